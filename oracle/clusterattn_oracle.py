@@ -1,0 +1,316 @@
+"""Plain fp64 statement of ClusterAttention* (transforms + diagonalized
+recursive splitting + top-k selection + striped mean-compensation).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, the smoke check and the
+benchmark's CPU-baseline leg, never by the product path.  Shares no code with
+the CUDA kernels.
+
+Every function works on ONE attention head (the method is per head, Section 3.1
+"Overview") and takes numpy arrays that it widens to float64.  The steps follow
+the paper's order and notation; no blocking, fusion or reordering is applied.
+numpy's `eigh`, `matmul` and `lexsort` serve as library steps.
+
+Pins (tests/test_oracle_*.py):
+  dense_attention ........ torch fp64 SDPA; hand-computed 2-key case
+  metric_q / psd_root .... ||R_q(k1-k2)||^2 == ||Q(k1-k2)||^2/n  (Section 3.2.2)
+  centered_scatter ....... D^T D == 2n K_c^T K_c by pair enumeration (Appendix B.2),
+                           shift invariance K_c(q+delta) == K_c q (Appendix B.1)
+  query_representation ... invariance to positive rescaling of q (Appendix B.2)
+  diagonalize ............ decorrelated coordinates, descending variance, isometry
+  split_point / recursive_split ... partition + size invariants (Section 3.1),
+                           d=1 closed form "sort and chunk", brute-force one-level cut
+  centroids / centroid_scores ..... mean pairwise logit identity, Jensen bound (Section 3.3.1)
+  select_topk ............ brute-force full sort
+  cluster_attention ...... all blocks kept == dense; c=1 == dense; eqs. (2)-(4);
+                           exact SMC error decomposition (Appendix A)
+Conventions of this build that the paper leaves open (subsample positions,
+round-half-up split point, fp32 rounding of the split coordinates, eigenvector
+sign) are "parity unpinned" by the paper: the oracle is their definition.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+F64 = np.float64
+
+
+# --------------------------------------------------------------------------
+# Eq. (1): dense bidirectional attention, softmax includes the 1/sqrt(d) scale
+# (Section 3.2.2 first paragraph; Section 3.3.1).
+# --------------------------------------------------------------------------
+def dense_attention(Q, K, V, scale=None, return_lse=False):
+    Q = np.asarray(Q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    if scale is None:
+        scale = 1.0 / np.sqrt(Q.shape[1])
+    logits = scale * (Q @ K.T)
+    mx = logits.max(axis=1, keepdims=True)
+    e = np.exp(logits - mx)
+    z = e.sum(axis=1, keepdims=True)
+    o = (e / z) @ V
+    if return_lse:
+        return o, (mx + np.log(z))[:, 0]
+    return o
+
+
+# --------------------------------------------------------------------------
+# Section 3.2.2 "Key clustering": M = Q^T Q / n.
+# --------------------------------------------------------------------------
+def metric_q(Q):
+    Q = np.asarray(Q, F64)
+    return (Q.T @ Q) / Q.shape[0]
+
+
+# --------------------------------------------------------------------------
+# Section 3.2.2 "Query clustering" / Appendix B.2: K_c^T K_c with K_c the key
+# matrix after subtracting the mean row.
+# --------------------------------------------------------------------------
+def centered_scatter(K):
+    K = np.asarray(K, F64)
+    Kc = K - K.mean(axis=0, keepdims=True)
+    return Kc.T @ Kc
+
+
+# --------------------------------------------------------------------------
+# Section 3.2.2: root of a PSD matrix by eigendecomposition, negative
+# eigenvalues clamped to zero; symmetric form E sqrt(L) E^T.
+# --------------------------------------------------------------------------
+def psd_root(A):
+    A = np.asarray(A, F64)
+    lam, E = np.linalg.eigh(0.5 * (A + A.T))
+    lam = np.maximum(lam, 0.0)
+    return (E * np.sqrt(lam)) @ E.T
+
+
+# Keys go to query space through R_q (Section 3.2.2, "project all keys through R_q").
+def transform_keys(K, R_q):
+    return np.asarray(K, F64) @ np.asarray(R_q, F64)   # rows: (R_q k)^T, R_q symmetric
+
+
+# r(q) = R_k q / |R_k q|  (Section 3.2.2, ranking form; Appendix B.2).
+# A row whose transformed norm underflows maps to the zero vector.
+def query_representation(Q, R_k):
+    Z = np.asarray(Q, F64) @ np.asarray(R_k, F64)
+    nrm = np.sqrt((Z * Z).sum(axis=1, keepdims=True))
+    out = np.zeros_like(Z)
+    ok = nrm[:, 0] >= 1e-30
+    out[ok] = Z[ok] / nrm[ok]
+    return out
+
+
+# --------------------------------------------------------------------------
+# Section 3.2.1 "Diagonalized recursive splitting": project the (transformed)
+# rows onto the principal components of the full set.  Centred covariance,
+# components in descending eigenvalue order; each eigenvector's sign is fixed
+# so that its entry of largest magnitude (lowest index on ties) is positive.
+# Returns (Y, eigenvalues, basis).
+# --------------------------------------------------------------------------
+def principal_basis(C):
+    lam, E = np.linalg.eigh(0.5 * (C + C.T))
+    order = np.argsort(-lam, kind="stable")
+    lam, E = lam[order], E[:, order]
+    for t in range(E.shape[1]):
+        j = int(np.argmax(np.abs(E[:, t])))
+        if E[j, t] < 0:
+            E[:, t] = -E[:, t]
+    return lam, E
+
+
+def diagonalize(X):
+    X = np.asarray(X, F64)
+    mu = X.mean(axis=0, keepdims=True)
+    Xc = X - mu
+    C = (Xc.T @ Xc) / X.shape[0]
+    lam, E = principal_basis(C)
+    return Xc @ E, lam, E
+
+
+# --------------------------------------------------------------------------
+# Section 3.2.1: the lower side of a split holds the multiple of c closest to
+# half of the set (half-way cases go up), so at most one final cluster is short
+# (Section 3.1).
+# --------------------------------------------------------------------------
+def split_point(s, c):
+    return c * ((s + c) // (2 * c))
+
+
+def subsample_positions(s, m):
+    """m evenly spaced positions inside a segment of s rows: floor(j*s/m)."""
+    return (np.arange(m, dtype=np.int64) * s) // m
+
+
+def choose_coordinate(sub):
+    """Coordinate of highest variance over the subsample rows `sub` [m, d]
+    (population variance; sums taken row after row in float64; lowest
+    coordinate on exact ties)."""
+    sub = np.asarray(sub, F64)
+    m = sub.shape[0]
+    mean = np.cumsum(sub, axis=0)[-1] / m
+    dev = sub - mean
+    var = np.cumsum(dev * dev, axis=0)[-1] / m
+    return int(np.argmax(var)), var
+
+
+def recursive_split(Y32, c, return_tree=False):
+    """Diagonalized recursive splitting (Section 3.2.1) on fp32 coordinates.
+
+    Y32 [N, d] float32: rows in principal-component coordinates.  Returns
+    perm [N] (position -> original row); cluster j is perm[j*c:(j+1)*c].
+    Every set keeps its rows in ascending original order, a split orders the
+    set by (coordinate value, original row) and sends the first L rows down.
+    """
+    Y32 = np.asarray(Y32)
+    assert Y32.dtype == np.float32
+    N, d = Y32.shape
+    perm = np.arange(N, dtype=np.int64)
+    work = [(0, N)]
+    tree = []
+    while work:
+        nxt = []
+        for lo, hi in work:
+            s = hi - lo
+            if s <= c:
+                continue
+            rows = perm[lo:hi].copy()
+            m = min(d, s)
+            sub = Y32[rows[subsample_positions(s, m)]]
+            t, _ = choose_coordinate(sub)
+            L = split_point(s, c)
+            keys = Y32[rows, t]
+            order = np.lexsort((rows, keys))        # by value, then original row
+            below = np.zeros(s, dtype=bool)
+            below[order[:L]] = True
+            perm[lo:lo + L] = rows[below]           # stable two-sided partition
+            perm[lo + L:hi] = rows[~below]
+            tree.append((lo, hi, t, L))
+            nxt.append((lo, lo + L))
+            nxt.append((lo + L, hi))
+        work = nxt
+    if return_tree:
+        return perm, tree
+    return perm
+
+
+# --------------------------------------------------------------------------
+# Section 3.1 / 3.3.1 / Appendix A: centroids are means over the actual members
+# in the ORIGINAL space; |c| is the member count.
+# --------------------------------------------------------------------------
+def centroids(X, perm, c):
+    X = np.asarray(X, F64)
+    N = X.shape[0]
+    n_c = -(-N // c)
+    cen = np.zeros((n_c, X.shape[1]), F64)
+    cnt = np.zeros(n_c, np.int64)
+    for j in range(n_c):
+        rows = perm[j * c:min((j + 1) * c, N)]
+        cen[j] = X[rows].mean(axis=0)
+        cnt[j] = len(rows)
+    return cen, cnt
+
+
+# Section 3.3.1: score = dot product of the two centroids.
+def centroid_scores(cq, ck):
+    return np.asarray(cq, F64) @ np.asarray(ck, F64).T
+
+
+# Section 3.3.2 top-k: the k best-scoring key clusters for each query cluster,
+# ties to the lower index, listed in ascending index order.
+def select_topk(scores, keep):
+    scores = np.asarray(scores, F64)
+    n_qc, n_kc = scores.shape
+    out = np.zeros((n_qc, keep), np.int64)
+    idx = np.arange(n_kc)
+    for i in range(n_qc):
+        order = np.lexsort((idx, -scores[i]))
+        out[i] = np.sort(order[:keep])
+    return out
+
+
+# --------------------------------------------------------------------------
+# Sparse attention over the selected clusters (eq. 2) with optional striped
+# mean-compensation (Appendix A, the expression for o-hat_S): an excluded
+# cluster enters numerator and denominator through its centroid key and value
+# with weight |c| * exp(q . k-bar / sqrt(d)).
+# `rows_of_cluster` lets the caller evaluate a sample of query clusters only.
+# --------------------------------------------------------------------------
+def cluster_attention(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx, compensate,
+                      ck=None, cv=None, count_k=None, scale=None, query_clusters=None):
+    Q = np.asarray(Q, F64)
+    K = np.asarray(K, F64)
+    V = np.asarray(V, F64)
+    N_q, d = Q.shape
+    N_k = K.shape[0]
+    n_kc = -(-N_k // c_k)
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    if compensate:
+        if ck is None:
+            ck, count_k = centroids(K, perm_k, c_k)
+        if cv is None:
+            cv, _ = centroids(V, perm_k, c_k)
+        ck = np.asarray(ck, F64)
+        cv = np.asarray(cv, F64)
+        count_k = np.asarray(count_k, F64)
+    O = np.zeros((N_q, V.shape[1]), F64)
+    lse = np.zeros(N_q, F64)
+    n_qc = -(-N_q // c_q)
+    todo = range(n_qc) if query_clusters is None else query_clusters
+    for i in todo:
+        rows = perm_q[i * c_q:min((i + 1) * c_q, N_q)]
+        sel = np.asarray(block_idx[i], np.int64)
+        members = np.concatenate([perm_k[j * c_k:min((j + 1) * c_k, N_k)] for j in sel])
+        logits = scale * (Q[rows] @ K[members].T)
+        values = V[members]
+        if compensate:
+            excluded = np.setdiff1d(np.arange(n_kc), sel)
+            if len(excluded):
+                lc = scale * (Q[rows] @ ck[excluded].T) + np.log(count_k[excluded])[None, :]
+                logits = np.concatenate([logits, lc], axis=1)
+                values = np.concatenate([values, cv[excluded]], axis=0)
+        mx = logits.max(axis=1, keepdims=True)
+        e = np.exp(logits - mx)
+        z = e.sum(axis=1, keepdims=True)
+        O[rows] = (e / z) @ values
+        lse[rows] = (mx + np.log(z))[:, 0]
+    return O, lse
+
+
+# --------------------------------------------------------------------------
+# The clustering stage for one head, steps in the paper's order:
+# metrics -> roots -> transforms -> global principal components -> fp32
+# coordinates -> recursive split -> centroids in the original space.
+# --------------------------------------------------------------------------
+def split_coordinates(Q, K):
+    """Returns (Yq32, Yk32): the fp32 coordinates the splitter reads."""
+    R_q = psd_root(metric_q(Q))
+    R_k = psd_root(centered_scatter(K))
+    Yk, _, _ = diagonalize(transform_keys(K, R_q))
+    Yq, _, _ = diagonalize(query_representation(Q, R_k))
+    return Yq.astype(np.float32), Yk.astype(np.float32)
+
+
+def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None):
+    if Yq32 is None or Yk32 is None:
+        Yq32, Yk32 = split_coordinates(Q, K)
+    perm_q = recursive_split(Yq32, c_q)
+    perm_k = recursive_split(Yk32, c_k)
+    cq, count_q = centroids(Q, perm_q, c_q)
+    ck, count_k = centroids(K, perm_k, c_k)
+    cv, _ = centroids(V, perm_k, c_k)
+    return dict(perm_q=perm_q, perm_k=perm_k, cq=cq, ck=ck, cv=cv,
+                count_q=count_q, count_k=count_k, Yq32=Yq32, Yk32=Yk32)
+
+
+def select_blocks(cq, ck, keep):
+    return select_topk(centroid_scores(cq, ck), keep)
+
+
+def clusterattention_forward(Q, K, V, c_q, c_k, keep, compensate, scale=None):
+    """Whole hot path for one head; returns (O, lse, clustering dict, block_idx)."""
+    cl = cluster_qk(Q, K, V, c_q, c_k)
+    block_idx = select_blocks(cl["cq"], cl["ck"], keep)
+    O, lse = cluster_attention(Q, K, V, cl["perm_q"], cl["perm_k"], c_q, c_k, block_idx,
+                               compensate, ck=cl["ck"], cv=cl["cv"], count_k=cl["count_k"],
+                               scale=scale)
+    return O, lse, cl, block_idx

@@ -1,0 +1,392 @@
+"""Pins of the fp64 oracle against what the paper and the mathematics fix.
+
+Each test checks an oracle function against something other than itself: an
+identity printed in the paper, a closed form, a brute-force enumeration, a
+special case that reduces to a textbook routine, or a library routine.
+"""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import clusterattn_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def rng(seed):
+    return np.random.default_rng(seed)
+
+
+# ---------------------------------------------------------------- dense (Eq. 1)
+def test_dense_matches_torch_sdpa_fp64():
+    r = rng(0)
+    Q, K, V = r.standard_normal((37, 16)), r.standard_normal((53, 16)), r.standard_normal((53, 16))
+    o = orc.dense_attention(Q, K, V)
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(Q)[None], torch.from_numpy(K)[None], torch.from_numpy(V)[None])[0].numpy()
+    assert np.abs(o - ref).max() < 1e-13
+
+
+def test_dense_two_keys_closed_form():
+    # one query, two keys: weights are a logistic function of the logit gap / sqrt(d)
+    q = np.array([[2.0, 0.0, 0.0, 0.0]])
+    K = np.array([[1.0, 0, 0, 0], [-1.0, 0, 0, 0]])
+    V = np.array([[1.0, 0, 0, 0], [0.0, 1.0, 0, 0]])
+    o, lse = orc.dense_attention(q, K, V, return_lse=True)
+    w0 = 1.0 / (1.0 + np.exp(-(2.0 - (-2.0)) / 2.0))     # sqrt(4) = 2
+    assert np.allclose(o[0, :2], [w0, 1 - w0], atol=1e-15)
+    assert np.isclose(lse[0], np.log(np.exp(1.0) + np.exp(-1.0)), atol=1e-15)
+
+
+# ------------------------------------------------- key metric (Section 3.2.2)
+def test_key_metric_root_gives_mean_squared_logit_difference():
+    r = rng(1)
+    Q = r.standard_normal((200, 12)) @ r.standard_normal((12, 12))
+    R = orc.psd_root(orc.metric_q(Q))
+    assert np.allclose(R, R.T, atol=1e-12)
+    for _ in range(20):
+        k1, k2 = r.standard_normal(12), r.standard_normal(12)
+        lhs = np.sum((R @ (k1 - k2)) ** 2)
+        rhs = np.sum((Q @ (k1 - k2)) ** 2) / Q.shape[0]
+        assert np.isclose(lhs, rhs, rtol=1e-10)
+        # inner product in the metric space
+        assert np.isclose((R @ k1) @ (R @ k2), k1 @ orc.metric_q(Q) @ k2, rtol=1e-9, atol=1e-9)
+    # rows of transform_keys are R_q k
+    K = r.standard_normal((5, 12))
+    assert np.allclose(orc.transform_keys(K, R), (R @ K.T).T, atol=1e-12)
+
+
+def test_psd_root_clamps_negative_eigenvalues_and_handles_rank_deficiency():
+    r = rng(2)
+    B = r.standard_normal((6, 3))
+    A = B @ B.T                                  # rank 3 of 6: zero-distance directions exist
+    R = orc.psd_root(A)
+    assert np.allclose(R @ R, A, atol=1e-10)
+    A_bad = A - 1e-9 * np.eye(6)                 # slightly indefinite
+    R2 = orc.psd_root(A_bad)
+    lam = np.linalg.eigvalsh(R2)
+    assert lam.min() > -1e-12 and np.allclose(R2 @ R2, A, atol=1e-7)
+    # diagonal case: root is the elementwise square root
+    D = np.diag([4.0, 9.0, 0.0, 1.0])
+    assert np.allclose(orc.psd_root(D), np.diag([2.0, 3.0, 0.0, 1.0]), atol=1e-14)
+
+
+# ------------------------------------------- query metric (Appendix B.1 / B.2)
+def test_pair_difference_operator_is_2n_times_centered_scatter():
+    r = rng(3)
+    n, d = 9, 4
+    K = r.standard_normal((n, d)) + 3.0
+    D = np.array([K[a] - K[b] for a in range(n) for b in range(n)])   # all ordered pairs
+    assert np.allclose(D.T @ D, 2 * n * orc.centered_scatter(K), atol=1e-10)
+
+
+def test_centered_key_representation_ignores_softmax_invariant_shifts():
+    r = rng(4)
+    n, d = 30, 6
+    K = r.standard_normal((n, d))
+    K[:, 5] = 0.7                                   # zero-variance direction: K e_5 = 0.7 * 1
+    delta = np.zeros(d)
+    delta[5] = 2.5
+    assert np.allclose(K @ delta, (0.7 * 2.5) * np.ones(n))
+    C = orc.centered_scatter(K)
+    R_k = orc.psd_root(C)
+    q = r.standard_normal(d)
+    Kc = K - K.mean(0)
+    assert np.allclose(Kc @ (q + delta), Kc @ q, atol=1e-12)
+    # same invariance through the root matrix: ||R_k delta|| = ||K_c delta|| = 0
+    assert np.linalg.norm(R_k @ delta) < 1e-6
+    # and softmax over the keys is indeed unchanged by the shift
+    a, b = K @ q, K @ (q + delta)
+    sa, sb = np.exp(a - a.max()), np.exp(b - b.max())
+    assert np.allclose(sa / sa.sum(), sb / sb.sum(), atol=1e-12)
+
+
+def test_query_representation_is_scale_invariant_and_unit_norm():
+    r = rng(5)
+    K = r.standard_normal((50, 8)) * np.arange(1, 9)
+    R_k = orc.psd_root(orc.centered_scatter(K))
+    Q = r.standard_normal((10, 8))
+    scales = r.uniform(0.1, 10.0, size=(10, 1))
+    a = orc.query_representation(Q, R_k)
+    b = orc.query_representation(Q * scales, R_k)
+    assert np.allclose(a, b, atol=1e-12)
+    assert np.allclose(np.linalg.norm(a, axis=1), 1.0, atol=1e-12)
+    assert np.allclose(a[0], (R_k @ Q[0]) / np.linalg.norm(R_k @ Q[0]), atol=1e-12)
+    zero = orc.query_representation(np.zeros((1, 8)), R_k)
+    assert np.all(zero == 0.0)
+
+
+# ---------------------------------------- diagonalization (Section 3.2.1, PCA)
+def test_diagonalize_is_pca_of_the_rows():
+    r = rng(6)
+    X = r.standard_normal((500, 7)) @ r.standard_normal((7, 7)) + 5.0
+    Y, lam, E = orc.diagonalize(X)
+    assert np.allclose(E.T @ E, np.eye(7), atol=1e-12)
+    assert np.all(np.diff(lam) <= 1e-12)                       # descending
+    cov = (Y.T @ Y) / X.shape[0]
+    assert np.allclose(cov, np.diag(lam), atol=1e-9)           # decorrelated, variances = eigenvalues
+    assert np.allclose(Y.mean(0), 0.0, atol=1e-10)
+    # pairwise distances are preserved (pure rotation of the centred rows)
+    assert np.isclose(np.linalg.norm(Y[3] - Y[11]), np.linalg.norm(X[3] - X[11]), rtol=1e-12)
+    # equivalent to the SVD of the centred data matrix up to column signs
+    _, s, Vt = np.linalg.svd(X - X.mean(0), full_matrices=False)
+    assert np.allclose(s ** 2 / X.shape[0], lam, rtol=1e-10)
+    assert np.allclose(np.abs(Vt), np.abs(E.T), atol=1e-8)
+    # sign convention
+    for t in range(7):
+        assert E[np.argmax(np.abs(E[:, t])), t] > 0
+
+
+def test_split_coordinates_do_not_depend_on_the_form_of_the_root():
+    # using E sqrt(L) instead of E sqrt(L) E^T rotates the transformed keys; the
+    # principal-component coordinates are the same up to per-coordinate sign.
+    r = rng(7)
+    Q = r.standard_normal((300, 6)) * np.array([3, 2, 1.5, 1, 0.5, 0.2])
+    K = r.standard_normal((400, 6)) @ r.standard_normal((6, 6))
+    M = orc.metric_q(Q)
+    lam, E = np.linalg.eigh(M)
+    R_sym = orc.psd_root(M)
+    R_alt = E * np.sqrt(np.maximum(lam, 0))
+    Y1, l1, _ = orc.diagonalize(K @ R_sym)
+    Y2, l2, _ = orc.diagonalize(K @ R_alt)
+    assert np.allclose(l1, l2, rtol=1e-9)
+    assert np.allclose(np.abs(Y1), np.abs(Y2), atol=1e-8)
+
+
+# ------------------------------------------------------ split sizes (Section 3.1)
+def test_split_point_rule_and_golden_shapes():
+    for c in (1, 2, 64, 128, 256):
+        for s in list(range(c + 1, 12 * c + 3)) + [32760, 75600, 131072]:
+            if s <= c:
+                continue
+            L = orc.split_point(s, c)
+            assert L % c == 0 and c <= L < s
+            # closest multiple of c to s/2; the half-way case goes up
+            cands = [m * c for m in range(1, s // c + 1) if m * c < s]
+            best = min(cands, key=lambda x: (abs(2 * x - s), -x))
+            assert L == best, (s, c, L, best)
+    with open(os.path.join(GOLDEN, "split_shapes.txt")) as f:
+        rows = [l.split() for l in f if l.strip() and not l.startswith("#")]
+    for N, c, n_clusters, short, levels in ((int(x) for x in r_) for r_ in rows):
+        sizes, depth = [N], 0
+        while any(s > c for s in sizes):
+            nxt = []
+            for s in sizes:
+                if s > c:
+                    L = orc.split_point(s, c)
+                    nxt += [L, s - L]
+                else:
+                    nxt.append(s)
+            sizes, depth = nxt, depth + 1
+        assert len(sizes) == n_clusters and depth == levels
+        shorts = [s for s in sizes if s != c]
+        assert shorts == ([short] if short else [])
+        assert sizes[-1] == (short if short else c)     # the short cluster is the last one
+
+
+# ------------------------------------------------- recursive split (Section 3.2.1)
+@pytest.mark.parametrize("N,c,d", [(1024, 64, 8), (1000, 64, 5), (777, 32, 3), (130, 128, 4),
+                                   (64, 64, 4), (50, 64, 4), (5 * 16 + 3, 16, 2)])
+def test_recursive_split_invariants(N, c, d):
+    r = rng(N + c)
+    Y = (r.standard_normal((N, d)) * np.linspace(3, 0.5, d)).astype(np.float32)
+    perm, tree = orc.recursive_split(Y, c, return_tree=True)
+    assert sorted(perm.tolist()) == list(range(N))              # clusters partition the rows
+    for lo, hi, t, L in tree:
+        assert L % c == 0 and 0 < L < hi - lo                   # lower side: multiple of c
+        left, right = perm[lo:lo + L], perm[lo + L:hi]
+        # ordered by (value, row): every row below sorts before every row above, along t
+        kl = max((Y[i, t], i) for i in left)
+        kr = min((Y[i, t], i) for i in right)
+        assert kl < kr
+    n_c = -(-N // c)
+    for j in range(n_c):
+        members = perm[j * c:(j + 1) * c]
+        assert len(members) == (c if j < n_c - 1 or N % c == 0 else N % c)
+        assert np.all(np.diff(members) > 0)                     # ascending original order inside a set
+
+
+def test_recursive_split_one_dimension_is_sort_and_chunk():
+    r = rng(11)
+    for N, c in [(256, 16), (250, 16), (96, 32)]:
+        y = r.standard_normal((N, 1)).astype(np.float32)
+        y[::7] = y[3]                                           # duplicates: ties go to the lower row
+        perm = orc.recursive_split(y, c)
+        order = sorted(range(N), key=lambda i: (y[i, 0], i))
+        for j in range(-(-N // c)):
+            assert sorted(order[j * c:(j + 1) * c]) == perm[j * c:(j + 1) * c].tolist()
+
+
+def test_recursive_split_single_level_is_median_cut_along_top_variance_coordinate():
+    # N = 2c: one PDDP-style step along the coordinate with the largest sampled variance
+    r = rng(12)
+    c, d = 8, 3
+    Y = r.standard_normal((2 * c, d)).astype(np.float32) * np.array([1.0, 4.0, 2.0], np.float32)
+    perm, tree = orc.recursive_split(Y, c, return_tree=True)
+    # brute force, written independently: subsample rows floor(j*s/m), m = min(d, s)
+    s, m = 2 * c, min(d, 2 * c)
+    sample = [Y[(j * s) // m].astype(np.float64) for j in range(m)]
+    var = []
+    for t in range(d):
+        vals = [row[t] for row in sample]
+        mu = sum(vals) / m
+        var.append(sum((v - mu) ** 2 for v in vals) / m)
+    t_star = max(range(d), key=lambda t: (var[t], -t))
+    assert tree == [(0, 2 * c, t_star, c)]
+    ranked = sorted(range(2 * c), key=lambda i: (Y[i, t_star], i))
+    assert sorted(ranked[:c]) == perm[:c].tolist() and sorted(ranked[c:]) == perm[c:].tolist()
+
+
+def test_choose_coordinate_ties_go_to_lowest_coordinate():
+    sub = np.zeros((4, 5))
+    sub[:, 2] = [1, -1, 1, -1]
+    sub[:, 4] = [1, -1, 1, -1]
+    t, var = orc.choose_coordinate(sub)
+    assert t == 2 and var[2] == var[4] == 1.0
+    assert orc.subsample_positions(10, 4).tolist() == [0, 2, 5, 7]
+
+
+def test_recursive_split_clusters_are_tighter_than_random_clusters():
+    # qualitative: Section 1.2 contrasts the method with random equal-size clusters
+    r = rng(13)
+    means = 3 * r.standard_normal((8, 16))
+    X = means[r.integers(0, 8, 2048)] + 0.3 * r.standard_normal((2048, 16))
+    Y, _, _ = orc.diagonalize(X)
+    perm = orc.recursive_split(Y.astype(np.float32), 64)
+
+    def within(p):
+        return sum(X[p[j * 64:(j + 1) * 64]].var(axis=0).sum() for j in range(32)) / 32
+    assert within(perm) < 0.5 * within(r.permutation(2048))
+
+
+# -------------------------------------------- centroids and scores (Section 3.3.1)
+def test_centroid_score_is_mean_pairwise_logit_and_jensen_bound():
+    r = rng(14)
+    N, d, c = 96, 8, 16
+    Q, K = r.standard_normal((N, d)), r.standard_normal((N + 5, d))
+    pq, pk = r.permutation(N), r.permutation(N + 5)
+    cq, nq = orc.centroids(Q, pq, c)
+    ck, nk = orc.centroids(K, pk, c)
+    assert nk.tolist() == [16] * 6 + [5] and nq.tolist() == [16] * 6
+    S = orc.centroid_scores(cq, ck)
+    for i, j in itertools.product(range(6), range(7)):
+        qs, ks = Q[pq[i * c:(i + 1) * c]], K[pk[j * c:min((j + 1) * c, N + 5)]]
+        pair = qs @ ks.T
+        assert np.isclose(S[i, j], pair.mean(), atol=1e-12)
+        assert np.exp(pair / np.sqrt(d)).mean() >= np.exp(S[i, j] / np.sqrt(d)) - 1e-12
+
+
+def test_select_topk_matches_full_sort_with_index_tie_break():
+    r = rng(15)
+    S = r.standard_normal((7, 20))
+    S[2, 5] = S[2, 9] = S[2, 14] = S[2].max() + 1.0          # three-way tie at the top
+    S[4, :] = 1.0                                             # all equal
+    for keep in (1, 2, 5, 20):
+        got = orc.select_topk(S, keep)
+        for i in range(7):
+            ranked = sorted(range(20), key=lambda j: (-S[i, j], j))
+            assert got[i].tolist() == sorted(ranked[:keep])
+    assert orc.select_topk(S, 2)[2].tolist() == [5, 9]
+    assert orc.select_topk(S, 3)[4].tolist() == [0, 1, 2]
+
+
+# ------------------------------------------------ attention (Section 1.2, Appendix A)
+def _setup(seed, N_q=48, N_k=60, d=8, c=4):
+    r = rng(seed)
+    Q, K, V = r.standard_normal((N_q, d)), 1.5 * r.standard_normal((N_k, d)), r.standard_normal((N_k, d))
+    return r, Q, K, V, r.permutation(N_q), r.permutation(N_k), c
+
+
+def test_all_blocks_kept_equals_dense():
+    r, Q, K, V, pq, pk, c = _setup(20, N_k=62)                 # 62 = 15*4 + 2: short key cluster
+    n_kc, n_qc = 16, 12
+    idx = np.tile(np.arange(n_kc), (n_qc, 1))
+    for comp in (False, True):
+        o, lse = orc.cluster_attention(Q, K, V, pq, pk, c, c, idx, comp)
+        od, lsed = orc.dense_attention(Q, K, V, return_lse=True)
+        assert np.abs(o - od).max() < 1e-12 and np.abs(lse - lsed).max() < 1e-12
+
+
+def test_cluster_size_one_makes_compensation_exact():
+    r, Q, K, V, pq, pk, _ = _setup(21, N_q=10, N_k=23)
+    idx = np.stack([np.sort(r.choice(23, 5, replace=False)) for _ in range(10)])
+    o, lse = orc.cluster_attention(Q, K, V, pq, pk, 1, 1, idx, True)
+    od, lsed = orc.dense_attention(Q, K, V, return_lse=True)
+    assert np.abs(o - od).max() < 1e-12 and np.abs(lse - lsed).max() < 1e-12
+    o_nc, _ = orc.cluster_attention(Q, K, V, pq, pk, 1, 1, idx, False)
+    assert np.abs(o_nc - od).max() > 1e-3                      # and it matters
+
+
+def test_uncompensated_output_and_error_split():
+    # eqs. (2)-(4): o_S over the selected keys; o - o_S = (1 - w_S)(o_Sbar - o_S)
+    r, Q, K, V, pq, pk, c = _setup(22)
+    n_kc, n_qc, keep = 15, 12, 4
+    idx = np.stack([np.sort(r.choice(n_kc, keep, replace=False)) for _ in range(n_qc)])
+    o_S, _ = orc.cluster_attention(Q, K, V, pq, pk, c, c, idx, False)
+    scale = 1 / np.sqrt(Q.shape[1])
+    for i in range(n_qc):
+        S = np.concatenate([pk[j * c:(j + 1) * c] for j in idx[i]])
+        Sbar = np.setdiff1d(np.arange(60), S)
+        for row in pq[i * c:(i + 1) * c]:
+            w = np.exp(scale * K @ Q[row])
+            w /= w.sum()
+            oS = (w[S] @ V[S]) / w[S].sum()
+            oSb = (w[Sbar] @ V[Sbar]) / w[Sbar].sum()
+            o = w @ V
+            assert np.allclose(o_S[row], oS, atol=1e-13)
+            assert np.allclose(o - o_S[row], (1 - w[S].sum()) * (oSb - oS), atol=1e-13)
+
+
+def test_compensated_error_decomposition():
+    # Appendix A: o - o_hat = sum_c |c| (delta_c (vbar_c - o_hat) + Cov_c(w, v)),
+    # the 1/d_hat form with (vbar_c - o), d_hat = 1 - sum_c |c| delta_c, delta_c >= 0.
+    r, Q, K, V, pq, pk, c = _setup(23, N_k=58)                 # last key cluster has 2 rows
+    N_k, n_kc, n_qc, keep = 58, 15, 12, 3
+    idx = np.stack([np.sort(r.choice(n_kc, keep, replace=False)) for _ in range(n_qc)])
+    o_hat, lse_hat = orc.cluster_attention(Q, K, V, pq, pk, c, c, idx, True)
+    od, lsed = orc.dense_attention(Q, K, V, return_lse=True)
+    scale = 1 / np.sqrt(Q.shape[1])
+    for i in range(n_qc):
+        excluded = np.setdiff1d(np.arange(n_kc), idx[i])
+        for row in pq[i * c:(i + 1) * c]:
+            e = np.exp(scale * K @ Q[row])
+            Z = e.sum()
+            w = e / Z
+            o = w @ V
+            jensen_hat, jensen_o, cov_sum, d_hat = 0.0, 0.0, 0.0, 1.0
+            for j in excluded:
+                mem = pk[j * c:min((j + 1) * c, N_k)]
+                n = len(mem)
+                kbar, vbar = K[mem].mean(0), V[mem].mean(0)
+                w_c = np.exp(scale * kbar @ Q[row]) / Z          # centroid weight, dense-normalised
+                delta = w[mem].mean() - w_c
+                assert delta >= -1e-15
+                cov = ((w[mem] - w[mem].mean())[:, None] * (V[mem] - vbar)).mean(0)
+                jensen_hat = jensen_hat + n * delta * (vbar - o_hat[row])
+                jensen_o = jensen_o + n * delta * (vbar - o)
+                cov_sum = cov_sum + n * cov
+                d_hat -= n * delta
+            assert np.allclose(o - o_hat[row], jensen_hat + cov_sum, atol=1e-13)
+            assert np.allclose(o - o_hat[row], (jensen_o + cov_sum) / d_hat, atol=1e-13)
+            # the compensated denominator is d_hat times the dense one
+            assert np.isclose(lse_hat[row], lsed[row] + np.log(d_hat), atol=1e-12)
+
+
+def test_forward_pipeline_shapes_and_convergence_to_dense():
+    # whole path on a small mixture: more kept blocks -> closer to dense; SMC helps
+    r = rng(30)
+    means = 3 * r.standard_normal((4, 16)) / 4
+    Q = means[r.integers(0, 4, 256)] + 0.5 * r.standard_normal((256, 16))
+    K = means[r.integers(0, 4, 256)] + 0.5 * r.standard_normal((256, 16))
+    V = r.standard_normal((256, 16))
+    od = orc.dense_attention(Q, K, V)
+    errs = []
+    for keep in (2, 8, 16):
+        o, _, cl, idx = orc.clusterattention_forward(Q, K, V, 16, 16, keep, True)
+        assert idx.shape == (16, keep) and np.all(np.diff(idx, axis=1) > 0)
+        assert sorted(cl["perm_k"].tolist()) == list(range(256))
+        errs.append(np.abs(o - od).max())
+    assert errs[2] < 1e-12 and errs[0] > errs[1] > errs[2]
