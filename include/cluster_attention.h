@@ -1,0 +1,140 @@
+/*
+ * libclusterattn — C ABI of the ClusterAttention hot path on one B200 (sm_100a).
+ *
+ * Three stages, one entry point each (the method's "clustering", "assignment"
+ * and "attention" parts, Section 3.1):
+ *   cluster_qk             transforms + diagonalized recursive splitting + centroids
+ *   select_blocks          centroid scoring + top-k key clusters per query cluster
+ *   cluster_attention_fwd  block-sparse attention over the selected cluster pairs
+ *                          with striped mean-compensation of the excluded clusters
+ *
+ * Conventions for every call
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte aligned,
+ *     dense row-major.  Inputs are never modified.  The library allocates no
+ *     device memory: scratch is a caller-provided workspace whose size
+ *     ca_workspace_bytes reports.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL is the
+ *     default stream).  Calls do not synchronise.
+ *   - Tensors are [batch, heads, rows, head_dim]; batch*heads independent problems.
+ *   - Return value: CA_OK or an error code; nothing is enqueued on error except
+ *     for CA_ERR_CUDA (a launch failed part-way).
+ *   - The first 256 bytes of a workspace hold a status word that kernels set when
+ *     a bounded wait expires (CA_ERR_TIMEOUT); ca_last_status reads it.
+ */
+#ifndef CLUSTER_ATTENTION_H_
+#define CLUSTER_ATTENTION_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  CA_OK = 0,
+  CA_ERR_INVALID_ARG = 1,  /* null pointer, bad size, keep out of range, misaligned pointer */
+  CA_ERR_UNSUPPORTED = 2,  /* dtype / head_dim / cluster size outside the supported set      */
+  CA_ERR_WORKSPACE = 3,    /* workspace null or smaller than ca_workspace_bytes reports      */
+  CA_ERR_CUDA = 4,         /* a CUDA runtime call or kernel launch failed                    */
+  CA_ERR_TIMEOUT = 5       /* (status word only) a bounded device-side wait gave up          */
+};
+
+enum { CA_DTYPE_FP32 = 0, CA_DTYPE_BF16 = 1 };
+
+/* cluster_qk flags */
+enum {
+  CA_Y_IN = 1,      /* Yq/Yk hold the split coordinates: skip the transforms (used by tests
+                       to feed the splitter the very same fp32 coordinates as the oracle)   */
+  CA_ATTN_FP32 = 2  /* cluster_attention_fwd: force the FP32 CUDA-core kernel for bf16 data  */
+};
+
+typedef struct {
+  int32_t batch, heads;
+  int32_t n_q, n_k;        /* query rows, key/value rows per head                            */
+  int32_t head_dim;        /* d (values have the same width); 64 or 128                      */
+  int32_t dtype;           /* CA_DTYPE_*: storage type of Q, K, V, Qp, Kp, Vp, O             */
+  int32_t cluster_q;       /* query cluster size c_q, a power of two in [16, 256]            */
+  int32_t cluster_k;       /* key cluster size c_k, a power of two in [16, 256]              */
+  int32_t keep;            /* kept key clusters per query cluster, 1 .. ceil(n_k/c_k)        */
+  int32_t compensate;      /* 0/1: striped mean-compensation off/on                          */
+  float softmax_scale;     /* 0 selects 1/sqrt(head_dim)                                     */
+  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32                                         */
+} ca_problem_t;
+
+/* Bytes of workspace each stage needs for this problem (any pointer may be NULL). */
+int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select_ws,
+                       size_t* attn_ws);
+
+/*
+ * Clustering (Section 3.2).  Per head, queries and keys separately:
+ *   M = Q^T Q / n_q, R_q = sqrt(M) (eigendecomposition, negative eigenvalues
+ *   clamped), keys -> K R_q; R_k = sqrt(K_c^T K_c) with K_c the centred keys,
+ *   queries -> r(q) = R_k q / |R_k q| (Section 3.2.2); both sets are projected
+ *   on their global principal components (Section 3.2.1, diagonalized variant);
+ *   the rows are split recursively: at each split the coordinate of highest
+ *   variance over min(d, |set|) evenly spaced rows of the set is chosen and the
+ *   set is cut so that the lower side holds the multiple of c closest to half
+ *   (ties in value go to the lower row index; half-way sizes go to the lower
+ *   side); every set keeps its rows in ascending original order.
+ * Outputs
+ *   perm_q [B,H,n_q], perm_k [B,H,n_k]  position -> original row; cluster j is
+ *        positions [j*c, min((j+1)*c, n)); only the last cluster can be short.
+ *   Qp,Kp,Vp [B,H,n_c*c,d]  rows gathered in cluster order (V follows the key
+ *        permutation); the short cluster is zero-padded to c rows.
+ *   cq,ck,cv [B,H,n_c,d] fp32  centroids: means over the actual members in the
+ *        original space (Section 3.3.1; Appendix A).
+ *   count_q,count_k [B,H,n_c]  member counts |c|.
+ *   Yq [B,H,n_q,d], Yk [B,H,n_k,d] fp32 split coordinates: input when
+ *        p->flags has CA_Y_IN, otherwise output (may be NULL: kept in ws).
+ */
+int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* V,
+               int32_t* perm_q, int32_t* perm_k, void* Qp, void* Kp, void* Vp,
+               float* cq, float* ck, float* cv, int32_t* count_q, int32_t* count_k,
+               float* Yq, float* Yk, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Assignment (Section 3.3).  score(i,j) = cq_i . ck_j (the mean logit of the two
+ * clusters); for each query cluster the `keep` best key clusters, ties to the
+ * lower index, written in ascending index order.
+ *   block_idx [B,H,n_qc,keep] int32.
+ */
+int select_blocks(const ca_problem_t* p, const float* cq, const float* ck,
+                  int32_t* block_idx, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Attention (eq. 2 over the selected clusters; Appendix A for compensation).
+ * For query row r of query cluster i, with s = softmax_scale:
+ *   entries  (s q_r.k_t, v_t)                 for every member t of a selected cluster
+ *   and, if p->compensate,
+ *            (s q_r.kbar_j + ln|c_j|, vbar_j) for every cluster j NOT selected;
+ *   O_r = softmax-weighted mean of the entry values; lse_r = log-sum-exp of the
+ *   entry logits.  Padding rows of the short cluster are masked.
+ * Accepts any valid permutation and block list (block_idx rows must be strictly
+ * ascending), so the stage can be driven by another clustering.
+ *   Qp,Kp,Vp, ck, cv, count_k, perm_q: as written by cluster_qk.
+ *   O [B,H,n_q,d] in ORIGINAL row order, storage dtype; lse [B,H,n_q] fp32 or NULL.
+ * bf16 storage runs on tcgen05 tensor cores with fp32 accumulation (head_dim
+ * 64/128, clusters 64..256 with c_q == 128 tiles); fp32 storage, other sizes, or
+ * CA_ATTN_FP32 run the FP32 CUDA-core kernel.
+ */
+int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
+                          const void* Vp, const float* ck, const float* cv,
+                          const int32_t* count_k, const int32_t* block_idx,
+                          const int32_t* perm_q, void* O, float* lse, void* ws,
+                          size_t ws_bytes, void* stream);
+
+/* Reads the status word of a workspace (synchronises the device). */
+int ca_last_status(const void* ws);
+
+/* Library version and the compute capability the kernels were built for. */
+const char* ca_version(void);
+
+/* Diagnostic: number of kernels this library has enqueued since it was loaded
+ * (host-side counter, not thread-safe). */
+unsigned long long ca_kernel_launches(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLUSTER_ATTENTION_H_ */

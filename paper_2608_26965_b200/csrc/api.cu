@@ -1,0 +1,204 @@
+// C entry points of libclusterattn: argument checks, workspace carving and the
+// order in which the kernels of each stage are enqueued.
+#include <math.h>
+
+#include "kernels.h"
+
+using namespace ca;
+
+namespace ca {
+unsigned long long g_kernel_launches = 0;
+}
+
+namespace {
+
+bool pow2(int x) { return x > 0 && (x & (x - 1)) == 0; }
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_problem(const ca_problem_t* p) {
+  if (!p) return CA_ERR_INVALID_ARG;
+  if (p->batch < 1 || p->heads < 1 || p->n_q < 1 || p->n_k < 1) return CA_ERR_INVALID_ARG;
+  if (p->head_dim != 64 && p->head_dim != 128) return CA_ERR_UNSUPPORTED;
+  if (p->dtype != CA_DTYPE_FP32 && p->dtype != CA_DTYPE_BF16) return CA_ERR_UNSUPPORTED;
+  if (!pow2(p->cluster_q) || !pow2(p->cluster_k)) return CA_ERR_INVALID_ARG;
+  if (p->cluster_q < 16 || p->cluster_q > 256 || p->cluster_k < 16 || p->cluster_k > 256)
+    return CA_ERR_UNSUPPORTED;
+  const int n_kc = ceil_div(p->n_k, p->cluster_k);
+  if (p->keep < 1 || p->keep > n_kc) return CA_ERR_INVALID_ARG;
+  if ((long long)p->batch * p->heads > 65535) return CA_ERR_UNSUPPORTED;
+  if (!(p->softmax_scale >= 0.f)) return CA_ERR_INVALID_ARG;
+  return CA_OK;
+}
+
+struct ClusterWs {
+  int* status;
+  float* partial;
+  double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
+  float *roots32, *basis32, *WK32, *biasK, *biasQ;
+  float *Qprime, *Yq, *Yk;
+  int32_t *perm_q_tmp, *perm_k_tmp;
+  uint32_t *keybuf_q, *keybuf_k;
+  size_t bytes;
+};
+
+ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool need_yk) {
+  ClusterWs w{};
+  Carver c(base);
+  const size_t P = (size_t)p->batch * p->heads, D = p->head_dim, DD = D * D;
+  w.status = c.take<int>(kStatusBytes / sizeof(int));
+  const bool transforms = !(p->flags & CA_Y_IN);
+  if (transforms) {
+    int cr, ncq, nck;
+    moments_chunking(p->n_q, (int)P, &cr, &ncq);
+    moments_chunking(p->n_k, (int)P, &cr, &nck);
+    const size_t nchunks = (size_t)(ncq > nck ? ncq : nck);
+    w.partial = c.take<float>(P * nchunks * (DD + D));
+    w.gramQ = c.take<double>(P * DD);  w.sumQ = c.take<double>(P * D);
+    w.gramK = c.take<double>(P * DD);  w.sumK = c.take<double>(P * D);
+    w.metric = c.take<double>(2 * P * DD);
+    w.roots = c.take<double>(2 * P * DD);
+    w.tmp = c.take<double>(P * DD);
+    w.cov = c.take<double>(2 * P * DD);
+    w.gramQp = c.take<double>(P * DD); w.sumQp = c.take<double>(P * D);
+    w.basis = c.take<double>(2 * P * DD);
+    w.WK = c.take<double>(P * DD);
+    w.roots32 = c.take<float>(2 * P * DD);
+    w.basis32 = c.take<float>(2 * P * DD);
+    w.WK32 = c.take<float>(P * DD);
+    w.biasK = c.take<float>(P * D);
+    w.biasQ = c.take<float>(P * D);
+    w.Qprime = c.take<float>(P * (size_t)p->n_q * D);
+    if (need_yq) w.Yq = c.take<float>(P * (size_t)p->n_q * D);
+    if (need_yk) w.Yk = c.take<float>(P * (size_t)p->n_k * D);
+  }
+  w.perm_q_tmp = c.take<int32_t>(P * (size_t)p->n_q);
+  w.perm_k_tmp = c.take<int32_t>(P * (size_t)p->n_k);
+  w.keybuf_q = c.take<uint32_t>(P * (size_t)p->n_q);
+  w.keybuf_k = c.take<uint32_t>(P * (size_t)p->n_k);
+  w.bytes = c.used();
+  return w;
+}
+
+#define CA_TRY(expr)               \
+  do {                             \
+    int _rc = (expr);              \
+    if (_rc != CA_OK) return _rc;  \
+  } while (0)
+
+}  // namespace
+
+extern "C" {
+
+const char* ca_version(void) { return "libclusterattn 0.1 (sm_100a)"; }
+
+unsigned long long ca_kernel_launches(void) { return g_kernel_launches; }
+
+int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select_ws, size_t* attn_ws) {
+  CA_TRY(check_problem(p));
+  if (cluster_ws) *cluster_ws = carve_cluster(p, nullptr, true, true).bytes;
+  if (select_ws) *select_ws = kStatusBytes;
+  if (attn_ws) *attn_ws = kStatusBytes;
+  return CA_OK;
+}
+
+int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* V, int32_t* perm_q,
+               int32_t* perm_k, void* Qp, void* Kp, void* Vp, float* cq, float* ck, float* cv,
+               int32_t* count_q, int32_t* count_k, float* Yq, float* Yk, void* ws, size_t ws_bytes,
+               void* stream) {
+  CA_TRY(check_problem(p));
+  const void* ptrs[] = {Q, K, V, perm_q, perm_k, Qp, Kp, Vp, cq, ck, cv, count_q, count_k};
+  for (const void* x : ptrs)
+    if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  const bool y_in = (p->flags & CA_Y_IN) != 0;
+  if (y_in && (!Yq || !Yk)) return CA_ERR_INVALID_ARG;
+  if ((Yq && !aligned16(Yq)) || (Yk && !aligned16(Yk))) return CA_ERR_INVALID_ARG;
+  if (!ws || !aligned16(ws)) return CA_ERR_WORKSPACE;
+  ClusterWs w = carve_cluster(p, ws, Yq == nullptr, Yk == nullptr);
+  if (ws_bytes < w.bytes) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int P = p->batch * p->heads, D = p->head_dim, DD = D * D;
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(w.status, 0, kStatusBytes, st));
+
+  const float* yq = Yq;
+  const float* yk = Yk;
+  if (!y_in) {
+    float* yq_out = Yq ? Yq : w.Yq;
+    float* yk_out = Yk ? Yk : w.Yk;
+    // metric matrices (Section 3.2.2)
+    CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
+    CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial, w.gramK, w.sumK, st));
+    double* M = w.metric;
+    double* CK = w.metric + (size_t)P * DD;
+    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, M, CK, st));
+    // roots R_q, R_k
+    CA_TRY(launch_eigh(w.metric, 2 * P, D, 0, w.roots, w.roots32, nullptr, st));
+    double* Rq = w.roots;
+    const float* Rk32 = w.roots32 + (size_t)P * DD;
+    // covariance of the transformed keys K R_q:  R_q C_K R_q / n_k
+    double* covK = w.cov;
+    double* covQ = w.cov + (size_t)P * DD;
+    CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, w.tmp, nullptr, st));
+    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, 1.0 / (double)p->n_k, covK, nullptr, st));
+    // query representation r(q) = R_k q / |R_k q| and its covariance
+    CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, 1, w.Qprime, st));
+    CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
+    CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
+    // global principal components of both transformed sets (Section 3.2.1)
+    CA_TRY(launch_eigh(w.cov, 2 * P, D, 1, w.basis, w.basis32, nullptr, st));
+    double* EK = w.basis;
+    double* EQ = w.basis + (size_t)P * DD;
+    const float* EQ32 = w.basis32 + (size_t)P * DD;
+    // keys: Y = (K - kbar) R_q E_K ; queries: Y = (r(q) - mean) E_Q
+    CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, w.WK, w.WK32, st));
+    CA_TRY(launch_bias(w.sumK, w.WK, P, D, p->n_k, w.biasK, st));
+    CA_TRY(launch_bias(w.sumQp, EQ, P, D, p->n_q, w.biasQ, st));
+    CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
+    CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, st));
+    yq = yq_out;
+    yk = yk_out;
+  }
+  CA_TRY(launch_split(yq, yk, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
+                      perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, st));
+  CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
+  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
+  CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+  return CA_OK;
+}
+
+int select_blocks(const ca_problem_t* p, const float* cq, const float* ck, int32_t* block_idx, void* ws,
+                  size_t ws_bytes, void* stream) {
+  CA_TRY(check_problem(p));
+  if (!cq || !ck || !block_idx || !aligned16(cq) || !aligned16(ck) || !aligned16(block_idx))
+    return CA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < kStatusBytes) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  const int P = p->batch * p->heads;
+  return launch_score_select(cq, ck, P, ceil_div(p->n_q, p->cluster_q), ceil_div(p->n_k, p->cluster_k),
+                             p->head_dim, p->keep, block_idx, st);
+}
+
+int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp, const void* Vp,
+                          const float* ck, const float* cv, const int32_t* count_k,
+                          const int32_t* block_idx, const int32_t* perm_q, void* O, float* lse, void* ws,
+                          size_t ws_bytes, void* stream) {
+  CA_TRY(check_problem(p));
+  const void* ptrs[] = {Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O};
+  for (const void* x : ptrs)
+    if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < kStatusBytes) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, scale, O, lse, st);
+}
+
+int ca_last_status(const void* ws) {
+  if (!ws) return CA_ERR_INVALID_ARG;
+  int status = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return CA_ERR_CUDA;
+  if (cudaMemcpy(&status, ws, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return CA_ERR_CUDA;
+  return status;
+}
+
+}  // extern "C"

@@ -1,0 +1,193 @@
+// FP32 CUDA-core kernel for block-sparse attention with striped
+// mean-compensation (eq. 2 over the selected clusters; Appendix A: an excluded
+// cluster enters through its centroid key and value with weight
+// |c| exp(q . kbar / sqrt(d)), in numerator and denominator).
+// Serves fp32 storage, unusual cluster sizes, and as an on-device cross-check of
+// the tensor-core kernel.  Flash-style online softmax, fp32 throughout.
+#include "kernels.h"
+
+namespace ca {
+
+constexpr int kRefQR = 16;       // query rows per CTA
+constexpr int kRefKT = 32;       // keys per staged tile
+constexpr int kRefThreads = 128;
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kRefThreads)
+attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __restrict__ Vp,
+                const float* __restrict__ ck, const float* __restrict__ cv,
+                const int32_t* __restrict__ count_k, const int32_t* __restrict__ block_idx,
+                const int32_t* __restrict__ perm_q, int n_q, int n_k, int c_q, int c_k, int keep,
+                int compensate, float scale, T* __restrict__ O, float* __restrict__ lse) {
+  constexpr int LD = D + 1;
+  constexpr int NC = D / 8;              // output columns per thread
+  extern __shared__ float smem[];
+  float* qs = smem;                      // [QR][LD]
+  float* ks = qs + kRefQR * LD;          // [KT][LD]
+  float* vs = ks + kRefKT * LD;          // [KT][LD]
+  float* ps = vs + kRefKT * LD;          // [QR][KT+1]
+  float* bias = ps + kRefQR * (kRefKT + 1);   // [KT] per-key additive term (ln|c| or -inf)
+  unsigned* selected = reinterpret_cast<unsigned*>(bias + kRefKT);   // bitmap over key clusters
+
+  const int n_qc = (n_q + c_q - 1) / c_q, n_kc = (n_k + c_k - 1) / c_k;
+  const int tiles_per_cluster = (c_q + kRefQR - 1) / kRefQR;
+  const int p = blockIdx.y;
+  const int qc = blockIdx.x / tiles_per_cluster;
+  const int r0 = (blockIdx.x % tiles_per_cluster) * kRefQR;
+  const int tid = threadIdx.x;
+  const int row = tid / 8, sub = tid % 8;
+  const size_t q_base = ((size_t)p * n_qc + qc) * (size_t)c_q;
+  const T* Kh = Kp + (size_t)p * n_kc * (size_t)c_k * D;
+  const T* Vh = Vp + (size_t)p * n_kc * (size_t)c_k * D;
+  const int32_t* sel = block_idx + ((size_t)p * n_qc + qc) * keep;
+  const int32_t* cnt = count_k + (size_t)p * n_kc;
+
+  for (int e = tid; e < kRefQR * D; e += kRefThreads) {
+    const int r = e / D, col = e % D;
+    const int pos = qc * c_q + r0 + r;
+    qs[r * LD + col] = (r0 + r < c_q && pos < n_q) ? to_f32<T>(Qp[(q_base + r0 + r) * D + col]) : 0.f;
+  }
+  const int words = (n_kc + 31) / 32;
+  for (int w = tid; w < words; w += kRefThreads) selected[w] = 0u;
+  __syncthreads();
+  for (int t = tid; t < keep; t += kRefThreads) atomicOr(&selected[sel[t] >> 5], 1u << (sel[t] & 31));
+
+  float m_run = -INFINITY, l_run = 0.f;
+  float acc[NC];
+#pragma unroll
+  for (int i = 0; i < NC; ++i) acc[i] = 0.f;
+
+  auto process_tile = [&]() {
+    // logits of this thread's 4 keys
+    float s[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] = 0.f;
+    for (int k = 0; k < D; ++k) {
+      const float q = qs[row * LD + k];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) s[i] = fmaf(q, ks[(sub + 8 * i) * LD + k], s[i]);
+    }
+    float tmax = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) { s[i] = s[i] * scale + bias[sub + 8 * i]; tmax = fmaxf(tmax, s[i]); }
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+    tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 4));
+    const float m_new = fmaxf(m_run, tmax);
+    float alpha = 1.f, psum = 0.f;
+    if (m_new > -INFINITY) {
+      alpha = expf(m_run - m_new);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float pv = expf(s[i] - m_new);
+        ps[row * (kRefKT + 1) + sub + 8 * i] = pv;
+        psum += pv;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) ps[row * (kRefKT + 1) + sub + 8 * i] = 0.f;
+    }
+    psum += __shfl_xor_sync(0xffffffffu, psum, 1);
+    psum += __shfl_xor_sync(0xffffffffu, psum, 2);
+    psum += __shfl_xor_sync(0xffffffffu, psum, 4);
+    l_run = l_run * alpha + psum;
+    m_run = m_new;
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < NC; ++i) acc[i] *= alpha;
+    for (int key = 0; key < kRefKT; ++key) {
+      const float pv = ps[row * (kRefKT + 1) + key];
+#pragma unroll
+      for (int i = 0; i < NC; ++i) acc[i] = fmaf(pv, vs[key * LD + sub + 8 * i], acc[i]);
+    }
+  };
+
+  // selected clusters: every member key
+  for (int t = 0; t < keep; ++t) {
+    const int j = sel[t];
+    const int members = cnt[j];
+    for (int t0 = 0; t0 < members; t0 += kRefKT) {
+      __syncthreads();
+      for (int e = tid; e < kRefKT * D; e += kRefThreads) {
+        const int r = e / D, col = e % D;
+        const bool ok = t0 + r < members;
+        const size_t g = ((size_t)j * c_k + t0 + r) * D + col;
+        ks[r * LD + col] = ok ? to_f32<T>(Kh[g]) : 0.f;
+        vs[r * LD + col] = ok ? to_f32<T>(Vh[g]) : 0.f;
+      }
+      if (tid < kRefKT) bias[tid] = (t0 + tid < members) ? 0.f : -INFINITY;
+      __syncthreads();
+      process_tile();
+    }
+  }
+  // excluded clusters through their centroids
+  if (compensate) {
+    const float* ckh = ck + (size_t)p * n_kc * D;
+    const float* cvh = cv + (size_t)p * n_kc * D;
+    for (int j0 = 0; j0 < n_kc; j0 += kRefKT) {
+      __syncthreads();
+      for (int e = tid; e < kRefKT * D; e += kRefThreads) {
+        const int r = e / D, col = e % D;
+        const bool ok = j0 + r < n_kc;
+        ks[r * LD + col] = ok ? ckh[(size_t)(j0 + r) * D + col] : 0.f;
+        vs[r * LD + col] = ok ? cvh[(size_t)(j0 + r) * D + col] : 0.f;
+      }
+      if (tid < kRefKT) {
+        const int j = j0 + tid;
+        const bool use = j < n_kc && !((selected[j >> 5] >> (j & 31)) & 1u);
+        bias[tid] = use ? logf((float)cnt[j]) : -INFINITY;
+      }
+      __syncthreads();
+      process_tile();
+    }
+  }
+
+  const int pos = qc * c_q + r0 + row;
+  if (r0 + row < c_q && pos < n_q) {
+    const int orig = perm_q[(size_t)p * n_q + pos];
+    const float inv = 1.f / l_run;
+    T* out = O + ((size_t)p * n_q + orig) * D;
+#pragma unroll
+    for (int i = 0; i < NC; ++i) out[sub + 8 * i] = from_f32<T>(acc[i] * inv);
+    if (lse && sub == 0) lse[(size_t)p * n_q + orig] = m_run + logf(l_run);
+  }
+}
+
+template <typename T>
+static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* Vp, const float* ck,
+                    const float* cv, const int32_t* count_k, const int32_t* block_idx,
+                    const int32_t* perm_q, float scale, T* O, float* lse, cudaStream_t st) {
+  const int P = pr.batch * pr.heads, D = pr.head_dim;
+  const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
+  const int tiles = ceil_div(pr.cluster_q, kRefQR);
+  const size_t smem = sizeof(float) * ((size_t)(kRefQR + 2 * kRefKT) * (D + 1) + kRefQR * (kRefKT + 1) + kRefKT) +
+                      sizeof(unsigned) * ((n_kc + 31) / 32);
+  dim3 grid(n_qc * tiles, P);
+  if (D == 64) {
+    auto k = attn_ref_kernel<T, 64>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, pr.n_q, pr.n_k,
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse);
+  } else {
+    auto k = attn_ref_kernel<T, 128>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, pr.n_q, pr.n_k,
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse);
+  }
+  CA_LAUNCH_CHECK();
+  return CA_OK;
+}
+
+int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
+                    const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
+                    const int32_t* perm_q, float scale, void* O, float* lse, cudaStream_t st) {
+  if (pr.dtype == CA_DTYPE_BF16)
+    return launch_t(pr, static_cast<const __nv_bfloat16*>(Qp), static_cast<const __nv_bfloat16*>(Kp),
+                    static_cast<const __nv_bfloat16*>(Vp), ck, cv, count_k, block_idx, perm_q, scale,
+                    static_cast<__nv_bfloat16*>(O), lse, st);
+  return launch_t(pr, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
+                  static_cast<const float*>(Vp), ck, cv, count_k, block_idx, perm_q, scale,
+                  static_cast<float*>(O), lse, st);
+}
+
+}  // namespace ca

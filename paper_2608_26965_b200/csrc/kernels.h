@@ -1,0 +1,47 @@
+// Host-side launchers of the library's kernels (internal; the public boundary
+// is include/cluster_attention.h).  Every launcher enqueues on `st` and returns
+// a CA_* code.
+#pragma once
+#include "common.cuh"
+
+namespace ca {
+
+// moments.cu
+int moments_chunking(int n_rows, int problems, int* chunk_rows, int* n_chunks);
+int launch_moments(const void* X, int dtype, int problems, int n_rows, int D, float* partial,
+                   double* gram, double* colsum, cudaStream_t st);
+int launch_transform_rows(const void* X, int dtype, int problems, int n_rows, int D, const float* W,
+                          const float* bias, int normalize, float* out, cudaStream_t st);
+
+// eigh.cu
+int launch_eigh(const double* A, int count, int D, int mode, double* out64, float* out32,
+                double* evals, cudaStream_t st);
+int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
+                  int n_k, double* M, double* CK, cudaStream_t st);
+int launch_covariance(const double* gram, const double* sum, int P, int D, int n, double* cov,
+                      cudaStream_t st);
+int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, double* C,
+                        float* C32, cudaStream_t st);
+int launch_bias(const double* sum, const double* W, int P, int D, int n, float* bias, cudaStream_t st);
+
+// split.cu
+int split_levels_for(int n, int c);
+int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
+                 int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
+                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st);
+
+// permute.cu
+int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P, int n, int D, int c,
+                            void* Xp, float* cen, int32_t* count, cudaStream_t st);
+
+// select.cu
+size_t select_smem_bytes(int n_kc, int D);
+int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n_kc, int D, int keep,
+                        int32_t* block_idx, cudaStream_t st);
+
+// attn_ref.cu
+int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
+                    const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
+                    const int32_t* perm_q, float scale, void* O, float* lse, cudaStream_t st);
+
+}  // namespace ca

@@ -1,0 +1,297 @@
+"""Parity of the CUDA path (through the C ABI) against the fp64 oracle.
+
+Integer results (permutations, block lists, counts, gathered rows) must match
+bit for bit; floating point within the tolerances stated in each test.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import clusterattn_oracle as orc
+from paper_2608_26965_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load_library()
+
+
+def to_dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is not None:
+        t = t.to(dtype)
+    return t.to(DEV).contiguous()
+
+
+def store(problem, a):
+    """float32 host array -> device tensor in the problem's storage type ([1,H,n,d])."""
+    return to_dev(a[None], binding.torch_dtype(problem))
+
+
+def random_y(seed, H, n, d, ties=False):
+    r = np.random.default_rng(seed)
+    y = (r.standard_normal((H, n, d)) * np.linspace(2.0, 0.2, d)).astype(np.float32)
+    if ties:
+        y = np.round(y * 2.0) / 2.0                 # heavy duplication, includes +-0
+        y[:, ::5, :] = -0.0
+    return y
+
+
+# ----------------------------------------------------------------------------
+# Splitter on the oracle's own fp32 coordinates: bit-exact permutation,
+# gathered rows, counts; centroids to fp32 rounding.
+# ----------------------------------------------------------------------------
+SPLIT_CASES = [
+    # H, n_q, n_k, d, c_q, c_k, dtype, ties
+    (2, 1024, 1024, 64, 64, 64, "fp32", False),       # the tiny configuration's shape
+    (2, 1000, 1531, 64, 64, 32, "fp32", False),       # ragged: short last clusters
+    (1, 50, 200, 64, 64, 128, "bf16", False),         # n <= c on one side, one split on the other
+    (2, 3000, 4099, 128, 128, 128, "bf16", True),     # many exact ties
+    (1, 2048, 40000, 64, 128, 128, "bf16", False),    # sets larger than the shared-memory window
+    (1, 640, 704, 128, 256, 16, "bf16", False),       # extreme cluster sizes
+]
+
+
+@pytest.mark.parametrize("H,n_q,n_k,d,c_q,c_k,dtype,ties", SPLIT_CASES)
+def test_split_and_gather_bit_exact(H, n_q, n_k, d, c_q, c_k, dtype, ties):
+    r = np.random.default_rng(n_q + n_k)
+    Yq, Yk = random_y(1, H, n_q, d, ties), random_y(2, H, n_k, d, ties)
+    Q = r.standard_normal((H, n_q, d)).astype(np.float32)
+    K = r.standard_normal((H, n_k, d)).astype(np.float32)
+    V = r.standard_normal((H, n_k, d)).astype(np.float32)
+    if dtype == "bf16":
+        Q, K, V = (inputs.round_to_bf16(x) for x in (Q, K, V))
+    p = binding.make_problem(1, H, n_q, n_k, d, dtype, c_q, c_k, 1, flags=binding.CA_Y_IN)
+    plan = binding.Plan(p, DEV)
+    plan.cluster_qk(store(p, Q), store(p, K), store(p, V), Yq=to_dev(Yq[None]), Yk=to_dev(Yk[None]))
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for h in range(H):
+        ref = orc.cluster_qk(Q[h], K[h], V[h], c_q, c_k, Yq32=Yq[h], Yk32=Yk[h])
+        pq, pk = plan.perm_q[0, h].cpu().numpy(), plan.perm_k[0, h].cpu().numpy()
+        assert np.array_equal(pq, ref["perm_q"]), "query permutation differs"
+        assert np.array_equal(pk, ref["perm_k"]), "key permutation differs"
+        assert np.array_equal(plan.count_q[0, h].cpu().numpy(), ref["count_q"])
+        assert np.array_equal(plan.count_k[0, h].cpu().numpy(), ref["count_k"])
+        for got, src, perm, n, c in ((plan.Qp, Q, pq, n_q, c_q), (plan.Kp, K, pk, n_k, c_k),
+                                     (plan.Vp, V, pk, n_k, c_k)):
+            g = got[0, h].float().cpu().numpy()
+            assert np.array_equal(g[:n], src[h][perm])            # rows moved, never changed
+            assert np.all(g[n:] == 0)                             # padding of the short cluster
+        for got, want in ((plan.cq, ref["cq"]), (plan.ck, ref["ck"]), (plan.cv, ref["cv"])):
+            assert np.abs(got[0, h].cpu().numpy() - want).max() < 2e-6 * max(1.0, np.abs(want).max())
+
+
+# ----------------------------------------------------------------------------
+# Full clustering stage: the device computes its own coordinates.  The oracle's
+# splitter run on the device's coordinates must give the same permutation, and
+# the coordinates must satisfy the basis-independent identities of the method.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("name,H,n_q,n_k", [("tiny", 2, 1024, 1024), ("tabular", 1, 2048, 6000),
+                                             ("video480", 1, 4000, 4000)])
+def test_cluster_qk_transforms_and_split(name, H, n_q, n_k):
+    w = inputs.WORKLOADS[name].scaled(heads=H, n_q=n_q, n_k=n_k)
+    if w.kind == "video":
+        w = w.scaled(grid=(5, 25, 32))
+    Q, K, V = inputs.generate(w)
+    p = binding.problem_from_workload(w)
+    plan = binding.Plan(p, DEV, keep_y=True)
+    plan.cluster_qk(store(p, Q), store(p, K), store(p, V))
+    torch.cuda.synchronize()
+    d = w.head_dim
+    for h in range(H):
+        Yq, Yk = plan.Yq[0, h].cpu().numpy(), plan.Yk[0, h].cpu().numpy()
+        # same split decisions as the oracle's splitter on these very coordinates
+        assert np.array_equal(plan.perm_q[0, h].cpu().numpy(), orc.recursive_split(Yq, w.cluster))
+        assert np.array_equal(plan.perm_k[0, h].cpu().numpy(), orc.recursive_split(Yk, w.cluster))
+        # key coordinates are an isometry of the query-aware metric:
+        # |Y_i - Y_j|^2 == (k_i - k_j)^T M (k_i - k_j), M = Q^T Q / n   (Section 3.2.2)
+        M = orc.metric_q(Q[h])
+        r = np.random.default_rng(h)
+        i, j = r.integers(0, n_k, 200), r.integers(0, n_k, 200)
+        dk = K[h][i].astype(np.float64) - K[h][j]
+        want = np.einsum("nd,de,ne->n", dk, M, dk)
+        got = ((Yk[i].astype(np.float64) - Yk[j]) ** 2).sum(1)
+        assert np.abs(got - want).max() <= 2e-3 * want.max()
+        # query coordinates are an isometry of r(q) = R_k q / |R_k q|
+        R_k = orc.psd_root(orc.centered_scatter(K[h]))
+        rq = orc.query_representation(Q[h], R_k)
+        i, j = r.integers(0, n_q, 200), r.integers(0, n_q, 200)
+        want = ((rq[i] - rq[j]) ** 2).sum(1)
+        got = ((Yq[i].astype(np.float64) - Yq[j]) ** 2).sum(1)
+        assert np.abs(got - want).max() <= 2e-3 * max(want.max(), 1e-12)
+        # principal components: centred, decorrelated, variance in descending order
+        for Y, ref in ((Yk, orc.diagonalize(orc.transform_keys(K[h], orc.psd_root(M)))[1]),
+                       (Yq, orc.diagonalize(rq)[1])):
+            Y = Y.astype(np.float64)
+            scale = ref[0]
+            assert np.abs(Y.mean(0)).max() < 1e-3 * np.sqrt(scale)
+            cov = (Y.T @ Y) / Y.shape[0]
+            assert np.abs(np.diag(cov) - ref).max() < 2e-3 * scale          # eigenvalues
+            off = cov - np.diag(np.diag(cov))
+            assert np.abs(off).max() < 2e-3 * scale
+    assert all(v == 0 for v in plan.last_status().values())
+
+
+# ----------------------------------------------------------------------------
+# Block selection on the oracle's centroids (rounded to fp32): exact lists.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("H,n_qc,n_kc,d,keep", [(2, 16, 16, 64, 4), (1, 37, 300, 128, 1), (1, 5, 300, 64, 300),
+                                                  (2, 130, 1024, 64, 128), (1, 9, 2049, 128, 77)])
+def test_select_blocks_exact(H, n_qc, n_kc, d, keep):
+    r = np.random.default_rng(n_qc * n_kc)
+    cq = r.standard_normal((H, n_qc, d)).astype(np.float32)
+    ck = r.standard_normal((H, n_kc, d)).astype(np.float32)
+    ck[:, 3] = ck[:, 1]                      # duplicate centroids: exact score ties
+    ck[:, n_kc - 1] = ck[:, 1]
+    if n_qc > 4:
+        cq[:, 4] = 0.0                       # a zero query centroid: every score ties at 0
+    c = 16
+    p = binding.make_problem(1, H, n_qc * c, n_kc * c, d, "fp32", c, c, keep)
+    plan = binding.Plan(p, DEV)
+    got = plan.select_blocks(to_dev(cq[None]), to_dev(ck[None])).cpu().numpy()[0]
+    torch.cuda.synchronize()
+    near_ties = 0
+    for h in range(H):
+        S = orc.centroid_scores(cq[h], ck[h])
+        want = orc.select_topk(S, keep)
+        for i in range(n_qc):
+            if np.array_equal(got[h, i], want[i]):
+                continue
+            # only a near-tie at the keep-th score may differ (summation order of the dot product)
+            srt = np.sort(S[i])[::-1]
+            gap = srt[keep - 1] - srt[keep] if keep < n_kc else np.inf
+            assert gap < 1e-12 * np.abs(S).max(), (h, i)
+            near_ties += 1
+            assert len(set(got[h, i])) == keep and np.all(np.diff(got[h, i]) > 0)
+    assert near_ties <= 0.001 * H * n_qc + 1
+
+
+# ----------------------------------------------------------------------------
+# Attention on the oracle's permutation and block lists.
+# ----------------------------------------------------------------------------
+def attention_case(w, H, keep, compensate, flags=0, perm_seed=None):
+    Q, K, V = inputs.generate(w.scaled(heads=H))
+    p = binding.problem_from_workload(w, heads=H, keep=keep, compensate=compensate, flags=flags)
+    plan = binding.Plan(p, DEV)
+    c = w.cluster
+    refs = []
+    arrs = {k: [] for k in ("perm_q", "Qp", "Kp", "Vp", "ck", "cv", "count_k", "idx")}
+    for h in range(H):
+        if perm_seed is None:
+            cl = orc.cluster_qk(Q[h], K[h], V[h], c, c)
+        else:                                # any valid permutation must work
+            r = np.random.default_rng(perm_seed + h)
+            pq, pk = r.permutation(w.n_q), r.permutation(w.n_k)
+            cq_, nq_ = orc.centroids(Q[h], pq, c)
+            ck_, nk_ = orc.centroids(K[h], pk, c)
+            cv_, _ = orc.centroids(V[h], pk, c)
+            cl = dict(perm_q=pq, perm_k=pk, cq=cq_, ck=ck_, cv=cv_, count_q=nq_, count_k=nk_)
+        idx = orc.select_blocks(cl["cq"], cl["ck"], keep)
+        ck32, cv32 = cl["ck"].astype(np.float32), cl["cv"].astype(np.float32)
+        o, lse = orc.cluster_attention(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c, c, idx, compensate,
+                                       ck=ck32, cv=cv32, count_k=cl["count_k"])
+        refs.append((o, lse))
+
+        def pad(x, perm, n):
+            out = np.zeros((-(-n // c) * c, x.shape[1]), np.float32)
+            out[:n] = x[perm]
+            return out
+        arrs["perm_q"].append(cl["perm_q"].astype(np.int32))
+        arrs["Qp"].append(pad(Q[h], cl["perm_q"], w.n_q))
+        arrs["Kp"].append(pad(K[h], cl["perm_k"], w.n_k))
+        arrs["Vp"].append(pad(V[h], cl["perm_k"], w.n_k))
+        arrs["ck"].append(ck32)
+        arrs["cv"].append(cv32)
+        arrs["count_k"].append(cl["count_k"].astype(np.int32))
+        arrs["idx"].append(idx.astype(np.int32))
+    st = {k: np.stack(v)[None] for k, v in arrs.items()}
+    dt = binding.torch_dtype(p)
+    O, lse = plan.cluster_attention_fwd(to_dev(st["Qp"], dt), to_dev(st["Kp"], dt), to_dev(st["Vp"], dt),
+                                        to_dev(st["ck"]), to_dev(st["cv"]), to_dev(st["count_k"]),
+                                        to_dev(st["idx"]), to_dev(st["perm_q"]))
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    return O[0].float().cpu().numpy(), lse[0].cpu().numpy(), refs
+
+
+@pytest.mark.parametrize("compensate", [True, False])
+def test_attention_fp32_tiny_configuration(compensate):
+    w = inputs.WORKLOADS["tiny"]
+    O, lse, refs = attention_case(w, 2, w.keep, compensate)
+    for h, (o_ref, lse_ref) in enumerate(refs):
+        assert np.abs(O[h] - o_ref).max() < 1e-5
+        assert np.abs(lse[h] - lse_ref).max() < 1e-5 * max(1.0, np.abs(lse_ref).max())
+
+
+@pytest.mark.parametrize("n_q,n_k,c,keep", [(1000, 1531, 64, 5), (300, 300, 128, 3), (260, 4000, 32, 125)])
+def test_attention_fp32_ragged_and_arbitrary_permutation(n_q, n_k, c, keep):
+    w = inputs.WORKLOADS["tiny"].scaled(n_q=n_q, n_k=n_k, cluster=c)
+    O, lse, refs = attention_case(w, 1, keep, True, perm_seed=7)
+    assert np.abs(O[0] - refs[0][0]).max() < 1e-5
+    assert np.abs(lse[0] - refs[0][1]).max() < 1e-5 * max(1.0, np.abs(refs[0][1]).max())
+
+
+def bf16_close(O, o_ref):
+    return np.abs(O - o_ref).max() <= 2e-2 and np.linalg.norm(O - o_ref) <= 5e-3 * np.linalg.norm(o_ref)
+
+
+@pytest.mark.parametrize("name,n_q,n_k,keep,compensate,flags", [
+    ("tabular", 1024, 4096, 4, True, 0), ("tabular", 1024, 4096, 4, False, 0),
+    ("video480", 1000, 1000, 2, True, 0), ("sweep", 2048, 2048, 16, True, 0),
+    ("tabular", 512, 2048, 4, True, binding.CA_ATTN_FP32),
+])
+def test_attention_bf16(name, n_q, n_k, keep, compensate, flags):
+    w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k)
+    if w.kind == "video":
+        w = w.scaled(grid=(5, 10, 20))
+    O, lse, refs = attention_case(w, 2, keep, compensate, flags=flags)
+    for h, (o_ref, lse_ref) in enumerate(refs):
+        assert bf16_close(O[h], o_ref), (np.abs(O[h] - o_ref).max(),
+                                         np.linalg.norm(O[h] - o_ref) / np.linalg.norm(o_ref))
+        assert np.abs(lse[h] - lse_ref).max() < 2e-2
+
+
+def test_all_blocks_kept_is_dense_attention_on_device():
+    w = inputs.WORKLOADS["tiny"]
+    O, lse, _ = attention_case(w, 1, w.n_kc, False)
+    Q, K, V = inputs.generate(w.scaled(heads=1))
+    od, lsed = orc.dense_attention(Q[0], K[0], V[0], return_lse=True)
+    assert np.abs(O[0] - od).max() < 1e-5 and np.abs(lse[0] - lsed).max() < 1e-5
+
+
+# ----------------------------------------------------------------------------
+# The whole path on the tiny configuration, every stage on the device.
+# ----------------------------------------------------------------------------
+def test_end_to_end_tiny_configuration():
+    w = inputs.WORKLOADS["tiny"]
+    Q, K, V = inputs.generate(w)
+    p = binding.problem_from_workload(w)
+    plan = binding.Plan(p, DEV, keep_y=True)
+    O = plan.forward(store(p, Q), store(p, K), store(p, V), want_lse=True)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    moved = 0
+    for h in range(w.heads):
+        pq, pk = plan.perm_q[0, h].cpu().numpy(), plan.perm_k[0, h].cpu().numpy()
+        idx = plan.block_idx[0, h].cpu().numpy()
+        # selection agrees with the oracle's on the device's own centroids
+        want_idx = orc.select_blocks(plan.cq[0, h].cpu().numpy(), plan.ck[0, h].cpu().numpy(), w.keep)
+        assert np.array_equal(idx, want_idx)
+        # attention agrees with the oracle's on the device's own clustering and selection
+        o_ref, lse_ref = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, w.cluster, w.cluster, idx, True,
+                                               ck=plan.ck[0, h].cpu().numpy(), cv=plan.cv[0, h].cpu().numpy(),
+                                               count_k=plan.count_k[0, h].cpu().numpy())
+        assert np.abs(O[0, h].cpu().numpy() - o_ref).max() < 1e-5
+        # informative: rows whose cluster differs from the all-oracle clustering
+        ref = orc.cluster_qk(Q[h], K[h], V[h], w.cluster, w.cluster)
+        for mine, theirs in ((pq, ref["perm_q"]), (pk, ref["perm_k"])):
+            a = {frozenset(mine[j * 64:(j + 1) * 64].tolist()) for j in range(16)}
+            b = {frozenset(theirs[j * 64:(j + 1) * 64].tolist()) for j in range(16)}
+            moved += 64 * len(a - b)
+    print(f"rows in clusters that differ from the all-fp64 clustering: {moved} of {4 * 1024}")
