@@ -1,0 +1,380 @@
+#!/usr/bin/env python
+"""Benchmark of the ClusterAttention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--workload tabular|video480|video720|sweep|tiny] [--no-cpu-baseline]
+
+One "step" is one pass of the whole hot path (cluster_qk + select_blocks +
+cluster_attention_fwd) over one batch of seeded synthetic input.  The default
+workload is the tabular-shaped configuration (8 heads, d=64, bf16, 16,384
+queries attending to 131,072 keys, clusters of 128, 1/8 of the key clusters
+kept, compensation on).  The metric is the throughput of the whole path in
+TFLOP/s over the computed blocks: 4*N_q*d*(keep*c + padded centroid columns)
+flops per head divided by the time of the step.
+
+With N > 1 (launched under torch.distributed.run) every rank runs an
+independent replica on its own GPU: heads are independent problems and the
+path has no exchange step, so there is no collective on the data path.
+
+`--impl reference` times the fp64 CPU oracle on a bounded sample of the same
+workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "clusterattention_hot_path_block_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="tabular")
+    ap.add_argument("--keep", type=int, default=0, help="override kept key clusters per query cluster")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-dense", action="store_true")
+    return ap.parse_args()
+
+
+def block_flops(w, heads, keep=None):
+    """Flops over the computed blocks: selected key rows plus centroid columns (padded to 128)."""
+    keep = w.keep if keep is None else keep
+    cols = keep * w.cluster + (-(-w.n_kc // 128) * 128 if w.compensate else 0)
+    return 4.0 * w.n_q * w.head_dim * cols * heads
+
+
+def dense_flops(w, heads):
+    return 4.0 * w.n_q * w.n_k * w.head_dim * heads
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+# ------------------------------------------------------------------------------
+# CPU oracle on a bounded sample (the reference arm and the cpu_baseline leg)
+# ------------------------------------------------------------------------------
+def oracle_sample_step(w, Q, K, V, n_query_clusters=8, budget_rows=32768):
+    """One oracle pass on a sample: a prefix of one head's rows (so clustering
+    stays within seconds) and `n_query_clusters` query clusters of attention.
+    Returns (flops over the blocks computed, seconds)."""
+    from oracle import clusterattn_oracle as orc
+    n_k = min(w.n_k, budget_rows)
+    n_q = min(w.n_q, budget_rows)
+    c = w.cluster
+    n_kc = -(-n_k // c)
+    keep = max(1, min(n_kc, round(w.keep * n_kc / w.n_kc)))
+    Qs, Ks, Vs = Q[:n_q], K[:n_k], V[:n_k]
+    t0 = time.perf_counter()
+    cl = orc.cluster_qk(Qs, Ks, Vs, c, c)
+    idx = orc.select_blocks(cl["cq"], cl["ck"], keep)
+    n_qc = -(-n_q // c)
+    sample = list(range(0, n_qc, max(1, n_qc // n_query_clusters)))[:n_query_clusters]
+    orc.cluster_attention(Qs, Ks, Vs, cl["perm_q"], cl["perm_k"], c, c, idx, w.compensate, ck=cl["ck"],
+                          cv=cl["cv"], count_k=cl["count_k"], query_clusters=sample)
+    dt = time.perf_counter() - t0
+    cols = keep * c + (n_kc if w.compensate else 0)
+    flops = 4.0 * len(sample) * c * w.head_dim * cols
+    desc = (f"1 head, first {n_q} queries x {n_k} keys of the workload: clustering and selection in full, "
+            f"attention on {len(sample)} of {n_qc} query clusters, keep={keep} of {n_kc}")
+    return flops, dt, desc
+
+
+def run_reference(args, w):
+    from paper_2608_26965_b200 import inputs
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    Q, K, V = inputs.generate_head(w, 0)
+    times, flops, desc = [], 0.0, ""
+    for i in range(args.warmup + args.steps):
+        flops, dt, desc = oracle_sample_step(w, Q, K, V, n_query_clusters=4, budget_rows=16384)
+        if i >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = flops * len(times) / total / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": host_cores(), "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.path = tempfile.mktemp(suffix=".csv")
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(device_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2])); power.append(float(f[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2608_26965_b200 import binding, build, inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    distributed = world > 1
+    if distributed:
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        build.build()
+    if distributed:
+        dist.barrier()
+    binding.load_library()
+
+    keep = args.keep or w.keep
+    heads = w.heads
+    p = binding.problem_from_workload(w, keep=keep)
+    dt = binding.torch_dtype(p)
+    Qh, Kh, Vh = inputs.generate(w)                        # every replica runs the same seeded batch
+    pin = lambda a: torch.from_numpy(a[None]).to(dt).pin_memory()
+    Q_host, K_host, V_host = pin(Qh), pin(Kh), pin(Vh)
+    Q, K, V = (t.to(dev, non_blocking=True) for t in (Q_host, K_host, V_host))
+    plan = binding.Plan(p, dev)
+    O_host = torch.empty(plan.O.shape, dtype=dt).pin_memory()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if distributed:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def max_over_ranks(x):
+        if not distributed:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def step(events=None):
+        if events is not None:
+            events[0].record(stream)
+        plan.cluster_qk(Q, K, V)
+        if events is not None:
+            events[1].record(stream)
+        plan.select_blocks()
+        if events is not None:
+            events[2].record(stream)
+        plan.cluster_attention_fwd(want_lse=False)
+        if events is not None:
+            events[3].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert all(v == 0 for v in plan.last_status().values()), plan.last_status()
+
+    # ---- timed region: device-resident inputs (larger than L2, so no flush is needed)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+    launches0 = binding.kernel_launches()
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    t_start = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    t_start.record(stream)
+    for i in range(args.steps):
+        step(ev[i])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = binding.kernel_launches() - launches0
+    total_ms = max_over_ranks(t_start.elapsed_time(t_end))
+    ms_per_step = total_ms / args.steps
+    stage_ms = {
+        "cluster_qk": float(np.mean([e[0].elapsed_time(e[1]) for e in ev])),
+        "select_blocks": float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
+        "cluster_attention_fwd": float(np.mean([e[2].elapsed_time(e[3]) for e in ev])),
+    }
+    flops_step = block_flops(w, heads, keep)
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e12
+
+    # ---- end to end through the same calls with HOST buffers (pinned), copies inside the region
+    e2e = None
+    if not args.no_e2e:
+        def e2e_step():
+            Q.copy_(Q_host, non_blocking=True)
+            K.copy_(K_host, non_blocking=True)
+            V.copy_(V_host, non_blocking=True)
+            step()
+            O_host.copy_(plan.O, non_blocking=True)
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(args.steps):
+            e2e_step()
+        b.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(a.elapsed_time(b)) / args.steps
+        nbytes = lambda t: t.numel() * t.element_size()
+        e2e = {"value": world * flops_step / (e2e_ms * 1e-3) / 1e12, "unit": UNIT, "ms_per_step": e2e_ms,
+               "h2d_bytes_per_step": nbytes(Q_host) + nbytes(K_host) + nbytes(V_host),
+               "d2h_bytes_per_step": nbytes(O_host)}
+
+    # ---- dense attention on the same GPU (library kernel with every block kept, and torch SDPA)
+    dense = None
+    if not args.no_dense and rank == 0:
+        dense = {}
+        try:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            with torch.no_grad():
+                for _ in range(2):
+                    torch.nn.functional.scaled_dot_product_attention(Q, K, V)
+                torch.cuda.synchronize()
+                a.record(stream)
+                for _ in range(5):
+                    torch.nn.functional.scaled_dot_product_attention(Q, K, V)
+                b.record(stream)
+                torch.cuda.synchronize()
+            dense["torch_sdpa_ms"] = a.elapsed_time(b) / 5
+            dense["torch_sdpa_tflops"] = dense_flops(w, heads) / (dense["torch_sdpa_ms"] * 1e-3) / 1e12
+            dense["speedup_vs_torch_sdpa"] = dense["torch_sdpa_ms"] / ms_per_step
+        except Exception as exc:  # noqa: BLE001
+            dense["torch_sdpa_error"] = str(exc)[:200]
+
+    if distributed:
+        dist.barrier()
+    if rank != 0:
+        if distributed:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    attn_ms = stage_ms["cluster_attention_fwd"]
+    attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.0 / 16.0
+    roofline = {
+        "kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": attn_tflops, "peak": peak,
+        "peak_source": f"{peak_kind} bf16 burst", "unit": "TFLOP/s", "frac": attn_tflops / peak,
+        "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+    }
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+        "config": {"workload": w.name, "heads": heads, "head_dim": w.head_dim, "n_q": w.n_q, "n_k": w.n_k,
+                   "cluster": w.cluster, "keep": keep, "n_kc": w.n_kc, "compensate": w.compensate,
+                   "parallelism": "replicas" if world > 1 else "single",
+                   "l2": "inputs larger than L2 (no flush)"},
+        "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),
+        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "dense": dense,
+    }
+    if not args.no_cpu_baseline:
+        # the oracle as it stands on whole heads until about 10 s of CPU work are spent
+        flops = secs = 0.0
+        used = 0
+        for h in range(heads):
+            f, s_, desc = oracle_sample_step(w, Qh[h], Kh[h], Vh[h], n_query_clusters=1 << 30,
+                                             budget_rows=1 << 30)
+            flops, secs, used = flops + f, secs + s_, used + 1
+            if secs > 10.0:
+                break
+        line["cpu_baseline"] = {"value": flops / secs / 1e12, "unit": UNIT, "cores": host_cores(),
+                                "kind": "oracle", "seconds": secs,
+                                "sample": f"{used} of {heads} heads in full (all stages, fp64 numpy)"}
+    print(json.dumps(line))
+    if distributed:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_2608_26965_b200 import inputs
+    w = inputs.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -172,7 +172,7 @@ class Plan:
         self.Yq = torch.empty((B, H, p.n_q, D), dtype=f32, device=dev) if keep_y else None
         self.Yk = torch.empty((B, H, p.n_k, D), dtype=f32, device=dev) if keep_y else None
         sizes = workspace_bytes(p)
-        self.ws = {k: torch.empty(max(v, 256), dtype=torch.uint8, device=dev) for k, v in sizes.items()}
+        self.ws = {k: torch.zeros(max(v, 256), dtype=torch.uint8, device=dev) for k, v in sizes.items()}
 
     # -- the three entry points ------------------------------------------------
     def cluster_qk(self, Q, K, V, Yq=None, Yk=None, stream=None):

@@ -99,7 +99,7 @@ def test_cluster_qk_transforms_and_split(name, H, n_q, n_k):
     if w.kind == "video":
         w = w.scaled(grid=(5, 25, 32))
     Q, K, V = inputs.generate(w)
-    p = binding.problem_from_workload(w)
+    p = binding.problem_from_workload(w, keep=min(w.keep, w.n_kc))
     plan = binding.Plan(p, DEV, keep_y=True)
     plan.cluster_qk(store(p, Q), store(p, K), store(p, V))
     torch.cuda.synchronize()
