@@ -97,7 +97,7 @@ int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select
   CA_TRY(check_problem(p));
   if (cluster_ws) *cluster_ws = carve_cluster(p, nullptr, true, true).bytes;
   if (select_ws) *select_ws = kStatusBytes;
-  if (attn_ws) *attn_ws = kStatusBytes;
+  if (attn_ws) *attn_ws = attn_tc_supported(*p) ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   return CA_OK;
 }
 
@@ -186,10 +186,14 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
   const void* ptrs[] = {Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O};
   for (const void* x : ptrs)
     if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
-  if (!ws || ws_bytes < kStatusBytes) return CA_ERR_WORKSPACE;
+  const bool tensor_cores = attn_tc_supported(*p);
+  const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
+  if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  if (tensor_cores)
+    return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, scale, O, lse, ws, st);
   return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, scale, O, lse, st);
 }
 

@@ -44,4 +44,11 @@ int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, cons
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* perm_q, float scale, void* O, float* lse, cudaStream_t st);
 
+// attn_tc.cu
+bool attn_tc_supported(const ca_problem_t& pr);
+size_t attn_tc_workspace_bytes(const ca_problem_t& pr);
+int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp, const float* ck,
+                   const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* perm_q,
+                   float scale, void* O, float* lse, void* ws, cudaStream_t st);
+
 }  // namespace ca
