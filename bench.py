@@ -51,6 +51,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="tabular")
     ap.add_argument("--keep", type=int, default=0, help="override kept key clusters per query cluster")
+    ap.add_argument("--heads", type=int, default=0, help="run only the first HEADS heads (profiling captures)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
@@ -370,6 +371,8 @@ def main():
     args = parse_args()
     from paper_2608_26965_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
+    if args.heads:
+        w = w.scaled(heads=args.heads)
     if args.impl == "reference":
         run_reference(args, w)
     else:

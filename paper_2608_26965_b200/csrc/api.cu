@@ -130,16 +130,17 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     double* M = w.metric;
     double* CK = w.metric + (size_t)P * DD;
     CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, M, CK, st));
-    // roots R_q, R_k
-    CA_TRY(launch_eigh(w.metric, 2 * P, D, 0, w.roots, w.roots32, nullptr, st));
+    // factors F_q F_q^T = M and F_k F_k^T = C_K (they stand in for the symmetric roots:
+    // any factor yields the same principal-component coordinates)
+    CA_TRY(launch_cholesky_factor(w.metric, 2 * P, D, w.roots, w.roots32, st));
     double* Rq = w.roots;
     const float* Rk32 = w.roots32 + (size_t)P * DD;
-    // covariance of the transformed keys K R_q:  R_q C_K R_q / n_k
+    // covariance of the transformed keys K F_q:  F_q^T C_K F_q / n_k
     double* covK = w.cov;
     double* covQ = w.cov + (size_t)P * DD;
-    CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, w.tmp, nullptr, st));
-    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, 1.0 / (double)p->n_k, covK, nullptr, st));
-    // query representation r(q) = R_k q / |R_k q| and its covariance
+    CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
+    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, 1.0 / (double)p->n_k, 0, covK, nullptr, st));
+    // query representation r(q) = F_k^T q / |F_k^T q| and its covariance
     CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, 1, w.Qprime, st));
     CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
@@ -148,8 +149,8 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     double* EK = w.basis;
     double* EQ = w.basis + (size_t)P * DD;
     const float* EQ32 = w.basis32 + (size_t)P * DD;
-    // keys: Y = (K - kbar) R_q E_K ; queries: Y = (r(q) - mean) E_Q
-    CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, w.WK, w.WK32, st));
+    // keys: Y = (K - kbar) F_q E_K ; queries: Y = (r(q) - mean) E_Q
+    CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, 0, w.WK, w.WK32, st));
     CA_TRY(launch_bias(w.sumK, w.WK, P, D, p->n_k, w.biasK, st));
     CA_TRY(launch_bias(w.sumQp, EQ, P, D, p->n_q, w.biasQ, st));
     CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));

@@ -12,7 +12,7 @@ template <int D>
 struct EighCfg {
   static constexpr int H = D / 2;                       // rotations per step
   static constexpr int NBLK = H * (H + 1) / 2;          // 2x2 blocks with k1 <= k2
-  static constexpr int THREADS = (D == 128) ? 1024 : 256;
+  static constexpr int THREADS = (D == 128) ? 1024 : 512;
   static constexpr int LDA = D + 1;
 };
 
@@ -71,7 +71,7 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
     if (tid == 0) {
       double o = 0.0, t = 0.0;
       for (int w = 0; w < NT / 32; ++w) { o += red[w]; t += red[32 + w]; }
-      *flag = (o <= 1e-28 * t) ? 1 : 0;
+      *flag = (o <= 1e-24 * t) ? 1 : 0;       // off-diagonal norm below 1e-12 of the matrix norm
     }
     __syncthreads();
     if (*flag) break;
@@ -200,6 +200,81 @@ int launch_eigh(const double* A, int count, int D, int mode, double* out64, floa
   return CA_OK;
 }
 
+
+// ---------------------------------------------------------------------------
+// Factor of a positive semi-definite matrix: lower-triangular F with F F^T = A
+// (right-looking Cholesky in double, one CTA per matrix).  A pivot that is not
+// above 1e-12 of the largest diagonal entry marks a direction in which the
+// (pseudo-)metric is zero: its column of F is set to zero, which is the
+// counterpart of clamping small or negative eigenvalues (Section 3.2.2).
+// Any factor of the metric matrix gives the same principal-component
+// coordinates as its symmetric root, because the two differ by a rotation.
+// ---------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(1024) cholesky_factor_kernel(const double* __restrict__ A_in,
+                                                               double* __restrict__ out64,
+                                                               float* __restrict__ out32) {
+  constexpr int LDA = D + 1;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* A = reinterpret_cast<double*>(smem_raw);       // [D][LDA], lower triangle is updated in place
+  __shared__ double s_tol;
+  __shared__ double s_inv;
+  const int tid = threadIdx.x, NT = blockDim.x;
+  const double* Ain = A_in + (size_t)blockIdx.x * D * D;
+  for (int e = tid; e < D * D; e += NT) {
+    const int i = e / D, j = e % D;
+    A[i * LDA + j] = 0.5 * (Ain[i * D + j] + Ain[j * D + i]);
+  }
+  __syncthreads();
+  if (tid == 0) {
+    double mx = 0.0;
+    for (int i = 0; i < D; ++i) mx = fmax(mx, A[i * LDA + i]);
+    s_tol = 1e-12 * mx;
+  }
+  __syncthreads();
+  for (int j = 0; j < D; ++j) {
+    if (tid == 0) {
+      const double piv = A[j * LDA + j];
+      s_inv = (piv > s_tol) ? rsqrt(piv) : 0.0;
+    }
+    __syncthreads();
+    const double inv = s_inv;
+    // column j of F (rows j..D-1); a dropped pivot gives a zero column
+    for (int i = j + tid; i < D; i += NT) A[i * LDA + j] *= inv;
+    __syncthreads();
+    // trailing update of the lower triangle
+    const int rem = D - 1 - j;
+    for (int e = tid; e < rem * rem; e += NT) {
+      const int i = j + 1 + e / rem, k = j + 1 + e % rem;
+      if (k <= i) A[i * LDA + k] -= A[i * LDA + j] * A[k * LDA + j];
+    }
+    __syncthreads();
+  }
+  double* o64 = out64 + (size_t)blockIdx.x * D * D;
+  float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
+  for (int e = tid; e < D * D; e += NT) {
+    const int i = e / D, j = e % D;
+    const double v = (j <= i) ? A[i * LDA + j] : 0.0;
+    o64[e] = v;
+    if (o32) o32[e] = (float)v;
+  }
+}
+
+int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st) {
+  const size_t smem = sizeof(double) * D * (D + 1);
+  if (D == 64) {
+    auto k = cholesky_factor_kernel<64>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<count, 512, smem, st>>>(A, out64, out32);
+  } else {
+    auto k = cholesky_factor_kernel<128>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<count, 1024, smem, st>>>(A, out64, out32);
+  }
+  CA_LAUNCH_CHECK();
+  return CA_OK;
+}
+
 // ---------------------------------------------------------------------------
 // d x d algebra in double (one CTA per problem unless noted).
 // ---------------------------------------------------------------------------
@@ -227,9 +302,10 @@ __global__ void covariance_kernel(const double* __restrict__ gram, const double*
   cov[o] = gram[o] / n - (sum[(size_t)p * D + i] / n) * (sum[(size_t)p * D + j] / n);
 }
 
-// C[p] = alpha * A[p] * B[p]; optional fp32 copy.
+// C[p] = alpha * op(A[p]) * B[p], op = transpose if trans_a; optional fp32 copy.
 __global__ void small_matmul_kernel(const double* __restrict__ A, const double* __restrict__ B, int D,
-                                    double alpha, double* __restrict__ C, float* __restrict__ C32) {
+                                    double alpha, int trans_a, double* __restrict__ C,
+                                    float* __restrict__ C32) {
   const int p = blockIdx.y;
   const double* Ap = A + (size_t)p * D * D;
   const double* Bp = B + (size_t)p * D * D;
@@ -237,7 +313,8 @@ __global__ void small_matmul_kernel(const double* __restrict__ A, const double* 
   if (e >= D * D) return;
   const int i = e / D, j = e % D;
   double s = 0.0;
-  for (int k = 0; k < D; ++k) s += Ap[i * D + k] * Bp[k * D + j];
+  if (trans_a) for (int k = 0; k < D; ++k) s += Ap[k * D + i] * Bp[k * D + j];
+  else for (int k = 0; k < D; ++k) s += Ap[i * D + k] * Bp[k * D + j];
   s *= alpha;
   C[(size_t)p * D * D + e] = s;
   if (C32) C32[(size_t)p * D * D + e] = (float)s;
@@ -267,9 +344,9 @@ int launch_covariance(const double* gram, const double* sum, int P, int D, int n
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
-int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, double* C,
-                        float* C32, cudaStream_t st) {
-  small_matmul_kernel<<<dim3(ceil_div(D * D, 256), P), 256, 0, st>>>(A, B, D, alpha, C, C32);
+int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
+                        double* C, float* C32, cudaStream_t st) {
+  small_matmul_kernel<<<dim3(ceil_div(D * D, 256), P), 256, 0, st>>>(A, B, D, alpha, trans_a, C, C32);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }

@@ -20,8 +20,9 @@ int launch_metric(const double* gramQ, const double* gramK, const double* sumK, 
                   int n_k, double* M, double* CK, cudaStream_t st);
 int launch_covariance(const double* gram, const double* sum, int P, int D, int n, double* cov,
                       cudaStream_t st);
-int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, double* C,
-                        float* C32, cudaStream_t st);
+int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
+                        double* C, float* C32, cudaStream_t st);
+int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st);
 int launch_bias(const double* sum, const double* W, int P, int D, int n, float* bias, cudaStream_t st);
 
 // split.cu
