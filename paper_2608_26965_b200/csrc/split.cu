@@ -1,5 +1,5 @@
 // Diagonalized recursive splitting (Section 3.2.1) on fp32 principal-component
-// coordinates.  One launch per tree level; one CTA per set of that level.
+// coordinates.
 //
 // A set [lo, lo+s) keeps its rows in ascending original order.  A split
 //   1. takes m = min(d, s) rows at positions floor(j*s/m), sums each coordinate
@@ -9,13 +9,29 @@
 //      smallest (value, row) along it, L = c * floor((s + c) / (2c));
 //   3. moves the L smallest rows to [lo, lo+L) and the others to [lo+L, lo+s),
 //      both sides keeping their order (stable partition by prefix sums).
-// Nothing here depends on floating-point rounding except step 1, whose
-// operation order is fixed, so the permutation is reproducible bit for bit.
+// Nothing depends on floating-point rounding except step 1, whose operation
+// order is fixed, so the permutation is reproducible bit for bit.
+//
+// Two kernels.  Large sets: one launch per tree level, a thread-block cluster of
+// up to 8 CTAs per set; each CTA keeps its slice of keys and rows in shared
+// memory, histograms and partition offsets are combined through distributed
+// shared memory (hardware cluster barriers, no spin waits).  Sets of at most
+// kTailRows rows: one CTA finishes the whole subtree in shared memory, all
+// subsets of a level side by side, and writes the permutation once.
+#include <climits>
+#include <cooperative_groups.h>
+
 #include "kernels.h"
 
 namespace ca {
 
-constexpr int kMaxSplitThreads = 1024;
+namespace cg = cooperative_groups;
+
+constexpr int kSplitThreads = 1024;
+constexpr int kSmemRowsMax = 24576;      // rows a CTA stages (8 bytes each)
+constexpr int kMaxCluster = 8;
+constexpr int kTailRowsMax = 4096;
+constexpr int kTailSegs = 32;            // subsets a tail CTA splits side by side
 
 struct SegmentRef { int lo, size, active; };
 
@@ -42,12 +58,33 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// variance of coordinate t over the subsample of a set (fixed operation order)
+__device__ __forceinline__ double subsample_variance(const float* __restrict__ Y, int D, int t,
+                                                     const int32_t* rows, bool identity, int lo, int s,
+                                                     int m) {
+  double sum = 0.0;
+  for (int j = 0; j < m; ++j) {
+    const int pos = (int)(((long long)j * s) / m);
+    const int row = identity ? lo + pos : rows[pos];
+    sum = __dadd_rn(sum, (double)__ldg(Y + (size_t)row * D + t));
+  }
+  const double mean = sum / (double)m;
+  double acc = 0.0;
+  for (int j = 0; j < m; ++j) {
+    const int pos = (int)(((long long)j * s) / m);
+    const int row = identity ? lo + pos : rows[pos];
+    const double dev = __dsub_rn((double)__ldg(Y + (size_t)row * D + t), mean);
+    acc = __dadd_rn(acc, __dmul_rn(dev, dev));
+  }
+  return acc / (double)m;
+}
+
 struct SplitSide {
   const float* Y;          // [P][n][D]
   const int32_t* perm_in;  // [P][n] or null (identity)
   int32_t* perm_out;       // [P][n]
-  uint32_t* keybuf;        // [P][n] staging for sets larger than the shared-memory window
-  int n, c, levels;
+  uint32_t* keybuf;        // [P][n] staging for sets larger than the shared-memory windows
+  int n, c, levels, tail_level;
 };
 
 struct SplitParams {
@@ -55,21 +92,29 @@ struct SplitParams {
   int D, level, problems, smem_rows;
 };
 
-__global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const SplitParams prm) {
+// ---------------------------------------------------------------------------
+// One level of the large sets.  grid.x = slots * cluster size.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitParams prm) {
+  cg::cluster_group cluster = cg::this_cluster();
+  const int csize = (int)cluster.num_blocks();
+  const int crank = (int)cluster.block_rank();
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem_raw);       // [smem_rows]
-  int32_t* s_rows = reinterpret_cast<int32_t*>(s_keys + prm.smem_rows);   // [smem_rows]
+  uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem_raw);                  // [smem_rows]
+  int32_t* s_rows = reinterpret_cast<int32_t*>(s_keys + prm.smem_rows);      // [smem_rows]
   __shared__ int s_hist[256];
+  __shared__ int s_total[256];
   __shared__ double s_var[128];
   __shared__ int s_sub[128];
   __shared__ int s_warp[2 * 32];
-  __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank
+  __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank, 3: chunk total
+  __shared__ int s_counts[2];      // this CTA's (less, equal) totals
 
   const int which = blockIdx.y / prm.problems;
   const int p = blockIdx.y % prm.problems;
   const SplitSide sd = prm.side[which];
-  if (prm.level >= sd.levels) return;
-  const SegmentRef seg = locate_segment(sd.n, sd.c, prm.level, blockIdx.x);
+  if (prm.level >= sd.tail_level) return;             // uniform over the cluster
+  const SegmentRef seg = locate_segment(sd.n, sd.c, prm.level, blockIdx.x / csize);
   if (!seg.active) return;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
   const int D = prm.D;
@@ -79,11 +124,12 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
   const int lo = seg.lo, s = seg.size;
 
   if (s <= sd.c) {                                   // final set: carry over
-    for (int i = tid; i < s; i += nt) pout[lo + i] = pin ? pin[lo + i] : lo + i;
+    if (crank == 0)
+      for (int i = tid; i < s; i += nt) pout[lo + i] = pin ? pin[lo + i] : lo + i;
     return;
   }
 
-  // ---- 1. coordinate of largest subsample variance
+  // ---- 1. coordinate of largest subsample variance (every CTA of the cluster computes it)
   const int m = min(D, s);
   if (tid < m) {
     const int pos = lo + (int)(((long long)tid * s) / m);
@@ -118,38 +164,51 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
   __syncthreads();
   const int coord = s_scalar[0];
 
-  // ---- 2. keys
-  const bool in_smem = s <= prm.smem_rows;
-  uint32_t* keys = in_smem ? s_keys : sd.keybuf + (size_t)p * sd.n + lo;
-  for (int i = tid; i < s; i += nt) {
-    const int row = pin ? pin[lo + i] : lo + i;
+  // ---- 2. keys of this CTA's slice [c0, c1) of the set
+  const int chunk = (s + csize - 1) / csize;
+  const int c0 = min(s, crank * chunk), c1 = min(s, c0 + chunk);
+  const int cs = c1 - c0;
+  const bool in_smem = cs <= prm.smem_rows;
+  uint32_t* keys = in_smem ? s_keys : sd.keybuf + (size_t)p * sd.n + lo + c0;
+  for (int i = tid; i < cs; i += nt) {
+    const int row = pin ? pin[lo + c0 + i] : lo + c0 + i;
     keys[i] = order_key(__ldg(Y + (size_t)row * D + coord));
     if (in_smem) s_rows[i] = row;
   }
   __syncthreads();
 
-  // ---- radix selection of the L-th smallest key (8 bits per pass)
+  // ---- radix selection of the L-th smallest key of the whole set (8 bits per pass)
   const int L = sd.c * ((s + sd.c) / (2 * sd.c));
   uint32_t prefix = 0, mask = 0;
   int remaining = L;                                // 1-based rank among the candidates
   for (int shift = 24; shift >= 0; shift -= 8) {
     for (int b = tid; b < 256; b += nt) s_hist[b] = 0;
     __syncthreads();
-    for (int i0 = 0; i0 < s; i0 += nt) {
+    for (int i0 = 0; i0 < cs; i0 += nt) {
       const int i = i0 + tid;
-      const bool ok = i < s;
+      const bool ok = i < cs;
       const uint32_t k = ok ? keys[i] : 0u;
       const bool cand = ok && ((k & mask) == prefix);
       const int bin = cand ? (int)((k >> shift) & 255u) : -1;
-      // one atomic per distinct bin in the warp
-      const unsigned peers = __match_any_sync(0xffffffffu, bin);
+      const unsigned peers = __match_any_sync(0xffffffffu, bin);   // one atomic per distinct bin
       if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+    }
+    if (csize > 1) {
+      cluster.sync();                                // every slice has counted
+      if (tid < 256) {
+        int sum = 0;
+        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(s_hist, r)[tid];
+        s_total[tid] = sum;
+      }
+    } else {
+      __syncthreads();
+      if (tid < 256) s_total[tid] = s_hist[tid];
     }
     __syncthreads();
     if (warp == 0) {
       int local[8]; int sum = 0;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { local[j] = s_hist[lane * 8 + j]; sum += local[j]; }
+      for (int j = 0; j < 8; ++j) { local[j] = s_total[lane * 8 + j]; sum += local[j]; }
       int incl = sum;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -165,7 +224,7 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
         before += local[j];
       }
     }
-    __syncthreads();
+    if (csize > 1) cluster.sync(); else __syncthreads();   // peers are done reading s_hist
     prefix |= (uint32_t)s_scalar[1] << shift;
     mask |= 255u << shift;
     remaining = s_scalar[2];
@@ -174,15 +233,36 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
   const uint32_t thr = prefix;
   const int eq_left = remaining;        // how many rows equal to the threshold go down
 
-  // ---- 3. stable two-sided partition
-  int less_before = 0, eq_before = 0;   // running totals over earlier positions
-  for (int i0 = 0; i0 < s; i0 += nt) {
+  // ---- 3. stable two-sided partition.  Offsets of this slice = totals of the earlier slices.
+  int less_before = 0, eq_before = 0;
+  if (csize > 1) {
+    int nl = 0, ne = 0;
+    for (int i = tid; i < cs; i += nt) {
+      const uint32_t k = keys[i];
+      nl += k < thr;
+      ne += k == thr;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+      nl += __shfl_xor_sync(0xffffffffu, nl, o);
+      ne += __shfl_xor_sync(0xffffffffu, ne, o);
+    }
+    if (tid == 0) { s_counts[0] = 0; s_counts[1] = 0; }
+    __syncthreads();
+    if (lane == 0) { atomicAdd(&s_counts[0], nl); atomicAdd(&s_counts[1], ne); }
+    cluster.sync();
+    for (int r = 0; r < crank; ++r) {
+      const int* rc = cluster.map_shared_rank(s_counts, r);
+      less_before += rc[0];
+      eq_before += rc[1];
+    }
+  }
+  for (int i0 = 0; i0 < cs; i0 += nt) {
     const int i = i0 + tid;
-    const bool ok = i < s;
+    const bool ok = i < cs;
     const uint32_t k = ok ? keys[i] : 0xffffffffu;
     const int is_less = (ok && k < thr) ? 1 : 0;
     const int is_eq = (ok && k == thr) ? 1 : 0;
-    int packed = is_less | (is_eq << 16);
+    const int packed = is_less | (is_eq << 16);
     int incl = packed;
     for (int o = 1; o < 32; o <<= 1) {
       const int v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -191,7 +271,7 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
     if (lane == 31) s_warp[warp] = incl;
     __syncthreads();
     if (warp == 0) {
-      int w = (lane < (nt >> 5)) ? s_warp[lane] : 0;
+      const int w = (lane < (nt >> 5)) ? s_warp[lane] : 0;
       int wi = w;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, wi, o);
@@ -207,8 +287,8 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
     if (ok) {
       const bool down = is_less || (is_eq && eq_here < eq_left);
       const int down_before = less_here + min(eq_here, eq_left);
-      const int row = in_smem ? s_rows[i] : (pin ? pin[lo + i] : lo + i);
-      const int dst = down ? lo + down_before : lo + L + (i - down_before);
+      const int row = in_smem ? s_rows[i] : (pin ? pin[lo + c0 + i] : lo + c0 + i);
+      const int dst = down ? lo + down_before : lo + L + (c0 + i - down_before);
       pout[dst] = row;
     }
     const int total = s_scalar[3];
@@ -216,71 +296,312 @@ __global__ void __launch_bounds__(kMaxSplitThreads) split_level_kernel(const Spl
     eq_before += total >> 16;
     __syncthreads();
   }
+  if (csize > 1) cluster.sync();                     // keep shared memory alive for the peers' reads
+}
+
+// ---------------------------------------------------------------------------
+// Subtree of a set of at most kTailRowsMax rows, finished by one CTA.
+// ---------------------------------------------------------------------------
+struct TailSmem {
+  int32_t rows[2][kTailRowsMax];
+  uint32_t keys[kTailRowsMax];
+  uint32_t scan[kTailRowsMax];            // inclusive (less | equal << 16) counts over positions
+  int hist[kTailSegs][256];
+  int seg_lo[2][2 * kTailSegs + 2];       // start of each subset (relative), +1 sentinel
+  int seg_coord[kTailSegs], seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
+  uint32_t seg_prefix[kTailSegs];
+  double best[kTailSegs][4];
+  int arg[kTailSegs][4];
+  int warp_tot[32];
+  int nseg[2];
+  int more;
+};
+
+__global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitParams prm) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  TailSmem& sm = *reinterpret_cast<TailSmem*>(smem_raw);
+  const int which = blockIdx.y / prm.problems;
+  const int p = blockIdx.y % prm.problems;
+  const SplitSide sd = prm.side[which];
+  const int level = sd.tail_level;
+  if ((int)blockIdx.x >= (1 << level)) return;
+  const SegmentRef root = locate_segment(sd.n, sd.c, level, blockIdx.x);
+  if (!root.active) return;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  constexpr int nt = kSplitThreads;
+  const int D = prm.D, c = sd.c;
+  const float* Y = sd.Y + (size_t)p * sd.n * D;
+  const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
+  int32_t* pout = sd.perm_out + (size_t)p * sd.n;
+  const int lo = root.lo, s0 = root.size;
+
+  for (int i = tid; i < s0; i += nt) sm.rows[0][i] = pin ? pin[lo + i] : lo + i;
+  if (tid == 0) { sm.seg_lo[0][0] = 0; sm.seg_lo[0][1] = s0; sm.nseg[0] = 1; sm.more = s0 > c; }
+  __syncthreads();
+
+  int cur = 0;
+  const int wps = D / 32;                            // warps per (subset, all coordinates)
+  while (sm.more) {
+    const int nseg = sm.nseg[cur];
+    const int* slo = sm.seg_lo[cur];
+    const int32_t* rows = sm.rows[cur];
+    int32_t* rows_next = sm.rows[cur ^ 1];
+
+    // ---- 1. coordinate of largest subsample variance for every subset that still splits
+    for (int task = tid; task < nseg * D; task += nt) {
+      const int g = task / D, t = task % D;
+      const int a = slo[g], sz = slo[g + 1] - a;
+      double v = -1.0;
+      if (sz > c) v = subsample_variance(Y, D, t, rows + a, false, 0, sz, min(D, sz));
+      // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
+      int at = t;
+      for (int o = 16; o > 0; o >>= 1) {
+        const double ov = __shfl_xor_sync(0xffffffffu, v, o);
+        const int oa = __shfl_xor_sync(0xffffffffu, at, o);
+        if (ov > v || (ov == v && oa < at)) { v = ov; at = oa; }
+      }
+      if (lane == 0) { sm.best[g][(t / 32)] = v; sm.arg[g][(t / 32)] = at; }
+    }
+    __syncthreads();
+    if (tid < nseg) {
+      const int a = slo[tid], sz = slo[tid + 1] - a;
+      double v = sm.best[tid][0]; int at = sm.arg[tid][0];
+      for (int w = 1; w < wps; ++w)
+        if (sm.best[tid][w] > v) { v = sm.best[tid][w]; at = sm.arg[tid][w]; }   // later warps hold higher coordinates
+      sm.seg_coord[tid] = at;
+      sm.seg_L[tid] = sz > c ? c * ((sz + c) / (2 * c)) : 0;
+      sm.seg_prefix[tid] = 0u;
+      sm.seg_rem[tid] = sm.seg_L[tid];
+    }
+    __syncthreads();
+
+    // ---- 2. keys; each position finds its subset by bisection of the start offsets
+    int my_seg[kTailRowsMax / kSplitThreads];
+#pragma unroll
+    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
+      const int i = tid + u * nt;
+      int g = 0;
+      if (i < s0) {
+        int hi = nseg;                                // slo[g] <= i < slo[g+1]
+        while (hi - g > 1) { const int mid = (g + hi) >> 1; if (slo[mid] <= i) g = mid; else hi = mid; }
+        const bool splits = slo[g + 1] - slo[g] > c;
+        if (splits) sm.keys[i] = order_key(__ldg(Y + (size_t)rows[i] * D + sm.seg_coord[g]));
+        else g = -1 - g;                              // final subset: carried over unchanged
+      } else {
+        g = INT_MIN;
+      }
+      my_seg[u] = g;
+    }
+    __syncthreads();
+
+    // ---- radix selection, all subsets side by side
+    uint32_t mask = 0;
+    for (int shift = 24; shift >= 0; shift -= 8) {
+      for (int e = tid; e < nseg * 256; e += nt) (&sm.hist[0][0])[e] = 0;
+      __syncthreads();
+#pragma unroll
+      for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
+        const int g = my_seg[u];
+        const bool live = g >= 0;
+        const uint32_t k = live ? sm.keys[tid + u * nt] : 0u;
+        const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
+        const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&(&sm.hist[0][0])[bin], __popc(peers));
+      }
+      __syncthreads();
+      for (int g = warp; g < nseg; g += nt / 32) {
+        const int remaining = sm.seg_rem[g];
+        if (sm.seg_L[g] == 0) continue;               // warp-uniform
+        int local[8]; int sum = 0;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) { local[j] = sm.hist[g][lane * 8 + j]; sum += local[j]; }
+        int incl = sum;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int v = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += v;
+        }
+        int before = incl - sum;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (before < remaining && remaining <= before + local[j]) {
+            sm.seg_digit[g] = lane * 8 + j;
+            sm.seg_rem[g] = remaining - before;
+          }
+          before += local[j];
+        }
+        __syncwarp();
+        if (lane == 0) sm.seg_prefix[g] |= (uint32_t)sm.seg_digit[g] << shift;
+      }
+      mask |= 255u << shift;
+      __syncthreads();
+    }
+
+    // ---- 3. stable partition of every subset: one scan over all positions
+    int carry = 0;
+#pragma unroll
+    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
+      const int i = tid + u * nt;
+      const int g = my_seg[u];
+      int packed = 0;
+      if (g >= 0) {
+        const uint32_t k = sm.keys[i], thr = sm.seg_prefix[g];
+        packed = (k < thr ? 1 : 0) | (k == thr ? 1 << 16 : 0);
+      }
+      int incl = packed;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      if (lane == 31) sm.warp_tot[warp] = incl;
+      __syncthreads();
+      int wbase = 0, total = 0;
+      for (int w = 0; w < nt / 32; ++w) {              // 32 broadcast reads
+        const int v = sm.warp_tot[w];
+        if (w < warp) wbase += v;
+        total += v;
+      }
+      if (i < kTailRowsMax) sm.scan[i] = (uint32_t)(carry + wbase + incl);
+      carry += total;
+      __syncthreads();
+    }
+#pragma unroll
+    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
+      const int i = tid + u * nt;
+      const int g = my_seg[u];
+      if (g == INT_MIN) continue;
+      if (g < 0) { rows_next[i] = rows[i]; continue; }
+      const int a = slo[g];
+      const uint32_t base = a > 0 ? sm.scan[a - 1] : 0u;
+      const uint32_t k = sm.keys[i], thr = sm.seg_prefix[g];
+      const int is_less = k < thr, is_eq = k == thr;
+      const uint32_t excl = sm.scan[i] - base - (uint32_t)(is_less | (is_eq << 16));
+      const int less_here = (int)(excl & 0xffffu), eq_here = (int)(excl >> 16);
+      const int eq_left = sm.seg_rem[g], L = sm.seg_L[g];
+      const bool down = is_less || (is_eq && eq_here < eq_left);
+      const int down_before = less_here + min(eq_here, eq_left);
+      const int dst = down ? a + down_before : a + L + (i - a - down_before);
+      rows_next[dst] = rows[i];
+    }
+    // ---- next level's subsets
+    if (tid == 0) {
+      int* nlo = sm.seg_lo[cur ^ 1];
+      int n2 = 0, more = 0;
+      for (int g = 0; g < nseg; ++g) {
+        const int a = slo[g], sz = slo[g + 1] - a;
+        nlo[n2++] = a;
+        if (sz > c) {
+          const int L = sm.seg_L[g];
+          nlo[n2++] = a + L;
+          more |= (L > c) | (sz - L > c);
+        }
+      }
+      nlo[n2] = s0;
+      sm.nseg[cur ^ 1] = n2;
+      sm.more = more;
+    }
+    __syncthreads();
+    cur ^= 1;
+  }
+  for (int i = tid; i < s0; i += nt) pout[lo + i] = sm.rows[cur][i];
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+static int next_size(int big, int c) {
+  const int L = c * ((big + c) / (2 * c));
+  return (L > big - L) ? L : big - L;
 }
 
 int split_levels_for(int n, int c) {
   int levels = 0;
-  // the largest set of each level follows the larger child
-  int big = n;
-  while (big > c) {
-    const int L = c * ((big + c) / (2 * c));
-    big = (L > big - L) ? L : big - L;
-    ++levels;
-  }
+  for (int big = n; big > c; big = next_size(big, c)) ++levels;   // the largest set follows the larger child
   return levels;
 }
 
 static int max_segment_at_level(int n, int c, int level) {
   int big = n;
-  for (int l = 0; l < level && big > c; ++l) {
-    const int L = c * ((big + c) / (2 * c));
-    big = (L > big - L) ? L : big - L;
-  }
+  for (int l = 0; l < level && big > c; ++l) big = next_size(big, c);
   return big;
 }
 
-// Runs all levels for both sides.  perm_a / perm_b are ping-pong buffers per
-// side; the final permutation lands in perm_final (which must be one of them,
-// chosen by the caller through split_final_buffer).
+static int tail_rows_for(int c) {
+  const int r = kTailSegs * c;
+  return r < kTailRowsMax ? r : kTailRowsMax;
+}
+
+// Levels [0, tail_level) run as per-level launches; the tail kernel finishes the rest.
+static int tail_level_for(int n, int c) {
+  int level = 0;
+  for (int big = n; big > tail_rows_for(c); big = next_size(big, c)) ++level;
+  return level;
+}
+
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
                  int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st) {
-  const int lev_q = split_levels_for(n_q, c_q), lev_k = split_levels_for(n_k, c_k);
-  const int levels = lev_q > lev_k ? lev_q : lev_k;
-  constexpr int kSmemRowsMax = 24576;                 // 192 KB of keys + rows
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(split_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kSmemRowsMax * 8));
-  // with no split to do (n <= c) one level still runs: it writes the identity
-  const int run_levels = levels > 0 ? levels : 1;
-  for (int level = 0; level < run_levels; ++level) {
-    SplitParams prm;
-    prm.D = D; prm.level = level; prm.problems = problems;
-    int max_seg = 1;
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(split_tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)sizeof(TailSmem)));
+  const int tail_q = tail_level_for(n_q, c_q), tail_k = tail_level_for(n_k, c_k);
+  const int top_levels = tail_q > tail_k ? tail_q : tail_k;
+  SplitParams prm;
+  prm.D = D; prm.problems = problems;
+  // per-level launches write alternately to tmp/out so that the tail kernel, which runs last,
+  // reads the buffer that is not the output
+  auto fill = [&](int level) {
     for (int w = 0; w < 2; ++w) {
       SplitSide& sd = prm.side[w];
-      const int n = w == 0 ? n_q : n_k, c = w == 0 ? c_q : c_k;
-      const int lev = w == 0 ? lev_q : lev_k;
       int32_t* out = w == 0 ? perm_q_out : perm_k_out;
       int32_t* tmp = w == 0 ? perm_q_tmp : perm_k_tmp;
-      const int side_levels = lev > 0 ? lev : 1;
-      // the last level of this side writes `out`; earlier levels alternate
-      const bool to_out = ((side_levels - 1 - level) % 2) == 0;
+      const int tail = w == 0 ? tail_q : tail_k;
       sd.Y = w == 0 ? Yq : Yk;
-      sd.perm_out = to_out ? out : tmp;
-      sd.perm_in = level == 0 ? nullptr : (to_out ? tmp : out);
       sd.keybuf = w == 0 ? keybuf_q : keybuf_k;
-      sd.n = n; sd.c = c; sd.levels = side_levels;
-      if (level < side_levels) {
-        const int ms = max_segment_at_level(n, c, level);
-        if (ms > max_seg) max_seg = ms;
+      sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
+      sd.levels = split_levels_for(sd.n, sd.c);
+      sd.tail_level = tail;
+      // level l of this side (l < tail) writes tmp if (tail - 1 - l) is even, else out;
+      // the tail kernel (level == tail) reads what level tail-1 wrote and writes out
+      const bool to_tmp = ((tail - 1 - level) % 2) == 0;
+      if (level < tail) {
+        sd.perm_out = to_tmp ? tmp : out;
+        sd.perm_in = level == 0 ? nullptr : (to_tmp ? out : tmp);
+      } else {
+        sd.perm_out = out;
+        sd.perm_in = tail == 0 ? nullptr : tmp;
       }
     }
-    prm.smem_rows = max_seg < kSmemRowsMax ? max_seg : kSmemRowsMax;
-    const int threads = max_seg >= 8192 ? 1024 : (max_seg >= 2048 ? 512 : 256);
-    dim3 grid(1u << level, 2 * problems);
-    split_level_kernel<<<grid, threads, (size_t)prm.smem_rows * 8, st>>>(prm);
+  };
+  for (int level = 0; level < top_levels; ++level) {
+    fill(level);
+    prm.level = level;
+    int max_seg = 1;
+    if (level < tail_q) max_seg = max_segment_at_level(n_q, c_q, level);
+    if (level < tail_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
+    int csize = 1;
+    while (csize < kMaxCluster && max_seg > csize * 8192) csize *= 2;
+    const int per_cta = (max_seg + csize - 1) / csize;
+    prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((1u << level) * csize, 2 * problems);
+    cfg.blockDim = dim3(kSplitThreads);
+    cfg.dynamicSmemBytes = (size_t)prm.smem_rows * 8;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, split_level_kernel, prm));
     CA_LAUNCH_CHECK();
   }
+  fill(top_levels);       // any level >= both tails selects the tail buffers
+  prm.level = top_levels;
+  prm.smem_rows = 0;
+  const int slots = 1 << (tail_q > tail_k ? tail_q : tail_k);
+  split_tail_kernel<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(TailSmem), st>>>(prm);
+  CA_LAUNCH_CHECK();
   return CA_OK;
 }
 

@@ -54,6 +54,9 @@ SPLIT_CASES = [
     (2, 3000, 4099, 128, 128, 128, "bf16", True),     # many exact ties
     (1, 2048, 40000, 64, 128, 128, "bf16", False),    # sets larger than the shared-memory window
     (1, 640, 704, 128, 256, 16, "bf16", False),       # extreme cluster sizes
+    (1, 16384, 131072, 64, 128, 128, "bf16", False),  # one head of the tabular shape: 8-CTA clusters at the top
+    (1, 5000, 200000, 64, 64, 128, "bf16", True),     # slices beyond the shared-memory window, with ties
+    (2, 32760, 32760, 128, 128, 128, "bf16", False),  # the video shape: odd cluster counts, short last cluster
 ]
 
 
