@@ -44,6 +44,20 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
     A[i * LDA + j] = 0.5 * (Ain[i * D + j] + Ain[j * D + i]);
     Vt[i * LDA + j] = (i == j) ? (VT)1 : (VT)0;
   }
+  // scale so that the largest diagonal entry is 1 (eigenvectors unchanged, eigenvalues scaled back)
+  __syncthreads();
+  if (tid == 0) {
+    double mx = 0.0;
+    for (int i = 0; i < D; ++i) mx = fmax(mx, fabs(A[i * LDA + i]));
+    red[0] = mx > 0.0 ? mx : 1.0;
+  }
+  __syncthreads();
+  const double a_scale = red[0];
+  {
+    const double inv = 1.0 / a_scale;
+    for (int e = tid; e < D * D; e += NT) A[(e / D) * LDA + (e % D)] *= inv;
+  }
+  __syncthreads();
   for (int e = tid; e < H * H; e += NT) {
     int k1 = e / H, k2 = e % H;
     if (k1 <= k2) {
@@ -82,12 +96,19 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
         if (tid == 0) { p = D - 1; q = round; }
         else { p = (round + tid) % (D - 1); q = (round - tid + (D - 1)) % (D - 1); }
         if (p > q) { int t = p; p = q; q = t; }
-        double apq = A[p * LDA + q], app = A[p * LDA + p], aqq = A[q * LDA + q];
+        const double apq = A[p * LDA + q], app = A[p * LDA + p], aqq = A[q * LDA + q];
+        // tan of the rotation angle: t = sgn / (|tau| + sqrt(1 + tau^2)), tau = (aqq - app) / (2 apq),
+        // rewritten as sgn |apq| / (|alpha| + hypot(alpha, apq)), alpha = (aqq - app) / 2.  t only needs
+        // single precision (an inexact angle leaves a residual of 1e-7 |apq|, removed by the next
+        // sweep); c = 1/sqrt(1 + t^2) and s = t c are formed in double so that the rotation is
+        // orthogonal to double precision.
         double c = 1.0, s = 0.0;
-        if (fabs(apq) > 1e-300) {
-          double tau = (aqq - app) / (2.0 * apq);
-          double t = (tau >= 0.0 ? 1.0 : -1.0) / (fabs(tau) + sqrt(1.0 + tau * tau));
-          c = 1.0 / sqrt(1.0 + t * t);
+        const double alpha = 0.5 * (aqq - app);
+        const float fa = (float)fabs(alpha), fb = (float)fabs(apq);   // entries are scaled to at most 1
+        if (fb > 0.f) {
+          const float tf = fb / (fa + sqrtf(fmaf(fa, fa, fb * fb)));
+          const double t = ((alpha >= 0.0) == (apq >= 0.0)) ? (double)tf : -(double)tf;
+          c = rsqrt(fma(t, t, 1.0));
           s = t * c;
         }
         pp[tid] = (short)p; qq[tid] = (short)q; rc[tid] = c; rs[tid] = s;
@@ -106,7 +127,6 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
         // rows: J1^T * B
         double n_pp = c1 * b_pp - s1 * b_qp, n_pq = c1 * b_pq - s1 * b_qq;
         double n_qp = s1 * b_pp + c1 * b_qp, n_qq = s1 * b_pq + c1 * b_qq;
-        if (k1 == k2) { n_pq = 0.0; n_qp = 0.0; }       // the annihilated pair
         A[p1 * LDA + p2] = n_pp; A[p1 * LDA + q2] = n_pq;
         A[q1 * LDA + p2] = n_qp; A[q1 * LDA + q2] = n_qq;
         if (k1 != k2) {
@@ -129,7 +149,7 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
 
   // eigenvalues on the diagonal
   double* lam = rc;          // reuse: [D] fits in rc+rs (H+H)
-  if (tid < D) lam[tid] = A[tid * LDA + tid];
+  if (tid < D) lam[tid] = A[tid * LDA + tid] * a_scale;
   __syncthreads();
   double* o64 = out64 + (size_t)blockIdx.x * D * D;
   float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;

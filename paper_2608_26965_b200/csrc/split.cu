@@ -58,22 +58,15 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// variance of coordinate t over the subsample of a set (fixed operation order)
-__device__ __forceinline__ double subsample_variance(const float* __restrict__ Y, int D, int t,
-                                                     const int32_t* rows, bool identity, int lo, int s,
-                                                     int m) {
+// Variance of coordinate t over a subsample staged in shared memory as tile[j*D + t], j < m.
+// The additions run in a fixed order (row after row) in double.
+__device__ __forceinline__ double staged_variance(const float* tile, int D, int t, int m) {
   double sum = 0.0;
-  for (int j = 0; j < m; ++j) {
-    const int pos = (int)(((long long)j * s) / m);
-    const int row = identity ? lo + pos : rows[pos];
-    sum = __dadd_rn(sum, (double)__ldg(Y + (size_t)row * D + t));
-  }
+  for (int j = 0; j < m; ++j) sum = __dadd_rn(sum, (double)tile[j * D + t]);
   const double mean = sum / (double)m;
   double acc = 0.0;
   for (int j = 0; j < m; ++j) {
-    const int pos = (int)(((long long)j * s) / m);
-    const int row = identity ? lo + pos : rows[pos];
-    const double dev = __dsub_rn((double)__ldg(Y + (size_t)row * D + t), mean);
+    const double dev = __dsub_rn((double)tile[j * D + t], mean);
     acc = __dadd_rn(acc, __dmul_rn(dev, dev));
   }
   return acc / (double)m;
@@ -136,17 +129,15 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
     s_sub[tid] = pin ? pin[pos] : pos;
   }
   __syncthreads();
-  if (tid < D) {
-    double sum = 0.0;
-    for (int j = 0; j < m; ++j) sum = __dadd_rn(sum, (double)__ldg(Y + (size_t)s_sub[j] * D + tid));
-    const double mean = sum / (double)m;
-    double acc = 0.0;
-    for (int j = 0; j < m; ++j) {
-      const double dev = __dsub_rn((double)__ldg(Y + (size_t)s_sub[j] * D + tid), mean);
-      acc = __dadd_rn(acc, __dmul_rn(dev, dev));
-    }
-    s_var[tid] = acc / (double)m;
+  {
+    // the subsample rows are staged by all threads (16-byte loads in flight together)
+    float4* stage4 = reinterpret_cast<float4*>(smem_raw);
+    const int q = D / 4;
+    for (int e = tid; e < m * q; e += nt)
+      stage4[e] = __ldg(reinterpret_cast<const float4*>(Y + (size_t)s_sub[e / q] * D) + (e % q));
   }
+  __syncthreads();
+  if (tid < D) s_var[tid] = staged_variance(reinterpret_cast<const float*>(smem_raw), D, tid, m);
   __syncthreads();
   if (warp == 0) {
     double best = -1.0; int arg = 0;
@@ -347,22 +338,42 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
     const int32_t* rows = sm.rows[cur];
     int32_t* rows_next = sm.rows[cur ^ 1];
 
-    // ---- 1. coordinate of largest subsample variance for every subset that still splits
-    for (int task = tid; task < nseg * D; task += nt) {
-      const int g = task / D, t = task % D;
-      const int a = slo[g], sz = slo[g + 1] - a;
-      double v = -1.0;
-      if (sz > c) v = subsample_variance(Y, D, t, rows + a, false, 0, sz, min(D, sz));
-      // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
-      int at = t;
-      for (int o = 16; o > 0; o >>= 1) {
-        const double ov = __shfl_xor_sync(0xffffffffu, v, o);
-        const int oa = __shfl_xor_sync(0xffffffffu, at, o);
-        if (ov > v || (ov == v && oa < at)) { v = ov; at = oa; }
+    // ---- 1. coordinate of largest subsample variance for every subset that still splits.
+    // The subsamples are staged, a few subsets at a time, in the 64 KB that keys/scan/hist
+    // occupy later in the level.
+    {
+      float* stage = reinterpret_cast<float*>(sm.keys);
+      const int per_group = (16384 / (D * D)) > 0 ? 16384 / (D * D) : 1;     // 4 (d=64) or 1 (d=128)
+      const int q = D / 4;
+      for (int g0 = 0; g0 < nseg; g0 += per_group) {
+        const int ng = min(per_group, nseg - g0);
+        for (int e = tid; e < ng * D * q; e += nt) {
+          const int gi = e / (D * q), j = (e / q) % D, c4 = e % q;
+          const int a = slo[g0 + gi], sz = slo[g0 + gi + 1] - a;
+          const int m = min(D, sz);
+          if (sz > c && j < m) {
+            const int row = rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)];
+            reinterpret_cast<float4*>(stage)[e] = __ldg(reinterpret_cast<const float4*>(Y + (size_t)row * D) + c4);
+          }
+        }
+        __syncthreads();
+        for (int task = tid; task < ng * D; task += nt) {
+          const int gi = task / D, t = task % D, g = g0 + gi;
+          const int sz = slo[g + 1] - slo[g];
+          double v = -1.0;
+          if (sz > c) v = staged_variance(stage + gi * D * D, D, t, min(D, sz));
+          // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
+          int at = t;
+          for (int o = 16; o > 0; o >>= 1) {
+            const double ov = __shfl_xor_sync(0xffffffffu, v, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, at, o);
+            if (ov > v || (ov == v && oa < at)) { v = ov; at = oa; }
+          }
+          if (lane == 0) { sm.best[g][(t / 32)] = v; sm.arg[g][(t / 32)] = at; }
+        }
+        __syncthreads();
       }
-      if (lane == 0) { sm.best[g][(t / 32)] = v; sm.arg[g][(t / 32)] = at; }
     }
-    __syncthreads();
     if (tid < nseg) {
       const int a = slo[tid], sz = slo[tid + 1] - a;
       double v = sm.best[tid][0]; int at = sm.arg[tid][0];
@@ -587,7 +598,8 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((1u << level) * csize, 2 * problems);
     cfg.blockDim = dim3(kSplitThreads);
-    cfg.dynamicSmemBytes = (size_t)prm.smem_rows * 8;
+    // keys + rows of the slice; the same space first stages the d x d subsample tile
+    cfg.dynamicSmemBytes = (size_t)prm.smem_rows * 8 > (size_t)D * D * 4 ? (size_t)prm.smem_rows * 8 : (size_t)D * D * 4;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
