@@ -145,7 +145,7 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
     // global principal components of both transformed sets (Section 3.2.1)
-    CA_TRY(launch_eigh(w.cov, 2 * P, D, 1, w.basis, w.basis32, nullptr, st));
+    CA_TRY(launch_eigh(w.cov, 2 * P, D, w.basis, w.basis32, nullptr, st));
     double* EK = w.basis;
     double* EQ = w.basis + (size_t)P * DD;
     const float* EQ32 = w.basis32 + (size_t)P * DD;

@@ -1,78 +1,120 @@
 // Batched symmetric eigendecomposition of d x d matrices (d = 64, 128) by
-// parallel cyclic Jacobi, one CTA per matrix, and the d x d algebra around it:
-// roots of the metric matrices (Section 3.2.2, negative eigenvalues clamped to
-// zero) and principal-component bases (Section 3.2.1).
+// parallel cyclic Jacobi, one CTA per matrix (principal-component bases,
+// Section 3.2.1), Cholesky factors of the metric matrices (Section 3.2.2), and
+// the d x d algebra around them.
 #include "kernels.h"
 
 namespace ca {
 
 constexpr int kMaxSweeps = 16;
+constexpr int kEighThreads = 1024;
 
 template <int D>
 struct EighCfg {
-  static constexpr int H = D / 2;                       // rotations per step
-  static constexpr int NBLK = H * (H + 1) / 2;          // 2x2 blocks with k1 <= k2
-  static constexpr int THREADS = (D == 128) ? 1024 : 512;
-  static constexpr int LDA = D + 1;
+  static constexpr int H = D / 2;                                   // rotations per step
+  static constexpr int NB = (H * H) / kEighThreads > 0 ? (H * H) / kEighThreads : 1;   // 2x2 blocks per thread
+  static constexpr int NV = (H * D / 4) / kEighThreads > 0 ? (H * D / 4) / kEighThreads : 1;
+  static constexpr int LDA = D + 4;                                 // 16-byte aligned rows, staggered banks
 };
 
-// mode 0: out = E sqrt(max(lambda,0)) E^T      (symmetric root)
-// mode 1: out = eigenvectors as columns, descending eigenvalue, each column's
-//         entry of largest magnitude (lowest row on ties) made positive
-template <int D, typename VT>
-__global__ void __launch_bounds__(EighCfg<D>::THREADS)
-eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out64,
-            float* __restrict__ out32, double* __restrict__ evals_out) {
+// Position permutation applied after every step (round-robin tournament): the
+// rows/columns sitting at positions (2k, 2k+1) are the pair rotated next.
+template <int D>
+__device__ __forceinline__ int next_position(int i) {
+  if (i == 0) return 0;
+  if (i & 1) return i == 1 ? 2 : i - 2;
+  return i == D - 2 ? D - 1 : i + 2;
+}
+
+template <typename T> struct Vec2;
+template <> struct Vec2<float> { using type = float2; };
+template <> struct Vec2<double> { using type = double2; };
+template <typename T> struct __align__(16) Vec4 { T x, y, z, w; };
+
+// Eigenvectors of symmetric d x d matrices by parallel cyclic Jacobi, one CTA per
+// matrix.  The matrix lives in shared memory in "position space": each step
+// rotates the d/2 adjacent pairs (2k, 2k+1) at once -- every thread transforms
+// 2x2 blocks J1^T B J2 read with vector loads from one copy of the matrix --
+// and stores the result into a second copy at the positions of the next
+// pairing, so pairs are always adjacent and a step needs two barriers.  The
+// rows of V^T follow the same permutation (their stores are deferred past the
+// barrier instead of being double-buffered).  AT is the working precision of
+// the matrix and of V (float for d = 128, where two double copies would not fit
+// in shared memory; the split coordinates are fp32 anyway).  Output:
+// eigenvectors as columns, descending eigenvalue, each column's entry of largest
+// magnitude (lowest row on ties) made positive.
+template <int D, typename AT>
+__global__ void __launch_bounds__(kEighThreads)
+eigh_kernel(const double* __restrict__ A_in, double* __restrict__ out64, float* __restrict__ out32,
+            double* __restrict__ evals_out) {
   using C = EighCfg<D>;
-  constexpr int H = C::H, LDA = C::LDA, NT = C::THREADS;
+  using V2 = typename Vec2<AT>::type;
+  constexpr int H = C::H, LDA = C::LDA, NT = kEighThreads;
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* A = reinterpret_cast<double*>(smem_raw);                 // [D][LDA]
-  VT* Vt = reinterpret_cast<VT*>(A + D * LDA);                     // [D][LDA]  (rows = eigenvectors)
-  double* rc = reinterpret_cast<double*>(Vt + D * LDA);            // [H]
-  double* rs = rc + H;                                             // [H]
-  double* red = rs + H;                                            // [64]
-  short* pp = reinterpret_cast<short*>(red + 64);                  // [H]
-  short* qq = pp + H;                                              // [H]
-  unsigned short* blk = reinterpret_cast<unsigned short*>(qq + H); // [NBLK] packed (k1<<8|k2)
-  int* flag = reinterpret_cast<int*>(blk + C::NBLK + (C::NBLK & 1));
+  AT* Abuf0 = reinterpret_cast<AT*>(smem_raw);                     // [D][LDA]
+  AT* Abuf1 = Abuf0 + D * LDA;                                     // [D][LDA]
+  AT* Vt = Abuf1 + D * LDA;                                        // [D][D]  (rows = eigenvectors)
+  AT* rc = Vt + D * D;                                             // [H]
+  AT* rs = rc + H;                                                 // [H]
+  double* red = reinterpret_cast<double*>(rs + H);                 // [64 + D]
+  int* flag = reinterpret_cast<int*>(red + 64 + D);
 
   const int tid = threadIdx.x;
   const double* Ain = A_in + (size_t)blockIdx.x * D * D;
-  for (int e = tid; e < D * D; e += NT) {
-    int i = e / D, j = e % D;
-    // symmetrise on load
-    A[i * LDA + j] = 0.5 * (Ain[i * D + j] + Ain[j * D + i]);
-    Vt[i * LDA + j] = (i == j) ? (VT)1 : (VT)0;
-  }
   // scale so that the largest diagonal entry is 1 (eigenvectors unchanged, eigenvalues scaled back)
-  __syncthreads();
-  if (tid == 0) {
+  if (tid < 32) {
     double mx = 0.0;
-    for (int i = 0; i < D; ++i) mx = fmax(mx, fabs(A[i * LDA + i]));
-    red[0] = mx > 0.0 ? mx : 1.0;
+    for (int i = tid; i < D; i += 32) mx = fmax(mx, fabs(Ain[i * D + i]));
+    for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (tid == 0) red[0] = mx > 0.0 ? mx : 1.0;
   }
   __syncthreads();
   const double a_scale = red[0];
   {
     const double inv = 1.0 / a_scale;
-    for (int e = tid; e < D * D; e += NT) A[(e / D) * LDA + (e % D)] *= inv;
-  }
-  __syncthreads();
-  for (int e = tid; e < H * H; e += NT) {
-    int k1 = e / H, k2 = e % H;
-    if (k1 <= k2) {
-      int idx = k1 * H - (k1 * (k1 - 1)) / 2 + (k2 - k1);
-      blk[idx] = (unsigned short)((k1 << 8) | k2);
+    for (int e = tid; e < D * D; e += NT) {
+      const int i = e / D, j = e % D;
+      Abuf0[i * LDA + j] = (AT)(0.5 * (Ain[i * D + j] + Ain[j * D + i]) * inv);   // symmetrise on load
+      Vt[e] = (i == j) ? (AT)1 : (AT)0;
     }
   }
   __syncthreads();
 
+  // fixed work assignment in position space
+  int rd[C::NB], w00[C::NB], w01[C::NB], w10[C::NB], w11[C::NB], bk1[C::NB], bk2[C::NB];
+#pragma unroll
+  for (int u = 0; u < C::NB; ++u) {
+    const int b = tid + u * NT;
+    const int k1 = (b / H) % H, k2 = b % H;
+    bk1[u] = k1; bk2[u] = k2;
+    rd[u] = (2 * k1) * LDA + 2 * k2;
+    const int p1 = next_position<D>(2 * k1) * LDA, q1 = next_position<D>(2 * k1 + 1) * LDA;
+    const int p2 = next_position<D>(2 * k2), q2 = next_position<D>(2 * k2 + 1);
+    w00[u] = p1 + p2; w01[u] = p1 + q2; w10[u] = q1 + p2; w11[u] = q1 + q2;
+  }
+  int vk[C::NV], vrd[C::NV], vw0[C::NV], vw1[C::NV];
+#pragma unroll
+  for (int u = 0; u < C::NV; ++u) {
+    const int e = tid + u * NT;
+    const int k = (e / (D / 4)) % H, i4 = e % (D / 4);
+    vk[u] = k;
+    vrd[u] = (2 * k) * D + 4 * i4;
+    vw0[u] = next_position<D>(2 * k) * D + 4 * i4;
+    vw1[u] = next_position<D>(2 * k + 1) * D + 4 * i4;
+  }
+  const bool blk_live = tid < H * H, v_live = tid < H * D / 4;      // only d = 64 leaves threads idle
+
+  AT* Acur = Abuf0;
+  AT* Anext = Abuf1;
+  Vec4<AT> nv0[C::NV], nv1[C::NV];
+  bool v_pending = false;
+  const double tol = sizeof(AT) == 4 ? 1e-12 : 1e-24;     // squared relative off-diagonal norm
   for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
     // convergence: off-diagonal mass against the whole matrix
     double off = 0.0, tot = 0.0;
     for (int e = tid; e < D * D; e += NT) {
-      int i = e / D, j = e % D;
-      double v = A[i * LDA + j];
+      const int i = e / D, j = e % D;
+      const double v = (double)Acur[i * LDA + j];
       tot += v * v;
       if (i != j) off += v * v;
     }
@@ -85,141 +127,134 @@ eigh_kernel(const double* __restrict__ A_in, int mode, double* __restrict__ out6
     if (tid == 0) {
       double o = 0.0, t = 0.0;
       for (int w = 0; w < NT / 32; ++w) { o += red[w]; t += red[32 + w]; }
-      *flag = (o <= 1e-24 * t) ? 1 : 0;       // off-diagonal norm below 1e-12 of the matrix norm
+      *flag = (o <= tol * t) ? 1 : 0;
     }
     __syncthreads();
     if (*flag) break;
 
-    for (int round = 0; round < D - 1; ++round) {
+    for (int step = 0; step < D - 1; ++step) {
+      // rotation of each adjacent pair; deferred stores of the previous step's V rows
       if (tid < H) {
-        int p, q;
-        if (tid == 0) { p = D - 1; q = round; }
-        else { p = (round + tid) % (D - 1); q = (round - tid + (D - 1)) % (D - 1); }
-        if (p > q) { int t = p; p = q; q = t; }
-        const double apq = A[p * LDA + q], app = A[p * LDA + p], aqq = A[q * LDA + q];
-        // tan of the rotation angle: t = sgn / (|tau| + sqrt(1 + tau^2)), tau = (aqq - app) / (2 apq),
-        // rewritten as sgn |apq| / (|alpha| + hypot(alpha, apq)), alpha = (aqq - app) / 2.  t only needs
-        // single precision (an inexact angle leaves a residual of 1e-7 |apq|, removed by the next
-        // sweep); c = 1/sqrt(1 + t^2) and s = t c are formed in double so that the rotation is
-        // orthogonal to double precision.
-        double c = 1.0, s = 0.0;
-        const double alpha = 0.5 * (aqq - app);
-        const float fa = (float)fabs(alpha), fb = (float)fabs(apq);   // entries are scaled to at most 1
+        const int p = 2 * tid, q = p + 1;
+        const float apq = (float)Acur[p * LDA + q];
+        const float alpha = 0.5f * ((float)Acur[q * LDA + q] - (float)Acur[p * LDA + p]);
+        // t = tan(angle) = sgn |apq| / (|alpha| + hypot(alpha, apq)); c = 1/sqrt(1 + t^2), s = t c.
+        // An inexact t only leaves a small residual in a_pq that the next sweep removes;
+        // c and s are formed in the working precision so that c^2 + s^2 = 1 to rounding.
+        AT c = (AT)1, s = (AT)0;
+        const float fa = fabsf(alpha), fb = fabsf(apq);
         if (fb > 0.f) {
           const float tf = fb / (fa + sqrtf(fmaf(fa, fa, fb * fb)));
-          const double t = ((alpha >= 0.0) == (apq >= 0.0)) ? (double)tf : -(double)tf;
-          c = rsqrt(fma(t, t, 1.0));
+          const AT t = ((alpha >= 0.f) == (apq >= 0.f)) ? (AT)tf : -(AT)tf;
+          if (sizeof(AT) == 4) c = (AT)rsqrtf((float)(t * t + (AT)1)); else c = (AT)rsqrt((double)(t * t + (AT)1));
           s = t * c;
         }
-        pp[tid] = (short)p; qq[tid] = (short)q; rc[tid] = c; rs[tid] = s;
+        rc[tid] = c; rs[tid] = s;
       }
-      __syncthreads();
-      // A <- J^T A J on 2x2 blocks (rows of pair k1, columns of pair k2), mirrored
-      for (int b = tid; b < C::NBLK; b += NT) {
-        const int k1 = blk[b] >> 8, k2 = blk[b] & 255;
-        const int p1 = pp[k1], q1 = qq[k1], p2 = pp[k2], q2 = qq[k2];
-        const double c1 = rc[k1], s1 = rs[k1], c2 = rc[k2], s2 = rs[k2];
-        double a_pp = A[p1 * LDA + p2], a_pq = A[p1 * LDA + q2];
-        double a_qp = A[q1 * LDA + p2], a_qq = A[q1 * LDA + q2];
-        // columns: B = blk * J2
-        double b_pp = c2 * a_pp - s2 * a_pq, b_pq = s2 * a_pp + c2 * a_pq;
-        double b_qp = c2 * a_qp - s2 * a_qq, b_qq = s2 * a_qp + c2 * a_qq;
-        // rows: J1^T * B
-        double n_pp = c1 * b_pp - s1 * b_qp, n_pq = c1 * b_pq - s1 * b_qq;
-        double n_qp = s1 * b_pp + c1 * b_qp, n_qq = s1 * b_pq + c1 * b_qq;
-        A[p1 * LDA + p2] = n_pp; A[p1 * LDA + q2] = n_pq;
-        A[q1 * LDA + p2] = n_qp; A[q1 * LDA + q2] = n_qq;
-        if (k1 != k2) {
-          A[p2 * LDA + p1] = n_pp; A[q2 * LDA + p1] = n_pq;
-          A[p2 * LDA + q1] = n_qp; A[q2 * LDA + q1] = n_qq;
+      if (v_pending && v_live) {
+#pragma unroll
+        for (int u = 0; u < C::NV; ++u) {
+          *reinterpret_cast<Vec4<AT>*>(&Vt[vw0[u]]) = nv0[u];
+          *reinterpret_cast<Vec4<AT>*>(&Vt[vw1[u]]) = nv1[u];
         }
       }
-      // V <- V J  (rows p, q of V^T)
-      for (int e = tid; e < H * D; e += NT) {
-        const int k = e / D, i = e % D;
-        const int p = pp[k], q = qq[k];
-        const VT c = (VT)rc[k], s = (VT)rs[k];
-        VT vp = Vt[p * LDA + i], vq = Vt[q * LDA + i];
-        Vt[p * LDA + i] = c * vp - s * vq;
-        Vt[q * LDA + i] = s * vp + c * vq;
-      }
       __syncthreads();
+      if (blk_live) {
+#pragma unroll
+        for (int u = 0; u < C::NB; ++u) {
+          const AT c1 = rc[bk1[u]], s1 = rs[bk1[u]], c2 = rc[bk2[u]], s2 = rs[bk2[u]];
+          const V2 r0 = *reinterpret_cast<const V2*>(&Acur[rd[u]]);
+          const V2 r1 = *reinterpret_cast<const V2*>(&Acur[rd[u] + LDA]);
+          // columns: B = blk * J2 ; rows: J1^T * B
+          const AT b_pp = c2 * r0.x - s2 * r0.y, b_pq = s2 * r0.x + c2 * r0.y;
+          const AT b_qp = c2 * r1.x - s2 * r1.y, b_qq = s2 * r1.x + c2 * r1.y;
+          Anext[w00[u]] = c1 * b_pp - s1 * b_qp; Anext[w01[u]] = c1 * b_pq - s1 * b_qq;
+          Anext[w10[u]] = s1 * b_pp + c1 * b_qp; Anext[w11[u]] = s1 * b_pq + c1 * b_qq;
+        }
+      }
+      if (v_live) {
+#pragma unroll
+        for (int u = 0; u < C::NV; ++u) {
+          const AT c = rc[vk[u]], s = rs[vk[u]];
+          const Vec4<AT> vp = *reinterpret_cast<const Vec4<AT>*>(&Vt[vrd[u]]);
+          const Vec4<AT> vq = *reinterpret_cast<const Vec4<AT>*>(&Vt[vrd[u] + D]);
+          nv0[u].x = c * vp.x - s * vq.x; nv0[u].y = c * vp.y - s * vq.y;
+          nv0[u].z = c * vp.z - s * vq.z; nv0[u].w = c * vp.w - s * vq.w;
+          nv1[u].x = s * vp.x + c * vq.x; nv1[u].y = s * vp.y + c * vq.y;
+          nv1[u].z = s * vp.z + c * vq.z; nv1[u].w = s * vp.w + c * vq.w;
+        }
+      }
+      v_pending = true;
+      __syncthreads();
+      AT* t = Acur; Acur = Anext; Anext = t;
     }
   }
+  if (v_pending && v_live) {
+#pragma unroll
+    for (int u = 0; u < C::NV; ++u) {
+      *reinterpret_cast<Vec4<AT>*>(&Vt[vw0[u]]) = nv0[u];
+      *reinterpret_cast<Vec4<AT>*>(&Vt[vw1[u]]) = nv1[u];
+    }
+  }
+  __syncthreads();
 
   // eigenvalues on the diagonal
-  double* lam = rc;          // reuse: [D] fits in rc+rs (H+H)
-  if (tid < D) lam[tid] = A[tid * LDA + tid] * a_scale;
+  double* lam = red + 64;
+  if (tid < D) lam[tid] = (double)Acur[tid * LDA + tid] * a_scale;
   __syncthreads();
   double* o64 = out64 + (size_t)blockIdx.x * D * D;
   float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
-  if (mode == 0) {
-    if (evals_out && tid < D) evals_out[(size_t)blockIdx.x * D + tid] = lam[tid];
-    __syncthreads();
-    if (tid < D) lam[tid] = sqrt(fmax(lam[tid], 0.0));
-    __syncthreads();
-    for (int e = tid; e < D * D; e += NT) {
-      const int i = e / D, j = e % D;
-      double s = 0.0;
-      for (int k = 0; k < D; ++k) s += (double)Vt[k * LDA + i] * lam[k] * (double)Vt[k * LDA + j];
-      o64[e] = s;
-      if (o32) o32[e] = (float)s;
+  // rank of each eigenvalue in descending order (ties: lower position first)
+  int* rank_of = reinterpret_cast<int*>(Anext);
+  float* sign_of = reinterpret_cast<float*>(rank_of + D);
+  if (tid < D) {
+    const double mine = lam[tid];
+    int rank = 0;
+    for (int k = 0; k < D; ++k) {
+      const double other = lam[k];
+      rank += (other > mine) || (other == mine && k < tid);
     }
-  } else {
-    // rank of each eigenvalue in descending order (ties: lower index first)
-    if (tid < D) {
-      const double mine = lam[tid];
-      int rank = 0;
-      for (int k = 0; k < D; ++k) {
-        const double other = lam[k];
-        rank += (other > mine) || (other == mine && k < tid);
-      }
-      // sign: entry of largest magnitude positive
-      double best = -1.0; double sgn = 1.0;
-      for (int i = 0; i < D; ++i) {
-        double v = (double)Vt[tid * LDA + i];
-        if (fabs(v) > best) { best = fabs(v); sgn = (v < 0.0) ? -1.0 : 1.0; }
-      }
-      // stash rank and sign: reuse A's first two rows
-      A[tid] = (double)rank;
-      A[LDA + tid] = sgn;
-      if (evals_out) evals_out[(size_t)blockIdx.x * D + rank] = mine;
+    // sign: entry of largest magnitude positive
+    double best = -1.0; float sgn = 1.f;
+    for (int i = 0; i < D; ++i) {
+      const double v = (double)Vt[tid * D + i];
+      if (fabs(v) > best) { best = fabs(v); sgn = (v < 0.0) ? -1.f : 1.f; }
     }
-    __syncthreads();
-    for (int e = tid; e < D * D; e += NT) {
-      const int k = e / D, i = e % D;           // eigenvector k, component i
-      const int col = (int)A[k];
-      const double v = A[LDA + k] * (double)Vt[k * LDA + i];
-      o64[i * D + col] = v;
-      if (o32) o32[i * D + col] = (float)v;
-    }
+    rank_of[tid] = rank;
+    sign_of[tid] = sgn;
+    if (evals_out) evals_out[(size_t)blockIdx.x * D + rank] = mine;
+  }
+  __syncthreads();
+  for (int e = tid; e < D * D; e += NT) {
+    const int k = e / D, i = e % D;           // eigenvector k, component i
+    const double v = (double)sign_of[k] * (double)Vt[k * D + i];
+    o64[i * D + rank_of[k]] = v;
+    if (o32) o32[i * D + rank_of[k]] = (float)v;
   }
 }
 
-template <int D, typename VT>
+template <int D, typename AT>
 static size_t eigh_smem() {
   using C = EighCfg<D>;
-  return sizeof(double) * D * C::LDA + sizeof(VT) * D * C::LDA + sizeof(double) * (2 * C::H + 64) +
-         sizeof(short) * 2 * C::H + sizeof(unsigned short) * (C::NBLK + 1) + 16;
+  return sizeof(AT) * (2 * D * C::LDA + D * D + 2 * C::H) + sizeof(double) * (64 + D) + 16;
 }
 
-int launch_eigh(const double* A, int count, int D, int mode, double* out64, float* out32,
-                double* evals, cudaStream_t st) {
+int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
+                cudaStream_t st) {
   if (D == 64) {
-    auto k = eigh_kernel<64, double>;
-    size_t smem = eigh_smem<64, double>();
+    auto k = eigh_kernel<64, float>;
+    size_t smem = eigh_smem<64, float>();
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, EighCfg<64>::THREADS, smem, st>>>(A, mode, out64, out32, evals);
+    k<<<count, kEighThreads, smem, st>>>(A, out64, out32, evals);
   } else {
     auto k = eigh_kernel<128, float>;
     size_t smem = eigh_smem<128, float>();
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, EighCfg<128>::THREADS, smem, st>>>(A, mode, out64, out32, evals);
+    k<<<count, kEighThreads, smem, st>>>(A, out64, out32, evals);
   }
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
-
 
 // ---------------------------------------------------------------------------
 // Factor of a positive semi-definite matrix: lower-triangular F with F F^T = A

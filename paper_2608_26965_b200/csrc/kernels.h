@@ -14,8 +14,8 @@ int launch_transform_rows(const void* X, int dtype, int problems, int n_rows, in
                           const float* bias, int normalize, float* out, cudaStream_t st);
 
 // eigh.cu
-int launch_eigh(const double* A, int count, int D, int mode, double* out64, float* out32,
-                double* evals, cudaStream_t st);
+int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
+                cudaStream_t st);
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
                   int n_k, double* M, double* CK, cudaStream_t st);
 int launch_covariance(const double* gram, const double* sum, int P, int D, int n, double* cov,
