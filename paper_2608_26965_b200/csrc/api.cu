@@ -36,6 +36,7 @@ struct ClusterWs {
   double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
   float *roots32, *basis32, *WK32, *biasK, *biasQ;
   float *Qprime, *Yq, *Yk;
+  __nv_bfloat16 *wt_hi, *wt_lo;
   int32_t *perm_q_tmp, *perm_k_tmp;
   uint32_t *keybuf_q, *keybuf_k;
   size_t bytes;
@@ -68,6 +69,8 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
     w.biasK = c.take<float>(P * D);
     w.biasQ = c.take<float>(P * D);
     w.Qprime = c.take<float>(P * (size_t)p->n_q * D);
+    w.wt_hi = c.take<__nv_bfloat16>(P * DD);
+    w.wt_lo = c.take<__nv_bfloat16>(P * DD);
     if (need_yq) w.Yq = c.take<float>(P * (size_t)p->n_q * D);
     if (need_yk) w.Yk = c.take<float>(P * (size_t)p->n_k * D);
   }
@@ -124,9 +127,18 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
   if (!y_in) {
     float* yq_out = Yq ? Yq : w.Yq;
     float* yk_out = Yk ? Yk : w.Yk;
+    // bf16 storage runs the O(n d^2) passes on the tensor cores; fp32 storage on the CUDA cores
+    const bool tc = p->dtype == CA_DTYPE_BF16;
+    __nv_bfloat16* qp_hi = reinterpret_cast<__nv_bfloat16*>(w.Qprime);          // r(q) as bf16 hi + lo parts
+    __nv_bfloat16* qp_lo = qp_hi + (size_t)P * p->n_q * D;
     // metric matrices (Section 3.2.2)
-    CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
-    CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial, w.gramK, w.sumK, st));
+    if (tc) {
+      CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
+      CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial, w.gramK, w.sumK, w.status, st));
+    } else {
+      CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
+      CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial, w.gramK, w.sumK, st));
+    }
     double* M = w.metric;
     double* CK = w.metric + (size_t)P * DD;
     CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, M, CK, st));
@@ -141,8 +153,14 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
     CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, 1.0 / (double)p->n_k, 0, covK, nullptr, st));
     // query representation r(q) = F_k^T q / |F_k^T q| and its covariance
-    CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, 1, w.Qprime, st));
-    CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
+    if (tc) {
+      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, 1, nullptr, qp_hi, qp_lo, w.wt_hi,
+                                 w.wt_lo, w.status, st));
+      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, w.status, st));
+    } else {
+      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, 1, w.Qprime, st));
+      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
+    }
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
     // global principal components of both transformed sets (Section 3.2.1)
     CA_TRY(launch_eigh(w.cov, 2 * P, D, w.basis, w.basis32, nullptr, st));
@@ -153,8 +171,15 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, 0, w.WK, w.WK32, st));
     CA_TRY(launch_bias(w.sumK, w.WK, P, D, p->n_k, w.biasK, st));
     CA_TRY(launch_bias(w.sumQp, EQ, P, D, p->n_q, w.biasQ, st));
-    CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
-    CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, st));
+    if (tc) {
+      CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr,
+                                 w.wt_hi, w.wt_lo, w.status, st));
+      CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr,
+                                 w.wt_hi, w.wt_lo, w.status, st));
+    } else {
+      CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
+      CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, st));
+    }
     yq = yq_out;
     yk = yk_out;
   }

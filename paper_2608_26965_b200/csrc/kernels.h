@@ -13,6 +13,16 @@ int launch_moments(const void* X, int dtype, int problems, int n_rows, int D, fl
 int launch_transform_rows(const void* X, int dtype, int problems, int n_rows, int D, const float* W,
                           const float* bias, int normalize, float* out, cudaStream_t st);
 
+int launch_gram_finalize(const float* partial, int problems, int n_chunks, int D, double* gram,
+                         double* colsum, cudaStream_t st);
+
+// tc_linear.cu (bf16 storage: tensor-core versions of the two kernels above)
+int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, float* partial,
+                   double* gram, double* colsum, int* status, cudaStream_t st);
+int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, const float* W,
+                        const float* bias, int normalize, float* out, void* out_hi, void* out_lo,
+                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st);
+
 // eigh.cu
 int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
                 cudaStream_t st);

@@ -84,6 +84,15 @@ int moments_chunking(int n_rows, int problems, int* chunk_rows, int* n_chunks) {
   return 0;
 }
 
+int launch_gram_finalize(const float* partial, int problems, int n_chunks, int D, double* gram,
+                         double* colsum, cudaStream_t st) {
+  const int elems = D * D + D;
+  gram_finalize_kernel<<<dim3(ceil_div(elems, 256), problems), 256, 0, st>>>(partial, n_chunks, elems, gram,
+                                                                              colsum, D * D);
+  CA_LAUNCH_CHECK();
+  return CA_OK;
+}
+
 template <typename T>
 static int launch_moments_t(const T* X, int problems, int n_rows, int D, float* partial,
                             double* gram, double* colsum, cudaStream_t st) {
@@ -93,11 +102,7 @@ static int launch_moments_t(const T* X, int problems, int n_rows, int D, float* 
   if (D == 64) gram_chunk_kernel<T, 64><<<grid, 256, 0, st>>>(X, n_rows, chunk_rows, n_chunks, partial);
   else gram_chunk_kernel<T, 128><<<grid, 256, 0, st>>>(X, n_rows, chunk_rows, n_chunks, partial);
   CA_LAUNCH_CHECK();
-  const int elems = D * D + D;
-  gram_finalize_kernel<<<dim3(ceil_div(elems, 256), problems), 256, 0, st>>>(partial, n_chunks, elems,
-                                                                              gram, colsum, D * D);
-  CA_LAUNCH_CHECK();
-  return CA_OK;
+  return launch_gram_finalize(partial, problems, n_chunks, D, gram, colsum, st);
 }
 
 int launch_moments(const void* X, int dtype, int problems, int n_rows, int D, float* partial,
