@@ -124,6 +124,37 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
                           const int32_t* perm_q, void* O, float* lse, void* ws,
                           size_t ws_bytes, void* stream);
 
+/*
+ * The attention stage without a caller-provided workspace.  (The paper has no
+ * counterpart for this entry point; it exists for deployment reasons only.)
+ *
+ * Meant for callers that cannot allocate device memory and therefore cannot
+ * supply a workspace: code inside a host framework's execute callback where
+ * allocation is not allowed, serving loops that must avoid the device-wide
+ * synchronisation an allocation implies, and processes whose device memory is
+ * already reserved by another pool.  Same computation, arguments and results
+ * as cluster_attention_fwd (inputs and outputs are still the caller's), but the
+ * scratch is a fixed array of ca_static_scratch_bytes() = 32 MiB that is part
+ * of the library image: every GPU that loads the library holds it until the
+ * process exits.  The call allocates and frees nothing.
+ *   - Limit: returns CA_ERR_WORKSPACE, enqueuing nothing, if the attention
+ *     workspace that ca_workspace_bytes reports for `p` exceeds the array.
+ *   - Set-up: the first call on each device looks up the array's device address
+ *     (with that device current).  Make that first call before any stream
+ *     capture is started.
+ *   - Sharing: every call on a device uses the same array, which keeps the
+ *     previous call's contents; the call itself clears the status word and
+ *     rewrites the centroid copies it needs.  Two calls whose kernels overlap on
+ *     the GPU (different streams) race on the array: serialise them.
+ * ca_static_last_status reads the array's status word (synchronises the device).
+ */
+size_t ca_static_scratch_bytes(void);
+int cluster_attention_fwd_static(const ca_problem_t* p, const void* Qp, const void* Kp,
+                                 const void* Vp, const float* ck, const float* cv,
+                                 const int32_t* count_k, const int32_t* block_idx,
+                                 const int32_t* perm_q, void* O, float* lse, void* stream);
+int ca_static_last_status(void);
+
 /* Reads the status word of a workspace (synchronises the device). */
 int ca_last_status(const void* ws);
 

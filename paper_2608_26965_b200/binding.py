@@ -25,7 +25,8 @@ CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
 CA_Y_IN, CA_ATTN_FP32 = 1, 2
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
-           "ca_last_status", "ca_version", "ca_kernel_launches")
+           "ca_last_status", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
+           "ca_static_scratch_bytes", "ca_static_last_status")
 
 
 class CaProblem(ctypes.Structure):
@@ -82,6 +83,12 @@ def load_library() -> ctypes.CDLL:
     lib.ca_version.restype = ctypes.c_char_p
     lib.ca_kernel_launches.argtypes = []
     lib.ca_kernel_launches.restype = ctypes.c_ulonglong
+    lib.cluster_attention_fwd_static.argtypes = [pp] + [vp] * 10 + [vp]
+    lib.cluster_attention_fwd_static.restype = ctypes.c_int
+    lib.ca_static_scratch_bytes.argtypes = []
+    lib.ca_static_scratch_bytes.restype = ctypes.c_size_t
+    lib.ca_static_last_status.argtypes = []
+    lib.ca_static_last_status.restype = ctypes.c_int
     _lib = lib
     return lib
 
@@ -252,6 +259,26 @@ def cluster_attention_fwd(problem: CaProblem, Qp, Kp, Vp, ck, cv, count_k, block
     if tuple(block_idx.shape[-2:]) != (problem.n_qc, problem.keep):
         raise ClusterAttnError("block_idx must be [B,H,n_qc,keep]")
     return plan.cluster_attention_fwd(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q)
+
+
+def cluster_attention_fwd_static(problem: CaProblem, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O,
+                                 lse=None, stream=None):
+    """The attention stage for callers that cannot allocate device memory (no
+    workspace argument: the library's fixed 32 MiB scratch array is used).  The
+    caller passes every input and the output tensors; nothing is allocated here
+    either.  Calls on one device share the scratch and must not overlap."""
+    lib = load_library()
+    args = [Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O]
+    for i, t in enumerate(args):
+        _require_cuda(t, f"arg{i}")
+    rc = lib.cluster_attention_fwd_static(ctypes.byref(problem), *[_ptr(t) for t in args], _ptr(lse),
+                                          _stream_ptr(stream))
+    _check(rc, "cluster_attention_fwd_static")
+    return O, lse
+
+
+def static_scratch_bytes() -> int:
+    return int(load_library().ca_static_scratch_bytes())
 
 
 def default_scale(problem: CaProblem) -> float:
