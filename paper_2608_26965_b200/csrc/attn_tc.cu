@@ -223,6 +223,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
+    long long T0 = 0, T1 = 0, T2 = 0, T3 = 0, tA, tB;
+    const bool dbg = (blockIdx.x == 5 && blockIdx.y == 0 && st == 0);
     for (int t = 0; t < total_tiles && ok; ++t) {
       // per-column additive term (log2 units): only tiles with masked or weighted columns need it.
       // `masked` depends on the tile only, so it is uniform over the 128 threads.
@@ -253,31 +255,49 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
 
+      tA = clock64();
       ok = __all_sync(0xffffffffu, mbar_wait(b_s_full, t & 1, abort_flag, prm.status));
       if (!ok) break;
       tc_fence_after();
-      uint32_t sr[4][32];
+      tB = clock64(); T0 += tB - tA;
+      // ---- pass 1: row maximum (TMEM chunks of 32 columns, the next load in flight while one is reduced)
+      uint32_t ra[32], rb[32];
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      auto reduce_max = [&](const uint32_t (&r)[32], int c4) {
+        if (masked) {
 #pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) tmem_ld32(tmem_s + lane_addr + c4 * 32, sr[c4]);
-      tmem_wait_ld();
-
-      float tmax = -INFINITY;
-      if (masked) {
-#pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const float x = fmaf(__uint_as_float(sr[c4][j]), prm.scale_log2, bz[c4 * 32 + j]);
-            sr[c4][j] = __float_as_uint(x);
-            tmax = fmaxf(tmax, x);
+          for (int j = 0; j < 32; j += 4) {
+            mx0 = fmaxf(mx0, fmaf(__uint_as_float(r[j]), prm.scale_log2, bz[c4 * 32 + j]));
+            mx1 = fmaxf(mx1, fmaf(__uint_as_float(r[j + 1]), prm.scale_log2, bz[c4 * 32 + j + 1]));
+            mx2 = fmaxf(mx2, fmaf(__uint_as_float(r[j + 2]), prm.scale_log2, bz[c4 * 32 + j + 2]));
+            mx3 = fmaxf(mx3, fmaf(__uint_as_float(r[j + 3]), prm.scale_log2, bz[c4 * 32 + j + 3]));
           }
-      } else {
+        } else {
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4)
-#pragma unroll
-          for (int j = 0; j < 32; ++j) tmax = fmaxf(tmax, __uint_as_float(sr[c4][j]));
-        tmax *= prm.scale_log2;
-      }
+          for (int j = 0; j < 32; j += 8) {
+            mx0 = fmaxf(mx0, fmaxf(__uint_as_float(r[j]), __uint_as_float(r[j + 1])));
+            mx1 = fmaxf(mx1, fmaxf(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])));
+            mx2 = fmaxf(mx2, fmaxf(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])));
+            mx3 = fmaxf(mx3, fmaxf(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
+          }
+        }
+      };
+      tmem_ld32(tmem_s + lane_addr, ra);
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr + 32, rb);
+      reduce_max(ra, 0);
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr + 64, ra);
+      reduce_max(rb, 1);
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr + 96, rb);
+      reduce_max(ra, 2);
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr, ra);             // first chunk again, for pass 2
+      reduce_max(rb, 3);
+      float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+      if (!masked) tmax *= prm.scale_log2;
+      tA = clock64(); T1 += tA - tB;
       // raise the reference maximum only when a tile exceeds it by the threshold
       const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
       if (__any_sync(0xffffffffu, raise)) {
@@ -288,6 +308,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         l_run *= alpha;
         if (t > 0) {                               // O holds the earlier tiles (their MMAs completed before S)
+          tmem_wait_ld();
 #pragma unroll
           for (int c4 = 0; c4 < D / 32; ++c4) {
             uint32_t o[32];
@@ -299,28 +320,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       }
+      // ---- pass 2: P = exp2(x - m), packed to bf16 over the S columns already consumed
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float psum = 0.f;
-#pragma unroll
-      for (int c4 = 0; c4 < 4; ++c4) {
+      float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+      auto exp_chunk = [&](const uint32_t (&r)[32], int c4) {
         uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-          float x0 = __uint_as_float(sr[c4][2 * j]), x1 = __uint_as_float(sr[c4][2 * j + 1]);
-          float p0, p1;
-          if (masked) { p0 = ex2_approx(x0 + neg_m); p1 = ex2_approx(x1 + neg_m); }
-          else { p0 = ex2_approx(fmaf(x0, prm.scale_log2, neg_m)); p1 = ex2_approx(fmaf(x1, prm.scale_log2, neg_m)); }
-          psum += p0 + p1;
+        for (int j = 0; j < 16; j += 2) {
+          float x0 = __uint_as_float(r[2 * j]), x1 = __uint_as_float(r[2 * j + 1]);
+          float x2 = __uint_as_float(r[2 * j + 2]), x3 = __uint_as_float(r[2 * j + 3]);
+          if (masked) {
+            x0 = fmaf(x0, prm.scale_log2, bz[c4 * 32 + 2 * j] + neg_m);
+            x1 = fmaf(x1, prm.scale_log2, bz[c4 * 32 + 2 * j + 1] + neg_m);
+            x2 = fmaf(x2, prm.scale_log2, bz[c4 * 32 + 2 * j + 2] + neg_m);
+            x3 = fmaf(x3, prm.scale_log2, bz[c4 * 32 + 2 * j + 3] + neg_m);
+          } else {
+            x0 = fmaf(x0, prm.scale_log2, neg_m); x1 = fmaf(x1, prm.scale_log2, neg_m);
+            x2 = fmaf(x2, prm.scale_log2, neg_m); x3 = fmaf(x3, prm.scale_log2, neg_m);
+          }
+          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
+          ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
           pk[j] = pack_bf16x2(p0, p1);
+          pk[j + 1] = pack_bf16x2(p2, p3);
         }
         tmem_st16(tmem_s + lane_addr + c4 * 16, pk);
-      }
+      };
+      // P chunk c overwrites S columns [16c, 16c+16), which pass 2 has read before (chunk c covers
+      // S columns [32c, 32c+32) >= 16c+16 only for c >= 1; chunk 0 is held in registers first)
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr + 32, rb);
+      tmem_wait_ld();                                // chunks 0 and 1 in registers before any P store
+      exp_chunk(ra, 0);
+      tmem_ld32(tmem_s + lane_addr + 64, ra);
+      exp_chunk(rb, 1);
+      tmem_wait_ld();
+      tmem_ld32(tmem_s + lane_addr + 96, rb);
+      exp_chunk(ra, 2);
+      tmem_wait_ld();
+      exp_chunk(rb, 3);
+      const float psum = (ps0 + ps1) + (ps2 + ps3);
       l_run += psum;
+      tB = clock64(); T2 += tB - tA;
       tmem_wait_st();
       tc_fence_before();
       mbar_arrive(b_p_ready);
+      tA = clock64(); T3 += tA - tB;
     }
 
+    if (dbg) { prm.status[8] = (int)(T0 >> 4); prm.status[9] = (int)(T1 >> 4); prm.status[10] = (int)(T2 >> 4); prm.status[11] = (int)(T3 >> 4); prm.status[12] = total_tiles; }
     // epilogue: O / l, rows back to their original positions
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_o_done, 0, abort_flag, prm.status));
     tc_fence_after();
