@@ -3,20 +3,24 @@
 // enters through its centroid key/value with weight |c| exp(q . kbar / sqrt(d))).
 //
 // One CTA per tile of 128 query rows (one query cluster, or half of a 256-row
-// one).  Key/value tiles of 128 rows stream through shared memory by TMA
-// (128-byte swizzle, 64-column panels).  For every tile
-//     S = Q K^T          tcgen05.mma, both operands in shared memory, S in TMEM
-//     P = exp2(S*c - m)  four softmax warps, one query row per thread; P is
-//                        written back over S in TMEM as packed bf16
-//     O += P V           tcgen05.mma, P from TMEM, V from shared memory (MN-major)
-// with a running maximum that is only raised when a tile exceeds it by 2^8
-// (the rescale of O in TMEM is then done by the softmax warps).  After the
-// selected clusters, the key centroids are streamed the same way as extra
-// "keys" (split into bf16 hi + lo parts so the logits keep fp32-level accuracy),
-// with logit bias ln|c| and selected clusters masked; their values are the
-// value centroids.  Warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 do the
+// one); two CTAs share an SM.  Key/value tiles of 128 rows stream through shared
+// memory by TMA (128-byte swizzle, 64-column panels).  The keys are consumed in
+// half-steps of 64, alternating between two 64-column score buffers in tensor
+// memory, so that the tensor core works on one half-step while the softmax
+// warps work on the other:
+//     S_b = Q K_h^T        tcgen05.mma, both operands in shared memory
+//     P_b = exp2(S_b c - m) four softmax warps, one query row per thread; P is
+//                          written back over S_b as packed bf16
+//     O  += P_b V_h        tcgen05.mma, P from tensor memory, V from shared memory (MN-major)
+// issued as S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  The running maximum is only
+// raised when a half-step exceeds it by 2^8; the softmax warps then rescale O in
+// tensor memory themselves after waiting for the one product that can still be
+// in flight.  After the selected clusters the key centroids are streamed as
+// extra keys, 64 per half-step: their tile holds bf16 hi parts in rows 0-63 and
+// lo parts in rows 64-127, accumulated by two products so the centroid logits
+// keep fp32-level accuracy; logit bias ln|c|, selected clusters masked; values are
+// the value centroids.  Warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 do the
 // softmax and the epilogue (rows scattered back to the original order).
-// Two CTAs share an SM so one's softmax overlaps the other's MMAs.
 #include "kernels.h"
 #include "tc_ptx.cuh"
 
@@ -26,7 +30,8 @@ using namespace ptx;
 
 constexpr int kTcThreads = 192;
 constexpr int kTile = 128;                 // query rows per CTA, key rows per tile
-constexpr uint32_t kTmemCols = 256;        // S: [0,128)  O: [128, 128+D)
+constexpr int kHalf = 64;                  // keys per half-step
+constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 template <int D>
@@ -39,9 +44,9 @@ struct TcCfg {
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + STAGES * TILE_BYTES;
-  static constexpr int OFF_BIAS = OFF_V + STAGES * TILE_BYTES;     // 2 x 128 floats
-  static constexpr int OFF_BAR = OFF_BIAS + 2 * kTile * 4;
-  static constexpr int NUM_BARS = 4 + 4 * STAGES;
+  static constexpr int OFF_BIAS = OFF_V + STAGES * TILE_BYTES;     // 4 x 64 floats
+  static constexpr int OFF_BAR = OFF_BIAS + 4 * kHalf * 4;
+  static constexpr int NUM_BARS = 8 + 4 * STAGES;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;           // tmem base, abort flag
   static constexpr int OFF_BITMAP = OFF_MISC + 16;
 };
@@ -53,7 +58,7 @@ struct TcParams {
   __nv_bfloat16* O;
   float* lse;
   int* status;
-  int n_q, n_k, c_q, c_k, keep, n_qc, n_kc, n_kc_pad, compensate, bitmap_words;
+  int n_q, n_k, c_q, c_k, keep, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
   float scale_log2;
 };
 
@@ -65,9 +70,8 @@ __host__ __device__ inline int selected_tiles(int keep, int c_k) {
 template <int D>
 __global__ void __launch_bounds__(kTcThreads, 2)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ckhi,
-               const __grid_constant__ CUtensorMap tm_cklo, const __grid_constant__ CUtensorMap tm_cv,
-               const TcParams prm) {
+               const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ck,
+               const __grid_constant__ CUtensorMap tm_cv, const TcParams prm) {
   using C = TcCfg<D>;
   extern __shared__ unsigned char smem_unaligned[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
@@ -76,12 +80,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t s_q = s_base + C::OFF_Q, s_k = s_base + C::OFF_K, s_v = s_base + C::OFF_V;
   float* bias = reinterpret_cast<float*>(smem + C::OFF_BIAS);
   const uint32_t bar0 = s_base + C::OFF_BAR;
-  // barrier indices
-  const uint32_t b_q_full = bar0, b_s_full = bar0 + 8, b_p_ready = bar0 + 16, b_o_done = bar0 + 24;
-  auto b_k_full = [&](int s) { return bar0 + 32 + 8 * s; };
-  auto b_k_empty = [&](int s) { return bar0 + 32 + 8 * (C::STAGES + s); };
-  auto b_v_full = [&](int s) { return bar0 + 32 + 8 * (2 * C::STAGES + s); };
-  auto b_v_empty = [&](int s) { return bar0 + 32 + 8 * (3 * C::STAGES + s); };
+  const uint32_t b_q_full = bar0, b_o_done = bar0 + 8;
+  auto b_s_full = [&](int b) { return bar0 + 16 + 8 * b; };
+  auto b_p_ready = [&](int b) { return bar0 + 32 + 8 * b; };
+  auto b_pv_done = [&](int b) { return bar0 + 48 + 8 * b; };
+  auto b_k_full = [&](int s) { return bar0 + 64 + 8 * s; };
+  auto b_k_empty = [&](int s) { return bar0 + 64 + 8 * (C::STAGES + s); };
+  auto b_v_full = [&](int s) { return bar0 + 64 + 8 * (2 * C::STAGES + s); };
+  auto b_v_empty = [&](int s) { return bar0 + 64 + 8 * (3 * C::STAGES + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
   unsigned* bitmap = reinterpret_cast<unsigned*>(smem + C::OFF_BITMAP);
@@ -92,14 +98,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int qc = blockIdx.x / tiles_per_qc, half = blockIdx.x % tiles_per_qc;
   const int32_t* sel = prm.block_idx + ((size_t)p * prm.n_qc + qc) * prm.keep;
   const int sel_tiles = selected_tiles(prm.keep, prm.c_k);
-  const int cen_tiles = prm.compensate ? prm.n_kc_pad / kTile : 0;
-  const int total_tiles = sel_tiles + cen_tiles;
+  const int cen_tiles = prm.compensate ? prm.cen_tiles : 0;
+  const int loads = sel_tiles + cen_tiles;             // K/V tile loads
+  const int steps = 2 * sel_tiles + cen_tiles;         // half-steps of 64 keys
 
   if (tid == 0) {
     mbar_init(b_q_full, 1);
-    mbar_init(b_s_full, 1);
-    mbar_init(b_p_ready, 128);
     mbar_init(b_o_done, 1);
+    for (int b = 0; b < 2; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 128); mbar_init(b_pv_done(b), 1); }
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(b_k_full(s), 1); mbar_init(b_k_empty(s), 1);
       mbar_init(b_v_full(s), 1); mbar_init(b_v_empty(s), 1);
@@ -124,7 +130,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int q_row = (p * prm.n_qc + qc) * prm.c_q + half * kTile;
       mbar_expect_tx(b_q_full, C::TILE_BYTES);
       for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(s_q + pn * C::PANEL_BYTES, &tm_q, pn * 64, q_row, b_q_full);
-      int kg = 0;                          // key load groups issued so far
       bool ok = true;
       auto load_rows = [&](uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
         for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(dst + pn * C::PANEL_BYTES, map, pn * 64, row, bar);
@@ -147,64 +152,75 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       };
-      for (int t = 0; t < total_tiles && ok; ++t) {
-        const int groups = t < sel_tiles ? 1 : 2;
-        for (int g = 0; g < groups && ok; ++g, ++kg) {
-          const int s = kg % C::STAGES;
-          if (kg >= C::STAGES) ok = mbar_wait(b_k_empty(s), ((kg / C::STAGES) - 1) & 1, abort_flag, prm.status);
-          if (!ok) break;
-          mbar_expect_tx(b_k_full(s), C::TILE_BYTES);
-          if (t < sel_tiles) load_selected(s_k + s * C::TILE_BYTES, &tm_k, t, b_k_full(s));
-          else load_rows(s_k + s * C::TILE_BYTES, g == 0 ? &tm_ckhi : &tm_cklo,
-                         p * prm.n_kc_pad + (t - sel_tiles) * kTile, b_k_full(s));
-        }
-        if (!ok) break;
+      for (int t = 0; t < loads && ok; ++t) {
         const int s = t % C::STAGES;
+        if (t >= C::STAGES) ok = mbar_wait(b_k_empty(s), ((t / C::STAGES) - 1) & 1, abort_flag, prm.status);
+        if (!ok) break;
+        mbar_expect_tx(b_k_full(s), C::TILE_BYTES);
+        if (t < sel_tiles) load_selected(s_k + s * C::TILE_BYTES, &tm_k, t, b_k_full(s));
+        else load_rows(s_k + s * C::TILE_BYTES, &tm_ck, (p * prm.cen_tiles + (t - sel_tiles)) * kTile, b_k_full(s));
         if (t >= C::STAGES) ok = mbar_wait(b_v_empty(s), ((t / C::STAGES) - 1) & 1, abort_flag, prm.status);
         if (!ok) break;
-        mbar_expect_tx(b_v_full(s), C::TILE_BYTES);
-        if (t < sel_tiles) load_selected(s_v + s * C::TILE_BYTES, &tm_v, t, b_v_full(s));
-        else load_rows(s_v + s * C::TILE_BYTES, &tm_cv, p * prm.n_kc_pad + (t - sel_tiles) * kTile, b_v_full(s));
+        if (t < sel_tiles) {
+          mbar_expect_tx(b_v_full(s), C::TILE_BYTES);
+          load_selected(s_v + s * C::TILE_BYTES, &tm_v, t, b_v_full(s));
+        } else {                                            // 64 value centroids
+          mbar_expect_tx(b_v_full(s), C::TILE_BYTES / 2);
+          load_rows(s_v + s * C::TILE_BYTES, &tm_cv, (p * prm.cen_tiles + (t - sel_tiles)) * kHalf, b_v_full(s));
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kTile, 0, 0);
+      constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, D, 0, 1);
       bool ok = mbar_wait(b_q_full, 0, abort_flag, prm.status);
-      int kg = 0;
-      for (int t = 0; t < total_tiles && ok; ++t) {
-        const int groups = t < sel_tiles ? 1 : 2;
-        for (int g = 0; g < groups && ok; ++g, ++kg) {
-          const int s = kg % C::STAGES;
-          ok = mbar_wait(b_k_full(s), (kg / C::STAGES) & 1, abort_flag, prm.status);
-          if (!ok) break;
+      // load index of half-step u (the shared-memory slot is the load index modulo the stages)
+      auto load_of = [&](int u) { return u < 2 * sel_tiles ? u >> 1 : sel_tiles + (u - 2 * sel_tiles); };
+      auto issue_s = [&](int u) {
+        const int L = load_of(u), s = L % C::STAGES, b = u & 1;
+        const bool centroid = u >= 2 * sel_tiles;
+        if (centroid || b == 0) {
+          if (!mbar_wait(b_k_full(s), (L / C::STAGES) & 1, abort_flag, prm.status)) return false;
           tc_fence_after();
+        }
+        const uint32_t kt = s_k + s * C::TILE_BYTES;
+        const int parts = centroid ? 2 : 1;               // centroid tile: hi rows 0-63, lo rows 64-127
+        for (int g = 0; g < parts; ++g) {
+          const uint32_t rows = (centroid ? g : b) * (kHalf * 128);   // 64 rows = 8192 bytes inside a panel
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
             const uint32_t off = (ks / 4) * C::PANEL_BYTES + (ks % 4) * 32;
             const uint64_t a = smem_desc_sw128(s_q + off, 16, 1024);
-            const uint64_t b = smem_desc_sw128(s_k + s * C::TILE_BYTES + off, 16, 1024);
-            mma_ss(tmem_s, a, b, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            const uint64_t bd = smem_desc_sw128(kt + rows + off, 16, 1024);
+            mma_ss(tmem_s + b * kHalf, a, bd, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
           }
-          mma_commit(b_k_empty(s));
         }
-        if (!ok) break;
-        mma_commit(b_s_full);
-        const int s = t % C::STAGES;
-        ok = mbar_wait(b_p_ready, t & 1, abort_flag, prm.status) &&
-             mbar_wait(b_v_full(s), (t / C::STAGES) & 1, abort_flag, prm.status);
+        if (centroid || b == 1) mma_commit(b_k_empty(s));
+        mma_commit(b_s_full(b));
+        return true;
+      };
+      if (ok && steps > 0) ok = issue_s(0);
+      if (ok && steps > 1) ok = issue_s(1);
+      for (int u = 0; u < steps && ok; ++u) {
+        const int L = load_of(u), s = L % C::STAGES, b = u & 1;
+        const bool centroid = u >= 2 * sel_tiles;
+        ok = mbar_wait(b_p_ready(b), (u >> 1) & 1, abort_flag, prm.status);
+        if (ok && (centroid || b == 0)) ok = mbar_wait(b_v_full(s), (L / C::STAGES) & 1, abort_flag, prm.status);
         if (!ok) break;
         tc_fence_after();
+        const uint32_t vt = s_v + s * C::TILE_BYTES + (centroid ? 0 : b) * (kHalf * 128);
 #pragma unroll
-        for (int ks = 0; ks < kTile / 16; ++ks) {
+        for (int ks = 0; ks < kHalf / 16; ++ks) {
           // V is MN-major: 16 key rows (2048 bytes) per step; panels along d
-          const uint64_t b = smem_desc_sw128(s_v + s * C::TILE_BYTES + ks * 2048, C::PANEL_BYTES, 1024);
-          mma_ts(tmem_o, tmem_s + ks * 8, b, idesc_pv, (t > 0 || ks > 0) ? 1u : 0u);
+          const uint64_t bd = smem_desc_sw128(vt + ks * 2048, C::PANEL_BYTES, 1024);
+          mma_ts(tmem_o, tmem_s + b * kHalf + ks * 8, bd, idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
         }
-        mma_commit(b_v_empty(s));
+        mma_commit(b_pv_done(b));
+        if (centroid || b == 1) mma_commit(b_v_empty(s));
+        if (u + 2 < steps) ok = issue_s(u + 2);
       }
       mma_commit(b_o_done);
     }
@@ -223,44 +239,46 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
     float m_ref = -INFINITY, l_run = 0.f;
     bool ok = true;
-    long long T0 = 0, T1 = 0, T2 = 0, T3 = 0, tA, tB;
-    const bool dbg = (blockIdx.x == 5 && blockIdx.y == 0 && st == 0);
-    for (int t = 0; t < total_tiles && ok; ++t) {
-      // per-column additive term (log2 units): only tiles with masked or weighted columns need it.
-      // `masked` depends on the tile only, so it is uniform over the 128 threads.
+    for (int u = 0; u < steps && ok; ++u) {
+      const int b = u & 1;
+      const uint32_t t_s = tmem_s + lane_addr + b * kHalf;
+      // per-column additive term (log2 units): only half-steps with masked or weighted columns need
+      // it.  `masked` depends on the half-step only, so it is uniform over the 128 threads.
       bool masked = false;
-      float* bz = bias + (t & 1) * kTile;
-      if (t < sel_tiles) {
-        bool use;
+      // four buffers: a thread can run at most two half-steps ahead of the slowest one
+      float* bz = bias + (u & 3) * kHalf;
+      if (u < 2 * sel_tiles) {
+        const int t = u >> 1;
+        bool use = true;
         if (prm.c_k >= kTile) {
           const int per = prm.c_k / kTile;
           const int members = cnt[sel[t / per]];
-          masked = members < prm.c_k;
-          use = st < members - (t % per) * kTile;
+          const int first = (t % per) * kTile + b * kHalf;      // row of this half-step's first column
+          masked = members < first + kHalf;
+          use = first + (st & 63) < members;
         } else {
-          const int per = kTile / prm.c_k;
-          for (int u = 0; u < per; ++u) {
-            const int e = t * per + u;
+          const int col0 = t * kTile + b * kHalf;                // position in the list of selected rows
+          const int per = prm.c_k >= kHalf ? 1 : kHalf / prm.c_k;
+          for (int x = 0; x < per; ++x) {
+            const int e = (col0 + x * prm.c_k) / prm.c_k;
             if (e >= prm.keep || cnt[sel[e]] < prm.c_k) masked = true;
           }
-          const int e = t * per + st / prm.c_k;
-          use = e < prm.keep && (st % prm.c_k) < cnt[sel[min(e, prm.keep - 1)]];
+          const int e = (col0 + (st & 63)) / prm.c_k;
+          use = e < prm.keep && ((col0 + (st & 63)) % prm.c_k) < cnt[sel[min(e, prm.keep - 1)]];
         }
-        if (masked) bz[st] = use ? 0.f : -INFINITY;
+        if (masked && st < kHalf) bz[st] = use ? 0.f : -INFINITY;
       } else {
         masked = true;
-        const int j = (t - sel_tiles) * kTile + st;
+        const int j = (u - 2 * sel_tiles) * kHalf + (st & 63);
         const bool use = j < prm.n_kc && !((bitmap[j >> 5] >> (j & 31)) & 1u);
-        bz[st] = use ? log2f((float)cnt[min(j, prm.n_kc - 1)]) : -INFINITY;
+        if (st < kHalf) bz[st] = use ? log2f((float)cnt[min(j, prm.n_kc - 1)]) : -INFINITY;
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
 
-      tA = clock64();
-      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full, t & 1, abort_flag, prm.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(b), (u >> 1) & 1, abort_flag, prm.status));
       if (!ok) break;
       tc_fence_after();
-      tB = clock64(); T0 += tB - tA;
-      // ---- pass 1: row maximum (TMEM chunks of 32 columns, the next load in flight while one is reduced)
+      // ---- pass 1: row maximum over the 64 columns
       uint32_t ra[32], rb[32];
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
       auto reduce_max = [&](const uint32_t (&r)[32], int c4) {
@@ -282,23 +300,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       };
-      tmem_ld32(tmem_s + lane_addr, ra);
+      tmem_ld32(t_s, ra);
+      tmem_ld32(t_s + 32, rb);
       tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr + 32, rb);
       reduce_max(ra, 0);
-      tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr + 64, ra);
       reduce_max(rb, 1);
-      tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr + 96, rb);
-      reduce_max(ra, 2);
-      tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr, ra);             // first chunk again, for pass 2
-      reduce_max(rb, 3);
       float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
       if (!masked) tmax *= prm.scale_log2;
-      tA = clock64(); T1 += tA - tB;
-      // raise the reference maximum only when a tile exceeds it by the threshold
+      // raise the reference maximum only when a half-step exceeds it by the threshold
       const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
       if (__any_sync(0xffffffffu, raise)) {
         float alpha = 1.f;
@@ -307,8 +316,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           m_ref = tmax;
         }
         l_run *= alpha;
-        if (t > 0) {                               // O holds the earlier tiles (their MMAs completed before S)
-          tmem_wait_ld();
+        if (u > 0) {
+          // S(u) complete means every product up to PV(u-2) is complete; PV(u-1) may still run
+          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done(b ^ 1), ((u - 1) >> 1) & 1, abort_flag, prm.status));
+          if (!ok) break;
+          tc_fence_after();
 #pragma unroll
           for (int c4 = 0; c4 < D / 32; ++c4) {
             uint32_t o[32];
@@ -320,7 +332,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           }
         }
       }
-      // ---- pass 2: P = exp2(x - m), packed to bf16 over the S columns already consumed
+      // ---- pass 2: P = exp2(x - m), packed to bf16 over the first 32 columns of the buffer
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
       auto exp_chunk = [&](const uint32_t (&r)[32], int c4) {
@@ -343,31 +355,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           pk[j] = pack_bf16x2(p0, p1);
           pk[j + 1] = pack_bf16x2(p2, p3);
         }
-        tmem_st16(tmem_s + lane_addr + c4 * 16, pk);
+        tmem_st16(t_s + c4 * 16, pk);       // both chunks are in registers: the stores cannot clobber unread S
       };
-      // P chunk c overwrites S columns [16c, 16c+16), which pass 2 has read before (chunk c covers
-      // S columns [32c, 32c+32) >= 16c+16 only for c >= 1; chunk 0 is held in registers first)
-      tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr + 32, rb);
-      tmem_wait_ld();                                // chunks 0 and 1 in registers before any P store
       exp_chunk(ra, 0);
-      tmem_ld32(tmem_s + lane_addr + 64, ra);
       exp_chunk(rb, 1);
-      tmem_wait_ld();
-      tmem_ld32(tmem_s + lane_addr + 96, rb);
-      exp_chunk(ra, 2);
-      tmem_wait_ld();
-      exp_chunk(rb, 3);
-      const float psum = (ps0 + ps1) + (ps2 + ps3);
-      l_run += psum;
-      tB = clock64(); T2 += tB - tA;
+      l_run += (ps0 + ps1) + (ps2 + ps3);
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(b_p_ready);
-      tA = clock64(); T3 += tA - tB;
+      mbar_arrive(b_p_ready(b));
     }
 
-    if (dbg) { prm.status[8] = (int)(T0 >> 4); prm.status[9] = (int)(T1 >> 4); prm.status[10] = (int)(T2 >> 4); prm.status[11] = (int)(T3 >> 4); prm.status[12] = total_tiles; }
     // epilogue: O / l, rows back to their original positions
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_o_done, 0, abort_flag, prm.status));
     tc_fence_after();
@@ -405,26 +402,27 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------
-// Centroids for the tensor-core path: key centroids as bf16 hi + lo parts, value
-// centroids as bf16, rows padded with zeros to a multiple of 128.
+// Centroids for the tensor-core path, 64 per tile: key tile = 64 rows of bf16 hi
+// parts followed by 64 rows of lo parts; value centroids as bf16.  Rows beyond
+// the last centroid are zero.
 // ---------------------------------------------------------------------------
 __global__ void centroid_prep_kernel(const float* __restrict__ ck, const float* __restrict__ cv, int n_kc,
-                                     int n_kc_pad, int D, __nv_bfloat16* __restrict__ hi,
-                                     __nv_bfloat16* __restrict__ lo, __nv_bfloat16* __restrict__ vb) {
+                                     int cen_tiles, int D, __nv_bfloat16* __restrict__ kmix,
+                                     __nv_bfloat16* __restrict__ vb) {
   const int p = blockIdx.y;
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= n_kc_pad * D) return;
-  const int j = e / D;
+  if (e >= cen_tiles * kHalf * D) return;
+  const int j = e / D, col = e % D;
   float k = 0.f, v = 0.f;
   if (j < n_kc) {
     k = ck[(size_t)p * n_kc * D + e];
     v = cv[(size_t)p * n_kc * D + e];
   }
   const __nv_bfloat16 h = __float2bfloat16_rn(k);
-  const size_t o = (size_t)p * n_kc_pad * D + e;
-  hi[o] = h;
-  lo[o] = __float2bfloat16_rn(k - __bfloat162float(h));
-  vb[o] = __float2bfloat16_rn(v);
+  const size_t tile = (size_t)p * cen_tiles + j / kHalf;
+  kmix[(tile * kTile + (j % kHalf)) * D + col] = h;
+  kmix[(tile * kTile + kHalf + (j % kHalf)) * D + col] = __float2bfloat16_rn(k - __bfloat162float(h));
+  vb[((size_t)p * cen_tiles * kHalf + j) * D + col] = __float2bfloat16_rn(v);
 }
 
 // ---------------------------------------------------------------------------
@@ -471,18 +469,18 @@ bool attn_tc_supported(const ca_problem_t& pr) {
 
 size_t attn_tc_workspace_bytes(const ca_problem_t& pr) {
   const size_t P = (size_t)pr.batch * pr.heads;
-  const size_t n_kc_pad = (size_t)align_up(ceil_div(pr.n_k, pr.cluster_k), kTile);
-  return kStatusBytes + 3 * align_up(P * n_kc_pad * pr.head_dim * sizeof(__nv_bfloat16), 256);
+  const size_t cen_tiles = (size_t)ceil_div(ceil_div(pr.n_k, pr.cluster_k), kHalf);
+  return kStatusBytes + align_up(P * cen_tiles * kTile * pr.head_dim * sizeof(__nv_bfloat16), 256) +
+         align_up(P * cen_tiles * kHalf * pr.head_dim * sizeof(__nv_bfloat16), 256);
 }
 
 template <int D>
-static int launch_tc_d(const ca_problem_t& pr, const CUtensorMap* maps, const TcParams& prm, dim3 grid,
-                       cudaStream_t st) {
+static int launch_tc_d(const CUtensorMap* maps, const TcParams& prm, dim3 grid, cudaStream_t st) {
   using C = TcCfg<D>;
   const size_t smem = 1024 + C::OFF_BITMAP + (size_t)prm.bitmap_words * 4;
   auto k = attn_tc_kernel<D>;
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-  k<<<grid, kTcThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], maps[5], prm);
+  k<<<grid, kTcThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
@@ -492,35 +490,34 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
                    float scale, void* O, float* lse, void* ws, cudaStream_t st) {
   const int P = pr.batch * pr.heads, D = pr.head_dim;
   const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
-  const int n_kc_pad = (int)align_up(n_kc, kTile);
+  const int cen_tiles = ceil_div(n_kc, kHalf);
   Carver c(ws);
   int* status = c.take<int>(kStatusBytes / sizeof(int));
-  __nv_bfloat16* hi = c.take<__nv_bfloat16>((size_t)P * n_kc_pad * D);
-  __nv_bfloat16* lo = c.take<__nv_bfloat16>((size_t)P * n_kc_pad * D);
-  __nv_bfloat16* vb = c.take<__nv_bfloat16>((size_t)P * n_kc_pad * D);
+  __nv_bfloat16* kmix = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kTile * D);
+  __nv_bfloat16* vb = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kHalf * D);
   if (pr.compensate) {
-    centroid_prep_kernel<<<dim3(ceil_div(n_kc_pad * D, 256), P), 256, 0, st>>>(ck, cv, n_kc, n_kc_pad, D, hi, lo, vb);
+    centroid_prep_kernel<<<dim3(ceil_div(cen_tiles * kHalf * D, 256), P), 256, 0, st>>>(ck, cv, n_kc, cen_tiles, D,
+                                                                                        kmix, vb);
     CA_LAUNCH_CHECK();
   }
-  CUtensorMap maps[6];
+  CUtensorMap maps[5];
   const int kbox = pr.cluster_k < kTile ? pr.cluster_k : kTile;
   bool ok = make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, kTile) &&
             make_map(&maps[1], Kp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
             make_map(&maps[2], Vp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
-            make_map(&maps[3], hi, (size_t)P * n_kc_pad, D, kTile) &&
-            make_map(&maps[4], lo, (size_t)P * n_kc_pad, D, kTile) &&
-            make_map(&maps[5], vb, (size_t)P * n_kc_pad, D, kTile);
+            make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kTile) &&
+            make_map(&maps[4], vb, (size_t)P * cen_tiles * kHalf, D, kHalf);
   if (!ok) return CA_ERR_CUDA;
   TcParams prm;
   prm.count_k = count_k; prm.block_idx = block_idx; prm.perm_q = perm_q;
   prm.O = static_cast<__nv_bfloat16*>(O); prm.lse = lse; prm.status = status;
   prm.n_q = pr.n_q; prm.n_k = pr.n_k; prm.c_q = pr.cluster_q; prm.c_k = pr.cluster_k; prm.keep = pr.keep;
-  prm.n_qc = n_qc; prm.n_kc = n_kc; prm.n_kc_pad = n_kc_pad; prm.compensate = pr.compensate;
-  prm.bitmap_words = (n_kc_pad + 31) / 32;
+  prm.n_qc = n_qc; prm.n_kc = n_kc; prm.cen_tiles = cen_tiles; prm.compensate = pr.compensate;
+  prm.bitmap_words = (cen_tiles * kHalf + 31) / 32;
   prm.scale_log2 = scale * 1.4426950408889634f;
   dim3 grid(n_qc * (pr.cluster_q / kTile), P);
-  if (D == 64) return launch_tc_d<64>(pr, maps, prm, grid, st);
-  return launch_tc_d<128>(pr, maps, prm, grid, st);
+  if (D == 64) return launch_tc_d<64>(maps, prm, grid, st);
+  return launch_tc_d<128>(maps, prm, grid, st);
 }
 
 }  // namespace ca
