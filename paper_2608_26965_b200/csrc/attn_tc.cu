@@ -33,6 +33,11 @@ constexpr int kTile = 128;                 // query rows per CTA, key rows per t
 constexpr int kHalf = 64;                  // keys per half-step
 constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+#ifndef CA_POLY_MODE
+#define CA_POLY_MODE 0
+#endif
+// share of the exponentials evaluated by polynomial on the FMA pipe: 0, 1/4, 3/8, 1/2
+constexpr int kPolyMode = CA_POLY_MODE;
 
 template <int D>
 struct TcCfg {
@@ -336,24 +341,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
       auto exp_chunk = [&](const uint32_t (&r)[32], int c4) {
+        // three sweeps over 32 independent elements (scale, exponential, sum + pack) so that the
+        // instruction stream never waits on a result produced a few instructions earlier
+        float x[32];
+        if (masked) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, bz[c4 * 32 + j] + neg_m);
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
+        }
+#pragma unroll
+        for (int j = 0; j < 32; ++j) {
+          const bool poly = (kPolyMode >= 1 && (j & 3) == 3) || (kPolyMode == 3 && (j & 3) == 1) ||
+                            (kPolyMode == 2 && (j & 7) == 1);
+          x[j] = poly ? ex2_poly(x[j]) : ex2_approx(x[j]);
+        }
         uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-          float x0 = __uint_as_float(r[2 * j]), x1 = __uint_as_float(r[2 * j + 1]);
-          float x2 = __uint_as_float(r[2 * j + 2]), x3 = __uint_as_float(r[2 * j + 3]);
-          if (masked) {
-            x0 = fmaf(x0, prm.scale_log2, bz[c4 * 32 + 2 * j] + neg_m);
-            x1 = fmaf(x1, prm.scale_log2, bz[c4 * 32 + 2 * j + 1] + neg_m);
-            x2 = fmaf(x2, prm.scale_log2, bz[c4 * 32 + 2 * j + 2] + neg_m);
-            x3 = fmaf(x3, prm.scale_log2, bz[c4 * 32 + 2 * j + 3] + neg_m);
-          } else {
-            x0 = fmaf(x0, prm.scale_log2, neg_m); x1 = fmaf(x1, prm.scale_log2, neg_m);
-            x2 = fmaf(x2, prm.scale_log2, neg_m); x3 = fmaf(x3, prm.scale_log2, neg_m);
-          }
-          const float p0 = ex2_approx(x0), p1 = ex2_approx(x1), p2 = ex2_approx(x2), p3 = ex2_approx(x3);
-          ps0 += p0; ps1 += p1; ps2 += p2; ps3 += p3;
-          pk[j] = pack_bf16x2(p0, p1);
-          pk[j + 1] = pack_bf16x2(p2, p3);
+        for (int j = 0; j < 32; j += 4) {
+          ps0 += x[j]; ps1 += x[j + 1]; ps2 += x[j + 2]; ps3 += x[j + 3];
+          pk[j / 2] = pack_bf16x2(x[j], x[j + 1]);
+          pk[j / 2 + 1] = pack_bf16x2(x[j + 2], x[j + 3]);
         }
         tmem_st16(t_s + c4 * 16, pk);       // both chunks are in registers: the stores cannot clobber unread S
       };

@@ -167,6 +167,19 @@ __device__ __forceinline__ float ex2_approx(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+// 2^x on the FMA pipe: round-to-nearest split x = n + f, |f| <= 1/2, cubic minimax
+// polynomial for 2^f (relative error 7.5e-5, far below bf16 resolution), exponent
+// added through the integer bits.  Used for a share of the softmax exponentials
+// so that the 16-per-clock special-function unit is not the only exp provider.
+__device__ __forceinline__ float ex2_poly(float x) {
+  x = fmaxf(x, -126.0f);
+  const float t = x + 12582912.0f;                     // 1.5 * 2^23: n lands in the low mantissa bits
+  const float f = x - (t - 12582912.0f);
+  float p = fmaf(0.05517165f, f, 0.24261113f);
+  p = fmaf(p, f, 0.69326097f);
+  p = fmaf(p, f, 0.99992806f);
+  return __int_as_float(__float_as_int(p) + (__float_as_int(t) << 23));
+}
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   uint32_t r;
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
