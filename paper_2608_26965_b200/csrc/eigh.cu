@@ -6,7 +6,7 @@
 
 namespace ca {
 
-constexpr int kMaxSweeps = 16;
+constexpr int kMaxSweeps = 12;
 constexpr int kEighThreads = 1024;
 
 template <int D>
@@ -108,7 +108,10 @@ eigh_kernel(const double* __restrict__ A_in, double* __restrict__ out64, float* 
   AT* Anext = Abuf1;
   Vec4<AT> nv0[C::NV], nv1[C::NV];
   bool v_pending = false;
-  const double tol = sizeof(AT) == 4 ? 1e-12 : 1e-24;     // squared relative off-diagonal norm
+  // Stop when the squared off-diagonal norm is below `tol` of the matrix norm, or when a sweep no
+  // longer reduces it fourfold (the rounding floor of the working precision has been reached).
+  const double tol = sizeof(AT) == 4 ? 1e-11 : 1e-24;
+  double prev_off = 1e300;       // used by thread 0 only
   for (int sweep = 0; sweep < kMaxSweeps; ++sweep) {
     // convergence: off-diagonal mass against the whole matrix
     double off = 0.0, tot = 0.0;
@@ -127,7 +130,8 @@ eigh_kernel(const double* __restrict__ A_in, double* __restrict__ out64, float* 
     if (tid == 0) {
       double o = 0.0, t = 0.0;
       for (int w = 0; w < NT / 32; ++w) { o += red[w]; t += red[32 + w]; }
-      *flag = (o <= tol * t) ? 1 : 0;
+      *flag = (o <= tol * t || (sweep >= 3 && o > 0.25 * prev_off)) ? 1 : 0;
+      prev_off = o;
     }
     __syncthreads();
     if (*flag) break;
