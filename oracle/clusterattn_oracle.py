@@ -140,15 +140,25 @@ def subsample_positions(s, m):
     return (np.arange(m, dtype=np.int64) * s) // m
 
 
+def interleaved_sum(x):
+    """Column sums of x [m, d] in a fixed order: eight partial sums over the rows
+    j = r, r+8, r+16, ... (each taken row after row), combined as
+    ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)).  The paper fixes no summation order; this
+    one is reproducible and lets eight workers share a column."""
+    parts = [np.cumsum(x[r::8], axis=0)[-1] if x[r::8].shape[0] else np.zeros(x.shape[1], F64)
+             for r in range(8)]
+    return ((parts[0] + parts[1]) + (parts[2] + parts[3])) + ((parts[4] + parts[5]) + (parts[6] + parts[7]))
+
+
 def choose_coordinate(sub):
     """Coordinate of highest variance over the subsample rows `sub` [m, d]
-    (population variance; sums taken row after row in float64; lowest
-    coordinate on exact ties)."""
+    (population variance in float64, sums in the order of `interleaved_sum`;
+    lowest coordinate on exact ties)."""
     sub = np.asarray(sub, F64)
     m = sub.shape[0]
-    mean = np.cumsum(sub, axis=0)[-1] / m
+    mean = interleaved_sum(sub) / m
     dev = sub - mean
-    var = np.cumsum(dev * dev, axis=0)[-1] / m
+    var = interleaved_sum(dev * dev) / m
     return int(np.argmax(var)), var
 
 

@@ -58,18 +58,42 @@ __device__ __forceinline__ uint32_t order_key(float x) {
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-// Variance of coordinate t over a subsample staged in shared memory as tile[j*D + t], j < m.
-// The additions run in a fixed order (row after row) in double.
-__device__ __forceinline__ double staged_variance(const float* tile, int D, int t, int m) {
-  double sum = 0.0;
-  for (int j = 0; j < m; ++j) sum = __dadd_rn(sum, (double)tile[j * D + t]);
-  const double mean = sum / (double)m;
-  double acc = 0.0;
-  for (int j = 0; j < m; ++j) {
-    const double dev = __dsub_rn((double)tile[j * D + t], mean);
-    acc = __dadd_rn(acc, __dmul_rn(dev, dev));
+// Variances of all coordinates over subsamples staged in shared memory, `ng` tiles of
+// tile[j*D + t], j < m_g.  Summation order (fixed, so the result is reproducible bit for
+// bit): eight partial sums over the rows j = r, r+8, ... taken row after row, combined
+// as ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)); first the mean, then the squared deviations.
+// part: [ng][8][D] doubles, out: [ng][D] doubles.  Called by all threads of the CTA.
+template <typename RowsOf>
+__device__ __forceinline__ void staged_variances(const float* tiles, int D, int ng, RowsOf rows_of,
+                                                 double* part, double* out, int tid, int nt) {
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int task = tid; task < ng * 8 * D; task += nt) {
+      const int gi = task / (8 * D), r = (task / D) % 8, t = task % D;
+      const int m = rows_of(gi);
+      const float* tile = tiles + gi * D * D;
+      double acc = 0.0;
+      if (pass == 0) {
+        for (int j = r; j < m; j += 8) acc = __dadd_rn(acc, (double)tile[j * D + t]);
+      } else {
+        const double mean = out[gi * D + t];
+        for (int j = r; j < m; j += 8) {
+          const double dev = __dsub_rn((double)tile[j * D + t], mean);
+          acc = __dadd_rn(acc, __dmul_rn(dev, dev));
+        }
+      }
+      part[(gi * 8 + r) * D + t] = acc;
+    }
+    __syncthreads();
+    for (int task = tid; task < ng * D; task += nt) {
+      const int gi = task / D, t = task % D;
+      const double* p = part + gi * 8 * D + t;
+      const double tot = __dadd_rn(__dadd_rn(__dadd_rn(p[0], p[D]), __dadd_rn(p[2 * D], p[3 * D])),
+                                   __dadd_rn(__dadd_rn(p[4 * D], p[5 * D]), __dadd_rn(p[6 * D], p[7 * D])));
+      const int m = rows_of(gi);
+      out[task] = m > 0 ? tot / (double)m : -1.0;
+    }
+    __syncthreads();
   }
-  return acc / (double)m;
 }
 
 struct SplitSide {
@@ -98,6 +122,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   __shared__ int s_hist[256];
   __shared__ int s_total[256];
   __shared__ double s_var[128];
+  __shared__ double s_part[8 * 128];
   __shared__ int s_sub[128];
   __shared__ int s_warp[2 * 32];
   __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank, 3: chunk total
@@ -137,8 +162,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
       stage4[e] = __ldg(reinterpret_cast<const float4*>(Y + (size_t)s_sub[e / q] * D) + (e % q));
   }
   __syncthreads();
-  if (tid < D) s_var[tid] = staged_variance(reinterpret_cast<const float*>(smem_raw), D, tid, m);
-  __syncthreads();
+  staged_variances(reinterpret_cast<const float*>(smem_raw), D, 1, [&](int) { return m; }, s_part, s_var, tid, nt);
   if (warp == 0) {
     double best = -1.0; int arg = 0;
     for (int t = lane; t < D; t += 32) {
@@ -301,6 +325,8 @@ struct TailSmem {
   int seg_lo[2][2 * kTailSegs + 2];       // start of each subset (relative), +1 sentinel
   int seg_coord[kTailSegs], seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
   uint32_t seg_prefix[kTailSegs];
+  double vpart[4 * 8 * 64];                // partial sums of the variance stage ([ng][8][D])
+  double vout[4 * 64];                     // means / variances ([ng][D])
   double best[kTailSegs][4];
   int arg[kTailSegs][4];
   int warp_tot[32];
@@ -357,11 +383,12 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
           }
         }
         __syncthreads();
+        staged_variances(stage, D, ng,
+                         [&](int gi) { const int sz = slo[g0 + gi + 1] - slo[g0 + gi]; return sz > c ? min(D, sz) : 0; },
+                         sm.vpart, sm.vout, tid, nt);
         for (int task = tid; task < ng * D; task += nt) {
           const int gi = task / D, t = task % D, g = g0 + gi;
-          const int sz = slo[g + 1] - slo[g];
-          double v = -1.0;
-          if (sz > c) v = staged_variance(stage + gi * D * D, D, t, min(D, sz));
+          double v = sm.vout[task];                    // -1 for a subset that is already final
           // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
           int at = t;
           for (int o = 16; o > 0; o >>= 1) {
