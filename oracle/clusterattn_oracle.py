@@ -140,25 +140,29 @@ def subsample_positions(s, m):
     return (np.arange(m, dtype=np.int64) * s) // m
 
 
-def interleaved_sum(x):
-    """Column sums of x [m, d] in a fixed order: eight partial sums over the rows
-    j = r, r+8, r+16, ... (each taken row after row), combined as
-    ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)).  The paper fixes no summation order; this
-    one is reproducible and lets eight workers share a column."""
-    parts = [np.cumsum(x[r::8], axis=0)[-1] if x[r::8].shape[0] else np.zeros(x.shape[1], F64)
-             for r in range(8)]
+def interleaved_sum32(x):
+    """Column sums of a float32 array x [m, d] in float32, in a fixed order: eight
+    partial sums over the rows j = r, r+8, r+16, ... (each taken row after row),
+    combined as ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)).  Every addition is one
+    IEEE single-precision operation, so any implementation that follows the
+    order gets the same bits."""
+    assert x.dtype == np.float32
+    zero = np.zeros(x.shape[1], np.float32)
+    parts = [np.cumsum(x[r::8], axis=0, dtype=np.float32)[-1] if x[r::8].shape[0] else zero for r in range(8)]
     return ((parts[0] + parts[1]) + (parts[2] + parts[3])) + ((parts[4] + parts[5]) + (parts[6] + parts[7]))
 
 
 def choose_coordinate(sub):
-    """Coordinate of highest variance over the subsample rows `sub` [m, d]
-    (population variance in float64, sums in the order of `interleaved_sum`;
-    lowest coordinate on exact ties)."""
-    sub = np.asarray(sub, F64)
-    m = sub.shape[0]
-    mean = interleaved_sum(sub) / m
+    """Coordinate of highest variance over the subsample rows `sub` [m, d]; lowest
+    coordinate on exact ties.  This estimate only feeds an argmax (a discrete
+    decision), so it is taken in the precision of the coordinates themselves,
+    float32, with a fixed operation order (`interleaved_sum32`; no fused
+    multiply-add): population variance, mean first, then squared deviations."""
+    sub = np.ascontiguousarray(sub, dtype=np.float32)
+    m = np.float32(sub.shape[0])
+    mean = interleaved_sum32(sub) / m
     dev = sub - mean
-    var = interleaved_sum(dev * dev) / m
+    var = interleaved_sum32(dev * dev) / m
     return int(np.argmax(var)), var
 
 

@@ -2,8 +2,8 @@
 // coordinates.
 //
 // A set [lo, lo+s) keeps its rows in ascending original order.  A split
-//   1. takes m = min(d, s) rows at positions floor(j*s/m), sums each coordinate
-//      over them row after row in double (mean, then squared deviations) and
+//   1. takes m = min(d, s) rows at positions floor(j*s/m), estimates the variance
+//      of each coordinate over them in float32 with a fixed operation order and
 //      picks the coordinate of largest variance, lowest index on exact ties;
 //   2. finds, by radix selection on order-preserving 32-bit keys, the L-th
 //      smallest (value, row) along it, L = c * floor((s + c) / (2c));
@@ -59,26 +59,27 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 }
 
 // Variances of all coordinates over subsamples staged in shared memory, `ng` tiles of
-// tile[j*D + t], j < m_g.  Summation order (fixed, so the result is reproducible bit for
-// bit): eight partial sums over the rows j = r, r+8, ... taken row after row, combined
-// as ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)); first the mean, then the squared deviations.
-// part: [ng][8][D] doubles, out: [ng][D] doubles.  Called by all threads of the CTA.
+// tile[j*D + t], j < m_g.  The estimate only feeds an argmax, so it is taken in float32 with
+// a fixed operation order (reproducible bit for bit; every operation rounded on its own, no
+// fused multiply-add): eight partial sums over the rows j = r, r+8, ... taken row after row,
+// combined as ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)); first the mean, then the squared
+// deviations.  part: [ng][8][D] floats, out: [ng][D] floats.  Called by all threads of the CTA.
 template <typename RowsOf>
 __device__ __forceinline__ void staged_variances(const float* tiles, int D, int ng, RowsOf rows_of,
-                                                 double* part, double* out, int tid, int nt) {
+                                                 float* part, float* out, int tid, int nt) {
   for (int pass = 0; pass < 2; ++pass) {
     for (int task = tid; task < ng * 8 * D; task += nt) {
       const int gi = task / (8 * D), r = (task / D) % 8, t = task % D;
       const int m = rows_of(gi);
       const float* tile = tiles + gi * D * D;
-      double acc = 0.0;
+      float acc = 0.f;
       if (pass == 0) {
-        for (int j = r; j < m; j += 8) acc = __dadd_rn(acc, (double)tile[j * D + t]);
+        for (int j = r; j < m; j += 8) acc = __fadd_rn(acc, tile[j * D + t]);
       } else {
-        const double mean = out[gi * D + t];
+        const float mean = out[gi * D + t];
         for (int j = r; j < m; j += 8) {
-          const double dev = __dsub_rn((double)tile[j * D + t], mean);
-          acc = __dadd_rn(acc, __dmul_rn(dev, dev));
+          const float dev = __fsub_rn(tile[j * D + t], mean);
+          acc = __fadd_rn(acc, __fmul_rn(dev, dev));
         }
       }
       part[(gi * 8 + r) * D + t] = acc;
@@ -86,11 +87,11 @@ __device__ __forceinline__ void staged_variances(const float* tiles, int D, int 
     __syncthreads();
     for (int task = tid; task < ng * D; task += nt) {
       const int gi = task / D, t = task % D;
-      const double* p = part + gi * 8 * D + t;
-      const double tot = __dadd_rn(__dadd_rn(__dadd_rn(p[0], p[D]), __dadd_rn(p[2 * D], p[3 * D])),
-                                   __dadd_rn(__dadd_rn(p[4 * D], p[5 * D]), __dadd_rn(p[6 * D], p[7 * D])));
+      const float* p = part + gi * 8 * D + t;
+      const float tot = __fadd_rn(__fadd_rn(__fadd_rn(p[0], p[D]), __fadd_rn(p[2 * D], p[3 * D])),
+                                  __fadd_rn(__fadd_rn(p[4 * D], p[5 * D]), __fadd_rn(p[6 * D], p[7 * D])));
       const int m = rows_of(gi);
-      out[task] = m > 0 ? tot / (double)m : -1.0;
+      out[task] = m > 0 ? __fdiv_rn(tot, (float)m) : -1.0f;
     }
     __syncthreads();
   }
@@ -121,8 +122,8 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   int32_t* s_rows = reinterpret_cast<int32_t*>(s_keys + prm.smem_rows);      // [smem_rows]
   __shared__ int s_hist[256];
   __shared__ int s_total[256];
-  __shared__ double s_var[128];
-  __shared__ double s_part[8 * 128];
+  __shared__ float s_var[128];
+  __shared__ float s_part[8 * 128];
   __shared__ int s_sub[128];
   __shared__ int s_warp[2 * 32];
   __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank, 3: chunk total
@@ -164,13 +165,13 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   __syncthreads();
   staged_variances(reinterpret_cast<const float*>(smem_raw), D, 1, [&](int) { return m; }, s_part, s_var, tid, nt);
   if (warp == 0) {
-    double best = -1.0; int arg = 0;
+    float best = -1.0f; int arg = 0;
     for (int t = lane; t < D; t += 32) {
-      const double v = s_var[t];
+      const float v = s_var[t];
       if (v > best) { best = v; arg = t; }
     }
     for (int o = 16; o > 0; o >>= 1) {
-      const double ob = __shfl_xor_sync(0xffffffffu, best, o);
+      const float ob = __shfl_xor_sync(0xffffffffu, best, o);
       const int oa = __shfl_xor_sync(0xffffffffu, arg, o);
       if (ob > best || (ob == best && oa < arg)) { best = ob; arg = oa; }
     }
@@ -325,9 +326,9 @@ struct TailSmem {
   int seg_lo[2][2 * kTailSegs + 2];       // start of each subset (relative), +1 sentinel
   int seg_coord[kTailSegs], seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
   uint32_t seg_prefix[kTailSegs];
-  double vpart[4 * 8 * 64];                // partial sums of the variance stage ([ng][8][D])
-  double vout[4 * 64];                     // means / variances ([ng][D])
-  double best[kTailSegs][4];
+  float vpart[4 * 8 * 64];                // partial sums of the variance stage ([ng][8][D])
+  float vout[4 * 64];                     // means / variances ([ng][D])
+  float best[kTailSegs][4];
   int arg[kTailSegs][4];
   int warp_tot[32];
   int nseg[2];
@@ -388,11 +389,11 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
                          sm.vpart, sm.vout, tid, nt);
         for (int task = tid; task < ng * D; task += nt) {
           const int gi = task / D, t = task % D, g = g0 + gi;
-          double v = sm.vout[task];                    // -1 for a subset that is already final
+          float v = sm.vout[task];                     // -1 for a subset that is already final
           // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
           int at = t;
           for (int o = 16; o > 0; o >>= 1) {
-            const double ov = __shfl_xor_sync(0xffffffffu, v, o);
+            const float ov = __shfl_xor_sync(0xffffffffu, v, o);
             const int oa = __shfl_xor_sync(0xffffffffu, at, o);
             if (ov > v || (ov == v && oa < at)) { v = ov; at = oa; }
           }
@@ -403,7 +404,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
     }
     if (tid < nseg) {
       const int a = slo[tid], sz = slo[tid + 1] - a;
-      double v = sm.best[tid][0]; int at = sm.arg[tid][0];
+      float v = sm.best[tid][0]; int at = sm.arg[tid][0];
       for (int w = 1; w < wps; ++w)
         if (sm.best[tid][w] > v) { v = sm.best[tid][w]; at = sm.arg[tid][w]; }   // later warps hold higher coordinates
       sm.seg_coord[tid] = at;
