@@ -97,6 +97,13 @@ __device__ __forceinline__ void staged_variances(const float* tiles, int D, int 
   }
 }
 
+// 16-byte asynchronous copy global -> shared (no registers held while in flight)
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
+  const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gmem_src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 struct SplitSide {
   const float* Y;          // [P][n][D]
   const int32_t* perm_in;  // [P][n] or null (identity)
@@ -160,7 +167,8 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
     float4* stage4 = reinterpret_cast<float4*>(smem_raw);
     const int q = D / 4;
     for (int e = tid; e < m * q; e += nt)
-      stage4[e] = __ldg(reinterpret_cast<const float4*>(Y + (size_t)s_sub[e / q] * D) + (e % q));
+      cp_async16(stage4 + e, reinterpret_cast<const float4*>(Y + (size_t)s_sub[e / q] * D) + (e % q));
+    cp_async_wait_all();
   }
   __syncthreads();
   staged_variances(reinterpret_cast<const float*>(smem_raw), D, 1, [&](int) { return m; }, s_part, s_var, tid, nt);
@@ -380,9 +388,10 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
           const int m = min(D, sz);
           if (sz > c && j < m) {
             const int row = rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)];
-            reinterpret_cast<float4*>(stage)[e] = __ldg(reinterpret_cast<const float4*>(Y + (size_t)row * D) + c4);
+            cp_async16(reinterpret_cast<float4*>(stage) + e, reinterpret_cast<const float4*>(Y + (size_t)row * D) + c4);
           }
         }
+        cp_async_wait_all();
         __syncthreads();
         staged_variances(stage, D, ng,
                          [&](int gi) { const int sz = slo[g0 + gi + 1] - slo[g0 + gi]; return sz > c ? min(D, sz) : 0; },
