@@ -64,8 +64,8 @@ __device__ __forceinline__ uint32_t order_key(float x) {
 // fused multiply-add): eight partial sums over the rows j = r, r+8, ... taken row after row,
 // combined as ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)); first the mean, then the squared
 // deviations.  part: [ng][8][D] floats, out: [ng][D] floats.  Called by all threads of the CTA.
-template <typename RowsOf>
-__device__ __forceinline__ void staged_variances(const float* tiles, int D, int ng, RowsOf rows_of,
+template <int D, typename RowsOf>
+__device__ __forceinline__ void staged_variances(const float* tiles, int ng, RowsOf rows_of,
                                                  float* part, float* out, int tid, int nt) {
   for (int pass = 0; pass < 2; ++pass) {
     for (int task = tid; task < ng * 8 * D; task += nt) {
@@ -120,6 +120,7 @@ struct SplitParams {
 // ---------------------------------------------------------------------------
 // One level of the large sets.  grid.x = slots * cluster size.
 // ---------------------------------------------------------------------------
+template <int D>
 __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitParams prm) {
   cg::cluster_group cluster = cg::this_cluster();
   const int csize = (int)cluster.num_blocks();
@@ -143,7 +144,6 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   const SegmentRef seg = locate_segment(sd.n, sd.c, prm.level, blockIdx.x / csize);
   if (!seg.active) return;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
-  const int D = prm.D;
   const float* Y = sd.Y + (size_t)p * sd.n * D;
   const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
   int32_t* pout = sd.perm_out + (size_t)p * sd.n;
@@ -165,13 +165,13 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   {
     // the subsample rows are staged by all threads (16-byte loads in flight together)
     float4* stage4 = reinterpret_cast<float4*>(smem_raw);
-    const int q = D / 4;
+    constexpr int q = D / 4;
     for (int e = tid; e < m * q; e += nt)
       cp_async16(stage4 + e, reinterpret_cast<const float4*>(Y + (size_t)s_sub[e / q] * D) + (e % q));
     cp_async_wait_all();
   }
   __syncthreads();
-  staged_variances(reinterpret_cast<const float*>(smem_raw), D, 1, [&](int) { return m; }, s_part, s_var, tid, nt);
+  staged_variances<D>(reinterpret_cast<const float*>(smem_raw), 1, [&](int) { return m; }, s_part, s_var, tid, nt);
   if (warp == 0) {
     float best = -1.0f; int arg = 0;
     for (int t = lane; t < D; t += 32) {
@@ -335,7 +335,8 @@ struct TailSmem {
   int seg_coord[kTailSegs], seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
   uint32_t seg_prefix[kTailSegs];
   float vpart[4 * 8 * 64];                // partial sums of the variance stage ([ng][8][D])
-  float vout[4 * 64];                     // means / variances ([ng][D])
+  float vout[4 * 64];
+  int sub_rows[4 * 64];                    // subsample rows of the subsets being staged                     // means / variances ([ng][D])
   float best[kTailSegs][4];
   int arg[kTailSegs][4];
   int warp_tot[32];
@@ -343,6 +344,7 @@ struct TailSmem {
   int more;
 };
 
+template <int D>
 __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitParams prm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   TailSmem& sm = *reinterpret_cast<TailSmem*>(smem_raw);
@@ -355,7 +357,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
   if (!root.active) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   constexpr int nt = kSplitThreads;
-  const int D = prm.D, c = sd.c;
+  const int c = sd.c;
   const float* Y = sd.Y + (size_t)p * sd.n * D;
   const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
   int32_t* pout = sd.perm_out + (size_t)p * sd.n;
@@ -366,7 +368,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
   __syncthreads();
 
   int cur = 0;
-  const int wps = D / 32;                            // warps per (subset, all coordinates)
+  constexpr int wps = D / 32;                            // warps per (subset, all coordinates)
   while (sm.more) {
     const int nseg = sm.nseg[cur];
     const int* slo = sm.seg_lo[cur];
@@ -378,22 +380,26 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
     // occupy later in the level.
     {
       float* stage = reinterpret_cast<float*>(sm.keys);
-      const int per_group = (16384 / (D * D)) > 0 ? 16384 / (D * D) : 1;     // 4 (d=64) or 1 (d=128)
-      const int q = D / 4;
+      constexpr int per_group = (16384 / (D * D)) > 0 ? 16384 / (D * D) : 1;     // 4 (d=64) or 1 (d=128)
+      constexpr int q = D / 4;
       for (int g0 = 0; g0 < nseg; g0 += per_group) {
         const int ng = min(per_group, nseg - g0);
-        for (int e = tid; e < ng * D * q; e += nt) {
-          const int gi = e / (D * q), j = (e / q) % D, c4 = e % q;
+        // rows of the subsamples (one division per row), then the tiles by asynchronous copies
+        for (int e = tid; e < ng * D; e += nt) {
+          const int gi = e / D, j = e % D;
           const int a = slo[g0 + gi], sz = slo[g0 + gi + 1] - a;
           const int m = min(D, sz);
-          if (sz > c && j < m) {
-            const int row = rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)];
-            cp_async16(reinterpret_cast<float4*>(stage) + e, reinterpret_cast<const float4*>(Y + (size_t)row * D) + c4);
-          }
+          sm.sub_rows[e] = (sz > c && j < m) ? rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)] : -1;
+        }
+        __syncthreads();
+        for (int e = tid; e < ng * D * q; e += nt) {
+          const int row = sm.sub_rows[e / q];
+          if (row >= 0)
+            cp_async16(reinterpret_cast<float4*>(stage) + e, reinterpret_cast<const float4*>(Y + (size_t)row * D) + (e % q));
         }
         cp_async_wait_all();
         __syncthreads();
-        staged_variances(stage, D, ng,
+        staged_variances<D>(stage, ng,
                          [&](int gi) { const int sz = slo[g0 + gi + 1] - slo[g0 + gi]; return sz > c ? min(D, sz) : 0; },
                          sm.vpart, sm.vout, tid, nt);
         for (int task = tid; task < ng * D; task += nt) {
@@ -589,9 +595,10 @@ static int tail_level_for(int n, int c) {
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
                  int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st) {
-  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(split_level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         kSmemRowsMax * 8));
-  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(split_tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  auto level_kernel = D == 64 ? split_level_kernel<64> : split_level_kernel<128>;
+  auto tail_kernel = D == 64 ? split_tail_kernel<64> : split_tail_kernel<128>;
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRowsMax * 8));
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(TailSmem)));
   const int tail_q = tail_level_for(n_q, c_q), tail_k = tail_level_for(n_k, c_k);
   const int top_levels = tail_q > tail_k ? tail_q : tail_k;
@@ -642,14 +649,14 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr; cfg.numAttrs = 1;
-    CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, split_level_kernel, prm));
+    CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, level_kernel, prm));
     CA_LAUNCH_CHECK();
   }
   fill(top_levels);       // any level >= both tails selects the tail buffers
   prm.level = top_levels;
   prm.smem_rows = 0;
   const int slots = 1 << (tail_q > tail_k ? tail_q : tail_k);
-  split_tail_kernel<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(TailSmem), st>>>(prm);
+  tail_kernel<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(TailSmem), st>>>(prm);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
