@@ -362,32 +362,72 @@ __global__ void covariance_kernel(const double* __restrict__ gram, const double*
 }
 
 // C[p] = alpha * op(A[p]) * B[p], op = transpose if trans_a; optional fp32 copy.
-__global__ void small_matmul_kernel(const double* __restrict__ A, const double* __restrict__ B, int D,
-                                    double alpha, int trans_a, double* __restrict__ C,
-                                    float* __restrict__ C32) {
-  const int p = blockIdx.y;
+// Operands are double in memory; the products are formed in float (FP64 throughput of the
+// CUDA cores is low on this part, and the results only feed fp32 projections).  One CTA of
+// 256 threads per 64 x 64 tile of C, 4 x 4 outputs per thread, 16-deep slices in shared memory.
+__global__ void __launch_bounds__(256) small_matmul_kernel(const double* __restrict__ A,
+                                                           const double* __restrict__ B, int D, double alpha,
+                                                           int trans_a, double* __restrict__ C,
+                                                           float* __restrict__ C32) {
+  __shared__ float As[16][64 + 4];     // As[k][i]
+  __shared__ float Bs[16][64 + 4];     // Bs[k][j]
+  const int p = blockIdx.z;
   const double* Ap = A + (size_t)p * D * D;
   const double* Bp = B + (size_t)p * D * D;
-  const int e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e >= D * D) return;
-  const int i = e / D, j = e % D;
-  double s = 0.0;
-  if (trans_a) for (int k = 0; k < D; ++k) s += Ap[k * D + i] * Bp[k * D + j];
-  else for (int k = 0; k < D; ++k) s += Ap[i * D + k] * Bp[k * D + j];
-  s *= alpha;
-  C[(size_t)p * D * D + e] = s;
-  if (C32) C32[(size_t)p * D * D + e] = (float)s;
+  const int i0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+  const int ti = threadIdx.x / 16, tj = threadIdx.x % 16;
+  float acc[4][4];
+#pragma unroll
+  for (int a = 0; a < 4; ++a)
+#pragma unroll
+    for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+  for (int k0 = 0; k0 < D; k0 += 16) {
+    for (int e = threadIdx.x; e < 16 * 64; e += 256) {
+      const int k = e / 64, x = e % 64;
+      As[k][x] = (float)(trans_a ? Ap[(size_t)(k0 + k) * D + i0 + x] : Ap[(size_t)(i0 + x) * D + k0 + k]);
+      Bs[k][x] = (float)Bp[(size_t)(k0 + k) * D + j0 + x];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < 16; ++k) {
+      float a[4], b[4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x) { a[x] = As[k][ti * 4 + x]; b[x] = Bs[k][tj * 4 + x]; }
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) acc[x][y] = fmaf(a[x], b[y], acc[x][y]);
+    }
+    __syncthreads();
+  }
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) {
+      const size_t o = (size_t)p * D * D + (size_t)(i0 + ti * 4 + x) * D + j0 + tj * 4 + y;
+      const double v = alpha * (double)acc[x][y];
+      C[o] = v;
+      if (C32) C32[o] = (float)v;
+    }
 }
 
-// bias[p][j] = - sum_i (sum[p][i] / n) * W[p][i][j]
+// bias[p][j] = - sum_i (sum[p][i] / n) * W[p][i][j]   (float accumulation, four independent chains)
 __global__ void bias_kernel(const double* __restrict__ sum, const double* __restrict__ W, int D, double n,
                             float* __restrict__ bias) {
   const int p = blockIdx.x;
   const int j = threadIdx.x;
   if (j >= D) return;
-  double s = 0.0;
-  for (int i = 0; i < D; ++i) s += (sum[(size_t)p * D + i] / n) * W[(size_t)p * D * D + i * D + j];
-  bias[(size_t)p * D + j] = (float)(-s);
+  const float inv_n = (float)(1.0 / n);
+  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+  const double* Wp = W + (size_t)p * D * D + j;
+  const double* sp = sum + (size_t)p * D;
+  for (int i = 0; i < D; i += 4) {
+    s0 = fmaf((float)sp[i] * inv_n, (float)Wp[(size_t)i * D], s0);
+    s1 = fmaf((float)sp[i + 1] * inv_n, (float)Wp[(size_t)(i + 1) * D], s1);
+    s2 = fmaf((float)sp[i + 2] * inv_n, (float)Wp[(size_t)(i + 2) * D], s2);
+    s3 = fmaf((float)sp[i + 3] * inv_n, (float)Wp[(size_t)(i + 3) * D], s3);
+  }
+  bias[(size_t)p * D + j] = -((s0 + s1) + (s2 + s3));
 }
 
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
@@ -405,7 +445,7 @@ int launch_covariance(const double* gram, const double* sum, int P, int D, int n
 }
 int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
                         double* C, float* C32, cudaStream_t st) {
-  small_matmul_kernel<<<dim3(ceil_div(D * D, 256), P), 256, 0, st>>>(A, B, D, alpha, trans_a, C, C32);
+  small_matmul_kernel<<<dim3(D / 64, D / 64, P), 256, 0, st>>>(A, B, D, alpha, trans_a, C, C32);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
