@@ -214,8 +214,13 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
       const uint32_t k = ok ? keys[i] : 0u;
       const bool cand = ok && ((k & mask) == prefix);
       const int bin = cand ? (int)((k >> shift) & 255u) : -1;
-      const unsigned peers = __match_any_sync(0xffffffffu, bin);   // one atomic per distinct bin
-      if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+      if (shift == 24) {
+        // leading digit: few distinct values in a warp (sign and exponent bits), one atomic per value
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+      } else if (cand) {
+        atomicAdd(&s_hist[bin], 1);                 // lower digits are spread out: plain atomics
+      }
     }
     if (csize > 1) {
       cluster.sync();                                // every slice has counted
@@ -460,8 +465,12 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
         const uint32_t k = live ? sm.keys[tid + u * nt] : 0u;
         const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
         const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&(&sm.hist[0][0])[bin], __popc(peers));
+        if (shift == 24) {
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&(&sm.hist[0][0])[bin], __popc(peers));
+        } else if (cand) {
+          atomicAdd(&(&sm.hist[0][0])[bin], 1);
+        }
       }
       __syncthreads();
       for (int g = warp; g < nseg; g += nt / 32) {
