@@ -194,10 +194,26 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   const int cs = c1 - c0;
   const bool in_smem = cs <= prm.smem_rows;
   uint32_t* keys = in_smem ? s_keys : sd.keybuf + (size_t)p * sd.n + lo + c0;
-  for (int i = tid; i < cs; i += nt) {
-    const int row = pin ? pin[lo + c0 + i] : lo + c0 + i;
-    keys[i] = order_key(__ldg(Y + (size_t)row * D + coord));
-    if (in_smem) s_rows[i] = row;
+  // gathers in batches of eight: the row indices first, then the coordinates, so that the
+  // memory latencies of a batch overlap
+  for (int i0 = tid; i0 < cs; i0 += 8 * nt) {
+    int row[8];
+    float val[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * nt;
+      row[u] = (i < cs) ? (pin ? __ldg(pin + lo + c0 + i) : lo + c0 + i) : 0;
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) val[u] = __ldg(Y + (size_t)row[u] * D + coord);
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+      const int i = i0 + u * nt;
+      if (i < cs) {
+        keys[i] = order_key(val[u]);
+        if (in_smem) s_rows[i] = row[u];
+      }
+    }
   }
   __syncthreads();
 
@@ -262,68 +278,57 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   const uint32_t thr = prefix;
   const int eq_left = remaining;        // how many rows equal to the threshold go down
 
-  // ---- 3. stable two-sided partition.  Offsets of this slice = totals of the earlier slices.
-  int less_before = 0, eq_before = 0;
-  if (csize > 1) {
-    int nl = 0, ne = 0;
-    for (int i = tid; i < cs; i += nt) {
-      const uint32_t k = keys[i];
-      nl += k < thr;
-      ne += k == thr;
-    }
-    for (int o = 16; o > 0; o >>= 1) {
-      nl += __shfl_xor_sync(0xffffffffu, nl, o);
-      ne += __shfl_xor_sync(0xffffffffu, ne, o);
-    }
-    if (tid == 0) { s_counts[0] = 0; s_counts[1] = 0; }
-    __syncthreads();
-    if (lane == 0) { atomicAdd(&s_counts[0], nl); atomicAdd(&s_counts[1], ne); }
-    cluster.sync();
-    for (int r = 0; r < crank; ++r) {
-      const int* rc = cluster.map_shared_rank(s_counts, r);
-      less_before += rc[0];
-      eq_before += rc[1];
-    }
+  // ---- 3. stable two-sided partition.  Every warp owns a contiguous run of the slice and walks
+  // it 32 positions at a time with ballots; offsets = totals of the earlier slices and warps.
+  const int nwarps = nt >> 5;
+  const int run = ((cs + nwarps - 1) / nwarps + 31) & ~31;       // positions per warp (multiple of 32)
+  const int w0 = min(cs, warp * run), w1 = min(cs, w0 + run);
+  int nl = 0, ne = 0;
+  for (int i0 = w0; i0 < w1; i0 += 32) {
+    const int i = i0 + lane;
+    const uint32_t k = (i < w1) ? keys[i] : 0xffffffffu;
+    nl += __popc(__ballot_sync(0xffffffffu, i < w1 && k < thr));
+    ne += __popc(__ballot_sync(0xffffffffu, i < w1 && k == thr));
   }
-  for (int i0 = 0; i0 < cs; i0 += nt) {
-    const int i = i0 + tid;
-    const bool ok = i < cs;
-    const uint32_t k = ok ? keys[i] : 0xffffffffu;
-    const int is_less = (ok && k < thr) ? 1 : 0;
-    const int is_eq = (ok && k == thr) ? 1 : 0;
-    const int packed = is_less | (is_eq << 16);
-    int incl = packed;
+  if (lane == 0) s_warp[warp] = nl | (ne << 16);       // a warp run holds fewer than 65536 positions
+  __syncthreads();
+  if (warp == 0) {
+    const int v = (lane < nwarps) ? s_warp[lane] : 0;
+    int vl = v & 0xffff, ve = v >> 16;
+    int il = vl, ie = ve;
     for (int o = 1; o < 32; o <<= 1) {
-      const int v = __shfl_up_sync(0xffffffffu, incl, o);
-      if (lane >= o) incl += v;
+      const int a = __shfl_up_sync(0xffffffffu, il, o), b = __shfl_up_sync(0xffffffffu, ie, o);
+      if (lane >= o) { il += a; ie += b; }
     }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-      const int w = (lane < (nt >> 5)) ? s_warp[lane] : 0;
-      int wi = w;
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, wi, o);
-        if (lane >= o) wi += v;
-      }
-      s_warp[32 + lane] = wi - w;                  // exclusive offset of each warp
-      if (lane == 31) s_scalar[3] = wi;            // chunk total
-    }
-    __syncthreads();
-    const int excl = incl - packed + s_warp[32 + warp];
-    const int less_here = less_before + (excl & 0xffff);
-    const int eq_here = eq_before + (excl >> 16);
+    s_hist[lane] = il - vl;                            // exclusive offsets per warp (s_hist is free now)
+    s_hist[32 + lane] = ie - ve;
+    if (lane == 31) { s_counts[0] = il; s_counts[1] = ie; }
+  }
+  if (csize > 1) cluster.sync(); else __syncthreads();
+  int less_before = s_hist[warp], eq_before = s_hist[32 + warp];
+  for (int r = 0; r < crank; ++r) {                     // totals of the earlier slices of the cluster
+    const int* rc = cluster.map_shared_rank(s_counts, r);
+    less_before += rc[0];
+    eq_before += rc[1];
+  }
+  const unsigned lt_mask = (1u << lane) - 1u;
+  for (int i0 = w0; i0 < w1; i0 += 32) {
+    const int i = i0 + lane;
+    const bool ok = i < w1;
+    const uint32_t k = ok ? keys[i] : 0xffffffffu;
+    const bool is_less = ok && k < thr, is_eq = ok && k == thr;
+    const unsigned bl = __ballot_sync(0xffffffffu, is_less), be = __ballot_sync(0xffffffffu, is_eq);
     if (ok) {
+      const int less_here = less_before + __popc(bl & lt_mask);
+      const int eq_here = eq_before + __popc(be & lt_mask);
       const bool down = is_less || (is_eq && eq_here < eq_left);
       const int down_before = less_here + min(eq_here, eq_left);
       const int row = in_smem ? s_rows[i] : (pin ? pin[lo + c0 + i] : lo + c0 + i);
       const int dst = down ? lo + down_before : lo + L + (c0 + i - down_before);
       pout[dst] = row;
     }
-    const int total = s_scalar[3];
-    less_before += total & 0xffff;
-    eq_before += total >> 16;
-    __syncthreads();
+    less_before += __popc(bl);
+    eq_before += __popc(be);
   }
   if (csize > 1) cluster.sync();                     // keep shared memory alive for the peers' reads
 }
