@@ -99,7 +99,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = blockIdx.y;
-  const int tiles_per_qc = prm.c_q / kTile;
+  // a query cluster of 256 rows takes two CTAs; one of 64 rows fills the upper half of a tile
+  // (the lower half is zeros and the warps that own those rows only keep the barriers going)
+  const int tiles_per_qc = prm.c_q >= kTile ? prm.c_q / kTile : 1;
+  const int q_rows = prm.c_q >= kTile ? kTile : prm.c_q;
   const int qc = blockIdx.x / tiles_per_qc, half = blockIdx.x % tiles_per_qc;
   const int32_t* sel = prm.block_idx + ((size_t)p * prm.n_qc + qc) * prm.keep;
   const int sel_tiles = selected_tiles(prm.keep, prm.c_k);
@@ -118,6 +121,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     *abort_flag = 0;
     fence_mbar_init();
   }
+  if (q_rows < kTile) {
+    // rows [q_rows, 128) of every Q panel: zeros (read by the tensor core through the async proxy)
+    for (int e = tid; e < C::PANELS * (kTile - q_rows) * 8; e += kTcThreads) {
+      const int pn = e / ((kTile - q_rows) * 8), rem = e % ((kTile - q_rows) * 8);
+      *reinterpret_cast<uint4*>(smem + C::OFF_Q + pn * C::PANEL_BYTES + q_rows * 128 + rem * 16) = make_uint4(0u, 0u, 0u, 0u);
+    }
+    fence_proxy_async();
+  }
   if (warp == 1) {                       // this warp owns the TMEM allocation
     tmem_alloc(smem_u32(tmem_slot), kTmemCols);
     tmem_relinquish();
@@ -133,7 +144,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (lane == 0) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
       const int q_row = (p * prm.n_qc + qc) * prm.c_q + half * kTile;
-      mbar_expect_tx(b_q_full, C::TILE_BYTES);
+      mbar_expect_tx(b_q_full, C::PANELS * q_rows * 128);
       for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(s_q + pn * C::PANEL_BYTES, &tm_q, pn * 64, q_row, b_q_full);
       bool ok = true;
       auto load_rows = [&](uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
@@ -283,6 +294,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(b), (u >> 1) & 1, abort_flag, prm.status));
       if (!ok) break;
       tc_fence_after();
+      if (quarter * 32 >= q_rows) {          // this warp's rows are padding of a 64-row query cluster
+        tc_fence_before();
+        mbar_arrive(b_p_ready(b));
+        continue;
+      }
       // ---- pass 1: row maximum over the 64 columns
       uint32_t ra[32], rb[32];
       float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -379,7 +395,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     tc_fence_after();
     if (ok) {                                          // warp-uniform: TMEM loads are warp-collective
       const int pos = qc * prm.c_q + half * kTile + row;
-      const bool live = pos < prm.n_q;                 // rows of the padding are not written
+      const bool live = row < q_rows && pos < prm.n_q;  // rows of the padding are not written
       const int orig = live ? prm.perm_q[(size_t)p * prm.n_q + pos] : 0;
       const float inv = 1.f / l_run;
       __nv_bfloat16* out = prm.O + ((size_t)p * prm.n_q + orig) * D;
@@ -469,7 +485,7 @@ static bool make_map(CUtensorMap* map, const void* base, size_t rows, int D, int
 
 bool attn_tc_supported(const ca_problem_t& pr) {
   if (pr.dtype != CA_DTYPE_BF16 || (pr.flags & CA_ATTN_FP32)) return false;
-  if (pr.cluster_q != 128 && pr.cluster_q != 256) return false;
+  if (pr.cluster_q != 64 && pr.cluster_q != 128 && pr.cluster_q != 256) return false;
   if (pr.cluster_k < 16 || pr.cluster_k > 256) return false;
   const int n_kc = ceil_div(pr.n_k, pr.cluster_k);
   if ((n_kc + 31) / 32 * 4 > 16384) return false;          // selected-cluster bitmap in shared memory
@@ -511,7 +527,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   }
   CUtensorMap maps[5];
   const int kbox = pr.cluster_k < kTile ? pr.cluster_k : kTile;
-  bool ok = make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, kTile) &&
+  bool ok = make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, pr.cluster_q < kTile ? pr.cluster_q : kTile) &&
             make_map(&maps[1], Kp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
             make_map(&maps[2], Vp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
             make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kTile) &&
@@ -524,7 +540,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   prm.n_qc = n_qc; prm.n_kc = n_kc; prm.cen_tiles = cen_tiles; prm.compensate = pr.compensate;
   prm.bitmap_words = (cen_tiles * kHalf + 31) / 32;
   prm.scale_log2 = scale * 1.4426950408889634f;
-  dim3 grid(n_qc * (pr.cluster_q / kTile), P);
+  dim3 grid(n_qc * (pr.cluster_q >= kTile ? pr.cluster_q / kTile : 1), P);
   if (D == 64) return launch_tc_d<64>(maps, prm, grid, st);
   return launch_tc_d<128>(maps, prm, grid, st);
 }

@@ -178,37 +178,38 @@ def test_select_blocks_exact(H, n_qc, n_kc, d, keep):
 # ----------------------------------------------------------------------------
 # Attention on the oracle's permutation and block lists.
 # ----------------------------------------------------------------------------
-def attention_case(w, H, keep, compensate, flags=0, perm_seed=None):
+def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=None):
     Q, K, V = inputs.generate(w.scaled(heads=H))
-    p = binding.problem_from_workload(w, heads=H, keep=keep, compensate=compensate, flags=flags)
+    c_q, c_k = w.cluster, (cluster_k or w.cluster)
+    p = binding.problem_from_workload(w, heads=H, keep=keep, compensate=compensate, flags=flags,
+                                      cluster_q=c_q, cluster_k=c_k)
     plan = binding.Plan(p, DEV)
-    c = w.cluster
     refs = []
     arrs = {k: [] for k in ("perm_q", "Qp", "Kp", "Vp", "ck", "cv", "count_k", "idx")}
     for h in range(H):
         if perm_seed is None:
-            cl = orc.cluster_qk(Q[h], K[h], V[h], c, c)
+            cl = orc.cluster_qk(Q[h], K[h], V[h], c_q, c_k)
         else:                                # any valid permutation must work
             r = np.random.default_rng(perm_seed + h)
             pq, pk = r.permutation(w.n_q), r.permutation(w.n_k)
-            cq_, nq_ = orc.centroids(Q[h], pq, c)
-            ck_, nk_ = orc.centroids(K[h], pk, c)
-            cv_, _ = orc.centroids(V[h], pk, c)
+            cq_, nq_ = orc.centroids(Q[h], pq, c_q)
+            ck_, nk_ = orc.centroids(K[h], pk, c_k)
+            cv_, _ = orc.centroids(V[h], pk, c_k)
             cl = dict(perm_q=pq, perm_k=pk, cq=cq_, ck=ck_, cv=cv_, count_q=nq_, count_k=nk_)
         idx = orc.select_blocks(cl["cq"], cl["ck"], keep)
         ck32, cv32 = cl["ck"].astype(np.float32), cl["cv"].astype(np.float32)
-        o, lse = orc.cluster_attention(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c, c, idx, compensate,
+        o, lse = orc.cluster_attention(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c_q, c_k, idx, compensate,
                                        ck=ck32, cv=cv32, count_k=cl["count_k"])
         refs.append((o, lse))
 
-        def pad(x, perm, n):
+        def pad(x, perm, n, c):
             out = np.zeros((-(-n // c) * c, x.shape[1]), np.float32)
             out[:n] = x[perm]
             return out
         arrs["perm_q"].append(cl["perm_q"].astype(np.int32))
-        arrs["Qp"].append(pad(Q[h], cl["perm_q"], w.n_q))
-        arrs["Kp"].append(pad(K[h], cl["perm_k"], w.n_k))
-        arrs["Vp"].append(pad(V[h], cl["perm_k"], w.n_k))
+        arrs["Qp"].append(pad(Q[h], cl["perm_q"], w.n_q, c_q))
+        arrs["Kp"].append(pad(K[h], cl["perm_k"], w.n_k, c_k))
+        arrs["Vp"].append(pad(V[h], cl["perm_k"], w.n_k, c_k))
         arrs["ck"].append(ck32)
         arrs["cv"].append(cv32)
         arrs["count_k"].append(cl["count_k"].astype(np.int32))
@@ -248,12 +249,21 @@ def bf16_close(O, o_ref):
     ("tabular", 1024, 4096, 4, True, 0), ("tabular", 1024, 4096, 4, False, 0),
     ("video480", 1000, 1000, 2, True, 0), ("sweep", 2048, 2048, 16, True, 0),
     ("tabular", 512, 2048, 4, True, binding.CA_ATTN_FP32),
+    ("sweep64", 1100, 3000, 9, True, 0),          # 64-row clusters on both sides, short last clusters
+    ("sweep256", 1024, 2100, 3, True, 0),         # 256-row clusters: two CTAs per query cluster
+    ("sweep32k", 640, 1000, 11, False, 0),        # 32-row key clusters packed four to a tile
 ])
 def test_attention_bf16(name, n_q, n_k, keep, compensate, flags):
-    w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k)
+    variants = {"sweep64": ("sweep", 64, 64), "sweep256": ("sweep", 256, 256), "sweep32k": ("sweep", 128, 32)}
+    cluster_k = None
+    if name in variants:
+        name, cq_, cluster_k = variants[name]
+        w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k, cluster=cq_)
+    else:
+        w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k)
     if w.kind == "video":
         w = w.scaled(grid=(5, 10, 20))
-    O, lse, refs = attention_case(w, 2, keep, compensate, flags=flags)
+    O, lse, refs = attention_case(w, 2, keep, compensate, flags=flags, cluster_k=cluster_k)
     for h, (o_ref, lse_ref) in enumerate(refs):
         assert bf16_close(O[h], o_ref), (np.abs(O[h] - o_ref).max(),
                                          np.linalg.norm(O[h] - o_ref) / np.linalg.norm(o_ref))
