@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="sweep workload: cluster size x kept fraction x compensation, one JSON line with all points")
     return ap.parse_args()
 
 
@@ -367,8 +369,78 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Cluster size 64/128/256 x kept fraction 1/32..1/2 x compensation on/off on the sweep
+    workload (16 heads, d=128, 131,072 tokens), plus dense attention on the same tensors."""
+    import torch
+
+    from paper_2608_26965_b200 import binding, build, inputs
+
+    build.build()
+    binding.load_library()
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    base = inputs.WORKLOADS["sweep"]
+    if args.heads:
+        base = base.scaled(heads=args.heads)
+    Qh, Kh, Vh = inputs.generate(base)
+    dt = torch.bfloat16
+    Q, K, V = (torch.from_numpy(a[None]).to(dt).to(dev) for a in (Qh, Kh, Vh))
+    stream = torch.cuda.current_stream()
+    peaks, peak_kind = load_peaks()
+
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        for _ in range(reps):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    with torch.no_grad():
+        dense_ms = timed(lambda: torch.nn.functional.scaled_dot_product_attention(Q, K, V), 3)
+    points = []
+    for c in (64, 128, 256):
+        n_kc = base.n_k // c
+        first = True
+        for frac in (1 / 32, 1 / 16, 1 / 8, 1 / 4, 1 / 2):
+            keep = inputs.keep_from_fraction(n_kc, frac)
+            for comp in (True, False):
+                w = base.scaled(cluster=c, keep=keep, compensate=comp)
+                p = binding.problem_from_workload(w)
+                plan = binding.Plan(p, dev)
+                if first:
+                    cluster_ms = timed(lambda: plan.cluster_qk(Q, K, V), args.steps)
+                    first = False
+                    kept = plan                      # clustering does not depend on keep / compensation
+                else:
+                    for name in ("perm_q", "perm_k", "Qp", "Kp", "Vp", "cq", "ck", "cv", "count_q", "count_k"):
+                        setattr(plan, name, getattr(kept, name))
+                select_ms = timed(lambda: plan.select_blocks(), args.steps)
+                attn_ms = timed(lambda: plan.cluster_attention_fwd(want_lse=False), args.steps)
+                assert all(v == 0 for v in plan.last_status().values())
+                flops = block_flops(w, w.heads, keep)
+                total = cluster_ms + select_ms + attn_ms
+                points.append({"cluster": c, "fraction": frac, "keep": keep, "compensate": comp,
+                               "cluster_qk_ms": cluster_ms, "select_ms": select_ms, "attn_ms": attn_ms,
+                               "total_ms": total, "attn_tflops": flops / attn_ms / 1e9,
+                               "attn_frac_of_peak": flops / attn_ms / 1e9 / peaks["bf16_tflops"],
+                               "speedup_vs_dense": dense_ms / total})
+                del plan
+    print(json.dumps({"metric": METRIC, "workload": "sweep", "heads": base.heads, "n": base.n_q,
+                      "head_dim": base.head_dim, "dense_sdpa_ms": dense_ms,
+                      "dense_sdpa_tflops": dense_flops(base, base.heads) / dense_ms / 1e9,
+                      "peak_tflops": peaks["bf16_tflops"], "peak_source": peak_kind, "points": points}))
+
+
 def main():
     args = parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     from paper_2608_26965_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
     if args.heads:
