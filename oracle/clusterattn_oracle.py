@@ -228,6 +228,20 @@ def centroid_scores(cq, ck):
     return np.asarray(cq, F64) @ np.asarray(ck, F64).T
 
 
+def centroid_scores_f32(cq, ck):
+    """The same scores in float32 with a fixed operation order: centroids rounded
+    to float32, terms added for k = 0, 1, ... with the product and the sum rounded
+    separately (no fused multiply-add).  The scores only feed the top-k decision,
+    which is therefore taken in the precision the device uses; any implementation
+    that follows the order gets the same bits."""
+    cq = np.ascontiguousarray(cq, dtype=np.float32)
+    ck = np.ascontiguousarray(ck, dtype=np.float32)
+    S = np.zeros((cq.shape[0], ck.shape[0]), np.float32)
+    for k in range(cq.shape[1]):
+        S = S + cq[:, k:k + 1] * ck[:, k][None, :]
+    return S
+
+
 # Section 3.3.2 top-k: the k best-scoring key clusters for each query cluster,
 # ties to the lower index, listed in ascending index order.
 def select_topk(scores, keep):
@@ -317,7 +331,7 @@ def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None):
 
 
 def select_blocks(cq, ck, keep):
-    return select_topk(centroid_scores(cq, ck), keep)
+    return select_topk(centroid_scores_f32(cq, ck), keep)
 
 
 def clusterattention_forward(Q, K, V, c_q, c_k, keep, compensate, scale=None):

@@ -1,6 +1,7 @@
 // Assignment (Section 3.3): centroid-centroid scores and exact top-k selection.
-// score(i, j) = cq_i . ck_j, accumulated in double (products of two floats are
-// exact in double, so the score is the correctly ordered sum of exact terms);
+// score(i, j) = cq_i . ck_j in float32 with a fixed operation order (terms added
+// for k = 0, 1, ..., product and sum rounded separately, no fused multiply-add),
+// so the scores -- and with them the selection -- are reproducible bit for bit;
 // the k best per query cluster by (score descending, index ascending), written
 // in ascending index order.
 #include "kernels.h"
@@ -10,10 +11,10 @@ namespace ca {
 constexpr int kSelectThreads = 256;
 constexpr int kSelectQT = 4;          // query clusters per CTA (key centroids are read once for all)
 
-__device__ __forceinline__ unsigned long long score_key(double s) {
-  if (s == 0.0) s = 0.0;
-  unsigned long long u = (unsigned long long)__double_as_longlong(s);
-  return (u >> 63) ? ~u : (u | 0x8000000000000000ull);
+__device__ __forceinline__ uint32_t score_key(float s) {
+  if (s == 0.0f) s = 0.0f;                        // -0 and +0 compare equal
+  const uint32_t u = __float_as_uint(s);
+  return (u >> 31) ? ~u : (u | 0x80000000u);
 }
 
 template <int D>
@@ -21,7 +22,7 @@ __global__ void __launch_bounds__(kSelectThreads)
 score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, int n_qc, int n_kc,
                     int keep, int32_t* __restrict__ block_idx) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);   // [QT][n_kc]
+  uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);                       // [QT][n_kc]
   float* qs = reinterpret_cast<float*>(keys + (size_t)kSelectQT * n_kc);        // [QT][D]
   __shared__ int s_hist[256];
   __shared__ int s_warp[64];
@@ -36,19 +37,19 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
   __syncthreads();
 
   for (int j = tid; j < n_kc; j += kSelectThreads) {
-    double acc[kSelectQT];
+    float acc[kSelectQT];
 #pragma unroll
-    for (int t = 0; t < kSelectQT; ++t) acc[t] = 0.0;
+    for (int t = 0; t < kSelectQT; ++t) acc[t] = 0.f;
     const float4* row = reinterpret_cast<const float4*>(ckp + (size_t)j * D);
     for (int k4 = 0; k4 < D / 4; ++k4) {
       const float4 kv = __ldg(row + k4);
 #pragma unroll
       for (int t = 0; t < kSelectQT; ++t) {
         const float* q = qs + t * D + k4 * 4;
-        acc[t] = fma((double)q[0], (double)kv.x, acc[t]);
-        acc[t] = fma((double)q[1], (double)kv.y, acc[t]);
-        acc[t] = fma((double)q[2], (double)kv.z, acc[t]);
-        acc[t] = fma((double)q[3], (double)kv.w, acc[t]);
+        acc[t] = __fadd_rn(acc[t], __fmul_rn(q[0], kv.x));
+        acc[t] = __fadd_rn(acc[t], __fmul_rn(q[1], kv.y));
+        acc[t] = __fadd_rn(acc[t], __fmul_rn(q[2], kv.z));
+        acc[t] = __fadd_rn(acc[t], __fmul_rn(q[3], kv.w));
       }
     }
 #pragma unroll
@@ -57,19 +58,19 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
   __syncthreads();
 
   for (int t = 0; t < nq; ++t) {
-    const unsigned long long* kt = keys + (size_t)t * n_kc;
+    const uint32_t* kt = keys + (size_t)t * n_kc;
     // radix selection of the keep-th largest key
-    unsigned long long prefix = 0, mask = 0;
+    uint32_t prefix = 0, mask = 0;
     int remaining = keep;
-    for (int shift = 56; shift >= 0; shift -= 8) {
+    for (int shift = 24; shift >= 0; shift -= 8) {
       s_hist[tid] = 0;                             // kSelectThreads == 256 bins
       __syncthreads();
       for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
         const int j = j0 + tid;
         const bool ok = j < n_kc;
-        const unsigned long long k = ok ? kt[j] : 0ull;
+        const uint32_t k = ok ? kt[j] : 0u;
         const bool cand = ok && ((k & mask) == prefix);
-        const int bin = cand ? (int)((k >> shift) & 255ull) : -1;
+        const int bin = cand ? (int)((k >> shift) & 255u) : -1;
         const unsigned peers = __match_any_sync(0xffffffffu, bin);
         if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
       }
@@ -95,12 +96,12 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
         }
       }
       __syncthreads();
-      prefix |= (unsigned long long)s_scalar[0] << shift;
-      mask |= 255ull << shift;
+      prefix |= (uint32_t)s_scalar[0] << shift;
+      mask |= 255u << shift;
       remaining = s_scalar[1];
       __syncthreads();
     }
-    const unsigned long long thr = prefix;
+    const uint32_t thr = prefix;
     const int eq_take = remaining;         // threshold-valued clusters taken, lowest indices first
 
     int32_t* out = block_idx + ((size_t)p * n_qc + q0 + t) * keep;
@@ -108,7 +109,7 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
     for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
       const int j = j0 + tid;
       const bool ok = j < n_kc;
-      const unsigned long long k = ok ? kt[j] : 0ull;
+      const uint32_t k = ok ? kt[j] : 0u;
       const int is_gt = (ok && k > thr) ? 1 : 0;
       const int is_eq = (ok && k == thr) ? 1 : 0;
       const int packed = is_gt | (is_eq << 16);
@@ -143,7 +144,7 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
 }
 
 size_t select_smem_bytes(int n_kc, int D) {
-  return (size_t)kSelectQT * n_kc * sizeof(unsigned long long) + (size_t)kSelectQT * D * sizeof(float);
+  return (size_t)kSelectQT * n_kc * sizeof(uint32_t) + (size_t)kSelectQT * D * sizeof(float);
 }
 
 int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n_kc, int D, int keep,

@@ -159,20 +159,9 @@ def test_select_blocks_exact(H, n_qc, n_kc, d, keep):
     plan = binding.Plan(p, DEV)
     got = plan.select_blocks(to_dev(cq[None]), to_dev(ck[None])).cpu().numpy()[0]
     torch.cuda.synchronize()
-    near_ties = 0
     for h in range(H):
-        S = orc.centroid_scores(cq[h], ck[h])
-        want = orc.select_topk(S, keep)
-        for i in range(n_qc):
-            if np.array_equal(got[h, i], want[i]):
-                continue
-            # only a near-tie at the keep-th score may differ (summation order of the dot product)
-            srt = np.sort(S[i])[::-1]
-            gap = srt[keep - 1] - srt[keep] if keep < n_kc else np.inf
-            assert gap < 1e-12 * np.abs(S).max(), (h, i)
-            near_ties += 1
-            assert len(set(got[h, i])) == keep and np.all(np.diff(got[h, i]) > 0)
-    assert near_ties <= 0.001 * H * n_qc + 1
+        # the scores are float32 with a fixed operation order on both sides: the lists are equal
+        assert np.array_equal(got[h], orc.select_blocks(cq[h], ck[h], keep)), h
 
 
 # ----------------------------------------------------------------------------

@@ -279,6 +279,21 @@ def test_centroid_score_is_mean_pairwise_logit_and_jensen_bound():
         assert np.exp(pair / np.sqrt(d)).mean() >= np.exp(S[i, j] / np.sqrt(d)) - 1e-12
 
 
+def test_float32_scores_follow_the_exact_scores():
+    r = rng(16)
+    cq, ck = r.standard_normal((9, 64)), r.standard_normal((40, 64))
+    S64 = orc.centroid_scores(cq.astype(np.float32), ck.astype(np.float32))
+    S32 = orc.centroid_scores_f32(cq, ck)
+    assert S32.dtype == np.float32 and np.abs(S32 - S64).max() < 2e-5 * np.abs(S64).max()
+    # brute force of the stated order on one entry
+    acc = np.float32(0)
+    for k in range(64):
+        acc = np.float32(acc + np.float32(np.float32(cq[3, k]) * np.float32(ck[7, k])))
+    assert acc == S32[3, 7]
+    # well separated scores: the selection is that of the exact scores
+    assert np.array_equal(orc.select_blocks(cq, ck, 5), orc.select_topk(S64, 5))
+
+
 def test_select_topk_matches_full_sort_with_index_tie_break():
     r = rng(15)
     S = r.standard_normal((7, 20))
