@@ -192,24 +192,19 @@ class ClockSampler:
 # ------------------------------------------------------------------------------
 def run_ours(args, w):
     import torch
-    import torch.distributed as dist
 
-    from paper_2608_26965_b200 import binding, build, inputs
+    from paper_2608_26965_b200 import binding, build, inputs, replicas
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, local, world = replicas.world()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
     torch.cuda.set_device(local)
     dev = f"cuda:{local}"
-    distributed = world > 1
-    if distributed:
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+    device = torch.device(dev)
+    distributed = replicas.init("nccl", device)
     if rank == 0:
         build.build()
-    if distributed:
-        dist.barrier()
+    replicas.barrier(device)
     binding.load_library()
 
     keep = args.keep or w.keep
@@ -225,17 +220,10 @@ def run_ours(args, w):
     stream = torch.cuda.current_stream()
 
     def barrier():
-        torch.cuda.synchronize()
-        if distributed:
-            dist.barrier()
-            torch.cuda.synchronize()
+        replicas.barrier(device)
 
     def max_over_ranks(x):
-        if not distributed:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return replicas.max_over_ranks(x, device)
 
     def step(events=None):
         if events is not None:
@@ -324,11 +312,9 @@ def run_ours(args, w):
         except Exception as exc:  # noqa: BLE001
             dense["torch_sdpa_error"] = str(exc)[:200]
 
-    if distributed:
-        dist.barrier()
+    barrier()
     if rank != 0:
-        if distributed:
-            dist.destroy_process_group()
+        replicas.shutdown()
         return
 
     peaks, peak_kind = load_peaks()
@@ -365,8 +351,7 @@ def run_ours(args, w):
                                 "kind": "oracle", "seconds": secs,
                                 "sample": f"{used} of {heads} heads in full (all stages, fp64 numpy)"}
     print(json.dumps(line))
-    if distributed:
-        dist.destroy_process_group()
+    replicas.shutdown()
 
 
 def run_sweep(args):
