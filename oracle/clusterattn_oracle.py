@@ -90,8 +90,10 @@ def transform_keys(K, R_q):
 
 # r(q) = R_k q / |R_k q|  (Section 3.2.2, ranking form; Appendix B.2).
 # A row whose transformed norm underflows maps to the zero vector.
-def query_representation(Q, R_k):
+def query_representation(Q, R_k, normalize=True):
     Z = np.asarray(Q, F64) @ np.asarray(R_k, F64)
+    if not normalize:        # adaptive-selection form (Section 3.2.2, Appendix B.1): r(q) = R_k q
+        return Z
     nrm = np.sqrt((Z * Z).sum(axis=1, keepdims=True))
     out = np.zeros_like(Z)
     ok = nrm[:, 0] >= 1e-30
@@ -256,6 +258,74 @@ def select_topk(scores, keep):
 
 
 # --------------------------------------------------------------------------
+# Section 3.3.2, adaptive selection: estimate the attention mass of every key
+# cluster from the centroids, |c_j| exp(qbar_i . kbar_j / sqrt(d)), and take the
+# most massive clusters until their share of the estimated mass reaches the
+# recall threshold, but never fewer than `min_count` (16 in the paper).  The
+# paper reaches this set through a two-pass 128-bin histogram; the definition
+# written out here is the exact greedy rule that the histogram approximates.
+#
+# The estimate only feeds discrete decisions (an order and a threshold
+# crossing), so it is taken in float32 with operations that any implementation
+# can reproduce bit for bit: 2^x by `exp2_f32` below, products and sums rounded
+# separately, the running sum taken in the order of decreasing mass.
+# --------------------------------------------------------------------------
+_EXP2_C = np.array([0.99992806, 0.69326097, 0.24261113, 0.05517165], np.float32)
+_LOG2E = np.float32(1.4426950408889634)
+
+
+def exp2_f32(x):
+    """2^x in float32 by a fixed recipe: clamp to [-126, 126], split x = n + f with n
+    the nearest integer (adding and subtracting 1.5 * 2^23), cubic polynomial in f
+    by Horner's rule with every product and sum rounded separately, scaling by
+    2^n.  Relative error 7.5e-5."""
+    x = np.minimum(np.maximum(np.asarray(x, np.float32), np.float32(-126.0)), np.float32(126.0))
+    magic = np.float32(12582912.0)
+    n = (x + magic) - magic
+    f = x - n
+    p = _EXP2_C[3] * f + _EXP2_C[2]
+    p = p * f + _EXP2_C[1]
+    p = p * f + _EXP2_C[0]
+    return np.ldexp(p, n.astype(np.int32)).astype(np.float32)
+
+
+def cluster_mass_f32(scores_f32, count_k, scale):
+    """Estimated attention mass of every key cluster for every query cluster,
+    relative to the row's best score: |c_j| 2^((s_ij - max_j s_ij) scale log2 e)."""
+    S = np.asarray(scores_f32, np.float32)
+    c = np.float32(np.float32(scale) * _LOG2E)
+    rel = (S - S.max(axis=1, keepdims=True)) * c
+    return exp2_f32(rel) * np.asarray(count_k, np.float32)[None, :]
+
+
+def select_adaptive(mass_f32, recall, min_count):
+    """Per query cluster: clusters in order of decreasing mass (ties: lower index);
+    the shortest prefix whose running float32 sum reaches recall * total, where the
+    total is the same running sum over all clusters; at least min_count clusters.
+    Returns a list of ascending index arrays (ragged)."""
+    mass = np.asarray(mass_f32, np.float32)
+    n_qc, n_kc = mass.shape
+    idx = np.arange(n_kc)
+    lists = []
+    for i in range(n_qc):
+        order = np.lexsort((idx, -mass[i]))
+        run = np.cumsum(mass[i][order], dtype=np.float32)
+        target = np.float32(np.float32(recall) * run[-1])
+        need = int(np.searchsorted(run, target, side="left")) + 1     # first prefix with run >= target
+        if recall >= 1.0:
+            need = n_kc                                               # full recall: every cluster, whatever rounding absorbs
+        need = min(n_kc, max(need, min_count))
+        lists.append(np.sort(order[:need]))
+    return lists
+
+
+def select_blocks_adaptive(cq, ck, count_k, recall, min_count=16, scale=None):
+    if scale is None:
+        scale = 1.0 / np.sqrt(np.asarray(cq).shape[1])
+    return select_adaptive(cluster_mass_f32(centroid_scores_f32(cq, ck), count_k, scale), recall, min_count)
+
+
+# --------------------------------------------------------------------------
 # Sparse attention over the selected clusters (eq. 2) with optional striped
 # mean-compensation (Appendix A, the expression for o-hat_S): an excluded
 # cluster enters numerator and denominator through its centroid key and value
@@ -309,18 +379,24 @@ def cluster_attention(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx, compensate,
 # metrics -> roots -> transforms -> global principal components -> fp32
 # coordinates -> recursive split -> centroids in the original space.
 # --------------------------------------------------------------------------
-def split_coordinates(Q, K):
-    """Returns (Yq32, Yk32): the fp32 coordinates the splitter reads."""
+def split_coordinates(Q, K, adaptive=False):
+    """Returns (Yq32, Yk32): the fp32 coordinates the splitter reads.  `adaptive`
+    selects the query representation that goes with adaptive selection: the
+    metric K_c^T K_c / n without normalisation (Appendix B.1) instead of the
+    normalised ranking form (Appendix B.2)."""
     R_q = psd_root(metric_q(Q))
-    R_k = psd_root(centered_scatter(K))
+    if adaptive:
+        R_k = psd_root(centered_scatter(K) / np.asarray(K).shape[0])
+    else:
+        R_k = psd_root(centered_scatter(K))
     Yk, _, _ = diagonalize(transform_keys(K, R_q))
-    Yq, _, _ = diagonalize(query_representation(Q, R_k))
+    Yq, _, _ = diagonalize(query_representation(Q, R_k, normalize=not adaptive))
     return Yq.astype(np.float32), Yk.astype(np.float32)
 
 
-def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None):
+def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None, adaptive=False):
     if Yq32 is None or Yk32 is None:
-        Yq32, Yk32 = split_coordinates(Q, K)
+        Yq32, Yk32 = split_coordinates(Q, K, adaptive)
     perm_q = recursive_split(Yq32, c_q)
     perm_k = recursive_split(Yk32, c_k)
     cq, count_q = centroids(Q, perm_q, c_q)

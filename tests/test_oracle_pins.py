@@ -308,6 +308,63 @@ def test_select_topk_matches_full_sort_with_index_tie_break():
     assert orc.select_topk(S, 3)[4].tolist() == [0, 1, 2]
 
 
+# ------------------------------------------------ adaptive selection (Section 3.3.2)
+def test_exp2_recipe_is_accurate_and_exact_on_integers():
+    x = np.linspace(-40, 10, 20001).astype(np.float32)
+    got = orc.exp2_f32(x).astype(np.float64)
+    assert np.abs(got / np.exp2(x.astype(np.float64)) - 1).max() < 1e-4
+    ints = np.arange(-20, 10).astype(np.float32)
+    assert np.abs(orc.exp2_f32(ints) / np.exp2(ints.astype(np.float64)) - 1).max() < 1e-4
+    assert orc.exp2_f32(np.float32(-1000.0)) < 1e-37            # clamped, no wrap-around
+
+
+def test_adaptive_selection_recall_minimality_and_limits():
+    r = rng(40)
+    d, n_qc, n_kc = 16, 7, 60
+    cq, ck = r.standard_normal((n_qc, d)) * 2, r.standard_normal((n_kc, d)) * 2
+    counts = r.integers(1, 9, n_kc)
+    scale = 1 / np.sqrt(d)
+    S = orc.centroid_scores(cq.astype(np.float32), ck.astype(np.float32))
+    exact_mass = counts[None, :] * np.exp(scale * (S - S.max(1, keepdims=True)))
+    for recall in (0.5, 0.9, 0.99):
+        lists = orc.select_blocks_adaptive(cq, ck, counts, recall, min_count=4, scale=scale)
+        for i, sel in enumerate(lists):
+            assert np.all(np.diff(sel) > 0) and len(sel) >= 4
+            m = exact_mass[i]
+            share = m[sel].sum() / m.sum()
+            assert share >= recall - 1e-3                       # reaches the recall (estimate precision 1e-4)
+            # greedy: every selected cluster is at least as massive as every excluded one
+            out = np.setdiff1d(np.arange(n_kc), sel)
+            assert m[sel].min() >= m[out].max() * (1 - 1e-3)
+            # minimal: without its least massive member the recall is missed (unless at the minimum count)
+            if len(sel) > 4:
+                assert (m[sel].sum() - m[sel].min()) / m.sum() < recall + 1e-3
+    # recall 1 takes everything, recall 0 takes the minimum count
+    assert all(len(x) == n_kc for x in orc.select_blocks_adaptive(cq, ck, counts, 1.0, 4, scale))
+    low = orc.select_blocks_adaptive(cq, ck, counts, 0.0, 5, scale)
+    assert all(len(x) == 5 for x in low)
+    # with equal cluster sizes the mass order is the score order: the minimum-count list is the top-k list
+    same = orc.select_blocks_adaptive(cq, ck, np.full(n_kc, 8), 0.0, 5, scale)
+    topk = orc.select_blocks(cq, ck, 5)
+    assert all(np.array_equal(a, b) for a, b in zip(same, topk))
+
+
+def test_unnormalised_query_representation_is_the_centred_key_metric():
+    # Appendix B.1: |r(q1) - r(q2)|^2 = |K_c (q1 - q2)|^2 / n, and softmax-invariant shifts vanish
+    r = rng(41)
+    K = r.standard_normal((80, 6)) @ r.standard_normal((6, 6)) + 2.0
+    n = K.shape[0]
+    R_k = orc.psd_root(orc.centered_scatter(K) / n)
+    Q = r.standard_normal((5, 6))
+    Z = orc.query_representation(Q, R_k, normalize=False)
+    Kc = K - K.mean(0)
+    for a in range(5):
+        for b in range(5):
+            assert np.isclose(((Z[a] - Z[b]) ** 2).sum(), ((Kc @ (Q[a] - Q[b])) ** 2).sum() / n, rtol=1e-9, atol=1e-12)
+    Yq, Yk = orc.split_coordinates(Q.repeat(20, 0) + 0.1 * r.standard_normal((100, 6)), K, adaptive=True)
+    assert Yq.dtype == np.float32 and Yq.shape == (100, 6)
+
+
 # ------------------------------------------------ attention (Section 1.2, Appendix A)
 def _setup(seed, N_q=48, N_k=60, d=8, c=4):
     r = rng(seed)
@@ -388,6 +445,18 @@ def test_compensated_error_decomposition():
             assert np.allclose(o - o_hat[row], (jensen_o + cov_sum) / d_hat, atol=1e-13)
             # the compensated denominator is d_hat times the dense one
             assert np.isclose(lse_hat[row], lsed[row] + np.log(d_hat), atol=1e-12)
+
+
+def test_attention_accepts_ragged_lists():
+    r, Q, K, V, pq, pk, c = _setup(24)
+    lists = [np.sort(r.choice(15, int(r.integers(1, 15)), replace=False)) for _ in range(12)]
+    o, lse = orc.cluster_attention(Q, K, V, pq, pk, c, c, lists, True)
+    # each query cluster equals the fixed-width call with its own list
+    for i, sel in enumerate(lists):
+        idx = np.tile(sel, (12, 1))
+        o_i, _ = orc.cluster_attention(Q, K, V, pq, pk, c, c, idx, True, query_clusters=[i])
+        rows = pq[i * c:(i + 1) * c]
+        assert np.abs(o[rows] - o_i[rows]).max() < 1e-14
 
 
 def test_forward_pipeline_shapes_and_convergence_to_dense():
