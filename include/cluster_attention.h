@@ -46,7 +46,10 @@ enum { CA_DTYPE_FP32 = 0, CA_DTYPE_BF16 = 1 };
 enum {
   CA_Y_IN = 1,      /* Yq/Yk hold the split coordinates: skip the transforms (used by tests
                        to feed the splitter the very same fp32 coordinates as the oracle)   */
-  CA_ATTN_FP32 = 2  /* cluster_attention_fwd: force the FP32 CUDA-core kernel for bf16 data  */
+  CA_ATTN_FP32 = 2, /* cluster_attention_fwd: force the FP32 CUDA-core kernel for bf16 data  */
+  CA_QUERY_UNNORMALIZED = 4 /* cluster_qk: queries are represented by R_k q with
+                       R_k = sqrt(K_c^T K_c / n_k), without the division by the norm: the
+                       form that goes with adaptive selection (Section 3.2.2, Appendix B.1) */
 };
 
 typedef struct {
@@ -59,7 +62,7 @@ typedef struct {
   int32_t keep;            /* kept key clusters per query cluster, 1 .. ceil(n_k/c_k)        */
   int32_t compensate;      /* 0/1: striped mean-compensation off/on                          */
   float softmax_scale;     /* 0 selects 1/sqrt(head_dim)                                     */
-  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32                                         */
+  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32 | CA_QUERY_UNNORMALIZED                 */
 } ca_problem_t;
 
 /* Bytes of workspace each stage needs for this problem (any pointer may be NULL). */
@@ -115,7 +118,7 @@ int select_blocks(const ca_problem_t* p, const float* cq, const float* ck,
  *   Qp,Kp,Vp, ck, cv, count_k, perm_q: as written by cluster_qk.
  *   O [B,H,n_q,d] in ORIGINAL row order, storage dtype; lse [B,H,n_q] fp32 or NULL.
  * bf16 storage runs on tcgen05 tensor cores with fp32 accumulation (head_dim
- * 64/128, clusters 64..256 with c_q == 128 tiles); fp32 storage, other sizes, or
+ * 64/128, c_q in {64, 128, 256}, c_k in 16..256); fp32 storage, other sizes, or
  * CA_ATTN_FP32 run the FP32 CUDA-core kernel.
  */
 int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
@@ -123,6 +126,42 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
                           const int32_t* count_k, const int32_t* block_idx,
                           const int32_t* perm_q, void* O, float* lse, void* ws,
                           size_t ws_bytes, void* stream);
+
+/*
+ * Adaptive assignment (Section 3.3.2): instead of a fixed count, each query
+ * cluster takes the key clusters of largest estimated attention mass until
+ * their share of the estimate reaches `recall`.  The estimate for the pair
+ * (i, j) is |c_j| exp(s cq_i . ck_j), s = softmax_scale.  All of it is float32
+ * with every product and sum rounded separately, in this order:
+ *   score = sum over k ascending of cq_ik ck_jk (as in select_blocks);
+ *   x = (score - max_j score) * (s * log2 e);   mass = 2^x * |c_j| with 2^x from
+ *   a cubic in the fractional part (x clamped to [-100, 100], nearest-integer
+ *   split, Horner's rule, coefficients 0.99992806, 0.69326097, 0.24261113,
+ *   0.05517165);  clusters in order of decreasing mass, ties to the lower index;
+ *   running sum in that order; the shortest prefix whose sum is >= recall * total
+ *   (total = the full running sum); recall >= 1 takes every cluster; never fewer
+ *   than min(min_count, n_kc).
+ *   block_idx [B,H,n_qc,n_kc] int32: row i holds keep_count[i] ascending cluster
+ *        indices, the rest of the row is -1.   keep_count [B,H,n_qc] int32.
+ * p->keep is not used (it must still be valid).  recall > 0, min_count >= 1.
+ */
+int select_blocks_adaptive(const ca_problem_t* p, const float* cq, const float* ck,
+                           const int32_t* count_k, float recall, int32_t min_count,
+                           int32_t* block_idx, int32_t* keep_count, void* ws,
+                           size_t ws_bytes, void* stream);
+
+/*
+ * cluster_attention_fwd over lists of different lengths: query cluster i attends
+ * the first keep_count[i] entries of row i of block_idx, whose rows are
+ * list_stride entries apart (n_kc for the output of select_blocks_adaptive).
+ * Everything else as in cluster_attention_fwd; p->keep is not used.
+ */
+int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const void* Kp,
+                                 const void* Vp, const float* ck, const float* cv,
+                                 const int32_t* count_k, const int32_t* block_idx,
+                                 const int32_t* keep_count, int32_t list_stride,
+                                 const int32_t* perm_q, void* O, float* lse, void* ws,
+                                 size_t ws_bytes, void* stream);
 
 /*
  * The attention stage without a caller-provided workspace.  (The paper has no

@@ -275,11 +275,11 @@ _LOG2E = np.float32(1.4426950408889634)
 
 
 def exp2_f32(x):
-    """2^x in float32 by a fixed recipe: clamp to [-126, 126], split x = n + f with n
+    """2^x in float32 by a fixed recipe: clamp to [-100, 100], split x = n + f with n
     the nearest integer (adding and subtracting 1.5 * 2^23), cubic polynomial in f
     by Horner's rule with every product and sum rounded separately, scaling by
     2^n.  Relative error 7.5e-5."""
-    x = np.minimum(np.maximum(np.asarray(x, np.float32), np.float32(-126.0)), np.float32(126.0))
+    x = np.minimum(np.maximum(np.asarray(x, np.float32), np.float32(-100.0)), np.float32(100.0))
     magic = np.float32(12582912.0)
     n = (x + magic) - magic
     f = x - n

@@ -22,7 +22,7 @@ CA_OK = 0
 ERRORS = {1: "CA_ERR_INVALID_ARG", 2: "CA_ERR_UNSUPPORTED", 3: "CA_ERR_WORKSPACE", 4: "CA_ERR_CUDA",
           5: "CA_ERR_TIMEOUT"}
 CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
-CA_Y_IN, CA_ATTN_FP32 = 1, 2
+CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED = 1, 2, 4
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
@@ -77,6 +77,10 @@ def load_library() -> ctypes.CDLL:
     lib.select_blocks.restype = ctypes.c_int
     lib.cluster_attention_fwd.argtypes = [pp] + [vp] * 11 + [sz, vp]
     lib.cluster_attention_fwd.restype = ctypes.c_int
+    lib.select_blocks_adaptive.argtypes = [pp, vp, vp, vp, ctypes.c_float, ctypes.c_int32, vp, vp, vp, sz, vp]
+    lib.select_blocks_adaptive.restype = ctypes.c_int
+    lib.cluster_attention_fwd_ragged.argtypes = [pp] + [vp] * 8 + [ctypes.c_int32] + [vp] * 4 + [sz, vp]
+    lib.cluster_attention_fwd_ragged.restype = ctypes.c_int
     lib.ca_last_status.argtypes = [vp]
     lib.ca_last_status.restype = ctypes.c_int
     lib.ca_version.argtypes = []
@@ -174,6 +178,8 @@ class Plan:
         self.count_q = torch.empty((B, H, p.n_qc), dtype=i32, device=dev)
         self.count_k = torch.empty((B, H, p.n_kc), dtype=i32, device=dev)
         self.block_idx = torch.empty((B, H, p.n_qc, p.keep), dtype=i32, device=dev)
+        self.block_idx_ragged = None
+        self.keep_count = None
         self.O = torch.empty((B, H, p.n_q, D), dtype=dt, device=dev)
         self.lse = torch.empty((B, H, p.n_q), dtype=f32, device=dev)
         self.Yq = torch.empty((B, H, p.n_q, D), dtype=f32, device=dev) if keep_y else None
@@ -231,6 +237,51 @@ class Plan:
         _check(rc, "cluster_attention_fwd")
         return self.O, (self.lse if want_lse else None)
 
+    def select_blocks_adaptive(self, recall: float, min_count: int = 16, cq=None, ck=None, count_k=None,
+                               stream=None):
+        """Adaptive assignment: returns (block_idx [B,H,n_qc,n_kc] padded with -1, keep_count [B,H,n_qc])."""
+        lib = load_library()
+        cq = self.cq if cq is None else cq
+        ck = self.ck if ck is None else ck
+        count_k = self.count_k if count_k is None else count_k
+        for name, t in (("cq", cq), ("ck", ck), ("count_k", count_k)):
+            _require_cuda(t, name)
+        pr = self.problem
+        if getattr(self, "block_idx_ragged", None) is None:
+            self.block_idx_ragged = torch.empty((pr.batch, pr.heads, pr.n_qc, pr.n_kc), dtype=torch.int32,
+                                                device=self.device)
+            self.keep_count = torch.empty((pr.batch, pr.heads, pr.n_qc), dtype=torch.int32, device=self.device)
+        ws = self.ws["select"]
+        rc = lib.select_blocks_adaptive(ctypes.byref(pr), _ptr(cq), _ptr(ck), _ptr(count_k), float(recall),
+                                        int(min_count), _ptr(self.block_idx_ragged), _ptr(self.keep_count),
+                                        _ptr(ws), ws.numel(), _stream_ptr(stream))
+        _check(rc, "select_blocks_adaptive")
+        return self.block_idx_ragged, self.keep_count
+
+    def cluster_attention_fwd_ragged(self, block_idx=None, keep_count=None, Qp=None, Kp=None, Vp=None, ck=None,
+                                     cv=None, count_k=None, perm_q=None, want_lse=True, stream=None):
+        lib = load_library()
+        block_idx = self.block_idx_ragged if block_idx is None else block_idx
+        keep_count = self.keep_count if keep_count is None else keep_count
+        args = [self.Qp if Qp is None else Qp, self.Kp if Kp is None else Kp, self.Vp if Vp is None else Vp,
+                self.ck if ck is None else ck, self.cv if cv is None else cv,
+                self.count_k if count_k is None else count_k, block_idx, keep_count]
+        perm_q = self.perm_q if perm_q is None else perm_q
+        for i, t in enumerate(args + [perm_q]):
+            _require_cuda(t, f"arg{i}")
+        ws = self.ws["attn"]
+        rc = lib.cluster_attention_fwd_ragged(ctypes.byref(self.problem), *[_ptr(t) for t in args],
+                                              int(block_idx.shape[-1]), _ptr(perm_q), _ptr(self.O),
+                                              _ptr(self.lse if want_lse else None), _ptr(ws), ws.numel(),
+                                              _stream_ptr(stream))
+        _check(rc, "cluster_attention_fwd_ragged")
+        return self.O, (self.lse if want_lse else None)
+
+    def forward_adaptive(self, Q, K, V, recall: float, min_count: int = 16, want_lse=False, stream=None):
+        self.cluster_qk(Q, K, V, stream=stream)
+        self.select_blocks_adaptive(recall, min_count, stream=stream)
+        return self.cluster_attention_fwd_ragged(want_lse=want_lse, stream=stream)
+
     def forward(self, Q, K, V, want_lse=False, stream=None):
         """The whole hot path: clustering, block selection, attention."""
         self.cluster_qk(Q, K, V, stream=stream)
@@ -259,6 +310,18 @@ def cluster_attention_fwd(problem: CaProblem, Qp, Kp, Vp, ck, cv, count_k, block
     if tuple(block_idx.shape[-2:]) != (problem.n_qc, problem.keep):
         raise ClusterAttnError("block_idx must be [B,H,n_qc,keep]")
     return plan.cluster_attention_fwd(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q)
+
+
+def select_blocks_adaptive(problem: CaProblem, cq, ck, count_k, recall: float, min_count: int = 16,
+                           plan: Optional[Plan] = None):
+    plan = plan or Plan(problem, device=str(cq.device))
+    return plan.select_blocks_adaptive(recall, min_count, cq, ck, count_k)
+
+
+def cluster_attention_fwd_ragged(problem: CaProblem, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, perm_q,
+                                 plan: Optional[Plan] = None):
+    plan = plan or Plan(problem, device=str(Qp.device))
+    return plan.cluster_attention_fwd_ragged(block_idx, keep_count, Qp, Kp, Vp, ck, cv, count_k, perm_q)
 
 
 def cluster_attention_fwd_static(problem: CaProblem, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O,

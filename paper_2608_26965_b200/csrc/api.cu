@@ -141,7 +141,11 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     }
     double* M = w.metric;
     double* CK = w.metric + (size_t)P * DD;
-    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, M, CK, st));
+    // the un-normalised query representation (Appendix B.1) takes the root of K_c^T K_c / n_k,
+    // the normalised one is indifferent to the factor and keeps the scatter matrix as it is
+    const bool unnormalized = (p->flags & CA_QUERY_UNNORMALIZED) != 0;
+    const double ck_scale = unnormalized ? 1.0 / (double)p->n_k : 1.0;
+    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, M, CK, st));
     // factors F_q F_q^T = M and F_k F_k^T = C_K (they stand in for the symmetric roots:
     // any factor yields the same principal-component coordinates)
     CA_TRY(launch_cholesky_factor(w.metric, 2 * P, D, w.roots, w.roots32, st));
@@ -151,14 +155,14 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     double* covK = w.cov;
     double* covQ = w.cov + (size_t)P * DD;
     CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
-    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, 1.0 / (double)p->n_k, 0, covK, nullptr, st));
+    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, unnormalized ? 1.0 : 1.0 / (double)p->n_k, 0, covK, nullptr, st));
     // query representation r(q) = F_k^T q / |F_k^T q| and its covariance
     if (tc) {
-      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, 1, nullptr, qp_hi, qp_lo, w.wt_hi,
+      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo, w.wt_hi,
                                  w.wt_lo, w.status, st));
       CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, w.status, st));
     } else {
-      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, 1, w.Qprime, st));
+      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, w.Qprime, st));
       CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
     }
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
@@ -219,8 +223,49 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
   CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
   if (tensor_cores)
-    return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, scale, O, lse, ws, st);
-  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, scale, O, lse, st);
+    return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, nullptr, p->keep, perm_q, scale, O, lse,
+                          ws, st);
+  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, nullptr, p->keep, perm_q, scale, O, lse, st);
+}
+
+int select_blocks_adaptive(const ca_problem_t* p, const float* cq, const float* ck, const int32_t* count_k,
+                           float recall, int32_t min_count, int32_t* block_idx, int32_t* keep_count,
+                           void* ws, size_t ws_bytes, void* stream) {
+  CA_TRY(check_problem(p));
+  const void* ptrs[] = {cq, ck, count_k, block_idx, keep_count};
+  for (const void* x : ptrs)
+    if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  if (!(recall > 0.f) || min_count < 1) return CA_ERR_INVALID_ARG;
+  if (!ws || ws_bytes < kStatusBytes) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  return launch_select_adaptive(cq, ck, count_k, p->batch * p->heads, ceil_div(p->n_q, p->cluster_q),
+                                ceil_div(p->n_k, p->cluster_k), p->head_dim, scale, recall, min_count,
+                                block_idx, keep_count, st);
+}
+
+int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const void* Kp, const void* Vp,
+                                 const float* ck, const float* cv, const int32_t* count_k,
+                                 const int32_t* block_idx, const int32_t* keep_count, int32_t list_stride,
+                                 const int32_t* perm_q, void* O, float* lse, void* ws, size_t ws_bytes,
+                                 void* stream) {
+  CA_TRY(check_problem(p));
+  const void* ptrs[] = {Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, perm_q, O};
+  for (const void* x : ptrs)
+    if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  if (list_stride < 1) return CA_ERR_INVALID_ARG;
+  const bool tensor_cores = attn_tc_supported(*p);
+  const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
+  if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  if (tensor_cores)
+    return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale,
+                          O, lse, ws, st);
+  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O,
+                         lse, st);
 }
 
 int ca_last_status(const void* ws) {

@@ -17,7 +17,8 @@ __global__ void __launch_bounds__(kRefThreads)
 attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __restrict__ Vp,
                 const float* __restrict__ ck, const float* __restrict__ cv,
                 const int32_t* __restrict__ count_k, const int32_t* __restrict__ block_idx,
-                const int32_t* __restrict__ perm_q, int n_q, int n_k, int c_q, int c_k, int keep,
+                const int32_t* __restrict__ keep_count, int list_stride,
+                const int32_t* __restrict__ perm_q, int n_q, int n_k, int c_q, int c_k, int keep_all,
                 int compensate, float scale, T* __restrict__ O, float* __restrict__ lse) {
   constexpr int LD = D + 1;
   constexpr int NC = D / 8;              // output columns per thread
@@ -39,7 +40,8 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
   const size_t q_base = ((size_t)p * n_qc + qc) * (size_t)c_q;
   const T* Kh = Kp + (size_t)p * n_kc * (size_t)c_k * D;
   const T* Vh = Vp + (size_t)p * n_kc * (size_t)c_k * D;
-  const int32_t* sel = block_idx + ((size_t)p * n_qc + qc) * keep;
+  const int32_t* sel = block_idx + ((size_t)p * n_qc + qc) * list_stride;
+  const int keep = keep_count ? keep_count[(size_t)p * n_qc + qc] : keep_all;   // ragged lists carry their length
   const int32_t* cnt = count_k + (size_t)p * n_kc;
 
   for (int e = tid; e < kRefQR * D; e += kRefThreads) {
@@ -156,7 +158,8 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
 template <typename T>
 static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* Vp, const float* ck,
                     const float* cv, const int32_t* count_k, const int32_t* block_idx,
-                    const int32_t* perm_q, float scale, T* O, float* lse, cudaStream_t st) {
+                    const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, T* O,
+                    float* lse, cudaStream_t st) {
   const int P = pr.batch * pr.heads, D = pr.head_dim;
   const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
   const int tiles = ceil_div(pr.cluster_q, kRefQR);
@@ -166,12 +169,14 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
   if (D == 64) {
     auto k = attn_ref_kernel<T, 64>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, pr.n_q, pr.n_k,
+    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
+                                        pr.n_q, pr.n_k,
                                         pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse);
   } else {
     auto k = attn_ref_kernel<T, 128>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, pr.n_q, pr.n_k,
+    k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
+                                        pr.n_q, pr.n_k,
                                         pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse);
   }
   CA_LAUNCH_CHECK();
@@ -180,13 +185,15 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
 
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
-                    const int32_t* perm_q, float scale, void* O, float* lse, cudaStream_t st) {
+                    const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
+                    float* lse, cudaStream_t st) {
   if (pr.dtype == CA_DTYPE_BF16)
     return launch_t(pr, static_cast<const __nv_bfloat16*>(Qp), static_cast<const __nv_bfloat16*>(Kp),
-                    static_cast<const __nv_bfloat16*>(Vp), ck, cv, count_k, block_idx, perm_q, scale,
+                    static_cast<const __nv_bfloat16*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride,
+                    perm_q, scale,
                     static_cast<__nv_bfloat16*>(O), lse, st);
   return launch_t(pr, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
-                  static_cast<const float*>(Vp), ck, cv, count_k, block_idx, perm_q, scale,
+                  static_cast<const float*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale,
                   static_cast<float*>(O), lse, st);
 }
 

@@ -59,11 +59,12 @@ struct TcCfg {
 struct TcParams {
   const int32_t* count_k;
   const int32_t* block_idx;
+  const int32_t* keep_count;      // per query cluster list length, or null: every list holds `keep` entries
   const int32_t* perm_q;
   __nv_bfloat16* O;
   float* lse;
   int* status;
-  int n_q, n_k, c_q, c_k, keep, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
+  int n_q, n_k, c_q, c_k, keep, list_stride, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
   float scale_log2;
 };
 
@@ -104,8 +105,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int tiles_per_qc = prm.c_q >= kTile ? prm.c_q / kTile : 1;
   const int q_rows = prm.c_q >= kTile ? kTile : prm.c_q;
   const int qc = blockIdx.x / tiles_per_qc, half = blockIdx.x % tiles_per_qc;
-  const int32_t* sel = prm.block_idx + ((size_t)p * prm.n_qc + qc) * prm.keep;
-  const int sel_tiles = selected_tiles(prm.keep, prm.c_k);
+  const int32_t* sel = prm.block_idx + ((size_t)p * prm.n_qc + qc) * prm.list_stride;
+  const int keep = prm.keep_count ? prm.keep_count[(size_t)p * prm.n_qc + qc] : prm.keep;
+  const int sel_tiles = selected_tiles(keep, prm.c_k);
   const int cen_tiles = prm.compensate ? prm.cen_tiles : 0;
   const int loads = sel_tiles + cen_tiles;             // K/V tile loads
   const int steps = 2 * sel_tiles + cen_tiles;         // half-steps of 64 keys
@@ -160,7 +162,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const int per = kTile / prm.c_k;
           for (int u = 0; u < per; ++u) {
             int e = t * per + u;
-            if (e >= prm.keep) e = prm.keep - 1;          // filler rows, masked by the softmax
+            if (e >= keep) e = keep - 1;          // filler rows, masked by the softmax
             const int j = sel[e];
             for (int pn = 0; pn < C::PANELS; ++pn)
               tma_load_2d(dst + pn * C::PANEL_BYTES + u * prm.c_k * 128, map, pn * 64,
@@ -250,7 +252,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     for (int w = st; w < prm.bitmap_words; w += 128) bitmap[w] = 0u;
     asm volatile("bar.sync 1, 128;" ::: "memory");
     if (prm.compensate)
-      for (int e = st; e < prm.keep; e += 128) atomicOr(&bitmap[sel[e] >> 5], 1u << (sel[e] & 31));
+      for (int e = st; e < keep; e += 128) atomicOr(&bitmap[sel[e] >> 5], 1u << (sel[e] & 31));
     asm volatile("bar.sync 1, 128;" ::: "memory");
 
     float m_ref = -INFINITY, l_run = 0.f;
@@ -277,10 +279,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const int per = prm.c_k >= kHalf ? 1 : kHalf / prm.c_k;
           for (int x = 0; x < per; ++x) {
             const int e = (col0 + x * prm.c_k) / prm.c_k;
-            if (e >= prm.keep || cnt[sel[e]] < prm.c_k) masked = true;
+            if (e >= keep || cnt[sel[e]] < prm.c_k) masked = true;
           }
           const int e = (col0 + (st & 63)) / prm.c_k;
-          use = e < prm.keep && ((col0 + (st & 63)) % prm.c_k) < cnt[sel[min(e, prm.keep - 1)]];
+          use = e < keep && ((col0 + (st & 63)) % prm.c_k) < cnt[sel[min(e, keep - 1)]];
         }
         if (masked && st < kHalf) bz[st] = use ? 0.f : -INFINITY;
       } else {
@@ -511,8 +513,9 @@ static int launch_tc_d(const CUtensorMap* maps, const TcParams& prm, dim3 grid, 
 }
 
 int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp, const float* ck,
-                   const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* perm_q,
-                   float scale, void* O, float* lse, void* ws, cudaStream_t st) {
+                   const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* keep_count,
+                   int list_stride, const int32_t* perm_q, float scale, void* O, float* lse, void* ws,
+                   cudaStream_t st) {
   const int P = pr.batch * pr.heads, D = pr.head_dim;
   const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
   const int cen_tiles = ceil_div(n_kc, kHalf);
@@ -534,7 +537,8 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
             make_map(&maps[4], vb, (size_t)P * cen_tiles * kHalf, D, kHalf);
   if (!ok) return CA_ERR_CUDA;
   TcParams prm;
-  prm.count_k = count_k; prm.block_idx = block_idx; prm.perm_q = perm_q;
+  prm.count_k = count_k; prm.block_idx = block_idx; prm.keep_count = keep_count; prm.perm_q = perm_q;
+  prm.list_stride = list_stride;
   prm.O = static_cast<__nv_bfloat16*>(O); prm.lse = lse; prm.status = status;
   prm.n_q = pr.n_q; prm.n_k = pr.n_k; prm.c_q = pr.cluster_q; prm.c_k = pr.cluster_k; prm.keep = pr.keep;
   prm.n_qc = n_qc; prm.n_kc = n_kc; prm.cen_tiles = cen_tiles; prm.compensate = pr.compensate;

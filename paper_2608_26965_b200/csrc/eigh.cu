@@ -340,14 +340,14 @@ int launch_cholesky_factor(const double* A, int count, int D, double* out64, flo
 // M = gramQ / n_q ;  C_K = gramK - sumK sumK^T / n_k   (centred scatter)
 __global__ void metric_kernel(const double* __restrict__ gramQ, const double* __restrict__ gramK,
                               const double* __restrict__ sumK, int D, double n_q, double n_k,
-                              double* __restrict__ M, double* __restrict__ CK) {
+                              double ck_scale, double* __restrict__ M, double* __restrict__ CK) {
   const int p = blockIdx.y;
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= D * D) return;
   const int i = e / D, j = e % D;
   const size_t o = (size_t)p * D * D + e;
   M[o] = gramQ[o] / n_q;
-  CK[o] = gramK[o] - sumK[(size_t)p * D + i] * sumK[(size_t)p * D + j] / n_k;
+  CK[o] = (gramK[o] - sumK[(size_t)p * D + i] * sumK[(size_t)p * D + j] / n_k) * ck_scale;
 }
 
 // Cov = gram / n - mean mean^T, mean = sum / n
@@ -431,9 +431,9 @@ __global__ void bias_kernel(const double* __restrict__ sum, const double* __rest
 }
 
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
-                  int n_k, double* M, double* CK, cudaStream_t st) {
+                  int n_k, double ck_scale, double* M, double* CK, cudaStream_t st) {
   metric_kernel<<<dim3(ceil_div(D * D, 256), P), 256, 0, st>>>(gramQ, gramK, sumK, D, (double)n_q,
-                                                                (double)n_k, M, CK);
+                                                                (double)n_k, ck_scale, M, CK);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }

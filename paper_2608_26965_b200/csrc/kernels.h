@@ -27,7 +27,7 @@ int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_
 int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
                 cudaStream_t st);
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
-                  int n_k, double* M, double* CK, cudaStream_t st);
+                  int n_k, double ck_scale, double* M, double* CK, cudaStream_t st);
 int launch_covariance(const double* gram, const double* sum, int P, int D, int n, double* cov,
                       cudaStream_t st);
 int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
@@ -47,19 +47,24 @@ int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P
 
 // select.cu
 size_t select_smem_bytes(int n_kc, int D);
+int launch_select_adaptive(const float* cq, const float* ck, const int32_t* count_k, int P, int n_qc, int n_kc,
+                           int D, float scale, float recall, int min_count, int32_t* block_idx,
+                           int32_t* keep_count, cudaStream_t st);
 int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n_kc, int D, int keep,
                         int32_t* block_idx, cudaStream_t st);
 
 // attn_ref.cu
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
-                    const int32_t* perm_q, float scale, void* O, float* lse, cudaStream_t st);
+                    const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
+                    float* lse, cudaStream_t st);
 
 // attn_tc.cu
 bool attn_tc_supported(const ca_problem_t& pr);
 size_t attn_tc_workspace_bytes(const ca_problem_t& pr);
 int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp, const float* ck,
-                   const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* perm_q,
-                   float scale, void* O, float* lse, void* ws, cudaStream_t st);
+                   const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* keep_count,
+                   int list_stride, const int32_t* perm_q, float scale, void* O, float* lse, void* ws,
+                   cudaStream_t st);
 
 }  // namespace ca

@@ -167,7 +167,7 @@ def test_select_blocks_exact(H, n_qc, n_kc, d, keep):
 # ----------------------------------------------------------------------------
 # Attention on the oracle's permutation and block lists.
 # ----------------------------------------------------------------------------
-def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=None):
+def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=None, adaptive=None):
     Q, K, V = inputs.generate(w.scaled(heads=H))
     c_q, c_k = w.cluster, (cluster_k or w.cluster)
     p = binding.problem_from_workload(w, heads=H, keep=keep, compensate=compensate, flags=flags,
@@ -185,7 +185,10 @@ def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=No
             ck_, nk_ = orc.centroids(K[h], pk, c_k)
             cv_, _ = orc.centroids(V[h], pk, c_k)
             cl = dict(perm_q=pq, perm_k=pk, cq=cq_, ck=ck_, cv=cv_, count_q=nq_, count_k=nk_)
-        idx = orc.select_blocks(cl["cq"], cl["ck"], keep)
+        if adaptive is None:
+            idx = orc.select_blocks(cl["cq"], cl["ck"], keep)
+        else:                                # lists of different lengths (Section 3.3.2)
+            idx = orc.select_blocks_adaptive(cl["cq"], cl["ck"], cl["count_k"], adaptive[0], adaptive[1])
         ck32, cv32 = cl["ck"].astype(np.float32), cl["cv"].astype(np.float32)
         o, lse = orc.cluster_attention(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c_q, c_k, idx, compensate,
                                        ck=ck32, cv=cv32, count_k=cl["count_k"])
@@ -202,12 +205,25 @@ def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=No
         arrs["ck"].append(ck32)
         arrs["cv"].append(cv32)
         arrs["count_k"].append(cl["count_k"].astype(np.int32))
-        arrs["idx"].append(idx.astype(np.int32))
+        if adaptive is None:
+            arrs["idx"].append(idx.astype(np.int32))
+        else:
+            padded = np.full((len(idx), p.n_kc), -1, np.int32)
+            for i, row in enumerate(idx):
+                padded[i, :len(row)] = row
+            arrs["idx"].append(padded)
+            arrs.setdefault("keep_count", []).append(np.array([len(row) for row in idx], np.int32))
     st = {k: np.stack(v)[None] for k, v in arrs.items()}
     dt = binding.torch_dtype(p)
-    O, lse = plan.cluster_attention_fwd(to_dev(st["Qp"], dt), to_dev(st["Kp"], dt), to_dev(st["Vp"], dt),
-                                        to_dev(st["ck"]), to_dev(st["cv"]), to_dev(st["count_k"]),
-                                        to_dev(st["idx"]), to_dev(st["perm_q"]))
+    if adaptive is None:
+        O, lse = plan.cluster_attention_fwd(to_dev(st["Qp"], dt), to_dev(st["Kp"], dt), to_dev(st["Vp"], dt),
+                                            to_dev(st["ck"]), to_dev(st["cv"]), to_dev(st["count_k"]),
+                                            to_dev(st["idx"]), to_dev(st["perm_q"]))
+    else:
+        O, lse = plan.cluster_attention_fwd_ragged(to_dev(st["idx"]), to_dev(st["keep_count"]),
+                                                   to_dev(st["Qp"], dt), to_dev(st["Kp"], dt), to_dev(st["Vp"], dt),
+                                                   to_dev(st["ck"]), to_dev(st["cv"]), to_dev(st["count_k"]),
+                                                   to_dev(st["perm_q"]))
     torch.cuda.synchronize()
     assert all(v == 0 for v in plan.last_status().values())
     return O[0].float().cpu().numpy(), lse[0].cpu().numpy(), refs
@@ -297,3 +313,100 @@ def test_end_to_end_tiny_configuration():
             b = {frozenset(theirs[j * 64:(j + 1) * 64].tolist()) for j in range(16)}
             moved += 64 * len(a - b)
     print(f"rows in clusters that differ from the all-fp64 clustering: {moved} of {4 * 1024}")
+
+
+# ----------------------------------------------------------------------------
+# Adaptive selection (Section 3.3.2): float32 mass estimates with a fixed recipe
+# on both sides, so lists and their lengths are equal bit for bit.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("H,n_qc,n_kc,d,spread", [(2, 16, 16, 64, 1.0), (1, 37, 300, 128, 1.0),
+                                                    (2, 130, 1024, 64, 3.0), (1, 9, 2049, 128, 0.2),
+                                                    (1, 20, 1500, 64, 12.0)])
+@pytest.mark.parametrize("recall,min_count", [(0.5, 1), (0.9, 16), (0.999, 4), (1.0, 1)])
+def test_select_blocks_adaptive_exact(H, n_qc, n_kc, d, spread, recall, min_count):
+    r = np.random.default_rng(n_qc * n_kc + d)
+    cq = (r.standard_normal((H, n_qc, d)) * spread).astype(np.float32)
+    ck = r.standard_normal((H, n_kc, d)).astype(np.float32)
+    ck[:, 3] = ck[:, 1]                      # duplicate centroids: equal masses, ordered by index
+    ck[:, n_kc - 1] = ck[:, 1]
+    if n_qc > 4:
+        cq[:, 4] = 0.0                       # every score equal: the mass is the member count alone
+    c = 16
+    count = np.full((H, n_kc), c, np.int32)
+    count[:, -1] = 5                         # a short last cluster weighs less
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    p = binding.make_problem(1, H, n_qc * c, n_kc * c - 11, d, "fp32", c, c, 1, softmax_scale=scale)
+    plan = binding.Plan(p, DEV)
+    idx, keep = plan.select_blocks_adaptive(recall, min_count, to_dev(cq[None]), to_dev(ck[None]),
+                                            to_dev(count[None]))
+    torch.cuda.synchronize()
+    idx, keep = idx.cpu().numpy()[0], keep.cpu().numpy()[0]
+    lengths = set()
+    for h in range(H):
+        want = orc.select_blocks_adaptive(cq[h], ck[h], count[h], recall, min_count, scale=scale)
+        for i, row in enumerate(want):
+            assert keep[h, i] == len(row), (h, i, keep[h, i], len(row))
+            assert np.array_equal(idx[h, i, :len(row)], row), (h, i)
+            assert (idx[h, i, len(row):] == -1).all()
+            lengths.add(len(row))
+    if recall < 1.0 and spread >= 1.0 and n_kc > 16:
+        assert len(lengths) > 1              # the case does exercise lists of different lengths
+
+
+@pytest.mark.parametrize("name,n_q,n_k,dtype_flags,recall", [
+    ("tiny", 1024, 1024, 0, 0.9),                      # fp32 storage: CUDA-core kernel
+    ("tabular", 1024, 4096, 0, 0.8),                   # bf16 on the tensor cores
+    ("tabular", 1000, 4000, binding.CA_ATTN_FP32, 0.95),
+    ("video480", 1000, 1000, 0, 0.9),
+    ("sweep64", 1100, 3000, 0, 0.9),
+])
+def test_attention_ragged_lists(name, n_q, n_k, dtype_flags, recall):
+    if name == "sweep64":
+        w = inputs.WORKLOADS["sweep"].scaled(n_q=n_q, n_k=n_k, cluster=64)
+    else:
+        w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k)
+    if w.kind == "video":
+        w = w.scaled(grid=(5, 10, 20))
+    O, lse, refs = attention_case(w, 2, 1, True, flags=dtype_flags, adaptive=(recall, 2))
+    for h, (o_ref, lse_ref) in enumerate(refs):
+        if w.dtype == "fp32":
+            assert np.abs(O[h] - o_ref).max() < 1e-5 and np.abs(lse[h] - lse_ref).max() < 1e-5
+        else:
+            assert bf16_close(O[h], o_ref)
+            assert np.abs(lse[h] - lse_ref).max() < 2e-2
+
+
+def test_end_to_end_adaptive_tiny_configuration():
+    """cluster_qk with the un-normalised query representation (Appendix B.1), adaptive
+    selection and attention over the resulting ragged lists, every stage on the device."""
+    w = inputs.WORKLOADS["tiny"]
+    Q, K, V = inputs.generate(w)
+    scale = float(np.float32(1.0 / np.sqrt(w.head_dim)))
+    p = binding.problem_from_workload(w, flags=binding.CA_QUERY_UNNORMALIZED, softmax_scale=scale)
+    plan = binding.Plan(p, DEV, keep_y=True)
+    O, lse = plan.forward_adaptive(store(p, Q), store(p, K), store(p, V), recall=0.9, min_count=2, want_lse=True)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for h in range(w.heads):
+        Yq = plan.Yq[0, h].cpu().numpy()
+        pq, pk = plan.perm_q[0, h].cpu().numpy(), plan.perm_k[0, h].cpu().numpy()
+        assert np.array_equal(pq, orc.recursive_split(Yq, w.cluster))
+        # query coordinates are an isometry of r(q) = R_k q, R_k = sqrt(K_c^T K_c / n)
+        R_k = orc.psd_root(orc.centered_scatter(K[h]) / w.n_k)
+        rq = orc.query_representation(Q[h], R_k, normalize=False)
+        r = np.random.default_rng(h)
+        i, j = r.integers(0, w.n_q, 200), r.integers(0, w.n_q, 200)
+        want = ((rq[i] - rq[j]) ** 2).sum(1)
+        got = ((Yq[i].astype(np.float64) - Yq[j]) ** 2).sum(1)
+        assert np.abs(got - want).max() <= 2e-3 * want.max()
+        lists = orc.select_blocks_adaptive(plan.cq[0, h].cpu().numpy(), plan.ck[0, h].cpu().numpy(),
+                                           plan.count_k[0, h].cpu().numpy(), 0.9, 2, scale=scale)
+        keep = plan.keep_count[0, h].cpu().numpy()
+        idx = plan.block_idx_ragged[0, h].cpu().numpy()
+        for i, row in enumerate(lists):
+            assert keep[i] == len(row) and np.array_equal(idx[i, :len(row)], row)
+        o_ref, lse_ref = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, w.cluster, w.cluster, lists, True,
+                                               ck=plan.ck[0, h].cpu().numpy(), cv=plan.cv[0, h].cpu().numpy(),
+                                               count_k=plan.count_k[0, h].cpu().numpy())
+        assert np.abs(O[0, h].cpu().numpy() - o_ref).max() < 1e-5
+        assert np.abs(lse[0, h].cpu().numpy() - lse_ref).max() < 1e-5
