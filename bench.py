@@ -52,11 +52,20 @@ def parse_args():
     ap.add_argument("--workload", default="tabular")
     ap.add_argument("--keep", type=int, default=0, help="override kept key clusters per query cluster")
     ap.add_argument("--heads", type=int, default=0, help="run only the first HEADS heads (profiling captures)")
+    ap.add_argument("--n-q", type=int, default=0, help="override the number of query rows per head")
+    ap.add_argument("--n-k", type=int, default=0, help="override the number of key rows per head")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-dense", action="store_true")
     ap.add_argument("--sweep", action="store_true",
                     help="sweep workload: cluster size x kept fraction x compensation, one JSON line with all points")
+    ap.add_argument("--adaptive", type=float, default=0.0, metavar="RECALL",
+                    help="adaptive mass-recall selection with this recall threshold (min count 16) and the "
+                         "un-normalised query representation, instead of a fixed count per query cluster")
+    ap.add_argument("--scaling", action="store_true",
+                    help="token-count sweep 8k..1M with per-stage times (64 kept blocks, and 10 %% of the blocks), "
+                         "eager launches and one replayed CUDA graph, against dense attention")
+    ap.add_argument("--max-tokens", type=int, default=1 << 20)
     return ap.parse_args()
 
 
@@ -209,7 +218,8 @@ def run_ours(args, w):
 
     keep = args.keep or w.keep
     heads = w.heads
-    p = binding.problem_from_workload(w, keep=keep)
+    adaptive = args.adaptive > 0.0
+    p = binding.problem_from_workload(w, keep=keep, flags=binding.CA_QUERY_UNNORMALIZED if adaptive else 0)
     dt = binding.torch_dtype(p)
     Qh, Kh, Vh = inputs.generate(w)                        # every replica runs the same seeded batch
     pin = lambda a: torch.from_numpy(a[None]).to(dt).pin_memory()
@@ -231,10 +241,16 @@ def run_ours(args, w):
         plan.cluster_qk(Q, K, V)
         if events is not None:
             events[1].record(stream)
-        plan.select_blocks()
+        if adaptive:
+            plan.select_blocks_adaptive(args.adaptive, 16)
+        else:
+            plan.select_blocks()
         if events is not None:
             events[2].record(stream)
-        plan.cluster_attention_fwd(want_lse=False)
+        if adaptive:
+            plan.cluster_attention_fwd_ragged(want_lse=False)
+        else:
+            plan.cluster_attention_fwd(want_lse=False)
         if events is not None:
             events[3].record(stream)
 
@@ -264,7 +280,8 @@ def run_ours(args, w):
         "select_blocks": float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
         "cluster_attention_fwd": float(np.mean([e[2].elapsed_time(e[3]) for e in ev])),
     }
-    flops_step = block_flops(w, heads, keep)
+    mean_keep = float(plan.keep_count.float().mean().item()) if adaptive else float(keep)
+    flops_step = block_flops(w, heads, mean_keep)
     value = world * flops_step / (ms_per_step * 1e-3) / 1e12
 
     # ---- end to end through the same calls with HOST buffers (pinned), copies inside the region
@@ -324,14 +341,16 @@ def run_ours(args, w):
     roofline = {
         "kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": attn_tflops, "peak": peak,
         "peak_source": f"{peak_kind} bf16 burst", "unit": "TFLOP/s", "frac": attn_tflops / peak,
-        "traffic": NCU_TRAFFIC_BYTES.get(w.name),
+        "traffic": None if (adaptive or args.keep or args.n_q or args.n_k or args.heads)
+        else NCU_TRAFFIC_BYTES.get(w.name),
     }
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "heads": heads, "head_dim": w.head_dim, "n_q": w.n_q, "n_k": w.n_k,
-                   "cluster": w.cluster, "keep": keep, "n_kc": w.n_kc, "compensate": w.compensate,
+                   "cluster": w.cluster, "keep": mean_keep if adaptive else keep, "n_kc": w.n_kc,
+                   "selection": f"adaptive recall {args.adaptive} min 16" if adaptive else "top-k", "compensate": w.compensate,
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "inputs larger than L2 (no flush)"},
         "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),
@@ -421,15 +440,91 @@ def run_sweep(args):
                       "peak_tflops": peaks["bf16_tflops"], "peak_source": peak_kind, "points": points}))
 
 
+def run_scaling(args):
+    """Token counts 8,192 .. 1,048,576 (self-attention, d = 64, 128-row clusters): per-stage
+    times with 64 kept blocks and with 10 % of the blocks kept, the same step replayed from a
+    CUDA graph, and dense attention on the same tensors."""
+    import torch
+
+    from paper_2608_26965_b200 import binding, build, inputs
+
+    build.build()
+    binding.load_library()
+    dev = "cuda:0"
+    torch.cuda.set_device(0)
+    heads = args.heads or 4
+    stream = torch.cuda.current_stream()
+    points = []
+    n = 8192
+    while n <= args.max_tokens:
+        base = inputs.WORKLOADS["tabular"].scaled(n_q=n, n_k=n, heads=heads)
+        Qh, Kh, Vh = inputs.generate(base)
+        Q, K, V = (torch.from_numpy(a[None]).to(torch.bfloat16).to(dev) for a in (Qh, Kh, Vh))
+        reps = max(2, min(args.steps, (1 << 22) // n))
+
+        def timed(fn, reps):
+            fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(reps):
+                fn()
+            b.record(stream)
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        with torch.no_grad():
+            dense_ms = timed(lambda: torch.nn.functional.scaled_dot_product_attention(Q, K, V), 1 if n > 200000 else 3)
+        n_kc = base.n_kc
+        for label, keep in (("64 blocks", min(64, n_kc)), ("10 %", max(1, round(0.1 * n_kc)))):
+            w = base.scaled(keep=keep)
+            plan = binding.Plan(binding.problem_from_workload(w), dev)
+            cluster_ms = timed(lambda: plan.cluster_qk(Q, K, V), reps)
+            select_ms = timed(lambda: plan.select_blocks(), reps)
+            attn_ms = timed(lambda: plan.cluster_attention_fwd(want_lse=False), reps)
+            eager_ms = timed(lambda: plan.forward(Q, K, V), reps)
+            assert all(v == 0 for v in plan.last_status().values())
+            # the same step captured once and replayed: no per-launch host cost
+            graph_ms = None
+            try:
+                side = torch.cuda.Stream()
+                side.wait_stream(stream)
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.stream(side):
+                    plan.forward(Q, K, V, stream=side)
+                    side.synchronize()
+                    with torch.cuda.graph(graph, stream=side):
+                        plan.forward(Q, K, V, stream=side)
+                stream.wait_stream(side)
+                graph_ms = timed(graph.replay, reps)
+                del graph
+            except Exception as exc:  # noqa: BLE001
+                graph_ms = f"capture failed: {str(exc)[:120]}"
+            points.append({"n": n, "kept": label, "keep": keep, "cluster_qk_ms": cluster_ms, "select_ms": select_ms,
+                           "attn_ms": attn_ms, "step_ms": eager_ms, "graph_step_ms": graph_ms, "dense_sdpa_ms": dense_ms,
+                           "speedup_vs_dense": dense_ms / eager_ms})
+            del plan
+        del Q, K, V
+        torch.cuda.empty_cache()
+        n *= 2
+    print(json.dumps({"metric": METRIC, "workload": "scaling", "heads": heads, "head_dim": 64, "cluster": 128,
+                      "points": points}))
+
+
 def main():
     args = parse_args()
     if args.sweep:
         run_sweep(args)
         return
+    if args.scaling:
+        run_scaling(args)
+        return
     from paper_2608_26965_b200 import inputs
     w = inputs.WORKLOADS[args.workload]
     if args.heads:
         w = w.scaled(heads=args.heads)
+    if args.n_q or args.n_k:
+        w = w.scaled(n_q=args.n_q or w.n_q, n_k=args.n_k or w.n_k)
     if args.impl == "reference":
         run_reference(args, w)
     else:
