@@ -169,12 +169,11 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     // global principal components of both transformed sets (Section 3.2.1)
     CA_TRY(launch_eigh(w.cov, 2 * P, D, w.basis, w.basis32, nullptr, st));
     double* EK = w.basis;
-    double* EQ = w.basis + (size_t)P * DD;
     const float* EQ32 = w.basis32 + (size_t)P * DD;
     // keys: Y = (K - kbar) F_q E_K ; queries: Y = (r(q) - mean) E_Q
     CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, 0, w.WK, w.WK32, st));
-    CA_TRY(launch_bias(w.sumK, w.WK, P, D, p->n_k, w.biasK, st));
-    CA_TRY(launch_bias(w.sumQp, EQ, P, D, p->n_q, w.biasQ, st));
+    CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st));
+    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, st));
     if (tc) {
       CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr,
                                  w.wt_hi, w.wt_lo, w.status, st));

@@ -1,0 +1,376 @@
+// Batched symmetric eigendecomposition of d x d matrices (d = 64, 128), one CTA
+// per matrix: Householder reduction to tridiagonal form, then the implicit-shift
+// QL iteration on the tridiagonal matrix (principal-component bases of
+// Section 3.2.1).  Working precision float32: the bases only feed fp32 split
+// coordinates.
+//
+// Phase 1 (all 8d threads, two barriers per reflector): for k = 0 .. d-3 the
+// reflector H_k = I - beta v v^T annihilates A[k+2.., k]; the trailing block is
+// updated as A - v w^T - w v^T with p = beta A v, w = p - (beta/2)(v.p) v, and
+// the transposed accumulated transform Qt <- H_k Qt is updated in the same two
+// stages.  Thread (r, q) = (tid / 8, tid % 8) keeps entries 4 (q + 8 t) + c of
+// row r of A and of column r of Qt in registers for the whole phase (the loops
+// are bound by instruction issue and latency, not by arithmetic); the eight
+// owners of row k+1 build the next reflector right after their update, inside
+// their warp, so no third barrier is needed.
+//
+// Phase 2: warp 0 runs the QL iteration on (diag, sub-diag) -- the search for a
+// negligible sub-diagonal entry uses all lanes, the rotation chase is one
+// dependent chain on lane 0 -- and hands each chase's rotations through a
+// double-buffered list to d consumer threads, which apply them to the rows of
+// Qt (thread t owns column t), pipelined with the next chase by named barriers.
+//
+// Output: eigenvectors as columns, descending eigenvalue, each column's entry of
+// largest magnitude (lowest row on ties) made positive.
+#include "kernels.h"
+
+namespace ca {
+
+namespace {
+
+// barrier ids are immediates so that the kernel reserves only the barriers it names
+__device__ __forceinline__ void named_sync(int id, int count) {
+  switch (id) {
+    case 1: asm volatile("bar.sync 1, %0;" ::"r"(count) : "memory"); break;
+    case 2: asm volatile("bar.sync 2, %0;" ::"r"(count) : "memory"); break;
+    case 3: asm volatile("bar.sync 3, %0;" ::"r"(count) : "memory"); break;
+    default: asm volatile("bar.sync 4, %0;" ::"r"(count) : "memory"); break;
+  }
+}
+__device__ __forceinline__ void named_arrive(int id, int count) {
+  switch (id) {
+    case 1: asm volatile("bar.arrive 1, %0;" ::"r"(count) : "memory"); break;
+    case 2: asm volatile("bar.arrive 2, %0;" ::"r"(count) : "memory"); break;
+    case 3: asm volatile("bar.arrive 3, %0;" ::"r"(count) : "memory"); break;
+    default: asm volatile("bar.arrive 4, %0;" ::"r"(count) : "memory"); break;
+  }
+}
+
+constexpr int kBarFull = 1;    // ids 1, 2: a rotation list is ready
+constexpr int kBarEmpty = 3;   // ids 3, 4: a rotation list has been applied
+constexpr int kMaxQlIterations = 64;
+
+}  // namespace
+
+template <int D>
+__global__ void __launch_bounds__(8 * D)
+eigh_tql_kernel(const double* __restrict__ A_in, double* __restrict__ out64, float* __restrict__ out32,
+                double* __restrict__ evals_out) {
+  constexpr int NT = 8 * D, LDA = D + 4;
+  constexpr int CH = D / 32;            // float4 chunks of a row per thread
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* A = reinterpret_cast<float*>(smem_raw);       // [D][LDA]
+  float* Qt = A + D * LDA;                             // [D][LDA]   written after phase 1; rows become the eigenvectors
+  float* vbuf = Qt + D * LDA;                          // [2][D]     reflector, zero above its first entry
+  float* pbuf = vbuf + 2 * D;                          // [D]
+  float* ubuf = pbuf + D;                              // [D]
+  float2* de = reinterpret_cast<float2*>(ubuf + D);    // [D]        (diagonal i, sub-diagonal coupling i and i+1)
+  float* beta = ubuf + 3 * D;                          // [2] (+2)
+  float* rot = beta + 4;                               // [2][2D]    (c, s) of the rotation of rows (i, i+1) at 2i
+  int* hdr = reinterpret_cast<int*>(rot + 4 * D);      // [2][4]     highest i, lowest i, end marker
+  __shared__ double s_scale;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int r = tid >> 3, q = tid & 7;
+  const double* Ain = A_in + (size_t)blockIdx.x * D * D;
+
+  // scale so that the largest diagonal entry is 1 (eigenvectors unchanged, eigenvalues scaled back)
+  if (tid < 32) {
+    double mx = 0.0;
+    for (int i = tid; i < D; i += 32) mx = fmax(mx, fabs(Ain[i * D + i]));
+    for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (tid == 0) s_scale = mx > 0.0 ? mx : 1.0;
+  }
+  __syncthreads();
+  const double a_scale = s_scale;
+  {
+    const double inv = 1.0 / a_scale;
+    for (int e = tid; e < D * D; e += NT) {
+      const int i = e / D, j = e % D;
+      A[i * LDA + j] = (float)(0.5 * (Ain[i * D + j] + Ain[j * D + i]) * inv);   // symmetrise on load
+    }
+  }
+  __syncthreads();
+
+  // This thread's parts of row r of A and of column r of Qt (the same index set: entries
+  // 4 (q + 8 t) + c), kept in registers for the whole reduction.  Qt starts as the identity.
+  float areg[CH][4], qreg[CH][4];
+#pragma unroll
+  for (int t = 0; t < CH; ++t) {
+    const int j0 = 4 * (q + 8 * t);
+    const float4 a = *reinterpret_cast<const float4*>(&A[r * LDA + j0]);
+    areg[t][0] = a.x; areg[t][1] = a.y; areg[t][2] = a.z; areg[t][3] = a.w;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) qreg[t][c] = (j0 + c == r) ? 1.f : 0.f;
+  }
+
+  // Iteration k applies reflector k (two stages) and then builds reflector k+1; k = -1 only builds.
+  for (int k = -1; k < D - 2; ++k) {
+    const int m0 = k + 1;
+    const float* v = vbuf + (k & 1) * D;
+    const float b = k >= 0 ? beta[k & 1] : 0.f;            // uniform over the CTA
+    const int t_first = m0 >> 5;                           // chunks below it hold only zeros of v
+    if (b != 0.f) {
+      // p = beta A v (rows >= m0), u = beta v^T Qt
+      float ps = 0.f, us = 0.f;
+#pragma unroll
+      for (int t = 0; t < CH; ++t) {
+        if (t < t_first) continue;
+        const float4 vv = *reinterpret_cast<const float4*>(&v[4 * (q + 8 * t)]);
+        ps = fmaf(areg[t][0], vv.x, ps); ps = fmaf(areg[t][1], vv.y, ps);
+        ps = fmaf(areg[t][2], vv.z, ps); ps = fmaf(areg[t][3], vv.w, ps);
+        us = fmaf(qreg[t][0], vv.x, us); us = fmaf(qreg[t][1], vv.y, us);
+        us = fmaf(qreg[t][2], vv.z, us); us = fmaf(qreg[t][3], vv.w, us);
+      }
+      ps += __shfl_xor_sync(0xffffffffu, ps, 1); us += __shfl_xor_sync(0xffffffffu, us, 1);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 2); us += __shfl_xor_sync(0xffffffffu, us, 2);
+      ps += __shfl_xor_sync(0xffffffffu, ps, 4); us += __shfl_xor_sync(0xffffffffu, us, 4);
+      if (q == 0) {
+        pbuf[r] = (r >= m0) ? b * ps : 0.f;
+        ubuf[r] = b * us;
+      }
+    }
+    __syncthreads();
+    if (b != 0.f) {
+      float kp = 0.f;
+      for (int j = lane; j < D; j += 32) kp = fmaf(v[j], pbuf[j], kp);
+      for (int o = 16; o > 0; o >>= 1) kp += __shfl_xor_sync(0xffffffffu, kp, o);
+      const float K = 0.5f * b * kp;
+      const float v_r = v[r];
+      const float w_r = pbuf[r] - K * v_r;
+      const float u_r = ubuf[r];
+      const bool live_row = r >= m0;
+#pragma unroll
+      for (int t = 0; t < CH; ++t) {
+        if (t < t_first) continue;
+        const int j0 = 4 * (q + 8 * t);
+        const float4 vv = *reinterpret_cast<const float4*>(&v[j0]);
+        if (live_row) {
+          const float4 pp = *reinterpret_cast<const float4*>(&pbuf[j0]);
+          areg[t][0] -= v_r * (pp.x - K * vv.x) + w_r * vv.x;
+          areg[t][1] -= v_r * (pp.y - K * vv.y) + w_r * vv.y;
+          areg[t][2] -= v_r * (pp.z - K * vv.z) + w_r * vv.z;
+          areg[t][3] -= v_r * (pp.w - K * vv.w) + w_r * vv.w;
+        }
+        qreg[t][0] = fmaf(-vv.x, u_r, qreg[t][0]); qreg[t][1] = fmaf(-vv.y, u_r, qreg[t][1]);
+        qreg[t][2] = fmaf(-vv.z, u_r, qreg[t][2]); qreg[t][3] = fmaf(-vv.w, u_r, qreg[t][3]);
+      }
+    }
+  // Reflector for row kn = k+1, built by the whole warp that holds the row's eight owners
+    // (the other groups of the warp go through the shuffles and write nothing).
+    const int kn = k + 1;
+    if (kn < D - 2 && warp == (kn >> 2)) {
+      const int mn = kn + 1;
+      float sig = 0.f, c_x0 = 0.f, c_kk = 0.f;              // candidates for A[kn][mn], A[kn][kn]
+#pragma unroll
+      for (int t = 0; t < CH; ++t) {
+        const int j0 = 4 * (q + 8 * t);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          const float a = areg[t][c];
+          const float xv = (j0 + c >= mn) ? a : 0.f;
+          sig = fmaf(xv, xv, sig);
+          if (j0 + c == mn) c_x0 = a;
+          if (j0 + c == kn) c_kk = a;
+        }
+      }
+      sig += __shfl_xor_sync(0xffffffffu, sig, 1);
+      sig += __shfl_xor_sync(0xffffffffu, sig, 2);
+      sig += __shfl_xor_sync(0xffffffffu, sig, 4);
+      const float x0 = __shfl_sync(0xffffffffu, c_x0, (lane & 24) | ((mn >> 2) & 7));
+      const float akk = __shfl_sync(0xffffffffu, c_kk, (lane & 24) | ((kn >> 2) & 7));
+      if (r == kn) {
+        const float rest = sig - x0 * x0;
+        float bn = 0.f, alpha = x0, v0 = 0.f;
+        const bool reflect = rest > 1e-30f;       // already tridiagonal in this column otherwise
+        if (reflect) {
+          const float rt = sqrtf(sig);
+          alpha = x0 >= 0.f ? -rt : rt;
+          v0 = x0 - alpha;
+          bn = 1.f / (sig + fabsf(x0) * rt);
+        }
+        float* vn = vbuf + (kn & 1) * D;
+#pragma unroll
+        for (int t = 0; t < CH; ++t) {
+          const int j0 = 4 * (q + 8 * t);
+          float4 o;
+          o.x = (reflect && j0 + 0 >= mn) ? (j0 + 0 == mn ? v0 : areg[t][0]) : 0.f;
+          o.y = (reflect && j0 + 1 >= mn) ? (j0 + 1 == mn ? v0 : areg[t][1]) : 0.f;
+          o.z = (reflect && j0 + 2 >= mn) ? (j0 + 2 == mn ? v0 : areg[t][2]) : 0.f;
+          o.w = (reflect && j0 + 3 >= mn) ? (j0 + 3 == mn ? v0 : areg[t][3]) : 0.f;
+          *reinterpret_cast<float4*>(&vn[j0]) = o;
+        }
+        if (q == 0) {
+          beta[kn & 1] = bn;
+          de[kn] = make_float2(akk, alpha);
+        }
+      }
+    }
+    __syncthreads();
+  }
+  // the last 2 x 2 block; the accumulated transform goes to shared memory for the rotations
+  if (q == 7 && r == D - 2) de[D - 2] = make_float2(areg[CH - 1][2], areg[CH - 1][3]);
+  if (q == 7 && r == D - 1) de[D - 1] = make_float2(areg[CH - 1][3], 0.f);
+#pragma unroll
+  for (int t = 0; t < CH; ++t)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) Qt[(4 * (q + 8 * t) + c) * LDA + r] = qreg[t][c];
+  __syncthreads();
+
+  // ---- implicit-shift QL on the tridiagonal matrix; rotations applied to the rows of Qt
+  constexpr int kParties = 32 + D;
+  if (warp == 0) {
+    int bsel = 0;
+    const float eps = 6e-8f;
+    for (int l = 0; l < D; ++l) {
+      for (int iter = 0; iter < kMaxQlIterations; ++iter) {
+        // first m >= l whose sub-diagonal entry is negligible (m = D-1 if none)
+        int m = D - 1;
+        for (int base = l; base < D - 1; base += 32) {
+          const int idx = base + lane;
+          bool small = false;
+          if (idx < D - 1) {
+            const float2 a = de[idx];
+            small = fabsf(a.y) <= eps * (fabsf(a.x) + fabsf(de[idx + 1].x));
+          }
+          const unsigned bal = __ballot_sync(0xffffffffu, small);
+          if (bal) { m = base + __ffs(bal) - 1; break; }
+        }
+        if (m == l) break;
+        named_sync(kBarEmpty + bsel, kParties);            // the list's previous contents have been applied
+        if (lane == 0) {
+          float2* rt = reinterpret_cast<float2*>(rot + bsel * 2 * D);
+          const float2 top = de[l];
+          float g = (de[l + 1].x - top.x) / (2.f * top.y);
+          float rr = sqrtf(fmaf(g, g, 1.f));
+          g = de[m].x - top.x + top.y / (g + (g >= 0.f ? rr : -rr));
+          float s = 1.f, c = 1.f, p = 0.f;
+          bool under = false;
+          int i = m - 1;
+          float2 cur = de[i];              // (d_i, e_i)
+          float d_i1 = de[i + 1].x;
+          for (; i >= l; --i) {
+            // operands of the next rotation, fetched ahead of the dependent chain
+            const float2 nxt = de[i > l ? i - 1 : l];
+            const float f = s * cur.y, bb = c * cur.y;
+            const float r2 = fmaf(f, f, g * g);
+            float rinv;
+            asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rinv) : "f"(r2));
+            const float p_old = p, d_old = d_i1;
+            s = f * rinv;
+            c = g * rinv;
+            g = d_i1 - p;
+            rr = fmaf(c, bb + bb, (cur.x - g) * s);
+            p = s * rr;
+            de[i + 1] = make_float2(g + p, r2 * rinv);       // new d_{i+1}; e_{i+1} = hypot(f, g)
+            g = fmaf(c, rr, -bb);
+            rt[i] = make_float2(c, s);
+            // The chase has died out (f = g = 0): deflate here.  Tested after the rotation has been
+            // formed so that the test is off the dependent chain; its results are discarded.
+            if (r2 < 1e-36f) {
+              de[i + 1] = make_float2(d_old - p_old, 0.f);
+              de[m].y = 0.f;
+              under = true;
+              break;
+            }
+            d_i1 = cur.x;          // d_i is the next step's d_{i+1}; it has not been modified yet
+            cur = nxt;
+          }
+          int lo = l;
+          if (!under) {
+            de[l] = make_float2(top.x - p, g);
+            de[m].y = 0.f;
+          } else {
+            lo = i + 1;
+          }
+          hdr[bsel * 4 + 0] = m - 1;
+          hdr[bsel * 4 + 1] = lo;
+          hdr[bsel * 4 + 2] = 0;
+        }
+        __syncwarp();
+        __threadfence_block();
+        named_arrive(kBarFull + bsel, kParties);
+        bsel ^= 1;
+      }
+    }
+    named_sync(kBarEmpty + bsel, kParties);
+    if (lane == 0) hdr[bsel * 4 + 2] = 1;                    // end marker
+    __syncwarp();
+    __threadfence_block();
+    named_arrive(kBarFull + bsel, kParties);
+    named_sync(kBarEmpty + (bsel ^ 1), kParties);            // the other list's last hand-back
+  } else if (tid < 32 + D) {
+    const int t = tid - 32;
+    named_arrive(kBarEmpty + 0, kParties);                   // both lists start out free
+    named_arrive(kBarEmpty + 1, kParties);
+    int bsel = 0;
+    while (true) {
+      named_sync(kBarFull + bsel, kParties);
+      if (hdr[bsel * 4 + 2]) break;
+      const int hi = hdr[bsel * 4 + 0], lo = hdr[bsel * 4 + 1];
+      const float* rt = rot + bsel * 2 * D;
+      float carry = Qt[(hi + 1) * LDA + t];
+      for (int i = hi; i >= lo; --i) {
+        const float c = rt[2 * i], s = rt[2 * i + 1];
+        const float zi = Qt[i * LDA + t];
+        Qt[(i + 1) * LDA + t] = fmaf(s, zi, c * carry);
+        carry = fmaf(c, zi, -s * carry);
+      }
+      Qt[lo * LDA + t] = carry;
+      __threadfence_block();
+      named_arrive(kBarEmpty + bsel, kParties);
+      bsel ^= 1;
+    }
+  }
+  __syncthreads();
+
+  // ---- order, sign and write out
+  double* lam = reinterpret_cast<double*>(A);                // A is free now
+  int* rank_of = reinterpret_cast<int*>(lam + D);
+  float* sign_of = reinterpret_cast<float*>(rank_of + D);
+  if (tid < D) lam[tid] = (double)de[tid].x * a_scale;
+  __syncthreads();
+  if (tid < D) {
+    const double mine = lam[tid];
+    int rank = 0;
+    for (int k = 0; k < D; ++k) {
+      const double other = lam[k];
+      rank += (other > mine) || (other == mine && k < tid);
+    }
+    float best = -1.f, sgn = 1.f;
+    for (int i = 0; i < D; ++i) {
+      const float v = Qt[tid * LDA + i];
+      if (fabsf(v) > best) { best = fabsf(v); sgn = (v < 0.f) ? -1.f : 1.f; }
+    }
+    rank_of[tid] = rank;
+    sign_of[tid] = sgn;
+    if (evals_out) evals_out[(size_t)blockIdx.x * D + rank] = mine;
+  }
+  __syncthreads();
+  double* o64 = out64 + (size_t)blockIdx.x * D * D;
+  float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
+  for (int e = tid; e < D * D; e += NT) {
+    const int k = e / D, i = e % D;           // eigenvector k, component i
+    const float v = sign_of[k] * Qt[k * LDA + i];
+    o64[i * D + rank_of[k]] = (double)v;
+    if (o32) o32[i * D + rank_of[k]] = v;
+  }
+}
+
+int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
+                cudaStream_t st) {
+  const size_t smem = sizeof(float) * ((size_t)2 * D * (D + 4) + 2 * D + 4 * D + 4 + 4 * D) + 8 * sizeof(int);
+  if (D == 64) {
+    auto k = eigh_tql_kernel<64>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<count, 8 * 64, smem, st>>>(A, out64, out32, evals);
+  } else {
+    auto k = eigh_tql_kernel<128>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    k<<<count, 8 * 128, smem, st>>>(A, out64, out32, evals);
+  }
+  CA_LAUNCH_CHECK();
+  return CA_OK;
+}
+
+}  // namespace ca

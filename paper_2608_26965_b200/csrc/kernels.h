@@ -33,7 +33,7 @@ int launch_covariance(const double* gram, const double* sum, int P, int D, int n
 int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
                         double* C, float* C32, cudaStream_t st);
 int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st);
-int launch_bias(const double* sum, const double* W, int P, int D, int n, float* bias, cudaStream_t st);
+int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st);
 
 // split.cu
 int split_levels_for(int n, int c);
