@@ -31,13 +31,8 @@ using namespace ptx;
 constexpr int kTcThreads = 192;
 constexpr int kTile = 128;                 // query rows per CTA, key rows per tile
 constexpr int kHalf = 64;                  // keys per half-step
-constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D)
+constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D) (+16 row-sum columns, d = 64)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-#ifndef CA_POLY_MODE
-#define CA_POLY_MODE 0
-#endif
-// share of the exponentials evaluated by polynomial on the FMA pipe: 0, 1/4, 3/8, 1/2
-constexpr int kPolyMode = CA_POLY_MODE;
 
 template <int D>
 struct TcCfg {
@@ -49,7 +44,12 @@ struct TcCfg {
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + STAGES * TILE_BYTES;
-  static constexpr int OFF_BIAS = OFF_V + STAGES * TILE_BYTES;     // 4 x 64 floats
+  // d = 64: the product P V is taken with 16 extra value columns that hold 1.0, so that the
+  // tensor core also delivers the row sums of P (the accumulator has no room for them at d = 128)
+  static constexpr bool ROWSUM_MMA = (D == 64);
+  static constexpr int PV_N = ROWSUM_MMA ? D + 16 : D;
+  static constexpr int OFF_ONES = OFF_V + STAGES * TILE_BYTES;      // 64 key rows x 128 bytes of bf16 ones
+  static constexpr int OFF_BIAS = OFF_ONES + (ROWSUM_MMA ? kHalf * 128 : 0);     // 4 x 64 floats
   static constexpr int OFF_BAR = OFF_BIAS + 4 * kHalf * 4;
   static constexpr int NUM_BARS = 8 + 4 * STAGES;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;           // tmem base, abort flag
@@ -97,6 +97,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
   unsigned* bitmap = reinterpret_cast<unsigned*>(smem + C::OFF_BITMAP);
+  // member counts of the selected clusters, in list order: looked up every half-step, so they are
+  // fetched from global memory once instead of sitting on each half-step's critical path
+  uint16_t* members_of = reinterpret_cast<uint16_t*>(bitmap + prm.bitmap_words);
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = blockIdx.y;
@@ -115,7 +118,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   if (tid == 0) {
     mbar_init(b_q_full, 1);
     mbar_init(b_o_done, 1);
-    for (int b = 0; b < 2; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 128); mbar_init(b_pv_done(b), 1); }
+    for (int b = 0; b < 2; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 4); mbar_init(b_pv_done(b), 1); }
     for (int s = 0; s < C::STAGES; ++s) {
       mbar_init(b_k_full(s), 1); mbar_init(b_k_empty(s), 1);
       mbar_init(b_v_full(s), 1); mbar_init(b_v_empty(s), 1);
@@ -129,6 +132,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int pn = e / ((kTile - q_rows) * 8), rem = e % ((kTile - q_rows) * 8);
       *reinterpret_cast<uint4*>(smem + C::OFF_Q + pn * C::PANEL_BYTES + q_rows * 128 + rem * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
+    fence_proxy_async();
+  }
+  if (C::ROWSUM_MMA) {
+    for (int e = tid; e < kHalf * 8; e += kTcThreads)
+      *reinterpret_cast<uint4*>(smem + C::OFF_ONES + e * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
     fence_proxy_async();
   }
   if (warp == 1) {                       // this warp owns the TMEM allocation
@@ -192,7 +200,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // ------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
-      constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, D, 0, 1);
+      constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
       bool ok = mbar_wait(b_q_full, 0, abort_flag, prm.status);
       // load index of half-step u (the shared-memory slot is the load index modulo the stages)
       auto load_of = [&](int u) { return u < 2 * sel_tiles ? u >> 1 : sel_tiles + (u - 2 * sel_tiles); };
@@ -233,7 +241,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
         for (int ks = 0; ks < kHalf / 16; ++ks) {
           // V is MN-major: 16 key rows (2048 bytes) per step; panels along d
-          const uint64_t bd = smem_desc_sw128(vt + ks * 2048, C::PANEL_BYTES, 1024);
+          // with the row-sum columns the panel after the values is the block of ones
+          const uint32_t next_panel = C::ROWSUM_MMA ? (s_base + C::OFF_ONES) - vt : (uint32_t)C::PANEL_BYTES;
+          const uint64_t bd = smem_desc_sw128(vt + ks * 2048, next_panel, 1024);
           mma_ts(tmem_o, tmem_s + b * kHalf + ks * 8, bd, idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
         }
         mma_commit(b_pv_done(b));
@@ -251,11 +261,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int32_t* cnt = prm.count_k + (size_t)p * prm.n_kc;
     for (int w = st; w < prm.bitmap_words; w += 128) bitmap[w] = 0u;
     asm volatile("bar.sync 1, 128;" ::: "memory");
-    if (prm.compensate)
-      for (int e = st; e < keep; e += 128) atomicOr(&bitmap[sel[e] >> 5], 1u << (sel[e] & 31));
+    for (int e = st; e < keep; e += 128) {
+      const int j = sel[e];
+      members_of[e] = (uint16_t)min(cnt[j], prm.c_k);
+      if (prm.compensate) atomicOr(&bitmap[j >> 5], 1u << (j & 31));
+    }
     asm volatile("bar.sync 1, 128;" ::: "memory");
 
     float m_ref = -INFINITY, l_run = 0.f;
+    const float inv_scale_log2 = 1.0f / prm.scale_log2;
+    const int ck_shift = __ffs(prm.c_k) - 1;
     bool ok = true;
     for (int u = 0; u < steps && ok; ++u) {
       const int b = u & 1;
@@ -266,23 +281,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // four buffers: a thread can run at most two half-steps ahead of the slowest one
       float* bz = bias + (u & 3) * kHalf;
       if (u < 2 * sel_tiles) {
+        // cluster sizes are powers of two: positions are split with shifts and masks
         const int t = u >> 1;
         bool use = true;
         if (prm.c_k >= kTile) {
-          const int per = prm.c_k / kTile;
-          const int members = cnt[sel[t / per]];
-          const int first = (t % per) * kTile + b * kHalf;      // row of this half-step's first column
+          const int e = t >> (ck_shift - 7);                      // c_k / 128 tiles per cluster
+          const int members = members_of[e];
+          const int first = ((t << 7) & (prm.c_k - 1)) + b * kHalf;   // row of this half-step's first column
           masked = members < first + kHalf;
           use = first + (st & 63) < members;
         } else {
           const int col0 = t * kTile + b * kHalf;                // position in the list of selected rows
-          const int per = prm.c_k >= kHalf ? 1 : kHalf / prm.c_k;
-          for (int x = 0; x < per; ++x) {
-            const int e = (col0 + x * prm.c_k) / prm.c_k;
-            if (e >= keep || cnt[sel[e]] < prm.c_k) masked = true;
-          }
-          const int e = (col0 + (st & 63)) / prm.c_k;
-          use = e < keep && ((col0 + (st & 63)) % prm.c_k) < cnt[sel[min(e, keep - 1)]];
+          const int e_first = col0 >> ck_shift, e_last = (col0 + kHalf - 1) >> ck_shift;
+          for (int e = e_first; e <= e_last; ++e)
+            if (e >= keep || members_of[e] < prm.c_k) masked = true;
+          const int e = (col0 + (st & 63)) >> ck_shift;
+          use = e < keep && ((col0 + (st & 63)) & (prm.c_k - 1)) < members_of[min(e, keep - 1)];
         }
         if (masked && st < kHalf) bz[st] = use ? 0.f : -INFINITY;
       } else {
@@ -298,38 +312,43 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tc_fence_after();
       if (quarter * 32 >= q_rows) {          // this warp's rows are padding of a 64-row query cluster
         tc_fence_before();
-        mbar_arrive(b_p_ready(b));
+        __syncwarp();
+        if (lane == 0) mbar_arrive(b_p_ready(b));
         continue;
       }
-      // ---- pass 1: row maximum over the 64 columns
-      uint32_t ra[32], rb[32];
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
-      auto reduce_max = [&](const uint32_t (&r)[32], int c4) {
-        if (masked) {
+      // The loops over the two 32-column chunks are kept rolled: the body of a half-step is
+      // executed by every softmax warp of both resident CTAs at different places, and an unrolled
+      // body does not stay in the instruction cache.
+      // ---- masked / weighted half-steps (short clusters, centroid columns): the additive term is
+      // folded into the scores in tensor memory first, so that the common path below has no bias
+      if (masked) {
+#pragma unroll 1
+        for (int c4 = 0; c4 < 2; ++c4) {
+          uint32_t r[32];
+          tmem_ld32(t_s + c4 * 32, r);
+          tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            mx0 = fmaxf(mx0, fmaf(__uint_as_float(r[j]), prm.scale_log2, bz[c4 * 32 + j]));
-            mx1 = fmaxf(mx1, fmaf(__uint_as_float(r[j + 1]), prm.scale_log2, bz[c4 * 32 + j + 1]));
-            mx2 = fmaxf(mx2, fmaf(__uint_as_float(r[j + 2]), prm.scale_log2, bz[c4 * 32 + j + 2]));
-            mx3 = fmaxf(mx3, fmaf(__uint_as_float(r[j + 3]), prm.scale_log2, bz[c4 * 32 + j + 3]));
-          }
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            mx0 = fmaxf(mx0, fmaxf(__uint_as_float(r[j]), __uint_as_float(r[j + 1])));
-            mx1 = fmaxf(mx1, fmaxf(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])));
-            mx2 = fmaxf(mx2, fmaxf(__uint_as_float(r[j + 4]), __uint_as_float(r[j + 5])));
-            mx3 = fmaxf(mx3, fmaxf(__uint_as_float(r[j + 6]), __uint_as_float(r[j + 7])));
-          }
+          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(fmaf(bz[c4 * 32 + j], inv_scale_log2, __uint_as_float(r[j])));
+          tmem_st32(t_s + c4 * 32, r);
         }
-      };
-      tmem_ld32(t_s, ra);
-      tmem_ld32(t_s + 32, rb);
-      tmem_wait_ld();
-      reduce_max(ra, 0);
-      reduce_max(rb, 1);
-      float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
-      if (!masked) tmax *= prm.scale_log2;
+        tmem_wait_st();
+      }
+      // ---- pass 1: row maximum over the 64 columns
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll 1
+      for (int c4 = 0; c4 < 2; ++c4) {
+        uint32_t r[32];
+        tmem_ld32(t_s + c4 * 32, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; j += 8) {
+          mx0 = max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          mx1 = max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          mx2 = max3(mx2, __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+          mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+        }
+      }
+      const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
       // raise the reference maximum only when a half-step exceeds it by the threshold
       const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
       if (__any_sync(0xffffffffu, raise)) {
@@ -338,13 +357,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           alpha = (m_ref == -INFINITY) ? 0.f : ex2_approx(m_ref - tmax);
           m_ref = tmax;
         }
-        l_run *= alpha;
+        if (!C::ROWSUM_MMA) l_run *= alpha;
         if (u > 0) {
           // S(u) complete means every product up to PV(u-2) is complete; PV(u-1) may still run
           ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done(b ^ 1), ((u - 1) >> 1) & 1, abort_flag, prm.status));
           if (!ok) break;
           tc_fence_after();
-#pragma unroll
+#pragma unroll 1
           for (int c4 = 0; c4 < D / 32; ++c4) {
             uint32_t o[32];
             tmem_ld32(tmem_o + lane_addr + c4 * 32, o);
@@ -353,43 +372,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
             tmem_st32(tmem_o + lane_addr + c4 * 32, o);
           }
+          if (C::ROWSUM_MMA) {
+            const uint32_t l = tmem_ld1(tmem_o + lane_addr + D);
+            tmem_wait_ld();
+            tmem_st1(tmem_o + lane_addr + D, __float_as_uint(__uint_as_float(l) * alpha));
+          }
         }
       }
-      // ---- pass 2: P = exp2(x - m), packed to bf16 over the first 32 columns of the buffer
+      // ---- pass 2: P = exp2(x - m), packed to bf16 over the first 32 columns of the buffer (chunk 0
+      // goes to columns [0,16) while chunk 1 is still unread in [32,64); chunk 1 to [16,32))
       const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
-      auto exp_chunk = [&](const uint32_t (&r)[32], int c4) {
-        // three sweeps over 32 independent elements (scale, exponential, sum + pack) so that the
-        // instruction stream never waits on a result produced a few instructions earlier
+#pragma unroll 1
+      for (int c4 = 0; c4 < 2; ++c4) {
+        uint32_t r[32];
+        tmem_ld32(t_s + c4 * 32, r);
+        tmem_wait_ld();
+        // The special-function unit takes one exponential per 8 cycles and sub-core: the other
+        // work of the chunk (scaling, sums, packing) is interleaved with the exponentials in groups
+        // of four, two groups behind, so that it issues in the shadow of that unit.
         float x[32];
-        if (masked) {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, bz[c4 * 32 + j] + neg_m);
-        } else {
-#pragma unroll
-          for (int j = 0; j < 32; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
-        }
-#pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const bool poly = (kPolyMode >= 1 && (j & 3) == 3) || (kPolyMode == 3 && (j & 3) == 1) ||
-                            (kPolyMode == 2 && (j & 7) == 1);
-          x[j] = poly ? ex2_poly(x[j]) : ex2_approx(x[j]);
-        }
         uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          ps0 += x[j]; ps1 += x[j + 1]; ps2 += x[j + 2]; ps3 += x[j + 3];
-          pk[j / 2] = pack_bf16x2(x[j], x[j + 1]);
-          pk[j / 2 + 1] = pack_bf16x2(x[j + 2], x[j + 3]);
+        for (int j = 0; j < 8; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
+#pragma unroll
+        for (int g = 0; g < 10; ++g) {
+          if (g < 8) {
+#pragma unroll
+            for (int j = 4 * g; j < 4 * g + 4; ++j) x[j] = ex2_approx(x[j]);
+          }
+          if (g + 2 < 8) {
+#pragma unroll
+            for (int j = 4 * (g + 2); j < 4 * (g + 2) + 4; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
+          }
+          if (g >= 2) {
+            const int j = 4 * (g - 2);
+            if (!C::ROWSUM_MMA) { ps0 += x[j]; ps1 += x[j + 1]; ps2 += x[j + 2]; ps3 += x[j + 3]; }
+            pk[j / 2] = pack_bf16x2(x[j], x[j + 1]);
+            pk[j / 2 + 1] = pack_bf16x2(x[j + 2], x[j + 3]);
+          }
         }
-        tmem_st16(t_s + c4 * 16, pk);       // both chunks are in registers: the stores cannot clobber unread S
-      };
-      exp_chunk(ra, 0);
-      exp_chunk(rb, 1);
-      l_run += (ps0 + ps1) + (ps2 + ps3);
+        tmem_st16(t_s + c4 * 16, pk);
+      }
+      if (!C::ROWSUM_MMA) l_run += (ps0 + ps1) + (ps2 + ps3);
+      // one arrival per warp: 128 arrivals on one barrier word would be serialised in shared memory
       tmem_wait_st();
       tc_fence_before();
-      mbar_arrive(b_p_ready(b));
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_p_ready(b));
     }
 
     // epilogue: O / l, rows back to their original positions
@@ -399,6 +429,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int pos = qc * prm.c_q + half * kTile + row;
       const bool live = row < q_rows && pos < prm.n_q;  // rows of the padding are not written
       const int orig = live ? prm.perm_q[(size_t)p * prm.n_q + pos] : 0;
+      if (C::ROWSUM_MMA) {                               // the sums of the rounded probabilities
+        l_run = __uint_as_float(tmem_ld1(tmem_o + lane_addr + D));
+        tmem_wait_ld();
+      }
       const float inv = 1.f / l_run;
       __nv_bfloat16* out = prm.O + ((size_t)p * prm.n_q + orig) * D;
 #pragma unroll
@@ -504,7 +538,7 @@ size_t attn_tc_workspace_bytes(const ca_problem_t& pr) {
 template <int D>
 static int launch_tc_d(const CUtensorMap* maps, const TcParams& prm, dim3 grid, cudaStream_t st) {
   using C = TcCfg<D>;
-  const size_t smem = 1024 + C::OFF_BITMAP + (size_t)prm.bitmap_words * 4;
+  const size_t smem = 1024 + C::OFF_BITMAP + (size_t)prm.bitmap_words * 4 + (((size_t)prm.list_stride * 2 + 15) & ~(size_t)15);
   auto k = attn_tc_kernel<D>;
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   k<<<grid, kTcThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
