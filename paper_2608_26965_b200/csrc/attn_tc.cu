@@ -33,6 +33,10 @@ constexpr int kTile = 128;                 // query rows per CTA, key rows per t
 constexpr int kHalf = 64;                  // keys per half-step
 constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D) (+16 row-sum columns, d = 64)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+#ifndef CA_STAGGER_NS
+#define CA_STAGGER_NS 400
+#endif
+constexpr unsigned kStaggerNs = CA_STAGGER_NS;
 
 template <int D>
 struct TcCfg {
@@ -48,10 +52,14 @@ struct TcCfg {
   // tensor core also delivers the row sums of P (the accumulator has no room for them at d = 128)
   static constexpr bool ROWSUM_MMA = (D == 64);
   static constexpr int PV_N = ROWSUM_MMA ? D + 16 : D;
+  // d = 64: tensor memory also has room for the query tile (32 columns of bf16 pairs), so Q K^T
+  // reads its A operand there instead of re-reading 4 KB of shared memory per instruction
+  static constexpr bool Q_IN_TMEM = (D == 64);
+  static constexpr int TMEM_Q = kTile + PV_N;               // first column of the query tile
   static constexpr int OFF_ONES = OFF_V + STAGES * TILE_BYTES;      // 64 key rows x 128 bytes of bf16 ones
   static constexpr int OFF_BIAS = OFF_ONES + (ROWSUM_MMA ? kHalf * 128 : 0);     // 4 x 64 floats
   static constexpr int OFF_BAR = OFF_BIAS + 4 * kHalf * 4;
-  static constexpr int NUM_BARS = 8 + 4 * STAGES;
+  static constexpr int NUM_BARS = 9 + 4 * STAGES;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;           // tmem base, abort flag
   static constexpr int OFF_BITMAP = OFF_MISC + 16;
 };
@@ -87,6 +95,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   float* bias = reinterpret_cast<float*>(smem + C::OFF_BIAS);
   const uint32_t bar0 = s_base + C::OFF_BAR;
   const uint32_t b_q_full = bar0, b_o_done = bar0 + 8;
+  const uint32_t b_q_tmem = bar0 + 8 * (C::NUM_BARS - 1);     // the query tile has been copied to tensor memory
   auto b_s_full = [&](int b) { return bar0 + 16 + 8 * b; };
   auto b_p_ready = [&](int b) { return bar0 + 32 + 8 * b; };
   auto b_pv_done = [&](int b) { return bar0 + 48 + 8 * b; };
@@ -117,6 +126,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   if (tid == 0) {
     mbar_init(b_q_full, 1);
+    mbar_init(b_q_tmem, 4);
     mbar_init(b_o_done, 1);
     for (int b = 0; b < 2; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 4); mbar_init(b_pv_done(b), 1); }
     for (int s = 0; s < C::STAGES; ++s) {
@@ -148,6 +158,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTile;
+  // Two CTAs share an SM and run the same loop at the same rate.  Started together they stay in
+  // phase: both sets of softmax warps want the special-function unit at the same time and both
+  // leave it idle at the same time.  The CTA that got the upper half of tensor memory starts a
+  // fraction of a half-step later, so that one CTA's exponentials run under the other's
+  // remaining work.
+  if ((tmem_base & 0xffffu) >= kTmemCols) __nanosleep(kStaggerNs);
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -202,8 +218,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
       bool ok = mbar_wait(b_q_full, 0, abort_flag, prm.status);
+      if (C::Q_IN_TMEM && ok) { ok = mbar_wait(b_q_tmem, 0, abort_flag, prm.status); tc_fence_after(); }
       // load index of half-step u (the shared-memory slot is the load index modulo the stages)
       auto load_of = [&](int u) { return u < 2 * sel_tiles ? u >> 1 : sel_tiles + (u - 2 * sel_tiles); };
+      const uint64_t q_desc0 = smem_desc_sw128(s_q, 16, 1024);
+      const uint64_t k_desc0 = smem_desc_sw128(s_k, 16, 1024);
       auto issue_s = [&](int u) {
         const int L = load_of(u), s = L % C::STAGES, b = u & 1;
         const bool centroid = u >= 2 * sel_tiles;
@@ -211,17 +230,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           if (!mbar_wait(b_k_full(s), (L / C::STAGES) & 1, abort_flag, prm.status)) return false;
           tc_fence_after();
         }
-        const uint32_t kt = s_k + s * C::TILE_BYTES;
+        // descriptors differ from a base one only in the start-address field (units of 16 bytes):
+        // the base descriptors are built once, the per-instruction part is an addition
         const int parts = centroid ? 2 : 1;               // centroid tile: hi rows 0-63, lo rows 64-127
         for (int g = 0; g < parts; ++g) {
           const uint32_t rows = (centroid ? g : b) * (kHalf * 128);   // 64 rows = 8192 bytes inside a panel
+          const uint64_t kd = k_desc0 + ((s * C::TILE_BYTES + rows) >> 4);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
-            const uint32_t off = (ks / 4) * C::PANEL_BYTES + (ks % 4) * 32;
-            const uint64_t a = smem_desc_sw128(s_q + off, 16, 1024);
-            const uint64_t bd = smem_desc_sw128(kt + rows + off, 16, 1024);
-            mma_ss(tmem_s + b * kHalf, a, bd, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            const uint32_t off16 = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
+            if (C::Q_IN_TMEM) mma_ts(tmem_s + b * kHalf, tmem_base + C::TMEM_Q + ks * 8, kd + off16, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            else mma_ss(tmem_s + b * kHalf, q_desc0 + off16, kd + off16, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
           }
         }
         if (centroid || b == 1) mma_commit(b_k_empty(s));
@@ -238,14 +258,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         const uint32_t vt = s_v + s * C::TILE_BYTES + (centroid ? 0 : b) * (kHalf * 128);
+        // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d.  With the row-sum
+        // columns the panel after the values is the block of ones, wherever the value tile sits.
+        const uint32_t next_panel = C::ROWSUM_MMA ? (s_base + C::OFF_ONES) - vt : (uint32_t)C::PANEL_BYTES;
+        const uint64_t vd = smem_desc_sw128(vt, next_panel, 1024);
+        const uint32_t p_cols = tmem_s + b * kHalf;
 #pragma unroll
-        for (int ks = 0; ks < kHalf / 16; ++ks) {
-          // V is MN-major: 16 key rows (2048 bytes) per step; panels along d
-          // with the row-sum columns the panel after the values is the block of ones
-          const uint32_t next_panel = C::ROWSUM_MMA ? (s_base + C::OFF_ONES) - vt : (uint32_t)C::PANEL_BYTES;
-          const uint64_t bd = smem_desc_sw128(vt + ks * 2048, next_panel, 1024);
-          mma_ts(tmem_o, tmem_s + b * kHalf + ks * 8, bd, idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
-        }
+        for (int ks = 0; ks < kHalf / 16; ++ks)
+          mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
         mma_commit(b_pv_done(b));
         if (centroid || b == 1) mma_commit(b_v_empty(s));
         if (u + 2 < steps) ok = issue_s(u + 2);
@@ -268,6 +288,22 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
 
+    if (C::Q_IN_TMEM) {
+      // this thread's query row: eight 16-byte chunks, stored at chunk position c ^ (row & 7)
+      bool q_ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status));
+      uint32_t qw[32];
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(smem + C::OFF_Q + row * 128 + ((c ^ (row & 7)) << 4));
+        qw[4 * c] = v.x; qw[4 * c + 1] = v.y; qw[4 * c + 2] = v.z; qw[4 * c + 3] = v.w;
+      }
+      (void)q_ok;
+      tmem_st32(tmem_base + C::TMEM_Q + lane_addr, qw);
+      tmem_wait_st();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(b_q_tmem);
+    }
     float m_ref = -INFINITY, l_run = 0.f;
     const float inv_scale_log2 = 1.0f / prm.scale_log2;
     const int ck_shift = __ffs(prm.c_k) - 1;
