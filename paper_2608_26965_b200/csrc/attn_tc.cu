@@ -214,11 +214,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // every lane runs the loop (waits and descriptor arithmetic stay warp-uniform); one elected
+    // lane issues the tensor-core instructions
+    {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
-      bool ok = mbar_wait(b_q_full, 0, abort_flag, prm.status);
-      if (C::Q_IN_TMEM && ok) { ok = mbar_wait(b_q_tmem, 0, abort_flag, prm.status); tc_fence_after(); }
+      bool ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status));
+      if (C::Q_IN_TMEM && ok) { ok = __all_sync(0xffffffffu, mbar_wait(b_q_tmem, 0, abort_flag, prm.status)); tc_fence_after(); }
       // load index of half-step u (the shared-memory slot is the load index modulo the stages)
       auto load_of = [&](int u) { return u < 2 * sel_tiles ? u >> 1 : sel_tiles + (u - 2 * sel_tiles); };
       const uint64_t q_desc0 = smem_desc_sw128(s_q, 16, 1024);
@@ -227,12 +229,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const int L = load_of(u), s = L % C::STAGES, b = u & 1;
         const bool centroid = u >= 2 * sel_tiles;
         if (centroid || b == 0) {
-          if (!mbar_wait(b_k_full(s), (L / C::STAGES) & 1, abort_flag, prm.status)) return false;
+          if (!__all_sync(0xffffffffu, mbar_wait(b_k_full(s), (L / C::STAGES) & 1, abort_flag, prm.status))) return false;
           tc_fence_after();
         }
         // descriptors differ from a base one only in the start-address field (units of 16 bytes):
         // the base descriptors are built once, the per-instruction part is an addition
         const int parts = centroid ? 2 : 1;               // centroid tile: hi rows 0-63, lo rows 64-127
+        if (elect_one()) {
         for (int g = 0; g < parts; ++g) {
           const uint32_t rows = (centroid ? g : b) * (kHalf * 128);   // 64 rows = 8192 bytes inside a panel
           const uint64_t kd = k_desc0 + ((s * C::TILE_BYTES + rows) >> 4);
@@ -246,6 +249,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         if (centroid || b == 1) mma_commit(b_k_empty(s));
         mma_commit(b_s_full(b));
+        }
+        __syncwarp();
         return true;
       };
       if (ok && steps > 0) ok = issue_s(0);
@@ -253,8 +258,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int u = 0; u < steps && ok; ++u) {
         const int L = load_of(u), s = L % C::STAGES, b = u & 1;
         const bool centroid = u >= 2 * sel_tiles;
-        ok = mbar_wait(b_p_ready(b), (u >> 1) & 1, abort_flag, prm.status);
-        if (ok && (centroid || b == 0)) ok = mbar_wait(b_v_full(s), (L / C::STAGES) & 1, abort_flag, prm.status);
+        ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(b), (u >> 1) & 1, abort_flag, prm.status));
+        if (ok && (centroid || b == 0)) ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(s), (L / C::STAGES) & 1, abort_flag, prm.status));
         if (!ok) break;
         tc_fence_after();
         const uint32_t vt = s_v + s * C::TILE_BYTES + (centroid ? 0 : b) * (kHalf * 128);
@@ -263,14 +268,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint32_t next_panel = C::ROWSUM_MMA ? (s_base + C::OFF_ONES) - vt : (uint32_t)C::PANEL_BYTES;
         const uint64_t vd = smem_desc_sw128(vt, next_panel, 1024);
         const uint32_t p_cols = tmem_s + b * kHalf;
+        if (elect_one()) {
 #pragma unroll
-        for (int ks = 0; ks < kHalf / 16; ++ks)
-          mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
-        mma_commit(b_pv_done(b));
-        if (centroid || b == 1) mma_commit(b_v_empty(s));
+          for (int ks = 0; ks < kHalf / 16; ++ks)
+            mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
+          mma_commit(b_pv_done(b));
+          if (centroid || b == 1) mma_commit(b_v_empty(s));
+        }
+        __syncwarp();
         if (u + 2 < steps) ok = issue_s(u + 2);
       }
-      mma_commit(b_o_done);
+      if (elect_one()) mma_commit(b_o_done);
     }
   } else {
     // ------------------------------------------------------------ softmax + epilogue (128 threads)

@@ -120,6 +120,15 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
                :: "r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
 }
 
+// One lane of a converged warp (the same one for the lifetime of the warp).  A warp whose lanes all
+// run the issuing loop keeps descriptors and addresses in uniform registers; only the tensor-core
+// instructions themselves are guarded by the elected lane.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+  return pred != 0;
+}
+
 // ---- tcgen05.mma ---------------------------------------------------------------------
 // Completion of all MMAs issued so far by this thread arrives on the mbarrier.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
