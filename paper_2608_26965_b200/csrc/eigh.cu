@@ -159,25 +159,33 @@ __global__ void __launch_bounds__(256) small_matmul_kernel(const double* __restr
     }
 }
 
-// bias[p][j] = - sum_i (sum[p][i] / n) * W[p][i][j]   (float accumulation, four independent chains)
-__global__ void __launch_bounds__(128) bias_kernel(const double* __restrict__ sum, const float* __restrict__ W,
-                                                   int D, double n, float* __restrict__ bias) {
-  __shared__ float mean[128];
+// bias[p][j] = - sum_i (sum[p][i] / n) * W[p][i][j].  Eight threads per output column, each with all of
+// its loads in flight at once; partial sums combined in a fixed order.
+template <int D>
+__global__ void __launch_bounds__(8 * D) bias_kernel(const double* __restrict__ sum, const float* __restrict__ W,
+                                                     double n, float* __restrict__ bias) {
+  constexpr int PER = D / 8;
+  __shared__ float mean[D];
+  __shared__ float part[8][D];
   const int p = blockIdx.x;
-  const int j = threadIdx.x;
-  if (j < D) mean[j] = (float)(sum[(size_t)p * D + j] / n);
+  const int j = threadIdx.x % D, g = threadIdx.x / D;
+  if (threadIdx.x < D) mean[threadIdx.x] = (float)(sum[(size_t)p * D + threadIdx.x] / n);
+  const float* Wp = W + (size_t)p * D * D + (size_t)g * PER * D + j;
+  float w[PER];
+#pragma unroll
+  for (int i = 0; i < PER; ++i) w[i] = Wp[(size_t)i * D];
   __syncthreads();
-  if (j >= D) return;
-  float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-  const float* Wp = W + (size_t)p * D * D + j;
-#pragma unroll 4
-  for (int i = 0; i < D; i += 4) {
-    s0 = fmaf(mean[i], Wp[(size_t)i * D], s0);
-    s1 = fmaf(mean[i + 1], Wp[(size_t)(i + 1) * D], s1);
-    s2 = fmaf(mean[i + 2], Wp[(size_t)(i + 2) * D], s2);
-    s3 = fmaf(mean[i + 3], Wp[(size_t)(i + 3) * D], s3);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < PER; ++i) s = fmaf(mean[g * PER + i], w[i], s);
+  part[g][j] = s;
+  __syncthreads();
+  if (g == 0) {
+    float t = 0.f;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) t += part[q][j];
+    bias[(size_t)p * D + j] = -t;
   }
-  bias[(size_t)p * D + j] = -((s0 + s1) + (s2 + s3));
 }
 
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
@@ -200,7 +208,8 @@ int launch_small_matmul(const double* A, const double* B, int P, int D, double a
   return CA_OK;
 }
 int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st) {
-  bias_kernel<<<P, 128, 0, st>>>(sum, W, D, (double)n, bias);
+  if (D == 64) bias_kernel<64><<<P, 512, 0, st>>>(sum, W, (double)n, bias);
+  else bias_kernel<128><<<P, 1024, 0, st>>>(sum, W, (double)n, bias);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
