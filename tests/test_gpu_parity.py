@@ -257,9 +257,11 @@ def bf16_close(O, o_ref):
     ("sweep64", 1100, 3000, 9, True, 0),          # 64-row clusters on both sides, short last clusters
     ("sweep256", 1024, 2100, 3, True, 0),         # 256-row clusters: two CTAs per query cluster
     ("sweep32k", 640, 1000, 11, False, 0),        # 32-row key clusters packed four to a tile
+    ("sweep64x128", 1100, 3000, 5, True, 0),      # 64 query rows x 128 key rows: the paper's block shape
 ])
 def test_attention_bf16(name, n_q, n_k, keep, compensate, flags):
-    variants = {"sweep64": ("sweep", 64, 64), "sweep256": ("sweep", 256, 256), "sweep32k": ("sweep", 128, 32)}
+    variants = {"sweep64": ("sweep", 64, 64), "sweep256": ("sweep", 256, 256), "sweep32k": ("sweep", 128, 32),
+                "sweep64x128": ("sweep", 64, 128)}
     cluster_k = None
     if name in variants:
         name, cq_, cluster_k = variants[name]
@@ -410,3 +412,26 @@ def test_end_to_end_adaptive_tiny_configuration():
                                                count_k=plan.count_k[0, h].cpu().numpy())
         assert np.abs(O[0, h].cpu().numpy() - o_ref).max() < 1e-5
         assert np.abs(lse[0, h].cpu().numpy() - lse_ref).max() < 1e-5
+
+
+def test_end_to_end_asymmetric_clusters_64_by_128():
+    """The block shape of the paper's attention kernel (64 query rows x 128 key rows) through every
+    stage on the device, bf16, d = 64: clustering with different cluster sizes on the two sides,
+    selection, attention; each stage checked against the oracle on the device's own inputs."""
+    w = inputs.WORKLOADS["tabular"].scaled(heads=2, n_q=2000, n_k=6000)
+    Q, K, V = inputs.generate(w)
+    p = binding.problem_from_workload(w, cluster_q=64, cluster_k=128, keep=6)
+    plan = binding.Plan(p, DEV, keep_y=True)
+    O = plan.forward(store(p, Q), store(p, K), store(p, V), want_lse=True)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for h in range(w.heads):
+        pq, pk = plan.perm_q[0, h].cpu().numpy(), plan.perm_k[0, h].cpu().numpy()
+        assert np.array_equal(pq, orc.recursive_split(plan.Yq[0, h].cpu().numpy(), 64))
+        assert np.array_equal(pk, orc.recursive_split(plan.Yk[0, h].cpu().numpy(), 128))
+        idx = plan.block_idx[0, h].cpu().numpy()
+        assert np.array_equal(idx, orc.select_blocks(plan.cq[0, h].cpu().numpy(), plan.ck[0, h].cpu().numpy(), 6))
+        o_ref, _ = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, 64, 128, idx, True,
+                                         ck=plan.ck[0, h].cpu().numpy(), cv=plan.cv[0, h].cpu().numpy(),
+                                         count_k=plan.count_k[0, h].cpu().numpy())
+        assert bf16_close(O[0, h].float().cpu().numpy(), o_ref)
