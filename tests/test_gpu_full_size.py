@@ -100,3 +100,47 @@ def test_video720_full_size_both_densities():
 
 def test_sweep_full_size_one_eighth():
     check_workload("sweep", sample_heads=[1, 14], clusters_per_head=4, split_heads=[9])
+
+
+def test_tabular_full_size_adaptive_selection():
+    """The adaptive path at the benchmark size, as `bench.py --adaptive 0.5` launches it:
+    un-normalised query representation, mass-recall selection, attention over ragged lists."""
+    build.build()
+    w = inputs.WORKLOADS["tabular"]
+    Q, K, V = inputs.generate(w)
+    scale = float(np.float32(1.0 / np.sqrt(w.head_dim)))
+    p = binding.problem_from_workload(w, flags=binding.CA_QUERY_UNNORMALIZED, softmax_scale=scale)
+    dt = binding.torch_dtype(p)
+    plan = binding.Plan(p, DEV, keep_y=True)
+    dev = lambda a: torch.from_numpy(a[None]).to(dt).to(DEV)
+    O, lse = plan.forward_adaptive(dev(Q), dev(K), dev(V), recall=0.5, min_count=16, want_lse=True)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    c = w.cluster
+    keep_all = plan.keep_count[0]
+    assert int(keep_all.min()) >= 16 and int(keep_all.max()) <= w.n_kc
+    idx_all = plan.block_idx_ragged[0]
+    pos = torch.arange(w.n_kc, device=DEV)[None, None, :]
+    live = pos < keep_all[..., None]
+    assert bool(((idx_all[..., 1:] > idx_all[..., :-1]) | ~live[..., 1:]).all())       # ascending inside the list
+    assert bool((idx_all[~live] == -1).all())                                          # padding behind it
+    r = np.random.default_rng(77)
+    for h in (1, 6):
+        Yq = plan.Yq[0, h].cpu().numpy()
+        pq, pk = plan.perm_q[0, h].cpu().numpy(), plan.perm_k[0, h].cpu().numpy()
+        assert np.array_equal(pq, orc.recursive_split(Yq, c))
+        ck, cv, cq = (t[0, h].cpu().numpy() for t in (plan.ck, plan.cv, plan.cq))
+        cnt = plan.count_k[0, h].cpu().numpy()
+        lists = orc.select_blocks_adaptive(cq, ck, cnt, 0.5, 16, scale=scale)
+        keep = keep_all[h].cpu().numpy()
+        idx = idx_all[h].cpu().numpy()
+        for i, row in enumerate(lists):
+            assert keep[i] == len(row) and np.array_equal(idx[i, :len(row)], row), (h, i)
+        qcs = sorted(r.choice(w.n_qc, 4, replace=False).tolist())
+        o_ref, lse_ref = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, c, c, lists, True, ck=ck, cv=cv,
+                                               count_k=cnt, query_clusters=qcs)
+        rows = np.concatenate([pq[i * c:(i + 1) * c] for i in qcs])
+        got = O[0, h].float().cpu().numpy()[rows]
+        assert np.abs(got - o_ref[rows]).max() <= 2e-2
+        assert np.linalg.norm(got - o_ref[rows]) <= 5e-3 * np.linalg.norm(o_ref[rows])
+        assert np.abs(lse[0, h].cpu().numpy()[rows] - lse_ref[rows]).max() < 2e-2
