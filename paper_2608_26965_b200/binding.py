@@ -19,6 +19,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libclusterattn.so")
 
 CA_OK = 0
+CA_ERR_INVALID_ARG, CA_ERR_UNSUPPORTED, CA_ERR_WORKSPACE, CA_ERR_CUDA, CA_ERR_TIMEOUT = 1, 2, 3, 4, 5
 ERRORS = {1: "CA_ERR_INVALID_ARG", 2: "CA_ERR_UNSUPPORTED", 3: "CA_ERR_WORKSPACE", 4: "CA_ERR_CUDA",
           5: "CA_ERR_TIMEOUT"}
 CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1

@@ -1,0 +1,99 @@
+"""Degenerate inputs and argument errors, through the C ABI on the device."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import clusterattn_oracle as orc
+from paper_2608_26965_b200 import binding, build, inputs
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    build.build()
+    binding.load_library()
+
+
+def dev(a, dtype=torch.float32):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(dtype).to(DEV)
+
+
+def test_identical_keys_give_the_mean_of_the_values():
+    """Every key equal (zero covariance: all pivots of the factorisation drop out, every split
+    coordinate ties and rows split in index order).  All logits of a query are equal, so the
+    compensated output is the plain mean of V whatever is selected (Appendix A: the centroid
+    stands for its members exactly when their weights are equal)."""
+    r = np.random.default_rng(5)
+    H, n_q, n_k, d, c = 2, 300, 1000, 64, 64
+    Q = r.standard_normal((H, n_q, d)).astype(np.float32)
+    K = np.tile(r.standard_normal((H, 1, d)).astype(np.float32), (1, n_k, 1))
+    V = r.standard_normal((H, n_k, d)).astype(np.float32)
+    p = binding.make_problem(1, H, n_q, n_k, d, "fp32", c, c, 3)
+    plan = binding.Plan(p, DEV)
+    O = plan.forward(dev(Q[None]), dev(K[None]), dev(V[None]), want_lse=True)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for h in range(H):
+        perm_k = plan.perm_k[0, h].cpu().numpy()
+        assert np.array_equal(np.sort(perm_k), np.arange(n_k))
+        assert np.array_equal(perm_k, np.arange(n_k))            # ties everywhere: index order survives
+        want = V[h].astype(np.float64).mean(0)
+        assert np.abs(O[0, h].cpu().numpy() - want).max() < 1e-5
+        # the oracle agrees on the clustering of the queries computed by the device
+        o_ref, _ = orc.cluster_attention(Q[h], K[h], V[h], plan.perm_q[0, h].cpu().numpy(), perm_k, c, c,
+                                         plan.block_idx[0, h].cpu().numpy(), True)
+        assert np.abs(O[0, h].cpu().numpy() - o_ref).max() < 1e-5
+
+
+def test_zero_queries_and_a_single_cluster():
+    """Q = 0: the metric is zero, r(q) is the zero vector, every score ties; n_k <= c: one key
+    cluster, kept by every query cluster; the result is dense attention with equal weights."""
+    r = np.random.default_rng(6)
+    H, n_q, n_k, d, c = 1, 200, 100, 128, 128
+    Q = np.zeros((H, n_q, d), np.float32)
+    K = r.standard_normal((H, n_k, d)).astype(np.float32)
+    V = r.standard_normal((H, n_k, d)).astype(np.float32)
+    p = binding.make_problem(1, H, n_q, n_k, d, "bf16", c, c, 1)
+    plan = binding.Plan(p, DEV)
+    O = plan.forward(dev(Q[None], torch.bfloat16), dev(K[None], torch.bfloat16), dev(V[None], torch.bfloat16))
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    assert int(plan.count_k[0, 0, 0]) == n_k and plan.count_k.numel() == 1
+    want = inputs.round_to_bf16(V[0]).astype(np.float64).mean(0)
+    assert np.abs(O[0, 0].float().cpu().numpy() - want).max() < 2e-2
+
+
+def test_argument_errors_enqueue_nothing():
+    lib = binding.load_library()
+    good = binding.make_problem(1, 1, 256, 256, 64, "bf16", 64, 64, 2)
+    plan = binding.Plan(good, DEV)
+    launches = binding.kernel_launches()
+
+    def attn(problem, ws=None, ws_bytes=None, block_idx=None):
+        ws = plan.ws["attn"] if ws is None else ws
+        args = [plan.Qp, plan.Kp, plan.Vp, plan.ck, plan.cv, plan.count_k,
+                plan.block_idx if block_idx is None else block_idx, plan.perm_q]
+        return lib.cluster_attention_fwd(ctypes.byref(problem), *[ctypes.c_void_p(t.data_ptr()) for t in args],
+                                         ctypes.c_void_p(plan.O.data_ptr()), None, ctypes.c_void_p(ws.data_ptr()),
+                                         ws.numel() if ws_bytes is None else ws_bytes, None)
+
+    assert attn(good.copy(keep=5)) == binding.CA_ERR_INVALID_ARG            # more than n_kc = 4
+    assert attn(good.copy(keep=0)) == binding.CA_ERR_INVALID_ARG
+    assert attn(good.copy(cluster_k=96)) == binding.CA_ERR_INVALID_ARG      # not a power of two
+    assert attn(good.copy(head_dim=96)) == binding.CA_ERR_UNSUPPORTED
+    assert attn(good.copy(n_q=0)) == binding.CA_ERR_INVALID_ARG
+    assert attn(good, ws_bytes=16) == binding.CA_ERR_WORKSPACE
+    odd = torch.empty(plan.block_idx.numel() + 1, dtype=torch.int32, device=DEV)[1:]   # 4-byte aligned only
+    assert attn(good, block_idx=odd) == binding.CA_ERR_INVALID_ARG
+    rc = lib.select_blocks_adaptive(ctypes.byref(good), ctypes.c_void_p(plan.cq.data_ptr()),
+                                    ctypes.c_void_p(plan.ck.data_ptr()), ctypes.c_void_p(plan.count_k.data_ptr()),
+                                    0.0, 16, ctypes.c_void_p(plan.block_idx.data_ptr()),
+                                    ctypes.c_void_p(plan.count_q.data_ptr()), ctypes.c_void_p(plan.ws["select"].data_ptr()),
+                                    plan.ws["select"].numel(), None)
+    assert rc == binding.CA_ERR_INVALID_ARG                                  # recall must be positive
+    torch.cuda.synchronize()
+    assert binding.kernel_launches() == launches                            # nothing was enqueued
