@@ -209,6 +209,133 @@ def recursive_split(Y32, c, return_tree=False):
 
 
 # --------------------------------------------------------------------------
+# Section 3.2.1 "Basic recursive splitting" (the variant of principal direction
+# divisive partitioning) with the metric injected into the power iteration, as
+# Section 5.2 proposes: no eigendecomposition, no transformed copy of the rows.
+# For rows x compared in the metric A = R R (R symmetric), the transformed rows
+# are x R and their first principal direction w satisfies w ~ (R C R) w with C
+# the covariance of the untransformed rows; in terms of u = R w the iteration is
+# u <- A C u and the projection of a row is x . u, so only A is needed.
+#
+# Every step is float32 with sequential sums (left to right from zero, each
+# product and sum rounded on its own), because the projections decide the
+# partition:
+#   subsample: m = min(d, s) rows at positions floor(j s / m) of the set;
+#   mean mu_k = (sum_i x_ik) / m;  z = x - mu;
+#   start: g = noise row of the node, gn = g / |g|; the root starts at gn, any
+#     other node at (u_parent + gn) / 2  (the parent's estimate and a random
+#     vector of the same norm, averaged);
+#   one iteration: v_i = sum_k z_ik u_k;  w_k = sum_i z_ik v_i;
+#     y_j = sum_k A_jk w_k;  u = y / |y|  (u is kept when |y| is 0 or not finite);
+#   projection of every row of the set: t = sum_k x_k u_k;
+#   split as in the diagonalized variant: order by (t, row), the first
+#   L = c floor((s + c) / (2c)) rows go down, both sides keep ascending row order.
+# Nodes are numbered level by level: node = 2^level - 1 + slot, where the bits of
+# slot, most significant first, are the path from the root (0 = lower side).
+# --------------------------------------------------------------------------
+def _seq_dot_rows(Z32, u32):
+    """sum_k Z[:, k] u[k] in float32, k ascending, product and sum rounded separately."""
+    acc = np.zeros(Z32.shape[0], np.float32)
+    for k in range(Z32.shape[1]):
+        acc = acc + Z32[:, k] * u32[k]
+    return acc
+
+
+def _seq_norm(v32):
+    s = np.float32(0.0)
+    for x in v32:
+        s = np.float32(s + np.float32(x * x))
+    return np.float32(np.sqrt(s))
+
+
+def basic_direction(sub32, A32, start32, iterations):
+    """Power iteration for the first principal direction of the subsample in the metric A
+    (dual form u <- A C u), float32 with the operation order stated above."""
+    sub32 = np.asarray(sub32, np.float32)
+    A32 = np.asarray(A32, np.float32)
+    m, d = sub32.shape
+    mu = np.zeros(d, np.float32)
+    for i in range(m):
+        mu = mu + sub32[i]
+    mu = mu / np.float32(m)
+    z = sub32 - mu[None, :]
+    u = np.asarray(start32, np.float32).copy()
+    for _ in range(iterations):
+        v = _seq_dot_rows(z, u)                        # [m]
+        w = np.zeros(d, np.float32)
+        for i in range(m):
+            w = w + z[i, :] * v[i]
+        y = _seq_dot_rows(A32, w)                      # y_j = sum_k A[j, k] w[k]
+        nrm = _seq_norm(y)
+        if nrm > 0 and np.isfinite(nrm):
+            u = y / nrm
+    return u
+
+
+def basic_start(noise_row32, parent_u32):
+    g = np.asarray(noise_row32, np.float32)
+    gn = g / _seq_norm(g)
+    if parent_u32 is None:
+        return gn
+    return (np.asarray(parent_u32, np.float32) + gn) * np.float32(0.5)
+
+
+def basic_recursive_split(X32, A32, noise32, c, iterations=3, return_tree=False):
+    """X32 [N, d] float32 rows (the stored values), A32 [d, d] metric, noise32
+    [2^levels - 1, d] normal deviates, one row per node.  Returns perm [N]."""
+    X32 = np.asarray(X32)
+    assert X32.dtype == np.float32
+    N, d = X32.shape
+    perm = np.arange(N, dtype=np.int64)
+    work = [(0, N, 0, None)]                # lo, hi, slot, parent direction
+    level = 0
+    tree = []
+    while work:
+        nxt = []
+        for lo, hi, slot, parent_u in work:
+            s = hi - lo
+            if s <= c:
+                continue
+            rows = perm[lo:hi].copy()
+            m = min(d, s)
+            node = (1 << level) - 1 + slot
+            u = basic_direction(X32[rows[subsample_positions(s, m)]], A32,
+                                basic_start(noise32[node], parent_u), iterations)
+            keys = _seq_dot_rows(X32[rows], u)
+            keys = np.where(keys == 0, np.float32(0.0), keys)      # -0 = +0
+            L = split_point(s, c)
+            order = np.lexsort((rows, keys))
+            below = np.zeros(s, dtype=bool)
+            below[order[:L]] = True
+            perm[lo:lo + L] = rows[below]
+            perm[lo + L:hi] = rows[~below]
+            tree.append((level, slot, lo, hi, L, u))
+            nxt.append((lo, lo + L, 2 * slot, u))
+            nxt.append((lo + L, hi, 2 * slot + 1, u))
+        work = nxt
+        level += 1
+    if return_tree:
+        return perm, tree
+    return perm
+
+
+def split_levels(n, c):
+    """Depth of the split tree: the largest set follows the larger child."""
+    levels, big = 0, n
+    while big > c:
+        L = split_point(big, c)
+        big = max(L, big - L)
+        levels += 1
+    return levels
+
+
+def basic_metrics(Q, K):
+    """Metrics of the basic variant: keys are compared in M = Q^T Q / n_q (Section 3.2.2),
+    queries in K_c^T K_c / n_k (the un-normalised representation, Appendix B.1); fp64."""
+    return centered_scatter(K) / np.asarray(K).shape[0], metric_q(Q)
+
+
+# --------------------------------------------------------------------------
 # Section 3.1 / 3.3.1 / Appendix A: centroids are means over the actual members
 # in the ORIGINAL space; |c| is the member count.
 # --------------------------------------------------------------------------

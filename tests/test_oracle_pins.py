@@ -262,6 +262,105 @@ def test_recursive_split_clusters_are_tighter_than_random_clusters():
     assert within(perm) < 0.5 * within(r.permutation(2048))
 
 
+# -------------------------------------------- basic recursive splitting (Section 3.2.1, Section 5.2)
+def test_basic_direction_converges_to_the_first_principal_component():
+    # identity metric, many iterations: the textbook power iteration on the centred covariance
+    r = rng(50)
+    sub = (r.standard_normal((12, 12)) * np.linspace(4, 0.2, 12)).astype(np.float32)
+    u = orc.basic_direction(sub, np.eye(12, dtype=np.float32), r.standard_normal(12).astype(np.float32), 200)
+    Z = sub.astype(np.float64) - sub.astype(np.float64).mean(0)
+    lam, E = np.linalg.eigh(Z.T @ Z)
+    assert abs(float(np.linalg.norm(u)) - 1) < 1e-5
+    assert abs(float(u.astype(np.float64) @ E[:, -1])) > 1 - 1e-4
+
+
+def test_basic_direction_with_injected_metric_equals_transforming_the_rows():
+    # u <- A C u on the rows x  ==  R (w <- C' w on the rows x R),  A = R R   (Section 5.2)
+    r = rng(51)
+    d = 10
+    B = r.standard_normal((d, d))
+    R = orc.psd_root(B @ B.T / d + 0.5 * np.eye(d))
+    A = R @ R
+    sub = r.standard_normal((d, d)) @ r.standard_normal((d, d))
+    u0 = r.standard_normal(d)
+    for p_iter in (1, 3, 6):
+        u = orc.basic_direction(sub.astype(np.float32), A.astype(np.float32), u0.astype(np.float32), p_iter)
+        w = orc.basic_direction((sub @ R).astype(np.float32), np.eye(d, dtype=np.float32),
+                                np.linalg.solve(R, u0).astype(np.float32), p_iter)
+        v = R @ w.astype(np.float64)
+        v /= np.linalg.norm(v)
+        assert np.abs(u.astype(np.float64) - v).max() < 2e-3
+        # and the projections order the rows alike: x . u  ~  (x R) . w
+        x = r.standard_normal((5, d))
+        assert np.allclose(x @ u.astype(np.float64), (x @ R) @ w.astype(np.float64) / np.linalg.norm(R @ w), atol=5e-3)
+
+
+def test_basic_split_tree_partitions_by_its_projections():
+    r = rng(52)
+    means = 3 * r.standard_normal((6, 8))
+    X = (means[r.integers(0, 6, 1000)] + 0.4 * r.standard_normal((1000, 8))).astype(np.float32)
+    c = 32
+    levels = orc.split_levels(1000, c)
+    noise = r.standard_normal(((1 << levels) - 1, 8)).astype(np.float32)
+    perm, tree = orc.basic_recursive_split(X, np.eye(8, dtype=np.float32), noise, c, 3, return_tree=True)
+    assert sorted(perm.tolist()) == list(range(1000))
+    sizes = [len(perm[j * c:(j + 1) * c]) for j in range(-(-1000 // c))]
+    assert sizes[:-1] == [c] * (len(sizes) - 1) and sizes[-1] == 1000 % c      # one short cluster, the last
+    for j in range(len(sizes)):
+        assert np.all(np.diff(perm[j * c:(j + 1) * c]) > 0)                     # ascending inside a set
+    # replay: every node sends down exactly the L smallest (projection, row) pairs of its set
+    check = np.arange(1000)
+    for level, slot, lo, hi, L, u in tree:
+        rows = check[lo:hi].copy()
+        t = (X[rows].astype(np.float64) @ u.astype(np.float64))
+        assert L == orc.split_point(hi - lo, c) and abs(float(np.linalg.norm(u)) - 1) < 1e-5
+        order = np.lexsort((rows, orc._seq_dot_rows(X[rows], u)))
+        down = np.sort(rows[order[:L]])
+        up = np.sort(rows[order[L:]])
+        assert t[np.isin(rows, down)].max() <= t[np.isin(rows, up)].min() + 1e-4   # a hyperplane cut
+        check[lo:lo + L], check[lo + L:hi] = down, up
+    assert np.array_equal(check, perm)
+
+    def within(p):
+        return sum(X[p[j * c:(j + 1) * c]].var(axis=0).sum() for j in range(31)) / 31
+    assert within(perm) < 0.5 * within(r.permutation(1000))
+
+
+def test_basic_split_start_vectors_and_one_dimension():
+    r = rng(53)
+    X = r.standard_normal((300, 4)).astype(np.float32)
+    levels = orc.split_levels(300, 50)
+    noise = r.standard_normal(((1 << levels) - 1, 4)).astype(np.float32)
+    _, tree = orc.basic_recursive_split(X, np.eye(4, dtype=np.float32), noise, 50, iterations=0, return_tree=True)
+    by_node = {(lv, sl): u for lv, sl, _, _, _, u in tree}
+    g0 = noise[0].astype(np.float64)
+    assert np.allclose(by_node[(0, 0)], g0 / np.linalg.norm(g0), atol=1e-6)       # the root starts at the noise
+    for (lv, sl), u in by_node.items():
+        if lv == 0:
+            continue
+        g = noise[(1 << lv) - 1 + sl].astype(np.float64)
+        want = 0.5 * (by_node[(lv - 1, sl >> 1)].astype(np.float64) + g / np.linalg.norm(g))
+        assert np.allclose(u, want, atol=1e-6)                                   # mean of parent and noise
+    # d = 1 with positive noise: the direction is +1 at every node (a one-row subsample has no
+    # variance, the start vector stays), so the method is "sort and cut into chunks"
+    x = r.standard_normal((257, 1)).astype(np.float32)
+    lv1 = orc.split_levels(257, 16)
+    perm = orc.basic_recursive_split(x, np.ones((1, 1), np.float32),
+                                     np.abs(r.standard_normal(((1 << lv1) - 1, 1))).astype(np.float32) + 0.1, 16, 2)
+    spans = sorted((x[perm[j * 16:(j + 1) * 16], 0].min(), x[perm[j * 16:(j + 1) * 16], 0].max()) for j in range(17))
+    assert all(spans[j][1] <= spans[j + 1][0] for j in range(16))
+
+
+def test_basic_metrics_are_the_two_metric_matrices():
+    r = rng(54)
+    Q, K = r.standard_normal((40, 5)), r.standard_normal((60, 5)) + 1.0
+    A_q, A_k = orc.basic_metrics(Q, K)
+    assert np.allclose(A_k, Q.T @ Q / 40)                         # keys in the query metric
+    Kc = K - K.mean(0)
+    assert np.allclose(A_q, Kc.T @ Kc / 60)                       # queries in the centred key metric
+    assert orc.split_levels(131072, 128) == 10 and orc.split_levels(32760, 128) == 8 and orc.split_levels(100, 128) == 0
+
+
 # -------------------------------------------- centroids and scores (Section 3.3.1)
 def test_centroid_score_is_mean_pairwise_logit_and_jensen_bound():
     r = rng(14)
