@@ -47,6 +47,8 @@ enum {
   CA_Y_IN = 1,      /* Yq/Yk hold the split coordinates: skip the transforms (used by tests
                        to feed the splitter the very same fp32 coordinates as the oracle)   */
   CA_ATTN_FP32 = 2, /* cluster_attention_fwd: force the FP32 CUDA-core kernel for bf16 data  */
+  CA_METRIC_IN = 8, /* cluster_qk_basic: A_q / A_k hold the metric matrices (used by tests to feed
+                       both sides the same float32 matrices)                                */
   CA_QUERY_UNNORMALIZED = 4 /* cluster_qk: queries are represented by R_k q with
                        R_k = sqrt(K_c^T K_c / n_k), without the division by the norm: the
                        form that goes with adaptive selection (Section 3.2.2, Appendix B.1) */
@@ -62,7 +64,7 @@ typedef struct {
   int32_t keep;            /* kept key clusters per query cluster, 1 .. ceil(n_k/c_k)        */
   int32_t compensate;      /* 0/1: striped mean-compensation off/on                          */
   float softmax_scale;     /* 0 selects 1/sqrt(head_dim)                                     */
-  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32 | CA_QUERY_UNNORMALIZED                 */
+  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32 | CA_QUERY_UNNORMALIZED | CA_METRIC_IN  */
 } ca_problem_t;
 
 /* Bytes of workspace each stage needs for this problem (any pointer may be NULL). */
@@ -95,6 +97,41 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
                int32_t* perm_q, int32_t* perm_k, void* Qp, void* Kp, void* Vp,
                float* cq, float* ck, float* cv, int32_t* count_q, int32_t* count_k,
                float* Yq, float* Yk, void* ws, size_t ws_bytes, void* stream);
+
+/*
+ * Clustering by basic recursive splitting (Section 3.2.1, the variant of principal
+ * direction divisive partitioning) with the metric injected into the power
+ * iteration (Section 5.2): no eigendecomposition and no transformed copy of the
+ * rows.  Rows x compared in a metric A = R R have the transformed rows x R, whose
+ * first principal direction w obeys w ~ (R C R) w, C the covariance of the
+ * rows; with u = R w that is u <- A C u, and a row projects to x . u.  Keys use
+ * A_k = Q^T Q / n_q, queries A_q = K_c^T K_c / n_k (the un-normalised
+ * representation, Appendix B.1).  Per set of s > c rows, all in float32 with
+ * sequential sums (each product and sum rounded on its own; the projections
+ * decide the partition, so the order of operations is part of the definition):
+ *   subsample: the min(d, s) rows at positions floor(j s / m) of the set;
+ *   mu_k = (sum_i x_ik) / m;  z = x - mu;
+ *   start vector: g / |g| at the root, (u_parent + g / |g|) / 2 elsewhere, g the
+ *   node's row of `noise` (normal deviates drawn by the caller);
+ *   `iterations` times: v_i = sum_k z_ik u_k; w_k = sum_i z_ik v_i;
+ *   y_j = sum_k A_jk w_k; u = y / |y| (kept when |y| is zero or not finite);
+ *   key of a row: t = sum_k x_k u_k; the set is split as in cluster_qk: the
+ *   L = c floor((s + c) / (2c)) smallest (t, row) go down, both sides keep their
+ *   rows in ascending order.
+ * Nodes are numbered 2^level - 1 + slot, the bits of slot (most significant
+ * first) being the path from the root, 0 = lower side.
+ *   noise_q [B,H,rows_q,d], noise_k [B,H,rows_k,d] fp32, rows as reported by
+ *        ca_basic_workspace_bytes (2^levels - 1).
+ *   A_q, A_k [B,H,d,d] fp32: output, or input when p->flags has CA_METRIC_IN.
+ *   iterations in 0 .. 64.  Other arguments and outputs as in cluster_qk.
+ */
+int ca_basic_workspace_bytes(const ca_problem_t* p, size_t* bytes, int32_t* noise_rows_q,
+                             int32_t* noise_rows_k);
+int cluster_qk_basic(const ca_problem_t* p, const void* Q, const void* K, const void* V,
+                     const float* noise_q, const float* noise_k, int32_t iterations,
+                     float* A_q, float* A_k, int32_t* perm_q, int32_t* perm_k, void* Qp,
+                     void* Kp, void* Vp, float* cq, float* ck, float* cv, int32_t* count_q,
+                     int32_t* count_k, void* ws, size_t ws_bytes, void* stream);
 
 /*
  * Assignment (Section 3.3).  score(i,j) = cq_i . ck_j (the mean logit of the two

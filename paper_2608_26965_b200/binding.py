@@ -23,7 +23,7 @@ CA_ERR_INVALID_ARG, CA_ERR_UNSUPPORTED, CA_ERR_WORKSPACE, CA_ERR_CUDA, CA_ERR_TI
 ERRORS = {1: "CA_ERR_INVALID_ARG", 2: "CA_ERR_UNSUPPORTED", 3: "CA_ERR_WORKSPACE", 4: "CA_ERR_CUDA",
           5: "CA_ERR_TIMEOUT"}
 CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
-CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED = 1, 2, 4
+CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN = 1, 2, 4, 8
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
@@ -82,6 +82,11 @@ def load_library() -> ctypes.CDLL:
     lib.select_blocks_adaptive.restype = ctypes.c_int
     lib.cluster_attention_fwd_ragged.argtypes = [pp] + [vp] * 8 + [ctypes.c_int32] + [vp] * 4 + [sz, vp]
     lib.cluster_attention_fwd_ragged.restype = ctypes.c_int
+    lib.ca_basic_workspace_bytes.argtypes = [pp, ctypes.POINTER(sz), ctypes.POINTER(ctypes.c_int32),
+                                             ctypes.POINTER(ctypes.c_int32)]
+    lib.ca_basic_workspace_bytes.restype = ctypes.c_int
+    lib.cluster_qk_basic.argtypes = [pp] + [vp] * 5 + [ctypes.c_int32] + [vp] * 13 + [sz, vp]
+    lib.cluster_qk_basic.restype = ctypes.c_int
     lib.ca_last_status.argtypes = [vp]
     lib.ca_last_status.restype = ctypes.c_int
     lib.ca_version.argtypes = []
@@ -237,6 +242,41 @@ class Plan:
                                        _stream_ptr(stream))
         _check(rc, "cluster_attention_fwd")
         return self.O, (self.lse if want_lse else None)
+
+    def basic_noise_rows(self):
+        """Rows of normal deviates per head that cluster_qk_basic reads (queries, keys)."""
+        lib = load_library()
+        b, rq, rk = ctypes.c_size_t(), ctypes.c_int32(), ctypes.c_int32()
+        _check(lib.ca_basic_workspace_bytes(ctypes.byref(self.problem), ctypes.byref(b), ctypes.byref(rq),
+                                            ctypes.byref(rk)), "ca_basic_workspace_bytes")
+        return rq.value, rk.value, b.value
+
+    def cluster_qk_basic(self, Q, K, V, noise_q, noise_k, iterations: int = 3, A_q=None, A_k=None, stream=None):
+        """cluster_qk_basic of the C library: basic recursive splitting with the metric injected into
+        the power iteration.  noise_q/noise_k: normal deviates [B,H,rows,d] (rows from basic_noise_rows).
+        A_q/A_k are inputs when the problem has CA_METRIC_IN, otherwise they are written."""
+        lib = load_library()
+        p = self.problem
+        for name, t in (("Q", Q), ("K", K), ("V", V), ("noise_q", noise_q), ("noise_k", noise_k)):
+            _require_cuda(t, name)
+        rq, rk, nbytes = self.basic_noise_rows()
+        if tuple(noise_q.shape[-2:]) != (rq, p.head_dim) or tuple(noise_k.shape[-2:]) != (rk, p.head_dim):
+            raise ClusterAttnError(f"noise must be [B,H,{rq},{p.head_dim}] and [B,H,{rk},{p.head_dim}]")
+        if p.flags & CA_METRIC_IN and (A_q is None or A_k is None):
+            raise ClusterAttnError("CA_METRIC_IN needs A_q and A_k")
+        shape = (p.batch, p.heads, p.head_dim, p.head_dim)
+        self.A_q = A_q if A_q is not None else torch.empty(shape, dtype=torch.float32, device=self.device)
+        self.A_k = A_k if A_k is not None else torch.empty(shape, dtype=torch.float32, device=self.device)
+        if self.ws.get("basic") is None or self.ws["basic"].numel() < nbytes:
+            self.ws["basic"] = torch.zeros(max(nbytes, 256), dtype=torch.uint8, device=self.device)
+        ws = self.ws["basic"]
+        rc = lib.cluster_qk_basic(ctypes.byref(p), _ptr(Q), _ptr(K), _ptr(V), _ptr(noise_q), _ptr(noise_k),
+                                  int(iterations), _ptr(self.A_q), _ptr(self.A_k), _ptr(self.perm_q),
+                                  _ptr(self.perm_k), _ptr(self.Qp), _ptr(self.Kp), _ptr(self.Vp), _ptr(self.cq),
+                                  _ptr(self.ck), _ptr(self.cv), _ptr(self.count_q), _ptr(self.count_k), _ptr(ws),
+                                  ws.numel(), _stream_ptr(stream))
+        _check(rc, "cluster_qk_basic")
+        return self
 
     def select_blocks_adaptive(self, recall: float, min_count: int = 16, cq=None, ck=None, count_k=None,
                                stream=None):

@@ -267,6 +267,92 @@ int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const vo
                          lse, st);
 }
 
+namespace {
+struct BasicWs {
+  int* status;
+  float* partial;
+  double *gramQ, *sumQ, *gramK, *sumK, *metric;
+  float *dirs_q, *dirs_k;
+  int32_t *perm_q_tmp, *perm_k_tmp;
+  uint32_t *keybuf_q, *keybuf_k;
+  int nodes_q, nodes_k;
+  size_t bytes;
+};
+BasicWs carve_basic(const ca_problem_t* p, void* base) {
+  BasicWs w{};
+  Carver c(base);
+  const size_t P = (size_t)p->batch * p->heads, D = p->head_dim, DD = D * D;
+  w.status = c.take<int>(kStatusBytes / sizeof(int));
+  int cr, ncq, nck;
+  moments_chunking(p->n_q, (int)P, &cr, &ncq);
+  moments_chunking(p->n_k, (int)P, &cr, &nck);
+  w.partial = c.take<float>(P * (size_t)(ncq > nck ? ncq : nck) * (DD + D));
+  w.gramQ = c.take<double>(P * DD);  w.sumQ = c.take<double>(P * D);
+  w.gramK = c.take<double>(P * DD);  w.sumK = c.take<double>(P * D);
+  w.metric = c.take<double>(2 * P * DD);
+  const int lq = split_levels_for(p->n_q, p->cluster_q), lk = split_levels_for(p->n_k, p->cluster_k);
+  w.nodes_q = (1 << (lq > 0 ? lq : 1)) - 1;
+  w.nodes_k = (1 << (lk > 0 ? lk : 1)) - 1;
+  w.dirs_q = c.take<float>(P * (size_t)w.nodes_q * D);
+  w.dirs_k = c.take<float>(P * (size_t)w.nodes_k * D);
+  w.perm_q_tmp = c.take<int32_t>(P * (size_t)p->n_q);
+  w.perm_k_tmp = c.take<int32_t>(P * (size_t)p->n_k);
+  w.keybuf_q = c.take<uint32_t>(P * (size_t)p->n_q);
+  w.keybuf_k = c.take<uint32_t>(P * (size_t)p->n_k);
+  w.bytes = c.used();
+  return w;
+}
+}  // namespace
+
+int ca_basic_workspace_bytes(const ca_problem_t* p, size_t* bytes, int32_t* noise_rows_q, int32_t* noise_rows_k) {
+  CA_TRY(check_problem(p));
+  const BasicWs w = carve_basic(p, nullptr);
+  if (bytes) *bytes = w.bytes;
+  if (noise_rows_q) *noise_rows_q = w.nodes_q;
+  if (noise_rows_k) *noise_rows_k = w.nodes_k;
+  return CA_OK;
+}
+
+int cluster_qk_basic(const ca_problem_t* p, const void* Q, const void* K, const void* V, const float* noise_q,
+                     const float* noise_k, int32_t iterations, float* A_q, float* A_k, int32_t* perm_q,
+                     int32_t* perm_k, void* Qp, void* Kp, void* Vp, float* cq, float* ck, float* cv,
+                     int32_t* count_q, int32_t* count_k, void* ws, size_t ws_bytes, void* stream) {
+  CA_TRY(check_problem(p));
+  const void* ptrs[] = {Q, K, V, noise_q, noise_k, A_q, A_k, perm_q, perm_k, Qp, Kp, Vp, cq, ck, cv, count_q, count_k};
+  for (const void* x : ptrs)
+    if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  if (iterations < 0 || iterations > 64) return CA_ERR_INVALID_ARG;
+  if (!ws || !aligned16(ws)) return CA_ERR_WORKSPACE;
+  const BasicWs w = carve_basic(p, ws);
+  if (ws_bytes < w.bytes) return CA_ERR_WORKSPACE;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const int P = p->batch * p->heads, D = p->head_dim;
+  const size_t DD = (size_t)D * D;
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(w.status, 0, kStatusBytes, st));
+  if (!(p->flags & CA_METRIC_IN)) {
+    // keys are compared in the query metric Q^T Q / n_q, queries in K_c^T K_c / n_k (Section 3.2.2)
+    if (p->dtype == CA_DTYPE_BF16) {
+      CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
+      CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial, w.gramK, w.sumK, w.status, st));
+    } else {
+      CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
+      CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial, w.gramK, w.sumK, st));
+    }
+    double* M = w.metric;
+    double* CK = w.metric + (size_t)P * DD;
+    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, 1.0 / (double)p->n_k, M, CK, st));
+    CA_TRY(launch_cast_f64_f32(M, A_k, (size_t)P * DD, st));
+    CA_TRY(launch_cast_f64_f32(CK, A_q, (size_t)P * DD, st));
+  }
+  CA_TRY(launch_split_basic(Q, K, p->dtype, A_q, A_k, noise_q, noise_k, w.dirs_q, w.dirs_k, iterations, P, D, p->n_q,
+                            p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp, perm_k, w.perm_k_tmp,
+                            w.keybuf_q, w.keybuf_k, st));
+  CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
+  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
+  CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+  return CA_OK;
+}
+
 int ca_last_status(const void* ws) {
   if (!ws) return CA_ERR_INVALID_ARG;
   int status = 0;

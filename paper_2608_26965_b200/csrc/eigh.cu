@@ -188,6 +188,16 @@ __global__ void __launch_bounds__(8 * D) bias_kernel(const double* __restrict__ 
   }
 }
 
+__global__ void cast_f64_f32_kernel(const double* __restrict__ src, float* __restrict__ dst, size_t count) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < count) dst[i] = (float)src[i];
+}
+int launch_cast_f64_f32(const double* src, float* dst, size_t count, cudaStream_t st) {
+  cast_f64_f32_kernel<<<(unsigned)((count + 255) / 256), 256, 0, st>>>(src, dst, count);
+  CA_LAUNCH_CHECK();
+  return CA_OK;
+}
+
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
                   int n_k, double ck_scale, double* M, double* CK, cudaStream_t st) {
   metric_kernel<<<dim3(ceil_div(D * D, 256), P), 256, 0, st>>>(gramQ, gramK, sumK, D, (double)n_q,

@@ -42,6 +42,13 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
                  int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st);
 
 // permute.cu
+int launch_split_basic(const void* Q, const void* K, int dtype, const float* A_q, const float* A_k,
+                       const float* noise_q, const float* noise_k, float* dirs_q, float* dirs_k, int iterations,
+                       int problems, int D, int n_q, int n_k, int c_q, int c_k, int32_t* perm_q_out,
+                       int32_t* perm_q_tmp, int32_t* perm_k_out, int32_t* perm_k_tmp, uint32_t* keybuf_q,
+                       uint32_t* keybuf_k, cudaStream_t st);
+int split_levels_for(int n, int c);
+int launch_cast_f64_f32(const double* src, float* dst, size_t count, cudaStream_t st);
 int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P, int n, int D, int c,
                             void* Xp, float* cen, int32_t* count, cudaStream_t st);
 

@@ -115,6 +115,7 @@ struct SplitSide {
 struct SplitParams {
   SplitSide side[2];
   int D, level, problems, smem_rows;
+  int keys_in;             // the keys of this level are already in keybuf (basic variant): no coordinate choice, no gather
 };
 
 // ---------------------------------------------------------------------------
@@ -157,6 +158,8 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
 
   // ---- 1. coordinate of largest subsample variance (every CTA of the cluster computes it)
   const int m = min(D, s);
+  int coord = 0;
+  if (!prm.keys_in) {
   if (tid < m) {
     const int pos = lo + (int)(((long long)tid * s) / m);
     s_sub[tid] = pin ? pin[pos] : pos;
@@ -186,7 +189,8 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
     if (lane == 0) s_scalar[0] = arg;
   }
   __syncthreads();
-  const int coord = s_scalar[0];
+  coord = s_scalar[0];
+  }
 
   // ---- 2. keys of this CTA's slice [c0, c1) of the set
   const int chunk = (s + csize - 1) / csize;
@@ -194,6 +198,16 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   const int cs = c1 - c0;
   const bool in_smem = cs <= prm.smem_rows;
   uint32_t* keys = in_smem ? s_keys : sd.keybuf + (size_t)p * sd.n + lo + c0;
+  if (prm.keys_in) {
+    // the projections of this level were turned into keys by another kernel, position by position
+    if (in_smem) {
+      const uint32_t* kin = sd.keybuf + (size_t)p * sd.n + lo + c0;
+      for (int i = tid; i < cs; i += nt) {
+        s_keys[i] = kin[i];
+        s_rows[i] = pin ? pin[lo + c0 + i] : lo + c0 + i;
+      }
+    }
+  } else {
   // gathers in batches of eight: the row indices first, then the coordinates, so that the
   // memory latencies of a batch overlap
   for (int i0 = tid; i0 < cs; i0 += 8 * nt) {
@@ -214,6 +228,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
         if (in_smem) s_rows[i] = row[u];
       }
     }
+  }
   }
   __syncthreads();
 
@@ -617,7 +632,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
   const int tail_q = tail_level_for(n_q, c_q), tail_k = tail_level_for(n_k, c_k);
   const int top_levels = tail_q > tail_k ? tail_q : tail_k;
   SplitParams prm;
-  prm.D = D; prm.problems = problems;
+  prm.D = D; prm.problems = problems; prm.keys_in = 0;
   // per-level launches write alternately to tmp/out so that the tail kernel, which runs last,
   // reads the buffer that is not the output
   auto fill = [&](int level) {
@@ -673,6 +688,242 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
   tail_kernel<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(TailSmem), st>>>(prm);
   CA_LAUNCH_CHECK();
   return CA_OK;
+}
+
+// ---------------------------------------------------------------------------
+// Basic recursive splitting (Section 3.2.1) with the metric injected into the
+// power iteration (Section 5.2): per set, the first principal direction of a
+// subsample in the metric A, in the dual form u <- A C u, then the projection
+// x . u of every row of the set as the key of the same select-and-partition step.
+// Every floating-point step is float32 with sequential sums (each product and
+// sum rounded on its own), because the projections decide the partition:
+//   subsample m = min(d, s) rows at positions floor(j s / m); mu_k = (sum_i x_ik) / m;
+//   z = x - mu; start g / |g| (root) or (u_parent + g / |g|) / 2, g the node's noise row;
+//   iteration: v_i = sum_k z_ik u_k; w_k = sum_i z_ik v_i; y_j = sum_k A_jk w_k; u = y / |y|.
+// Nodes are numbered 2^level - 1 + slot.
+// ---------------------------------------------------------------------------
+struct BasicSide {
+  const void* X;           // [P][n][D] rows in the storage type
+  const float* A;          // [P][D][D] metric
+  const float* noise;      // [P][nodes][D]
+  float* dirs;             // [P][nodes][D] directions of every node (output, read by the children)
+  const int32_t* perm_in;  // [P][n] or null (identity)
+  uint32_t* keybuf;        // [P][n]
+  int n, c, levels, nodes;
+};
+struct BasicParams {
+  BasicSide side[2];
+  int level, problems, iterations;
+};
+
+__device__ __forceinline__ float seq_norm(const float* v, int d) {
+  float s = 0.f;
+  for (int j = 0; j < d; ++j) s = __fadd_rn(s, __fmul_rn(v[j], v[j]));
+  return __fsqrt_rn(s);
+}
+
+// One CTA of D threads per (slot, side, head).
+template <typename T, int D>
+__global__ void __launch_bounds__(D) basic_direction_kernel(const BasicParams prm) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  float* z = reinterpret_cast<float*>(smem_raw);       // [m][D + 1]
+  __shared__ float u[D], v[D], w[D], y[D], g[D];
+  constexpr int LD = D + 1;
+  const int which = blockIdx.y / prm.problems, p = blockIdx.y % prm.problems;
+  const BasicSide sd = prm.side[which];
+  if (prm.level >= sd.levels) return;
+  const SegmentRef seg = locate_segment(sd.n, sd.c, prm.level, blockIdx.x);
+  if (!seg.active || seg.size <= sd.c) return;
+  const int tid = threadIdx.x;
+  const int s = seg.size, lo = seg.lo, m = min(D, s);
+  const T* X = static_cast<const T*>(sd.X) + (size_t)p * sd.n * D;
+  const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
+  const int node = (1 << prm.level) - 1 + (int)blockIdx.x;
+  // subsample rows, one row per thread, then centred column by column
+  if (tid < m) {
+    const int pos = lo + (int)(((long long)tid * s) / m);
+    const int row = pin ? pin[pos] : pos;
+    const T* xr = X + (size_t)row * D;
+    for (int k = 0; k < D; ++k) z[tid * LD + k] = to_f32<T>(xr[k]);
+  }
+  g[tid] = sd.noise[((size_t)p * sd.nodes + node) * D + tid];
+  __syncthreads();
+  {
+    float mu = 0.f;                                      // thread k: column k, rows in order
+    for (int i = 0; i < m; ++i) mu = __fadd_rn(mu, z[i * LD + tid]);
+    mu = __fdiv_rn(mu, (float)m);
+    for (int i = 0; i < m; ++i) z[i * LD + tid] = __fsub_rn(z[i * LD + tid], mu);
+    const float gn = __fdiv_rn(g[tid], seq_norm(g, D));
+    float start = gn;
+    if (prm.level > 0) {
+      const int parent = (1 << (prm.level - 1)) - 1 + ((int)blockIdx.x >> 1);
+      start = __fmul_rn(__fadd_rn(sd.dirs[((size_t)p * sd.nodes + parent) * D + tid], gn), 0.5f);
+    }
+    u[tid] = start;
+  }
+  __syncthreads();
+  for (int it = 0; it < prm.iterations; ++it) {
+    if (tid < m) {
+      float acc = 0.f;
+      for (int k = 0; k < D; ++k) acc = __fadd_rn(acc, __fmul_rn(z[tid * LD + k], u[k]));
+      v[tid] = acc;
+    }
+    __syncthreads();
+    {
+      float acc = 0.f;
+      for (int i = 0; i < m; ++i) acc = __fadd_rn(acc, __fmul_rn(z[i * LD + tid], v[i]));
+      w[tid] = acc;
+    }
+    __syncthreads();
+    {
+      const float* Ar = sd.A + ((size_t)p * D + tid) * D;
+      float acc = 0.f;
+      for (int k = 0; k < D; ++k) acc = __fadd_rn(acc, __fmul_rn(Ar[k], w[k]));
+      y[tid] = acc;
+    }
+    __syncthreads();
+    const float nrm = seq_norm(y, D);                    // every thread takes the same sequential sum
+    if (nrm > 0.f && isfinite(nrm)) u[tid] = __fdiv_rn(y[tid], nrm);
+    __syncthreads();
+  }
+  sd.dirs[((size_t)p * sd.nodes + node) * D + tid] = u[tid];
+}
+
+// Keys of one level: one thread per position; the set of a position follows from the size rule.
+template <typename T, int D>
+__global__ void __launch_bounds__(256) basic_keys_kernel(const BasicParams prm) {
+  const int which = blockIdx.y / prm.problems, p = blockIdx.y % prm.problems;
+  const BasicSide sd = prm.side[which];
+  if (prm.level >= sd.levels) return;
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= sd.n) return;
+  int lo = 0, size = sd.n, slot = 0;
+  for (int l = 0; l < prm.level; ++l) {
+    if (size <= sd.c) return;                           // a final set: nothing to split at this level
+    const int L = sd.c * ((size + sd.c) / (2 * sd.c));
+    if (i < lo + L) { size = L; slot = 2 * slot; } else { lo += L; size -= L; slot = 2 * slot + 1; }
+  }
+  if (size <= sd.c) return;
+  const int node = (1 << prm.level) - 1 + slot;
+  const float* u = sd.dirs + ((size_t)p * sd.nodes + node) * D;
+  const int row = sd.perm_in ? sd.perm_in[(size_t)p * sd.n + i] : i;
+  const T* xr = static_cast<const T*>(sd.X) + ((size_t)p * sd.n + row) * D;
+  float t = 0.f;
+  if (sizeof(T) == 2) {
+    const uint4* x4 = reinterpret_cast<const uint4*>(xr);
+    for (int k8 = 0; k8 < D / 8; ++k8) {
+      const uint4 q = __ldg(x4 + k8);
+      const uint32_t wds[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const float a = __uint_as_float(wds[e] << 16), b = __uint_as_float(wds[e] & 0xffff0000u);
+        t = __fadd_rn(t, __fmul_rn(a, __ldg(u + k8 * 8 + 2 * e)));
+        t = __fadd_rn(t, __fmul_rn(b, __ldg(u + k8 * 8 + 2 * e + 1)));
+      }
+    }
+  } else {
+    const float4* x4 = reinterpret_cast<const float4*>(xr);
+    for (int k4 = 0; k4 < D / 4; ++k4) {
+      const float4 q = __ldg(x4 + k4);
+      t = __fadd_rn(t, __fmul_rn(q.x, __ldg(u + k4 * 4)));
+      t = __fadd_rn(t, __fmul_rn(q.y, __ldg(u + k4 * 4 + 1)));
+      t = __fadd_rn(t, __fmul_rn(q.z, __ldg(u + k4 * 4 + 2)));
+      t = __fadd_rn(t, __fmul_rn(q.w, __ldg(u + k4 * 4 + 3)));
+    }
+  }
+  sd.keybuf[(size_t)p * sd.n + i] = order_key(t);
+}
+
+template <typename T>
+static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const float* A_k, const float* noise_q,
+                                const float* noise_k, float* dirs_q, float* dirs_k, int iterations, int problems,
+                                int D, int n_q, int n_k, int c_q, int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp,
+                                int32_t* perm_k_out, int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k,
+                                cudaStream_t st) {
+  auto level_kernel = D == 64 ? split_level_kernel<64> : split_level_kernel<128>;
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRowsMax * 8));
+  const int lev_q = split_levels_for(n_q, c_q), lev_k = split_levels_for(n_k, c_k);
+  // a side without any split still needs one launch to write the identity permutation
+  const int run_q = lev_q > 0 ? lev_q : 1, run_k = lev_k > 0 ? lev_k : 1;
+  const int top = run_q > run_k ? run_q : run_k;
+  BasicParams bp;
+  bp.problems = problems; bp.iterations = iterations;
+  SplitParams prm;
+  prm.D = D; prm.problems = problems; prm.keys_in = 1;
+  for (int level = 0; level < top; ++level) {
+    for (int w = 0; w < 2; ++w) {
+      const int run = w == 0 ? run_q : run_k;
+      int32_t* out = w == 0 ? perm_q_out : perm_k_out;
+      int32_t* tmp = w == 0 ? perm_q_tmp : perm_k_tmp;
+      // the last level of a side writes its output buffer, the ones before alternate
+      const bool to_tmp = ((run - 1 - level) % 2) != 0;
+      SplitSide& sd = prm.side[w];
+      sd.Y = nullptr;
+      sd.keybuf = w == 0 ? keybuf_q : keybuf_k;
+      sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
+      sd.levels = w == 0 ? lev_q : lev_k;
+      sd.tail_level = run;                               // every level runs as a launch of its own
+      sd.perm_out = to_tmp ? tmp : out;
+      sd.perm_in = level == 0 ? nullptr : (to_tmp ? out : tmp);
+      BasicSide& bs = bp.side[w];
+      bs.X = w == 0 ? static_cast<const void*>(Q) : static_cast<const void*>(K);
+      bs.A = w == 0 ? A_q : A_k;
+      bs.noise = w == 0 ? noise_q : noise_k;
+      bs.dirs = w == 0 ? dirs_q : dirs_k;
+      bs.perm_in = sd.perm_in; bs.keybuf = sd.keybuf;
+      bs.n = sd.n; bs.c = sd.c; bs.levels = sd.levels;
+      bs.nodes = (1 << (sd.levels > 0 ? sd.levels : 1)) - 1;
+    }
+    bp.level = level; prm.level = level;
+    const size_t dsmem = (size_t)D * (D + 1) * sizeof(float);
+    if (D == 64) {
+      auto dk = basic_direction_kernel<T, 64>;
+      CA_RETURN_IF_CUDA(cudaFuncSetAttribute(dk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dsmem));
+      dk<<<dim3(1u << level, 2 * problems), 64, dsmem, st>>>(bp);
+    } else {
+      auto dk = basic_direction_kernel<T, 128>;
+      CA_RETURN_IF_CUDA(cudaFuncSetAttribute(dk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dsmem));
+      dk<<<dim3(1u << level, 2 * problems), 128, dsmem, st>>>(bp);
+    }
+    CA_LAUNCH_CHECK();
+    const int n_max = n_q > n_k ? n_q : n_k;
+    if (D == 64) basic_keys_kernel<T, 64><<<dim3(ceil_div(n_max, 256), 2 * problems), 256, 0, st>>>(bp);
+    else basic_keys_kernel<T, 128><<<dim3(ceil_div(n_max, 256), 2 * problems), 256, 0, st>>>(bp);
+    CA_LAUNCH_CHECK();
+    int max_seg = 1;
+    if (level < run_q) max_seg = max_segment_at_level(n_q, c_q, level);
+    if (level < run_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
+    int csize = 1;
+    while (csize < kMaxCluster && max_seg > csize * 8192) csize *= 2;
+    const int per_cta = (max_seg + csize - 1) / csize;
+    prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((1u << level) * csize, 2 * problems);
+    cfg.blockDim = dim3(kSplitThreads);
+    cfg.dynamicSmemBytes = (size_t)prm.smem_rows * 8 > 16 ? (size_t)prm.smem_rows * 8 : 16;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, level_kernel, prm));
+    CA_LAUNCH_CHECK();
+  }
+  return CA_OK;
+}
+
+int launch_split_basic(const void* Q, const void* K, int dtype, const float* A_q, const float* A_k,
+                       const float* noise_q, const float* noise_k, float* dirs_q, float* dirs_k, int iterations,
+                       int problems, int D, int n_q, int n_k, int c_q, int c_k, int32_t* perm_q_out,
+                       int32_t* perm_q_tmp, int32_t* perm_k_out, int32_t* perm_k_tmp, uint32_t* keybuf_q,
+                       uint32_t* keybuf_k, cudaStream_t st) {
+  if (dtype == CA_DTYPE_BF16)
+    return launch_split_basic_t(static_cast<const __nv_bfloat16*>(Q), static_cast<const __nv_bfloat16*>(K), A_q, A_k,
+                                noise_q, noise_k, dirs_q, dirs_k, iterations, problems, D, n_q, n_k, c_q, c_k,
+                                perm_q_out, perm_q_tmp, perm_k_out, perm_k_tmp, keybuf_q, keybuf_k, st);
+  return launch_split_basic_t(static_cast<const float*>(Q), static_cast<const float*>(K), A_q, A_k, noise_q, noise_k,
+                              dirs_q, dirs_k, iterations, problems, D, n_q, n_k, c_q, c_k, perm_q_out, perm_q_tmp,
+                              perm_k_out, perm_k_tmp, keybuf_q, keybuf_k, st);
 }
 
 }  // namespace ca
