@@ -62,6 +62,9 @@ def parse_args():
     ap.add_argument("--adaptive", type=float, default=0.0, metavar="RECALL",
                     help="adaptive mass-recall selection with this recall threshold (min count 16) and the "
                          "un-normalised query representation, instead of a fixed count per query cluster")
+    ap.add_argument("--basic", type=int, default=-1, metavar="ITERATIONS",
+                    help="cluster with basic recursive splitting (power iteration with the injected metric, "
+                         "this many iterations per split) instead of the diagonalized variant")
     ap.add_argument("--scaling", action="store_true",
                     help="token-count sweep 8k..1M with per-stage times (64 kept blocks, and 10 %% of the blocks), "
                          "eager launches and one replayed CUDA graph, against dense attention")
@@ -235,10 +238,24 @@ def run_ours(args, w):
     def max_over_ranks(x):
         return replicas.max_over_ranks(x, device)
 
+    basic = args.basic >= 0
+    if basic:
+        rows_q, rows_k, _ = plan.basic_noise_rows()
+        gen = torch.Generator(device=dev)
+        gen.manual_seed(26082696)
+        noise_q = torch.randn((1, heads, rows_q, w.head_dim), generator=gen, device=dev)
+        noise_k = torch.randn((1, heads, rows_k, w.head_dim), generator=gen, device=dev)
+
+    def clustering(Qd, Kd, Vd):
+        if basic:
+            plan.cluster_qk_basic(Qd, Kd, Vd, noise_q, noise_k, args.basic)
+        else:
+            plan.cluster_qk(Qd, Kd, Vd)
+
     def step(events=None):
         if events is not None:
             events[0].record(stream)
-        plan.cluster_qk(Q, K, V)
+        clustering(Q, K, V)
         if events is not None:
             events[1].record(stream)
         if adaptive:
@@ -309,7 +326,7 @@ def run_ours(args, w):
                 ev_in[bsel].record(h2d)
             stream.wait_event(ev_in[bsel])
             Qd, Kd, Vd = sets[bsel]
-            plan.cluster_qk(Qd, Kd, Vd)
+            clustering(Qd, Kd, Vd)
             ev_free[bsel].record(stream)                      # only the clustering stage reads the inputs
             if adaptive:
                 plan.select_blocks_adaptive(args.adaptive, 16)
@@ -385,7 +402,7 @@ def run_ours(args, w):
     roofline = {
         "kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": attn_tflops, "peak": peak,
         "peak_source": f"{peak_kind} bf16 burst", "unit": "TFLOP/s", "frac": attn_tflops / peak,
-        "traffic": None if (adaptive or args.keep or args.n_q or args.n_k or args.heads)
+        "traffic": None if (adaptive or basic or args.keep or args.n_q or args.n_k or args.heads)
         else NCU_TRAFFIC_BYTES.get(w.name),
     }
     line = {
@@ -394,7 +411,9 @@ def run_ours(args, w):
         "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "heads": heads, "head_dim": w.head_dim, "n_q": w.n_q, "n_k": w.n_k,
                    "cluster": w.cluster, "keep": mean_keep if adaptive else keep, "n_kc": w.n_kc,
-                   "selection": f"adaptive recall {args.adaptive} min 16" if adaptive else "top-k", "compensate": w.compensate,
+                   "selection": f"adaptive recall {args.adaptive} min 16" if adaptive else "top-k",
+                   "clustering": f"basic recursive splitting, {args.basic} power iterations" if basic
+                   else "diagonalized recursive splitting", "compensate": w.compensate,
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "inputs larger than L2 (no flush)"},
         "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),

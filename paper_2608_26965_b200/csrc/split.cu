@@ -255,14 +255,14 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
     }
     if (csize > 1) {
       cluster.sync();                                // every slice has counted
-      if (tid < 256) {
+      for (int b = tid; b < 256; b += nt) {
         int sum = 0;
-        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(s_hist, r)[tid];
-        s_total[tid] = sum;
+        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(s_hist, r)[b];
+        s_total[b] = sum;
       }
     } else {
       __syncthreads();
-      if (tid < 256) s_total[tid] = s_hist[tid];
+      for (int b = tid; b < 256; b += nt) s_total[b] = s_hist[b];
     }
     __syncthreads();
     if (warp == 0) {
@@ -744,7 +744,27 @@ __global__ void __launch_bounds__(D) basic_direction_kernel(const BasicParams pr
     const int pos = lo + (int)(((long long)tid * s) / m);
     const int row = pin ? pin[pos] : pos;
     const T* xr = X + (size_t)row * D;
-    for (int k = 0; k < D; ++k) z[tid * LD + k] = to_f32<T>(xr[k]);
+    if (sizeof(T) == 2) {                                // 16-byte loads, all in flight together
+      uint4 q[D / 8];
+#pragma unroll
+      for (int k8 = 0; k8 < D / 8; ++k8) q[k8] = __ldg(reinterpret_cast<const uint4*>(xr) + k8);
+#pragma unroll
+      for (int k8 = 0; k8 < D / 8; ++k8) {
+        const uint32_t wds[4] = {q[k8].x, q[k8].y, q[k8].z, q[k8].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          z[tid * LD + k8 * 8 + 2 * e] = __uint_as_float(wds[e] << 16);
+          z[tid * LD + k8 * 8 + 2 * e + 1] = __uint_as_float(wds[e] & 0xffff0000u);
+        }
+      }
+    } else {
+#pragma unroll 8
+      for (int k4 = 0; k4 < D / 4; ++k4) {
+        const float4 q = __ldg(reinterpret_cast<const float4*>(xr) + k4);
+        z[tid * LD + k4 * 4] = q.x; z[tid * LD + k4 * 4 + 1] = q.y;
+        z[tid * LD + k4 * 4 + 2] = q.z; z[tid * LD + k4 * 4 + 3] = q.w;
+      }
+    }
   }
   g[tid] = sd.noise[((size_t)p * sd.nodes + node) * D + tid];
   __syncthreads();
@@ -899,7 +919,10 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
     prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((1u << level) * csize, 2 * problems);
-    cfg.blockDim = dim3(kSplitThreads);
+    // deep levels hold many small sets: a CTA per set with about four rows per thread
+    int threads = 128;
+    while (threads < kSplitThreads && threads * 4 < per_cta) threads *= 2;
+    cfg.blockDim = dim3(threads);
     cfg.dynamicSmemBytes = (size_t)prm.smem_rows * 8 > 16 ? (size_t)prm.smem_rows * 8 : 16;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
