@@ -144,3 +144,31 @@ def test_tabular_full_size_adaptive_selection():
         assert np.abs(got - o_ref[rows]).max() <= 2e-2
         assert np.linalg.norm(got - o_ref[rows]) <= 5e-3 * np.linalg.norm(o_ref[rows])
         assert np.abs(lse[0, h].cpu().numpy()[rows] - lse_ref[rows]).max() < 2e-2
+
+
+def test_tabular_full_size_basic_splitting():
+    """Basic recursive splitting at the benchmark size, as `bench.py --basic 3` launches it: the
+    oracle's splitter on the device's metric matrices reproduces the permutation of 131,072 keys and
+    16,384 queries of a sampled head bit for bit; invariants on every head."""
+    build.build()
+    w = inputs.WORKLOADS["tabular"]
+    Q, K, V = inputs.generate(w)
+    p = binding.problem_from_workload(w)
+    dt = binding.torch_dtype(p)
+    plan = binding.Plan(p, DEV)
+    rows_q, rows_k, _ = plan.basic_noise_rows()
+    r = np.random.default_rng(11)
+    nq = r.standard_normal((w.heads, rows_q, w.head_dim)).astype(np.float32)
+    nk = r.standard_normal((w.heads, rows_k, w.head_dim)).astype(np.float32)
+    dev = lambda a, t=torch.float32: torch.from_numpy(a[None]).to(t).to(DEV)
+    plan.cluster_qk_basic(dev(Q, dt), dev(K, dt), dev(V, dt), dev(nq), dev(nk), 3)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for perm, n in ((plan.perm_q[0], w.n_q), (plan.perm_k[0], w.n_k)):
+        srt = torch.sort(perm, dim=1).values
+        assert torch.equal(srt, torch.arange(n, device=DEV, dtype=torch.int32).expand_as(srt))
+    assert int(plan.count_k.sum()) == w.heads * w.n_k and int(plan.count_k.min()) == w.cluster
+    h = 4
+    A_q, A_k = plan.A_q[0, h].cpu().numpy(), plan.A_k[0, h].cpu().numpy()
+    assert np.array_equal(plan.perm_k[0, h].cpu().numpy(), orc.basic_recursive_split(K[h], A_k, nk[h], w.cluster, 3))
+    assert np.array_equal(plan.perm_q[0, h].cpu().numpy(), orc.basic_recursive_split(Q[h], A_q, nq[h], w.cluster, 3))
