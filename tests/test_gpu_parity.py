@@ -57,6 +57,7 @@ SPLIT_CASES = [
     (1, 16384, 131072, 64, 128, 128, "bf16", False),  # one head of the tabular shape: 8-CTA clusters at the top
     (1, 5000, 200000, 64, 64, 128, "bf16", True),     # slices beyond the shared-memory window, with ties
     (2, 32760, 32760, 128, 128, 128, "bf16", False),  # the video shape: odd cluster counts, short last cluster
+    (1, 4096, 1048576, 64, 128, 128, "bf16", False),  # a million rows: 13 levels, 8 with thread-block clusters
 ]
 
 
