@@ -138,6 +138,9 @@ int cluster_qk_basic(const ca_problem_t* p, const void* Q, const void* K, const 
  * clusters); for each query cluster the `keep` best key clusters, ties to the
  * lower index, written in ascending index order.
  *   block_idx [B,H,n_qc,keep] int32.
+ * With 2048 key clusters or more and a workspace as large as ca_workspace_bytes
+ * reports, the scores are first computed in tiles into the workspace (same
+ * operation order, same bits); a workspace of 256 bytes selects the fused kernel.
  */
 int select_blocks(const ca_problem_t* p, const float* cq, const float* ck,
                   int32_t* block_idx, void* ws, size_t ws_bytes, void* stream);

@@ -99,7 +99,9 @@ unsigned long long ca_kernel_launches(void) { return g_kernel_launches; }
 int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select_ws, size_t* attn_ws) {
   CA_TRY(check_problem(p));
   if (cluster_ws) *cluster_ws = carve_cluster(p, nullptr, true, true).bytes;
-  if (select_ws) *select_ws = kStatusBytes;
+  if (select_ws)
+    *select_ws = kStatusBytes + sizeof(float) * select_score_floats(p->batch * p->heads, ceil_div(p->n_q, p->cluster_q),
+                                                                    ceil_div(p->n_k, p->cluster_k));
   if (attn_ws) *attn_ws = attn_tc_supported(*p) ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   return CA_OK;
 }
@@ -203,8 +205,11 @@ int select_blocks(const ca_problem_t* p, const float* cq, const float* ck, int32
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
   const int P = p->batch * p->heads;
+  // room behind the status block holds tiles of scores when there are many key clusters
+  float* score_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
+  const size_t score_floats = aligned16(ws) ? (ws_bytes - kStatusBytes) / sizeof(float) : 0;
   return launch_score_select(cq, ck, P, ceil_div(p->n_q, p->cluster_q), ceil_div(p->n_k, p->cluster_k),
-                             p->head_dim, p->keep, block_idx, st);
+                             p->head_dim, p->keep, block_idx, score_ws, score_floats, st);
 }
 
 int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp, const void* Vp,
@@ -239,9 +244,11 @@ int select_blocks_adaptive(const ca_problem_t* p, const float* cq, const float* 
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
+  float* score_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
+  const size_t score_floats = aligned16(ws) ? (ws_bytes - kStatusBytes) / sizeof(float) : 0;
   return launch_select_adaptive(cq, ck, count_k, p->batch * p->heads, ceil_div(p->n_q, p->cluster_q),
                                 ceil_div(p->n_k, p->cluster_k), p->head_dim, scale, recall, min_count,
-                                block_idx, keep_count, st);
+                                block_idx, keep_count, score_ws, score_floats, st);
 }
 
 int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const void* Kp, const void* Vp,

@@ -53,12 +53,13 @@ int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P
                             void* Xp, float* cen, int32_t* count, cudaStream_t st);
 
 // select.cu
-size_t select_smem_bytes(int n_kc, int D);
+size_t select_smem_bytes(int n_kc, int D, int qt);
 int launch_select_adaptive(const float* cq, const float* ck, const int32_t* count_k, int P, int n_qc, int n_kc,
                            int D, float scale, float recall, int min_count, int32_t* block_idx,
-                           int32_t* keep_count, cudaStream_t st);
+                           int32_t* keep_count, float* score_ws, size_t score_floats, cudaStream_t st);
+size_t select_score_floats(int P, int n_qc, int n_kc);
 int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n_kc, int D, int keep,
-                        int32_t* block_idx, cudaStream_t st);
+                        int32_t* block_idx, float* score_ws, size_t score_floats, cudaStream_t st);
 
 // attn_ref.cu
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,

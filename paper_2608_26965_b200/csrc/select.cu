@@ -10,6 +10,7 @@ namespace ca {
 
 constexpr int kSelectThreads = 256;
 constexpr int kSelectQT = 4;          // query clusters per CTA (key centroids are read once for all)
+constexpr int kSelectTiledMinClusters = 2048;   // from here on the scores are computed in tiles first
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   if (s == 0.0f) s = 0.0f;                        // -0 and +0 compare equal
@@ -17,34 +18,44 @@ __device__ __forceinline__ uint32_t score_key(float s) {
   return (u >> 31) ? ~u : (u | 0x80000000u);
 }
 
-template <int D>
+// QT query clusters per CTA: 4 when the CTA computes the scores itself (the key centroids are read
+// once for the four), 1 when the scores come from memory (less shared memory, more CTAs per SM).
+template <int D, int QT>
 __global__ void __launch_bounds__(kSelectThreads)
 score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, int n_qc, int n_kc,
-                    int keep, int32_t* __restrict__ block_idx) {
+                    int keep, int32_t* __restrict__ block_idx, const float* __restrict__ scores, int row0,
+                    int chunk_rows) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);                       // [QT][n_kc]
-  float* qs = reinterpret_cast<float*>(keys + (size_t)kSelectQT * n_kc);        // [QT][D]
+  float* qs = reinterpret_cast<float*>(keys + (size_t)QT * n_kc);        // [QT][D]
   __shared__ int s_hist[256];
   __shared__ int s_warp[64];
   __shared__ int s_scalar[4];
   const int p = blockIdx.y;
-  const int q0 = blockIdx.x * kSelectQT;
-  const int nq = min(kSelectQT, n_qc - q0);
+  const int q0 = row0 + blockIdx.x * QT;
+  const int nq = min(QT, min(n_qc, row0 + chunk_rows) - q0);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* cqp = cq + ((size_t)p * n_qc + q0) * D;
   const float* ckp = ck + (size_t)p * n_kc * D;
-  for (int e = tid; e < kSelectQT * D; e += kSelectThreads) qs[e] = (e < nq * D) ? cqp[e] : 0.f;
+  if (scores) {
+    // the scores of this chunk of rows were computed by score_tile_kernel (same operation order)
+    for (int t = 0; t < nq; ++t) {
+      const float* srow = scores + ((size_t)p * chunk_rows + (q0 - row0 + t)) * n_kc;
+      for (int j = tid; j < n_kc; j += kSelectThreads) keys[(size_t)t * n_kc + j] = score_key(__ldg(srow + j));
+    }
+  } else {
+  for (int e = tid; e < QT * D; e += kSelectThreads) qs[e] = (e < nq * D) ? cqp[e] : 0.f;
   __syncthreads();
 
   for (int j = tid; j < n_kc; j += kSelectThreads) {
-    float acc[kSelectQT];
+    float acc[QT];
 #pragma unroll
-    for (int t = 0; t < kSelectQT; ++t) acc[t] = 0.f;
+    for (int t = 0; t < QT; ++t) acc[t] = 0.f;
     const float4* row = reinterpret_cast<const float4*>(ckp + (size_t)j * D);
     for (int k4 = 0; k4 < D / 4; ++k4) {
       const float4 kv = __ldg(row + k4);
 #pragma unroll
-      for (int t = 0; t < kSelectQT; ++t) {
+      for (int t = 0; t < QT; ++t) {
         const float* q = qs + t * D + k4 * 4;
         acc[t] = __fadd_rn(acc[t], __fmul_rn(q[0], kv.x));
         acc[t] = __fadd_rn(acc[t], __fmul_rn(q[1], kv.y));
@@ -53,7 +64,8 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
       }
     }
 #pragma unroll
-    for (int t = 0; t < kSelectQT; ++t) keys[(size_t)t * n_kc + j] = score_key(acc[t]);
+    for (int t = 0; t < QT; ++t) keys[(size_t)t * n_kc + j] = score_key(acc[t]);
+  }
   }
   __syncthreads();
 
@@ -71,8 +83,13 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
         const uint32_t k = ok ? kt[j] : 0u;
         const bool cand = ok && ((k & mask) == prefix);
         const int bin = cand ? (int)((k >> shift) & 255u) : -1;
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+        if (shift == 24) {
+          // leading digit (sign and exponent bits): few distinct values in a warp, one atomic per value
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+        } else if (cand) {
+          atomicAdd(&s_hist[bin], 1);                // lower digits are spread out: plain atomics
+        }
       }
       __syncthreads();
       if (warp == 0) {
@@ -143,25 +160,138 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
   }
 }
 
-size_t select_smem_bytes(int n_kc, int D) {
-  return (size_t)kSelectQT * n_kc * sizeof(uint32_t) + (size_t)kSelectQT * D * sizeof(float);
+size_t select_smem_bytes(int n_kc, int D, int qt) {
+  return (size_t)qt * n_kc * sizeof(uint32_t) + (size_t)qt * D * sizeof(float);
+}
+
+// ---------------------------------------------------------------------------
+// Scores of a chunk of query clusters against every key cluster, 64 x 64 tiles.
+// Used when there are many key clusters: the fused kernels re-read all key
+// centroids for every few query clusters, which is bound by L2 traffic.  Every
+// score is accumulated for k = 0, 1, ... with separately rounded product and sum,
+// exactly as in the fused kernels, so both paths give the same bits.
+//   scores [P][chunk_rows][n_kc]
+// ---------------------------------------------------------------------------
+template <int D>
+__global__ void __launch_bounds__(256)
+score_tile_kernel(const float* __restrict__ cq, const float* __restrict__ ck, int n_qc, int n_kc, int row0,
+                  int chunk_rows, float* __restrict__ scores) {
+  extern __shared__ __align__(16) float tile_smem[];
+  float* As = tile_smem;                 // [D][64]  As[k][i]
+  float* Bs = tile_smem + D * 64;        // [D][64]  Bs[k][j]
+  const int p = blockIdx.z;
+  const int i0 = row0 + blockIdx.y * 64, j0 = blockIdx.x * 64;
+  const int row_end = min(n_qc, row0 + chunk_rows);
+  const int tid = threadIdx.x;
+  const float* cqp = cq + (size_t)p * n_qc * D;
+  const float* ckp = ck + (size_t)p * n_kc * D;
+  for (int e = tid; e < 64 * (D / 4); e += 256) {
+    const int r = e / (D / 4), k4 = e % (D / 4);
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (i0 + r < row_end) a = __ldg(reinterpret_cast<const float4*>(cqp + (size_t)(i0 + r) * D) + k4);
+    if (j0 + r < n_kc) b = __ldg(reinterpret_cast<const float4*>(ckp + (size_t)(j0 + r) * D) + k4);
+    As[(k4 * 4 + 0) * 64 + r] = a.x; As[(k4 * 4 + 1) * 64 + r] = a.y;
+    As[(k4 * 4 + 2) * 64 + r] = a.z; As[(k4 * 4 + 3) * 64 + r] = a.w;
+    Bs[(k4 * 4 + 0) * 64 + r] = b.x; Bs[(k4 * 4 + 1) * 64 + r] = b.y;
+    Bs[(k4 * 4 + 2) * 64 + r] = b.z; Bs[(k4 * 4 + 3) * 64 + r] = b.w;
+  }
+  __syncthreads();
+  const int ti = tid / 16, tj = tid % 16;
+  float acc[4][4];
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+#pragma unroll 4
+  for (int k = 0; k < D; ++k) {
+    const float4 a = *reinterpret_cast<const float4*>(&As[k * 64 + ti * 4]);
+    const float4 b = *reinterpret_cast<const float4*>(&Bs[k * 64 + tj * 4]);
+    const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) acc[x][y] = __fadd_rn(acc[x][y], __fmul_rn(av[x], bv[y]));
+  }
+#pragma unroll
+  for (int x = 0; x < 4; ++x) {
+    const int i = i0 + ti * 4 + x;
+    if (i >= row_end) continue;
+    float* out = scores + ((size_t)p * chunk_rows + (i - row0)) * n_kc + j0 + tj * 4;
+    if (j0 + tj * 4 + 3 < n_kc && (n_kc & 3) == 0) {
+      *reinterpret_cast<float4*>(out) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+    } else {
+#pragma unroll
+      for (int y = 0; y < 4; ++y)
+        if (j0 + tj * 4 + y < n_kc) out[y] = acc[x][y];
+    }
+  }
+}
+
+// rows of scores that fit the workspace (a multiple of 64), or 0: use the fused kernels
+int select_chunk_rows(int P, int n_qc, int n_kc, size_t score_floats) {
+  if (n_kc < kSelectTiledMinClusters || score_floats == 0) return 0;
+  size_t rows = score_floats / ((size_t)P * n_kc);
+  if (rows >= (size_t)n_qc) return n_qc;
+  rows = rows / 64 * 64;
+  return (int)rows;
+}
+
+size_t select_score_floats(int P, int n_qc, int n_kc) {
+  if (n_kc < kSelectTiledMinClusters) return 0;
+  const size_t all = (size_t)P * n_qc * n_kc;
+  const size_t budget = (size_t)64 << 20;            // 256 MB of scores at a time
+  const size_t least = (size_t)P * 64 * n_kc;        // at least one 64-row chunk
+  size_t take = all < budget ? all : budget;
+  if (take < least) take = least;
+  return (take + 63) / 64 * 64;
+}
+
+template <int D>
+static int launch_score_tiles(const float* cq, const float* ck, int P, int n_qc, int n_kc, int row0, int chunk_rows,
+                              float* scores, cudaStream_t st) {
+  auto k = score_tile_kernel<D>;
+  const size_t smem = (size_t)2 * D * 64 * sizeof(float);
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int rows = min(chunk_rows, n_qc - row0);
+  k<<<dim3(ceil_div(n_kc, 64), ceil_div(rows, 64), P), 256, smem, st>>>(cq, ck, n_qc, n_kc, row0, chunk_rows, scores);
+  CA_LAUNCH_CHECK();
+  return CA_OK;
 }
 
 int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n_kc, int D, int keep,
-                        int32_t* block_idx, cudaStream_t st) {
-  const size_t smem = select_smem_bytes(n_kc, D);
-  if (smem > 200 * 1024) return CA_ERR_UNSUPPORTED;
-  dim3 grid(ceil_div(n_qc, kSelectQT), P);
-  if (D == 64) {
-    auto k = score_select_kernel<64>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx);
-  } else {
-    auto k = score_select_kernel<128>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx);
+                        int32_t* block_idx, float* score_ws, size_t score_floats, cudaStream_t st) {
+  const int chunk = select_chunk_rows(P, n_qc, n_kc, score_ws ? score_floats : 0);
+  if (chunk == 0) {
+    const size_t smem = select_smem_bytes(n_kc, D, kSelectQT);
+    if (smem > 200 * 1024) return CA_ERR_UNSUPPORTED;
+    dim3 grid(ceil_div(n_qc, kSelectQT), P);
+    if (D == 64) {
+      auto k = score_select_kernel<64, kSelectQT>;
+      CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      k<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx, nullptr, 0, n_qc);
+    } else {
+      auto k = score_select_kernel<128, kSelectQT>;
+      CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+      k<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx, nullptr, 0, n_qc);
+    }
+    CA_LAUNCH_CHECK();
+    return CA_OK;
   }
-  CA_LAUNCH_CHECK();
+  const size_t smem = select_smem_bytes(n_kc, D, 1);
+  if (smem > 200 * 1024) return CA_ERR_UNSUPPORTED;
+  auto k64 = score_select_kernel<64, 1>;
+  auto k128 = score_select_kernel<128, 1>;
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k64, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k128, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  for (int row0 = 0; row0 < n_qc; row0 += chunk) {
+    const int rows = min(chunk, n_qc - row0);
+    if (D == 64) { int rc = launch_score_tiles<64>(cq, ck, P, n_qc, n_kc, row0, chunk, score_ws, st); if (rc != CA_OK) return rc; }
+    else { int rc = launch_score_tiles<128>(cq, ck, P, n_qc, n_kc, row0, chunk, score_ws, st); if (rc != CA_OK) return rc; }
+    dim3 grid(rows, P);
+    if (D == 64) k64<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx, score_ws, row0, chunk);
+    else k128<<<grid, kSelectThreads, smem, st>>>(cq, ck, n_qc, n_kc, keep, block_idx, score_ws, row0, chunk);
+    CA_LAUNCH_CHECK();
+  }
   return CA_OK;
 }
 
@@ -197,7 +327,8 @@ __global__ void __launch_bounds__(256)
 select_adaptive_kernel(const float* __restrict__ cq, const float* __restrict__ ck,
                        const int32_t* __restrict__ count_k, int n_qc, int n_kc, int n_pad, float c_log2,
                        float recall, int min_count, int32_t* __restrict__ block_idx,
-                       int32_t* __restrict__ keep_count) {
+                       int32_t* __restrict__ keep_count, const float* __restrict__ scores, int row0,
+                       int chunk_rows) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);   // [n_pad] (mass, ~index)
   float* score = reinterpret_cast<float*>(keys + n_pad);                         // [n_kc]
@@ -205,13 +336,21 @@ select_adaptive_kernel(const float* __restrict__ cq, const float* __restrict__ c
   __shared__ float s_red[8];
   __shared__ int s_warp[64];
   __shared__ int s_need;
-  const int p = blockIdx.y, i = blockIdx.x;
+  const int p = blockIdx.y, i = row0 + blockIdx.x;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* ckp = ck + (size_t)p * n_kc * D;
   const int32_t* cnt = count_k + (size_t)p * n_kc;
   for (int e = tid; e < D; e += 256) qs[e] = cq[((size_t)p * n_qc + i) * D + e];
   __syncthreads();
   float mx = -INFINITY;
+  if (scores) {
+    const float* srow = scores + ((size_t)p * chunk_rows + (i - row0)) * n_kc;
+    for (int j = tid; j < n_kc; j += 256) {
+      const float v = __ldg(srow + j);
+      score[j] = v;
+      mx = fmaxf(mx, v);
+    }
+  } else
   for (int j = tid; j < n_kc; j += 256) {
     float acc = 0.f;
     const float4* row = reinterpret_cast<const float4*>(ckp + (size_t)j * D);
@@ -303,23 +442,36 @@ select_adaptive_kernel(const float* __restrict__ cq, const float* __restrict__ c
 
 int launch_select_adaptive(const float* cq, const float* ck, const int32_t* count_k, int P, int n_qc, int n_kc,
                            int D, float scale, float recall, int min_count, int32_t* block_idx,
-                           int32_t* keep_count, cudaStream_t st) {
+                           int32_t* keep_count, float* score_ws, size_t score_floats, cudaStream_t st) {
   int n_pad = 1;
   while (n_pad < n_kc) n_pad <<= 1;
   const size_t smem = (size_t)n_pad * 8 + (size_t)n_kc * 4 + (size_t)D * 4;
   if (smem > 200 * 1024) return CA_ERR_UNSUPPORTED;
   const float c_log2 = scale * 1.4426950408889634f;      // one float32 product, as in the definition
-  dim3 grid(n_qc, P);
-  if (D == 64) {
-    auto k = select_adaptive_kernel<64>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, 256, smem, st>>>(cq, ck, count_k, n_qc, n_kc, n_pad, c_log2, recall, min_count, block_idx, keep_count);
-  } else {
-    auto k = select_adaptive_kernel<128>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<grid, 256, smem, st>>>(cq, ck, count_k, n_qc, n_kc, n_pad, c_log2, recall, min_count, block_idx, keep_count);
+  auto k64 = select_adaptive_kernel<64>;
+  auto k128 = select_adaptive_kernel<128>;
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k64, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k128, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  const int chunk = select_chunk_rows(P, n_qc, n_kc, score_ws ? score_floats : 0);
+  const int step = chunk == 0 ? n_qc : chunk;
+  for (int row0 = 0; row0 < n_qc; row0 += step) {
+    const int rows = min(step, n_qc - row0);
+    const float* scores = nullptr;
+    if (chunk != 0) {
+      int rc = D == 64 ? launch_score_tiles<64>(cq, ck, P, n_qc, n_kc, row0, chunk, score_ws, st)
+                       : launch_score_tiles<128>(cq, ck, P, n_qc, n_kc, row0, chunk, score_ws, st);
+      if (rc != CA_OK) return rc;
+      scores = score_ws;
+    }
+    dim3 grid(rows, P);
+    if (D == 64)
+      k64<<<grid, 256, smem, st>>>(cq, ck, count_k, n_qc, n_kc, n_pad, c_log2, recall, min_count, block_idx,
+                                   keep_count, scores, row0, step);
+    else
+      k128<<<grid, 256, smem, st>>>(cq, ck, count_k, n_qc, n_kc, n_pad, c_log2, recall, min_count, block_idx,
+                                    keep_count, scores, row0, step);
+    CA_LAUNCH_CHECK();
   }
-  CA_LAUNCH_CHECK();
   return CA_OK;
 }
 
