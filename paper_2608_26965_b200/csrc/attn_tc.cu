@@ -8,10 +8,12 @@
 // half-steps of 64, alternating between two 64-column score buffers in tensor
 // memory, so that the tensor core works on one half-step while the softmax
 // warps work on the other:
-//     S_b = Q K_h^T        tcgen05.mma, both operands in shared memory
+//     S_b = Q K_h^T        tcgen05.mma, K from shared memory; Q from shared memory (d = 128) or from a
+//                          copy in tensor memory (d = 64)
 //     P_b = exp2(S_b c - m) four softmax warps, one query row per thread; P is
 //                          written back over S_b as packed bf16
-//     O  += P_b V_h        tcgen05.mma, P from tensor memory, V from shared memory (MN-major)
+//     O  += P_b V_h        tcgen05.mma, P from tensor memory, V from shared memory (MN-major); at
+//                          d = 64 V is followed by 16 columns of ones, which makes the row sums of P
 // issued as S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  The running maximum is only
 // raised when a half-step exceeds it by 2^8; the softmax warps then rescale O in
 // tensor memory themselves after waiting for the one product that can still be
@@ -19,8 +21,10 @@
 // extra keys, 64 per half-step: their tile holds bf16 hi parts in rows 0-63 and
 // lo parts in rows 64-127, accumulated by two products so the centroid logits
 // keep fp32-level accuracy; logit bias ln|c|, selected clusters masked; values are
-// the value centroids.  Warp 0 issues TMA, warp 1 issues MMAs, warps 2-5 do the
-// softmax and the epilogue (rows scattered back to the original order).
+// the value centroids.  Block lists may be ragged (a length per query cluster).
+// Warp 0 issues TMA, warp 1 issues MMAs (all lanes run the loop, one elected lane
+// issues), warps 2-5 do the softmax and the epilogue (rows scattered back to the
+// original order).
 #include "kernels.h"
 #include "tc_ptx.cuh"
 

@@ -3,7 +3,9 @@
 // for k = 0, 1, ..., product and sum rounded separately, no fused multiply-add),
 // so the scores -- and with them the selection -- are reproducible bit for bit;
 // the k best per query cluster by (score descending, index ascending), written
-// in ascending index order.
+// in ascending index order.  With few key clusters one kernel scores and
+// selects; with many, the scores are computed in tiles first (score_tile_kernel).
+// The second half of the file is the adaptive (mass-recall) selection.
 #include "kernels.h"
 
 namespace ca {

@@ -18,6 +18,10 @@
 // shared memory (hardware cluster barriers, no spin waits).  Sets of at most
 // kTailRows rows: one CTA finishes the whole subtree in shared memory, all
 // subsets of a level side by side, and writes the permutation once.
+//
+// The basic variant of the splitting (a power iteration per set instead of a
+// coordinate choice, at the end of this file) computes its keys in kernels of
+// its own and reuses the per-level kernel for selection and partition.
 #include <climits>
 #include <cooperative_groups.h>
 
