@@ -436,3 +436,37 @@ def test_end_to_end_asymmetric_clusters_64_by_128():
                                          ck=plan.ck[0, h].cpu().numpy(), cv=plan.cv[0, h].cpu().numpy(),
                                          count_k=plan.count_k[0, h].cpu().numpy())
         assert bf16_close(O[0, h].float().cpu().numpy(), o_ref)
+
+
+# ----------------------------------------------------------------------------
+# Selection on random shapes: both the fused kernel and, from 2,048 key clusters
+# on, the tiled scores + one row per CTA; top-k and adaptive, exact lists.
+# ----------------------------------------------------------------------------
+@pytest.mark.parametrize("seed", range(8))
+def test_selection_random_shapes_exact(seed):
+    r = np.random.default_rng(1000 + seed)
+    d = int(r.choice([64, 128]))
+    H = int(r.integers(1, 3))
+    n_qc = int(r.integers(1, 200))
+    n_kc = int(r.choice([r.integers(1, 300), r.integers(2048, 2600)]))
+    keep = int(r.integers(1, n_kc + 1))
+    cq = (r.standard_normal((H, n_qc, d)) * r.uniform(0.2, 4.0)).astype(np.float32)
+    ck = r.standard_normal((H, n_kc, d)).astype(np.float32)
+    dup = r.integers(0, n_kc, max(1, n_kc // 10))
+    ck[:, dup] = ck[:, dup[0]][:, None, :]                  # a tenth of the key centroids coincide
+    count = r.integers(1, 17, (H, n_kc)).astype(np.int32)
+    c = 16
+    scale = float(np.float32(1.0 / np.sqrt(d)))
+    p = binding.make_problem(1, H, n_qc * c, n_kc * c, d, "fp32", c, c, keep, softmax_scale=scale)
+    plan = binding.Plan(p, DEV)
+    got = plan.select_blocks(to_dev(cq[None]), to_dev(ck[None])).cpu().numpy()[0]
+    recall = float(r.choice([0.3, 0.7, 0.95]))
+    min_count = int(r.integers(1, 20))
+    idx, kc = plan.select_blocks_adaptive(recall, min_count, to_dev(cq[None]), to_dev(ck[None]), to_dev(count[None]))
+    torch.cuda.synchronize()
+    idx, kc = idx.cpu().numpy()[0], kc.cpu().numpy()[0]
+    for h in range(H):
+        assert np.array_equal(got[h], orc.select_blocks(cq[h], ck[h], keep)), (seed, h)
+        want = orc.select_blocks_adaptive(cq[h], ck[h], count[h], recall, min_count, scale=scale)
+        for i, row in enumerate(want):
+            assert kc[h, i] == len(row) and np.array_equal(idx[h, i, :len(row)], row), (seed, h, i)
