@@ -470,3 +470,29 @@ def test_selection_random_shapes_exact(seed):
         want = orc.select_blocks_adaptive(cq[h], ck[h], count[h], recall, min_count, scale=scale)
         for i, row in enumerate(want):
             assert kc[h, i] == len(row) and np.array_equal(idx[h, i, :len(row)], row), (seed, h, i)
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_attention_random_shapes(seed):
+    """Random sizes, cluster sizes, densities and arbitrary permutations (ragged tails on both
+    sides); bf16 on the tensor-core kernel and fp32 on the CUDA-core kernel."""
+    r = np.random.default_rng(2000 + seed)
+    base = "tabular" if r.integers(0, 2) == 0 else "sweep"              # d = 64 / d = 128
+    c_q = int(r.choice([64, 128, 256]))
+    c_k = int(r.choice([16, 32, 64, 128, 256]))
+    n_q = int(r.integers(c_q // 2, 5 * c_q))
+    n_k = int(r.integers(c_k, 40 * c_k))
+    n_kc = -(-n_k // c_k)
+    keep = int(r.integers(1, n_kc + 1))
+    compensate = bool(r.integers(0, 2))
+    w = inputs.WORKLOADS[base].scaled(n_q=n_q, n_k=n_k, cluster=c_q)
+    if seed % 5 == 4:
+        w = w.scaled(dtype="fp32")
+    O, lse, refs = attention_case(w, 2, keep, compensate, perm_seed=seed, cluster_k=c_k)
+    for h, (o_ref, lse_ref) in enumerate(refs):
+        if w.dtype == "fp32":
+            assert np.abs(O[h] - o_ref).max() < 1e-5 and np.abs(lse[h] - lse_ref).max() < 1e-5, (seed, h)
+        else:
+            assert bf16_close(O[h], o_ref), (seed, h, c_q, c_k, n_q, n_k, keep, compensate,
+                                             np.abs(O[h] - o_ref).max())
+            assert np.abs(lse[h] - lse_ref).max() < 2e-2
