@@ -35,35 +35,43 @@ using namespace ptx;
 constexpr int kTcThreads = 192;
 constexpr int kTile = 128;                 // query rows per CTA, key rows per tile
 constexpr int kHalf = 64;                  // keys per half-step
-constexpr uint32_t kTmemCols = 256;        // S_a: [0,64)  S_b: [64,128)  O: [128, 128+D) (+16 row-sum columns, d = 64)
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
-#ifndef CA_STAGGER_NS
-#define CA_STAGGER_NS 400
-#endif
-constexpr unsigned kStaggerNs = CA_STAGGER_NS;
 
 template <int D>
 struct TcCfg {
   static constexpr int PANELS = D / 64;
-  static constexpr int PANEL_BYTES = kTile * 128;            // 128 rows x 128 bytes
+  static constexpr int PANEL_BYTES = kTile * 128;            // query tile: 128 rows x 128 bytes per panel
   static constexpr int TILE_BYTES = PANELS * PANEL_BYTES;
-  static constexpr int STAGES = (D == 64) ? 2 : 1;
+  static constexpr int HALF_PANEL_BYTES = kHalf * 128;       // key/value slot: 64 rows x 128 bytes per panel
+  static constexpr int HALF_BYTES = PANELS * HALF_PANEL_BYTES;
+  // Per CTA the half-steps form one dependent chain (scores -> softmax -> P V -> next scores) whose
+  // length is set by latencies, not by any pipe, and an SM has throughput to spare: what counts is
+  // the number of such chains per SM.  d = 64: one 64-column score buffer + 64 output columns =
+  // 128 columns of tensor memory and 48 KB of shared memory per CTA, four CTAs per SM.  d = 128: the
+  // output alone takes 128 columns; two score buffers, 256 columns, two CTAs per SM.
+  static constexpr int NBUF = (D == 64) ? 1 : 2;
+  static constexpr int NBAR = 2;                              // barrier rings (>= every lead below)
+  static constexpr uint32_t TMEM_COLS = (D == 64) ? 128 : 256;
+  static constexpr int CTAS_PER_SM = (D == 64) ? 4 : 2;
+  // key and value slots of 64 rows (one half-step each; a centroid half-step takes two key slots).
+  // The keys of half-step i are loaded once S(i - K_LEAD) has completed, so the slots of at most
+  // K_LEAD half-steps are live (K_LEAD_CEN for centroid half-steps); likewise for the values.
+  static constexpr int NK = 2;
+  static constexpr int NV = 2;
+  static constexpr int K_LEAD = 2;
+  static constexpr int K_LEAD_CEN = 1;
+  static constexpr bool ROWSUM_MMA = false;
+  static constexpr int PV_N = D;
+  static constexpr bool Q_IN_TMEM = false;
+  static constexpr int TMEM_Q = 0;
   // shared memory layout (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-  static constexpr int OFF_V = OFF_K + STAGES * TILE_BYTES;
-  // d = 64: the product P V is taken with 16 extra value columns that hold 1.0, so that the
-  // tensor core also delivers the row sums of P (the accumulator has no room for them at d = 128)
-  static constexpr bool ROWSUM_MMA = (D == 64);
-  static constexpr int PV_N = ROWSUM_MMA ? D + 16 : D;
-  // d = 64: tensor memory also has room for the query tile (32 columns of bf16 pairs), so Q K^T
-  // reads its A operand there instead of re-reading 4 KB of shared memory per instruction
-  static constexpr bool Q_IN_TMEM = (D == 64);
-  static constexpr int TMEM_Q = kTile + PV_N;               // first column of the query tile
-  static constexpr int OFF_ONES = OFF_V + STAGES * TILE_BYTES;      // 64 key rows x 128 bytes of bf16 ones
-  static constexpr int OFF_BIAS = OFF_ONES + (ROWSUM_MMA ? kHalf * 128 : 0);     // 4 x 64 floats
-  static constexpr int OFF_BAR = OFF_BIAS + 4 * kHalf * 4;
-  static constexpr int NUM_BARS = 9 + 4 * STAGES;
+  static constexpr int OFF_V = OFF_K + NK * HALF_BYTES;
+  static constexpr int OFF_ONES = OFF_V + NV * HALF_BYTES;
+  static constexpr int OFF_BIAS = OFF_ONES;                         // 8 x 64 floats
+  static constexpr int OFF_BAR = OFF_BIAS + 8 * kHalf * 4;
+  static constexpr int NUM_BARS = 3 + 3 * NBAR + NK + NV;           // q_full, o_done, q_tmem, three rings, per slot
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;           // tmem base, abort flag
   static constexpr int OFF_BITMAP = OFF_MISC + 16;
 };
@@ -86,7 +94,7 @@ __host__ __device__ inline int selected_tiles(int keep, int c_k) {
 }
 
 template <int D>
-__global__ void __launch_bounds__(kTcThreads, 2)
+__global__ void __launch_bounds__(kTcThreads, TcCfg<D>::CTAS_PER_SM)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ck,
                const __grid_constant__ CUtensorMap tm_cv, const TcParams prm) {
@@ -98,15 +106,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t s_q = s_base + C::OFF_Q, s_k = s_base + C::OFF_K, s_v = s_base + C::OFF_V;
   float* bias = reinterpret_cast<float*>(smem + C::OFF_BIAS);
   const uint32_t bar0 = s_base + C::OFF_BAR;
-  const uint32_t b_q_full = bar0, b_o_done = bar0 + 8;
-  const uint32_t b_q_tmem = bar0 + 8 * (C::NUM_BARS - 1);     // the query tile has been copied to tensor memory
-  auto b_s_full = [&](int b) { return bar0 + 16 + 8 * b; };
-  auto b_p_ready = [&](int b) { return bar0 + 32 + 8 * b; };
-  auto b_pv_done = [&](int b) { return bar0 + 48 + 8 * b; };
-  auto b_k_full = [&](int s) { return bar0 + 64 + 8 * s; };
-  auto b_k_empty = [&](int s) { return bar0 + 64 + 8 * (C::STAGES + s); };
-  auto b_v_full = [&](int s) { return bar0 + 64 + 8 * (2 * C::STAGES + s); };
-  auto b_v_empty = [&](int s) { return bar0 + 64 + 8 * (3 * C::STAGES + s); };
+  const uint32_t b_q_full = bar0, b_o_done = bar0 + 8, b_q_tmem = bar0 + 16;
+  auto b_s_full = [&](int b) { return bar0 + 24 + 8 * b; };
+  auto b_p_ready = [&](int b) { return bar0 + 24 + 8 * (C::NBAR + b); };
+  auto b_pv_done = [&](int b) { return bar0 + 24 + 8 * (2 * C::NBAR + b); };
+  auto b_k_full = [&](int s) { return bar0 + 24 + 8 * (3 * C::NBAR + s); };
+  auto b_v_full = [&](int s) { return bar0 + 24 + 8 * (3 * C::NBAR + C::NK + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
   unsigned* bitmap = reinterpret_cast<unsigned*>(smem + C::OFF_BITMAP);
@@ -125,18 +130,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int keep = prm.keep_count ? prm.keep_count[(size_t)p * prm.n_qc + qc] : prm.keep;
   const int sel_tiles = selected_tiles(keep, prm.c_k);
   const int cen_tiles = prm.compensate ? prm.cen_tiles : 0;
-  const int loads = sel_tiles + cen_tiles;             // K/V tile loads
   const int steps = 2 * sel_tiles + cen_tiles;         // half-steps of 64 keys
 
   if (tid == 0) {
     mbar_init(b_q_full, 1);
     mbar_init(b_q_tmem, 4);
     mbar_init(b_o_done, 1);
-    for (int b = 0; b < 2; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 4); mbar_init(b_pv_done(b), 1); }
-    for (int s = 0; s < C::STAGES; ++s) {
-      mbar_init(b_k_full(s), 1); mbar_init(b_k_empty(s), 1);
-      mbar_init(b_v_full(s), 1); mbar_init(b_v_empty(s), 1);
-    }
+    for (int b = 0; b < C::NBAR; ++b) { mbar_init(b_s_full(b), 1); mbar_init(b_p_ready(b), 4); mbar_init(b_pv_done(b), 1); }
+    for (int s = 0; s < C::NK; ++s) mbar_init(b_k_full(s), 1);
+    for (int s = 0; s < C::NV; ++s) mbar_init(b_v_full(s), 1);
     *abort_flag = 0;
     fence_mbar_init();
   }
@@ -154,23 +156,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     fence_proxy_async();
   }
   if (warp == 1) {                       // this warp owns the TMEM allocation
-    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tmem_alloc(smem_u32(tmem_slot), C::TMEM_COLS);
     tmem_relinquish();
   }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + kTile;
-  // Two CTAs share an SM and run the same loop at the same rate.  Started together they stay in
-  // phase: both sets of softmax warps want the special-function unit at the same time and both
-  // leave it idle at the same time.  The CTA that got the upper half of tensor memory starts a
-  // fraction of a half-step later, so that one CTA's exponentials run under the other's
-  // remaining work.
-  if ((tmem_base & 0xffffu) >= kTmemCols) __nanosleep(kStaggerNs);
+  const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + C::NBUF * kHalf;
+  // key slots used before half-step u (a centroid half-step takes two: hi and lo parts)
+  auto kslot_of = [&](int u) { return u < 2 * sel_tiles ? u : 2 * sel_tiles + 2 * (u - 2 * sel_tiles); };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
+    // Loads run in the order the tensor core consumes them: the keys of half-step i (needed by
+    // S(i), issued NBUF half-steps early) and the values of half-step i - NBUF.  A slot is free
+    // again when the product that read it has completed, which is what the barriers s_full and
+    // pv_done of that half-step announce; no separate "empty" barriers or commits.
     if (lane == 0) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
       const int q_row = (p * prm.n_qc + qc) * prm.c_q + half * kTile;
@@ -178,41 +180,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(s_q + pn * C::PANEL_BYTES, &tm_q, pn * 64, q_row, b_q_full);
       bool ok = true;
       auto load_rows = [&](uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
-        for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(dst + pn * C::PANEL_BYTES, map, pn * 64, row, bar);
+        for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(dst + pn * C::HALF_PANEL_BYTES, map, pn * 64, row, bar);
       };
-      // rows of a selected-cluster tile: sub-boxes of min(c_k, 128) rows
-      auto load_selected = [&](uint32_t dst, const CUtensorMap* map, int t, uint32_t bar) {
-        if (prm.c_k >= kTile) {
-          const int per = prm.c_k / kTile;
-          const int j = sel[t / per];
-          load_rows(dst, map, (p * prm.n_kc + j) * prm.c_k + (t % per) * kTile, bar);
+      // the 64 rows of half-step u of the selected clusters: one box, or several boxes of c_k rows
+      auto load_selected = [&](uint32_t dst, const CUtensorMap* map, int u, uint32_t bar) {
+        if (prm.c_k >= kHalf) {
+          const int pos = u * kHalf;                       // position in the concatenated selected rows
+          const int j = sel[min(pos / prm.c_k, keep - 1)];     // a filler half-step repeats the last cluster (masked)
+          load_rows(dst, map, (p * prm.n_kc + j) * prm.c_k + pos % prm.c_k, bar);
         } else {
-          const int per = kTile / prm.c_k;
-          for (int u = 0; u < per; ++u) {
-            int e = t * per + u;
-            if (e >= keep) e = keep - 1;          // filler rows, masked by the softmax
+          const int per = kHalf / prm.c_k;
+          for (int x = 0; x < per; ++x) {
+            int e = u * per + x;
+            if (e >= keep) e = keep - 1;                   // filler rows, masked by the softmax
             const int j = sel[e];
             for (int pn = 0; pn < C::PANELS; ++pn)
-              tma_load_2d(dst + pn * C::PANEL_BYTES + u * prm.c_k * 128, map, pn * 64,
+              tma_load_2d(dst + pn * C::HALF_PANEL_BYTES + x * prm.c_k * 128, map, pn * 64,
                           (p * prm.n_kc + j) * prm.c_k, bar);
           }
         }
       };
-      for (int t = 0; t < loads && ok; ++t) {
-        const int s = t % C::STAGES;
-        if (t >= C::STAGES) ok = mbar_wait(b_k_empty(s), ((t / C::STAGES) - 1) & 1, abort_flag, prm.status);
-        if (!ok) break;
-        mbar_expect_tx(b_k_full(s), C::TILE_BYTES);
-        if (t < sel_tiles) load_selected(s_k + s * C::TILE_BYTES, &tm_k, t, b_k_full(s));
-        else load_rows(s_k + s * C::TILE_BYTES, &tm_ck, (p * prm.cen_tiles + (t - sel_tiles)) * kTile, b_k_full(s));
-        if (t >= C::STAGES) ok = mbar_wait(b_v_empty(s), ((t / C::STAGES) - 1) & 1, abort_flag, prm.status);
-        if (!ok) break;
-        if (t < sel_tiles) {
-          mbar_expect_tx(b_v_full(s), C::TILE_BYTES);
-          load_selected(s_v + s * C::TILE_BYTES, &tm_v, t, b_v_full(s));
-        } else {                                            // 64 value centroids
-          mbar_expect_tx(b_v_full(s), C::TILE_BYTES / 2);
-          load_rows(s_v + s * C::TILE_BYTES, &tm_cv, (p * prm.cen_tiles + (t - sel_tiles)) * kHalf, b_v_full(s));
+      // A slot is reused when the product that read it has completed.  Products complete in the
+      // order of their issue, so it is enough to wait for a later one; the one waited for is chosen
+      // so that its barrier cannot complete another phase before this thread has looked (the next
+      // product on the same score buffer needs the very load that follows the wait).
+      for (int i = 0; i < steps + C::NBUF && ok; ++i) {
+        if (i < steps) {
+          const bool centroid = i >= 2 * sel_tiles;
+          const int parts = centroid ? 2 : 1;
+          const int w = i - (centroid ? C::K_LEAD_CEN : C::K_LEAD);
+          if (w >= 0) ok = mbar_wait(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          for (int g = 0; g < parts && ok; ++g) {
+            const int kc = kslot_of(i) + g, slot = kc % C::NK;
+            mbar_expect_tx(b_k_full(slot), C::HALF_BYTES);
+            const uint32_t dst = s_k + slot * C::HALF_BYTES;
+            if (!centroid) load_selected(dst, &tm_k, i, b_k_full(slot));
+            else load_rows(dst, &tm_ck, (p * prm.cen_tiles + (i - 2 * sel_tiles)) * kTile + g * kHalf, b_k_full(slot));
+          }
+        }
+        const int j = i - C::NBUF;
+        if (j >= 0 && ok) {
+          const int slot = j % C::NV;
+          const int w = j - C::NV;
+          if (w >= 0) ok = mbar_wait(b_pv_done(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          if (!ok) break;
+          mbar_expect_tx(b_v_full(slot), C::HALF_BYTES);
+          const uint32_t dst = s_v + slot * C::HALF_BYTES;
+          if (j < 2 * sel_tiles) load_selected(dst, &tm_v, j, b_v_full(slot));
+          else load_rows(dst, &tm_cv, (p * prm.cen_tiles + (j - 2 * sel_tiles)) * kHalf, b_v_full(slot));
         }
       }
     }
@@ -224,63 +239,52 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
       bool ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status));
-      if (C::Q_IN_TMEM && ok) { ok = __all_sync(0xffffffffu, mbar_wait(b_q_tmem, 0, abort_flag, prm.status)); tc_fence_after(); }
-      // load index of half-step u (the shared-memory slot is the load index modulo the stages)
-      auto load_of = [&](int u) { return u < 2 * sel_tiles ? u >> 1 : sel_tiles + (u - 2 * sel_tiles); };
+      // descriptors differ from a base one only in the start-address field (units of 16 bytes):
+      // the base descriptors are built once, the per-instruction part is an addition
       const uint64_t q_desc0 = smem_desc_sw128(s_q, 16, 1024);
       const uint64_t k_desc0 = smem_desc_sw128(s_k, 16, 1024);
+      const uint64_t v_desc0 = smem_desc_sw128(s_v, C::HALF_PANEL_BYTES, 1024);
       auto issue_s = [&](int u) {
-        const int L = load_of(u), s = L % C::STAGES, b = u & 1;
+        const int buf = u % C::NBUF;
         const bool centroid = u >= 2 * sel_tiles;
-        if (centroid || b == 0) {
-          if (!__all_sync(0xffffffffu, mbar_wait(b_k_full(s), (L / C::STAGES) & 1, abort_flag, prm.status))) return false;
-          tc_fence_after();
-        }
-        // descriptors differ from a base one only in the start-address field (units of 16 bytes):
-        // the base descriptors are built once, the per-instruction part is an addition
-        const int parts = centroid ? 2 : 1;               // centroid tile: hi rows 0-63, lo rows 64-127
-        if (elect_one()) {
+        const int parts = centroid ? 2 : 1;               // centroid keys: bf16 hi parts, then lo parts
         for (int g = 0; g < parts; ++g) {
-          const uint32_t rows = (centroid ? g : b) * (kHalf * 128);   // 64 rows = 8192 bytes inside a panel
-          const uint64_t kd = k_desc0 + ((s * C::TILE_BYTES + rows) >> 4);
+          const int kc = kslot_of(u) + g, slot = kc % C::NK;
+          if (!__all_sync(0xffffffffu, mbar_wait(b_k_full(slot), (kc / C::NK) & 1, abort_flag, prm.status))) return false;
+          tc_fence_after();
+          if (elect_one()) {
+            const uint64_t kd = k_desc0 + ((slot * C::HALF_BYTES) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
-            const uint32_t off16 = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
-            if (C::Q_IN_TMEM) mma_ts(tmem_s + b * kHalf, tmem_base + C::TMEM_Q + ks * 8, kd + off16, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
-            else mma_ss(tmem_s + b * kHalf, q_desc0 + off16, kd + off16, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            for (int ks = 0; ks < D / 16; ++ks) {
+              // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
+              const uint32_t qoff = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
+              const uint32_t koff = ((ks / 4) * C::HALF_PANEL_BYTES + (ks % 4) * 32) >> 4;
+              mma_ss(tmem_s + buf * kHalf, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            }
+            if (g == parts - 1) mma_commit(b_s_full(u % C::NBAR));
           }
+          __syncwarp();
         }
-        if (centroid || b == 1) mma_commit(b_k_empty(s));
-        mma_commit(b_s_full(b));
-        }
-        __syncwarp();
         return true;
       };
-      if (ok && steps > 0) ok = issue_s(0);
-      if (ok && steps > 1) ok = issue_s(1);
+      for (int u = 0; u < C::NBUF && u < steps && ok; ++u) ok = issue_s(u);
       for (int u = 0; u < steps && ok; ++u) {
-        const int L = load_of(u), s = L % C::STAGES, b = u & 1;
-        const bool centroid = u >= 2 * sel_tiles;
-        ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(b), (u >> 1) & 1, abort_flag, prm.status));
-        if (ok && (centroid || b == 0)) ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(s), (L / C::STAGES) & 1, abort_flag, prm.status));
+        const int buf = u % C::NBUF, slot = u % C::NV;
+        ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(slot), (u / C::NV) & 1, abort_flag, prm.status));
         if (!ok) break;
         tc_fence_after();
-        const uint32_t vt = s_v + s * C::TILE_BYTES + (centroid ? 0 : b) * (kHalf * 128);
-        // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d.  With the row-sum
-        // columns the panel after the values is the block of ones, wherever the value tile sits.
-        const uint32_t next_panel = C::ROWSUM_MMA ? (s_base + C::OFF_ONES) - vt : (uint32_t)C::PANEL_BYTES;
-        const uint64_t vd = smem_desc_sw128(vt, next_panel, 1024);
-        const uint32_t p_cols = tmem_s + b * kHalf;
+        // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d
+        const uint64_t vd = v_desc0 + ((slot * C::HALF_BYTES) >> 4);
+        const uint32_t p_cols = tmem_s + buf * kHalf;
         if (elect_one()) {
 #pragma unroll
           for (int ks = 0; ks < kHalf / 16; ++ks)
             mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(b_pv_done(b));
-          if (centroid || b == 1) mma_commit(b_v_empty(s));
+          mma_commit(b_pv_done(u % C::NBAR));
         }
         __syncwarp();
-        if (u + 2 < steps) ok = issue_s(u + 2);
+        if (u + C::NBUF < steps) ok = issue_s(u + C::NBUF);
       }
       if (elect_one()) mma_commit(b_o_done);
     }
@@ -321,13 +325,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     const int ck_shift = __ffs(prm.c_k) - 1;
     bool ok = true;
     for (int u = 0; u < steps && ok; ++u) {
-      const int b = u & 1;
-      const uint32_t t_s = tmem_s + lane_addr + b * kHalf;
+      const int b = u & 1;                               // half of a 128-row tile (geometry of the keys)
+      const int buf = u % C::NBUF;                       // score buffer
+      const uint32_t t_s = tmem_s + lane_addr + buf * kHalf;
       // per-column additive term (log2 units): only half-steps with masked or weighted columns need
       // it.  `masked` depends on the half-step only, so it is uniform over the 128 threads.
       bool masked = false;
-      // four buffers: a thread can run at most two half-steps ahead of the slowest one
-      float* bz = bias + (u & 3) * kHalf;
+      // eight buffers: a thread can run at most NBUF half-steps ahead of the slowest one
+      float* bz = bias + (u & 7) * kHalf;
       if (u < 2 * sel_tiles) {
         // cluster sizes are powers of two: positions are split with shifts and masks
         const int t = u >> 1;
@@ -355,13 +360,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
 
-      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(b), (u >> 1) & 1, abort_flag, prm.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
       if (!ok) break;
       tc_fence_after();
       if (quarter * 32 >= q_rows) {          // this warp's rows are padding of a 64-row query cluster
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(b_p_ready(b));
+        if (lane == 0) mbar_arrive(b_p_ready(u % C::NBAR));
         continue;
       }
       // The loops over the two 32-column chunks are kept rolled: the body of a half-step is
@@ -407,8 +412,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         if (!C::ROWSUM_MMA) l_run *= alpha;
         if (u > 0) {
-          // S(u) complete means every product up to PV(u-2) is complete; PV(u-1) may still run
-          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done(b ^ 1), ((u - 1) >> 1) & 1, abort_flag, prm.status));
+          // products complete in the order of their issue: once P V (u-1) is complete, all earlier are
+          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status));
           if (!ok) break;
           tc_fence_after();
 #pragma unroll 1
@@ -467,7 +472,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       tmem_wait_st();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(b_p_ready(b));
+      if (lane == 0) mbar_arrive(b_p_ready(u % C::NBAR));
     }
 
     // epilogue: O / l, rows back to their original positions
@@ -507,7 +512,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem_base, kTmemCols);
+  if (warp == 1) tmem_dealloc(tmem_base, C::TMEM_COLS);
 }
 
 // ---------------------------------------------------------------------------
@@ -611,11 +616,11 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
     CA_LAUNCH_CHECK();
   }
   CUtensorMap maps[5];
-  const int kbox = pr.cluster_k < kTile ? pr.cluster_k : kTile;
+  const int kbox = pr.cluster_k < kHalf ? pr.cluster_k : kHalf;      // key/value slots hold 64 rows
   bool ok = make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, pr.cluster_q < kTile ? pr.cluster_q : kTile) &&
             make_map(&maps[1], Kp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
             make_map(&maps[2], Vp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
-            make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kTile) &&
+            make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kHalf) &&
             make_map(&maps[4], vb, (size_t)P * cen_tiles * kHalf, D, kHalf);
   if (!ok) return CA_ERR_CUDA;
   TcParams prm;
