@@ -36,7 +36,7 @@ struct ClusterWs {
   double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
   float *roots32, *basis32, *WK32, *biasK, *biasQ;
   float *Qprime, *Yq, *Yk;
-  __nv_bfloat16 *wt_hi, *wt_lo;
+  __nv_bfloat16 *wt_hi, *wt_lo, *wt2_hi, *wt2_lo;
   int32_t *perm_q_tmp, *perm_k_tmp;
   uint32_t *keybuf_q, *keybuf_k;
   size_t bytes;
@@ -71,6 +71,8 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
     w.Qprime = c.take<float>(P * (size_t)p->n_q * D);
     w.wt_hi = c.take<__nv_bfloat16>(P * DD);
     w.wt_lo = c.take<__nv_bfloat16>(P * DD);
+    w.wt2_hi = c.take<__nv_bfloat16>(P * DD);
+    w.wt2_lo = c.take<__nv_bfloat16>(P * DD);
     if (need_yq) w.Yq = c.take<float>(P * (size_t)p->n_q * D);
     if (need_yk) w.Yk = c.take<float>(P * (size_t)p->n_k * D);
   }
@@ -80,6 +82,30 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
   w.keybuf_k = c.take<uint32_t>(P * (size_t)p->n_k);
   w.bytes = c.used();
   return w;
+}
+
+// The query side and the key side of cluster_qk are independent once the two factors exist.  The
+// query side runs on a second stream that forks from the caller's stream and joins it again
+// before the call returns (events only: nothing waits on the host, and a stream capture of the
+// caller's stream picks the side stream up as a parallel branch).  One stream and two events per
+// device, created at the first call on that device.
+struct SideStream {
+  cudaStream_t stream = nullptr;
+  cudaEvent_t fork = nullptr, join = nullptr;
+  bool ready = false;
+};
+SideStream* side_stream() {
+  static SideStream table[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  SideStream& s = table[dev];
+  if (!s.ready) {
+    if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    s.ready = true;
+  }
+  return &s;
 }
 
 #define CA_TRY(expr)               \
@@ -153,43 +179,62 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_cholesky_factor(w.metric, 2 * P, D, w.roots, w.roots32, st));
     double* Rq = w.roots;
     const float* Rk32 = w.roots32 + (size_t)P * DD;
-    // covariance of the transformed keys K F_q:  F_q^T C_K F_q / n_k
     double* covK = w.cov;
     double* covQ = w.cov + (size_t)P * DD;
+    // ---- fork: the query side continues on the side stream
+    SideStream* side = side_stream();
+    if (!side) return CA_ERR_CUDA;
+    cudaStream_t sq = side->stream;
+    CA_RETURN_IF_CUDA(cudaEventRecord(side->fork, st));
+    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(sq, side->fork, 0));
+    // query representation r(q) = F_k^T q / |F_k^T q|, its covariance, its principal components,
+    // the coordinates Y = (r(q) - mean) E_Q
+    const float* EQ32 = w.basis32 + (size_t)P * DD;
+    if (tc) {
+      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
+                                 w.wt2_hi, w.wt2_lo, w.status, sq));
+      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, w.status, sq));
+    } else {
+      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
+      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, sq));
+    }
+    CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, sq));
+    CA_TRY(launch_eigh(covQ, P, D, w.basis + (size_t)P * DD, w.basis32 + (size_t)P * DD, nullptr, sq));
+    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, sq));
+    if (tc) {
+      CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
+                                 w.wt2_lo, w.status, sq));
+    } else {
+      CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
+    }
+    CA_TRY(launch_split(yq_out, nullptr, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
+                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 1, sq));
+    CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, sq));
+    CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
+    // ---- key side on the caller's stream: covariance of the transformed keys K F_q
+    // (F_q^T C_K F_q / n_k, d x d algebra), its principal components, Y = (K - kbar) F_q E_K
     CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
     CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, unnormalized ? 1.0 : 1.0 / (double)p->n_k, 0, covK, nullptr, st));
-    // query representation r(q) = F_k^T q / |F_k^T q| and its covariance
-    if (tc) {
-      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo, w.wt_hi,
-                                 w.wt_lo, w.status, st));
-      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, w.status, st));
-    } else {
-      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, w.Qprime, st));
-      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, st));
-    }
-    CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, st));
-    // global principal components of both transformed sets (Section 3.2.1)
-    CA_TRY(launch_eigh(w.cov, 2 * P, D, w.basis, w.basis32, nullptr, st));
-    double* EK = w.basis;
-    const float* EQ32 = w.basis32 + (size_t)P * DD;
-    // keys: Y = (K - kbar) F_q E_K ; queries: Y = (r(q) - mean) E_Q
-    CA_TRY(launch_small_matmul(Rq, EK, P, D, 1.0, 0, w.WK, w.WK32, st));
+    CA_TRY(launch_eigh(covK, P, D, w.basis, w.basis32, nullptr, st));
+    CA_TRY(launch_small_matmul(Rq, w.basis, P, D, 1.0, 0, w.WK, w.WK32, st));
     CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st));
-    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, st));
     if (tc) {
-      CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr,
-                                 w.wt_hi, w.wt_lo, w.status, st));
-      CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr,
-                                 w.wt_hi, w.wt_lo, w.status, st));
+      CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
+                                 w.wt_lo, w.status, st));
     } else {
       CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
-      CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, st));
     }
-    yq = yq_out;
-    yk = yk_out;
+    CA_TRY(launch_split(nullptr, yk_out, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
+                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 2, st));
+    CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
+    CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+    // ---- join
+    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->join, 0));
+    return CA_OK;
   }
+  // coordinates given by the caller: split and gather only
   CA_TRY(launch_split(yq, yk, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
-                      perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, st));
+                      perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 3, st));
   CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
   CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
   CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));

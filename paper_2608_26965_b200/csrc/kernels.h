@@ -39,7 +39,7 @@ int launch_bias(const double* sum, const float* W, int P, int D, int n, float* b
 int split_levels_for(int n, int c);
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
-                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st);
+                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st);
 
 // permute.cu
 int launch_split_basic(const void* Q, const void* K, int dtype, const float* A_q, const float* A_k,

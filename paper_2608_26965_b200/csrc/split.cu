@@ -114,6 +114,7 @@ struct SplitSide {
   int32_t* perm_out;       // [P][n]
   uint32_t* keybuf;        // [P][n] staging for sets larger than the shared-memory windows
   int n, c, levels, tail_level;
+  int active;              // 0: this launch leaves the side alone (the two sides can run on different streams)
 };
 
 struct SplitParams {
@@ -145,7 +146,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   const int which = blockIdx.y / prm.problems;
   const int p = blockIdx.y % prm.problems;
   const SplitSide sd = prm.side[which];
-  if (prm.level >= sd.tail_level) return;             // uniform over the cluster
+  if (!sd.active || prm.level >= sd.tail_level) return;   // uniform over the cluster
   const SegmentRef seg = locate_segment(sd.n, sd.c, prm.level, blockIdx.x / csize);
   if (!seg.active) return;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
@@ -381,7 +382,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
   const int p = blockIdx.y % prm.problems;
   const SplitSide sd = prm.side[which];
   const int level = sd.tail_level;
-  if ((int)blockIdx.x >= (1 << level)) return;
+  if (!sd.active || (int)blockIdx.x >= (1 << level)) return;
   const SegmentRef root = locate_segment(sd.n, sd.c, level, blockIdx.x);
   if (!root.active) return;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -627,14 +628,17 @@ static int tail_level_for(int n, int c) {
 
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
-                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, cudaStream_t st) {
+                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st) {
+  // sides: bit 0 = queries, bit 1 = keys
   auto level_kernel = D == 64 ? split_level_kernel<64> : split_level_kernel<128>;
   auto tail_kernel = D == 64 ? split_tail_kernel<64> : split_tail_kernel<128>;
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRowsMax * 8));
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(tail_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)sizeof(TailSmem)));
+  const bool do_q = (sides & 1) != 0, do_k = (sides & 2) != 0;
   const int tail_q = tail_level_for(n_q, c_q), tail_k = tail_level_for(n_k, c_k);
-  const int top_levels = tail_q > tail_k ? tail_q : tail_k;
+  const int top_q = do_q ? tail_q : 0, top_k = do_k ? tail_k : 0;
+  const int top_levels = top_q > top_k ? top_q : top_k;
   SplitParams prm;
   prm.D = D; prm.problems = problems; prm.keys_in = 0;
   // per-level launches write alternately to tmp/out so that the tail kernel, which runs last,
@@ -650,6 +654,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
       sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
       sd.levels = split_levels_for(sd.n, sd.c);
       sd.tail_level = tail;
+      sd.active = (w == 0 ? do_q : do_k) ? 1 : 0;
       // level l of this side (l < tail) writes tmp if (tail - 1 - l) is even, else out;
       // the tail kernel (level == tail) reads what level tail-1 wrote and writes out
       const bool to_tmp = ((tail - 1 - level) % 2) == 0;
@@ -666,8 +671,8 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
     fill(level);
     prm.level = level;
     int max_seg = 1;
-    if (level < tail_q) max_seg = max_segment_at_level(n_q, c_q, level);
-    if (level < tail_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
+    if (level < top_q) max_seg = max_segment_at_level(n_q, c_q, level);
+    if (level < top_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
     int csize = 1;
     while (csize < kMaxCluster && max_seg > csize * 8192) csize *= 2;
     const int per_cta = (max_seg + csize - 1) / csize;
@@ -688,7 +693,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
   fill(top_levels);       // any level >= both tails selects the tail buffers
   prm.level = top_levels;
   prm.smem_rows = 0;
-  const int slots = 1 << (tail_q > tail_k ? tail_q : tail_k);
+  const int slots = 1 << ((do_q ? tail_q : 0) > (do_k ? tail_k : 0) ? (do_q ? tail_q : 0) : (do_k ? tail_k : 0));
   tail_kernel<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(TailSmem), st>>>(prm);
   CA_LAUNCH_CHECK();
   return CA_OK;
@@ -887,6 +892,7 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
       sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
       sd.levels = w == 0 ? lev_q : lev_k;
       sd.tail_level = run;                               // every level runs as a launch of its own
+      sd.active = 1;
       sd.perm_out = to_tmp ? tmp : out;
       sd.perm_in = level == 0 ? nullptr : (to_tmp ? out : tmp);
       BasicSide& bs = bp.side[w];
