@@ -36,6 +36,7 @@ constexpr int kTcThreads = 192;
 constexpr int kTile = 128;                 // query rows per CTA, key rows per tile
 constexpr int kHalf = 64;                  // keys per half-step
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
+constexpr float kDanger = 96.0f;            // log2 units: exp2 arguments stay below this
 
 template <int D>
 struct TcCfg {
@@ -60,7 +61,6 @@ struct TcCfg {
   static constexpr int NV = 2;
   static constexpr int K_LEAD = 2;
   static constexpr int K_LEAD_CEN = 1;
-  static constexpr bool ROWSUM_MMA = false;
   static constexpr int PV_N = D;
   static constexpr bool Q_IN_TMEM = false;
   static constexpr int TMEM_Q = 0;
@@ -68,8 +68,7 @@ struct TcCfg {
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
   static constexpr int OFF_V = OFF_K + NK * HALF_BYTES;
-  static constexpr int OFF_ONES = OFF_V + NV * HALF_BYTES;
-  static constexpr int OFF_BIAS = OFF_ONES;                         // 8 x 64 floats
+  static constexpr int OFF_BIAS = OFF_V + NV * HALF_BYTES;                     // 8 x 64 floats
   static constexpr int OFF_BAR = OFF_BIAS + 8 * kHalf * 4;
   static constexpr int NUM_BARS = 3 + 3 * NBAR + NK + NV;           // q_full, o_done, q_tmem, three rings, per slot
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;           // tmem base, abort flag
@@ -84,6 +83,7 @@ struct TcParams {
   __nv_bfloat16* O;
   float* lse;
   int* status;
+  int32_t* redo;                  // [B*H, n_qc, 2] per CTA: scores left the range of the fast softmax
   int n_q, n_k, c_q, c_k, keep, list_stride, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
   float scale_log2;
 };
@@ -114,6 +114,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   auto b_v_full = [&](int s) { return bar0 + 24 + 8 * (3 * C::NBAR + C::NK + s); };
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_MISC);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 4);
+  volatile int* redo_flag = reinterpret_cast<volatile int*>(smem + C::OFF_MISC + 8);
   unsigned* bitmap = reinterpret_cast<unsigned*>(smem + C::OFF_BITMAP);
   // member counts of the selected clusters, in list order: looked up every half-step, so they are
   // fetched from global memory once instead of sitting on each half-step's critical path
@@ -140,6 +141,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     for (int s = 0; s < C::NK; ++s) mbar_init(b_k_full(s), 1);
     for (int s = 0; s < C::NV; ++s) mbar_init(b_v_full(s), 1);
     *abort_flag = 0;
+    *redo_flag = 0;
     fence_mbar_init();
   }
   if (q_rows < kTile) {
@@ -148,11 +150,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int pn = e / ((kTile - q_rows) * 8), rem = e % ((kTile - q_rows) * 8);
       *reinterpret_cast<uint4*>(smem + C::OFF_Q + pn * C::PANEL_BYTES + q_rows * 128 + rem * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
-    fence_proxy_async();
-  }
-  if (C::ROWSUM_MMA) {
-    for (int e = tid; e < kHalf * 8; e += kTcThreads)
-      *reinterpret_cast<uint4*>(smem + C::OFF_ONES + e * 16) = make_uint4(0x3F803F80u, 0x3F803F80u, 0x3F803F80u, 0x3F803F80u);
     fence_proxy_async();
   }
   if (warp == 1) {                       // this warp owns the TMEM allocation
@@ -244,47 +241,60 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const uint64_t q_desc0 = smem_desc_sw128(s_q, 16, 1024);
       const uint64_t k_desc0 = smem_desc_sw128(s_k, 16, 1024);
       const uint64_t v_desc0 = smem_desc_sw128(s_v, C::HALF_PANEL_BYTES, 1024);
-      auto issue_s = [&](int u) {
-        const int buf = u % C::NBUF;
-        const bool centroid = u >= 2 * sel_tiles;
-        const int parts = centroid ? 2 : 1;               // centroid keys: bf16 hi parts, then lo parts
-        for (int g = 0; g < parts; ++g) {
-          const int kc = kslot_of(u) + g, slot = kc % C::NK;
-          if (!__all_sync(0xffffffffu, mbar_wait(b_k_full(slot), (kc / C::NK) & 1, abort_flag, prm.status))) return false;
-          tc_fence_after();
-          if (elect_one()) {
-            const uint64_t kd = k_desc0 + ((slot * C::HALF_BYTES) >> 4);
-#pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-              // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
-              const uint32_t qoff = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
-              const uint32_t koff = ((ks / 4) * C::HALF_PANEL_BYTES + (ks % 4) * 32) >> 4;
-              mma_ss(tmem_s + buf * kHalf, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
-            }
-            if (g == parts - 1) mma_commit(b_s_full(u % C::NBAR));
-          }
-          __syncwarp();
+      // The tensor core sits idle between the softmax's arrival and the next product, so that
+      // stretch is kept short: everything a product needs besides the probabilities -- its key and
+      // value slots (loaded long before) and their descriptors -- is waited for and computed BEFORE
+      // the wait for the softmax, and P V (u) and S(u + NBUF) are then issued back to back.
+      auto wait_keys = [&](int un) {
+        const int parts = un >= 2 * sel_tiles ? 2 : 1;      // centroid keys: bf16 hi parts, then lo parts
+        bool got = true;
+        for (int g = 0; g < parts && got; ++g) {
+          const int kc = kslot_of(un) + g;
+          got = __all_sync(0xffffffffu, mbar_wait(b_k_full(kc % C::NK), (kc / C::NK) & 1, abort_flag, prm.status));
         }
-        return true;
+        return got;
       };
-      for (int u = 0; u < C::NBUF && u < steps && ok; ++u) ok = issue_s(u);
-      for (int u = 0; u < steps && ok; ++u) {
-        const int buf = u % C::NBUF, slot = u % C::NV;
-        ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(slot), (u / C::NV) & 1, abort_flag, prm.status));
+      auto fire_s = [&](int un) {                           // elected lane
+        const int parts = un >= 2 * sel_tiles ? 2 : 1;
+        const uint32_t d_cols = tmem_s + (un % C::NBUF) * kHalf;
+        for (int g = 0; g < parts; ++g) {
+          const int slot = (kslot_of(un) + g) % C::NK;
+          const uint64_t kd = k_desc0 + ((slot * C::HALF_BYTES) >> 4);
+#pragma unroll
+          for (int ks = 0; ks < D / 16; ++ks) {
+            // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
+            const uint32_t qoff = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
+            const uint32_t koff = ((ks / 4) * C::HALF_PANEL_BYTES + (ks % 4) * 32) >> 4;
+            mma_ss(d_cols, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+          }
+        }
+        mma_commit(b_s_full(un % C::NBAR));
+      };
+      for (int u = 0; u < C::NBUF && u < steps && ok; ++u) {
+        ok = wait_keys(u);
         if (!ok) break;
         tc_fence_after();
+        if (elect_one()) fire_s(u);
+        __syncwarp();
+      }
+      for (int u = 0; u < steps && ok; ++u) {
+        const int slot = u % C::NV, un = u + C::NBUF;
+        ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(slot), (u / C::NV) & 1, abort_flag, prm.status));
+        if (ok && un < steps) ok = wait_keys(un);
         // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d
         const uint64_t vd = v_desc0 + ((slot * C::HALF_BYTES) >> 4);
-        const uint32_t p_cols = tmem_s + buf * kHalf;
+        const uint32_t p_cols = tmem_s + (u % C::NBUF) * kHalf;
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
+        if (!ok) break;
+        tc_fence_after();
         if (elect_one()) {
 #pragma unroll
           for (int ks = 0; ks < kHalf / 16; ++ks)
             mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
           mma_commit(b_pv_done(u % C::NBAR));
+          if (un < steps) fire_s(un);
         }
         __syncwarp();
-        if (u + C::NBUF < steps) ok = issue_s(u + C::NBUF);
       }
       if (elect_one()) mma_commit(b_o_done);
     }
@@ -320,7 +330,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       __syncwarp();
       if (lane == 0) mbar_arrive(b_q_tmem);
     }
-    float m_ref = -INFINITY, l_run = 0.f;
+    float m_ref = -INFINITY, l_run = 0.f, pend = 0.f;
     const float inv_scale_log2 = 1.0f / prm.scale_log2;
     const int ck_shift = __ffs(prm.c_k) - 1;
     bool ok = true;
@@ -386,31 +396,52 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         tmem_wait_st();
       }
-      // ---- pass 1: row maximum over the 64 columns
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      // ---- reference maximum.  The softmax needs no exact row maximum, only a reference m_ref
+      // that keeps exp2(x - m_ref) in range.  The first half-step of a row (and any later one while
+      // the row has seen only masked columns) measures the maximum of its scores first; afterwards
+      // the maximum of a half-step is gathered while its exponentials are computed, and a row
+      // whose values exceeded 2^threshold moves its reference up at the start of the NEXT
+      // half-step (`pend`).  Values between 2^threshold and 2^kDanger are exact all the same: P is
+      // bf16, which has the exponent range of fp32, and O and l are fp32.  A jump beyond 2^kDanger
+      // within one half-step may overflow: the CTA then marks its query tile in `redo`, and the
+      // launcher's second pass recomputes marked tiles with the fp32 kernel (exact row maxima).
+      float alpha = 1.f;
+      bool rescale;
+      if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll 1
-      for (int c4 = 0; c4 < 2; ++c4) {
-        uint32_t r[32];
-        tmem_ld32(t_s + c4 * 32, r);
-        tmem_wait_ld();
+        for (int c4 = 0; c4 < 2; ++c4) {
+          uint32_t r[32];
+          tmem_ld32(t_s + c4 * 32, r);
+          tmem_wait_ld();
 #pragma unroll
-        for (int j = 0; j < 32; j += 8) {
-          mx0 = max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          mx1 = max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-          mx2 = max3(mx2, __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-          mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+          for (int j = 0; j < 32; j += 8) {
+            mx0 = max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+            mx1 = max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+            mx2 = max3(mx2, __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+            mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+          }
         }
-      }
-      const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
-      // raise the reference maximum only when a half-step exceeds it by the threshold
-      const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
-      if (__any_sync(0xffffffffu, raise)) {
-        float alpha = 1.f;
+        const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
+        const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         if (raise) {
           alpha = (m_ref == -INFINITY) ? 0.f : ex2_approx(m_ref - tmax);
           m_ref = tmax;
+        } else if (pend > 0.f) {
+          alpha = ex2_approx(-pend);
+          m_ref += pend;
         }
-        if (!C::ROWSUM_MMA) l_run *= alpha;
+        rescale = __any_sync(0xffffffffu, raise || pend > 0.f);
+      } else {
+        if (pend > 0.f) {
+          alpha = ex2_approx(-pend);
+          m_ref += pend;
+        }
+        rescale = __any_sync(0xffffffffu, pend > 0.f);
+      }
+      pend = 0.f;
+      if (rescale) {
+        l_run *= alpha;
         if (u > 0) {
           // products complete in the order of their issue: once P V (u-1) is complete, all earlier are
           ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status));
@@ -425,49 +456,62 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             for (int j = 0; j < 32; ++j) o[j] = __float_as_uint(__uint_as_float(o[j]) * alpha);
             tmem_st32(tmem_o + lane_addr + c4 * 32, o);
           }
-          if (C::ROWSUM_MMA) {
-            const uint32_t l = tmem_ld1(tmem_o + lane_addr + D);
-            tmem_wait_ld();
-            tmem_st1(tmem_o + lane_addr + D, __float_as_uint(__uint_as_float(l) * alpha));
-          }
         }
       }
-      // ---- pass 2: P = exp2(x - m), packed to bf16 over the first 32 columns of the buffer (chunk 0
+      // ---- P = exp2(x - m_ref), packed to bf16 over the first 32 columns of the buffer (chunk 0
       // goes to columns [0,16) while chunk 1 is still unread in [32,64); chunk 1 to [16,32))
-      const float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      float ps0 = 0.f, ps1 = 0.f, ps2 = 0.f, ps3 = 0.f;
+      float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
+      const f32x2 sc2 = pack2(prm.scale_log2, prm.scale_log2);
+      float cm0 = -INFINITY, cm1 = -INFINITY;            // maximum of x - m_ref over the half-step
 #pragma unroll 1
       for (int c4 = 0; c4 < 2; ++c4) {
         uint32_t r[32];
         tmem_ld32(t_s + c4 * 32, r);
         tmem_wait_ld();
-        // The special-function unit takes one exponential per 8 cycles and sub-core: the other
-        // work of the chunk (scaling, sums, packing) is interleaved with the exponentials in groups
-        // of four, two groups behind, so that it issues in the shadow of that unit.
+        // The special-function unit takes one exponential per 8 cycles and sub-core and is the
+        // busiest unit of the kernel at d = 64: scaling and sums use two-value fp32 instructions,
+        // and the other work of the chunk is interleaved with the exponentials in groups of four,
+        // two groups behind, so that it issues in the shadow of that unit.
         float x[32];
         uint32_t pk[16];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
+        const f32x2 nm2 = pack2(neg_m, neg_m);
+        f32x2 s01 = pack2(0.f, 0.f), s23 = s01;
+        auto scale4 = [&](int j) {
+          unpack2(fma2(pack2(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), sc2, nm2), x[j], x[j + 1]);
+          unpack2(fma2(pack2(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), sc2, nm2), x[j + 2], x[j + 3]);
+        };
+        scale4(0);
+        scale4(4);
 #pragma unroll
         for (int g = 0; g < 10; ++g) {
           if (g < 8) {
+            const int j = 4 * g;
+            cm0 = max3(cm0, x[j], x[j + 1]);
+            cm1 = max3(cm1, x[j + 2], x[j + 3]);
 #pragma unroll
-            for (int j = 4 * g; j < 4 * g + 4; ++j) x[j] = ex2_approx(x[j]);
+            for (int e = j; e < j + 4; ++e) x[e] = ex2_approx(x[e]);
           }
-          if (g + 2 < 8) {
-#pragma unroll
-            for (int j = 4 * (g + 2); j < 4 * (g + 2) + 4; ++j) x[j] = fmaf(__uint_as_float(r[j]), prm.scale_log2, neg_m);
-          }
+          if (g + 2 < 8) scale4(4 * (g + 2));
           if (g >= 2) {
             const int j = 4 * (g - 2);
-            if (!C::ROWSUM_MMA) { ps0 += x[j]; ps1 += x[j + 1]; ps2 += x[j + 2]; ps3 += x[j + 3]; }
+            s01 = add2(s01, pack2(x[j], x[j + 1]));
+            s23 = add2(s23, pack2(x[j + 2], x[j + 3]));
             pk[j / 2] = pack_bf16x2(x[j], x[j + 1]);
             pk[j / 2 + 1] = pack_bf16x2(x[j + 2], x[j + 3]);
           }
         }
+        float sa, sb, sc, sd;
+        unpack2(s01, sa, sb);
+        unpack2(s23, sc, sd);
+        const float chunk_sum = (sa + sb) + (sc + sd);
+        l_run += chunk_sum;
         tmem_st16(t_s + c4 * 16, pk);
       }
-      if (!C::ROWSUM_MMA) l_run += (ps0 + ps1) + (ps2 + ps3);
+      {
+        const float hm = fmaxf(cm0, cm1);
+        if (hm > kRescaleThreshold) pend = ceilf(hm);
+        if (__any_sync(0xffffffffu, hm > kDanger)) *redo_flag = 1;
+      }
       // one arrival per warp: 128 arrivals on one barrier word would be serialised in shared memory
       tmem_wait_st();
       tc_fence_before();
@@ -482,10 +526,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int pos = qc * prm.c_q + half * kTile + row;
       const bool live = row < q_rows && pos < prm.n_q;  // rows of the padding are not written
       const int orig = live ? prm.perm_q[(size_t)p * prm.n_q + pos] : 0;
-      if (C::ROWSUM_MMA) {                               // the sums of the rounded probabilities
-        l_run = __uint_as_float(tmem_ld1(tmem_o + lane_addr + D));
-        tmem_wait_ld();
-      }
       const float inv = 1.f / l_run;
       __nv_bfloat16* out = prm.O + ((size_t)p * prm.n_q + orig) * D;
 #pragma unroll
@@ -513,6 +553,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   tc_fence_before();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem_base, C::TMEM_COLS);
+  // one word per CTA, written on every launch: 1 = this tile is to be recomputed
+  if (tid == 0) prm.redo[((size_t)p * prm.n_qc + qc) * 2 + half] = *redo_flag;
 }
 
 // ---------------------------------------------------------------------------
@@ -584,8 +626,10 @@ bool attn_tc_supported(const ca_problem_t& pr) {
 size_t attn_tc_workspace_bytes(const ca_problem_t& pr) {
   const size_t P = (size_t)pr.batch * pr.heads;
   const size_t cen_tiles = (size_t)ceil_div(ceil_div(pr.n_k, pr.cluster_k), kHalf);
+  const size_t n_qc = (size_t)ceil_div(pr.n_q, pr.cluster_q);
   return kStatusBytes + align_up(P * cen_tiles * kTile * pr.head_dim * sizeof(__nv_bfloat16), 256) +
-         align_up(P * cen_tiles * kHalf * pr.head_dim * sizeof(__nv_bfloat16), 256);
+         align_up(P * cen_tiles * kHalf * pr.head_dim * sizeof(__nv_bfloat16), 256) +
+         align_up(P * n_qc * 2 * sizeof(int32_t), 256);
 }
 
 template <int D>
@@ -610,6 +654,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   int* status = c.take<int>(kStatusBytes / sizeof(int));
   __nv_bfloat16* kmix = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kTile * D);
   __nv_bfloat16* vb = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kHalf * D);
+  int32_t* redo = c.take<int32_t>((size_t)P * n_qc * 2);
   if (pr.compensate) {
     centroid_prep_kernel<<<dim3(ceil_div(cen_tiles * kHalf * D, 256), P), 256, 0, st>>>(ck, cv, n_kc, cen_tiles, D,
                                                                                         kmix, vb);
@@ -626,14 +671,18 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   TcParams prm;
   prm.count_k = count_k; prm.block_idx = block_idx; prm.keep_count = keep_count; prm.perm_q = perm_q;
   prm.list_stride = list_stride;
-  prm.O = static_cast<__nv_bfloat16*>(O); prm.lse = lse; prm.status = status;
+  prm.O = static_cast<__nv_bfloat16*>(O); prm.lse = lse; prm.status = status; prm.redo = redo;
   prm.n_q = pr.n_q; prm.n_k = pr.n_k; prm.c_q = pr.cluster_q; prm.c_k = pr.cluster_k; prm.keep = pr.keep;
   prm.n_qc = n_qc; prm.n_kc = n_kc; prm.cen_tiles = cen_tiles; prm.compensate = pr.compensate;
   prm.bitmap_words = (cen_tiles * kHalf + 31) / 32;
   prm.scale_log2 = scale * 1.4426950408889634f;
   dim3 grid(n_qc * (pr.cluster_q >= kTile ? pr.cluster_q / kTile : 1), P);
-  if (D == 64) return launch_tc_d<64>(maps, prm, grid, st);
-  return launch_tc_d<128>(maps, prm, grid, st);
+  const int rc = D == 64 ? launch_tc_d<64>(maps, prm, grid, st) : launch_tc_d<128>(maps, prm, grid, st);
+  if (rc != CA_OK) return rc;
+  // second pass: query tiles whose scores left the range of the fast softmax (a climb of more than
+  // 2^96 within 64 keys) are recomputed by the fp32 kernel; its CTAs return at once for the others
+  return launch_attn_ref(pr, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O, lse,
+                         st, redo, (int)grid.x / n_qc);
 }
 
 }  // namespace ca

@@ -97,3 +97,54 @@ def test_argument_errors_enqueue_nothing():
     assert rc == binding.CA_ERR_INVALID_ARG                                  # recall must be positive
     torch.cuda.synchronize()
     assert binding.kernel_launches() == launches                            # nothing was enqueued
+
+
+def _bf16_round(a):
+    return torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(torch.bfloat16).float().numpy()
+
+
+@pytest.mark.parametrize("d,c_k,compensate", [(64, 128, False), (64, 32, True), (128, 128, True), (128, 32, False),
+                                              (64, 64, True)])
+def test_attention_scores_that_rise_along_the_list(d, c_k, compensate):
+    """Key blocks listed in an order in which the scores of a row climb by tens and by hundreds of
+    binary orders of magnitude from one block to the next, and fall by as much for other rows: the
+    running reference of the online softmax (Section 3.1: exact softmax over the kept blocks) has
+    to follow without overflow, whatever it was before.  With 32-row key clusters the climb happens
+    in the middle of a 64-column half-step."""
+    r = np.random.default_rng(31 + d + c_k)
+    H, n_q, c_q = 1, 300, 128
+    gains = np.array([0.0, 2.0, 4.0, 60.0, 62.0, 30.0, 600.0, 610.0, 100.0, 1200.0, 1.0, 3.0])
+    n_kc = len(gains)
+    n_k = n_kc * c_k - 5                                     # short last cluster
+    e = np.zeros(d); e[:4] = 0.5                             # unit direction
+    a = r.uniform(2.0, 5.0, n_q) * np.where(r.random(n_q) < 0.25, -1.0, 1.0)
+    Q = _bf16_round(a[:, None] * e[None] + 0.3 * r.standard_normal((n_q, d)))
+    K = _bf16_round(np.repeat(gains, c_k)[:n_k, None] * e[None] + 0.3 * r.standard_normal((n_k, d)))
+    V = _bf16_round(r.standard_normal((n_k, d)))
+    perm_q, perm_k = np.arange(n_q), np.arange(n_k)
+    n_qc = -(-n_q // c_q)
+    keep = 10
+    idx = np.stack([np.arange(keep), np.arange(keep), np.r_[np.arange(5, keep), np.arange(5)]])[:n_qc].astype(np.int32)
+    ck, count_k = orc.centroids(K, perm_k, c_k)
+    cv, _ = orc.centroids(V, perm_k, c_k)
+    ck32, cv32 = ck.astype(np.float32), cv.astype(np.float32)
+    o_ref, lse_ref = orc.cluster_attention(Q, K, V, perm_q, perm_k, c_q, c_k, idx, compensate,
+                                           ck=ck32, cv=cv32, count_k=count_k)
+    p = binding.make_problem(1, H, n_q, n_k, d, "bf16", c_q, c_k, keep, compensate)
+    plan = binding.Plan(p, DEV)
+
+    def pad(x, n, c):
+        out = np.zeros((-(-n // c) * c, x.shape[1]), np.float32)
+        out[:n] = x
+        return out
+    bf = torch.bfloat16
+    O, lse = plan.cluster_attention_fwd(dev(pad(Q, n_q, c_q)[None, None], bf), dev(pad(K, n_k, c_k)[None, None], bf),
+                                        dev(pad(V, n_k, c_k)[None, None], bf), dev(ck32[None, None]),
+                                        dev(cv32[None, None]), dev(count_k[None, None], torch.int32),
+                                        dev(idx[None, None], torch.int32), dev(perm_q[None, None], torch.int32))
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    O, lse = O[0, 0].float().cpu().numpy(), lse[0, 0].cpu().numpy()
+    assert np.isfinite(O).all() and np.isfinite(lse).all()
+    assert np.abs(O - o_ref).max() <= 2e-2 and np.linalg.norm(O - o_ref) <= 5e-3 * np.linalg.norm(o_ref)
+    assert np.abs(lse - lse_ref).max() <= 2e-2 + 1e-4 * np.abs(lse_ref).max()
