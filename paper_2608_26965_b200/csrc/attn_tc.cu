@@ -254,12 +254,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         }
         return got;
       };
-      auto fire_s = [&](int un) {                           // elected lane
-        const int parts = un >= 2 * sel_tiles ? 2 : 1;
-        const uint32_t d_cols = tmem_s + (un % C::NBUF) * kHalf;
+      // first key slot and number of parts of S(un); fire_s (elected lane) issues it
+      auto fire_s = [&](uint32_t d_cols, int kc0, int parts, uint32_t bar) {
         for (int g = 0; g < parts; ++g) {
-          const int slot = (kslot_of(un) + g) % C::NK;
-          const uint64_t kd = k_desc0 + ((slot * C::HALF_BYTES) >> 4);
+          const uint64_t kd = k_desc0 + ((((kc0 + g) % C::NK) * C::HALF_BYTES) >> 4);
 #pragma unroll
           for (int ks = 0; ks < D / 16; ++ks) {
             // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
@@ -268,13 +266,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             mma_ss(d_cols, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
           }
         }
-        mma_commit(b_s_full(un % C::NBAR));
+        mma_commit(bar);
       };
       for (int u = 0; u < C::NBUF && u < steps && ok; ++u) {
         ok = wait_keys(u);
         if (!ok) break;
         tc_fence_after();
-        if (elect_one()) fire_s(u);
+        if (elect_one())
+          fire_s(tmem_s + (u % C::NBUF) * kHalf, kslot_of(u), u >= 2 * sel_tiles ? 2 : 1, b_s_full(u % C::NBAR));
         __syncwarp();
       }
       for (int u = 0; u < steps && ok; ++u) {
@@ -284,6 +283,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d
         const uint64_t vd = v_desc0 + ((slot * C::HALF_BYTES) >> 4);
         const uint32_t p_cols = tmem_s + (u % C::NBUF) * kHalf;
+        const uint32_t s_cols = tmem_s + (un % C::NBUF) * kHalf, s_bar = b_s_full(un % C::NBAR), pv_bar = b_pv_done(u % C::NBAR);
+        const int s_kc0 = kslot_of(un), s_parts = un >= steps ? 0 : (un >= 2 * sel_tiles ? 2 : 1);
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
         if (!ok) break;
         tc_fence_after();
@@ -291,8 +292,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
 #pragma unroll
           for (int ks = 0; ks < kHalf / 16; ++ks)
             mma_ts(tmem_o, p_cols + ks * 8, vd + (uint64_t)(ks * (2048 >> 4)), idesc_pv, (u > 0 || ks > 0) ? 1u : 0u);
-          mma_commit(b_pv_done(u % C::NBAR));
-          if (un < steps) fire_s(un);
+          mma_commit(pv_bar);
+          if (s_parts) fire_s(s_cols, s_kc0, s_parts, s_bar);
         }
         __syncwarp();
       }
@@ -406,24 +407,28 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // within one half-step may overflow: the CTA then marks its query tile in `redo`, and the
       // launcher's second pass recomputes marked tiles with the fp32 kernel (exact row maxima).
       float alpha = 1.f;
-      bool rescale;
-      if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
-        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      bool rescale = false;
+      if (__any_sync(0xffffffffu, m_ref == -INFINITY || pend > 0.f)) {
+        bool raise = false;
+        float tmax = 0.f;
+        if (__any_sync(0xffffffffu, m_ref == -INFINITY)) {
+          float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
 #pragma unroll 1
-        for (int c4 = 0; c4 < 2; ++c4) {
-          uint32_t r[32];
-          tmem_ld32(t_s + c4 * 32, r);
-          tmem_wait_ld();
+          for (int c4 = 0; c4 < 2; ++c4) {
+            uint32_t r[32];
+            tmem_ld32(t_s + c4 * 32, r);
+            tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; j += 8) {
-            mx0 = max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-            mx1 = max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-            mx2 = max3(mx2, __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
-            mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+            for (int j = 0; j < 32; j += 8) {
+              mx0 = max3(mx0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+              mx1 = max3(mx1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+              mx2 = max3(mx2, __uint_as_float(r[j + 4]), __uint_as_float(r[j + 5]));
+              mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
+            }
           }
+          tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
+          raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         }
-        const float tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
-        const bool raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         if (raise) {
           alpha = (m_ref == -INFINITY) ? 0.f : ex2_approx(m_ref - tmax);
           m_ref = tmax;
@@ -432,12 +437,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           m_ref += pend;
         }
         rescale = __any_sync(0xffffffffu, raise || pend > 0.f);
-      } else {
-        if (pend > 0.f) {
-          alpha = ex2_approx(-pend);
-          m_ref += pend;
-        }
-        rescale = __any_sync(0xffffffffu, pend > 0.f);
       }
       pend = 0.f;
       if (rescale) {
