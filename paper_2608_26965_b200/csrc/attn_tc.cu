@@ -206,7 +206,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const bool centroid = i >= 2 * sel_tiles;
           const int parts = centroid ? 2 : 1;
           const int w = i - (centroid ? C::K_LEAD_CEN : C::K_LEAD);
-          if (w >= 0) ok = mbar_wait(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          if (w >= 0) ok = mbar_wait_relaxed(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
           for (int g = 0; g < parts && ok; ++g) {
             const int kc = kslot_of(i) + g, slot = kc % C::NK;
             mbar_expect_tx(b_k_full(slot), C::HALF_BYTES);
@@ -219,7 +219,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (j >= 0 && ok) {
           const int slot = j % C::NV;
           const int w = j - C::NV;
-          if (w >= 0) ok = mbar_wait(b_pv_done(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          if (w >= 0) ok = mbar_wait_relaxed(b_pv_done(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
           if (!ok) break;
           mbar_expect_tx(b_v_full(slot), C::HALF_BYTES);
           const uint32_t dst = s_v + slot * C::HALF_BYTES;
