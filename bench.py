@@ -395,6 +395,48 @@ def run_ours(args, w):
         replicas.shutdown()
         return
 
+    # ---- supplementary: the same steps (a) replayed from one CUDA graph, (b) with two steps in
+    # flight on two streams and two sets of buffers.  Neither is the headline; both say how much of a
+    # step is launch gaps and latency-bound clustering that another step could fill.
+    overlap = None
+    if not (args.no_e2e or adaptive or basic):
+        def timed_steps(fn, n):
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn(n)
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / n
+        overlap = {}
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(stream)
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                plan.forward(Q, K, V, stream=side)
+                side.synchronize()
+                with torch.cuda.graph(graph, stream=side):
+                    plan.forward(Q, K, V, stream=side)
+            overlap["cuda_graph_ms_per_step"] = timed_steps(lambda n: [graph.replay() for _ in range(n)], args.steps)
+            del graph
+        except Exception as exc:                               # noqa: BLE001
+            overlap["cuda_graph_ms_per_step"] = f"capture failed: {str(exc)[:120]}"
+        plans = [plan, binding.Plan(p, dev)]
+        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+
+        def two_in_flight(n):
+            for st_ in streams:
+                st_.wait_stream(torch.cuda.current_stream())
+            for i in range(n):
+                plans[i & 1].forward(Q, K, V, stream=streams[i & 1])
+            for st_ in streams:
+                torch.cuda.current_stream().wait_stream(st_)
+        two_in_flight(4)
+        overlap["two_steps_in_flight_ms_per_step"] = timed_steps(two_in_flight, args.steps)
+        assert all(v == 0 for pl in plans for v in pl.last_status().values())
+        del plans[1]
+
     peaks, peak_kind = load_peaks()
     attn_ms = stage_ms["cluster_attention_fwd"]
     attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
@@ -418,6 +460,7 @@ def run_ours(args, w):
                    "l2": "inputs larger than L2 (no flush)"},
         "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),
         "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "dense": dense,
+        "overlap": overlap,
     }
     if not args.no_cpu_baseline:
         # the oracle as it stands on whole heads until about 10 s of CPU work are spent
