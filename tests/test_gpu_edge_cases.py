@@ -103,16 +103,18 @@ def _bf16_round(a):
     return torch.from_numpy(np.ascontiguousarray(a, np.float32)).to(torch.bfloat16).float().numpy()
 
 
-@pytest.mark.parametrize("d,c_k,compensate", [(64, 128, False), (64, 32, True), (128, 128, True), (128, 32, False),
-                                              (64, 64, True)])
-def test_attention_scores_that_rise_along_the_list(d, c_k, compensate):
+@pytest.mark.parametrize("d,c_q,c_k,compensate", [(64, 128, 128, False), (64, 128, 32, True), (128, 128, 128, True),
+                                                  (128, 128, 32, False), (64, 128, 64, True),
+                                                  (64, 256, 128, True),      # two CTAs per query cluster
+                                                  (128, 64, 128, False)])    # half-filled query tile
+def test_attention_scores_that_rise_along_the_list(d, c_q, c_k, compensate):
     """Key blocks listed in an order in which the scores of a row climb by tens and by hundreds of
     binary orders of magnitude from one block to the next, and fall by as much for other rows: the
     running reference of the online softmax (Section 3.1: exact softmax over the kept blocks) has
     to follow without overflow, whatever it was before.  With 32-row key clusters the climb happens
     in the middle of a 64-column half-step."""
     r = np.random.default_rng(31 + d + c_k)
-    H, n_q, c_q = 1, 300, 128
+    H, n_q = 1, 300 if c_q < 256 else 700
     gains = np.array([0.0, 2.0, 4.0, 60.0, 62.0, 30.0, 600.0, 610.0, 100.0, 1200.0, 1.0, 3.0])
     n_kc = len(gains)
     n_k = n_kc * c_k - 5                                     # short last cluster
@@ -124,7 +126,8 @@ def test_attention_scores_that_rise_along_the_list(d, c_k, compensate):
     perm_q, perm_k = np.arange(n_q), np.arange(n_k)
     n_qc = -(-n_q // c_q)
     keep = 10
-    idx = np.stack([np.arange(keep), np.arange(keep), np.r_[np.arange(5, keep), np.arange(5)]])[:n_qc].astype(np.int32)
+    lists = [np.arange(keep), np.arange(keep), np.r_[np.arange(5, keep), np.arange(5)]]
+    idx = np.stack([lists[i % 3] for i in range(n_qc)]).astype(np.int32)
     ck, count_k = orc.centroids(K, perm_k, c_k)
     cv, _ = orc.centroids(V, perm_k, c_k)
     ck32, cv32 = ck.astype(np.float32), cv.astype(np.float32)
