@@ -35,12 +35,21 @@ struct ClusterWs {
   float* partial;
   double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
   float *roots32, *basis32, *WK32, *biasK, *biasQ;
-  float *Qprime, *Yq, *Yk;
+  float *Qprime, *Yq, *Yk, *Ytq, *Ytk;
   __nv_bfloat16 *wt_hi, *wt_lo, *wt2_hi, *wt2_lo;
   int32_t *perm_q_tmp, *perm_k_tmp;
   uint32_t *keybuf_q, *keybuf_k;
   size_t bytes;
 };
+
+// A level of the splitter reads one coordinate of every row of a set, rows scattered: from the
+// row-major coordinates that costs a 128-byte DRAM line per row and level.  A coordinate-major copy
+// makes it a 4-byte read inside an L2-resident column, at the price of writing the coordinates a
+// second time (4 d bytes per row): worth it when levels x 128 > 1.5 x 4 d (long sequences, d = 64).
+static bool use_yt(const ca_problem_t* p, int n, int c) {
+  const bool tc = p->dtype == CA_DTYPE_BF16 && (p->head_dim == 64 || p->head_dim == 128);
+  return tc && !(p->flags & CA_Y_IN) && split_top_levels_for(n, c) * 128 >= 6 * p->head_dim;
+}
 
 ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool need_yk) {
   ClusterWs w{};
@@ -75,6 +84,9 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
     w.wt2_lo = c.take<__nv_bfloat16>(P * DD);
     if (need_yq) w.Yq = c.take<float>(P * (size_t)p->n_q * D);
     if (need_yk) w.Yk = c.take<float>(P * (size_t)p->n_k * D);
+    // coordinate-major copies of the split coordinates, where they pay (use_yt)
+    if (use_yt(p, p->n_q, p->cluster_q)) w.Ytq = c.take<float>(P * (size_t)p->n_q * D);
+    if (use_yt(p, p->n_k, p->cluster_k)) w.Ytk = c.take<float>(P * (size_t)p->n_k * D);
   }
   w.perm_q_tmp = c.take<int32_t>(P * (size_t)p->n_q);
   w.perm_k_tmp = c.take<int32_t>(P * (size_t)p->n_k);
@@ -203,12 +215,12 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, sq));
     if (tc) {
       CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
-                                 w.wt2_lo, w.status, sq));
+                                 w.wt2_lo, w.status, sq, w.Ytq));
     } else {
       CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
     }
     CA_TRY(launch_split(yq_out, nullptr, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
-                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 1, sq));
+                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 1, sq, w.Ytq, nullptr));
     CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, sq));
     CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
     // ---- key side on the caller's stream: covariance of the transformed keys K F_q
@@ -220,12 +232,12 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st));
     if (tc) {
       CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
-                                 w.wt_lo, w.status, st));
+                                 w.wt_lo, w.status, st, w.Ytk));
     } else {
       CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
     }
     CA_TRY(launch_split(nullptr, yk_out, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
-                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 2, st));
+                        perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 2, st, nullptr, w.Ytk));
     CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
     CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
     // ---- join

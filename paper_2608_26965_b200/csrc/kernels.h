@@ -21,7 +21,7 @@ int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows,
                    double* gram, double* colsum, int* status, cudaStream_t st);
 int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, const float* W,
                         const float* bias, int normalize, float* out, void* out_hi, void* out_lo,
-                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st);
+                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t = nullptr);
 
 // eigh.cu
 int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
@@ -37,9 +37,12 @@ int launch_bias(const double* sum, const float* W, int P, int D, int n, float* b
 
 // split.cu
 int split_levels_for(int n, int c);
+// levels that run as per-level launches over whole sets (the rest is finished per subtree)
+int split_top_levels_for(int n, int c);
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
-                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st);
+                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st,
+                 const float* Ytq = nullptr, const float* Ytk = nullptr);
 
 // permute.cu
 int launch_split_basic(const void* Q, const void* K, int dtype, const float* A_q, const float* A_k,

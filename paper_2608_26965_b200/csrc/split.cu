@@ -110,6 +110,7 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 
 struct SplitSide {
   const float* Y;          // [P][n][D]
+  const float* Yt;         // [P][D][n] the same coordinates, coordinate-major, or null
   const int32_t* perm_in;  // [P][n] or null (identity)
   int32_t* perm_out;       // [P][n]
   uint32_t* keybuf;        // [P][n] staging for sets larger than the shared-memory windows
@@ -151,6 +152,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   if (!seg.active) return;
   const int tid = threadIdx.x, nt = blockDim.x, lane = tid & 31, warp = tid >> 5;
   const float* Y = sd.Y + (size_t)p * sd.n * D;
+  const float* Yt = sd.Yt ? sd.Yt + (size_t)p * sd.n * D : nullptr;
   const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
   int32_t* pout = sd.perm_out + (size_t)p * sd.n;
   const int lo = seg.lo, s = seg.size;
@@ -224,7 +226,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
       row[u] = (i < cs) ? (pin ? __ldg(pin + lo + c0 + i) : lo + c0 + i) : 0;
     }
 #pragma unroll
-    for (int u = 0; u < 8; ++u) val[u] = __ldg(Y + (size_t)row[u] * D + coord);
+    for (int u = 0; u < 8; ++u) val[u] = Yt ? __ldg(Yt + (size_t)coord * sd.n + row[u]) : __ldg(Y + (size_t)row[u] * D + coord);
 #pragma unroll
     for (int u = 0; u < 8; ++u) {
       const int i = i0 + u * nt;
@@ -389,6 +391,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
   constexpr int nt = kSplitThreads;
   const int c = sd.c;
   const float* Y = sd.Y + (size_t)p * sd.n * D;
+  const float* Yt = sd.Yt ? sd.Yt + (size_t)p * sd.n * D : nullptr;
   const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
   int32_t* pout = sd.perm_out + (size_t)p * sd.n;
   const int lo = root.lo, s0 = root.size;
@@ -469,7 +472,8 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
         int hi = nseg;                                // slo[g] <= i < slo[g+1]
         while (hi - g > 1) { const int mid = (g + hi) >> 1; if (slo[mid] <= i) g = mid; else hi = mid; }
         const bool splits = slo[g + 1] - slo[g] > c;
-        if (splits) sm.keys[i] = order_key(__ldg(Y + (size_t)rows[i] * D + sm.seg_coord[g]));
+        if (splits) sm.keys[i] = order_key(Yt ? __ldg(Yt + (size_t)sm.seg_coord[g] * sd.n + rows[i])
+                                              : __ldg(Y + (size_t)rows[i] * D + sm.seg_coord[g]));
         else g = -1 - g;                              // final subset: carried over unchanged
       } else {
         g = INT_MIN;
@@ -626,9 +630,12 @@ static int tail_level_for(int n, int c) {
   return level;
 }
 
+int split_top_levels_for(int n, int c) { return tail_level_for(n, c); }
+
 int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q, int n_k, int c_q,
                  int c_k, int32_t* perm_q_out, int32_t* perm_q_tmp, int32_t* perm_k_out,
-                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st) {
+                 int32_t* perm_k_tmp, uint32_t* keybuf_q, uint32_t* keybuf_k, int sides, cudaStream_t st,
+                 const float* Ytq, const float* Ytk) {
   // sides: bit 0 = queries, bit 1 = keys
   auto level_kernel = D == 64 ? split_level_kernel<64> : split_level_kernel<128>;
   auto tail_kernel = D == 64 ? split_tail_kernel<64> : split_tail_kernel<128>;
@@ -650,6 +657,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
       int32_t* tmp = w == 0 ? perm_q_tmp : perm_k_tmp;
       const int tail = w == 0 ? tail_q : tail_k;
       sd.Y = w == 0 ? Yq : Yk;
+      sd.Yt = w == 0 ? Ytq : Ytk;
       sd.keybuf = w == 0 ? keybuf_q : keybuf_k;
       sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
       sd.levels = split_levels_for(sd.n, sd.c);
@@ -888,6 +896,7 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
       const bool to_tmp = ((run - 1 - level) % 2) != 0;
       SplitSide& sd = prm.side[w];
       sd.Y = nullptr;
+      sd.Yt = nullptr;
       sd.keybuf = w == 0 ? keybuf_q : keybuf_k;
       sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
       sd.levels = w == 0 ? lev_q : lev_k;

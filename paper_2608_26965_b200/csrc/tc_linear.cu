@@ -186,6 +186,7 @@ struct LinCfg {
 
 struct LinParams {
   const float* bias;      // [P][D] or null
+  float* out_t;           // [P][D][n_rows] or null: the fp32 result once more, coordinate-major
   int* status;
   int n_rows, tiles_per_cta, has_lo, stages, normalize, out_split;
 };
@@ -317,6 +318,18 @@ transform_tc_kernel(const __grid_constant__ CUtensorMap tm_xhi, const __grid_con
         const float inv = nrm >= 1e-30f ? 1.f / nrm : 0.f;
 #pragma unroll
         for (int j = 0; j < D; ++j) v[j] *= inv;
+      }
+      if (prm.out_t) {
+        // coordinate-major copy: for one coordinate the 128 threads of the tile write 512
+        // consecutive bytes.  The splitter gathers one coordinate of scattered rows per level; from
+        // this layout that is a 4-byte read inside an L2-resident column instead of one DRAM line
+        // per row of the row-major result.
+        const int grow = (t_begin + t) * kRows + row;
+        if (grow < prm.n_rows) {
+          float* dst = prm.out_t + (size_t)p * D * prm.n_rows + grow;
+#pragma unroll
+          for (int j = 0; j < D; ++j) dst[(size_t)j * prm.n_rows] = v[j];
+        }
       }
       // the previous tile's stores must have finished reading the staging buffer
       if (st == 0) tma_store_wait_read();
@@ -467,12 +480,12 @@ int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows,
 
 int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, const float* W,
                         const float* bias, int normalize, float* out, void* out_hi, void* out_lo,
-                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st) {
+                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t) {
   weight_prep_kernel<<<dim3(ceil_div(D * D, 256), problems), 256, 0, st>>>(
       W, D, static_cast<__nv_bfloat16*>(wt_hi), static_cast<__nv_bfloat16*>(wt_lo));
   CA_LAUNCH_CHECK();
   LinParams prm;
-  prm.bias = bias; prm.status = status; prm.n_rows = n_rows; prm.has_lo = X_lo ? 1 : 0;
+  prm.bias = bias; prm.out_t = out ? out_t : nullptr; prm.status = status; prm.n_rows = n_rows; prm.has_lo = X_lo ? 1 : 0;
   prm.normalize = normalize; prm.out_split = out ? 0 : 1;
   const int tile = kRows * D * 2 * (X_lo ? 2 : 1);
   const int fixed = 2 * D * D * 2 + kRows * D * 4 + 4096;
