@@ -92,10 +92,11 @@ int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select
  *   count_q,count_k [B,H,n_c]  member counts |c|.
  *   Yq [B,H,n_q,d], Yk [B,H,n_k,d] fp32 split coordinates: input when
  *        p->flags has CA_Y_IN, otherwise output (may be NULL: kept in ws).
- * Once the two factors exist the query side and the key side are independent:
- * the query side is enqueued on a second stream of the library (one per device,
- * created together with two events at the first call on that device) that forks
- * from `stream` and joins it again before the call returns.  Nothing waits on the
+ * The chain from Q to the key side (metric, its factor, key projection, key split)
+ * and the chain from K to the query side need each other only through C_K: the
+ * second one is enqueued on a second stream of the library (one per device,
+ * created together with three events at the first call on that device) that forks
+ * from `stream` at the start of the call and joins it again before the call returns.  Nothing waits on the
  * host; a capture of `stream` records the side stream as a parallel branch (make
  * the first call on a device before capturing).
  */

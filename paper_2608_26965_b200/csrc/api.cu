@@ -32,7 +32,7 @@ int check_problem(const ca_problem_t* p) {
 
 struct ClusterWs {
   int* status;
-  float* partial;
+  float *partial, *partial2;           // chunk sums of the Gram kernels, one buffer per stream
   double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
   float *roots32, *basis32, *WK32, *biasK, *biasQ;
   float *Qprime, *Yq, *Yk, *Ytq, *Ytk;
@@ -63,6 +63,7 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
     moments_chunking(p->n_k, (int)P, &cr, &nck);
     const size_t nchunks = (size_t)(ncq > nck ? ncq : nck);
     w.partial = c.take<float>(P * nchunks * (DD + D));
+    w.partial2 = c.take<float>(P * nchunks * (DD + D));
     w.gramQ = c.take<double>(P * DD);  w.sumQ = c.take<double>(P * D);
     w.gramK = c.take<double>(P * DD);  w.sumK = c.take<double>(P * D);
     w.metric = c.take<double>(2 * P * DD);
@@ -103,7 +104,7 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
 // device, created at the first call on that device.
 struct SideStream {
   cudaStream_t stream = nullptr;
-  cudaEvent_t fork = nullptr, join = nullptr;
+  cudaEvent_t fork = nullptr, mid = nullptr, join = nullptr;
   bool ready = false;
 };
 SideStream* side_stream() {
@@ -114,6 +115,7 @@ SideStream* side_stream() {
   if (!s.ready) {
     if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    if (cudaEventCreateWithFlags(&s.mid, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
     s.ready = true;
   }
@@ -171,44 +173,49 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     const bool tc = p->dtype == CA_DTYPE_BF16;
     __nv_bfloat16* qp_hi = reinterpret_cast<__nv_bfloat16*>(w.Qprime);          // r(q) as bf16 hi + lo parts
     __nv_bfloat16* qp_lo = qp_hi + (size_t)P * p->n_q * D;
-    // metric matrices (Section 3.2.2)
-    if (tc) {
-      CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
-      CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial, w.gramK, w.sumK, w.status, st));
-    } else {
-      CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
-      CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial, w.gramK, w.sumK, st));
-    }
+    // metric matrices (Section 3.2.2) and their factors F_q F_q^T = M, F_k F_k^T = C_K (they stand
+    // in for the symmetric roots: any factor yields the same principal-component coordinates).  The
+    // un-normalised query representation (Appendix B.1) takes the root of K_c^T K_c / n_k, the
+    // normalised one is indifferent to the factor and keeps the scatter matrix as it is.
+    // M and F_q come from Q on the caller's stream and lead into the key side; C_K and F_k come from
+    // K on the side stream and lead into the query side: the fork is at the very start, and the
+    // key side only waits for C_K (event `mid`).
     double* M = w.metric;
     double* CK = w.metric + (size_t)P * DD;
-    // the un-normalised query representation (Appendix B.1) takes the root of K_c^T K_c / n_k,
-    // the normalised one is indifferent to the factor and keeps the scatter matrix as it is
     const bool unnormalized = (p->flags & CA_QUERY_UNNORMALIZED) != 0;
     const double ck_scale = unnormalized ? 1.0 / (double)p->n_k : 1.0;
-    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, M, CK, st));
-    // factors F_q F_q^T = M and F_k F_k^T = C_K (they stand in for the symmetric roots:
-    // any factor yields the same principal-component coordinates)
-    CA_TRY(launch_cholesky_factor(w.metric, 2 * P, D, w.roots, w.roots32, st));
     double* Rq = w.roots;
     const float* Rk32 = w.roots32 + (size_t)P * DD;
     double* covK = w.cov;
     double* covQ = w.cov + (size_t)P * DD;
-    // ---- fork: the query side continues on the side stream
     SideStream* side = side_stream();
     if (!side) return CA_ERR_CUDA;
     cudaStream_t sq = side->stream;
     CA_RETURN_IF_CUDA(cudaEventRecord(side->fork, st));
     CA_RETURN_IF_CUDA(cudaStreamWaitEvent(sq, side->fork, 0));
+    if (tc) {
+      CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
+      CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial2, w.gramK, w.sumK, w.status, sq));
+    } else {
+      CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
+      CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial2, w.gramK, w.sumK, sq));
+    }
+    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, M, nullptr, st));
+    CA_TRY(launch_cholesky_factor(M, P, D, w.roots, w.roots32, st));
+    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, nullptr, CK, sq));
+    CA_RETURN_IF_CUDA(cudaEventRecord(side->mid, sq));
+    CA_TRY(launch_cholesky_factor(CK, P, D, w.roots + (size_t)P * DD, w.roots32 + (size_t)P * DD, sq));
+    // ---- query side (side stream)
     // query representation r(q) = F_k^T q / |F_k^T q|, its covariance, its principal components,
     // the coordinates Y = (r(q) - mean) E_Q
     const float* EQ32 = w.basis32 + (size_t)P * DD;
     if (tc) {
       CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
                                  w.wt2_hi, w.wt2_lo, w.status, sq));
-      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, w.status, sq));
+      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, w.status, sq));
     } else {
       CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
-      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial, w.gramQp, w.sumQp, sq));
+      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, sq));
     }
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, sq));
     CA_TRY(launch_eigh(covQ, P, D, w.basis + (size_t)P * DD, w.basis32 + (size_t)P * DD, nullptr, sq));
@@ -225,6 +232,7 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
     // ---- key side on the caller's stream: covariance of the transformed keys K F_q
     // (F_q^T C_K F_q / n_k, d x d algebra), its principal components, Y = (K - kbar) F_q E_K
+    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->mid, 0));
     CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
     CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, unnormalized ? 1.0 : 1.0 / (double)p->n_k, 0, covK, nullptr, st));
     CA_TRY(launch_eigh(covK, P, D, w.basis, w.basis32, nullptr, st));

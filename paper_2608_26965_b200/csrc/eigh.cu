@@ -85,13 +85,14 @@ int launch_cholesky_factor(const double* A, int count, int D, double* out64, flo
 __global__ void metric_kernel(const double* __restrict__ gramQ, const double* __restrict__ gramK,
                               const double* __restrict__ sumK, int D, double n_q, double n_k,
                               double ck_scale, double* __restrict__ M, double* __restrict__ CK) {
+  // either output may be left out (null): the two come from different streams in cluster_qk
   const int p = blockIdx.y;
   const int e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= D * D) return;
   const int i = e / D, j = e % D;
   const size_t o = (size_t)p * D * D + e;
-  M[o] = gramQ[o] / n_q;
-  CK[o] = (gramK[o] - sumK[(size_t)p * D + i] * sumK[(size_t)p * D + j] / n_k) * ck_scale;
+  if (M) M[o] = gramQ[o] / n_q;
+  if (CK) CK[o] = (gramK[o] - sumK[(size_t)p * D + i] * sumK[(size_t)p * D + j] / n_k) * ck_scale;
 }
 
 // Cov = gram / n - mean mean^T, mean = sum / n
