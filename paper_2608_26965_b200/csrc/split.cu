@@ -682,7 +682,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
     if (level < top_q) max_seg = max_segment_at_level(n_q, c_q, level);
     if (level < top_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
     int csize = 1;
-    while (csize < kMaxCluster && max_seg > csize * 8192) csize *= 2;
+    while (csize < kMaxCluster && max_seg > csize * 16384) csize *= 2;
     const int per_cta = (max_seg + csize - 1) / csize;
     prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
     cudaLaunchConfig_t cfg = {};
@@ -933,7 +933,7 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
     if (level < run_q) max_seg = max_segment_at_level(n_q, c_q, level);
     if (level < run_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
     int csize = 1;
-    while (csize < kMaxCluster && max_seg > csize * 8192) csize *= 2;
+    while (csize < kMaxCluster && max_seg > csize * 16384) csize *= 2;
     const int per_cta = (max_seg + csize - 1) / csize;
     prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
     cudaLaunchConfig_t cfg = {};
