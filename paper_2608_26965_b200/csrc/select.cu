@@ -30,9 +30,9 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* keys = reinterpret_cast<uint32_t*>(smem_raw);                       // [QT][n_kc]
   float* qs = reinterpret_cast<float*>(keys + (size_t)QT * n_kc);        // [QT][D]
-  __shared__ int s_hist[256];
-  __shared__ int s_warp[64];
-  __shared__ int s_scalar[4];
+  __shared__ int s_hist[QT][256];
+  __shared__ int s_warp[QT][64];
+  __shared__ int s_scalar[QT][4];
   const int p = blockIdx.y;
   const int q0 = row0 + blockIdx.x * QT;
   const int nq = min(QT, min(n_qc, row0 + chunk_rows) - q0);
@@ -71,94 +71,121 @@ score_select_kernel(const float* __restrict__ cq, const float* __restrict__ ck, 
   }
   __syncthreads();
 
-  for (int t = 0; t < nq; ++t) {
-    const uint32_t* kt = keys + (size_t)t * n_kc;
-    // radix selection of the keep-th largest key
-    uint32_t prefix = 0, mask = 0;
-    int remaining = keep;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      s_hist[tid] = 0;                             // kSelectThreads == 256 bins
-      __syncthreads();
-      for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
-        const int j = j0 + tid;
-        const bool ok = j < n_kc;
-        const uint32_t k = ok ? kt[j] : 0u;
-        const bool cand = ok && ((k & mask) == prefix);
+  // ---- radix selection of the keep-th largest key, the QT rows side by side (one set of barriers
+  // for all of them: a row on its own is bound by the barriers of its passes, not by work)
+  uint32_t prefix[QT], mask = 0;
+  int remaining[QT];
+#pragma unroll
+  for (int t = 0; t < QT; ++t) { prefix[t] = 0; remaining[t] = keep; }
+  for (int shift = 24; shift >= 0; shift -= 8) {
+#pragma unroll
+    for (int t = 0; t < QT; ++t) s_hist[t][tid] = 0;                 // kSelectThreads == 256 bins
+    __syncthreads();
+    for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
+      const int j = j0 + tid;
+      const bool ok = j < n_kc;
+#pragma unroll
+      for (int t = 0; t < QT; ++t) {
+        if (t >= nq) break;
+        const uint32_t k = ok ? keys[(size_t)t * n_kc + j] : 0u;
+        const bool cand = ok && ((k & mask) == prefix[t]);
         const int bin = cand ? (int)((k >> shift) & 255u) : -1;
         if (shift == 24) {
           // leading digit (sign and exponent bits): few distinct values in a warp, one atomic per value
           const unsigned peers = __match_any_sync(0xffffffffu, bin);
-          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[t][bin], __popc(peers));
         } else if (cand) {
-          atomicAdd(&s_hist[bin], 1);                // lower digits are spread out: plain atomics
+          atomicAdd(&s_hist[t][bin], 1);               // lower digits are spread out: plain atomics
         }
       }
-      __syncthreads();
-      if (warp == 0) {
-        // bins from the top: lane 0 owns bins 255..248
-        int local[8]; int sum = 0;
-#pragma unroll
-        for (int b = 0; b < 8; ++b) { local[b] = s_hist[255 - (lane * 8 + b)]; sum += local[b]; }
-        int incl = sum;
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += v;
-        }
-        int before = incl - sum;
-#pragma unroll
-        for (int b = 0; b < 8; ++b) {
-          if (before < remaining && remaining <= before + local[b]) {
-            s_scalar[0] = 255 - (lane * 8 + b);
-            s_scalar[1] = remaining - before;
-          }
-          before += local[b];
-        }
-      }
-      __syncthreads();
-      prefix |= (uint32_t)s_scalar[0] << shift;
-      mask |= 255u << shift;
-      remaining = s_scalar[1];
-      __syncthreads();
     }
-    const uint32_t thr = prefix;
-    const int eq_take = remaining;         // threshold-valued clusters taken, lowest indices first
-
-    int32_t* out = block_idx + ((size_t)p * n_qc + q0 + t) * keep;
-    int gt_before = 0, eq_before = 0;
-    for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
-      const int j = j0 + tid;
-      const bool ok = j < n_kc;
-      const uint32_t k = ok ? kt[j] : 0u;
-      const int is_gt = (ok && k > thr) ? 1 : 0;
-      const int is_eq = (ok && k == thr) ? 1 : 0;
-      const int packed = is_gt | (is_eq << 16);
-      int incl = packed;
+    __syncthreads();
+    if (warp < nq) {
+      // warp t scans row t's bins from the top: lane 0 owns bins 255..248
+      int local[8]; int sum = 0;
+#pragma unroll
+      for (int b = 0; b < 8; ++b) { local[b] = s_hist[warp][255 - (lane * 8 + b)]; sum += local[b]; }
+      int incl = sum;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
       }
-      if (lane == 31) s_warp[warp] = incl;
-      __syncthreads();
-      if (warp == 0) {
-        const int w = (lane < kSelectThreads / 32) ? s_warp[lane] : 0;
-        int wi = w;
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(0xffffffffu, wi, o);
-          if (lane >= o) wi += v;
+      int before = incl - sum;
+      int rem = 0;
+#pragma unroll
+      for (int t = 0; t < QT; ++t) if (t == warp) rem = remaining[t];
+#pragma unroll
+      for (int b = 0; b < 8; ++b) {
+        if (before < rem && rem <= before + local[b]) {
+          s_scalar[warp][0] = 255 - (lane * 8 + b);
+          s_scalar[warp][1] = rem - before;
         }
-        s_warp[32 + lane] = wi - w;
-        if (lane == 31) s_scalar[2] = wi;
+        before += local[b];
       }
-      __syncthreads();
-      const int excl = incl - packed + s_warp[32 + warp];
-      const int gt_here = gt_before + (excl & 0xffff);
-      const int eq_here = eq_before + (excl >> 16);
-      if (ok && (is_gt || (is_eq && eq_here < eq_take))) out[gt_here + min(eq_here, eq_take)] = j;
-      const int total = s_scalar[2];
-      gt_before += total & 0xffff;
-      eq_before += total >> 16;
-      __syncthreads();
     }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < QT; ++t) {
+      if (t < nq) {
+        prefix[t] |= (uint32_t)s_scalar[t][0] << shift;
+        remaining[t] = s_scalar[t][1];
+      }
+    }
+    mask |= 255u << shift;
+    // the next pass's first barrier (after the bins are cleared) orders these reads before the
+    // next writes of s_scalar
+  }
+
+  // ---- output, ascending index: keys above the threshold, then threshold-valued ones, lowest
+  // indices first, until the list is full; again all rows per barrier
+  int gt_before[QT], eq_before[QT];
+#pragma unroll
+  for (int t = 0; t < QT; ++t) { gt_before[t] = 0; eq_before[t] = 0; }
+  for (int j0 = 0; j0 < n_kc; j0 += kSelectThreads) {
+    const int j = j0 + tid;
+    const bool ok = j < n_kc;
+    int packed[QT], incl[QT];
+#pragma unroll
+    for (int t = 0; t < QT; ++t) {
+      const uint32_t k = (ok && t < nq) ? keys[(size_t)t * n_kc + j] : 0u;
+      const int is_gt = (ok && t < nq && k > prefix[t]) ? 1 : 0;
+      const int is_eq = (ok && t < nq && k == prefix[t]) ? 1 : 0;
+      packed[t] = is_gt | (is_eq << 16);
+      int v = packed[t];
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, v, o);
+        if (lane >= o) v += u;
+      }
+      incl[t] = v;
+      if (lane == 31) s_warp[t][warp] = v;
+    }
+    __syncthreads();
+    if (warp < QT) {
+      const int w = (lane < kSelectThreads / 32) ? s_warp[warp][lane] : 0;
+      int wi = w;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += v;
+      }
+      s_warp[warp][32 + lane] = wi - w;
+      if (lane == 31) s_scalar[warp][2] = wi;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int t = 0; t < QT; ++t) {
+      if (t >= nq) break;
+      const int excl = incl[t] - packed[t] + s_warp[t][32 + warp];
+      const int gt_here = gt_before[t] + (excl & 0xffff);
+      const int eq_here = eq_before[t] + (excl >> 16);
+      const int eq_take = remaining[t];    // threshold-valued clusters taken, lowest indices first
+      const bool is_gt = (packed[t] & 1) != 0, is_eq = (packed[t] >> 16) != 0;
+      int32_t* out = block_idx + ((size_t)p * n_qc + q0 + t) * keep;
+      if (is_gt || (is_eq && eq_here < eq_take)) out[gt_here + min(eq_here, eq_take)] = j;
+      const int total = s_scalar[t][2];
+      gt_before[t] += total & 0xffff;
+      eq_before[t] += total >> 16;
+    }
+    __syncthreads();
   }
 }
 
