@@ -290,6 +290,7 @@ def run_ours(args, w):
     barrier()
     clocks = sampler.stop() if sampler else None
     launches = binding.kernel_launches() - launches0
+    recomputed = plan.recomputed_clusters()           # 0: no query cluster left the tensor-core kernel
     total_ms = max_over_ranks(t_start.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     stage_ms = {
@@ -459,7 +460,8 @@ def run_ours(args, w):
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "inputs larger than L2 (no flush)"},
         "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),
-        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "dense": dense,
+        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "recomputed_clusters": int(recomputed),
+        "clocks": clocks, "dense": dense,
         "overlap": overlap,
     }
     if not args.no_cpu_baseline:

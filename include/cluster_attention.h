@@ -244,6 +244,14 @@ int ca_static_last_status(void);
 /* Reads the status word of a workspace (synchronises the device). */
 int ca_last_status(const void* ws);
 
+/* Statistics of an attention workspace (synchronises the device): how many query clusters the
+ * second pass of cluster_attention_fwd has recomputed with the fp32 kernel since the workspace
+ * was zero-filled.  The tensor-core kernel keeps the reference of its online softmax (Section
+ * 3.1: exact softmax over the kept blocks) one half-step behind; a query cluster whose scores
+ * climb by more than 2^96 within 64 keys leaves its range and is recomputed.  Returns the count
+ * (>= 0), or minus an error code. */
+int ca_attn_recomputed(const void* ws);
+
 /* Library version and the compute capability the kernels were built for. */
 const char* ca_version(void);
 

@@ -26,7 +26,7 @@ CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
 CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN = 1, 2, 4, 8
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
-           "ca_last_status", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
+           "ca_last_status", "ca_attn_recomputed", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
            "ca_static_scratch_bytes", "ca_static_last_status")
 
 
@@ -89,6 +89,8 @@ def load_library() -> ctypes.CDLL:
     lib.cluster_qk_basic.restype = ctypes.c_int
     lib.ca_last_status.argtypes = [vp]
     lib.ca_last_status.restype = ctypes.c_int
+    lib.ca_attn_recomputed.argtypes = [vp]
+    lib.ca_attn_recomputed.restype = ctypes.c_int
     lib.ca_version.argtypes = []
     lib.ca_version.restype = ctypes.c_char_p
     lib.ca_kernel_launches.argtypes = []
@@ -332,6 +334,15 @@ class Plan:
     def last_status(self) -> Dict[str, int]:
         lib = load_library()
         return {k: lib.ca_last_status(_ptr(v)) for k, v in self.ws.items()}
+
+    def recomputed_clusters(self) -> int:
+        """Query clusters that the second pass of the attention call has recomputed with the fp32
+        kernel since this plan was made (ca_attn_recomputed of the C library)."""
+        lib = load_library()
+        n = lib.ca_attn_recomputed(_ptr(self.ws["attn"]))
+        if n < 0:
+            _check(-n, "ca_attn_recomputed")
+        return n
 
 
 # -- functional forms with the C names ------------------------------------------

@@ -425,6 +425,15 @@ int cluster_qk_basic(const ca_problem_t* p, const void* Q, const void* K, const 
   return CA_OK;
 }
 
+int ca_attn_recomputed(const void* ws) {
+  if (!ws) return -CA_ERR_INVALID_ARG;
+  int count = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess) return -CA_ERR_CUDA;
+  if (cudaMemcpy(&count, static_cast<const int*>(ws) + 1, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return -CA_ERR_CUDA;
+  return count;
+}
+
 int ca_last_status(const void* ws) {
   if (!ws) return CA_ERR_INVALID_ARG;
   int status = 0;

@@ -20,7 +20,7 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
                 const int32_t* __restrict__ keep_count, int list_stride,
                 const int32_t* __restrict__ perm_q, int n_q, int n_k, int c_q, int c_k, int keep_all,
                 int compensate, float scale, T* __restrict__ O, float* __restrict__ lse,
-                const int32_t* __restrict__ redo, int redo_tiles) {
+                const int32_t* __restrict__ redo, int redo_tiles, int* __restrict__ redo_count) {
   constexpr int LD = D + 1;
   constexpr int NC = D / 8;              // output columns per thread
   extern __shared__ float smem[];
@@ -46,6 +46,7 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
     bool marked = false;
     for (int t = 0; t < redo_tiles; ++t) marked |= redo[((size_t)p * n_qc + qc) * 2 + t] != 0;
     if (!marked) return;
+    if (threadIdx.x == 0 && redo_count) atomicAdd(redo_count, 1);   // statistics: clusters recomputed
   }
   const size_t q_base = ((size_t)p * n_qc + qc) * (size_t)c_q;
   const T* Kh = Kp + (size_t)p * n_kc * (size_t)c_k * D;
@@ -174,7 +175,7 @@ template <typename T>
 static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* Vp, const float* ck,
                     const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, T* O,
-                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles) {
+                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles, int* redo_count) {
   const int P = pr.batch * pr.heads, D = pr.head_dim;
   const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
   const int tiles = ceil_div(pr.cluster_q, kRefQR);
@@ -186,13 +187,13 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
                                         pr.n_q, pr.n_k,
-                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles);
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles, redo_count);
   } else {
     auto k = attn_ref_kernel<T, 128>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
                                         pr.n_q, pr.n_k,
-                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles);
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles, redo_count);
   }
   CA_LAUNCH_CHECK();
   return CA_OK;
@@ -201,15 +202,15 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
-                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles) {
+                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles, int* redo_count) {
   if (pr.dtype == CA_DTYPE_BF16)
     return launch_t(pr, static_cast<const __nv_bfloat16*>(Qp), static_cast<const __nv_bfloat16*>(Kp),
                     static_cast<const __nv_bfloat16*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride,
                     perm_q, scale,
-                    static_cast<__nv_bfloat16*>(O), lse, st, redo, redo_tiles);
+                    static_cast<__nv_bfloat16*>(O), lse, st, redo, redo_tiles, redo_count);
   return launch_t(pr, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
                   static_cast<const float*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale,
-                  static_cast<float*>(O), lse, st, redo, redo_tiles);
+                  static_cast<float*>(O), lse, st, redo, redo_tiles, redo_count);
 }
 
 }  // namespace ca

@@ -681,7 +681,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   // second pass: query tiles whose scores left the range of the fast softmax (a climb of more than
   // 2^96 within 64 keys) are recomputed by the fp32 kernel; its CTAs return at once for the others
   return launch_attn_ref(pr, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O, lse,
-                         st, redo, (int)grid.x / n_qc);
+                         st, redo, (int)grid.x / n_qc, status + 1);
 }
 
 }  // namespace ca

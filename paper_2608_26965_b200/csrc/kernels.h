@@ -68,7 +68,8 @@ int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
-                    float* lse, cudaStream_t st, const int32_t* redo = nullptr, int redo_tiles = 0);
+                    float* lse, cudaStream_t st, const int32_t* redo = nullptr, int redo_tiles = 0,
+                    int* redo_count = nullptr);
 
 // attn_tc.cu
 bool attn_tc_supported(const ca_problem_t& pr);

@@ -149,5 +149,8 @@ def test_attention_scores_that_rise_along_the_list(d, c_q, c_k, compensate):
     assert all(v == 0 for v in plan.last_status().values())
     O, lse = O[0, 0].float().cpu().numpy(), lse[0, 0].cpu().numpy()
     assert np.isfinite(O).all() and np.isfinite(lse).all()
+    # the climbs of 2^300 and 2^600 leave the range of the tensor-core kernel's late reference:
+    # those query clusters went through the second pass
+    assert plan.recomputed_clusters() > 0
     assert np.abs(O - o_ref).max() <= 2e-2 and np.linalg.norm(O - o_ref) <= 5e-3 * np.linalg.norm(o_ref)
     assert np.abs(lse - lse_ref).max() <= 2e-2 + 1e-4 * np.abs(lse_ref).max()

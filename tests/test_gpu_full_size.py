@@ -35,6 +35,7 @@ def run_workload(name, keep=None):
     O = plan.forward(dev(Q), dev(K), dev(V), want_lse=True)
     torch.cuda.synchronize()
     assert all(v == 0 for v in plan.last_status().values())
+    assert plan.recomputed_clusters() == 0          # everything stayed on the tensor-core kernel
     return w, Q, K, V, plan, O
 
 
@@ -116,6 +117,7 @@ def test_tabular_full_size_adaptive_selection():
     O, lse = plan.forward_adaptive(dev(Q), dev(K), dev(V), recall=0.5, min_count=16, want_lse=True)
     torch.cuda.synchronize()
     assert all(v == 0 for v in plan.last_status().values())
+    assert plan.recomputed_clusters() == 0          # everything stayed on the tensor-core kernel
     c = w.cluster
     keep_all = plan.keep_count[0]
     assert int(keep_all.min()) >= 16 and int(keep_all.max()) <= w.n_kc
@@ -164,6 +166,7 @@ def test_tabular_full_size_basic_splitting():
     plan.cluster_qk_basic(dev(Q, dt), dev(K, dt), dev(V, dt), dev(nq), dev(nk), 3)
     torch.cuda.synchronize()
     assert all(v == 0 for v in plan.last_status().values())
+    assert plan.recomputed_clusters() == 0          # everything stayed on the tensor-core kernel
     for perm, n in ((plan.perm_q[0], w.n_q), (plan.perm_k[0], w.n_k)):
         srt = torch.sort(perm, dim=1).values
         assert torch.equal(srt, torch.arange(n, device=DEV, dtype=torch.int32).expand_as(srt))
