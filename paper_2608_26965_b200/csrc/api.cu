@@ -246,8 +246,7 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     }
     CA_TRY(launch_split(nullptr, yk_out, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
                         perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 2, st, nullptr, w.Ytk));
-    CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
-    CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+    CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
     // ---- join
     CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->join, 0));
     return CA_OK;
@@ -256,8 +255,7 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
   CA_TRY(launch_split(yq, yk, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
                       perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 3, st));
   CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
-  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
-  CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
   return CA_OK;
 }
 
@@ -420,8 +418,7 @@ int cluster_qk_basic(const ca_problem_t* p, const void* Q, const void* K, const 
                             p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp, perm_k, w.perm_k_tmp,
                             w.keybuf_q, w.keybuf_k, st));
   CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
-  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st));
-  CA_TRY(launch_permute_centroid(V, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Vp, cv, nullptr, st));
+  CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
   return CA_OK;
 }
 

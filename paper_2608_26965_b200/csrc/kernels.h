@@ -53,7 +53,8 @@ int launch_split_basic(const void* Q, const void* K, int dtype, const float* A_q
 int split_levels_for(int n, int c);
 int launch_cast_f64_f32(const double* src, float* dst, size_t count, cudaStream_t st);
 int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P, int n, int D, int c,
-                            void* Xp, float* cen, int32_t* count, cudaStream_t st);
+                            void* Xp, float* cen, int32_t* count, cudaStream_t st, const void* X2 = nullptr,
+                            void* Xp2 = nullptr, float* cen2 = nullptr);
 
 // select.cu
 size_t select_smem_bytes(int n_kc, int D, int qt);

@@ -7,13 +7,20 @@ namespace ca {
 
 // One CTA (128 threads) per cluster.  A row is VEC 16-byte vectors; thread t owns
 // vector t % VEC of rows t / VEC, t / VEC + G, ...  Row sums are combined in a
-// fixed order, so the centroids are reproducible.
+// fixed order, so the centroids are reproducible.  A second tensor gathered by the same
+// permutation (the values next to the keys) rides along as blockIdx.z = 1.
 template <typename T, int D>
-__global__ void __launch_bounds__(128) permute_centroid_kernel(const T* __restrict__ X,
+__global__ void __launch_bounds__(128) permute_centroid_kernel(const T* __restrict__ X0, const T* __restrict__ X1,
                                                                const int32_t* __restrict__ perm, int n,
-                                                               int c, int n_c, T* __restrict__ Xp,
-                                                               float* __restrict__ centroid,
-                                                               int32_t* __restrict__ count) {
+                                                               int c, int n_c, T* __restrict__ Xp0,
+                                                               T* __restrict__ Xp1,
+                                                               float* __restrict__ centroid0,
+                                                               float* __restrict__ centroid1,
+                                                               int32_t* __restrict__ count0) {
+  const T* X = blockIdx.z ? X1 : X0;
+  T* Xp = blockIdx.z ? Xp1 : Xp0;
+  float* centroid = blockIdx.z ? centroid1 : centroid0;
+  int32_t* count = blockIdx.z ? nullptr : count0;
   constexpr int EPV = 16 / sizeof(T);          // elements per 16-byte vector
   constexpr int VEC = D / EPV;                 // vectors per row
   constexpr int G = 128 / VEC;                 // rows in flight
@@ -50,22 +57,26 @@ __global__ void __launch_bounds__(128) permute_centroid_kernel(const T* __restri
 }
 
 template <typename T>
-static int launch_t(const T* X, const int32_t* perm, int P, int n, int D, int c, T* Xp, float* cen,
-                    int32_t* count, cudaStream_t st) {
+static int launch_t(const T* X, const T* X2, const int32_t* perm, int P, int n, int D, int c, T* Xp, T* Xp2,
+                    float* cen, float* cen2, int32_t* count, cudaStream_t st) {
   const int n_c = ceil_div(n, c);
-  dim3 grid(n_c, P);
-  if (D == 64) permute_centroid_kernel<T, 64><<<grid, 128, 0, st>>>(X, perm, n, c, n_c, Xp, cen, count);
-  else permute_centroid_kernel<T, 128><<<grid, 128, 0, st>>>(X, perm, n, c, n_c, Xp, cen, count);
+  dim3 grid(n_c, P, X2 ? 2 : 1);
+  if (D == 64)
+    permute_centroid_kernel<T, 64><<<grid, 128, 0, st>>>(X, X2, perm, n, c, n_c, Xp, Xp2, cen, cen2, count);
+  else
+    permute_centroid_kernel<T, 128><<<grid, 128, 0, st>>>(X, X2, perm, n, c, n_c, Xp, Xp2, cen, cen2, count);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
 
 int launch_permute_centroid(const void* X, int dtype, const int32_t* perm, int P, int n, int D, int c,
-                            void* Xp, float* cen, int32_t* count, cudaStream_t st) {
+                            void* Xp, float* cen, int32_t* count, cudaStream_t st, const void* X2, void* Xp2,
+                            float* cen2) {
   if (dtype == CA_DTYPE_BF16)
-    return launch_t(static_cast<const __nv_bfloat16*>(X), perm, P, n, D, c,
-                    static_cast<__nv_bfloat16*>(Xp), cen, count, st);
-  return launch_t(static_cast<const float*>(X), perm, P, n, D, c, static_cast<float*>(Xp), cen, count, st);
+    return launch_t(static_cast<const __nv_bfloat16*>(X), static_cast<const __nv_bfloat16*>(X2), perm, P, n, D, c,
+                    static_cast<__nv_bfloat16*>(Xp), static_cast<__nv_bfloat16*>(Xp2), cen, cen2, count, st);
+  return launch_t(static_cast<const float*>(X), static_cast<const float*>(X2), perm, P, n, D, c,
+                  static_cast<float*>(Xp), static_cast<float*>(Xp2), cen, cen2, count, st);
 }
 
 }  // namespace ca
