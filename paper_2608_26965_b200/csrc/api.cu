@@ -171,6 +171,9 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     float* yk_out = Yk ? Yk : w.Yk;
     // bf16 storage runs the O(n d^2) passes on the tensor cores; fp32 storage on the CUDA cores
     const bool tc = p->dtype == CA_DTYPE_BF16;
+    // d = 64: the one CTA per head that computes the bias also lays the weights out for the
+    // tensor-core projection (one launch less on each side); at d = 128 that is too much for one CTA
+    const bool fold = tc && D == 64;
     __nv_bfloat16* qp_hi = reinterpret_cast<__nv_bfloat16*>(w.Qprime);          // r(q) as bf16 hi + lo parts
     __nv_bfloat16* qp_lo = qp_hi + (size_t)P * p->n_q * D;
     // metric matrices (Section 3.2.2) and their factors F_q F_q^T = M, F_k F_k^T = C_K (they stand
@@ -219,10 +222,10 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     }
     CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, sq));
     CA_TRY(launch_eigh(covQ, P, D, w.basis + (size_t)P * DD, w.basis32 + (size_t)P * DD, nullptr, sq));
-    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, sq));
+    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, sq, fold ? w.wt2_hi : nullptr, fold ? w.wt2_lo : nullptr));
     if (tc) {
       CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
-                                 w.wt2_lo, w.status, sq, w.Ytq));
+                                 w.wt2_lo, w.status, sq, w.Ytq, fold));
     } else {
       CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
     }
@@ -237,10 +240,10 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, unnormalized ? 1.0 : 1.0 / (double)p->n_k, 0, covK, nullptr, st));
     CA_TRY(launch_eigh(covK, P, D, w.basis, w.basis32, nullptr, st));
     CA_TRY(launch_small_matmul(Rq, w.basis, P, D, 1.0, 0, w.WK, w.WK32, st));
-    CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st));
+    CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st, fold ? w.wt_hi : nullptr, fold ? w.wt_lo : nullptr));
     if (tc) {
       CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
-                                 w.wt_lo, w.status, st, w.Ytk));
+                                 w.wt_lo, w.status, st, w.Ytk, fold));
     } else {
       CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
     }

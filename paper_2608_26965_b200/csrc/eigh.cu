@@ -161,10 +161,13 @@ __global__ void __launch_bounds__(256) small_matmul_kernel(const double* __restr
 }
 
 // bias[p][j] = - sum_i (sum[p][i] / n) * W[p][i][j].  Eight threads per output column, each with all of
-// its loads in flight at once; partial sums combined in a fixed order.
+// its loads in flight at once; partial sums combined in a fixed order.  The same CTA also lays W out
+// for the tensor-core projection (W^T as bf16 hi + lo parts, [D out][D in]) when asked to.
 template <int D>
 __global__ void __launch_bounds__(8 * D) bias_kernel(const double* __restrict__ sum, const float* __restrict__ W,
-                                                     double n, float* __restrict__ bias) {
+                                                     double n, float* __restrict__ bias,
+                                                     __nv_bfloat16* __restrict__ wt_hi,
+                                                     __nv_bfloat16* __restrict__ wt_lo) {
   constexpr int PER = D / 8;
   __shared__ float mean[D];
   __shared__ float part[8][D];
@@ -186,6 +189,15 @@ __global__ void __launch_bounds__(8 * D) bias_kernel(const double* __restrict__ 
 #pragma unroll
     for (int q = 0; q < 8; ++q) t += part[q][j];
     bias[(size_t)p * D + j] = -t;
+  }
+  if (wt_hi) {
+    for (int e = threadIdx.x; e < D * D; e += 8 * D) {
+      const int o = e / D, k = e % D;
+      const float w = W[(size_t)p * D * D + k * D + o];
+      const __nv_bfloat16 h = __float2bfloat16_rn(w);
+      wt_hi[(size_t)p * D * D + e] = h;
+      wt_lo[(size_t)p * D * D + e] = __float2bfloat16_rn(w - __bfloat162float(h));
+    }
   }
 }
 
@@ -218,9 +230,12 @@ int launch_small_matmul(const double* A, const double* B, int P, int D, double a
   CA_LAUNCH_CHECK();
   return CA_OK;
 }
-int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st) {
-  if (D == 64) bias_kernel<64><<<P, 512, 0, st>>>(sum, W, (double)n, bias);
-  else bias_kernel<128><<<P, 1024, 0, st>>>(sum, W, (double)n, bias);
+int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st,
+                void* wt_hi, void* wt_lo) {
+  __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(wt_hi);
+  __nv_bfloat16* lo = static_cast<__nv_bfloat16*>(wt_lo);
+  if (D == 64) bias_kernel<64><<<P, 512, 0, st>>>(sum, W, (double)n, bias, hi, lo);
+  else bias_kernel<128><<<P, 1024, 0, st>>>(sum, W, (double)n, bias, hi, lo);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }

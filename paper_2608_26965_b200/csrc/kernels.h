@@ -21,7 +21,8 @@ int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows,
                    double* gram, double* colsum, int* status, cudaStream_t st);
 int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, const float* W,
                         const float* bias, int normalize, float* out, void* out_hi, void* out_lo,
-                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t = nullptr);
+                        void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t = nullptr,
+                        bool weights_ready = false);
 
 // eigh.cu
 int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
@@ -33,7 +34,8 @@ int launch_covariance(const double* gram, const double* sum, int P, int D, int n
 int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
                         double* C, float* C32, cudaStream_t st);
 int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st);
-int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st);
+int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st,
+                void* wt_hi = nullptr, void* wt_lo = nullptr);
 
 // split.cu
 int split_levels_for(int n, int c);
