@@ -63,67 +63,6 @@ __global__ void __launch_bounds__(1024) cholesky_factor_kernel(const double* __r
   }
 }
 
-// One barrier per column: column j of F goes straight to the outputs, the trailing block is
-// updated from the unscaled column (a_ik -= a_ij a_kj / pivot), and the thread that produces the next
-// pivot also leaves its reciprocal and reciprocal root for the next column.
-template <int D>
-__global__ void __launch_bounds__(1024) cholesky_factor_1b_kernel(const double* __restrict__ A_in,
-                                                               double* __restrict__ out64,
-                                                               float* __restrict__ out32) {
-  constexpr int LDA = D + 1;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* A = reinterpret_cast<double*>(smem_raw);       // [D][LDA], lower triangle is updated in place
-  __shared__ double s_tol;
-  __shared__ double s_inv[2], s_inv2[2];                 // 1 / sqrt(pivot), 1 / pivot; by column parity
-  const int tid = threadIdx.x, NT = blockDim.x;
-  const double* Ain = A_in + (size_t)blockIdx.x * D * D;
-  double* o64 = out64 + (size_t)blockIdx.x * D * D;
-  float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
-  for (int e = tid; e < D * D; e += NT) {
-    const int i = e / D, j = e % D;
-    A[i * LDA + j] = 0.5 * (Ain[i * D + j] + Ain[j * D + i]);
-    if (j > i) {                                         // F is lower-triangular
-      o64[e] = 0.0;
-      if (o32) o32[e] = 0.f;
-    }
-  }
-  __syncthreads();
-  if (tid == 0) {
-    double mx = 0.0;
-    for (int i = 0; i < D; ++i) mx = fmax(mx, A[i * LDA + i]);
-    const double tol = 1e-12 * mx, piv = A[0];
-    s_tol = tol;
-    const double r = (piv > tol) ? rsqrt(piv) : 0.0;
-    s_inv[0] = r;
-    s_inv2[0] = r * r;
-  }
-  __syncthreads();
-  const double tol = s_tol;
-  for (int j = 0; j < D; ++j) {
-    const double inv = s_inv[j & 1], inv2 = s_inv2[j & 1];
-    // column j of F (rows j..D-1); a dropped pivot gives a zero column and no update
-    for (int i = j + tid; i < D; i += NT) {
-      const double v = A[i * LDA + j] * inv;
-      o64[i * D + j] = v;
-      if (o32) o32[i * D + j] = (float)v;
-    }
-    const int rem = D - 1 - j;
-    for (int e = tid; e < rem * rem; e += NT) {
-      const int i = j + 1 + e / rem, k = j + 1 + e % rem;
-      if (k <= i) {
-        const double a = A[i * LDA + k] - A[i * LDA + j] * A[k * LDA + j] * inv2;
-        A[i * LDA + k] = a;
-        if (i == j + 1 && k == j + 1) {                  // the next pivot
-          const double r = (a > tol) ? rsqrt(a) : 0.0;
-          s_inv[(j + 1) & 1] = r;
-          s_inv2[(j + 1) & 1] = r * r;
-        }
-      }
-    }
-    __syncthreads();
-  }
-}
-
 int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st) {
   const size_t smem = sizeof(double) * D * (D + 1);
   if (D == 64) {
@@ -131,8 +70,7 @@ int launch_cholesky_factor(const double* A, int count, int D, double* out64, flo
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<count, 512, smem, st>>>(A, out64, out32);
   } else {
-    // d = 128: the one-barrier form is the faster one (185 -> ~120 us); at d = 64 the three-barrier form is
-    auto k = cholesky_factor_1b_kernel<128>;
+    auto k = cholesky_factor_kernel<128>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<count, 1024, smem, st>>>(A, out64, out32);
   }
