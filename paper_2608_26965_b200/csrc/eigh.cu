@@ -21,7 +21,7 @@ __global__ void __launch_bounds__(1024) cholesky_factor_kernel(const double* __r
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* A = reinterpret_cast<double*>(smem_raw);       // [D][LDA], lower triangle is updated in place
   __shared__ double s_tol;
-  __shared__ double s_inv;
+  __shared__ double s_inv, s_l10, s_inv1;
   const int tid = threadIdx.x, NT = blockDim.x;
   const double* Ain = A_in + (size_t)blockIdx.x * D * D;
   for (int e = tid; e < D * D; e += NT) {
@@ -35,21 +35,34 @@ __global__ void __launch_bounds__(1024) cholesky_factor_kernel(const double* __r
     s_tol = 1e-12 * mx;
   }
   __syncthreads();
-  for (int j = 0; j < D; ++j) {
+  // two columns per round (three barriers for the pair): thread 0 prepares both pivots -- the second
+  // one after its update by the first column -- then every row scales its two entries, then the
+  // trailing block takes the rank-2 update
+  for (int j = 0; j < D; j += 2) {
     if (tid == 0) {
-      const double piv = A[j * LDA + j];
-      s_inv = (piv > s_tol) ? rsqrt(piv) : 0.0;
+      const double piv0 = A[j * LDA + j];
+      const double inv0 = (piv0 > s_tol) ? rsqrt(piv0) : 0.0;
+      const double l10 = A[(j + 1) * LDA + j] * inv0;
+      const double piv1 = A[(j + 1) * LDA + j + 1] - l10 * l10;
+      s_inv = inv0;
+      s_l10 = l10;
+      s_inv1 = (piv1 > s_tol) ? rsqrt(piv1) : 0.0;
     }
     __syncthreads();
-    const double inv = s_inv;
-    // column j of F (rows j..D-1); a dropped pivot gives a zero column
-    for (int i = j + tid; i < D; i += NT) A[i * LDA + j] *= inv;
+    const double inv0 = s_inv, l10 = s_l10, inv1 = s_inv1;
+    // columns j and j+1 of F; a dropped pivot gives a zero column
+    for (int i = j + tid; i < D; i += NT) {
+      const double c0 = A[i * LDA + j] * inv0;
+      A[i * LDA + j] = c0;
+      if (i > j) A[i * LDA + j + 1] = (A[i * LDA + j + 1] - c0 * l10) * inv1;
+    }
     __syncthreads();
     // trailing update of the lower triangle
-    const int rem = D - 1 - j;
+    const int rem = D - 2 - j;
     for (int e = tid; e < rem * rem; e += NT) {
-      const int i = j + 1 + e / rem, k = j + 1 + e % rem;
-      if (k <= i) A[i * LDA + k] -= A[i * LDA + j] * A[k * LDA + j];
+      const int i = j + 2 + e / rem, k = j + 2 + e % rem;
+      if (k <= i)
+        A[i * LDA + k] -= A[i * LDA + j] * A[k * LDA + j] + A[i * LDA + j + 1] * A[k * LDA + j + 1];
     }
     __syncthreads();
   }
