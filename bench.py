@@ -40,7 +40,7 @@ UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 # DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None = not captured.
-NCU_TRAFFIC_BYTES = {"tabular": 570.0e6, "video480": 1269.0e6}   # scaled by heads from the 4- and 8-head captures in profiles/
+NCU_TRAFFIC_BYTES = {"tabular": 554.2e6, "video480": 1269.0e6}   # scaled by heads from the 4- and 8-head captures in profiles/
 
 
 def parse_args():
