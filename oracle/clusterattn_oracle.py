@@ -19,10 +19,21 @@ Pins (tests/test_oracle_*.py):
   diagonalize ............ decorrelated coordinates, descending variance, isometry
   split_point / recursive_split ... partition + size invariants (Section 3.1),
                            d=1 closed form "sort and chunk", brute-force one-level cut
+  split_coordinates ...... squared distances of the key coordinates == (k1-k2)^T (Q^T Q/n) (k1-k2)
+                           and of the query coordinates == the distance of r(q) written with
+                           K_c alone (no root), both query representations (Section 3.2.2,
+                           Appendix B.1 / B.2); sign rule independent of the root's form
   centroids / centroid_scores ..... mean pairwise logit identity, Jensen bound (Section 3.3.1)
   select_topk ............ brute-force full sort
   cluster_attention ...... all blocks kept == dense; c=1 == dense; eqs. (2)-(4);
                            exact SMC error decomposition (Appendix A)
+  *_f32 helpers .......... hand-computed sums whose bits depend on the order of the additions;
+                           the fp64 decisions on inputs without near-ties
+Decisions (which coordinate a split takes, which key clusters are kept) are DEFINED by the
+float64 functions `choose_coordinate`, `centroid_scores` + `select_topk`.  The `_f32` functions
+beside them restate the same quantities in float32 with a fixed operation order; they exist so
+that a float32 implementation can be compared bit for bit, and the tests count where the two
+decisions differ (only at near-ties).
 Conventions of this build that the paper leaves open (subsample positions,
 round-half-up split point, fp32 rounding of the split coordinates, eigenvector
 sign) are "parity unpinned" by the paper: the oracle is their definition.
@@ -104,27 +115,34 @@ def query_representation(Q, R_k, normalize=True):
 # --------------------------------------------------------------------------
 # Section 3.2.1 "Diagonalized recursive splitting": project the (transformed)
 # rows onto the principal components of the full set.  Centred covariance,
-# components in descending eigenvalue order; each eigenvector's sign is fixed
-# so that its entry of largest magnitude (lowest index on ties) is positive.
+# components in descending eigenvalue order.  The paper leaves the sign of a
+# component open; it is fixed here through the map from the ORIGINAL space:
+# with `lift` = the matrix R that produced the transformed rows (keys: x R_q,
+# queries: R_k q before normalisation), component t is oriented so that the
+# entry of largest magnitude (lowest index on ties) of column t of R E is
+# positive.  R E does not change when R is replaced by another root R U of the
+# same metric (E becomes U^T E), so the coordinates, signs included, are a
+# function of the metric alone.  Without `lift` the rule applies to E itself.
 # Returns (Y, eigenvalues, basis).
 # --------------------------------------------------------------------------
-def principal_basis(C):
+def principal_basis(C, lift=None):
     lam, E = np.linalg.eigh(0.5 * (C + C.T))
     order = np.argsort(-lam, kind="stable")
     lam, E = lam[order], E[:, order]
+    W = E if lift is None else np.asarray(lift, F64) @ E
     for t in range(E.shape[1]):
-        j = int(np.argmax(np.abs(E[:, t])))
-        if E[j, t] < 0:
+        j = int(np.argmax(np.abs(W[:, t])))
+        if W[j, t] < 0:
             E[:, t] = -E[:, t]
     return lam, E
 
 
-def diagonalize(X):
+def diagonalize(X, lift=None):
     X = np.asarray(X, F64)
     mu = X.mean(axis=0, keepdims=True)
     Xc = X - mu
     C = (Xc.T @ Xc) / X.shape[0]
-    lam, E = principal_basis(C)
+    lam, E = principal_basis(C, lift)
     return Xc @ E, lam, E
 
 
@@ -155,11 +173,21 @@ def interleaved_sum32(x):
 
 
 def choose_coordinate(sub):
-    """Coordinate of highest variance over the subsample rows `sub` [m, d]; lowest
-    coordinate on exact ties.  This estimate only feeds an argmax (a discrete
-    decision), so it is taken in the precision of the coordinates themselves,
-    float32, with a fixed operation order (`interleaved_sum32`; no fused
-    multiply-add): population variance, mean first, then squared deviations."""
+    """Section 3.2.1: the coordinate of highest variance over the subsample rows
+    `sub` [m, d] (population variance, float64); lowest coordinate on exact ties.
+    This is the definition of the decision."""
+    sub = np.asarray(sub, F64)
+    var = ((sub - sub.mean(axis=0, keepdims=True)) ** 2).mean(axis=0)
+    return int(np.argmax(var)), var
+
+
+def choose_coordinate_f32(sub):
+    """The same decision restated in float32 with a fixed operation order
+    (`interleaved_sum32`; no fused multiply-add): mean first, then squared
+    deviations.  Not a definition: a helper against which a float32
+    implementation can be compared bit for bit.  It can differ from
+    `choose_coordinate` only where the two largest variances lie within the
+    rounding error of a float32 sum of m terms."""
     sub = np.ascontiguousarray(sub, dtype=np.float32)
     m = np.float32(sub.shape[0])
     mean = interleaved_sum32(sub) / m
@@ -168,13 +196,15 @@ def choose_coordinate(sub):
     return int(np.argmax(var)), var
 
 
-def recursive_split(Y32, c, return_tree=False):
+def recursive_split(Y32, c, return_tree=False, choose=choose_coordinate):
     """Diagonalized recursive splitting (Section 3.2.1) on fp32 coordinates.
 
     Y32 [N, d] float32: rows in principal-component coordinates.  Returns
     perm [N] (position -> original row); cluster j is perm[j*c:(j+1)*c].
     Every set keeps its rows in ascending original order, a split orders the
     set by (coordinate value, original row) and sends the first L rows down.
+    `choose` picks the split coordinate from the subsample (the float64
+    definition unless the float32 restatement is asked for).
     """
     Y32 = np.asarray(Y32)
     assert Y32.dtype == np.float32
@@ -191,7 +221,7 @@ def recursive_split(Y32, c, return_tree=False):
             rows = perm[lo:hi].copy()
             m = min(d, s)
             sub = Y32[rows[subsample_positions(s, m)]]
-            t, _ = choose_coordinate(sub)
+            t, _ = choose(sub)
             L = split_point(s, c)
             keys = Y32[rows, t]
             order = np.lexsort((rows, keys))        # by value, then original row
@@ -319,6 +349,11 @@ def basic_recursive_split(X32, A32, noise32, c, iterations=3, return_tree=False)
     return perm
 
 
+def recursive_split_f32(Y32, c, return_tree=False):
+    """`recursive_split` with every coordinate chosen by `choose_coordinate_f32`."""
+    return recursive_split(Y32, c, return_tree, choose=choose_coordinate_f32)
+
+
 def split_levels(n, c):
     """Depth of the split tree: the largest set follows the larger child."""
     levels, big = 0, n
@@ -358,11 +393,12 @@ def centroid_scores(cq, ck):
 
 
 def centroid_scores_f32(cq, ck):
-    """The same scores in float32 with a fixed operation order: centroids rounded
-    to float32, terms added for k = 0, 1, ... with the product and the sum rounded
-    separately (no fused multiply-add).  The scores only feed the top-k decision,
-    which is therefore taken in the precision the device uses; any implementation
-    that follows the order gets the same bits."""
+    """The same scores restated in float32 with a fixed operation order: centroids
+    rounded to float32, terms added for k = 0, 1, ... with the product and the sum
+    rounded separately (no fused multiply-add).  Not a definition: a helper against
+    which a float32 implementation can be compared bit for bit; the selection it
+    leads to can differ from that of `centroid_scores` only where the k-th and
+    (k+1)-th scores lie within float32 rounding of each other."""
     cq = np.ascontiguousarray(cq, dtype=np.float32)
     ck = np.ascontiguousarray(ck, dtype=np.float32)
     S = np.zeros((cq.shape[0], ck.shape[0]), np.float32)
@@ -516,16 +552,17 @@ def split_coordinates(Q, K, adaptive=False):
         R_k = psd_root(centered_scatter(K) / np.asarray(K).shape[0])
     else:
         R_k = psd_root(centered_scatter(K))
-    Yk, _, _ = diagonalize(transform_keys(K, R_q))
-    Yq, _, _ = diagonalize(query_representation(Q, R_k, normalize=not adaptive))
+    Yk, _, _ = diagonalize(transform_keys(K, R_q), lift=R_q)
+    Yq, _, _ = diagonalize(query_representation(Q, R_k, normalize=not adaptive), lift=R_k)
     return Yq.astype(np.float32), Yk.astype(np.float32)
 
 
-def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None, adaptive=False):
+def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None, adaptive=False, f32_decisions=False):
     if Yq32 is None or Yk32 is None:
         Yq32, Yk32 = split_coordinates(Q, K, adaptive)
-    perm_q = recursive_split(Yq32, c_q)
-    perm_k = recursive_split(Yk32, c_k)
+    choose = choose_coordinate_f32 if f32_decisions else choose_coordinate
+    perm_q = recursive_split(Yq32, c_q, choose=choose)
+    perm_k = recursive_split(Yk32, c_k, choose=choose)
     cq, count_q = centroids(Q, perm_q, c_q)
     ck, count_k = centroids(K, perm_k, c_k)
     cv, _ = centroids(V, perm_k, c_k)
@@ -534,6 +571,12 @@ def cluster_qk(Q, K, V, c_q, c_k, Yq32=None, Yk32=None, adaptive=False):
 
 
 def select_blocks(cq, ck, keep):
+    """Section 3.3: the `keep` best key clusters per query cluster by the float64 scores."""
+    return select_topk(centroid_scores(cq, ck), keep)
+
+
+def select_blocks_f32(cq, ck, keep):
+    """The same selection on the float32 restatement of the scores (`centroid_scores_f32`)."""
     return select_topk(centroid_scores_f32(cq, ck), keep)
 
 

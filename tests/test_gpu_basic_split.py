@@ -102,7 +102,7 @@ def test_basic_split_with_device_metrics_and_attention(name, H, n_q, n_k):
         assert np.array_equal(pq, orc.basic_recursive_split(Q[h], A_q, nq[h], c, 3))
         assert np.array_equal(pk, orc.basic_recursive_split(K[h], A_k, nk[h], c, 3))
         idx = plan.block_idx[0, h].cpu().numpy()
-        assert np.array_equal(idx, orc.select_blocks(plan.cq[0, h].cpu().numpy(), plan.ck[0, h].cpu().numpy(), p.keep))
+        assert np.array_equal(idx, orc.select_blocks_f32(plan.cq[0, h].cpu().numpy(), plan.ck[0, h].cpu().numpy(), p.keep))
         o_ref, lse_ref = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, c, c, idx, True,
                                                ck=plan.ck[0, h].cpu().numpy(), cv=plan.cv[0, h].cpu().numpy(),
                                                count_k=plan.count_k[0, h].cpu().numpy())

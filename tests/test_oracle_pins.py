@@ -141,8 +141,9 @@ def test_diagonalize_is_pca_of_the_rows():
 
 
 def test_split_coordinates_do_not_depend_on_the_form_of_the_root():
-    # using E sqrt(L) instead of E sqrt(L) E^T rotates the transformed keys; the
-    # principal-component coordinates are the same up to per-coordinate sign.
+    # using E sqrt(L), or a Cholesky factor, instead of E sqrt(L) E^T rotates the
+    # transformed keys; the principal-component coordinates are the same, and with the
+    # sign taken from the map out of the original space (lift) the signs are the same too.
     r = rng(7)
     Q = r.standard_normal((300, 6)) * np.array([3, 2, 1.5, 1, 0.5, 0.2])
     K = r.standard_normal((400, 6)) @ r.standard_normal((6, 6))
@@ -150,10 +151,58 @@ def test_split_coordinates_do_not_depend_on_the_form_of_the_root():
     lam, E = np.linalg.eigh(M)
     R_sym = orc.psd_root(M)
     R_alt = E * np.sqrt(np.maximum(lam, 0))
+    R_chol = np.linalg.cholesky(M)
+    assert np.allclose(R_alt @ R_alt.T, M) and np.allclose(R_chol @ R_chol.T, M)
     Y1, l1, _ = orc.diagonalize(K @ R_sym)
     Y2, l2, _ = orc.diagonalize(K @ R_alt)
     assert np.allclose(l1, l2, rtol=1e-9)
     assert np.allclose(np.abs(Y1), np.abs(Y2), atol=1e-8)
+    Y1, _, E1 = orc.diagonalize(K @ R_sym, lift=R_sym)
+    for R in (R_alt, R_chol):
+        Y2, _, E2 = orc.diagonalize(K @ R, lift=R)
+        assert np.allclose(Y1, Y2, atol=1e-8)                 # signs included
+        assert np.allclose(R_sym @ E1, R @ E2, atol=1e-8)     # the map from the original space is the same
+    W = R_sym @ E1
+    for t in range(6):
+        assert W[np.argmax(np.abs(W[:, t])), t] > 0
+
+
+# ---------------------------- the clustering stage's coordinates (Section 3.2.2, Appendix B)
+@pytest.mark.parametrize("adaptive", [False, True])
+def test_split_coordinates_carry_the_two_metrics(adaptive):
+    """Keys are compared in the metric of the queries and queries in the metric of the centred
+    keys: which root goes to which side, the 1/n of the un-normalised form and the normalisation
+    of the ranking form are all fixed by distances written WITHOUT any matrix root."""
+    r = rng(70 + adaptive)
+    d, n_q, n_k = 7, 90, 130
+    Q = (r.standard_normal((n_q, d)) * np.linspace(3.0, 0.3, d)) @ r.standard_normal((d, d)) + 0.5
+    K = (r.standard_normal((n_k, d)) * np.linspace(0.2, 2.0, d)) @ r.standard_normal((d, d)) - 1.0
+    Yq, Yk = orc.split_coordinates(Q, K, adaptive=adaptive)
+    assert Yq.dtype == np.float32 and Yk.dtype == np.float32
+    assert Yq.shape == (n_q, d) and Yk.shape == (n_k, d)
+    Yq, Yk = Yq.astype(np.float64), Yk.astype(np.float64)
+    Kc = K - K.mean(0)
+    # keys: |y_i - y_j|^2 = |Q (k_i - k_j)|^2 / n_q      (Section 3.2.2, key clustering)
+    for i, j in zip(r.integers(0, n_k, 40), r.integers(0, n_k, 40)):
+        want = ((Q @ (K[i] - K[j])) ** 2).sum() / n_q
+        assert np.isclose(((Yk[i] - Yk[j]) ** 2).sum(), want, rtol=2e-5, atol=1e-9)
+    for i, j in zip(r.integers(0, n_q, 40), r.integers(0, n_q, 40)):
+        a, b = Kc @ Q[i], Kc @ Q[j]                     # K_c q: the logits up to a per-query shift
+        if adaptive:                                    # Appendix B.1: |K_c (q_i - q_j)|^2 / n_k
+            want = ((a - b) ** 2).sum() / n_k
+        else:                                           # Appendix B.2: unit vectors K_c q / |K_c q|
+            want = 2.0 - 2.0 * (a @ b) / np.sqrt((a @ a) * (b @ b))
+        assert np.isclose(((Yq[i] - Yq[j]) ** 2).sum(), want, rtol=2e-5, atol=1e-7)
+    # both sets are centred and decorrelated with variances in descending order
+    for Y in (Yq, Yk):
+        cov = Y.T @ Y / Y.shape[0]
+        off = cov - np.diag(np.diag(cov))
+        assert np.abs(Y.mean(0)).max() < 1e-5 * np.sqrt(cov[0, 0])
+        assert np.abs(off).max() < 1e-5 * cov[0, 0] and np.all(np.diff(np.diag(cov)) <= 1e-6 * cov[0, 0])
+    # swapping the sides must fail the same checks (the two metrics differ on this input)
+    Yq_s, Yk_s = (y.astype(np.float64) for y in orc.split_coordinates(K[:n_q], Q, adaptive=adaptive))
+    i, j = 3, 11
+    assert not np.isclose(((Yk_s[i] - Yk_s[j]) ** 2).sum(), ((Q @ (Q[i] - Q[j])) ** 2).sum() / n_q, rtol=1e-2)
 
 
 # ------------------------------------------------------ split sizes (Section 3.1)
@@ -244,9 +293,76 @@ def test_choose_coordinate_ties_go_to_lowest_coordinate():
     sub = np.zeros((4, 5))
     sub[:, 2] = [1, -1, 1, -1]
     sub[:, 4] = [1, -1, 1, -1]
-    t, var = orc.choose_coordinate(sub)
-    assert t == 2 and var[2] == var[4] == 1.0
+    for choose in (orc.choose_coordinate, orc.choose_coordinate_f32):
+        t, var = choose(sub)
+        assert t == 2 and var[2] == var[4] == 1.0
     assert orc.subsample_positions(10, 4).tolist() == [0, 2, 5, 7]
+
+
+def test_choose_coordinate_is_the_population_variance_argmax():
+    r = rng(17)
+    sub = r.standard_normal((9, 6)) * np.array([1.0, 3.0, 2.0, 3.5, 0.1, 1.0]) + 10.0
+    t, var = orc.choose_coordinate(sub)
+    brute = [sum((x - sum(col) / 9) ** 2 for x in col) / 9 for col in sub.T.tolist()]
+    assert np.allclose(var, brute, rtol=1e-12) and t == int(np.argmax(brute))
+    assert np.allclose(var, np.var(sub, axis=0), rtol=1e-12)       # library routine, ddof = 0
+
+
+def test_interleaved_sum32_follows_the_stated_order():
+    """Inputs on which the order of the float32 additions decides the bits.  Expected values
+    worked out by hand from: 2^24 + 1 rounds to 2^24 (tie to even), 2^24 + 2 is exact."""
+    big = np.float32(2.0 ** 24)
+
+    def column(m, **rows):
+        x = np.zeros((m, 1), np.float32)
+        for k, v in rows.items():
+            x[int(k[1:])] = v
+        return x
+    # rows 0 and 8 feed partial sum p0, rows 1 and 9 feed p1:
+    # p0 = rn(2^24 + 1) = 2^24, p1 = 1 + 1 = 2, total 2^24 + 2 (row after row: stays at 2^24)
+    x = column(16, r0=big, r8=1.0, r1=1.0, r9=1.0)
+    assert orc.interleaved_sum32(x)[0] == big + np.float32(2.0)
+    assert np.cumsum(x[:, 0], dtype=np.float32)[-1] == big
+    # p0 = rn(2^24 + 1) = 2^24, p1 = 1: rn(2^24 + 1) = 2^24
+    # (partial sums over blocks of consecutive rows would add rows 8 and 9 first: 2^24 + 2)
+    assert orc.interleaved_sum32(column(16, r0=big, r8=1.0, r9=1.0))[0] == big
+    # the tree ((p0+p1)+(p2+p3)) + ((p4+p5)+(p6+p7)) with p0 = 2^24 and seven ones:
+    # (2^24 + 2) + 4 = 2^24 + 6 (left to right over the partial sums: stays at 2^24)
+    y = np.ones((8, 1), np.float32)
+    y[0] = big
+    assert orc.interleaved_sum32(y)[0] == big + np.float32(6.0)
+    # p0 = 2^24, p1 = p5 = 1: (2^24 + 1 -> 2^24) + (0 + 1) -> 2^24
+    # (pairing p0 with p4 and p1 with p5 first would give 2^24 + 2)
+    assert orc.interleaved_sum32(column(8, r0=big, r1=1.0, r5=1.0))[0] == big
+    # p0 = 2^24, p1 = p3 = 1: ((2^24 + 1 -> 2^24) + (0 + 1)) -> 2^24
+    # (pairing p0 with p2 and p1 with p3 first would give 2^24 + 2)
+    assert orc.interleaved_sum32(column(8, r0=big, r1=1.0, r3=1.0))[0] == big
+    # fewer than eight rows, and one sum per column
+    w = np.array([[1.0, 2.0], [3.0, 4.0], [5.0, 6.0]], np.float32)
+    assert orc.interleaved_sum32(w).tolist() == [9.0, 12.0]
+
+
+def test_float32_coordinate_choice_differs_from_the_definition_only_at_near_ties():
+    """Two columns whose variances are almost equal: the float32 restatement may pick the other
+    one, and when it does the two variances lie within the rounding error of a float32 sum."""
+    r = rng(18)
+    differ = 0
+    for trial in range(3000):
+        m = int(r.choice([16, 64, 128]))
+        col = r.standard_normal(m)
+        other = r.permutation(col) * (1.0 + r.uniform(-3e-7, 3e-7))
+        sub = np.stack([col, other, 0.3 * r.standard_normal(m)], axis=1).astype(np.float32)
+        t64, v64 = orc.choose_coordinate(sub)
+        t32, _ = orc.choose_coordinate_f32(sub)
+        if t64 != t32:
+            differ += 1
+            top = np.sort(v64)[::-1]
+            assert (top[0] - top[1]) <= (m / 8 + 8) * 2.0 ** -23 * top[0]
+    assert differ > 0                                          # the search does reach disagreements
+    # well separated variances: the same decision
+    for trial in range(200):
+        sub = (r.standard_normal((64, 8)) * np.linspace(2.0, 0.5, 8)).astype(np.float32)
+        assert orc.choose_coordinate(sub)[0] == orc.choose_coordinate_f32(sub)[0]
 
 
 def test_recursive_split_clusters_are_tighter_than_random_clusters():
@@ -389,8 +505,9 @@ def test_float32_scores_follow_the_exact_scores():
     for k in range(64):
         acc = np.float32(acc + np.float32(np.float32(cq[3, k]) * np.float32(ck[7, k])))
     assert acc == S32[3, 7]
-    # well separated scores: the selection is that of the exact scores
-    assert np.array_equal(orc.select_blocks(cq, ck, 5), orc.select_topk(S64, 5))
+    # well separated scores: the float32 restatement selects what the definition selects
+    assert np.array_equal(orc.select_blocks_f32(cq, ck, 5), orc.select_topk(S64, 5))
+    assert np.array_equal(orc.select_blocks(cq.astype(np.float32), ck.astype(np.float32), 5), orc.select_topk(S64, 5))
 
 
 def test_select_topk_matches_full_sort_with_index_tie_break():
