@@ -19,7 +19,9 @@
  *   - Return value: CA_OK or an error code; nothing is enqueued on error except
  *     for CA_ERR_CUDA (a launch failed part-way).
  *   - The first 256 bytes of a workspace hold a status word that kernels set when
- *     a bounded wait expires (CA_ERR_TIMEOUT); ca_last_status reads it.
+ *     a bounded wait expires (CA_ERR_TIMEOUT) or an index supplied by the caller
+ *     is out of range (CA_ERR_BAD_INDEX); ca_last_status reads it.  Every call
+ *     clears it on its stream before its kernels run.
  */
 #ifndef CLUSTER_ATTENTION_H_
 #define CLUSTER_ATTENTION_H_
@@ -37,7 +39,9 @@ enum {
   CA_ERR_UNSUPPORTED = 2,  /* dtype / head_dim / cluster size outside the supported set      */
   CA_ERR_WORKSPACE = 3,    /* workspace null or smaller than ca_workspace_bytes reports      */
   CA_ERR_CUDA = 4,         /* a CUDA runtime call or kernel launch failed                    */
-  CA_ERR_TIMEOUT = 5       /* (status word only) a bounded device-side wait gave up          */
+  CA_ERR_TIMEOUT = 5,      /* (status word only) a bounded device-side wait gave up          */
+  CA_ERR_BAD_INDEX = 6     /* (status word only) a block list entry, a list length or a perm_q
+                              entry was out of range; the access was skipped                  */
 };
 
 enum { CA_DTYPE_FP32 = 0, CA_DTYPE_BF16 = 1 };
@@ -73,11 +77,17 @@ int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select
 
 /*
  * Clustering (Section 3.2).  Per head, queries and keys separately:
- *   M = Q^T Q / n_q, R_q = sqrt(M) (eigendecomposition, negative eigenvalues
- *   clamped), keys -> K R_q; R_k = sqrt(K_c^T K_c) with K_c the centred keys,
- *   queries -> r(q) = R_k q / |R_k q| (Section 3.2.2); both sets are projected
- *   on their global principal components (Section 3.2.1, diagonalized variant);
- *   the rows are split recursively: at each split the coordinate of highest
+ *   M = Q^T Q / n_q, keys -> K R_q with R_q a root of M; R_k a root of K_c^T K_c
+ *   with K_c the centred keys, queries -> r(q) = R_k q / |R_k q| (Section 3.2.2);
+ *   both sets are projected on their global principal components (Section 3.2.1,
+ *   diagonalized variant).  The roots are Cholesky factors F F^T = M (a pivot at
+ *   or below 1e-12 of the largest diagonal entry gives a zero column: the
+ *   counterpart of clamping non-positive eigenvalues): the principal-component
+ *   coordinates are the same for every root of the same matrix.  Component t is
+ *   oriented so that the entry of largest magnitude of column t of the map from
+ *   the original space to the coordinates (F E, E the principal directions) is
+ *   positive, which does not depend on the root either.
+ *   The rows are split recursively: at each split the coordinate of highest
  *   variance over min(d, |set|) evenly spaced rows of the set is chosen and the
  *   set is cut so that the lower side holds the multiple of c closest to half
  *   (ties in value go to the lower row index; half-way sizes go to the lower
@@ -222,15 +232,20 @@ int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const vo
  * as cluster_attention_fwd (inputs and outputs are still the caller's), but the
  * scratch is a fixed array of ca_static_scratch_bytes() = 32 MiB that is part
  * of the library image: every GPU that loads the library holds it until the
- * process exits.  The call allocates and frees nothing.
+ * process exits.  After the set-up described below a call allocates and frees
+ * nothing.
  *   - Limit: returns CA_ERR_WORKSPACE, enqueuing nothing, if the attention
  *     workspace that ca_workspace_bytes reports for `p` exceeds the array.
  *   - Set-up: the first call on each device looks up the array's device address
- *     (with that device current).  Make that first call before any stream
- *     capture is started.
+ *     (with that device current).  Under CUDA's lazy module loading that lookup
+ *     is also what loads the library's device code on that GPU and reserves the
+ *     32 MiB, so the first call can take longer, may synchronise the device, and
+ *     returns CA_ERR_CUDA if the memory cannot be had.  Make that first call
+ *     before any stream capture is started.
  *   - Sharing: every call on a device uses the same array, which keeps the
  *     previous call's contents; the call itself clears the status word and
- *     rewrites the centroid copies it needs.  Two calls whose kernels overlap on
+ *     rewrites the centroid copies it needs (the counter that
+ *     ca_attn_recomputed reports keeps adding up over the life of the process).  Two calls whose kernels overlap on
  *     the GPU (different streams) race on the array: serialise them.
  * ca_static_last_status reads the array's status word (synchronises the device).
  */
@@ -241,16 +256,25 @@ int cluster_attention_fwd_static(const ca_problem_t* p, const void* Qp, const vo
                                  const int32_t* perm_q, void* O, float* lse, void* stream);
 int ca_static_last_status(void);
 
-/* Reads the status word of a workspace (synchronises the device). */
+/* Reads the status word of a workspace as the last call on it left it (synchronises the device). */
 int ca_last_status(const void* ws);
 
 /* Statistics of an attention workspace (synchronises the device): how many query clusters the
- * second pass of cluster_attention_fwd has recomputed with the fp32 kernel since the workspace
- * was zero-filled.  The tensor-core kernel keeps the reference of its online softmax (Section
- * 3.1: exact softmax over the kept blocks) one half-step behind; a query cluster whose scores
- * climb by more than 2^96 within 64 keys leaves its range and is recomputed.  Returns the count
- * (>= 0), or minus an error code. */
+ * second pass of the attention calls on this workspace has recomputed with the fp32 kernel, summed
+ * over all calls since the caller zero-filled the workspace (the calls only add to the counter,
+ * the last word of the 256-byte status block).  The tensor-core kernel keeps the reference of its
+ * online softmax (Section 3.1: exact softmax over the kept blocks) one half-step behind; a query
+ * cluster whose scores climb by more than 2^96 within 64 keys leaves its range and is recomputed.
+ * Returns the count (>= 0), or minus an error code. */
 int ca_attn_recomputed(const void* ws);
+
+/* Diagnostic hook for tests of the failure path (process-wide, not thread-safe; affects the
+ * attention calls issued after it).  wait_limit_cycles: SM cycles after which a device-side wait
+ * of the tensor-core attention kernel gives up (<= 0 restores the default of about two seconds).
+ * skip_key_load: the loader leaves out the key rows of this half-step (64 keys) of every query
+ * tile, so that the waits for them run out: the kernel records CA_ERR_TIMEOUT, releases its tensor
+ * memory and returns, and the output of the call is undefined; -1 restores normal operation. */
+void ca_debug_attn_wait(long long wait_limit_cycles, int skip_key_load);
 
 /* Library version and the compute capability the kernels were built for. */
 const char* ca_version(void);

@@ -20,14 +20,16 @@ LIB_PATH = os.path.join(_HERE, "libclusterattn.so")
 
 CA_OK = 0
 CA_ERR_INVALID_ARG, CA_ERR_UNSUPPORTED, CA_ERR_WORKSPACE, CA_ERR_CUDA, CA_ERR_TIMEOUT = 1, 2, 3, 4, 5
+CA_ERR_BAD_INDEX = 6
 ERRORS = {1: "CA_ERR_INVALID_ARG", 2: "CA_ERR_UNSUPPORTED", 3: "CA_ERR_WORKSPACE", 4: "CA_ERR_CUDA",
-          5: "CA_ERR_TIMEOUT"}
+          5: "CA_ERR_TIMEOUT", 6: "CA_ERR_BAD_INDEX"}
 CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
 CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN = 1, 2, 4, 8
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_attn_recomputed", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
-           "ca_static_scratch_bytes", "ca_static_last_status")
+           "ca_static_scratch_bytes", "ca_static_last_status", "select_blocks_adaptive",
+           "cluster_attention_fwd_ragged", "ca_basic_workspace_bytes", "cluster_qk_basic", "ca_debug_attn_wait")
 
 
 class CaProblem(ctypes.Structure):
@@ -101,6 +103,8 @@ def load_library() -> ctypes.CDLL:
     lib.ca_static_scratch_bytes.restype = ctypes.c_size_t
     lib.ca_static_last_status.argtypes = []
     lib.ca_static_last_status.restype = ctypes.c_int
+    lib.ca_debug_attn_wait.argtypes = [ctypes.c_longlong, ctypes.c_int]
+    lib.ca_debug_attn_wait.restype = None
     _lib = lib
     return lib
 
@@ -336,8 +340,8 @@ class Plan:
         return {k: lib.ca_last_status(_ptr(v)) for k, v in self.ws.items()}
 
     def recomputed_clusters(self) -> int:
-        """Query clusters that the second pass of the attention call has recomputed with the fp32
-        kernel since this plan was made (ca_attn_recomputed of the C library)."""
+        """Query clusters that the second pass of the attention calls on this plan has recomputed
+        with the fp32 kernel, summed over all calls since the plan was made (ca_attn_recomputed)."""
         lib = load_library()
         n = lib.ca_attn_recomputed(_ptr(self.ws["attn"]))
         if n < 0:

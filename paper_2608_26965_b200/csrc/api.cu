@@ -33,7 +33,7 @@ int check_problem(const ca_problem_t* p) {
 struct ClusterWs {
   int* status;
   float *partial, *partial2;           // chunk sums of the Gram kernels, one buffer per stream
-  double *gramQ, *sumQ, *gramK, *sumK, *metric, *roots, *tmp, *cov, *gramQp, *sumQp, *basis, *WK;
+  double *gramQ, *sumQ, *gramK, *sumK, *roots, *gramQp, *sumQp;
   float *roots32, *basis32, *WK32, *biasK, *biasQ;
   float *Qprime, *Yq, *Yk, *Ytq, *Ytk;
   __nv_bfloat16 *wt_hi, *wt_lo, *wt2_hi, *wt2_lo;
@@ -66,13 +66,8 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
     w.partial2 = c.take<float>(P * nchunks * (DD + D));
     w.gramQ = c.take<double>(P * DD);  w.sumQ = c.take<double>(P * D);
     w.gramK = c.take<double>(P * DD);  w.sumK = c.take<double>(P * D);
-    w.metric = c.take<double>(2 * P * DD);
     w.roots = c.take<double>(2 * P * DD);
-    w.tmp = c.take<double>(P * DD);
-    w.cov = c.take<double>(2 * P * DD);
     w.gramQp = c.take<double>(P * DD); w.sumQp = c.take<double>(P * D);
-    w.basis = c.take<double>(2 * P * DD);
-    w.WK = c.take<double>(P * DD);
     w.roots32 = c.take<float>(2 * P * DD);
     w.basis32 = c.take<float>(2 * P * DD);
     w.WK32 = c.take<float>(P * DD);
@@ -100,8 +95,8 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
 // The query side and the key side of cluster_qk are independent once the two factors exist.  The
 // query side runs on a second stream that forks from the caller's stream and joins it again
 // before the call returns (events only: nothing waits on the host, and a stream capture of the
-// caller's stream picks the side stream up as a parallel branch).  One stream and two events per
-// device, created at the first call on that device.
+// caller's stream picks the side stream up as a parallel branch).  One stream and three events
+// (fork, C_K ready, join) per device, created at the first call on that device.
 struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, mid = nullptr, join = nullptr;
@@ -171,26 +166,21 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     float* yk_out = Yk ? Yk : w.Yk;
     // bf16 storage runs the O(n d^2) passes on the tensor cores; fp32 storage on the CUDA cores
     const bool tc = p->dtype == CA_DTYPE_BF16;
-    // d = 64: the one CTA per head that computes the bias also lays the weights out for the
-    // tensor-core projection (one launch less on each side); at d = 128 that is too much for one CTA
-    const bool fold = tc && D == 64;
     __nv_bfloat16* qp_hi = reinterpret_cast<__nv_bfloat16*>(w.Qprime);          // r(q) as bf16 hi + lo parts
     __nv_bfloat16* qp_lo = qp_hi + (size_t)P * p->n_q * D;
-    // metric matrices (Section 3.2.2) and their factors F_q F_q^T = M, F_k F_k^T = C_K (they stand
-    // in for the symmetric roots: any factor yields the same principal-component coordinates).  The
+    // Factors F_q F_q^T = M = Q^T Q / n_q and F_k F_k^T = C_K (Section 3.2.2; they stand in for the
+    // symmetric roots: any factor yields the same principal-component coordinates).  The
     // un-normalised query representation (Appendix B.1) takes the root of K_c^T K_c / n_k, the
-    // normalised one is indifferent to the factor and keeps the scatter matrix as it is.
-    // M and F_q come from Q on the caller's stream and lead into the key side; C_K and F_k come from
-    // K on the side stream and lead into the query side: the fork is at the very start, and the
-    // key side only waits for C_K (event `mid`).
-    double* M = w.metric;
-    double* CK = w.metric + (size_t)P * DD;
+    // normalised one is indifferent to the scale and keeps the scatter matrix as it is.
+    // F_q comes from Q on the caller's stream and leads into the key side; F_k comes from K on the
+    // side stream and leads into the query side: the fork is at the very start, and the key side
+    // only waits for the Gram matrix and column sums of K (event `mid`), from which its
+    // principal-component kernel forms C_K itself.
     const bool unnormalized = (p->flags & CA_QUERY_UNNORMALIZED) != 0;
     const double ck_scale = unnormalized ? 1.0 / (double)p->n_k : 1.0;
-    double* Rq = w.roots;
-    const float* Rk32 = w.roots32 + (size_t)P * DD;
-    double* covK = w.cov;
-    double* covQ = w.cov + (size_t)P * DD;
+    double* Fq = w.roots;
+    double* Fk = w.roots + (size_t)P * DD;
+    const float* Fk32 = w.roots32 + (size_t)P * DD;
     SideStream* side = side_stream();
     if (!side) return CA_ERR_CUDA;
     cudaStream_t sq = side->stream;
@@ -203,29 +193,35 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
       CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
       CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial2, w.gramK, w.sumK, sq));
     }
-    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, M, nullptr, st));
-    CA_TRY(launch_cholesky_factor(M, P, D, w.roots, w.roots32, st));
-    CA_TRY(launch_metric(w.gramQ, w.gramK, w.sumK, P, D, p->n_q, p->n_k, ck_scale, nullptr, CK, sq));
     CA_RETURN_IF_CUDA(cudaEventRecord(side->mid, sq));
-    CA_TRY(launch_cholesky_factor(CK, P, D, w.roots + (size_t)P * DD, w.roots32 + (size_t)P * DD, sq));
+    CA_TRY(launch_cholesky_factor(w.gramQ, nullptr, 1.0, 1.0 / (double)p->n_q, P, D, Fq, w.roots32, nullptr, nullptr, st));
+    CA_TRY(launch_cholesky_factor(w.gramK, w.sumK, (double)p->n_k, ck_scale, P, D, Fk, w.roots32 + (size_t)P * DD,
+                                  tc ? w.wt2_hi : nullptr, tc ? w.wt2_lo : nullptr, sq));
     // ---- query side (side stream)
-    // query representation r(q) = F_k^T q / |F_k^T q|, its covariance, its principal components,
-    // the coordinates Y = (r(q) - mean) E_Q
-    const float* EQ32 = w.basis32 + (size_t)P * DD;
+    // query representation r(q) = F_k^T q / |F_k^T q|, its covariance and principal components E_Q
+    // (one kernel), the coordinates Y = (r(q) - mean) E_Q
+    float* EQ32 = w.basis32 + (size_t)P * DD;
     if (tc) {
-      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
-                                 w.wt2_hi, w.wt2_lo, w.status, sq));
+      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
+                                 w.wt2_hi, w.wt2_lo, w.status, sq, nullptr, true));
       CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, w.status, sq));
     } else {
-      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Rk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
+      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
       CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, sq));
     }
-    CA_TRY(launch_covariance(w.gramQp, w.sumQp, P, D, p->n_q, covQ, sq));
-    CA_TRY(launch_eigh(covQ, P, D, w.basis + (size_t)P * DD, w.basis32 + (size_t)P * DD, nullptr, sq));
-    CA_TRY(launch_bias(w.sumQp, EQ32, P, D, p->n_q, w.biasQ, sq, fold ? w.wt2_hi : nullptr, fold ? w.wt2_lo : nullptr));
+    {
+      PcaArgs a{};
+      a.mode = kPcaQueries;
+      a.gram = w.gramQp; a.sum = w.sumQp; a.n = (double)p->n_q;
+      a.lift = Fk; a.out_lifted = 0;
+      a.mean_sum = w.sumQp; a.mean_n = (double)p->n_q;
+      a.W32 = EQ32; a.bias = w.biasQ;
+      a.wt_hi = tc ? w.wt2_hi : nullptr; a.wt_lo = tc ? w.wt2_lo : nullptr;
+      CA_TRY(launch_pca(a, P, D, sq));
+    }
     if (tc) {
       CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
-                                 w.wt2_lo, w.status, sq, w.Ytq, fold));
+                                 w.wt2_lo, w.status, sq, w.Ytq, true));
     } else {
       CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
     }
@@ -234,16 +230,23 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, sq));
     CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
     // ---- key side on the caller's stream: covariance of the transformed keys K F_q
-    // (F_q^T C_K F_q / n_k, d x d algebra), its principal components, Y = (K - kbar) F_q E_K
+    // (F_q^T C_K F_q / n_k, d x d algebra), its principal components E_K and the projection
+    // W = F_q E_K with its bias in one kernel; Y = (K - kbar) W
     CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->mid, 0));
-    CA_TRY(launch_small_matmul(Rq, CK, P, D, 1.0, 1, w.tmp, nullptr, st));
-    CA_TRY(launch_small_matmul(w.tmp, Rq, P, D, unnormalized ? 1.0 : 1.0 / (double)p->n_k, 0, covK, nullptr, st));
-    CA_TRY(launch_eigh(covK, P, D, w.basis, w.basis32, nullptr, st));
-    CA_TRY(launch_small_matmul(Rq, w.basis, P, D, 1.0, 0, w.WK, w.WK32, st));
-    CA_TRY(launch_bias(w.sumK, w.WK32, P, D, p->n_k, w.biasK, st, fold ? w.wt_hi : nullptr, fold ? w.wt_lo : nullptr));
+    {
+      PcaArgs a{};
+      a.mode = kPcaKeys;
+      a.gram = w.gramK; a.sum = w.sumK; a.n = (double)p->n_k; a.c_scale = ck_scale;
+      a.alpha = unnormalized ? 1.0 : 1.0 / (double)p->n_k;
+      a.lift = Fq; a.out_lifted = 1;
+      a.mean_sum = w.sumK; a.mean_n = (double)p->n_k;
+      a.W32 = w.WK32; a.bias = w.biasK;
+      a.wt_hi = tc ? w.wt_hi : nullptr; a.wt_lo = tc ? w.wt_lo : nullptr;
+      CA_TRY(launch_pca(a, P, D, st));
+    }
     if (tc) {
       CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
-                                 w.wt_lo, w.status, st, w.Ytk, fold));
+                                 w.wt_lo, w.status, st, w.Ytk, true));
     } else {
       CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
     }
@@ -290,12 +293,13 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
   const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusClearBytes, st));
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
   if (tensor_cores)
     return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, nullptr, p->keep, perm_q, scale, O, lse,
                           ws, st);
-  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, nullptr, p->keep, perm_q, scale, O, lse, st);
+  return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, nullptr, p->keep, perm_q, scale, O, lse,
+                         static_cast<int*>(ws), st);
 }
 
 int select_blocks_adaptive(const ca_problem_t* p, const float* cq, const float* ck, const int32_t* count_k,
@@ -331,13 +335,13 @@ int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const vo
   const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusBytes, st));
+  CA_RETURN_IF_CUDA(cudaMemsetAsync(ws, 0, kStatusClearBytes, st));
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
   if (tensor_cores)
     return launch_attn_tc(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale,
                           O, lse, ws, st);
   return launch_attn_ref(*p, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O,
-                         lse, st);
+                         lse, static_cast<int*>(ws), st);
 }
 
 namespace {
@@ -429,9 +433,13 @@ int ca_attn_recomputed(const void* ws) {
   if (!ws) return -CA_ERR_INVALID_ARG;
   int count = 0;
   if (cudaDeviceSynchronize() != cudaSuccess) return -CA_ERR_CUDA;
-  if (cudaMemcpy(&count, static_cast<const int*>(ws) + 1, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+  if (cudaMemcpy(&count, static_cast<const int*>(ws) + kRecomputedWord, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
     return -CA_ERR_CUDA;
   return count;
+}
+
+void ca_debug_attn_wait(long long wait_limit_cycles, int skip_key_load) {
+  attn_tc_set_debug(wait_limit_cycles, skip_key_load);
 }
 
 int ca_last_status(const void* ws) {

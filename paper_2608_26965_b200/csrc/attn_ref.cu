@@ -20,7 +20,8 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
                 const int32_t* __restrict__ keep_count, int list_stride,
                 const int32_t* __restrict__ perm_q, int n_q, int n_k, int c_q, int c_k, int keep_all,
                 int compensate, float scale, T* __restrict__ O, float* __restrict__ lse,
-                const int32_t* __restrict__ redo, int redo_tiles, int* __restrict__ redo_count) {
+                int* __restrict__ status, const int32_t* __restrict__ redo, int redo_tiles,
+                int* __restrict__ redo_count) {
   constexpr int LD = D + 1;
   constexpr int NC = D / 8;              // output columns per thread
   extern __shared__ float smem[];
@@ -52,13 +53,24 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
   const T* Kh = Kp + (size_t)p * n_kc * (size_t)c_k * D;
   const T* Vh = Vp + (size_t)p * n_kc * (size_t)c_k * D;
   const int32_t* sel = block_idx + ((size_t)p * n_qc + qc) * list_stride;
-  const int keep = keep_count ? keep_count[(size_t)p * n_qc + qc] : keep_all;   // ragged lists carry their length
+  int keep = keep_count ? keep_count[(size_t)p * n_qc + qc] : keep_all;   // ragged lists carry their length
+  // indices from the caller are range-checked before use: a bad one sets CA_ERR_BAD_INDEX (6) in the
+  // status word and is skipped (a list length is clamped to its row, a cluster that does not exist
+  // is left out, a row of O that does not exist is not written)
+  if (keep < 0 || keep > list_stride) {
+    if (tid == 0) atomicCAS(status, 0, 6);
+    keep = keep < 0 ? 0 : list_stride;
+  }
   const int32_t* cnt = count_k + (size_t)p * n_kc;
 
   const int words = (n_kc + 31) / 32;
   for (int w = tid; w < words; w += kRefThreads) selected[w] = 0u;
   __syncthreads();
-  for (int t = tid; t < keep; t += kRefThreads) atomicOr(&selected[sel[t] >> 5], 1u << (sel[t] & 31));
+  for (int t = tid; t < keep; t += kRefThreads) {
+    const int j = sel[t];
+    if (j < 0 || j >= n_kc) atomicCAS(status, 0, 6);
+    else atomicOr(&selected[j >> 5], 1u << (j & 31));
+  }
 
   for (int r0 = r0_first; r0 < r0_end; r0 += kRefQR) {
     __syncthreads();                       // the previous tile's readers are done with the staged rows
@@ -122,7 +134,8 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
     // selected clusters: every member key
     for (int t = 0; t < keep; ++t) {
       const int j = sel[t];
-      const int members = cnt[j];
+      if (j < 0 || j >= n_kc) continue;                  // flagged above
+      const int members = min(max(cnt[j], 0), c_k);
       for (int t0 = 0; t0 < members; t0 += kRefKT) {
         __syncthreads();
         for (int e = tid; e < kRefKT * D; e += kRefThreads) {
@@ -162,11 +175,17 @@ attn_ref_kernel(const T* __restrict__ Qp, const T* __restrict__ Kp, const T* __r
     const int pos = qc * c_q + r0 + row;
     if (r0 + row < c_q && pos < n_q) {
       const int orig = perm_q[(size_t)p * n_q + pos];
-      const float inv = 1.f / l_run;
-      T* out = O + ((size_t)p * n_q + orig) * D;
+      if (orig < 0 || orig >= n_q) {
+        atomicCAS(status, 0, 6);
+      } else {
+        // a row without a single live entry (an empty list without compensation): zeros, lse = -inf
+        const bool empty = !(l_run > 0.f);
+        const float inv = empty ? 0.f : 1.f / l_run;
+        T* out = O + ((size_t)p * n_q + orig) * D;
 #pragma unroll
-      for (int i = 0; i < NC; ++i) out[sub + 8 * i] = from_f32<T>(acc[i] * inv);
-      if (lse && sub == 0) lse[(size_t)p * n_q + orig] = m_run + logf(l_run);
+        for (int i = 0; i < NC; ++i) out[sub + 8 * i] = from_f32<T>(acc[i] * inv);
+        if (lse && sub == 0) lse[(size_t)p * n_q + orig] = empty ? -INFINITY : m_run + logf(l_run);
+      }
     }
   }   // tiles of the cluster
 }
@@ -175,7 +194,8 @@ template <typename T>
 static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* Vp, const float* ck,
                     const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, T* O,
-                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles, int* redo_count) {
+                    float* lse, int* status, cudaStream_t st, const int32_t* redo, int redo_tiles,
+                    int* redo_count) {
   const int P = pr.batch * pr.heads, D = pr.head_dim;
   const int n_qc = ceil_div(pr.n_q, pr.cluster_q), n_kc = ceil_div(pr.n_k, pr.cluster_k);
   const int tiles = ceil_div(pr.cluster_q, kRefQR);
@@ -187,13 +207,13 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
                                         pr.n_q, pr.n_k,
-                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles, redo_count);
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, status, redo, redo_tiles, redo_count);
   } else {
     auto k = attn_ref_kernel<T, 128>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     k<<<grid, kRefThreads, smem, st>>>(Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q,
                                         pr.n_q, pr.n_k,
-                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, redo, redo_tiles, redo_count);
+                                        pr.cluster_q, pr.cluster_k, pr.keep, pr.compensate, scale, O, lse, status, redo, redo_tiles, redo_count);
   }
   CA_LAUNCH_CHECK();
   return CA_OK;
@@ -202,15 +222,16 @@ static int launch_t(const ca_problem_t& pr, const T* Qp, const T* Kp, const T* V
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
-                    float* lse, cudaStream_t st, const int32_t* redo, int redo_tiles, int* redo_count) {
+                    float* lse, int* status, cudaStream_t st, const int32_t* redo, int redo_tiles,
+                    int* redo_count) {
   if (pr.dtype == CA_DTYPE_BF16)
     return launch_t(pr, static_cast<const __nv_bfloat16*>(Qp), static_cast<const __nv_bfloat16*>(Kp),
                     static_cast<const __nv_bfloat16*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride,
                     perm_q, scale,
-                    static_cast<__nv_bfloat16*>(O), lse, st, redo, redo_tiles, redo_count);
+                    static_cast<__nv_bfloat16*>(O), lse, status, st, redo, redo_tiles, redo_count);
   return launch_t(pr, static_cast<const float*>(Qp), static_cast<const float*>(Kp),
                   static_cast<const float*>(Vp), ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale,
-                  static_cast<float*>(O), lse, st, redo, redo_tiles, redo_count);
+                  static_cast<float*>(O), lse, status, st, redo, redo_tiles, redo_count);
 }
 
 }  // namespace ca

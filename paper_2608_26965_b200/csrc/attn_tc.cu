@@ -2,29 +2,36 @@
 // cores (eq. 2 over the selected clusters; Appendix A: an excluded cluster
 // enters through its centroid key/value with weight |c| exp(q . kbar / sqrt(d))).
 //
-// One CTA per tile of 128 query rows (one query cluster, or half of a 256-row
-// one); two CTAs share an SM.  Key/value tiles of 128 rows stream through shared
-// memory by TMA (128-byte swizzle, 64-column panels).  The keys are consumed in
-// half-steps of 64, alternating between two 64-column score buffers in tensor
-// memory, so that the tensor core works on one half-step while the softmax
-// warps work on the other:
-//     S_b = Q K_h^T        tcgen05.mma, K from shared memory; Q from shared memory (d = 128) or from a
-//                          copy in tensor memory (d = 64)
+// One CTA per tile of 128 query rows (one query cluster, half of a 256-row one,
+// or a 64-row one in a half-filled tile).  Per CTA the half-steps of 64 keys form
+// one dependent chain, so what counts is the number of chains per SM: at d = 64 a
+// CTA holds one 64-column score buffer and 64 output columns in tensor memory and
+// four CTAs share an SM; at d = 128 two score buffers and 128 output columns, two
+// CTAs per SM (TcCfg).  Key and value rows stream through shared memory by TMA in
+// slots of 64 rows (128-byte swizzle, 64-column panels), loaded in the order the
+// tensor core consumes them:
+//     S_b = Q K_h^T        tcgen05.mma, Q and K from shared memory (K-major)
 //     P_b = exp2(S_b c - m) four softmax warps, one query row per thread; P is
-//                          written back over S_b as packed bf16
-//     O  += P_b V_h        tcgen05.mma, P from tensor memory, V from shared memory (MN-major); at
-//                          d = 64 V is followed by 16 columns of ones, which makes the row sums of P
-// issued as S(0) S(1) | PV(0) S(2) | PV(1) S(3) | ...  The running maximum is only
-// raised when a half-step exceeds it by 2^8; the softmax warps then rescale O in
-// tensor memory themselves after waiting for the one product that can still be
-// in flight.  After the selected clusters the key centroids are streamed as
-// extra keys, 64 per half-step: their tile holds bf16 hi parts in rows 0-63 and
-// lo parts in rows 64-127, accumulated by two products so the centroid logits
-// keep fp32-level accuracy; logit bias ln|c|, selected clusters masked; values are
-// the value centroids.  Block lists may be ragged (a length per query cluster).
-// Warp 0 issues TMA, warp 1 issues MMAs (all lanes run the loop, one elected lane
-// issues), warps 2-5 do the softmax and the epilogue (rows scattered back to the
-// original order).
+//                          written back over S_b as packed bf16; row sums in fp32
+//                          registers
+//     O  += P_b V_h        tcgen05.mma, P from tensor memory, V from shared memory (MN-major)
+// issued as S(0) [S(1)] | PV(0) S(NBUF) | PV(1) S(NBUF + 1) | ...  The softmax keeps
+// a reference m per row instead of the exact running maximum: it is measured on a
+// row's first half-step, afterwards gathered with the exponentials and raised one
+// half-step late (by an integer, when a half-step exceeded it by 2^8), the softmax
+// warps then rescale O in tensor memory themselves after waiting for the one
+// product that can still be in flight; a climb beyond 2^96 inside one half-step
+// marks the tile for the second pass of the fp32 kernel.  After the selected
+// clusters the key centroids are streamed as extra keys, 64 per half-step: their
+// tile holds bf16 hi parts in rows 0-63 and lo parts in rows 64-127, accumulated
+// by two products so the centroid logits keep fp32-level accuracy; logit bias
+// ln|c|, selected clusters masked; values are the value centroids.  Block lists
+// may be ragged (a length per query cluster).  Warp 0 issues TMA, warp 1 issues
+// MMAs (all lanes run the loop, one elected lane issues), warps 2-5 do the softmax
+// and the epilogue (rows scattered back to the original order).
+// Indices that come from the caller (block lists, list lengths, perm_q) are range-
+// checked before use: a bad one sets CA_ERR_BAD_INDEX in the status word and the
+// access is skipped (the cluster is masked, the row is not written).
 #include "kernels.h"
 #include "tc_ptx.cuh"
 
@@ -86,7 +93,11 @@ struct TcParams {
   int32_t* redo;                  // [B*H, n_qc, 2] per CTA: scores left the range of the fast softmax
   int n_q, n_k, c_q, c_k, keep, list_stride, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
   float scale_log2;
+  long long wait_limit;           // SM cycles after which a barrier wait gives up (CA_ERR_TIMEOUT)
+  int skip_key_load;              // diagnostic hook: the loader leaves out the keys of this half-step (-1: none)
 };
+
+constexpr int kErrBadIndex = 6;   // CA_ERR_BAD_INDEX
 
 // key rows of the selected clusters are consumed in tiles of 128 rows
 __host__ __device__ inline int selected_tiles(int keep, int c_k) {
@@ -128,7 +139,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const int q_rows = prm.c_q >= kTile ? kTile : prm.c_q;
   const int qc = blockIdx.x / tiles_per_qc, half = blockIdx.x % tiles_per_qc;
   const int32_t* sel = prm.block_idx + ((size_t)p * prm.n_qc + qc) * prm.list_stride;
-  const int keep = prm.keep_count ? prm.keep_count[(size_t)p * prm.n_qc + qc] : prm.keep;
+  int keep = prm.keep_count ? prm.keep_count[(size_t)p * prm.n_qc + qc] : prm.keep;
+  if (keep < 0 || keep > prm.list_stride) {            // a list length that does not fit its row
+    if (tid == 0) atomicCAS(prm.status, 0, kErrBadIndex);
+    keep = keep < 0 ? 0 : prm.list_stride;
+  }
   const int sel_tiles = selected_tiles(keep, prm.c_k);
   const int cen_tiles = prm.compensate ? prm.cen_tiles : 0;
   const int steps = 2 * sel_tiles + cen_tiles;         // half-steps of 64 keys
@@ -183,14 +198,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       auto load_selected = [&](uint32_t dst, const CUtensorMap* map, int u, uint32_t bar) {
         if (prm.c_k >= kHalf) {
           const int pos = u * kHalf;                       // position in the concatenated selected rows
-          const int j = sel[min(pos / prm.c_k, keep - 1)];     // a filler half-step repeats the last cluster (masked)
+          int j = sel[min(pos / prm.c_k, keep - 1)];     // a filler half-step repeats the last cluster (masked)
+          j = min(max(j, 0), prm.n_kc - 1);                // out-of-range entries are flagged and masked by the softmax warps
           load_rows(dst, map, (p * prm.n_kc + j) * prm.c_k + pos % prm.c_k, bar);
         } else {
           const int per = kHalf / prm.c_k;
           for (int x = 0; x < per; ++x) {
             int e = u * per + x;
             if (e >= keep) e = keep - 1;                   // filler rows, masked by the softmax
-            const int j = sel[e];
+            const int j = min(max(sel[e], 0), prm.n_kc - 1);
             for (int pn = 0; pn < C::PANELS; ++pn)
               tma_load_2d(dst + pn * C::HALF_PANEL_BYTES + x * prm.c_k * 128, map, pn * 64,
                           (p * prm.n_kc + j) * prm.c_k, bar);
@@ -206,9 +222,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           const bool centroid = i >= 2 * sel_tiles;
           const int parts = centroid ? 2 : 1;
           const int w = i - (centroid ? C::K_LEAD_CEN : C::K_LEAD);
-          if (w >= 0) ok = mbar_wait_relaxed(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          if (w >= 0) ok = mbar_wait_relaxed(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit);
           for (int g = 0; g < parts && ok; ++g) {
             const int kc = kslot_of(i) + g, slot = kc % C::NK;
+            if (i == prm.skip_key_load) continue;          // diagnostic: this slot never fills, its waiters time out
             mbar_expect_tx(b_k_full(slot), C::HALF_BYTES);
             const uint32_t dst = s_k + slot * C::HALF_BYTES;
             if (!centroid) load_selected(dst, &tm_k, i, b_k_full(slot));
@@ -219,7 +236,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (j >= 0 && ok) {
           const int slot = j % C::NV;
           const int w = j - C::NV;
-          if (w >= 0) ok = mbar_wait_relaxed(b_pv_done(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status);
+          if (w >= 0) ok = mbar_wait_relaxed(b_pv_done(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit);
           if (!ok) break;
           mbar_expect_tx(b_v_full(slot), C::HALF_BYTES);
           const uint32_t dst = s_v + slot * C::HALF_BYTES;
@@ -235,7 +252,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     {
       constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
-      bool ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status));
+      bool ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status, prm.wait_limit));
       // descriptors differ from a base one only in the start-address field (units of 16 bytes):
       // the base descriptors are built once, the per-instruction part is an addition
       const uint64_t q_desc0 = smem_desc_sw128(s_q, 16, 1024);
@@ -250,7 +267,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         bool got = true;
         for (int g = 0; g < parts && got; ++g) {
           const int kc = kslot_of(un) + g;
-          got = __all_sync(0xffffffffu, mbar_wait(b_k_full(kc % C::NK), (kc / C::NK) & 1, abort_flag, prm.status));
+          got = __all_sync(0xffffffffu, mbar_wait(b_k_full(kc % C::NK), (kc / C::NK) & 1, abort_flag, prm.status, prm.wait_limit));
         }
         return got;
       };
@@ -278,14 +295,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       for (int u = 0; u < steps && ok; ++u) {
         const int slot = u % C::NV, un = u + C::NBUF;
-        ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(slot), (u / C::NV) & 1, abort_flag, prm.status));
+        ok = __all_sync(0xffffffffu, mbar_wait(b_v_full(slot), (u / C::NV) & 1, abort_flag, prm.status, prm.wait_limit));
         if (ok && un < steps) ok = wait_keys(un);
         // V is MN-major: 16 key rows (2048 bytes) per instruction; panels along d
         const uint64_t vd = v_desc0 + ((slot * C::HALF_BYTES) >> 4);
         const uint32_t p_cols = tmem_s + (u % C::NBUF) * kHalf;
         const uint32_t s_cols = tmem_s + (un % C::NBUF) * kHalf, s_bar = b_s_full(un % C::NBAR), pv_bar = b_pv_done(u % C::NBAR);
         const int s_kc0 = kslot_of(un), s_parts = un >= steps ? 0 : (un >= 2 * sel_tiles ? 2 : 1);
-        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
+        if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
         if (!ok) break;
         tc_fence_after();
         if (elect_one()) {
@@ -310,14 +327,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     asm volatile("bar.sync 1, 128;" ::: "memory");
     for (int e = st; e < keep; e += 128) {
       const int j = sel[e];
-      members_of[e] = (uint16_t)min(cnt[j], prm.c_k);
+      if (j < 0 || j >= prm.n_kc) {                        // not a key cluster: flagged, all of its columns masked
+        atomicCAS(prm.status, 0, kErrBadIndex);
+        members_of[e] = 0;
+        continue;
+      }
+      members_of[e] = (uint16_t)min(max(cnt[j], 0), prm.c_k);
       if (prm.compensate) atomicOr(&bitmap[j >> 5], 1u << (j & 31));
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
 
     if (C::Q_IN_TMEM) {
       // this thread's query row: eight 16-byte chunks, stored at chunk position c ^ (row & 7)
-      bool q_ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status));
+      bool q_ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status, prm.wait_limit));
       uint32_t qw[32];
 #pragma unroll
       for (int c = 0; c < 8; ++c) {
@@ -371,7 +393,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
 
-      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status));
+      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
       if (!ok) break;
       tc_fence_after();
       if (quarter * 32 >= q_rows) {          // this warp's rows are padding of a 64-row query cluster
@@ -443,7 +465,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         l_run *= alpha;
         if (u > 0) {
           // products complete in the order of their issue: once P V (u-1) is complete, all earlier are
-          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
           if (!ok) break;
           tc_fence_after();
 #pragma unroll 1
@@ -519,13 +541,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
 
     // epilogue: O / l, rows back to their original positions
-    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_o_done, 0, abort_flag, prm.status));
+    if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_o_done, 0, abort_flag, prm.status, prm.wait_limit));
     tc_fence_after();
     if (ok) {                                          // warp-uniform: TMEM loads are warp-collective
       const int pos = qc * prm.c_q + half * kTile + row;
-      const bool live = row < q_rows && pos < prm.n_q;  // rows of the padding are not written
-      const int orig = live ? prm.perm_q[(size_t)p * prm.n_q + pos] : 0;
-      const float inv = 1.f / l_run;
+      bool live = row < q_rows && pos < prm.n_q;        // rows of the padding are not written
+      int orig = live ? prm.perm_q[(size_t)p * prm.n_q + pos] : 0;
+      if (orig < 0 || orig >= prm.n_q) {                // not a row of O: flagged, nothing written
+        atomicCAS(prm.status, 0, kErrBadIndex);
+        live = false;
+        orig = 0;
+      }
+      // a row without a single live entry (an empty list without compensation): zeros, lse = -inf
+      const bool empty = !(l_run > 0.f);
+      const float inv = empty ? 0.f : 1.f / l_run;
       __nv_bfloat16* out = prm.O + ((size_t)p * prm.n_q + orig) * D;
 #pragma unroll
       for (int c4 = 0; c4 < D / 32; ++c4) {
@@ -541,11 +570,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
             w.y = pack_bf16x2(__uint_as_float(o[8 * v + 2]) * inv, __uint_as_float(o[8 * v + 3]) * inv);
             w.z = pack_bf16x2(__uint_as_float(o[8 * v + 4]) * inv, __uint_as_float(o[8 * v + 5]) * inv);
             w.w = pack_bf16x2(__uint_as_float(o[8 * v + 6]) * inv, __uint_as_float(o[8 * v + 7]) * inv);
+            if (empty) w = make_uint4(0u, 0u, 0u, 0u);   // no product was issued: the accumulator holds no data
             dst[v] = w;
           }
         }
       }
-      if (live && prm.lse) prm.lse[(size_t)p * prm.n_q + orig] = (m_ref + log2f(l_run)) * 0.6931471805599453f;
+      if (live && prm.lse)
+        prm.lse[(size_t)p * prm.n_q + orig] = empty ? -INFINITY : (m_ref + log2f(l_run)) * 0.6931471805599453f;
     }
   }
 
@@ -642,6 +673,15 @@ static int launch_tc_d(const CUtensorMap* maps, const TcParams& prm, dim3 grid, 
   return CA_OK;
 }
 
+namespace {
+long long g_wait_limit = kWaitLimitCycles;   // host-side settings of the diagnostic hook
+int g_skip_key_load = -1;
+}  // namespace
+void attn_tc_set_debug(long long wait_limit_cycles, int skip_key_load) {
+  g_wait_limit = wait_limit_cycles > 0 ? wait_limit_cycles : kWaitLimitCycles;
+  g_skip_key_load = skip_key_load;
+}
+
 int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp, const float* ck,
                    const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* keep_count,
                    int list_stride, const int32_t* perm_q, float scale, void* O, float* lse, void* ws,
@@ -675,13 +715,15 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   prm.n_qc = n_qc; prm.n_kc = n_kc; prm.cen_tiles = cen_tiles; prm.compensate = pr.compensate;
   prm.bitmap_words = (cen_tiles * kHalf + 31) / 32;
   prm.scale_log2 = scale * 1.4426950408889634f;
+  prm.wait_limit = g_wait_limit;
+  prm.skip_key_load = g_skip_key_load;
   dim3 grid(n_qc * (pr.cluster_q >= kTile ? pr.cluster_q / kTile : 1), P);
   const int rc = D == 64 ? launch_tc_d<64>(maps, prm, grid, st) : launch_tc_d<128>(maps, prm, grid, st);
   if (rc != CA_OK) return rc;
   // second pass: query tiles whose scores left the range of the fast softmax (a climb of more than
   // 2^96 within 64 keys) are recomputed by the fp32 kernel; its CTAs return at once for the others
   return launch_attn_ref(pr, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O, lse,
-                         st, redo, (int)grid.x / n_qc, status + 1);
+                         status, st, redo, (int)grid.x / n_qc, status + kRecomputedWord);
 }
 
 }  // namespace ca

@@ -8,8 +8,12 @@
 
 namespace ca {
 
-// Status block at the start of every workspace.
+// Status block at the start of every workspace: word 0 is the status code (CA_OK or the first
+// error a kernel recorded); every call clears the first kStatusClearBytes on its stream.  The last
+// word is a counter that calls only add to (query clusters recomputed by the second attention pass).
 constexpr size_t kStatusBytes = 256;
+constexpr size_t kStatusClearBytes = 252;
+constexpr int kRecomputedWord = 63;
 
 extern unsigned long long g_kernel_launches;   // kernels enqueued since the library was loaded
 

@@ -1,27 +1,40 @@
-// Batched symmetric eigendecomposition of d x d matrices (d = 64, 128), one CTA
-// per matrix: Householder reduction to tridiagonal form, then the implicit-shift
-// QL iteration on the tridiagonal matrix (principal-component bases of
-// Section 3.2.1).  Working precision float32: the bases only feed fp32 split
-// coordinates.
+// Principal components of the transformed rows (Section 3.2.1, diagonalized
+// variant), one CTA per head and side: builds the d x d covariance, decomposes
+// it, and writes the projection that the split coordinates are computed with.
 //
-// Phase 1 (all 8d threads, two barriers per reflector): for k = 0 .. d-3 the
-// reflector H_k = I - beta v v^T annihilates A[k+2.., k]; the trailing block is
-// updated as A - v w^T - w v^T with p = beta A v, w = p - (beta/2)(v.p) v, and
-// the transposed accumulated transform Qt <- H_k Qt is updated in the same two
-// stages.  Thread (r, q) = (tid / 8, tid % 8) keeps entries 4 (q + 8 t) + c of
-// row r of A and of column r of Qt in registers for the whole phase (the loops
-// are bound by instruction issue and latency, not by arithmetic); the eight
-// owners of row k+1 build the next reflector right after their update, inside
-// their warp, so no third barrier is needed.
+// Prologue.  Keys: the transformed keys K F (F F^T = M the query metric, Section
+// 3.2.2) have covariance F^T C_K F / n_k with C_K the centred scatter of the keys,
+// formed here from the Gram matrix and the column sums of K (two d x d x d
+// products in shared memory, no pass over the data).  Queries: the covariance of
+// the representation r(q) from its Gram matrix and column sums.
 //
-// Phase 2: warp 0 runs the QL iteration on (diag, sub-diag) -- the search for a
-// negligible sub-diagonal entry uses all lanes, the rotation chase is one
-// dependent chain on lane 0 -- and hands each chase's rotations through a
-// double-buffered list to d consumer threads, which apply them to the rows of
-// Qt (thread t owns column t), pipelined with the next chase by named barriers.
+// Decomposition (d = 64, 128; float32: the bases only feed fp32 coordinates):
+// Householder reduction to tridiagonal form, then the implicit-shift QL
+// iteration.  Phase 1 (all 8d threads, two barriers per reflector): for
+// k = 0 .. d-3 the reflector H_k = I - beta v v^T annihilates A[k+2.., k]; the
+// trailing block is updated as A - v w^T - w v^T with p = beta A v,
+// w = p - (beta/2)(v.p) v, and the transposed accumulated transform
+// Qt <- H_k Qt is updated in the same two stages.  Thread (r, q) =
+// (tid / 8, tid % 8) keeps entries 4 (q + 8 t) + c of row r of A and of column r
+// of Qt in registers for the whole phase (the loops are bound by instruction
+// issue and latency, not by arithmetic); the eight owners of row k+1 build the
+// next reflector right after their update, inside their warp, so no third
+// barrier is needed.  Phase 2: warp 0 runs the QL iteration on (diag, sub-diag)
+// -- the search for a negligible sub-diagonal entry uses all lanes, the rotation
+// chase is one dependent chain on lane 0 -- and hands each chase's rotations
+// through a double-buffered list to d consumer threads, which apply them to the
+// rows of Qt (thread t owns column t), pipelined with the next chase by named
+// barriers.
 //
-// Output: eigenvectors as columns, descending eigenvalue, each column's entry of
-// largest magnitude (lowest row on ties) made positive.
+// Epilogue.  Components in order of descending eigenvalue.  With E the
+// eigenvectors and F the factor that produced the transformed rows, the map from
+// the original space to the coordinates is F E; component t is oriented so that
+// the entry of largest magnitude (lowest row on ties) of column t of F E is
+// positive -- a rule that gives the same signs whatever root of the metric F is.
+// Written out: the projection matrix (F E for the keys, which are projected
+// straight from K; E for the queries, whose representation is already stored),
+// its bias -mean . W, and W^T as bf16 hi + lo parts for the tensor-core
+// projection.
 #include "kernels.h"
 
 namespace ca {
@@ -52,16 +65,35 @@ constexpr int kMaxQlIterations = 64;
 
 }  // namespace
 
+// this thread's columns j = 4 (q + 8 t) + c of  acc[j] = sum_k x(k) Y[k][j]
+template <int D, typename XF>
+__device__ __forceinline__ void row_times_matrix(XF x_of_k, const float* __restrict__ Y, int lda, int q,
+                                                 float (&acc)[D / 32][4]) {
+#pragma unroll
+  for (int t = 0; t < D / 32; ++t)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) acc[t][c] = 0.f;
+#pragma unroll 4
+  for (int k = 0; k < D; ++k) {
+    const float x = x_of_k(k);
+#pragma unroll
+    for (int t = 0; t < D / 32; ++t) {
+      const float4 y = *reinterpret_cast<const float4*>(&Y[k * lda + 4 * (q + 8 * t)]);
+      acc[t][0] = fmaf(x, y.x, acc[t][0]); acc[t][1] = fmaf(x, y.y, acc[t][1]);
+      acc[t][2] = fmaf(x, y.z, acc[t][2]); acc[t][3] = fmaf(x, y.w, acc[t][3]);
+    }
+  }
+}
+
 template <int D>
-__global__ void __launch_bounds__(8 * D)
-eigh_tql_kernel(const double* __restrict__ A_in, double* __restrict__ out64, float* __restrict__ out32,
-                double* __restrict__ evals_out) {
+__global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   constexpr int NT = 8 * D, LDA = D + 4;
   constexpr int CH = D / 32;            // float4 chunks of a row per thread
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* A = reinterpret_cast<float*>(smem_raw);       // [D][LDA]
   float* Qt = A + D * LDA;                             // [D][LDA]   written after phase 1; rows become the eigenvectors
-  float* vbuf = Qt + D * LDA;                          // [2][D]     reflector, zero above its first entry
+  float* L = Qt + D * LDA;                             // [D][LDA]   the factor F (lift of the sign rule)
+  float* vbuf = L + D * LDA;                           // [2][D]     reflector, zero above its first entry
   float* pbuf = vbuf + 2 * D;                          // [D]
   float* ubuf = pbuf + D;                              // [D]
   float2* de = reinterpret_cast<float2*>(ubuf + D);    // [D]        (diagonal i, sub-diagonal coupling i and i+1)
@@ -72,23 +104,71 @@ eigh_tql_kernel(const double* __restrict__ A_in, double* __restrict__ out64, flo
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = tid >> 3, q = tid & 7;
-  const double* Ain = A_in + (size_t)blockIdx.x * D * D;
+  const size_t mat = (size_t)blockIdx.x * D * D;
 
-  // scale so that the largest diagonal entry is 1 (eigenvectors unchanged, eigenvalues scaled back)
-  if (tid < 32) {
-    double mx = 0.0;
-    for (int i = tid; i < D; i += 32) mx = fmax(mx, fabs(Ain[i * D + i]));
-    for (int o = 16; o > 0; o >>= 1) mx = fmax(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (tid == 0) s_scale = mx > 0.0 ? mx : 1.0;
+  // ---- prologue: the matrix to decompose, in A
+  if (a.lift) {
+    const double* F = a.lift + mat;
+    for (int e = tid; e < D * D; e += NT) L[(e / D) * LDA + e % D] = (float)F[e];
   }
+  if (a.mode == kPcaKeys) {
+    // C = (gram - s s^T / n) c_scale, the centred scatter of the keys; then alpha F^T C F
+    const double* G = a.gram + mat;
+    const double* sm = a.sum + (size_t)blockIdx.x * D;
+    for (int e = tid; e < D * D; e += NT) {
+      const int i = e / D, j = e % D;
+      A[i * LDA + j] = (float)((G[e] - sm[i] * sm[j] / a.n) * a.c_scale);
+    }
+    __syncthreads();
+    float acc[CH][4];
+    row_times_matrix<D>([&](int k) { return L[k * LDA + r]; }, A, LDA, q, acc);        // (F^T C)[r][.]
+#pragma unroll
+    for (int t = 0; t < CH; ++t)
+      *reinterpret_cast<float4*>(&Qt[r * LDA + 4 * (q + 8 * t)]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+    __syncthreads();
+    row_times_matrix<D>([&](int k) { return Qt[r * LDA + k]; }, L, LDA, q, acc);       // ((F^T C) F)[r][.]
+    const float al = (float)a.alpha;
+#pragma unroll
+    for (int t = 0; t < CH; ++t)
+      *reinterpret_cast<float4*>(&A[r * LDA + 4 * (q + 8 * t)]) =
+          make_float4(al * acc[t][0], al * acc[t][1], al * acc[t][2], al * acc[t][3]);
+  } else if (a.mode == kPcaQueries) {
+    // covariance of the stored representation: gram / n - mean mean^T
+    const double* G = a.gram + mat;
+    const double* sm = a.sum + (size_t)blockIdx.x * D;
+    for (int e = tid; e < D * D; e += NT) {
+      const int i = e / D, j = e % D;
+      A[i * LDA + j] = (float)(G[e] / a.n - (sm[i] / a.n) * (sm[j] / a.n));
+    }
+  } else {
+    const double* Ain = a.A_in + mat;
+    for (int e = tid; e < D * D; e += NT) A[(e / D) * LDA + e % D] = (float)Ain[e];
+  }
+  __syncthreads();
+  // symmetrise, and scale so that the largest diagonal entry is 1 (eigenvectors unchanged,
+  // eigenvalues scaled back at the end)
+  if (tid < 32) {
+    float mx = 0.f;
+    for (int i = tid; i < D; i += 32) mx = fmaxf(mx, fabsf(A[i * LDA + i]));
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (tid == 0) s_scale = mx > 0.f ? (double)mx : 1.0;
+  }
+  float sym[CH][4];
+#pragma unroll
+  for (int t = 0; t < CH; ++t)
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const int j = 4 * (q + 8 * t) + c;
+      sym[t][c] = 0.5f * (A[r * LDA + j] + A[j * LDA + r]);
+    }
   __syncthreads();
   const double a_scale = s_scale;
   {
-    const double inv = 1.0 / a_scale;
-    for (int e = tid; e < D * D; e += NT) {
-      const int i = e / D, j = e % D;
-      A[i * LDA + j] = (float)(0.5 * (Ain[i * D + j] + Ain[j * D + i]) * inv);   // symmetrise on load
-    }
+    const float inv = (float)(1.0 / a_scale);
+#pragma unroll
+    for (int t = 0; t < CH; ++t)
+      *reinterpret_cast<float4*>(&A[r * LDA + 4 * (q + 8 * t)]) =
+          make_float4(sym[t][0] * inv, sym[t][1] * inv, sym[t][2] * inv, sym[t][3] * inv);
   }
   __syncthreads();
 
@@ -324,12 +404,35 @@ eigh_tql_kernel(const double* __restrict__ A_in, double* __restrict__ out64, flo
   }
   __syncthreads();
 
-  // ---- order, sign and write out
-  double* lam = reinterpret_cast<double*>(A);                // A is free now
-  int* rank_of = reinterpret_cast<int*>(lam + D);
-  float* sign_of = reinterpret_cast<float*>(rank_of + D);
-  if (tid < D) lam[tid] = (double)de[tid].x * a_scale;
+  // ---- the map from the original space, W = F E (W[i][j] = sum_k F[i][k] Qt[j][k]), into A
+  constexpr int PER = D / 8;
+  if (a.lift) {
+    float acc[PER];
+#pragma unroll
+    for (int t = 0; t < PER; ++t) acc[t] = 0.f;
+    for (int k = 0; k < D; k += 4) {
+      const float4 f = *reinterpret_cast<const float4*>(&L[r * LDA + k]);
+#pragma unroll
+      for (int t = 0; t < PER; ++t) {
+        const float4 ev = *reinterpret_cast<const float4*>(&Qt[(q + 8 * t) * LDA + k]);
+        acc[t] = fmaf(f.x, ev.x, acc[t]); acc[t] = fmaf(f.y, ev.y, acc[t]);
+        acc[t] = fmaf(f.z, ev.z, acc[t]); acc[t] = fmaf(f.w, ev.w, acc[t]);
+      }
+    }
+#pragma unroll
+    for (int t = 0; t < PER; ++t) A[r * LDA + q + 8 * t] = acc[t];
+  }
+  // ---- order, sign, bias
+  double* lam = reinterpret_cast<double*>(vbuf);             // [D] doubles over vbuf's 2D floats
+  int* rank_of = reinterpret_cast<int*>(pbuf);
+  float* sign_of = ubuf;
+  float* mean = rot;                                         // the rotation lists are free now
+  if (tid < D) {
+    lam[tid] = (double)de[tid].x * a_scale;
+    mean[tid] = a.mean_sum ? (float)(a.mean_sum[(size_t)blockIdx.x * D + tid] / a.mean_n) : 0.f;
+  }
   __syncthreads();
+  const bool lifted_out = a.lift && a.out_lifted;
   if (tid < D) {
     const double mine = lam[tid];
     int rank = 0;
@@ -337,37 +440,47 @@ eigh_tql_kernel(const double* __restrict__ A_in, double* __restrict__ out64, flo
       const double other = lam[k];
       rank += (other > mine) || (other == mine && k < tid);
     }
-    float best = -1.f, sgn = 1.f;
+    // sign rule on column tid of F E (of E when no factor is given); bias = -mean . (output column)
+    float best = -1.f, sgn = 1.f, dot = 0.f;
     for (int i = 0; i < D; ++i) {
-      const float v = Qt[tid * LDA + i];
-      if (fabsf(v) > best) { best = fabsf(v); sgn = (v < 0.f) ? -1.f : 1.f; }
+      const float e_i = Qt[tid * LDA + i];
+      const float w_i = a.lift ? A[i * LDA + tid] : e_i;
+      if (fabsf(w_i) > best) { best = fabsf(w_i); sgn = (w_i < 0.f) ? -1.f : 1.f; }
+      dot = fmaf(mean[i], lifted_out ? w_i : e_i, dot);
     }
     rank_of[tid] = rank;
     sign_of[tid] = sgn;
-    if (evals_out) evals_out[(size_t)blockIdx.x * D + rank] = mine;
+    if (a.bias) a.bias[(size_t)blockIdx.x * D + rank] = -sgn * dot;
+    if (a.evals) a.evals[(size_t)blockIdx.x * D + rank] = mine;
   }
   __syncthreads();
-  double* o64 = out64 + (size_t)blockIdx.x * D * D;
-  float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
+  // projection matrix [in i][out rank(j)], fp32, and its transpose as bf16 hi + lo parts
   for (int e = tid; e < D * D; e += NT) {
-    const int k = e / D, i = e % D;           // eigenvector k, component i
-    const float v = sign_of[k] * Qt[k * LDA + i];
-    o64[i * D + rank_of[k]] = (double)v;
-    if (o32) o32[i * D + rank_of[k]] = v;
+    const int i = e / D, j = e % D;
+    const float v = sign_of[j] * (lifted_out ? A[i * LDA + j] : Qt[j * LDA + i]);
+    a.W32[mat + (size_t)i * D + rank_of[j]] = v;
+  }
+  if (a.wt_hi) {
+    for (int e = tid; e < D * D; e += NT) {
+      const int j = e / D, i = e % D;
+      const float v = sign_of[j] * (lifted_out ? A[i * LDA + j] : Qt[j * LDA + i]);
+      const __nv_bfloat16 h = __float2bfloat16_rn(v);
+      a.wt_hi[mat + (size_t)rank_of[j] * D + i] = h;
+      a.wt_lo[mat + (size_t)rank_of[j] * D + i] = __float2bfloat16_rn(v - __bfloat162float(h));
+    }
   }
 }
 
-int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
-                cudaStream_t st) {
-  const size_t smem = sizeof(float) * ((size_t)2 * D * (D + 4) + 2 * D + 4 * D + 4 + 4 * D) + 8 * sizeof(int);
+int launch_pca(const PcaArgs& args, int count, int D, cudaStream_t st) {
+  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 2 * D + 4 * D + 4 + 4 * D) + 8 * sizeof(int);
   if (D == 64) {
     auto k = eigh_tql_kernel<64>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, 8 * 64, smem, st>>>(A, out64, out32, evals);
+    k<<<count, 8 * 64, smem, st>>>(args);
   } else {
     auto k = eigh_tql_kernel<128>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, 8 * 128, smem, st>>>(A, out64, out32, evals);
+    k<<<count, 8 * 128, smem, st>>>(args);
   }
   CA_LAUNCH_CHECK();
   return CA_OK;

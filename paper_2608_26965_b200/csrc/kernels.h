@@ -24,18 +24,37 @@ int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_
                         void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t = nullptr,
                         bool weights_ready = false);
 
+// eigh_tql.cu: covariance + principal components + projection matrix of one side, one CTA per head
+enum { kPcaMatrix = 0, kPcaKeys = 1, kPcaQueries = 2 };
+struct PcaArgs {
+  int mode;                 // what is decomposed:
+                            //   kPcaMatrix   A_in as given
+                            //   kPcaKeys     alpha F^T C F,  C = (gram - s s^T / n) c_scale,  F = lift
+                            //   kPcaQueries  gram / n - (s / n)(s / n)^T
+  const double* A_in;       // [P][D][D]
+  const double* gram;       // [P][D][D]
+  const double* sum;        // [P][D]
+  double n, c_scale, alpha;
+  const double* lift;       // [P][D][D] factor F of the metric the rows were transformed with (sign rule:
+                            // column t of F E); null: the sign rule applies to E itself
+  int out_lifted;           // 1: the projection written is F E (rows are projected from the original
+                            // space); 0: E (rows are already transformed)
+  const double* mean_sum;   // [P][D] column sums of the rows that will be projected, and their count:
+  double mean_n;            //   bias = -(mean_sum / mean_n) . projection   (null: zero bias)
+  float* W32;               // [P][D in][D out] projection matrix
+  float* bias;              // [P][D] or null
+  __nv_bfloat16* wt_hi;     // [P][D out][D in] transposed projection as bf16 hi + lo parts, or null
+  __nv_bfloat16* wt_lo;
+  double* evals;            // [P][D] eigenvalues in descending order, or null
+};
+int launch_pca(const PcaArgs& args, int count, int D, cudaStream_t st);
+
 // eigh.cu
-int launch_eigh(const double* A, int count, int D, double* out64, float* out32, double* evals,
-                cudaStream_t st);
 int launch_metric(const double* gramQ, const double* gramK, const double* sumK, int P, int D, int n_q,
                   int n_k, double ck_scale, double* M, double* CK, cudaStream_t st);
-int launch_covariance(const double* gram, const double* sum, int P, int D, int n, double* cov,
-                      cudaStream_t st);
-int launch_small_matmul(const double* A, const double* B, int P, int D, double alpha, int trans_a,
-                        double* C, float* C32, cudaStream_t st);
-int launch_cholesky_factor(const double* A, int count, int D, double* out64, float* out32, cudaStream_t st);
-int launch_bias(const double* sum, const float* W, int P, int D, int n, float* bias, cudaStream_t st,
-                void* wt_hi = nullptr, void* wt_lo = nullptr);
+// factor of gram * scale (sum null) or of (gram - s s^T / n) * scale
+int launch_cholesky_factor(const double* gram, const double* sum, double n, double scale, int count, int D,
+                           double* out64, float* out32, void* wt_hi, void* wt_lo, cudaStream_t st);
 
 // split.cu
 int split_levels_for(int n, int c);
@@ -71,7 +90,7 @@ int launch_score_select(const float* cq, const float* ck, int P, int n_qc, int n
 int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp,
                     const float* ck, const float* cv, const int32_t* count_k, const int32_t* block_idx,
                     const int32_t* keep_count, int list_stride, const int32_t* perm_q, float scale, void* O,
-                    float* lse, cudaStream_t st, const int32_t* redo = nullptr, int redo_tiles = 0,
+                    float* lse, int* status, cudaStream_t st, const int32_t* redo = nullptr, int redo_tiles = 0,
                     int* redo_count = nullptr);
 
 // attn_tc.cu
@@ -81,5 +100,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
                    const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* keep_count,
                    int list_stride, const int32_t* perm_q, float scale, void* O, float* lse, void* ws,
                    cudaStream_t st);
+// diagnostic hook of the attention kernel (see ca_debug_attn_wait in the public header)
+void attn_tc_set_debug(long long wait_limit_cycles, int skip_key_load);
 
 }  // namespace ca

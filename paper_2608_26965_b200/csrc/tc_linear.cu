@@ -481,7 +481,7 @@ int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows,
 int launch_transform_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, const float* W,
                         const float* bias, int normalize, float* out, void* out_hi, void* out_lo,
                         void* wt_hi, void* wt_lo, int* status, cudaStream_t st, float* out_t, bool weights_ready) {
-  if (!weights_ready) {               // otherwise launch_bias has already laid W out
+  if (!weights_ready) {               // otherwise the kernel that produced W has laid it out
     weight_prep_kernel<<<dim3(ceil_div(D * D, 256), problems), 256, 0, st>>>(
         W, D, static_cast<__nv_bfloat16*>(wt_hi), static_cast<__nv_bfloat16*>(wt_lo));
     CA_LAUNCH_CHECK();

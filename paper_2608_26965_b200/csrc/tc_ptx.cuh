@@ -38,20 +38,20 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 
-// Bounded wait.  Gives up after about `kWaitLimitCycles` SM cycles (or as soon as
-// another thread of the CTA gave up): records CA_ERR_TIMEOUT in the status word,
-// raises the CTA's abort flag and returns false.  Callers keep going without
-// further waiting so that the kernel always terminates and releases its TMEM.
+// Bounded wait.  Gives up after about `limit` SM cycles (or as soon as another
+// thread of the CTA gave up): records CA_ERR_TIMEOUT in the status word, raises
+// the CTA's abort flag and returns false.  Callers keep going without further
+// waiting so that the kernel always terminates and releases its TMEM.
 constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          int* status) {
+                                          int* status, long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         atomicExch(status, 5 /* CA_ERR_TIMEOUT */);
         return false;
@@ -64,7 +64,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // sleeps between polls, so that it does not take issue slots from the warps that share its
 // sub-core.
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                                  int* status) {
+                                                  int* status, long long limit = kWaitLimitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
@@ -72,7 +72,7 @@ __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity,
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0) {
       if (*abort_flag) return false;
-      if (clock64() - t0 > kWaitLimitCycles) {
+      if (clock64() - t0 > limit) {
         *abort_flag = 1;
         atomicExch(status, 5 /* CA_ERR_TIMEOUT */);
         return false;

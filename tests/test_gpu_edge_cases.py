@@ -154,3 +154,147 @@ def test_attention_scores_that_rise_along_the_list(d, c_q, c_k, compensate):
     assert plan.recomputed_clusters() > 0
     assert np.abs(O - o_ref).max() <= 2e-2 and np.linalg.norm(O - o_ref) <= 5e-3 * np.linalg.norm(o_ref)
     assert np.abs(lse - lse_ref).max() <= 2e-2 + 1e-4 * np.abs(lse_ref).max()
+
+
+# ----------------------------------------------------------------------------
+# Indices that come from the caller are checked before use; waits are bounded.
+# ----------------------------------------------------------------------------
+def _attention_inputs(dtype, d, n_q, n_k, c, keep, seed):
+    """A valid attention problem on an arbitrary permutation: host arrays + device tensors."""
+    r = np.random.default_rng(seed)
+    Q = _bf16_round(r.standard_normal((n_q, d)))
+    K = _bf16_round(r.standard_normal((n_k, d)))
+    V = _bf16_round(r.standard_normal((n_k, d)))
+    perm_q, perm_k = r.permutation(n_q), r.permutation(n_k)
+    n_qc, n_kc = -(-n_q // c), -(-n_k // c)
+    idx = np.stack([np.sort(r.choice(n_kc, keep, replace=False)) for _ in range(n_qc)]).astype(np.int32)
+    ck, count_k = orc.centroids(K, perm_k, c)
+    cv, _ = orc.centroids(V, perm_k, c)
+
+    def pad(x, perm, n):
+        out = np.zeros((-(-n // c) * c, d), np.float32)
+        out[:n] = x[perm]
+        return out
+    dt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    t = dict(Qp=dev(pad(Q, perm_q, n_q)[None, None], dt), Kp=dev(pad(K, perm_k, n_k)[None, None], dt),
+             Vp=dev(pad(V, perm_k, n_k)[None, None], dt), ck=dev(ck.astype(np.float32)[None, None]),
+             cv=dev(cv.astype(np.float32)[None, None]), count_k=dev(count_k[None, None], torch.int32))
+    host = dict(Q=Q, K=K, V=V, perm_q=perm_q, perm_k=perm_k, idx=idx, ck=ck.astype(np.float32),
+                cv=cv.astype(np.float32), count_k=count_k)
+    return host, t
+
+
+@pytest.mark.parametrize("dtype,d,c", [("bf16", 64, 128), ("bf16", 128, 32), ("fp32", 64, 64)])
+def test_forged_indices_are_reported_and_skipped(dtype, d, c):
+    """A block list with entries that are no key clusters and a perm_q entry that is no row of O:
+    the call reports CA_ERR_BAD_INDEX in the status word, treats the forged clusters as absent (the
+    oracle on the list without them gives the same rows) and leaves the forged row unwritten."""
+    n_q, n_k, keep = 5 * c + 17, 9 * c + 3, 4
+    host, t = _attention_inputs(dtype, d, n_q, n_k, c, keep, seed=91)
+    n_kc = -(-n_k // c)
+    idx = host["idx"].copy()
+    idx[2, 1] = n_kc + 5
+    idx[2, 3] = -7
+    perm_q = host["perm_q"].astype(np.int32).copy()
+    forged_pos = 3 * c + 5
+    lost_row = int(perm_q[forged_pos])
+    perm_q[forged_pos] = n_q + 3
+    p = binding.make_problem(1, 1, n_q, n_k, d, dtype, c, c, keep, True)
+    plan = binding.Plan(p, DEV)
+    plan.O.fill_(7.0)
+    plan.lse.fill_(7.0)
+    O, lse = plan.cluster_attention_fwd(t["Qp"], t["Kp"], t["Vp"], t["ck"], t["cv"], t["count_k"],
+                                        dev(idx[None, None], torch.int32), dev(perm_q[None, None], torch.int32))
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == binding.CA_ERR_BAD_INDEX
+    O, lse = O[0, 0].float().cpu().numpy(), lse[0, 0].cpu().numpy()
+    assert np.isfinite(O).all() and np.isfinite(lse).all()
+    assert (O[lost_row] == 7.0).all() and lse[lost_row] == 7.0          # not written
+    lists = [row[(row >= 0) & (row < n_kc)] for row in idx]
+    o_ref, lse_ref = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
+                                           lists, True, ck=host["ck"], cv=host["cv"], count_k=host["count_k"])
+    rows = np.setdiff1d(np.arange(n_q), [lost_row])
+    tol = 1e-5 if dtype == "fp32" else 2e-2
+    assert np.abs(O[rows] - o_ref[rows]).max() <= tol and np.abs(lse[rows] - lse_ref[rows]).max() <= tol
+    # the next call on the same workspace with valid indices is clean
+    plan.cluster_attention_fwd(t["Qp"], t["Kp"], t["Vp"], t["ck"], t["cv"], t["count_k"],
+                               dev(host["idx"][None, None], torch.int32),
+                               dev(host["perm_q"].astype(np.int32)[None, None], torch.int32))
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == 0
+
+
+@pytest.mark.parametrize("dtype,compensate", [("bf16", True), ("bf16", False), ("fp32", False)])
+def test_ragged_list_lengths_of_zero_and_beyond_the_row(dtype, compensate):
+    """cluster_attention_fwd_ragged with a list of length 0 (with compensation: centroids only;
+    without: no entry at all, the rows are zeros with lse = -inf) and with a length beyond the row
+    (clamped to the row and reported)."""
+    d, c, n_q, n_k = 64, 64, 4 * 64, 6 * 64
+    host, t = _attention_inputs(dtype, d, n_q, n_k, c, 6, seed=92)
+    n_kc = 6
+    idx = np.tile(np.arange(n_kc, dtype=np.int32), (4, 1))
+    keep_count = np.array([3, 0, 6, 2], np.int32)
+    p = binding.make_problem(1, 1, n_q, n_k, d, dtype, c, c, 1, compensate)
+    plan = binding.Plan(p, DEV)
+    args = (t["Qp"], t["Kp"], t["Vp"], t["ck"], t["cv"], t["count_k"], dev(host["perm_q"].astype(np.int32)[None, None], torch.int32))
+    O, lse = plan.cluster_attention_fwd_ragged(dev(idx[None, None], torch.int32), dev(keep_count[None, None], torch.int32), *args)
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == 0
+    O, lse = O[0, 0].float().cpu().numpy(), lse[0, 0].cpu().numpy()
+    lists = [idx[i, :keep_count[i]] for i in range(4)]
+    tol = 1e-5 if dtype == "fp32" else 2e-2
+    empty_rows = host["perm_q"][c:2 * c]
+    others = np.setdiff1d(np.arange(n_q), empty_rows)
+    if compensate:
+        o_ref, lse_ref = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
+                                               lists, True, ck=host["ck"], cv=host["cv"], count_k=host["count_k"])
+        assert np.abs(O - o_ref).max() <= tol and np.abs(lse - lse_ref).max() <= tol
+    else:
+        lists_ne = [l if len(l) else np.array([0]) for l in lists]
+        o_ref, lse_ref = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
+                                               lists_ne, False)
+        assert np.abs(O[others] - o_ref[others]).max() <= tol
+        assert (O[empty_rows] == 0).all() and np.isneginf(lse[empty_rows]).all()
+    # a length beyond the row: reported, clamped to the row
+    keep_count[3] = n_kc + 4
+    O2, _ = plan.cluster_attention_fwd_ragged(dev(idx[None, None], torch.int32), dev(keep_count[None, None], torch.int32), *args)
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == binding.CA_ERR_BAD_INDEX
+    lists[3] = idx[3]
+    o_ref, _ = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
+                                     [l if len(l) else np.array([0]) for l in lists], compensate,
+                                     ck=host["ck"], cv=host["cv"], count_k=host["count_k"])
+    rows = host["perm_q"][3 * c:4 * c]
+    assert np.abs(O2[0, 0].float().cpu().numpy()[rows] - o_ref[rows]).max() <= tol
+
+
+@pytest.mark.parametrize("d", [64, 128])
+def test_a_wait_that_runs_out_ends_the_kernel_with_a_status(d):
+    """The loader of the tensor-core attention kernel is told (diagnostic hook) to leave out the key
+    rows of one half-step, with the limit of the device-side waits set to about a millisecond: the
+    waits for those rows run out, the kernel records CA_ERR_TIMEOUT, releases its tensor memory and
+    returns.  With the hook cleared the next call on the same workspace is correct again."""
+    lib = binding.load_library()
+    c, n_q, n_k, keep = 128, 512, 1024, 3
+    host, t = _attention_inputs("bf16", d, n_q, n_k, c, keep, seed=93)
+    p = binding.make_problem(1, 1, n_q, n_k, d, "bf16", c, c, keep, True)
+    plan = binding.Plan(p, DEV)
+    args = (t["Qp"], t["Kp"], t["Vp"], t["ck"], t["cv"], t["count_k"], dev(host["idx"][None, None], torch.int32),
+            dev(host["perm_q"].astype(np.int32)[None, None], torch.int32))
+    good = plan.cluster_attention_fwd(*args)[0].clone()
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == 0
+    try:
+        lib.ca_debug_attn_wait(2_000_000, 2)
+        plan.cluster_attention_fwd(*args)
+        torch.cuda.synchronize()
+        assert plan.last_status()["attn"] == binding.CA_ERR_TIMEOUT
+    finally:
+        lib.ca_debug_attn_wait(0, -1)
+    again = plan.cluster_attention_fwd(*args)[0]
+    torch.cuda.synchronize()
+    assert plan.last_status()["attn"] == 0
+    assert torch.equal(again, good)
+    o_ref, _ = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
+                                     host["idx"], True, ck=host["ck"], cv=host["cv"], count_k=host["count_k"])
+    assert np.abs(again[0, 0].float().cpu().numpy() - o_ref).max() <= 2e-2

@@ -21,7 +21,7 @@ def lib():
 def declared_functions():
     text = open(os.path.join(ROOT, "include", "cluster_attention.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    return sorted(set(re.findall(r"\b(?:int|const char\*|unsigned long long|size_t)\s+(\w+)\s*\(", text)))
+    return sorted(set(re.findall(r"\b(?:int|void|const char\*|unsigned long long|size_t)\s+(\w+)\s*\(", text)))
 
 
 def test_header_declarations_are_exported(lib):
