@@ -520,7 +520,8 @@ def cluster_attention(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx, compensate,
     for i in todo:
         rows = perm_q[i * c_q:min((i + 1) * c_q, N_q)]
         sel = np.asarray(block_idx[i], np.int64)
-        members = np.concatenate([perm_k[j * c_k:min((j + 1) * c_k, N_k)] for j in sel])
+        members = (np.concatenate([perm_k[j * c_k:min((j + 1) * c_k, N_k)] for j in sel]) if len(sel)
+                   else np.zeros(0, np.int64))          # S empty: with compensation every cluster enters by its centroid
         logits = scale * (Q[rows] @ K[members].T)
         values = V[members]
         if compensate:
