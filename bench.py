@@ -39,8 +39,33 @@ METRIC = "clusterattention_hot_path_block_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
-# DRAM bytes per launch of the dominant kernel from an ncu capture (see profiles/); None = not captured.
-NCU_TRAFFIC_BYTES = {"tabular": 554.2e6, "video480": 1269.0e6}   # scaled by heads from the 4- and 8-head captures in profiles/
+# DRAM bytes per launch of the dominant kernel from the ncu captures summarised under profiles/
+# (4- and 8-head captures scaled by the head count).  Each figure is tied to the kernel source it
+# was captured from: sha256 of csrc/attn_tc.cu + csrc/tc_ptx.cuh, first 16 hex digits.  When the
+# source has changed since, the bench prints null instead of a stale figure.
+NCU_TRAFFIC = {
+    "tabular": {"bytes": 554.2e6, "source": "", "commit": "4457068"},
+    "video480": {"bytes": 1269.0e6, "source": "", "commit": "6755999"},
+}
+# FP32 FMA rate of the CUDA cores, the roof of kernels bound by plain arithmetic (centroid scoring,
+# the fp32 attention kernel): 148 SMs x 128 FMA lanes x 2 flops x 1.965 GHz (the maximum SM clock).
+FP32_ALU_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+
+def attn_source_digest():
+    import hashlib
+    h = hashlib.sha256()
+    for name in ("attn_tc.cu", "tc_ptx.cuh"):
+        with open(os.path.join(ROOT, "paper_2608_26965_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload_name):
+    rec = NCU_TRAFFIC.get(workload_name)
+    if rec is None or rec["source"] != attn_source_digest():
+        return None, None
+    return rec["bytes"], rec["commit"]
 
 
 def parse_args():
@@ -69,6 +94,9 @@ def parse_args():
                     help="token-count sweep 8k..1M with per-stage times (64 kept blocks, and 10 %% of the blocks), "
                          "eager launches and one replayed CUDA graph, against dense attention")
     ap.add_argument("--max-tokens", type=int, default=1 << 20)
+    ap.add_argument("--secondary", default="video480", metavar="WORKLOAD",
+                    help="also report stage times and the attention roofline of this workload (10 steps); "
+                         "'' switches it off")
     return ap.parse_args()
 
 
@@ -165,7 +193,7 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "50",
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "20",
                  "-i", str(device_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -197,6 +225,133 @@ class ClockSampler:
             pass
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
                 "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------
+# per-kernel rooflines of the clustering and selection stages
+# ------------------------------------------------------------------------------
+def split_level_counts(n, c):
+    """(levels run as per-level launches over whole sets, levels finished inside the subtree kernel):
+    sets of more than min(32 c, 4096) rows take a launch per level."""
+    def nxt(big):
+        L = c * ((big + c) // (2 * c))
+        return max(L, big - L)
+    levels, top, big = 0, 0, n
+    tail_rows = min(32 * c, 4096)
+    while big > c:
+        if big > tail_rows:
+            top += 1
+        levels += 1
+        big = nxt(big)
+    return top, levels - top
+
+
+def stage_rooflines(w, heads, group_ms, hbm_gbs, peak_kind):
+    """Algorithmic bytes (flops for the scoring) of every kernel group of cluster_qk and
+    select_blocks, its device time per step (the library's own CUDA-event timers, each group timed
+    alone), and the fraction of the roof that bounds it."""
+    b = 2 if w.dtype == "bf16" else 4
+    d, nq, nk, c = w.head_dim, w.n_q, w.n_k, w.cluster
+    top_q, tail_q = split_level_counts(nq, c)
+    top_k, tail_k = split_level_counts(nk, c)
+    sub = lambda nodes: nodes * d * d * 4                      # subsample rows read by `nodes` sets
+    algo = {
+        # Gram matrices of Q, K and of the query representation r(q) (stored as two bf16 halves / fp32)
+        "gram": heads * ((nq + nk) * d * b + nq * d * 4),
+        # Q -> r(q) (4 bytes per element out), r(q) -> Y_q, K -> Y_k (fp32 coordinates out)
+        "transform": heads * (nq * d * (b + 4) + nq * d * 8 + nk * d * (b + 4)),
+        # per level and side: a key and a row index read, a row index written, plus the subsample tiles
+        "split_levels": heads * (12 * (nq * top_q + nk * top_k) + sub((1 << top_q) - 1) + sub((1 << top_k) - 1)),
+        "split_tail": heads * (12 * (nq * tail_q + nk * tail_k)
+                               + sub(max(0, w.n_qc - (1 << top_q))) + sub(max(0, w.n_kc - (1 << top_k)))),
+        # Q, K and V rows read once and written once in cluster order
+        "permute_centroid": heads * 2 * (nq + 2 * nk) * d * b,
+    }
+    out = {}
+    for name, nbytes in algo.items():
+        ms = group_ms.get(name)
+        if not ms:
+            continue
+        gbs = nbytes / (ms * 1e-3) / 1e9
+        out[name] = {"bound": "hbm", "algorithmic_bytes": nbytes, "ms": ms, "achieved": gbs, "unit": "GB/s",
+                     "peak": hbm_gbs, "peak_source": f"{peak_kind} HBM copy", "frac": gbs / hbm_gbs}
+    for name in ("cholesky_factor", "principal_components"):
+        if group_ms.get(name):
+            out[name] = {"bound": "latency", "ms": group_ms[name],
+                         "note": "d x d work on one CTA per head and side: no roofline, wall time only"}
+    ms = group_ms.get("score_select")
+    if ms:
+        flops = 2.0 * w.n_qc * w.n_kc * d * heads
+        tf = flops / (ms * 1e-3) / 1e12
+        out["score_select"] = {"bound": "alu", "algorithmic_flops": flops, "ms": ms, "achieved": tf, "unit": "TFLOP/s",
+                               "peak": FP32_ALU_TFLOPS, "peak_source": "148 SMs x 128 FMA lanes x 2 x 1.965 GHz",
+                               "frac": tf / FP32_ALU_TFLOPS,
+                               "algorithmic_bytes": heads * ((w.n_qc + w.n_kc) * d * 4 + w.n_qc * w.keep * 4),
+                               "hbm_frac": heads * ((w.n_qc + w.n_kc) * d * 4 + w.n_qc * w.keep * 4) / (ms * 1e-3) / 1e9 / hbm_gbs}
+    return out
+
+
+def library_dense_ms(torch, binding, w, Q, K, V, dev, reps=3):
+    """Dense attention through the library's own kernel: every key cluster kept, compensation off,
+    identity permutation (the inputs themselves are the cluster-ordered tensors)."""
+    p = binding.problem_from_workload(w, keep=w.n_kc, compensate=False)
+    plan = binding.Plan(p, dev)
+    c = w.cluster
+    for dst, src, n in ((plan.Qp, Q, w.n_q), (plan.Kp, K, w.n_k), (plan.Vp, V, w.n_k)):
+        dst.zero_()
+        dst[:, :, :n].copy_(src)
+    plan.perm_q.copy_(torch.arange(w.n_q, dtype=torch.int32, device=dev).expand_as(plan.perm_q))
+    counts = torch.full((w.n_kc,), c, dtype=torch.int32, device=dev)
+    counts[-1] = w.n_k - (w.n_kc - 1) * c
+    plan.count_k.copy_(counts.expand_as(plan.count_k))
+    plan.block_idx.copy_(torch.arange(w.n_kc, dtype=torch.int32, device=dev).expand_as(plan.block_idx))
+    plan.ck.zero_()
+    plan.cv.zero_()
+    plan.cluster_attention_fwd(want_lse=False)
+    torch.cuda.synchronize()
+    a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        plan.cluster_attention_fwd(want_lse=False)
+    b_.record()
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    return a.elapsed_time(b_) / reps
+
+
+def secondary_workload(torch, binding, inputs, name, dev, steps, peaks):
+    """Stage times and the attention roofline fraction of another workload (d = 128), so that the
+    record of the default run also carries the video-shaped configuration."""
+    w = inputs.WORKLOADS[name]
+    p = binding.problem_from_workload(w)
+    dt = binding.torch_dtype(p)
+    Q, K, V = (torch.from_numpy(a[None]).to(dt).to(dev) for a in inputs.generate(w))
+    plan = binding.Plan(p, dev)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        plan.forward(Q, K, V)
+    torch.cuda.synchronize()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    for e in ev:
+        e[0].record(stream)
+        plan.cluster_qk(Q, K, V)
+        e[1].record(stream)
+        plan.select_blocks()
+        e[2].record(stream)
+        plan.cluster_attention_fwd(want_lse=False)
+        e[3].record(stream)
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values()) and plan.recomputed_clusters() == 0
+    stage = {"cluster_qk": float(np.mean([e[0].elapsed_time(e[1]) for e in ev])),
+             "select_blocks": float(np.mean([e[1].elapsed_time(e[2]) for e in ev])),
+             "cluster_attention_fwd": float(np.mean([e[2].elapsed_time(e[3]) for e in ev]))}
+    flops = block_flops(w, w.heads)
+    tf = flops / (stage["cluster_attention_fwd"] * 1e-3) / 1e12
+    return {"workload": name, "heads": w.heads, "head_dim": w.head_dim, "n_q": w.n_q, "n_k": w.n_k, "keep": w.keep,
+            "steps": steps, "stage_ms": stage, "ms_per_step": float(np.mean([e[0].elapsed_time(e[3]) for e in ev])),
+            "block_flops_per_step": flops,
+            "roofline": {"kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": tf,
+                         "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tf / peaks["bf16_tflops"]}}
 
 
 # ------------------------------------------------------------------------------
@@ -271,6 +426,9 @@ def run_ours(args, w):
         if events is not None:
             events[3].record(stream)
 
+    # the clock sampler runs from before the warm-up until after the sustained leg below, so that a
+    # short timed region still has clock samples under the same load around it
+    sampler = ClockSampler(local) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         step()
     barrier()
@@ -279,7 +437,6 @@ def run_ours(args, w):
     # ---- timed region: device-resident inputs (larger than L2, so no flush is needed)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
     launches0 = binding.kernel_launches()
-    sampler = ClockSampler(local) if rank == 0 else None
     barrier()
     t_start = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
@@ -288,9 +445,34 @@ def run_ours(args, w):
         step(ev[i])
     t_end.record(stream)
     barrier()
-    clocks = sampler.stop() if sampler else None
     launches = binding.kernel_launches() - launches0
-    recomputed = plan.recomputed_clusters()           # 0: no query cluster left the tensor-core kernel
+    # ---- sustained leg (not the headline): the same step back to back for about a second, so that the
+    # clock sampler sees this load for long enough; its time per step is reported beside the headline
+    sustained = None
+    if rank == 0:
+        n_sus = max(args.steps, int(1000.0 / max(t_start.elapsed_time(t_end) / args.steps, 0.05)))
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(n_sus):
+            step()
+        s1.record(stream)
+        torch.cuda.synchronize()
+        sustained = {"steps": n_sus, "ms_per_step": s0.elapsed_time(s1) / n_sus}
+    clocks = sampler.stop() if sampler else None
+    if clocks is not None:
+        clocks["window"] = "warm-up, timed region and the sustained leg (same step, about one second)"
+        clocks["sustained_leg"] = sustained
+    recomputed = plan.recomputed_clusters()           # 0 over every step so far: nothing left the tensor-core kernel
+    # ---- per-kernel times of the clustering and selection stages (the library's own timers, each
+    # kernel group alone on the stream), outside the timed region
+    group_ms = {}
+    if rank == 0 and not basic:
+        binding.profile(True)
+        n_prof = 5
+        for _ in range(n_prof):
+            step()
+        group_ms = {k: v["ms"] / n_prof for k, v in binding.profile_read().items() if v["scopes"]}
+        binding.profile(False)
     total_ms = max_over_ranks(t_start.elapsed_time(t_end))
     ms_per_step = total_ms / args.steps
     stage_ms = {
@@ -390,6 +572,13 @@ def run_ours(args, w):
             dense["speedup_vs_torch_sdpa"] = dense["torch_sdpa_ms"] / ms_per_step
         except Exception as exc:  # noqa: BLE001
             dense["torch_sdpa_error"] = str(exc)[:200]
+        if w.dtype == "bf16":
+            dense["library_ms"] = library_dense_ms(torch, binding, w, Q, K, V, dev)
+            dense["library_tflops"] = dense_flops(w, heads) / (dense["library_ms"] * 1e-3) / 1e12
+        candidates = [dense[k] for k in ("torch_sdpa_ms", "library_ms") if k in dense]
+        if candidates:
+            dense["fastest_ms"] = min(candidates)
+            dense["speedup_vs_fastest_dense"] = dense["fastest_ms"] / ms_per_step
 
     barrier()
     if rank != 0:
@@ -441,13 +630,21 @@ def run_ours(args, w):
     peaks, peak_kind = load_peaks()
     attn_ms = stage_ms["cluster_attention_fwd"]
     attn_tflops = flops_step / (attn_ms * 1e-3) / 1e12
-    peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.0 / 16.0
-    roofline = {
-        "kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": attn_tflops, "peak": peak,
-        "peak_source": f"{peak_kind} bf16 burst", "unit": "TFLOP/s", "frac": attn_tflops / peak,
-        "traffic": None if (adaptive or basic or args.keep or args.n_q or args.n_k or args.heads)
-        else NCU_TRAFFIC_BYTES.get(w.name),
-    }
+    traffic, traffic_commit = (None, None) if (adaptive or basic or args.keep or args.n_q or args.n_k or args.heads) \
+        else ncu_traffic(w.name)
+    if w.dtype == "bf16":
+        roofline = {"kernel": "cluster_attention_fwd", "bound": "tensor", "achieved": attn_tflops,
+                    "peak": peaks["bf16_tflops"], "peak_source": f"{peak_kind} bf16 burst", "unit": "TFLOP/s",
+                    "frac": attn_tflops / peaks["bf16_tflops"], "traffic": traffic, "traffic_capture_commit": traffic_commit}
+    else:           # fp32 storage runs the CUDA-core kernel: bound by the FP32 FMA rate
+        roofline = {"kernel": "cluster_attention_fwd", "bound": "alu", "achieved": attn_tflops, "peak": FP32_ALU_TFLOPS,
+                    "peak_source": "148 SMs x 128 FMA lanes x 2 x 1.965 GHz", "unit": "TFLOP/s",
+                    "frac": attn_tflops / FP32_ALU_TFLOPS, "traffic": None}
+    stages = stage_rooflines(w.scaled(keep=keep), heads, group_ms, peaks["hbm_gbs"], peak_kind) if group_ms else None
+    secondary = None
+    if args.secondary and args.secondary != w.name and world == 1 and w.name == "tabular" \
+            and not (adaptive or basic or args.keep or args.n_q or args.n_k or args.heads):
+        secondary = secondary_workload(torch, binding, inputs, args.secondary, dev, 10, peaks)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -460,9 +657,10 @@ def run_ours(args, w):
                    "parallelism": "replicas" if world > 1 else "single",
                    "l2": "inputs larger than L2 (no flush)"},
         "stage_ms": stage_ms, "block_flops_per_step": flops_step, "dense_flops": dense_flops(w, heads),
-        "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "recomputed_clusters": int(recomputed),
+        "roofline": roofline, "stage_rooflines": stages, "kernel_group_ms": group_ms or None,
+        "e2e": e2e, "gpu_launches": int(launches), "recomputed_clusters": int(recomputed),
         "clocks": clocks, "dense": dense,
-        "overlap": overlap,
+        "overlap": overlap, "secondary": secondary,
     }
     if not args.no_cpu_baseline:
         # the oracle as it stands on whole heads until about 10 s of CPU work are spent

@@ -276,6 +276,21 @@ int ca_attn_recomputed(const void* ws);
  * memory and returns, and the output of the call is undefined; -1 restores normal operation. */
 void ca_debug_attn_wait(long long wait_limit_cycles, int skip_key_load);
 
+/*
+ * Per-kernel-group device times (a measuring aid; process-wide, not thread-safe).
+ * ca_profile(1) switches the timers on: every call issued afterwards records CUDA events around
+ * its kernel groups, and cluster_qk runs its two sides one after the other on the caller's stream
+ * (instead of side by side on two streams) so that every group is timed alone.  ca_profile(0)
+ * switches them off.  The first ca_profile(1) creates the events (make it before a stream capture).
+ * ca_profile_read synchronises the device, returns the number of groups and, for group g, its
+ * name (static string), the summed device time in ms and the number of timed scopes since the
+ * timers were switched on or last read; then it starts counting afresh.  Groups: gram,
+ * cholesky_factor, principal_components, transform, split_levels, split_tail, permute_centroid,
+ * score_select, centroid_prep, attn_tc, attn_second_pass.  Any output pointer may be NULL.
+ */
+int ca_profile(int enable);
+int ca_profile_read(int max_groups, const char** names, float* ms, int* scopes);
+
 /* Library version and the compute capability the kernels were built for. */
 const char* ca_version(void);
 

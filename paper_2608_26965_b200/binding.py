@@ -29,7 +29,8 @@ CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN = 1, 2, 4, 8
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_attn_recomputed", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
            "ca_static_scratch_bytes", "ca_static_last_status", "select_blocks_adaptive",
-           "cluster_attention_fwd_ragged", "ca_basic_workspace_bytes", "cluster_qk_basic", "ca_debug_attn_wait")
+           "cluster_attention_fwd_ragged", "ca_basic_workspace_bytes", "cluster_qk_basic", "ca_debug_attn_wait",
+           "ca_profile", "ca_profile_read")
 
 
 class CaProblem(ctypes.Structure):
@@ -105,8 +106,32 @@ def load_library() -> ctypes.CDLL:
     lib.ca_static_last_status.restype = ctypes.c_int
     lib.ca_debug_attn_wait.argtypes = [ctypes.c_longlong, ctypes.c_int]
     lib.ca_debug_attn_wait.restype = None
+    lib.ca_profile.argtypes = [ctypes.c_int]
+    lib.ca_profile.restype = ctypes.c_int
+    lib.ca_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float),
+                                    ctypes.POINTER(ctypes.c_int)]
+    lib.ca_profile_read.restype = ctypes.c_int
     _lib = lib
     return lib
+
+
+def profile(enable: bool) -> None:
+    """Switches the library's per-kernel-group timers on or off (ca_profile)."""
+    _check(load_library().ca_profile(1 if enable else 0), "ca_profile")
+
+
+def profile_read() -> Dict[str, Dict[str, float]]:
+    """Device time in ms and number of timed scopes per kernel group since the timers were switched
+    on or last read (ca_profile_read; synchronises the device)."""
+    lib = load_library()
+    n = 16
+    names = (ctypes.c_char_p * n)()
+    ms = (ctypes.c_float * n)()
+    scopes = (ctypes.c_int * n)()
+    got = lib.ca_profile_read(n, names, ms, scopes)
+    if got < 0:
+        _check(-got, "ca_profile_read")
+    return {names[i].decode(): {"ms": float(ms[i]), "scopes": int(scopes[i])} for i in range(got)}
 
 
 def kernel_launches() -> int:

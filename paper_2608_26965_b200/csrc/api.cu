@@ -8,7 +8,38 @@ using namespace ca;
 
 namespace ca {
 unsigned long long g_kernel_launches = 0;
+
+// ---- per-kernel-group timers (off unless ca_profile(1) was called) ------------------------------
+namespace {
+constexpr int kProfPairs = 512;
+struct Profiler {
+  bool on = false;
+  int used = 0;
+  cudaEvent_t begin[kProfPairs], end[kProfPairs];
+  int group[kProfPairs];
+  int open_pair[kProfGroups];
+  int created = 0;
+} g_prof;
+const char* const kProfNames[kProfGroups] = {
+    "gram", "cholesky_factor", "principal_components", "transform", "split_levels", "split_tail",
+    "permute_centroid", "score_select", "centroid_prep", "attn_tc", "attn_second_pass"};
+}  // namespace
+bool prof_enabled() { return g_prof.on; }
+void prof_mark(int group, cudaStream_t st, bool begin) {
+  if (!g_prof.on) return;
+  if (begin) {
+    if (g_prof.used >= g_prof.created) return;            // out of pairs: the scope is not timed
+    const int i = g_prof.used++;
+    g_prof.group[i] = group;
+    g_prof.open_pair[group] = i;
+    cudaEventRecord(g_prof.begin[i], st);
+  } else {
+    const int i = g_prof.open_pair[group];
+    if (i >= 0) cudaEventRecord(g_prof.end[i], st);
+    g_prof.open_pair[group] = -1;
+  }
 }
+}  // namespace ca
 
 namespace {
 
@@ -131,6 +162,41 @@ const char* ca_version(void) { return "libclusterattn 0.1 (sm_100a)"; }
 
 unsigned long long ca_kernel_launches(void) { return g_kernel_launches; }
 
+int ca_profile(int enable) {
+  if (enable) {
+    while (g_prof.created < kProfPairs) {
+      if (cudaEventCreate(&g_prof.begin[g_prof.created]) != cudaSuccess) return CA_ERR_CUDA;
+      if (cudaEventCreate(&g_prof.end[g_prof.created]) != cudaSuccess) return CA_ERR_CUDA;
+      ++g_prof.created;
+    }
+    g_prof.used = 0;
+    for (int g = 0; g < kProfGroups; ++g) g_prof.open_pair[g] = -1;
+  }
+  g_prof.on = enable != 0;
+  return CA_OK;
+}
+
+int ca_profile_read(int max_groups, const char** names, float* ms, int* scopes) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return -CA_ERR_CUDA;
+  float total[kProfGroups] = {};
+  int count[kProfGroups] = {};
+  for (int i = 0; i < g_prof.used; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, g_prof.begin[i], g_prof.end[i]) != cudaSuccess) { (void)cudaGetLastError(); continue; }
+    total[g_prof.group[i]] += t;
+    ++count[g_prof.group[i]];
+  }
+  g_prof.used = 0;
+  int n = 0;
+  for (int g = 0; g < kProfGroups && n < max_groups; ++g) {
+    if (names) names[n] = kProfNames[g];
+    if (ms) ms[n] = total[g];
+    if (scopes) scopes[n] = count[g];
+    ++n;
+  }
+  return n;
+}
+
 int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select_ws, size_t* attn_ws) {
   CA_TRY(check_problem(p));
   if (cluster_ws) *cluster_ws = carve_cluster(p, nullptr, true, true).bytes;
@@ -183,33 +249,54 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
     const float* Fk32 = w.roots32 + (size_t)P * DD;
     SideStream* side = side_stream();
     if (!side) return CA_ERR_CUDA;
-    cudaStream_t sq = side->stream;
-    CA_RETURN_IF_CUDA(cudaEventRecord(side->fork, st));
-    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(sq, side->fork, 0));
-    if (tc) {
-      CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
-      CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial2, w.gramK, w.sumK, w.status, sq));
-    } else {
-      CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
-      CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial2, w.gramK, w.sumK, sq));
+    // while the per-kernel timers are on, both sides run on the caller's stream, one kernel after
+    // the other, so that every kernel group is timed alone
+    const bool serial = prof_enabled();
+    cudaStream_t sq = serial ? st : side->stream;
+    if (!serial) {
+      CA_RETURN_IF_CUDA(cudaEventRecord(side->fork, st));
+      CA_RETURN_IF_CUDA(cudaStreamWaitEvent(sq, side->fork, 0));
     }
-    CA_RETURN_IF_CUDA(cudaEventRecord(side->mid, sq));
-    CA_TRY(launch_cholesky_factor(w.gramQ, nullptr, 1.0, 1.0 / (double)p->n_q, P, D, Fq, w.roots32, nullptr, nullptr, st));
-    CA_TRY(launch_cholesky_factor(w.gramK, w.sumK, (double)p->n_k, ck_scale, P, D, Fk, w.roots32 + (size_t)P * DD,
-                                  tc ? w.wt2_hi : nullptr, tc ? w.wt2_lo : nullptr, sq));
+    {
+      ProfScope ps(kProfGram, st);
+      if (tc) {
+        CA_TRY(launch_gram_tc(Q, nullptr, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, w.status, st));
+        CA_TRY(launch_gram_tc(K, nullptr, P, p->n_k, D, w.partial2, w.gramK, w.sumK, w.status, sq));
+      } else {
+        CA_TRY(launch_moments(Q, p->dtype, P, p->n_q, D, w.partial, w.gramQ, w.sumQ, st));
+        CA_TRY(launch_moments(K, p->dtype, P, p->n_k, D, w.partial2, w.gramK, w.sumK, sq));
+      }
+    }
+    if (!serial) CA_RETURN_IF_CUDA(cudaEventRecord(side->mid, sq));
+    {
+      ProfScope ps(kProfFactor, st);
+      CA_TRY(launch_cholesky_factor(w.gramQ, nullptr, 1.0, 1.0 / (double)p->n_q, P, D, Fq, w.roots32, nullptr, nullptr, st));
+      CA_TRY(launch_cholesky_factor(w.gramK, w.sumK, (double)p->n_k, ck_scale, P, D, Fk, w.roots32 + (size_t)P * DD,
+                                    tc ? w.wt2_hi : nullptr, tc ? w.wt2_lo : nullptr, sq));
+    }
     // ---- query side (side stream)
     // query representation r(q) = F_k^T q / |F_k^T q|, its covariance and principal components E_Q
     // (one kernel), the coordinates Y = (r(q) - mean) E_Q
     float* EQ32 = w.basis32 + (size_t)P * DD;
-    if (tc) {
-      CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
-                                 w.wt2_hi, w.wt2_lo, w.status, sq, nullptr, true));
-      CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, w.status, sq));
-    } else {
-      CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
-      CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, sq));
+    {
+      ProfScope ps(kProfTransform, sq);
+      if (tc) {
+        CA_TRY(launch_transform_tc(Q, nullptr, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, nullptr, qp_hi, qp_lo,
+                                   w.wt2_hi, w.wt2_lo, w.status, sq, nullptr, true));
+      } else {
+        CA_TRY(launch_transform_rows(Q, p->dtype, P, p->n_q, D, Fk32, nullptr, unnormalized ? 0 : 1, w.Qprime, sq));
+      }
     }
     {
+      ProfScope ps(kProfGram, sq);
+      if (tc) {
+        CA_TRY(launch_gram_tc(qp_hi, qp_lo, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, w.status, sq));
+      } else {
+        CA_TRY(launch_moments(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, w.partial2, w.gramQp, w.sumQp, sq));
+      }
+    }
+    {
+      ProfScope ps(kProfPca, sq);
       PcaArgs a{};
       a.mode = kPcaQueries;
       a.gram = w.gramQp; a.sum = w.sumQp; a.n = (double)p->n_q;
@@ -219,21 +306,28 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
       a.wt_hi = tc ? w.wt2_hi : nullptr; a.wt_lo = tc ? w.wt2_lo : nullptr;
       CA_TRY(launch_pca(a, P, D, sq));
     }
-    if (tc) {
-      CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
-                                 w.wt2_lo, w.status, sq, w.Ytq, true));
-    } else {
-      CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
+    {
+      ProfScope ps(kProfTransform, sq);
+      if (tc) {
+        CA_TRY(launch_transform_tc(qp_hi, qp_lo, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, nullptr, nullptr, w.wt2_hi,
+                                   w.wt2_lo, w.status, sq, w.Ytq, true));
+      } else {
+        CA_TRY(launch_transform_rows(w.Qprime, CA_DTYPE_FP32, P, p->n_q, D, EQ32, w.biasQ, 0, yq_out, sq));
+      }
     }
     CA_TRY(launch_split(yq_out, nullptr, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
                         perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 1, sq, w.Ytq, nullptr));
-    CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, sq));
-    CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
+    {
+      ProfScope ps(kProfPermute, sq);
+      CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, sq));
+    }
+    if (!serial) CA_RETURN_IF_CUDA(cudaEventRecord(side->join, sq));
     // ---- key side on the caller's stream: covariance of the transformed keys K F_q
     // (F_q^T C_K F_q / n_k, d x d algebra), its principal components E_K and the projection
     // W = F_q E_K with its bias in one kernel; Y = (K - kbar) W
-    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->mid, 0));
+    if (!serial) CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->mid, 0));
     {
+      ProfScope ps(kProfPca, st);
       PcaArgs a{};
       a.mode = kPcaKeys;
       a.gram = w.gramK; a.sum = w.sumK; a.n = (double)p->n_k; a.c_scale = ck_scale;
@@ -244,22 +338,29 @@ int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* 
       a.wt_hi = tc ? w.wt_hi : nullptr; a.wt_lo = tc ? w.wt_lo : nullptr;
       CA_TRY(launch_pca(a, P, D, st));
     }
-    if (tc) {
-      CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
-                                 w.wt_lo, w.status, st, w.Ytk, true));
-    } else {
-      CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
+    {
+      ProfScope ps(kProfTransform, st);
+      if (tc) {
+        CA_TRY(launch_transform_tc(K, nullptr, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, nullptr, nullptr, w.wt_hi,
+                                   w.wt_lo, w.status, st, w.Ytk, true));
+      } else {
+        CA_TRY(launch_transform_rows(K, p->dtype, P, p->n_k, D, w.WK32, w.biasK, 0, yk_out, st));
+      }
     }
     CA_TRY(launch_split(nullptr, yk_out, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
                         perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 2, st, nullptr, w.Ytk));
-    CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
+    {
+      ProfScope ps(kProfPermute, st);
+      CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
+    }
     // ---- join
-    CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->join, 0));
+    if (!serial) CA_RETURN_IF_CUDA(cudaStreamWaitEvent(st, side->join, 0));
     return CA_OK;
   }
   // coordinates given by the caller: split and gather only
   CA_TRY(launch_split(yq, yk, P, D, p->n_q, p->n_k, p->cluster_q, p->cluster_k, perm_q, w.perm_q_tmp,
                       perm_k, w.perm_k_tmp, w.keybuf_q, w.keybuf_k, 3, st));
+  ProfScope ps(kProfPermute, st);
   CA_TRY(launch_permute_centroid(Q, p->dtype, perm_q, P, p->n_q, D, p->cluster_q, Qp, cq, count_q, st));
   CA_TRY(launch_permute_centroid(K, p->dtype, perm_k, P, p->n_k, D, p->cluster_k, Kp, ck, count_k, st, V, Vp, cv));
   return CA_OK;
@@ -277,6 +378,7 @@ int select_blocks(const ca_problem_t* p, const float* cq, const float* ck, int32
   // room behind the status block holds tiles of scores when there are many key clusters
   float* score_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
   const size_t score_floats = aligned16(ws) ? (ws_bytes - kStatusBytes) / sizeof(float) : 0;
+  ProfScope ps(kProfSelect, st);
   return launch_score_select(cq, ck, P, ceil_div(p->n_q, p->cluster_q), ceil_div(p->n_k, p->cluster_k),
                              p->head_dim, p->keep, block_idx, score_ws, score_floats, st);
 }
@@ -316,6 +418,7 @@ int select_blocks_adaptive(const ca_problem_t* p, const float* cq, const float* 
   const float scale = p->softmax_scale > 0.f ? p->softmax_scale : 1.0f / sqrtf((float)p->head_dim);
   float* score_ws = reinterpret_cast<float*>(static_cast<char*>(ws) + kStatusBytes);
   const size_t score_floats = aligned16(ws) ? (ws_bytes - kStatusBytes) / sizeof(float) : 0;
+  ProfScope ps(kProfSelect, st);
   return launch_select_adaptive(cq, ck, count_k, p->batch * p->heads, ceil_div(p->n_q, p->cluster_q),
                                 ceil_div(p->n_k, p->cluster_k), p->head_dim, scale, recall, min_count,
                                 block_idx, keep_count, score_ws, score_floats, st);

@@ -695,6 +695,7 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   __nv_bfloat16* vb = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kHalf * D);
   int32_t* redo = c.take<int32_t>((size_t)P * n_qc * 2);
   if (pr.compensate) {
+    ProfScope ps(kProfAttnPrep, st);
     centroid_prep_kernel<<<dim3(ceil_div(cen_tiles * kHalf * D, 256), P), 256, 0, st>>>(ck, cv, n_kc, cen_tiles, D,
                                                                                         kmix, vb);
     CA_LAUNCH_CHECK();
@@ -718,8 +719,13 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   prm.wait_limit = g_wait_limit;
   prm.skip_key_load = g_skip_key_load;
   dim3 grid(n_qc * (pr.cluster_q >= kTile ? pr.cluster_q / kTile : 1), P);
-  const int rc = D == 64 ? launch_tc_d<64>(maps, prm, grid, st) : launch_tc_d<128>(maps, prm, grid, st);
+  int rc;
+  {
+    ProfScope ps(kProfAttn, st);
+    rc = D == 64 ? launch_tc_d<64>(maps, prm, grid, st) : launch_tc_d<128>(maps, prm, grid, st);
+  }
   if (rc != CA_OK) return rc;
+  ProfScope ps(kProfAttnSecond, st);
   // second pass: query tiles whose scores left the range of the fast softmax (a climb of more than
   // 2^96 within 64 keys) are recomputed by the fp32 kernel; its CTAs return at once for the others
   return launch_attn_ref(pr, Qp, Kp, Vp, ck, cv, count_k, block_idx, keep_count, list_stride, perm_q, scale, O, lse,

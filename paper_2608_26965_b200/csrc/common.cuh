@@ -36,6 +36,22 @@ inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
     }                                                       \
   } while (0)
 
+// Per-kernel-group device times (ca_profile / ca_profile_read of the public header).  A scope
+// records a pair of CUDA events around the launches it encloses when profiling is on.
+enum ProfGroup {
+  kProfGram = 0, kProfFactor, kProfPca, kProfTransform, kProfSplitLevels, kProfSplitTail, kProfPermute,
+  kProfSelect, kProfAttnPrep, kProfAttn, kProfAttnSecond, kProfGroups
+};
+bool prof_enabled();
+void prof_mark(int group, cudaStream_t st, bool begin);
+struct ProfScope {
+  int group;
+  cudaStream_t st;
+  bool on;
+  ProfScope(int g, cudaStream_t s) : group(g), st(s), on(prof_enabled()) { if (on) prof_mark(group, st, true); }
+  ~ProfScope() { if (on) prof_mark(group, st, false); }
+};
+
 template <typename T>
 __device__ __forceinline__ float to_f32(T x);
 template <>

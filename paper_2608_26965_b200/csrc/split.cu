@@ -675,6 +675,7 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
       }
     }
   };
+  if (top_levels > 0 && prof_enabled()) prof_mark(kProfSplitLevels, st, true);
   for (int level = 0; level < top_levels; ++level) {
     fill(level);
     prm.level = level;
@@ -698,6 +699,8 @@ int launch_split(const float* Yq, const float* Yk, int problems, int D, int n_q,
     CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, level_kernel, prm));
     CA_LAUNCH_CHECK();
   }
+  if (top_levels > 0 && prof_enabled()) prof_mark(kProfSplitLevels, st, false);
+  ProfScope ps(kProfSplitTail, st);
   fill(top_levels);       // any level >= both tails selects the tail buffers
   prm.level = top_levels;
   prm.smem_rows = 0;

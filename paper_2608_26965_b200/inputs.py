@@ -16,7 +16,9 @@ workload's storage type (bf16 workloads are rounded to bf16, nearest-even).
 """
 from __future__ import annotations
 
+import concurrent.futures
 import math
+import os
 from dataclasses import dataclass, replace
 from typing import Optional, Sequence, Tuple
 
@@ -166,7 +168,26 @@ def generate_head(w: Workload, head: int):
 
 
 def generate(w: Workload, heads: Optional[Sequence[int]] = None):
-    """Stacked [H', n, d] float32 arrays for the listed heads (default: all)."""
+    """Stacked [H', n, d] float32 arrays for the listed heads (default: all).  Heads are drawn
+    from their own generator streams, so they are produced side by side on the host's cores; the
+    values do not depend on how many threads run."""
     heads = list(range(w.heads)) if heads is None else list(heads)
-    parts = [generate_head(w, h) for h in heads]
-    return tuple(np.stack([p[i] for p in parts]) for i in range(3))
+    d = w.head_dim
+    out = (np.empty((len(heads), w.n_q, d), np.float32), np.empty((len(heads), w.n_k, d), np.float32),
+           np.empty((len(heads), w.n_k, d), np.float32))
+
+    def one(slot):
+        for dst, src in zip(out, generate_head(w, heads[slot])):
+            dst[slot] = src
+
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except AttributeError:
+        cores = os.cpu_count() or 1
+    workers = max(1, min(len(heads), cores))
+    if workers == 1:
+        one(0)
+    else:
+        with concurrent.futures.ThreadPoolExecutor(max_workers=workers) as pool:
+            list(pool.map(one, range(len(heads))))
+    return out

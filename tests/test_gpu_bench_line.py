@@ -33,3 +33,22 @@ def test_bench_line_has_the_contract_keys():
     assert line["gpu_launches"] > 0 and line["gpu_launches"] % line["steps"] == 0
     assert line["recomputed_clusters"] == 0                   # the timed path is the tensor-core kernel
     assert "sm_mhz" in line["clocks"] and "reasons" in line["clocks"]
+    assert line["clocks"]["samples"] > 0 and line["clocks"]["sm_mhz"] > 0     # even with five timed steps
+    # the clustering and selection kernels each against the roof that bounds them
+    stages = line["stage_rooflines"]
+    for name in ("gram", "transform", "split_levels", "split_tail", "permute_centroid"):
+        st = stages[name]
+        assert st["bound"] == "hbm" and st["ms"] > 0 and 0 < st["frac"] < 1.2
+        assert abs(st["frac"] - st["achieved"] / st["peak"]) < 1e-9
+    assert stages["score_select"]["bound"] == "alu" and 0 < stages["score_select"]["frac"] < 1.2
+    assert stages["principal_components"]["ms"] > 0
+    # the step's stages are made of these groups: their sum cannot be far below the clustering stage
+    clustering = sum(stages[n]["ms"] for n in ("gram", "cholesky_factor", "principal_components", "transform",
+                                               "split_levels", "split_tail", "permute_centroid"))
+    assert clustering > 0.8 * line["stage_ms"]["cluster_qk"]
+    # dense attention on the same GPU: torch's kernel and the library's own, the faster is the denominator
+    dense = line["dense"]
+    assert dense["library_ms"] > 0 and dense["fastest_ms"] == min(dense["library_ms"], dense["torch_sdpa_ms"])
+    assert dense["speedup_vs_fastest_dense"] > 1.0
+    sec = line["secondary"]
+    assert sec["workload"] == "video480" and sec["head_dim"] == 128 and 0 < sec["roofline"]["frac"] < 1.2
