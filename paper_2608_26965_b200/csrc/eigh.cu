@@ -6,109 +6,118 @@ namespace ca {
 
 // ---------------------------------------------------------------------------
 // Factor of a positive semi-definite matrix: lower-triangular F with F F^T = A
-// (right-looking Cholesky in double, one CTA per matrix).  A pivot that is not
-// above 1e-12 of the largest diagonal entry marks a direction in which the
-// (pseudo-)metric is zero: its column of F is set to zero, which is the
+// (right-looking Cholesky in double, one CTA of 8 d threads per matrix).  A pivot
+// that is not above 1e-12 of the largest diagonal entry marks a direction in
+// which the (pseudo-)metric is zero: its column of F is set to zero, which is the
 // counterpart of clamping small or negative eigenvalues (Section 3.2.2).
 // Any factor of the metric matrix gives the same principal-component
 // coordinates as its symmetric root, because the two differ by a rotation.
-// ---------------------------------------------------------------------------
+//
 // The matrix is formed on load from a Gram matrix and column sums: gram * scale (the query metric
 // M = Q^T Q / n_q, `sum` null) or (gram - s s^T / n) * scale (the centred scatter of the keys).
 // Besides F in double and float, F^T can be written as bf16 hi + lo parts, the layout in which the
 // tensor-core projection takes its weights (the query representation multiplies by F).
-template <int D>
-__global__ void __launch_bounds__(1024) cholesky_factor_kernel(const double* __restrict__ gram,
-                                                               const double* __restrict__ sum, double n,
-                                                               double scale, double* __restrict__ out64,
-                                                               float* __restrict__ out32,
-                                                               __nv_bfloat16* __restrict__ wt_hi,
-                                                               __nv_bfloat16* __restrict__ wt_lo) {
-  constexpr int LDA = D + 1;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  double* A = reinterpret_cast<double*>(smem_raw);       // [D][LDA], lower triangle is updated in place
-  __shared__ double s_tol;
-  __shared__ double s_inv, s_l10, s_inv1;
-  const int tid = threadIdx.x, NT = blockDim.x;
+//
+// Thread (r, q) = (tid / 8, tid % 8) keeps the entries k = q (mod 8) of row r of the lower triangle
+// in registers for the whole elimination.  Step j needs column j, which its owners publish to
+// shared memory during step j - 1 (right after their last update of it), so a step takes one
+// barrier; the trailing block takes A[i][k] -= A[i][j] A[k][j] / pivot_j with the unscaled
+// column, and the columns are scaled by 1 / sqrt(pivot) at the end.  The one division of a step
+// (double-precision division is slow on this part) is made by the thread that completes the next
+// pivot, also a step ahead.  A dropped pivot (reciprocal 0) leaves the trailing block alone and
+// gives a zero column.
+// ---------------------------------------------------------------------------
+template <int D, typename T>
+__global__ void __launch_bounds__(8 * D) cholesky_factor_kernel(const double* __restrict__ gram,
+                                                                const double* __restrict__ sum, double n,
+                                                                double scale, double* __restrict__ out64,
+                                                                float* __restrict__ out32,
+                                                                __nv_bfloat16* __restrict__ wt_hi,
+                                                                __nv_bfloat16* __restrict__ wt_lo) {
+  constexpr int PER = D / 8;
+  __shared__ T colbuf[2][D];       // column j of the trailing matrix, rows > j (two in rotation)
+  __shared__ T pivots[D];          // diagonal entries; afterwards 1 / sqrt(pivot) per column
+  __shared__ T s_ip[2];
+  __shared__ T s_tol;
+  const T kDrop = sizeof(T) == 8 ? (T)1e-12 : (T)1e-6;   // share of the largest diagonal entry below which a pivot drops out
+  const int tid = threadIdx.x;
+  const int r = tid >> 3, q = tid & 7;
   const double* G = gram + (size_t)blockIdx.x * D * D;
   const double* sm = sum ? sum + (size_t)blockIdx.x * D : nullptr;
-  for (int e = tid; e < D * D; e += NT) {
-    const int i = e / D, j = e % D;
-    const double centre = sm ? sm[i] * sm[j] / n : 0.0;
-    A[i * LDA + j] = (0.5 * (G[i * D + j] + G[j * D + i]) - centre) * scale;
+  // double-precision operations are scarce on this part: two per element here (the centring needs
+  // them: the Gram matrix is n mean^2 + scatter), none in the elimination
+  const double row_term = sm ? sm[r] * (scale / n) : 0.0;
+  T a[PER];
+#pragma unroll
+  for (int t = 0; t < PER; ++t) {
+    const int k = q + 8 * t;
+    a[t] = (T)0;
+    if (k <= r) a[t] = (T)(sm ? fma(-row_term, sm[k], G[r * D + k] * scale) : G[r * D + k] * scale);
+    if (k == r) pivots[r] = a[t];
+    if (k == 0) colbuf[0][r] = a[t];
   }
   __syncthreads();
-  if (tid == 0) {
-    double mx = 0.0;
-    for (int i = 0; i < D; ++i) mx = fmax(mx, A[i * LDA + i]);
-    s_tol = 1e-12 * mx;
-  }
-  __syncthreads();
-  // two columns per round (three barriers for the pair): thread 0 prepares both pivots -- the second
-  // one after its update by the first column -- then every row scales its two entries, then the
-  // trailing block takes the rank-2 update
-  for (int j = 0; j < D; j += 2) {
+  if (tid < 32) {
+    T mx = (T)0;
+    for (int i = tid; i < D; i += 32) mx = max(mx, pivots[i]);
+    for (int o = 16; o > 0; o >>= 1) mx = max(mx, __shfl_xor_sync(0xffffffffu, mx, o));
     if (tid == 0) {
-      const double piv0 = A[j * LDA + j];
-      const double inv0 = (piv0 > s_tol) ? rsqrt(piv0) : 0.0;
-      const double l10 = A[(j + 1) * LDA + j] * inv0;
-      const double piv1 = A[(j + 1) * LDA + j + 1] - l10 * l10;
-      s_inv = inv0;
-      s_l10 = l10;
-      s_inv1 = (piv1 > s_tol) ? rsqrt(piv1) : 0.0;
+      s_tol = kDrop * mx;
+      s_ip[0] = pivots[0] > kDrop * mx ? (T)1 / pivots[0] : (T)0;
     }
-    __syncthreads();
-    const double inv0 = s_inv, l10 = s_l10, inv1 = s_inv1;
-    // columns j and j+1 of F; a dropped pivot gives a zero column
-    for (int i = j + tid; i < D; i += NT) {
-      const double c0 = A[i * LDA + j] * inv0;
-      A[i * LDA + j] = c0;
-      if (i > j) A[i * LDA + j + 1] = (A[i * LDA + j + 1] - c0 * l10) * inv1;
-    }
-    __syncthreads();
-    // trailing update of the lower triangle
-    const int rem = D - 2 - j;
-    for (int e = tid; e < rem * rem; e += NT) {
-      const int i = j + 2 + e / rem, k = j + 2 + e % rem;
-      if (k <= i)
-        A[i * LDA + k] -= A[i * LDA + j] * A[k * LDA + j] + A[i * LDA + j + 1] * A[k * LDA + j + 1];
+  }
+  __syncthreads();
+  const T tol = s_tol;
+  for (int j = 0; j < D - 1; ++j) {
+    if (r > j) {                                          // rows up to j are final
+      const T* col = colbuf[j & 1];
+      const T f = col[r] * s_ip[j & 1];
+#pragma unroll
+      for (int t = 0; t < PER; ++t) {
+        if (8 * t + 7 <= j) continue;                     // uniform: these columns are final
+        const int k = q + 8 * t;
+        if (k > j && k <= r) {
+          a[t] -= f * col[k];
+          if (k == j + 1) {                               // column j + 1 is complete: publish it
+            colbuf[(j + 1) & 1][r] = a[t];
+            if (r == j + 1) s_ip[(j + 1) & 1] = a[t] > tol ? (T)1 / a[t] : (T)0;
+          }
+        }
+      }
     }
     __syncthreads();
   }
+#pragma unroll
+  for (int t = 0; t < PER; ++t)
+    if (q + 8 * t == r) pivots[r] = a[t];
+  __syncthreads();
+  if (tid < D) pivots[tid] = pivots[tid] > tol ? (T)rsqrt((double)pivots[tid]) : (T)0;
+  __syncthreads();
   double* o64 = out64 + (size_t)blockIdx.x * D * D;
   float* o32 = out32 ? out32 + (size_t)blockIdx.x * D * D : nullptr;
-  for (int e = tid; e < D * D; e += NT) {
-    const int i = e / D, j = e % D;
-    const double v = (j <= i) ? A[i * LDA + j] : 0.0;
-    o64[e] = v;
-    if (o32) o32[e] = (float)v;
-  }
-  if (wt_hi) {
-    // F^T [out j][in i] = F[i][j] as bf16 hi + lo
-    for (int e = tid; e < D * D; e += NT) {
-      const int j = e / D, i = e % D;
-      const float v = (j <= i) ? (float)A[i * LDA + j] : 0.f;
-      const __nv_bfloat16 h = __float2bfloat16_rn(v);
-      wt_hi[(size_t)blockIdx.x * D * D + e] = h;
-      wt_lo[(size_t)blockIdx.x * D * D + e] = __float2bfloat16_rn(v - __bfloat162float(h));
+#pragma unroll
+  for (int t = 0; t < PER; ++t) {
+    const int k = q + 8 * t;
+    const double v = (k <= r) ? (double)(a[t] * pivots[k]) : 0.0;
+    o64[r * D + k] = v;
+    if (o32) o32[r * D + k] = (float)v;
+    if (wt_hi) {                                          // F^T [out k][in r] = F[r][k] as bf16 hi + lo
+      const float vf = (float)v;
+      const __nv_bfloat16 h = __float2bfloat16_rn(vf);
+      wt_hi[(size_t)blockIdx.x * D * D + (size_t)k * D + r] = h;
+      wt_lo[(size_t)blockIdx.x * D * D + (size_t)k * D + r] = __float2bfloat16_rn(vf - __bfloat162float(h));
     }
   }
 }
 
+typedef double CholT;   // arithmetic of the elimination (float32 was measured: no faster, and less exact)
+
 int launch_cholesky_factor(const double* gram, const double* sum, double n, double scale, int count, int D,
                            double* out64, float* out32, void* wt_hi, void* wt_lo, cudaStream_t st) {
-  const size_t smem = sizeof(double) * D * (D + 1);
   __nv_bfloat16* hi = static_cast<__nv_bfloat16*>(wt_hi);
   __nv_bfloat16* lo = static_cast<__nv_bfloat16*>(wt_lo);
-  if (D == 64) {
-    auto k = cholesky_factor_kernel<64>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, 512, smem, st>>>(gram, sum, n, scale, out64, out32, hi, lo);
-  } else {
-    auto k = cholesky_factor_kernel<128>;
-    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    k<<<count, 1024, smem, st>>>(gram, sum, n, scale, out64, out32, hi, lo);
-  }
+  if (D == 64) cholesky_factor_kernel<64, CholT><<<count, 8 * 64, 0, st>>>(gram, sum, n, scale, out64, out32, hi, lo);
+  else cholesky_factor_kernel<128, CholT><<<count, 8 * 128, 0, st>>>(gram, sum, n, scale, out64, out32, hi, lo);
   CA_LAUNCH_CHECK();
   return CA_OK;
 }

@@ -113,11 +113,13 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   }
   if (a.mode == kPcaKeys) {
     // C = (gram - s s^T / n) c_scale, the centred scatter of the keys; then alpha F^T C F
+    // (double-precision operations are scarce on this part: no division per element)
     const double* G = a.gram + mat;
     const double* sm = a.sum + (size_t)blockIdx.x * D;
+    const double cs = a.c_scale, cn = a.c_scale / a.n;
     for (int e = tid; e < D * D; e += NT) {
       const int i = e / D, j = e % D;
-      A[i * LDA + j] = (float)((G[e] - sm[i] * sm[j] / a.n) * a.c_scale);
+      A[i * LDA + j] = (float)fma(-cn * sm[i], sm[j], G[e] * cs);
     }
     __syncthreads();
     float acc[CH][4];
@@ -136,9 +138,10 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
     // covariance of the stored representation: gram / n - mean mean^T
     const double* G = a.gram + mat;
     const double* sm = a.sum + (size_t)blockIdx.x * D;
+    const double inv_n = 1.0 / a.n, inv_n2 = inv_n * inv_n;
     for (int e = tid; e < D * D; e += NT) {
       const int i = e / D, j = e % D;
-      A[i * LDA + j] = (float)(G[e] / a.n - (sm[i] / a.n) * (sm[j] / a.n));
+      A[i * LDA + j] = (float)fma(-inv_n2 * sm[i], sm[j], G[e] * inv_n);
     }
   } else {
     const double* Ain = a.A_in + mat;
