@@ -29,6 +29,10 @@ Pins (tests/test_oracle_*.py):
                            exact SMC error decomposition (Appendix A)
   *_f32 helpers .......... hand-computed sums whose bits depend on the order of the additions;
                            the fp64 decisions on inputs without near-ties
+  round_to_minifloat / quantize_* / cluster_attention_quantized_qk ... the table of all E4M3
+                           numbers written out from the format's definition, hand-rounded values,
+                           a hand-computed 2 x 2 case, and the limit of many mantissa bits
+                           (= the unquantised attention)
 Decisions (which coordinate a split takes, which key clusters are kept) are DEFINED by the
 float64 functions `choose_coordinate`, `centroid_scores` + `select_topk`.  The `_f32` functions
 beside them restate the same quantities in float32 with a fixed operation order; they exist so
@@ -536,6 +540,91 @@ def cluster_attention(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx, compensate,
         O[rows] = (e / z) @ values
         lse[rows] = (mx + np.log(z))[:, 0]
     return O, lse
+
+
+# --------------------------------------------------------------------------
+# Quantised Q K^T (Section 3.1: the block-sparse kernel the paper runs is a
+# quantised one; Section 5.1 names "the quantization in the kernel we use" as a
+# source of its error).  The paper does not print that kernel's scheme; the
+# variant defined here is: queries and keys are stored as 8-bit floating point
+# numbers with 4 exponent and 3 mantissa bits (E4M3: bias 7, largest finite
+# value 448, no infinities, subnormals down to 2^-9), each query ROW with its own
+# scale, each key CLUSTER with one scale, the key centroids of the compensation
+# with one scale per run of 64 centroids; probabilities and values are not
+# quantised.  A scale maps the largest magnitude of its group to 448.  Because
+# floating point decides the stored codes, scales and scaled values are taken in
+# float32 with IEEE operations that any implementation reproduces bit for bit:
+#   amax = max |x| over the group;  inv = 448 / amax;  s = amax / 448
+#   (both 0 when amax is 0);  code = E4M3(x * inv), round to nearest, ties to
+#   even, saturating;  the value the logits see is  s * code.
+# Products of two such values and their sums are then exact in float64, so the
+# quantised attention is `cluster_attention` on the de-quantised tensors.
+# `man_bits` generalises the format (more mantissa bits, same exponent range):
+# with enough of them the quantisation disappears, which pins the rest.
+# --------------------------------------------------------------------------
+def round_to_minifloat(y, man_bits=3, min_exp=-6, max_value=448.0):
+    """Rounds float values to the nearest number of the form +-(1 + m / 2^man_bits) 2^e,
+    e >= min_exp, or +-(m / 2^man_bits) 2^min_exp below that (subnormals); ties go to the even
+    mantissa; magnitudes beyond max_value saturate.  Exact arithmetic in float64."""
+    y = np.asarray(y, F64)
+    mag = np.abs(y)
+    e = np.floor(np.log2(np.where(mag > 0, mag, 1.0)))
+    e = np.maximum(e, min_exp)
+    step = np.exp2(e - man_bits)                    # spacing of the representable numbers around |y|
+    q = np.rint(mag / step) * step                  # np.rint rounds halves to even
+    q = np.minimum(q, max_value)
+    return np.sign(y) * q
+
+
+def quantize_group_e4m3(x32, man_bits=3):
+    """One group with one scale.  Returns (s, codes) with the de-quantised values s * codes."""
+    x32 = np.asarray(x32, np.float32)
+    amax = np.float32(np.abs(x32).max()) if x32.size else np.float32(0)
+    if amax == 0:
+        return np.float32(0), np.zeros(x32.shape, F64)
+    inv = np.float32(448.0) / amax                  # float32 division
+    s = amax / np.float32(448.0)
+    scaled = (x32 * inv).astype(np.float32)         # float32 product
+    return s, round_to_minifloat(scaled, man_bits)
+
+
+def quantize_qk(Q, K, perm_k, c_k, ck=None, man_bits=3):
+    """De-quantised (Q~, K~, ck~) of the scheme above: per query row, per key cluster (the rows
+    perm_k[j c_k : (j+1) c_k]), per run of 64 key centroids.  float64 arrays."""
+    Q = np.asarray(Q, np.float32)
+    K = np.asarray(K, np.float32)
+    Qd = np.zeros(Q.shape, F64)
+    for r in range(Q.shape[0]):
+        s, code = quantize_group_e4m3(Q[r], man_bits)
+        Qd[r] = F64(s) * code
+    Kd = np.zeros(K.shape, F64)
+    N_k = K.shape[0]
+    for j in range(-(-N_k // c_k)):
+        rows = perm_k[j * c_k:min((j + 1) * c_k, N_k)]
+        s, code = quantize_group_e4m3(K[rows], man_bits)
+        Kd[rows] = F64(s) * code
+    ckd = None
+    if ck is not None:
+        ck = np.asarray(ck, np.float32)
+        ckd = np.zeros(ck.shape, F64)
+        for j0 in range(0, ck.shape[0], 64):
+            s, code = quantize_group_e4m3(ck[j0:j0 + 64], man_bits)
+            ckd[j0:j0 + 64] = F64(s) * code
+    return Qd, Kd, ckd
+
+
+def cluster_attention_quantized_qk(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx, compensate,
+                                   ck=None, cv=None, count_k=None, scale=None, query_clusters=None, man_bits=3):
+    """`cluster_attention` with Q K^T (and the centroid logits) taken on the quantised queries, keys
+    and key centroids; values, value centroids and counts as given."""
+    if compensate and ck is None:
+        ck, count_k = centroids(K, perm_k, c_k)
+        ck = ck.astype(np.float32)
+    if compensate and cv is None:
+        cv, _ = centroids(V, perm_k, c_k)
+    Qd, Kd, ckd = quantize_qk(Q, K, perm_k, c_k, ck if compensate else None, man_bits)
+    return cluster_attention(Qd, Kd, V, perm_q, perm_k, c_q, c_k, block_idx, compensate, ck=ckd, cv=cv,
+                             count_k=count_k, scale=scale, query_clusters=query_clusters)
 
 
 # --------------------------------------------------------------------------

@@ -690,3 +690,88 @@ def test_forward_pipeline_shapes_and_convergence_to_dense():
         assert sorted(cl["perm_k"].tolist()) == list(range(256))
         errs.append(np.abs(o - od).max())
     assert errs[2] < 1e-12 and errs[0] > errs[1] > errs[2]
+
+
+# ------------------------------------------------ quantised Q K^T (Section 3.1, Section 5.1)
+def _all_e4m3_values():
+    """Every finite non-negative E4M3 number from the format's definition: 4 exponent bits (bias 7),
+    3 mantissa bits, exponent field 0 = subnormals, the all-ones code is not a number."""
+    vals = [m / 8.0 * 2.0 ** -6 for m in range(8)]
+    for e in range(1, 16):
+        for m in range(8):
+            if e == 15 and m == 7:
+                continue
+            vals.append((1 + m / 8.0) * 2.0 ** (e - 7))
+    return np.array(vals)
+
+
+def test_e4m3_rounding_matches_the_format():
+    vals = _all_e4m3_values()
+    assert len(vals) == 127 and vals.max() == 448.0 and vals[1] == 2.0 ** -9
+    # representable numbers are fixed points, both signs
+    assert np.array_equal(orc.round_to_minifloat(vals), vals)
+    assert np.array_equal(orc.round_to_minifloat(-vals), -vals)
+    # every real rounds to the nearest table entry; exact halves go to the even mantissa
+    r = rng(60)
+    y = np.concatenate([r.uniform(0, 460, 4000), r.uniform(0, 0.05, 2000), 2.0 ** r.uniform(-12, 9, 2000)])
+    got = orc.round_to_minifloat(y)
+    nearest = vals[np.abs(y[:, None] - vals[None, :]).argmin(axis=1)]
+    assert np.array_equal(got, nearest)
+    assert orc.round_to_minifloat(1.0625) == 1.0            # half-way between 1 (mantissa 000) and 1.125 (001)
+    assert orc.round_to_minifloat(1.1875) == 1.25           # half-way between 1.125 (001) and 1.25 (010)
+    assert orc.round_to_minifloat(2.0 ** -10) == 0.0        # half-way between 0 and the smallest subnormal
+    assert orc.round_to_minifloat(3 * 2.0 ** -10) == 2.0 ** -8
+    assert orc.round_to_minifloat(1e9) == 448.0 and orc.round_to_minifloat(-465.0) == -448.0
+    assert orc.round_to_minifloat(464.0) == 448.0           # beyond the largest number: saturates
+
+
+def test_group_quantisation_scales_the_largest_magnitude_to_448():
+    x = np.array([[0.5, -3.0, 1.0], [0.0, 2.9, -0.011]], np.float32)
+    s, code = orc.quantize_group_e4m3(x)
+    assert s == np.float32(3.0) / np.float32(448.0) and code[0, 1] == -448.0
+    # by hand: inv = 448/3; 0.5 * inv = 74.67 -> spacing 8 in [64, 128): 72;  1.0 * inv = 149.33 -> spacing 16: 144
+    assert code[0, 0] == 72.0 and code[0, 2] == 144.0 and code[1, 0] == 0.0
+    assert code[1, 1] == 448.0                              # 433.07 -> spacing 32 in [256, 512): 416 or 448, nearer 448
+    assert code[1, 2] == -1.625                             # -1.6427 -> spacing 0.125 in [1, 2): -1.625
+    zero_s, zero_code = orc.quantize_group_e4m3(np.zeros((2, 3), np.float32))
+    assert zero_s == 0 and not zero_code.any()
+
+
+def test_quantised_attention_two_by_two_by_hand():
+    # one query, two keys in two clusters of one key each, d = 2, both kept
+    Q = np.array([[1.0, 0.3]], np.float32)
+    K = np.array([[2.0, 0.1], [-1.0, 1.0]], np.float32)
+    V = np.array([[1.0, 0.0], [0.0, 1.0]])
+    o, lse = orc.cluster_attention_quantized_qk(Q, K, V, np.arange(1), np.arange(2), 1, 1, np.array([[0, 1]]), False,
+                                                scale=1.0)
+    # query row: amax 1, inv 448: codes (448, 134.4 -> spacing 16: 128) -> (1, 128/448)
+    # key 0: amax 2: codes (448, 22.4 -> spacing 2 in [16, 32): 22) -> (2, 2 * 22/448);  key 1: amax 1: (-1, 1) exact
+    q = np.array([1.0, 128.0 / 448.0])
+    k0 = np.array([2.0, 2.0 * 22.0 / 448.0])
+    k1 = np.array([-1.0, 1.0])
+    l0, l1 = q @ k0, q @ k1
+    w0 = 1.0 / (1.0 + np.exp(l1 - l0))
+    assert np.allclose(o[0], [w0, 1 - w0], atol=1e-6)       # float32 scales: 1e-7 relative
+    assert np.isclose(lse[0], np.log(np.exp(l0) + np.exp(l1)), atol=1e-6)
+
+
+def test_quantised_attention_tends_to_the_unquantised_one():
+    r, Q, K, V, pq, pk, c = _setup(61, N_k=58)
+    Q, K = Q.astype(np.float32), K.astype(np.float32)
+    idx = np.stack([np.sort(r.choice(15, 4, replace=False)) for _ in range(12)])
+    ck, cnt = orc.centroids(K, pk, c)
+    ck32 = ck.astype(np.float32)
+    exact, lse_exact = orc.cluster_attention(Q, K, V, pq, pk, c, c, idx, True, ck=ck32, count_k=cnt)
+    errs = []
+    for bits in (3, 7, 12, 23):
+        o, lse = orc.cluster_attention_quantized_qk(Q, K, V, pq, pk, c, c, idx, True, ck=ck32, count_k=cnt, man_bits=bits)
+        errs.append(np.abs(o - exact).max())
+    assert errs[0] > errs[1] > errs[2] > errs[3]            # every added mantissa bit brings it closer
+    assert errs[0] > 1e-3 and errs[3] < 2e-6                # 3 bits matter; 23 bits leave float32 rounding of the scales
+    # the scales alone do not change anything that the codes do not: a tensor of representable
+    # numbers with group maximum 448 passes through unchanged
+    vals = _all_e4m3_values()
+    X = r.choice(vals, (6, 8)).astype(np.float32)
+    X[:, 0] = 448.0
+    Qd, Kd, _ = orc.quantize_qk(X, X, np.arange(6), 2)
+    assert np.array_equal(Qd, X.astype(np.float64)) and np.array_equal(Kd, X.astype(np.float64))
