@@ -53,6 +53,7 @@ enum {
   CA_ATTN_FP32 = 2, /* cluster_attention_fwd: force the FP32 CUDA-core kernel for bf16 data  */
   CA_METRIC_IN = 8, /* cluster_qk_basic: A_q / A_k hold the metric matrices (used by tests to feed
                        both sides the same float32 matrices)                                */
+  CA_ATTN_FP8_QK = 16, /* cluster_attention_fwd: Q K^T on 8-bit floating point operands (see there) */
   CA_QUERY_UNNORMALIZED = 4 /* cluster_qk: queries are represented by R_k q with
                        R_k = sqrt(K_c^T K_c / n_k), without the division by the norm: the
                        form that goes with adaptive selection (Section 3.2.2, Appendix B.1) */
@@ -68,7 +69,7 @@ typedef struct {
   int32_t keep;            /* kept key clusters per query cluster, 1 .. ceil(n_k/c_k)        */
   int32_t compensate;      /* 0/1: striped mean-compensation off/on                          */
   float softmax_scale;     /* 0 selects 1/sqrt(head_dim)                                     */
-  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32 | CA_QUERY_UNNORMALIZED | CA_METRIC_IN  */
+  int32_t flags;           /* CA_Y_IN | CA_ATTN_FP32 | CA_QUERY_UNNORMALIZED | CA_METRIC_IN | CA_ATTN_FP8_QK */
 } ca_problem_t;
 
 /* Bytes of workspace each stage needs for this problem (any pointer may be NULL). */
@@ -177,6 +178,18 @@ int select_blocks(const ca_problem_t* p, const float* cq, const float* ck,
  * bf16 storage runs on tcgen05 tensor cores with fp32 accumulation (head_dim
  * 64/128, c_q in {64, 128, 256}, c_k in 16..256); fp32 storage, other sizes, or
  * CA_ATTN_FP32 run the FP32 CUDA-core kernel.
+ *
+ * CA_ATTN_FP8_QK (off by default; bf16 storage, head_dim 128, c_k >= 64, else
+ * CA_ERR_UNSUPPORTED): the variant with a quantised Q K^T (Section 3.1: the kernel
+ * the paper runs is a quantised one; Section 5.1).  Queries, keys and the key
+ * centroids of the compensation are turned into E4M3 codes (4 exponent bits, 3
+ * mantissa bits, largest value 448) inside the call: one scale per query row, per
+ * key cluster and per run of 64 key centroids, scale = (largest magnitude of the
+ * group) / 448, code = E4M3(x * (448 / largest magnitude)) rounded to nearest even,
+ * all in float32.  The logits are (code_q . code_k) * scale_q * scale_k * s; the
+ * probabilities, the values and the value centroids are not quantised.  The
+ * workspace is larger (ca_workspace_bytes with the flag set).  Query tiles that the
+ * second pass recomputes (see ca_attn_recomputed) are recomputed unquantised.
  */
 int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
                           const void* Vp, const float* ck, const float* cv,

@@ -24,7 +24,7 @@ CA_ERR_BAD_INDEX = 6
 ERRORS = {1: "CA_ERR_INVALID_ARG", 2: "CA_ERR_UNSUPPORTED", 3: "CA_ERR_WORKSPACE", 4: "CA_ERR_CUDA",
           5: "CA_ERR_TIMEOUT", 6: "CA_ERR_BAD_INDEX"}
 CA_DTYPE_FP32, CA_DTYPE_BF16 = 0, 1
-CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN = 1, 2, 4, 8
+CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN, CA_ATTN_FP8_QK = 1, 2, 4, 8, 16
 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_attn_recomputed", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",

@@ -391,6 +391,7 @@ int cluster_attention_fwd(const ca_problem_t* p, const void* Qp, const void* Kp,
   const void* ptrs[] = {Qp, Kp, Vp, ck, cv, count_k, block_idx, perm_q, O};
   for (const void* x : ptrs)
     if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
+  if ((p->flags & CA_ATTN_FP8_QK) && !attn_tc_fp8_supported(*p)) return CA_ERR_UNSUPPORTED;
   const bool tensor_cores = attn_tc_supported(*p);
   const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;
@@ -434,6 +435,7 @@ int cluster_attention_fwd_ragged(const ca_problem_t* p, const void* Qp, const vo
   for (const void* x : ptrs)
     if (!x || !aligned16(x)) return CA_ERR_INVALID_ARG;
   if (list_stride < 1) return CA_ERR_INVALID_ARG;
+  if ((p->flags & CA_ATTN_FP8_QK) && !attn_tc_fp8_supported(*p)) return CA_ERR_UNSUPPORTED;
   const bool tensor_cores = attn_tc_supported(*p);
   const size_t need = tensor_cores ? attn_tc_workspace_bytes(*p) : kStatusBytes;
   if (!ws || !aligned16(ws) || ws_bytes < need) return CA_ERR_WORKSPACE;

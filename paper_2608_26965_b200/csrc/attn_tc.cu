@@ -45,13 +45,20 @@ constexpr int kHalf = 64;                  // keys per half-step
 constexpr float kRescaleThreshold = 8.0f;  // log2 units
 constexpr float kDanger = 96.0f;            // log2 units: exp2 arguments stay below this
 
-template <int D>
+// F8: queries, keys and key centroids arrive as E4M3 codes (one byte per element: a 128-byte row
+// of a panel holds 128 of them) and Q K^T runs as kind::f8f6f4 products; values stay bf16.
+template <int D, bool F8 = false>
 struct TcCfg {
-  static constexpr int PANELS = D / 64;
+  static constexpr int PANELS = D / 64;                      // value panels (bf16: 64 elements per 128-byte row)
+  static constexpr int QK_PANELS = F8 ? D / 128 : D / 64;    // query / key panels
+  static constexpr int QK_PANEL_COLS = F8 ? 128 : 64;        // elements per panel row
+  static constexpr int QK_KSTEP = F8 ? 32 : 16;              // elements per tensor-core instruction (32 bytes)
   static constexpr int PANEL_BYTES = kTile * 128;            // query tile: 128 rows x 128 bytes per panel
-  static constexpr int TILE_BYTES = PANELS * PANEL_BYTES;
+  static constexpr int TILE_BYTES = QK_PANELS * PANEL_BYTES;
   static constexpr int HALF_PANEL_BYTES = kHalf * 128;       // key/value slot: 64 rows x 128 bytes per panel
-  static constexpr int HALF_BYTES = PANELS * HALF_PANEL_BYTES;
+  static constexpr int HALF_BYTES = PANELS * HALF_PANEL_BYTES;        // a value slot
+  static constexpr int KHALF_BYTES = QK_PANELS * HALF_PANEL_BYTES;    // a key slot
+  static constexpr int CEN_PARTS = F8 ? 1 : 2;               // key slots of a centroid half-step (bf16: hi and lo parts)
   // Per CTA the half-steps form one dependent chain (scores -> softmax -> P V -> next scores) whose
   // length is set by latencies, not by any pipe, and an SM has throughput to spare: what counts is
   // the number of such chains per SM.  d = 64: one 64-column score buffer + 64 output columns =
@@ -74,7 +81,7 @@ struct TcCfg {
   // shared memory layout (offsets from a 1024-byte aligned base)
   static constexpr int OFF_Q = 0;
   static constexpr int OFF_K = OFF_Q + TILE_BYTES;
-  static constexpr int OFF_V = OFF_K + NK * HALF_BYTES;
+  static constexpr int OFF_V = OFF_K + NK * KHALF_BYTES;
   static constexpr int OFF_BIAS = OFF_V + NV * HALF_BYTES;                     // 8 x 64 floats
   static constexpr int OFF_BAR = OFF_BIAS + 8 * kHalf * 4;
   static constexpr int NUM_BARS = 3 + 3 * NBAR + NK + NV;           // q_full, o_done, q_tmem, three rings, per slot
@@ -93,6 +100,11 @@ struct TcParams {
   int32_t* redo;                  // [B*H, n_qc, 2] per CTA: scores left the range of the fast softmax
   int n_q, n_k, c_q, c_k, keep, list_stride, n_qc, n_kc, cen_tiles, compensate, bitmap_words;
   float scale_log2;
+  // quantised Q K^T: de-quantisation scales of the query rows [B*H*n_qc*c_q], of the key clusters
+  // [B*H*n_kc] and of the runs of 64 key centroids [B*H*cen_tiles]; null otherwise
+  const float* q_scale;
+  const float* k_scale;
+  const float* c_scale;
   long long wait_limit;           // SM cycles after which a barrier wait gives up (CA_ERR_TIMEOUT)
   int skip_key_load;              // diagnostic hook: the loader leaves out the keys of this half-step (-1: none)
 };
@@ -104,12 +116,12 @@ __host__ __device__ inline int selected_tiles(int keep, int c_k) {
   return c_k >= kTile ? keep * (c_k / kTile) : (keep * c_k + kTile - 1) / kTile;
 }
 
-template <int D>
-__global__ void __launch_bounds__(kTcThreads, TcCfg<D>::CTAS_PER_SM)
+template <int D, bool F8>
+__global__ void __launch_bounds__(kTcThreads, TcCfg<D, F8>::CTAS_PER_SM)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_ck,
                const __grid_constant__ CUtensorMap tm_cv, const TcParams prm) {
-  using C = TcCfg<D>;
+  using C = TcCfg<D, F8>;
   extern __shared__ unsigned char smem_unaligned[];
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_unaligned) + 1023) & ~uintptr_t(1023));
@@ -130,6 +142,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   // member counts of the selected clusters, in list order: looked up every half-step, so they are
   // fetched from global memory once instead of sitting on each half-step's critical path
   uint16_t* members_of = reinterpret_cast<uint16_t*>(bitmap + prm.bitmap_words);
+  // quantised Q K^T: de-quantisation scale of every selected key cluster, in list order
+  float* kscale_of = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(members_of) +
+                                              (((size_t)prm.list_stride * 2 + 15) & ~(size_t)15));
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int p = blockIdx.y;
@@ -161,7 +176,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   }
   if (q_rows < kTile) {
     // rows [q_rows, 128) of every Q panel: zeros (read by the tensor core through the async proxy)
-    for (int e = tid; e < C::PANELS * (kTile - q_rows) * 8; e += kTcThreads) {
+    for (int e = tid; e < C::QK_PANELS * (kTile - q_rows) * 8; e += kTcThreads) {
       const int pn = e / ((kTile - q_rows) * 8), rem = e % ((kTile - q_rows) * 8);
       *reinterpret_cast<uint4*>(smem + C::OFF_Q + pn * C::PANEL_BYTES + q_rows * 128 + rem * 16) = make_uint4(0u, 0u, 0u, 0u);
     }
@@ -177,7 +192,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
   const uint32_t tmem_s = tmem_base, tmem_o = tmem_base + C::NBUF * kHalf;
   // key slots used before half-step u (a centroid half-step takes two: hi and lo parts)
-  auto kslot_of = [&](int u) { return u < 2 * sel_tiles ? u : 2 * sel_tiles + 2 * (u - 2 * sel_tiles); };
+  auto kslot_of = [&](int u) { return u < 2 * sel_tiles ? u : 2 * sel_tiles + C::CEN_PARTS * (u - 2 * sel_tiles); };
 
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
@@ -188,27 +203,31 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     if (lane == 0) {
       prefetch_tensormap(&tm_q); prefetch_tensormap(&tm_k); prefetch_tensormap(&tm_v);
       const int q_row = (p * prm.n_qc + qc) * prm.c_q + half * kTile;
-      mbar_expect_tx(b_q_full, C::PANELS * q_rows * 128);
-      for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(s_q + pn * C::PANEL_BYTES, &tm_q, pn * 64, q_row, b_q_full);
+      mbar_expect_tx(b_q_full, C::QK_PANELS * q_rows * 128);
+      for (int pn = 0; pn < C::QK_PANELS; ++pn)
+        tma_load_2d(s_q + pn * C::PANEL_BYTES, &tm_q, pn * C::QK_PANEL_COLS, q_row, b_q_full);
       bool ok = true;
-      auto load_rows = [&](uint32_t dst, const CUtensorMap* map, int row, uint32_t bar) {
-        for (int pn = 0; pn < C::PANELS; ++pn) tma_load_2d(dst + pn * C::HALF_PANEL_BYTES, map, pn * 64, row, bar);
+      // `key`: rows of keys or key centroids (their panels), otherwise rows of values
+      auto load_rows = [&](uint32_t dst, const CUtensorMap* map, int row, uint32_t bar, bool key) {
+        const int panels = key ? C::QK_PANELS : C::PANELS, cols = key ? C::QK_PANEL_COLS : 64;
+        for (int pn = 0; pn < panels; ++pn) tma_load_2d(dst + pn * C::HALF_PANEL_BYTES, map, pn * cols, row, bar);
       };
       // the 64 rows of half-step u of the selected clusters: one box, or several boxes of c_k rows
-      auto load_selected = [&](uint32_t dst, const CUtensorMap* map, int u, uint32_t bar) {
+      auto load_selected = [&](uint32_t dst, const CUtensorMap* map, int u, uint32_t bar, bool key) {
         if (prm.c_k >= kHalf) {
           const int pos = u * kHalf;                       // position in the concatenated selected rows
           int j = sel[min(pos / prm.c_k, keep - 1)];     // a filler half-step repeats the last cluster (masked)
           j = min(max(j, 0), prm.n_kc - 1);                // out-of-range entries are flagged and masked by the softmax warps
-          load_rows(dst, map, (p * prm.n_kc + j) * prm.c_k + pos % prm.c_k, bar);
+          load_rows(dst, map, (p * prm.n_kc + j) * prm.c_k + pos % prm.c_k, bar, key);
         } else {
           const int per = kHalf / prm.c_k;
           for (int x = 0; x < per; ++x) {
             int e = u * per + x;
             if (e >= keep) e = keep - 1;                   // filler rows, masked by the softmax
             const int j = min(max(sel[e], 0), prm.n_kc - 1);
-            for (int pn = 0; pn < C::PANELS; ++pn)
-              tma_load_2d(dst + pn * C::HALF_PANEL_BYTES + x * prm.c_k * 128, map, pn * 64,
+            const int panels = key ? C::QK_PANELS : C::PANELS, cols = key ? C::QK_PANEL_COLS : 64;
+            for (int pn = 0; pn < panels; ++pn)
+              tma_load_2d(dst + pn * C::HALF_PANEL_BYTES + x * prm.c_k * 128, map, pn * cols,
                           (p * prm.n_kc + j) * prm.c_k, bar);
           }
         }
@@ -220,16 +239,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       for (int i = 0; i < steps + C::NBUF && ok; ++i) {
         if (i < steps) {
           const bool centroid = i >= 2 * sel_tiles;
-          const int parts = centroid ? 2 : 1;
+          const int parts = centroid ? C::CEN_PARTS : 1;
           const int w = i - (centroid ? C::K_LEAD_CEN : C::K_LEAD);
           if (w >= 0) ok = mbar_wait_relaxed(b_s_full(w % C::NBAR), (w / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit);
           for (int g = 0; g < parts && ok; ++g) {
             const int kc = kslot_of(i) + g, slot = kc % C::NK;
             if (i == prm.skip_key_load) continue;          // diagnostic: this slot never fills, its waiters time out
-            mbar_expect_tx(b_k_full(slot), C::HALF_BYTES);
-            const uint32_t dst = s_k + slot * C::HALF_BYTES;
-            if (!centroid) load_selected(dst, &tm_k, i, b_k_full(slot));
-            else load_rows(dst, &tm_ck, (p * prm.cen_tiles + (i - 2 * sel_tiles)) * kTile + g * kHalf, b_k_full(slot));
+            mbar_expect_tx(b_k_full(slot), C::KHALF_BYTES);
+            const uint32_t dst = s_k + slot * C::KHALF_BYTES;
+            if (!centroid) load_selected(dst, &tm_k, i, b_k_full(slot), true);
+            else load_rows(dst, &tm_ck, (p * prm.cen_tiles + (i - 2 * sel_tiles)) * (C::CEN_PARTS * kHalf) + g * kHalf,
+                           b_k_full(slot), true);
           }
         }
         const int j = i - C::NBUF;
@@ -240,8 +260,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
           if (!ok) break;
           mbar_expect_tx(b_v_full(slot), C::HALF_BYTES);
           const uint32_t dst = s_v + slot * C::HALF_BYTES;
-          if (j < 2 * sel_tiles) load_selected(dst, &tm_v, j, b_v_full(slot));
-          else load_rows(dst, &tm_cv, (p * prm.cen_tiles + (j - 2 * sel_tiles)) * kHalf, b_v_full(slot));
+          if (j < 2 * sel_tiles) load_selected(dst, &tm_v, j, b_v_full(slot), false);
+          else load_rows(dst, &tm_cv, (p * prm.cen_tiles + (j - 2 * sel_tiles)) * kHalf, b_v_full(slot), false);
         }
       }
     }
@@ -250,7 +270,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     // every lane runs the loop (waits and descriptor arithmetic stay warp-uniform); one elected
     // lane issues the tensor-core instructions
     {
-      constexpr uint32_t idesc_qk = idesc_bf16_f32(kTile, kHalf, 0, 0);
+      constexpr uint32_t idesc_qk = F8 ? idesc_e4m3_f32(kTile, kHalf) : idesc_bf16_f32(kTile, kHalf, 0, 0);
       constexpr uint32_t idesc_pv = idesc_bf16_f32(kTile, C::PV_N, 0, 1);
       bool ok = __all_sync(0xffffffffu, mbar_wait(b_q_full, 0, abort_flag, prm.status, prm.wait_limit));
       // descriptors differ from a base one only in the start-address field (units of 16 bytes):
@@ -263,7 +283,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // value slots (loaded long before) and their descriptors -- is waited for and computed BEFORE
       // the wait for the softmax, and P V (u) and S(u + NBUF) are then issued back to back.
       auto wait_keys = [&](int un) {
-        const int parts = un >= 2 * sel_tiles ? 2 : 1;      // centroid keys: bf16 hi parts, then lo parts
+        const int parts = un >= 2 * sel_tiles ? C::CEN_PARTS : 1;      // centroid keys as bf16: hi parts, then lo parts
         bool got = true;
         for (int g = 0; g < parts && got; ++g) {
           const int kc = kslot_of(un) + g;
@@ -274,13 +294,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // first key slot and number of parts of S(un); fire_s (elected lane) issues it
       auto fire_s = [&](uint32_t d_cols, int kc0, int parts, uint32_t bar) {
         for (int g = 0; g < parts; ++g) {
-          const uint64_t kd = k_desc0 + ((((kc0 + g) % C::NK) * C::HALF_BYTES) >> 4);
+          const uint64_t kd = k_desc0 + ((((kc0 + g) % C::NK) * C::KHALF_BYTES) >> 4);
 #pragma unroll
-          for (int ks = 0; ks < D / 16; ++ks) {
-            // K-major operands: 16 elements (32 bytes) per step inside a 64-column panel
+          for (int ks = 0; ks < D / C::QK_KSTEP; ++ks) {
+            // K-major operands: 32 bytes (16 bf16 or 32 E4M3 elements) per step, four steps per panel
             const uint32_t qoff = ((ks / 4) * C::PANEL_BYTES + (ks % 4) * 32) >> 4;
             const uint32_t koff = ((ks / 4) * C::HALF_PANEL_BYTES + (ks % 4) * 32) >> 4;
-            mma_ss(d_cols, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            if (F8) mma_ss_f8(d_cols, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
+            else mma_ss(d_cols, q_desc0 + qoff, kd + koff, idesc_qk, (g > 0 || ks > 0) ? 1u : 0u);
           }
         }
         mma_commit(bar);
@@ -290,7 +311,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (!ok) break;
         tc_fence_after();
         if (elect_one())
-          fire_s(tmem_s + (u % C::NBUF) * kHalf, kslot_of(u), u >= 2 * sel_tiles ? 2 : 1, b_s_full(u % C::NBAR));
+          fire_s(tmem_s + (u % C::NBUF) * kHalf, kslot_of(u), u >= 2 * sel_tiles ? C::CEN_PARTS : 1, b_s_full(u % C::NBAR));
         __syncwarp();
       }
       for (int u = 0; u < steps && ok; ++u) {
@@ -301,7 +322,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         const uint64_t vd = v_desc0 + ((slot * C::HALF_BYTES) >> 4);
         const uint32_t p_cols = tmem_s + (u % C::NBUF) * kHalf;
         const uint32_t s_cols = tmem_s + (un % C::NBUF) * kHalf, s_bar = b_s_full(un % C::NBAR), pv_bar = b_pv_done(u % C::NBAR);
-        const int s_kc0 = kslot_of(un), s_parts = un >= steps ? 0 : (un >= 2 * sel_tiles ? 2 : 1);
+        const int s_kc0 = kslot_of(un), s_parts = un >= steps ? 0 : (un >= 2 * sel_tiles ? C::CEN_PARTS : 1);
         if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_p_ready(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
         if (!ok) break;
         tc_fence_after();
@@ -330,9 +351,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (j < 0 || j >= prm.n_kc) {                        // not a key cluster: flagged, all of its columns masked
         atomicCAS(prm.status, 0, kErrBadIndex);
         members_of[e] = 0;
+        if (F8) kscale_of[e] = 0.f;
         continue;
       }
       members_of[e] = (uint16_t)min(max(cnt[j], 0), prm.c_k);
+      if (F8) kscale_of[e] = prm.k_scale[(size_t)p * prm.n_kc + j];
       if (prm.compensate) atomicOr(&bitmap[j >> 5], 1u << (j & 31));
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -354,8 +377,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       if (lane == 0) mbar_arrive(b_q_tmem);
     }
     float m_ref = -INFINITY, l_run = 0.f, pend = 0.f;
-    const float inv_scale_log2 = 1.0f / prm.scale_log2;
     const int ck_shift = __ffs(prm.c_k) - 1;
+    // factor from a raw score to log2 units: the softmax scale, and with quantised Q K^T the scale
+    // of this thread's query row (times, per half-step, the scale of the key cluster or centroid run)
+    float row_sc = prm.scale_log2;
+    if (F8) {
+      const int qrow = (p * prm.n_qc + qc) * prm.c_q + half * kTile + (row < q_rows ? row : 0);
+      row_sc *= prm.q_scale[qrow];
+    }
     bool ok = true;
     for (int u = 0; u < steps && ok; ++u) {
       const int b = u & 1;                               // half of a 128-row tile (geometry of the keys)
@@ -392,6 +421,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (st < kHalf) bz[st] = use ? log2f((float)cnt[min(j, prm.n_kc - 1)]) : -INFINITY;
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
+      // scale of this half-step's scores.  A zero scale (an all-zero query row or key group) makes
+      // every logit 0: the raw scores are then dropped and the additive terms enter with scale 1.
+      float sc_used = prm.scale_log2;
+      bool keep_raw = true;
+      if (F8) {
+        const float ks = u < 2 * sel_tiles ? kscale_of[min((u * kHalf) >> ck_shift, max(keep - 1, 0))]
+                                           : prm.c_scale[(size_t)p * prm.cen_tiles + (u - 2 * sel_tiles)];
+        const float sc_eff = row_sc * ks;
+        keep_raw = sc_eff > 0.f;
+        sc_used = keep_raw ? sc_eff : (masked ? 1.f : 0.f);
+      }
 
       ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
       if (!ok) break;
@@ -408,13 +448,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // ---- masked / weighted half-steps (short clusters, centroid columns): the additive term is
       // folded into the scores in tensor memory first, so that the common path below has no bias
       if (masked) {
+        const float inv_scale_log2 = __fdividef(1.f, sc_used);
+        const float raw_factor = keep_raw ? 1.f : 0.f;
 #pragma unroll 1
         for (int c4 = 0; c4 < 2; ++c4) {
           uint32_t r[32];
           tmem_ld32(t_s + c4 * 32, r);
           tmem_wait_ld();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(fmaf(bz[c4 * 32 + j], inv_scale_log2, __uint_as_float(r[j])));
+          for (int j = 0; j < 32; ++j) {
+            const float raw = F8 ? __uint_as_float(r[j]) * raw_factor : __uint_as_float(r[j]);
+            r[j] = __float_as_uint(fmaf(bz[c4 * 32 + j], inv_scale_log2, raw));
+          }
           tmem_st32(t_s + c4 * 32, r);
         }
         tmem_wait_st();
@@ -448,7 +493,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
               mx3 = max3(mx3, __uint_as_float(r[j + 6]), __uint_as_float(r[j + 7]));
             }
           }
-          tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * prm.scale_log2;
+          tmax = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * sc_used;
           raise = tmax > m_ref + kRescaleThreshold || (m_ref == -INFINITY && tmax > -INFINITY);
         }
         if (raise) {
@@ -482,7 +527,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       // ---- P = exp2(x - m_ref), packed to bf16 over the first 32 columns of the buffer (chunk 0
       // goes to columns [0,16) while chunk 1 is still unread in [32,64); chunk 1 to [16,32))
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
-      const f32x2 sc2 = pack2(prm.scale_log2, prm.scale_log2);
+      const f32x2 sc2 = pack2(sc_used, sc_used);
       float cm0 = -INFINITY, cm1 = -INFINITY;            // maximum of x - m_ref over the half-step
 #pragma unroll 1
       for (int c4 = 0; c4 < 2; ++c4) {
@@ -631,15 +676,16 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
-// bf16 matrix [rows, D] row-major; box = 64 columns x box_rows rows, 128-byte swizzle
-static bool make_map(CUtensorMap* map, const void* base, size_t rows, int D, int box_rows) {
+// matrix [rows, D] row-major of bf16 (or of one-byte codes); box = one 128-byte panel row (64 bf16
+// or 128 codes) x box_rows rows, 128-byte swizzle
+static bool make_map(CUtensorMap* map, const void* base, size_t rows, int D, int box_rows, bool bytes = false) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-  cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)D * (bytes ? 1 : 2)};
+  cuuint32_t box[2] = {bytes ? 128u : 64u, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+  return fn(map, bytes ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -653,20 +699,34 @@ bool attn_tc_supported(const ca_problem_t& pr) {
   return true;
 }
 
+// quantised Q K^T: head dimension 128 (one 128-byte panel row of codes), key clusters of at least
+// 64 rows (one scale per half-step)
+bool attn_tc_fp8_supported(const ca_problem_t& pr) {
+  return attn_tc_supported(pr) && pr.head_dim == 128 && pr.cluster_k >= kHalf;
+}
+
 size_t attn_tc_workspace_bytes(const ca_problem_t& pr) {
   const size_t P = (size_t)pr.batch * pr.heads;
   const size_t cen_tiles = (size_t)ceil_div(ceil_div(pr.n_k, pr.cluster_k), kHalf);
   const size_t n_qc = (size_t)ceil_div(pr.n_q, pr.cluster_q);
-  return kStatusBytes + align_up(P * cen_tiles * kTile * pr.head_dim * sizeof(__nv_bfloat16), 256) +
-         align_up(P * cen_tiles * kHalf * pr.head_dim * sizeof(__nv_bfloat16), 256) +
-         align_up(P * n_qc * 2 * sizeof(int32_t), 256);
+  size_t bytes = kStatusBytes + align_up(P * cen_tiles * kTile * pr.head_dim * sizeof(__nv_bfloat16), 256) +
+                 align_up(P * cen_tiles * kHalf * pr.head_dim * sizeof(__nv_bfloat16), 256) +
+                 align_up(P * n_qc * 2 * sizeof(int32_t), 256);
+  if (pr.flags & CA_ATTN_FP8_QK) {
+    const size_t n_kc = (size_t)ceil_div(pr.n_k, pr.cluster_k), D = pr.head_dim;
+    const size_t q_rows = P * n_qc * pr.cluster_q, k_rows = P * n_kc * pr.cluster_k;
+    bytes += align_up(q_rows * D, 256) + align_up(q_rows * 4, 256) + align_up(k_rows * D, 256) +
+             align_up(P * n_kc * 4, 256) + align_up(P * cen_tiles * kHalf * D, 256) + align_up(P * cen_tiles * 4, 256);
+  }
+  return bytes;
 }
 
-template <int D>
+template <int D, bool F8>
 static int launch_tc_d(const CUtensorMap* maps, const TcParams& prm, dim3 grid, cudaStream_t st) {
-  using C = TcCfg<D>;
-  const size_t smem = 1024 + C::OFF_BITMAP + (size_t)prm.bitmap_words * 4 + (((size_t)prm.list_stride * 2 + 15) & ~(size_t)15);
-  auto k = attn_tc_kernel<D>;
+  using C = TcCfg<D, F8>;
+  const size_t smem = 1024 + C::OFF_BITMAP + (size_t)prm.bitmap_words * 4 + (((size_t)prm.list_stride * 2 + 15) & ~(size_t)15) +
+                      (F8 ? (size_t)prm.list_stride * 4 : 0);
+  auto k = attn_tc_kernel<D, F8>;
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
   k<<<grid, kTcThreads, smem, st>>>(maps[0], maps[1], maps[2], maps[3], maps[4], prm);
   CA_LAUNCH_CHECK();
@@ -694,6 +754,20 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   __nv_bfloat16* kmix = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kTile * D);
   __nv_bfloat16* vb = c.take<__nv_bfloat16>((size_t)P * cen_tiles * kHalf * D);
   int32_t* redo = c.take<int32_t>((size_t)P * n_qc * 2);
+  const bool f8 = (pr.flags & CA_ATTN_FP8_QK) != 0;
+  unsigned char *q8 = nullptr, *k8 = nullptr, *c8 = nullptr;
+  float *sq = nullptr, *sk = nullptr, *sc = nullptr;
+  if (f8) {
+    // queries, keys and key centroids as E4M3 codes with their scales (quantize.cu)
+    const size_t q_rows = (size_t)P * n_qc * pr.cluster_q, k_rows = (size_t)P * n_kc * pr.cluster_k;
+    q8 = c.take<unsigned char>(q_rows * D);  sq = c.take<float>(q_rows);
+    k8 = c.take<unsigned char>(k_rows * D);  sk = c.take<float>((size_t)P * n_kc);
+    c8 = c.take<unsigned char>((size_t)P * cen_tiles * kHalf * D);  sc = c.take<float>((size_t)P * cen_tiles);
+    ProfScope ps(kProfAttnPrep, st);
+    const int rq = launch_quantize_qk(Qp, Kp, pr.compensate ? ck : nullptr, P, n_qc, pr.cluster_q, n_kc, pr.cluster_k,
+                                      cen_tiles, D, q8, sq, k8, sk, c8, sc, st);
+    if (rq != CA_OK) return rq;
+  }
   if (pr.compensate) {
     ProfScope ps(kProfAttnPrep, st);
     centroid_prep_kernel<<<dim3(ceil_div(cen_tiles * kHalf * D, 256), P), 256, 0, st>>>(ck, cv, n_kc, cen_tiles, D,
@@ -702,11 +776,17 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   }
   CUtensorMap maps[5];
   const int kbox = pr.cluster_k < kHalf ? pr.cluster_k : kHalf;      // key/value slots hold 64 rows
-  bool ok = make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, pr.cluster_q < kTile ? pr.cluster_q : kTile) &&
-            make_map(&maps[1], Kp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
-            make_map(&maps[2], Vp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
-            make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kHalf) &&
+  const int qbox = pr.cluster_q < kTile ? pr.cluster_q : kTile;
+  bool ok = make_map(&maps[2], Vp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
             make_map(&maps[4], vb, (size_t)P * cen_tiles * kHalf, D, kHalf);
+  if (f8)
+    ok = ok && make_map(&maps[0], q8, (size_t)P * n_qc * pr.cluster_q, D, qbox, true) &&
+         make_map(&maps[1], k8, (size_t)P * n_kc * pr.cluster_k, D, kbox, true) &&
+         make_map(&maps[3], c8, (size_t)P * cen_tiles * kHalf, D, kHalf, true);
+  else
+    ok = ok && make_map(&maps[0], Qp, (size_t)P * n_qc * pr.cluster_q, D, qbox) &&
+         make_map(&maps[1], Kp, (size_t)P * n_kc * pr.cluster_k, D, kbox) &&
+         make_map(&maps[3], kmix, (size_t)P * cen_tiles * kTile, D, kHalf);
   if (!ok) return CA_ERR_CUDA;
   TcParams prm;
   prm.count_k = count_k; prm.block_idx = block_idx; prm.keep_count = keep_count; prm.perm_q = perm_q;
@@ -718,11 +798,13 @@ int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const
   prm.scale_log2 = scale * 1.4426950408889634f;
   prm.wait_limit = g_wait_limit;
   prm.skip_key_load = g_skip_key_load;
+  prm.q_scale = sq; prm.k_scale = sk; prm.c_scale = sc;
   dim3 grid(n_qc * (pr.cluster_q >= kTile ? pr.cluster_q / kTile : 1), P);
   int rc;
   {
     ProfScope ps(kProfAttn, st);
-    rc = D == 64 ? launch_tc_d<64>(maps, prm, grid, st) : launch_tc_d<128>(maps, prm, grid, st);
+    if (f8) rc = launch_tc_d<128, true>(maps, prm, grid, st);
+    else rc = D == 64 ? launch_tc_d<64, false>(maps, prm, grid, st) : launch_tc_d<128, false>(maps, prm, grid, st);
   }
   if (rc != CA_OK) return rc;
   ProfScope ps(kProfAttnSecond, st);

@@ -95,6 +95,11 @@ int launch_attn_ref(const ca_problem_t& pr, const void* Qp, const void* Kp, cons
 
 // attn_tc.cu
 bool attn_tc_supported(const ca_problem_t& pr);
+bool attn_tc_fp8_supported(const ca_problem_t& pr);
+// quantize.cu: E4M3 codes and scales of the cluster-ordered queries, keys and the key centroids
+int launch_quantize_qk(const void* Qp, const void* Kp, const float* ck, int P, int n_qc, int c_q, int n_kc, int c_k,
+                       int cen_tiles, int D, unsigned char* q8, float* sq, unsigned char* k8, float* sk,
+                       unsigned char* c8, float* sc, cudaStream_t st);
 size_t attn_tc_workspace_bytes(const ca_problem_t& pr);
 int launch_attn_tc(const ca_problem_t& pr, const void* Qp, const void* Kp, const void* Vp, const float* ck,
                    const float* cv, const int32_t* count_k, const int32_t* block_idx, const int32_t* keep_count,

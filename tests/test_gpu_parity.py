@@ -181,7 +181,7 @@ def test_select_blocks_exact(H, n_qc, n_kc, d, keep):
 # ----------------------------------------------------------------------------
 # Attention on the oracle's permutation and block lists.
 # ----------------------------------------------------------------------------
-def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=None, adaptive=None):
+def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=None, adaptive=None, quantized=False):
     Q, K, V = inputs.generate(w.scaled(heads=H))
     c_q, c_k = w.cluster, (cluster_k or w.cluster)
     p = binding.problem_from_workload(w, heads=H, keep=keep, compensate=compensate, flags=flags,
@@ -204,8 +204,9 @@ def attention_case(w, H, keep, compensate, flags=0, perm_seed=None, cluster_k=No
         else:                                # lists of different lengths (Section 3.3.2)
             idx = orc.select_blocks_adaptive(cl["cq"], cl["ck"], cl["count_k"], adaptive[0], adaptive[1])
         ck32, cv32 = cl["ck"].astype(np.float32), cl["cv"].astype(np.float32)
-        o, lse = orc.cluster_attention(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c_q, c_k, idx, compensate,
-                                       ck=ck32, cv=cv32, count_k=cl["count_k"])
+        attend = orc.cluster_attention_quantized_qk if quantized else orc.cluster_attention
+        o, lse = attend(Q[h], K[h], V[h], cl["perm_q"], cl["perm_k"], c_q, c_k, idx, compensate,
+                        ck=ck32, cv=cv32, count_k=cl["count_k"])
         refs.append((o, lse))
 
         def pad(x, perm, n, c):
@@ -289,6 +290,40 @@ def test_attention_bf16(name, n_q, n_k, keep, compensate, flags):
         assert bf16_close(O[h], o_ref), (np.abs(O[h] - o_ref).max(),
                                          np.linalg.norm(O[h] - o_ref) / np.linalg.norm(o_ref))
         assert np.abs(lse[h] - lse_ref).max() < 2e-2
+
+
+@pytest.mark.parametrize("name,n_q,n_k,c_q,c_k,keep,compensate,perm_seed", [
+    ("video480", 1000, 1000, 128, 128, 2, True, None),     # short last clusters, centroid columns
+    ("sweep", 2048, 2048, 128, 128, 16, True, None),       # all blocks kept but none short
+    ("sweep", 1100, 3000, 64, 64, 9, True, 5),             # 64-row clusters: one key scale per half-step
+    ("sweep", 1100, 3000, 64, 128, 5, False, None),        # the paper's block shape, no compensation
+    ("sweep", 1024, 2100, 256, 256, 3, True, 6),           # two CTAs per query cluster, two tiles per key cluster
+])
+def test_attention_with_quantised_qk(name, n_q, n_k, c_q, c_k, keep, compensate, perm_seed):
+    """CA_ATTN_FP8_QK: Q K^T on E4M3 codes with a scale per query row, per key cluster and per run
+    of 64 key centroids (Section 3.1 / 5.1: the paper's kernel is a quantised one).  The codes are
+    taken in float32 the same way on both sides and their products are exact, so the result is held
+    to the bf16 tolerances against the oracle's attention on the de-quantised tensors -- and it
+    differs visibly from the unquantised attention."""
+    w = inputs.WORKLOADS[name].scaled(n_q=n_q, n_k=n_k, cluster=c_q)
+    if w.kind == "video":
+        w = w.scaled(grid=(5, 10, 20))
+    O, lse, refs = attention_case(w, 2, keep, compensate, flags=binding.CA_ATTN_FP8_QK, cluster_k=c_k,
+                                  perm_seed=perm_seed, quantized=True)
+    _, _, plain = attention_case(w, 2, keep, compensate, cluster_k=c_k, perm_seed=perm_seed)
+    for h, (o_ref, lse_ref) in enumerate(refs):
+        assert bf16_close(O[h], o_ref), (np.abs(O[h] - o_ref).max(), np.linalg.norm(O[h] - o_ref) / np.linalg.norm(o_ref))
+        assert np.abs(lse[h] - lse_ref).max() < 2e-2
+        # the quantisation itself is a larger step than the tolerance of the comparison
+        assert np.linalg.norm(plain[h][0] - o_ref) > 2 * np.linalg.norm(O[h] - o_ref)
+
+
+def test_quantised_qk_is_refused_where_it_is_not_built():
+    p = binding.make_problem(1, 1, 512, 512, 64, "bf16", 128, 128, 2, flags=binding.CA_ATTN_FP8_QK)
+    plan = binding.Plan(p.copy(flags=0), DEV)
+    plan.problem = p
+    with pytest.raises(binding.ClusterAttnError, match="CA_ERR_UNSUPPORTED"):
+        plan.cluster_attention_fwd()
 
 
 def test_all_blocks_kept_is_dense_attention_on_device():
