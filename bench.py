@@ -94,6 +94,8 @@ def parse_args():
                     help="token-count sweep 8k..1M with per-stage times (64 kept blocks, and 10 %% of the blocks), "
                          "eager launches and one replayed CUDA graph, against dense attention")
     ap.add_argument("--max-tokens", type=int, default=1 << 20)
+    ap.add_argument("--fp8-qk", action="store_true",
+                    help="attention with Q K^T on E4M3 codes (CA_ATTN_FP8_QK; head dimension 128 only)")
     ap.add_argument("--secondary", default="video480", metavar="WORKLOAD",
                     help="also report stage times and the attention roofline of this workload (10 steps); "
                          "'' switches it off")
@@ -377,7 +379,8 @@ def run_ours(args, w):
     keep = args.keep or w.keep
     heads = w.heads
     adaptive = args.adaptive > 0.0
-    p = binding.problem_from_workload(w, keep=keep, flags=binding.CA_QUERY_UNNORMALIZED if adaptive else 0)
+    p = binding.problem_from_workload(w, keep=keep, flags=(binding.CA_QUERY_UNNORMALIZED if adaptive else 0) |
+                                      (binding.CA_ATTN_FP8_QK if args.fp8_qk else 0))
     dt = binding.torch_dtype(p)
     Qh, Kh, Vh = inputs.generate(w)                        # every replica runs the same seeded batch
     pin = lambda a: torch.from_numpy(a[None]).to(dt).pin_memory()
@@ -652,6 +655,7 @@ def run_ours(args, w):
         "config": {"workload": w.name, "heads": heads, "head_dim": w.head_dim, "n_q": w.n_q, "n_k": w.n_k,
                    "cluster": w.cluster, "keep": mean_keep if adaptive else keep, "n_kc": w.n_kc,
                    "selection": f"adaptive recall {args.adaptive} min 16" if adaptive else "top-k",
+                   "qk_operands": "e4m3 (per-row / per-cluster scales)" if args.fp8_qk else w.dtype,
                    "clustering": f"basic recursive splitting, {args.basic} power iterations" if basic
                    else "diagonalized recursive splitting", "compensate": w.compensate,
                    "parallelism": "replicas" if world > 1 else "single",

@@ -41,7 +41,7 @@ def generated(w):
     return _GENERATED[key]
 
 
-def run_workload(name, keep=None, cluster=None, compensate=None, **shape):
+def run_workload(name, keep=None, cluster=None, compensate=None, flags=0, **shape):
     build.build()
     w = inputs.WORKLOADS[name]
     if shape:
@@ -53,7 +53,7 @@ def run_workload(name, keep=None, cluster=None, compensate=None, **shape):
     if compensate is not None:
         w = w.scaled(compensate=compensate)
     Q, K, V = generated(w)
-    p = binding.problem_from_workload(w)
+    p = binding.problem_from_workload(w, flags=flags)
     dt = binding.torch_dtype(p)
     plan = binding.Plan(p, DEV, keep_y=True)
     dev = lambda a: torch.from_numpy(a[None]).to(dt).to(DEV)
@@ -65,8 +65,9 @@ def run_workload(name, keep=None, cluster=None, compensate=None, **shape):
 
 
 def check_workload(name, sample_heads, clusters_per_head, split_heads, keep=None, cluster=None, compensate=None,
-                   chain_heads=(), **shape):
-    w, Q, K, V, plan, O = run_workload(name, keep, cluster, compensate, **shape)
+                   chain_heads=(), quantized=False, **shape):
+    w, Q, K, V, plan, O = run_workload(name, keep, cluster, compensate,
+                                       flags=binding.CA_ATTN_FP8_QK if quantized else 0, **shape)
     c = w.cluster
     label = f"{name} c={c} keep={w.keep}"
     # ---- invariants for every head
@@ -107,8 +108,9 @@ def check_workload(name, sample_heads, clusters_per_head, split_heads, keep=None
         qcs = sorted(r.choice(w.n_qc, clusters_per_head, replace=False).tolist())
         if w.n_q % c:
             qcs[-1] = w.n_qc - 1                 # include the short cluster
-        o_ref, lse_ref = orc.cluster_attention(Q[h], K[h], V[h], pq, pk, c, c, idx, w.compensate, ck=ck, cv=cv,
-                                               count_k=plan.count_k[0, h].cpu().numpy(), query_clusters=qcs)
+        attend = orc.cluster_attention_quantized_qk if quantized else orc.cluster_attention
+        o_ref, lse_ref = attend(Q[h], K[h], V[h], pq, pk, c, c, idx, w.compensate, ck=ck, cv=cv,
+                                count_k=plan.count_k[0, h].cpu().numpy(), query_clusters=qcs)
         rows = np.concatenate([pq[i * c:min((i + 1) * c, w.n_q)] for i in qcs])
         got = O[0, h].float().cpu().numpy()[rows]
         worst_abs = max(worst_abs, np.abs(got - o_ref[rows]).max())
@@ -125,6 +127,12 @@ def test_tabular_full_size():
 
 def test_video480_full_size():
     check_workload("video480", sample_heads=[0, 17, 39], clusters_per_head=4, split_heads=[11], chain_heads=[11])
+
+
+def test_video480_full_size_quantised_qk():
+    """The video-shaped workload with Q K^T on E4M3 codes (CA_ATTN_FP8_QK), as `bench.py --workload
+    video480 --fp8-qk` launches it; sampled query clusters against the oracle's quantised attention."""
+    check_workload("video480", sample_heads=[5, 33], clusters_per_head=4, split_heads=[], quantized=True)
 
 
 def test_video720_full_size_both_densities():
