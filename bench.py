@@ -44,8 +44,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # was captured from: sha256 of csrc/attn_tc.cu + csrc/tc_ptx.cuh, first 16 hex digits.  When the
 # source has changed since, the bench prints null instead of a stale figure.
 NCU_TRAFFIC = {
-    "tabular": {"bytes": 554.2e6, "source": "", "commit": "4457068"},
-    "video480": {"bytes": 1269.0e6, "source": "", "commit": "6755999"},
+    "tabular": {"bytes": 568.3e6, "source": "6b538db0b9316f3e", "commit": "8346370"},
+    "video480": {"bytes": 1274.8e6, "source": "6b538db0b9316f3e", "commit": "8346370"},
 }
 # FP32 FMA rate of the CUDA cores, the roof of kernels bound by plain arithmetic (centroid scoring,
 # the fp32 attention kernel): 148 SMs x 128 FMA lanes x 2 flops x 1.965 GHz (the maximum SM clock).
@@ -94,6 +94,8 @@ def parse_args():
                     help="token-count sweep 8k..1M with per-stage times (64 kept blocks, and 10 %% of the blocks), "
                          "eager launches and one replayed CUDA graph, against dense attention")
     ap.add_argument("--max-tokens", type=int, default=1 << 20)
+    ap.add_argument("--bare", action="store_true",
+                    help="timed steps only: no sustained leg, no per-kernel timers (for captures under a profiler)")
     ap.add_argument("--fp8-qk", action="store_true",
                     help="attention with Q K^T on E4M3 codes (CA_ATTN_FP8_QK; head dimension 128 only)")
     ap.add_argument("--secondary", default="video480", metavar="WORKLOAD",
@@ -452,7 +454,7 @@ def run_ours(args, w):
     # ---- sustained leg (not the headline): the same step back to back for about a second, so that the
     # clock sampler sees this load for long enough; its time per step is reported beside the headline
     sustained = None
-    if rank == 0:
+    if rank == 0 and not args.bare:
         n_sus = max(args.steps, int(1000.0 / max(t_start.elapsed_time(t_end) / args.steps, 0.05)))
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s0.record(stream)
@@ -469,7 +471,7 @@ def run_ours(args, w):
     # ---- per-kernel times of the clustering and selection stages (the library's own timers, each
     # kernel group alone on the stream), outside the timed region
     group_ms = {}
-    if rank == 0 and not basic:
+    if rank == 0 and not basic and not args.bare:
         binding.profile(True)
         n_prof = 5
         for _ in range(n_prof):
@@ -643,6 +645,17 @@ def run_ours(args, w):
         roofline = {"kernel": "cluster_attention_fwd", "bound": "alu", "achieved": attn_tflops, "peak": FP32_ALU_TFLOPS,
                     "peak_source": "148 SMs x 128 FMA lanes x 2 x 1.965 GHz", "unit": "TFLOP/s",
                     "frac": attn_tflops / FP32_ALU_TFLOPS, "traffic": None}
+    if w.dtype == "bf16" and w.head_dim == 64:
+        # At d = 64 the exponentials bound the kernel before the tensor pipe does: a half-step of 64 keys
+        # is 2 x (128 x 64 x 64) multiply-adds = 2^21 flops of tensor work per query tile and
+        # 128 x 64 = 8192 exponentials, which the special-function unit of an SM takes 512 cycles for
+        # (16 per cycle: 4 sub-cores x 1 warp instruction per 8 cycles): at most 4096 flops per cycle
+        # and SM, i.e. 148 SMs x 4096 x 1.965 GHz.
+        sfu_peak = 148 * 4096 * 1.965e9 / 1e12
+        roofline["second_bound"] = {"name": "special-function unit (exp2 of the softmax)", "peak": sfu_peak,
+                                    "unit": "TFLOP/s", "frac": attn_tflops / sfu_peak,
+                                    "derivation": "8192 exp2 per 2^21 tensor flops; 16 exp2 per cycle and SM; "
+                                                  "148 SMs x 4096 flops/cycle x 1.965 GHz"}
     stages = stage_rooflines(w.scaled(keep=keep), heads, group_ms, peaks["hbm_gbs"], peak_kind) if group_ms else None
     secondary = None
     if args.secondary and args.secondary != w.name and world == 1 and w.name == "tabular" \
