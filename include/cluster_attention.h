@@ -105,11 +105,14 @@ int ca_workspace_bytes(const ca_problem_t* p, size_t* cluster_ws, size_t* select
  *        p->flags has CA_Y_IN, otherwise output (may be NULL: kept in ws).
  * The chain from Q to the key side (metric, its factor, key projection, key split)
  * and the chain from K to the query side need each other only through C_K: the
- * second one is enqueued on a second stream of the library (one per device,
- * created together with three events at the first call on that device) that forks
- * from `stream` at the start of the call and joins it again before the call returns.  Nothing waits on the
- * host; a capture of `stream` records the side stream as a parallel branch (make
- * the first call on a device before capturing).
+ * second one is enqueued on a side stream of the library (a pool of four per
+ * device, taken in turn, created together with their events at the first call on
+ * that device) that forks from `stream` at the start of the call and joins it
+ * again before the call returns.  Nothing waits on the host; a capture of `stream`
+ * records the side stream as a parallel branch (make the first call on a device
+ * before capturing).  The calls of this library may be issued from several host
+ * threads; ca_profile, ca_debug_attn_wait and the workspaces themselves are not
+ * synchronised (one workspace serves one call at a time).
  */
 int cluster_qk(const ca_problem_t* p, const void* Q, const void* K, const void* V,
                int32_t* perm_q, int32_t* perm_k, void* Qp, void* Kp, void* Vp,
@@ -308,7 +311,7 @@ int ca_profile_read(int max_groups, const char** names, float* ms, int* scopes);
 const char* ca_version(void);
 
 /* Diagnostic: number of kernels this library has enqueued since it was loaded
- * (host-side counter, not thread-safe). */
+ * (host-side atomic counter). */
 unsigned long long ca_kernel_launches(void);
 
 #ifdef __cplusplus

@@ -2,12 +2,15 @@
 // order in which the kernels of each stage are enqueued.
 #include <math.h>
 
+#include <atomic>
+#include <mutex>
+
 #include "kernels.h"
 
 using namespace ca;
 
 namespace ca {
-unsigned long long g_kernel_launches = 0;
+std::atomic<unsigned long long> g_kernel_launches{0};
 
 // ---- per-kernel-group timers (off unless ca_profile(1) was called) ------------------------------
 namespace {
@@ -126,26 +129,33 @@ ClusterWs carve_cluster(const ca_problem_t* p, void* base, bool need_yq, bool ne
 // The query side and the key side of cluster_qk are independent once the two factors exist.  The
 // query side runs on a second stream that forks from the caller's stream and joins it again
 // before the call returns (events only: nothing waits on the host, and a stream capture of the
-// caller's stream picks the side stream up as a parallel branch).  One stream and three events
-// (fork, C_K ready, join) per device, created at the first call on that device.
+// caller's stream picks the side stream up as a parallel branch).  A pool of four side streams, each
+// with three events (fork, Gram matrix of K ready, join), per device, created at the first call on
+// that device; calls take them in turn, so that up to four calls in flight on different caller
+// streams (from one or several host threads) do not share a side stream.
 struct SideStream {
   cudaStream_t stream = nullptr;
   cudaEvent_t fork = nullptr, mid = nullptr, join = nullptr;
-  bool ready = false;
 };
+constexpr int kSidePool = 4;
 SideStream* side_stream() {
-  static SideStream table[64];
+  static SideStream table[64][kSidePool];
+  static bool ready[64] = {};
+  static unsigned next[64] = {};
+  static std::mutex guard;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  SideStream& s = table[dev];
-  if (!s.ready) {
-    if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s.mid, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-    s.ready = true;
+  std::lock_guard<std::mutex> lock(guard);
+  if (!ready[dev]) {
+    for (SideStream& s : table[dev]) {
+      if (cudaStreamCreateWithFlags(&s.stream, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&s.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&s.mid, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+      if (cudaEventCreateWithFlags(&s.join, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    }
+    ready[dev] = true;
   }
-  return &s;
+  return &table[dev][next[dev]++ % kSidePool];
 }
 
 #define CA_TRY(expr)               \
@@ -160,7 +170,7 @@ extern "C" {
 
 const char* ca_version(void) { return "libclusterattn 0.1 (sm_100a)"; }
 
-unsigned long long ca_kernel_launches(void) { return g_kernel_launches; }
+unsigned long long ca_kernel_launches(void) { return g_kernel_launches.load(); }
 
 int ca_profile(int enable) {
   if (enable) {

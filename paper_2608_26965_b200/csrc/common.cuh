@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/cluster_attention.h"
 
 namespace ca {
@@ -15,7 +17,7 @@ constexpr size_t kStatusBytes = 256;
 constexpr size_t kStatusClearBytes = 252;
 constexpr int kRecomputedWord = 63;
 
-extern unsigned long long g_kernel_launches;   // kernels enqueued since the library was loaded
+extern std::atomic<unsigned long long> g_kernel_launches;   // kernels enqueued since the library was loaded
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }

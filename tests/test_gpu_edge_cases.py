@@ -298,3 +298,44 @@ def test_a_wait_that_runs_out_ends_the_kernel_with_a_status(d):
     o_ref, _ = orc.cluster_attention(host["Q"], host["K"], host["V"], host["perm_q"], host["perm_k"], c, c,
                                      host["idx"], True, ck=host["ck"], cv=host["cv"], count_k=host["count_k"])
     assert np.abs(again[0, 0].float().cpu().numpy() - o_ref).max() <= 2e-2
+
+
+def test_two_host_threads_on_two_streams_give_the_sequential_results():
+    """Two plans driven from two host threads on their own streams at the same time (the library's
+    side streams come from a pool, its launch counter is atomic): every output equals the one of the
+    same call made alone."""
+    import threading
+    w = inputs.WORKLOADS["tabular"].scaled(heads=2, n_q=4096, n_k=16384, keep=16)
+    data = [inputs.generate(w.scaled(config_id=w.config_id + 7 * i)) for i in range(2)]
+    p = binding.problem_from_workload(w)
+    tensors = [[torch.from_numpy(a[None]).to(torch.bfloat16).to(DEV) for a in d] for d in data]
+    alone = []
+    for t in tensors:
+        plan = binding.Plan(p, DEV)
+        O = plan.forward(*t, want_lse=True)
+        torch.cuda.synchronize()
+        alone.append([x.clone() for x in (O, plan.lse, plan.perm_q, plan.perm_k, plan.block_idx)])
+    plans = [binding.Plan(p, DEV) for _ in range(2)]
+    streams = [torch.cuda.Stream() for _ in range(2)]
+    errors = []
+
+    def work(i):
+        try:
+            with torch.cuda.device(0):
+                for _ in range(5):
+                    plans[i].forward(*tensors[i], want_lse=True, stream=streams[i])
+                streams[i].synchronize()
+        except Exception as exc:      # noqa: BLE001
+            errors.append(exc)
+    threads = [threading.Thread(target=work, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    for i in range(2):
+        assert all(v == 0 for v in plans[i].last_status().values())
+        got = (plans[i].O, plans[i].lse, plans[i].perm_q, plans[i].perm_k, plans[i].block_idx)
+        for a, b in zip(got, alone[i]):
+            assert torch.equal(a, b)
