@@ -632,18 +632,21 @@ def cluster_attention_quantized_qk(Q, K, V, perm_q, perm_k, c_q, c_k, block_idx,
 # metrics -> roots -> transforms -> global principal components -> fp32
 # coordinates -> recursive split -> centroids in the original space.
 # --------------------------------------------------------------------------
-def split_coordinates(Q, K, adaptive=False):
+def split_coordinates(Q, K, adaptive=False, return_maps=False):
     """Returns (Yq32, Yk32): the fp32 coordinates the splitter reads.  `adaptive`
     selects the query representation that goes with adaptive selection: the
     metric K_c^T K_c / n without normalisation (Appendix B.1) instead of the
-    normalised ranking form (Appendix B.2)."""
+    normalised ranking form (Appendix B.2).  With `return_maps` also the two
+    matrices R E (root times principal directions) whose columns fix the signs."""
     R_q = psd_root(metric_q(Q))
     if adaptive:
         R_k = psd_root(centered_scatter(K) / np.asarray(K).shape[0])
     else:
         R_k = psd_root(centered_scatter(K))
-    Yk, _, _ = diagonalize(transform_keys(K, R_q), lift=R_q)
-    Yq, _, _ = diagonalize(query_representation(Q, R_k, normalize=not adaptive), lift=R_k)
+    Yk, _, Ek = diagonalize(transform_keys(K, R_q), lift=R_q)
+    Yq, _, Eq = diagonalize(query_representation(Q, R_k, normalize=not adaptive), lift=R_k)
+    if return_maps:
+        return Yq.astype(np.float32), Yk.astype(np.float32), R_k @ Eq, R_q @ Ek
     return Yq.astype(np.float32), Yk.astype(np.float32)
 
 

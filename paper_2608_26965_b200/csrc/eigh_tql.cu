@@ -47,7 +47,11 @@ __device__ __forceinline__ void named_sync(int id, int count) {
     case 1: asm volatile("bar.sync 1, %0;" ::"r"(count) : "memory"); break;
     case 2: asm volatile("bar.sync 2, %0;" ::"r"(count) : "memory"); break;
     case 3: asm volatile("bar.sync 3, %0;" ::"r"(count) : "memory"); break;
-    default: asm volatile("bar.sync 4, %0;" ::"r"(count) : "memory"); break;
+    case 4: asm volatile("bar.sync 4, %0;" ::"r"(count) : "memory"); break;
+    case 5: asm volatile("bar.sync 5, %0;" ::"r"(count) : "memory"); break;
+    case 6: asm volatile("bar.sync 6, %0;" ::"r"(count) : "memory"); break;
+    case 7: asm volatile("bar.sync 7, %0;" ::"r"(count) : "memory"); break;
+    default: asm volatile("bar.sync 8, %0;" ::"r"(count) : "memory"); break;
   }
 }
 __device__ __forceinline__ void named_arrive(int id, int count) {
@@ -55,13 +59,130 @@ __device__ __forceinline__ void named_arrive(int id, int count) {
     case 1: asm volatile("bar.arrive 1, %0;" ::"r"(count) : "memory"); break;
     case 2: asm volatile("bar.arrive 2, %0;" ::"r"(count) : "memory"); break;
     case 3: asm volatile("bar.arrive 3, %0;" ::"r"(count) : "memory"); break;
-    default: asm volatile("bar.arrive 4, %0;" ::"r"(count) : "memory"); break;
+    case 4: asm volatile("bar.arrive 4, %0;" ::"r"(count) : "memory"); break;
+    case 5: asm volatile("bar.arrive 5, %0;" ::"r"(count) : "memory"); break;
+    case 6: asm volatile("bar.arrive 6, %0;" ::"r"(count) : "memory"); break;
+    case 7: asm volatile("bar.arrive 7, %0;" ::"r"(count) : "memory"); break;
+    default: asm volatile("bar.arrive 8, %0;" ::"r"(count) : "memory"); break;
   }
 }
 
-constexpr int kBarFull = 1;    // ids 1, 2: a rotation list is ready
-constexpr int kBarEmpty = 3;   // ids 3, 4: a rotation list has been applied
 constexpr int kMaxQlIterations = 64;
+
+// ---- implicit-shift QL on rows [l0, l1) of a tridiagonal matrix (de[i] = (diagonal i, coupling of
+// i and i + 1); the coupling at l1 - 1 is not part of the block).  One warp: the search for a
+// negligible sub-diagonal entry uses all lanes, the rotation chase is one dependent chain on lane 0.
+// Each chase's rotations go through a double-buffered list (rot, hdr) to the consumer threads, which
+// apply them to the rows of Qt; bar_full / bar_empty are the first of two named barriers each.
+__device__ __forceinline__ void ql_producer(float2* de, int l0, int l1, float* rot, int* hdr, int rot_stride,
+                                            int bar_full, int bar_empty, int parties, int lane) {
+  int bsel = 0;
+  const float eps = 6e-8f;
+  for (int l = l0; l < l1; ++l) {
+    for (int iter = 0; iter < kMaxQlIterations; ++iter) {
+      // first m >= l whose sub-diagonal entry is negligible (m = l1 - 1 if none)
+      int m = l1 - 1;
+      for (int base = l; base < l1 - 1; base += 32) {
+        const int idx = base + lane;
+        bool small = false;
+        if (idx < l1 - 1) {
+          const float2 a = de[idx];
+          small = fabsf(a.y) <= eps * (fabsf(a.x) + fabsf(de[idx + 1].x));
+        }
+        const unsigned bal = __ballot_sync(0xffffffffu, small);
+        if (bal) { m = base + __ffs(bal) - 1; break; }
+      }
+      if (m == l) break;
+      named_sync(bar_empty + bsel, parties);             // the list's previous contents have been applied
+      if (lane == 0) {
+        float2* rt = reinterpret_cast<float2*>(rot + bsel * rot_stride);
+        const float2 top = de[l];
+        float g = (de[l + 1].x - top.x) / (2.f * top.y);
+        float rr = sqrtf(fmaf(g, g, 1.f));
+        g = de[m].x - top.x + top.y / (g + (g >= 0.f ? rr : -rr));
+        float s = 1.f, c = 1.f, p = 0.f;
+        bool under = false;
+        int i = m - 1;
+        float2 cur = de[i];              // (d_i, e_i)
+        float d_i1 = de[i + 1].x;
+        for (; i >= l; --i) {
+          // operands of the next rotation, fetched ahead of the dependent chain
+          const float2 nxt = de[i > l ? i - 1 : l];
+          const float f = s * cur.y, bb = c * cur.y;
+          const float r2 = fmaf(f, f, g * g);
+          float rinv;
+          asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rinv) : "f"(r2));
+          const float p_old = p, d_old = d_i1;
+          s = f * rinv;
+          c = g * rinv;
+          g = d_i1 - p;
+          rr = fmaf(c, bb + bb, (cur.x - g) * s);
+          p = s * rr;
+          de[i + 1] = make_float2(g + p, r2 * rinv);       // new d_{i+1}; e_{i+1} = hypot(f, g)
+          g = fmaf(c, rr, -bb);
+          rt[i] = make_float2(c, s);
+          // The chase has died out (f = g = 0): deflate here.  Tested after the rotation has been
+          // formed so that the test is off the dependent chain; its results are discarded.
+          if (r2 < 1e-36f) {
+            de[i + 1] = make_float2(d_old - p_old, 0.f);
+            de[m].y = 0.f;
+            under = true;
+            break;
+          }
+          d_i1 = cur.x;          // d_i is the next step's d_{i+1}; it has not been modified yet
+          cur = nxt;
+        }
+        int lo = l;
+        if (!under) {
+          de[l] = make_float2(top.x - p, g);
+          de[m].y = 0.f;
+        } else {
+          lo = i + 1;
+        }
+        hdr[bsel * 4 + 0] = m - 1;
+        hdr[bsel * 4 + 1] = lo;
+        hdr[bsel * 4 + 2] = 0;
+      }
+      __syncwarp();
+      __threadfence_block();
+      named_arrive(bar_full + bsel, parties);
+      bsel ^= 1;
+    }
+  }
+  named_sync(bar_empty + bsel, parties);
+  if (lane == 0) hdr[bsel * 4 + 2] = 1;                    // end marker
+  __syncwarp();
+  __threadfence_block();
+  named_arrive(bar_full + bsel, parties);
+  named_sync(bar_empty + (bsel ^ 1), parties);             // the other list's last hand-back
+}
+
+// consumer thread of column t (t >= ncols: only keeps the barriers going)
+__device__ __forceinline__ void ql_consumer(float* Qt, int lda, int t, int ncols, const float* rot, const int* hdr,
+                                            int rot_stride, int bar_full, int bar_empty, int parties) {
+  named_arrive(bar_empty + 0, parties);                    // both lists start out free
+  named_arrive(bar_empty + 1, parties);
+  int bsel = 0;
+  while (true) {
+    named_sync(bar_full + bsel, parties);
+    if (hdr[bsel * 4 + 2]) break;
+    if (t < ncols) {
+      const int hi = hdr[bsel * 4 + 0], lo = hdr[bsel * 4 + 1];
+      const float* rt = rot + bsel * rot_stride;
+      float carry = Qt[(hi + 1) * lda + t];
+      for (int i = hi; i >= lo; --i) {
+        const float c = rt[2 * i], s = rt[2 * i + 1];
+        const float zi = Qt[i * lda + t];
+        Qt[(i + 1) * lda + t] = fmaf(s, zi, c * carry);
+        carry = fmaf(c, zi, -s * carry);
+      }
+      Qt[lo * lda + t] = carry;
+    }
+    __threadfence_block();
+    named_arrive(bar_empty + bsel, parties);
+    bsel ^= 1;
+  }
+}
 
 }  // namespace
 
@@ -92,14 +213,15 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   float* A = reinterpret_cast<float*>(smem_raw);       // [D][LDA]
   float* Qt = A + D * LDA;                             // [D][LDA]   written after phase 1; rows become the eigenvectors
-  float* L = Qt + D * LDA;                             // [D][LDA]   the factor F (lift of the sign rule)
-  float* vbuf = L + D * LDA;                           // [2][D]     reflector, zero above its first entry
+  float* L = Qt + D * LDA;                             // [D][LDA]   the factor F (prologue, sign rule); the merged basis in between
+  float* vbuf = A + 3 * D * LDA;                       // [2][D]     reflector, zero above its first entry
   float* pbuf = vbuf + 2 * D;                          // [D]
   float* ubuf = pbuf + D;                              // [D]
   float2* de = reinterpret_cast<float2*>(ubuf + D);    // [D]        (diagonal i, sub-diagonal coupling i and i+1)
   float* beta = ubuf + 3 * D;                          // [2] (+2)
-  float* rot = beta + 4;                               // [2][2D]    (c, s) of the rotation of rows (i, i+1) at 2i
-  int* hdr = reinterpret_cast<int*>(rot + 4 * D);      // [2][4]     highest i, lowest i, end marker
+  float* rot = beta + 4;                               // [2][2][2D] per half: (c, s) of the rotation of rows (i, i+1) at 2i
+  int* hdr = reinterpret_cast<int*>(rot + 8 * D);      // [2][2][4]  highest i, lowest i, end marker
+  float* scratch = reinterpret_cast<float*>(hdr + 16); // [16 D]     arrays of the merge
   __shared__ double s_scale;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -300,110 +422,222 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
     for (int c = 0; c < 4; ++c) Qt[(4 * (q + 8 * t) + c) * LDA + r] = qreg[t][c];
   __syncthreads();
 
-  // ---- implicit-shift QL on the tridiagonal matrix; rotations applied to the rows of Qt
-  constexpr int kParties = 32 + D;
-  if (warp == 0) {
-    int bsel = 0;
-    const float eps = 6e-8f;
-    for (int l = 0; l < D; ++l) {
-      for (int iter = 0; iter < kMaxQlIterations; ++iter) {
-        // first m >= l whose sub-diagonal entry is negligible (m = D-1 if none)
-        int m = D - 1;
-        for (int base = l; base < D - 1; base += 32) {
-          const int idx = base + lane;
-          bool small = false;
-          if (idx < D - 1) {
-            const float2 a = de[idx];
-            small = fabsf(a.y) <= eps * (fabsf(a.x) + fabsf(de[idx + 1].x));
-          }
-          const unsigned bal = __ballot_sync(0xffffffffu, small);
-          if (bal) { m = base + __ffs(bal) - 1; break; }
-        }
-        if (m == l) break;
-        named_sync(kBarEmpty + bsel, kParties);            // the list's previous contents have been applied
-        if (lane == 0) {
-          float2* rt = reinterpret_cast<float2*>(rot + bsel * 2 * D);
-          const float2 top = de[l];
-          float g = (de[l + 1].x - top.x) / (2.f * top.y);
-          float rr = sqrtf(fmaf(g, g, 1.f));
-          g = de[m].x - top.x + top.y / (g + (g >= 0.f ? rr : -rr));
-          float s = 1.f, c = 1.f, p = 0.f;
-          bool under = false;
-          int i = m - 1;
-          float2 cur = de[i];              // (d_i, e_i)
-          float d_i1 = de[i + 1].x;
-          for (; i >= l; --i) {
-            // operands of the next rotation, fetched ahead of the dependent chain
-            const float2 nxt = de[i > l ? i - 1 : l];
-            const float f = s * cur.y, bb = c * cur.y;
-            const float r2 = fmaf(f, f, g * g);
-            float rinv;
-            asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(rinv) : "f"(r2));
-            const float p_old = p, d_old = d_i1;
-            s = f * rinv;
-            c = g * rinv;
-            g = d_i1 - p;
-            rr = fmaf(c, bb + bb, (cur.x - g) * s);
-            p = s * rr;
-            de[i + 1] = make_float2(g + p, r2 * rinv);       // new d_{i+1}; e_{i+1} = hypot(f, g)
-            g = fmaf(c, rr, -bb);
-            rt[i] = make_float2(c, s);
-            // The chase has died out (f = g = 0): deflate here.  Tested after the rotation has been
-            // formed so that the test is off the dependent chain; its results are discarded.
-            if (r2 < 1e-36f) {
-              de[i + 1] = make_float2(d_old - p_old, 0.f);
-              de[m].y = 0.f;
-              under = true;
-              break;
+  // ---- phase 2: divide and conquer.  T = diag(T1, T2) + rho u u^T with rho = |b|, b the coupling of
+  // rows KH-1 and KH, u = e_{KH-1} + sign(b) e_{KH}, and b subtracted from the two diagonal entries it
+  // touches.  The two halves are independent tridiagonal problems: each gets its own QL warp and its
+  // own consumer threads (rows of Qt of its half), side by side.  An extra column of Qt (index D, in
+  // the row padding) starts as u and goes through the same rotations: afterwards it holds z = Q^T u.
+  constexpr int KH = D / 2;
+  constexpr int kParties = D + 64;                         // a QL warp + D + 1 columns rounded up to warps
+  float* rot_top = rot;
+  float* rot_bot = rot + 4 * D;
+  int* hdr_top = hdr;
+  int* hdr_bot = hdr + 8;
+  __shared__ float s_rho, s_theta, s_z2sum;
+  if (tid == 0) {
+    const float bk = de[KH - 1].y;
+    s_rho = fabsf(bk);
+    s_theta = bk < 0.f ? -1.f : 1.f;
+    de[KH - 1] = make_float2(de[KH - 1].x - fabsf(bk), 0.f);
+    de[KH].x -= fabsf(bk);
+  }
+  for (int i = tid; i < D; i += NT) Qt[i * LDA + D] = 0.f;
+  __syncthreads();
+  if (tid == 0) { Qt[(KH - 1) * LDA + D] = 1.f; Qt[KH * LDA + D] = s_theta; }
+  __syncthreads();
+  if (warp == 0) ql_producer(de, 0, KH, rot_top, hdr_top, 2 * D, 1, 3, kParties, lane);
+  else if (warp == 1) ql_producer(de, KH, D, rot_bot, hdr_bot, 2 * D, 5, 7, kParties, lane);
+  else if (tid < 64 + D + 32) ql_consumer(Qt, LDA, tid - 64, D + 1, rot_top, hdr_top, 2 * D, 1, 3, kParties);
+  else if (tid < 64 + 2 * (D + 32)) ql_consumer(Qt, LDA, tid - 64 - (D + 32), D + 1, rot_bot, hdr_bot, 2 * D, 5, 7, kParties);
+  __syncthreads();
+
+  // ---- merge: eigen-decomposition of diag(d) + rho2 z z^T, d the eigenvalues of the halves, z scaled
+  // to unit length (rho2 = 2 rho).  Sorted poles, deflation of negligible weights and of poles that
+  // coincide (a plane rotation of their two eigenvectors), the roots of the secular equation
+  // 1 + rho2 sum_j z_j^2 / (d_j - x) = 0 by bisection on the offset from the nearer pole (eight threads
+  // per root), the weights recomputed from the roots so that the eigenvectors come out orthogonal
+  // (Gu and Eisenstat), eigenvectors u_i[j] = zhat_j / (d_j - x_i), and the product with the halves'
+  // eigenvectors.
+  {
+    float* ds = scratch;                                   // poles in ascending order
+    float* zs = ds + D;
+    int* ord = reinterpret_cast<int*>(zs + D);             // sorted position -> row of Qt
+    int* keep_row = ord + D;                               // kept pole -> row of Qt
+    float* kd = reinterpret_cast<float*>(keep_row + D);    // kept poles, weights
+    float* kz = kd + D;
+    int* korg = reinterpret_cast<int*>(kz + D);            // root -> pole its offset is measured from
+    float* kmu = reinterpret_cast<float*>(korg + D);
+    float* kzh = kmu + D;
+    float* gc = kzh + D;                                   // plane rotations of the deflation
+    float* gs = gc + D;
+    int* ga = reinterpret_cast<int*>(gs + D);
+    int* gb = ga + D;
+    int* defl_row = gb + D;                                // deflated: row of Qt, eigenvalue
+    float* defl_d = reinterpret_cast<float*>(defl_row + D);
+    int* counts = reinterpret_cast<int*>(defl_d + D);      // kept, rotations, deflated, skip
+    if (tid < D) {
+      const float mine = de[tid].x;
+      int rank = 0;
+      for (int k = 0; k < D; ++k) {
+        const float other = de[k].x;
+        rank += (other < mine) || (other == mine && k < tid);
+      }
+      ord[rank] = tid;
+    }
+    __syncthreads();
+    if (tid < D) {
+      ds[tid] = de[ord[tid]].x;
+      zs[tid] = Qt[ord[tid] * LDA + D] * 0.70710678f;
+    }
+    __syncthreads();
+    if (tid == 0) {
+      const float rho2 = 2.f * s_rho;
+      float dmax = 0.f, zmax = 0.f;
+      for (int j = 0; j < D; ++j) { dmax = fmaxf(dmax, fabsf(ds[j])); zmax = fmaxf(zmax, fabsf(zs[j])); }
+      const float tol = 8.f * 6e-8f * fmaxf(dmax, zmax);
+      int K = 0, ng = 0, nd = 0, prev = -1;
+      if (rho2 * zmax <= tol) {
+        counts[3] = 1;                                     // the halves do not couple: nothing to merge
+      } else {
+        counts[3] = 0;
+        for (int j = 0; j < D; ++j) {
+          if (rho2 * fabsf(zs[j]) <= tol) { defl_row[nd] = ord[j]; defl_d[nd] = ds[j]; ++nd; continue; }
+          if (prev >= 0) {
+            float sn = zs[prev], cs = zs[j];
+            const float tau = sqrtf(fmaf(cs, cs, sn * sn));
+            const float t = ds[j] - ds[prev];
+            cs = cs / tau;
+            sn = -sn / tau;
+            if (fabsf(t * cs * sn) <= tol) {               // the two poles coincide: rotate the weight into one
+              zs[j] = tau;
+              zs[prev] = 0.f;
+              gc[ng] = cs; gs[ng] = sn; ga[ng] = ord[prev]; gb[ng] = ord[j]; ++ng;
+              const float tt = ds[prev] * cs * cs + ds[j] * sn * sn;
+              ds[j] = ds[prev] * sn * sn + ds[j] * cs * cs;
+              ds[prev] = tt;
+              --K;                                         // prev is the last kept pole
+              defl_row[nd] = ord[prev]; defl_d[nd] = tt; ++nd;
             }
-            d_i1 = cur.x;          // d_i is the next step's d_{i+1}; it has not been modified yet
-            cur = nxt;
           }
-          int lo = l;
-          if (!under) {
-            de[l] = make_float2(top.x - p, g);
-            de[m].y = 0.f;
-          } else {
-            lo = i + 1;
-          }
-          hdr[bsel * 4 + 0] = m - 1;
-          hdr[bsel * 4 + 1] = lo;
-          hdr[bsel * 4 + 2] = 0;
+          keep_row[K] = ord[j]; kd[K] = ds[j]; kz[K] = zs[j]; ++K;
+          prev = j;
         }
-        __syncwarp();
-        __threadfence_block();
-        named_arrive(kBarFull + bsel, kParties);
-        bsel ^= 1;
+        float z2 = 0.f;
+        for (int j = 0; j < K; ++j) z2 = fmaf(kz[j], kz[j], z2);
+        s_z2sum = z2;
       }
+      counts[0] = K; counts[1] = ng; counts[2] = nd;
     }
-    named_sync(kBarEmpty + bsel, kParties);
-    if (lane == 0) hdr[bsel * 4 + 2] = 1;                    // end marker
-    __syncwarp();
-    __threadfence_block();
-    named_arrive(kBarFull + bsel, kParties);
-    named_sync(kBarEmpty + (bsel ^ 1), kParties);            // the other list's last hand-back
-  } else if (tid < 32 + D) {
-    const int t = tid - 32;
-    named_arrive(kBarEmpty + 0, kParties);                   // both lists start out free
-    named_arrive(kBarEmpty + 1, kParties);
-    int bsel = 0;
-    while (true) {
-      named_sync(kBarFull + bsel, kParties);
-      if (hdr[bsel * 4 + 2]) break;
-      const int hi = hdr[bsel * 4 + 0], lo = hdr[bsel * 4 + 1];
-      const float* rt = rot + bsel * 2 * D;
-      float carry = Qt[(hi + 1) * LDA + t];
-      for (int i = hi; i >= lo; --i) {
-        const float c = rt[2 * i], s = rt[2 * i + 1];
-        const float zi = Qt[i * LDA + t];
-        Qt[(i + 1) * LDA + t] = fmaf(s, zi, c * carry);
-        carry = fmaf(c, zi, -s * carry);
+    __syncthreads();
+    if (!counts[3]) {
+      const int K = counts[0], ng = counts[1], nd = counts[2];
+      const float rho2 = 2.f * s_rho;
+      // rotations of the deflation on the rows of Qt (one column per thread, in the order recorded)
+      if (tid < D) {
+        for (int g = 0; g < ng; ++g) {
+          const float x = Qt[ga[g] * LDA + tid], y = Qt[gb[g] * LDA + tid];
+          Qt[ga[g] * LDA + tid] = gc[g] * x + gs[g] * y;
+          Qt[gb[g] * LDA + tid] = gc[g] * y - gs[g] * x;
+        }
       }
-      Qt[lo * LDA + t] = carry;
-      __threadfence_block();
-      named_arrive(kBarEmpty + bsel, kParties);
-      bsel ^= 1;
+      // roots: group i = tid / 8 of eight threads, each with the poles j = sub (mod 8)
+      const int gi = tid >> 3, sub = tid & 7;
+      const bool live = gi < K;
+      {
+        const int i = live ? gi : 0;
+        auto fval = [&](int org, float m) {
+          const float d0 = kd[org];
+          float acc = 0.f;
+          for (int j = sub; j < K; j += 8) acc += (kz[j] * kz[j]) / ((kd[j] - d0) - m);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+          acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+          return fmaf(rho2, acc, 1.f);
+        };
+        // the last root lies in (d_{K-1}, d_{K-1} + rho2 |z|^2); every other one between two poles
+        int org = i;
+        const bool last = i >= K - 1;
+        const float width = last ? rho2 * s_z2sum : kd[i + 1] - kd[i];
+        const float mid = 0.5f * width;
+        const float f_mid = fval(i, mid);                  // every thread of the warp takes part
+        float lo_m = 0.f, hi_m = width;
+        if (!last) {
+          if (f_mid >= 0.f) hi_m = mid;                    // root in the left half: offset from pole i
+          else { org = i + 1; lo_m = -mid; hi_m = 0.f; }   // offset from pole i + 1
+        }
+        for (int it = 0; it < 64; ++it) {                  // a fixed count: the groups of a warp stay in step
+          const float m = 0.5f * (lo_m + hi_m);
+          const float fm = fval(org, m);
+          if (m != lo_m && m != hi_m) {
+            if (fm > 0.f) hi_m = m; else lo_m = m;
+          }
+        }
+        if (live && sub == 0) { korg[gi] = org; kmu[gi] = 0.5f * (lo_m + hi_m); }
+      }
+      __syncthreads();
+      // weights recomputed from the roots: zhat_j^2 = prod_i (x_i - d_j) / (rho2 prod_{i != j} (d_i - d_j))
+      {
+        const int j = live ? gi : 0;
+        float prod = 1.f;
+        for (int i = sub; i < K; i += 8) {
+          const float num = (kd[korg[i]] - kd[j]) + kmu[i];
+          prod *= (i == j) ? num / rho2 : num / (kd[i] - kd[j]);
+        }
+        prod *= __shfl_xor_sync(0xffffffffu, prod, 1);
+        prod *= __shfl_xor_sync(0xffffffffu, prod, 2);
+        prod *= __shfl_xor_sync(0xffffffffu, prod, 4);
+        if (live && sub == 0) kzh[gi] = copysignf(sqrtf(fabsf(prod)), kz[gi]);
+      }
+      __syncthreads();
+      // eigenvector i over the kept poles, normalised, as row i of A; its eigenvalue
+      {
+        const int i = live ? gi : 0;
+        const float d0 = kd[korg[i]], mu = kmu[i];
+        float nrm = 0.f;
+        for (int j = sub; j < K; j += 8) {
+          const float v = kzh[j] / ((kd[j] - d0) - mu);
+          nrm = fmaf(v, v, nrm);
+        }
+        nrm += __shfl_xor_sync(0xffffffffu, nrm, 1);
+        nrm += __shfl_xor_sync(0xffffffffu, nrm, 2);
+        nrm += __shfl_xor_sync(0xffffffffu, nrm, 4);
+        const float inv = rsqrtf(nrm);
+        if (live)
+          for (int j = sub; j < K; j += 8) A[gi * LDA + j] = kzh[j] / ((kd[j] - d0) - mu) * inv;
+      }
+      __syncthreads();
+      // rows of the merged basis into L: row i = sum_j A[i][j] Qt[keep_row[j]] (i < K), then the deflated rows
+      for (int i = r; i < K; i += NT / 8) {
+        float acc[CH][4];
+#pragma unroll
+        for (int t = 0; t < CH; ++t)
+#pragma unroll
+          for (int c = 0; c < 4; ++c) acc[t][c] = 0.f;
+        for (int j = 0; j < K; ++j) {
+          const float x = A[i * LDA + j];
+          const float* src = Qt + keep_row[j] * LDA;
+#pragma unroll
+          for (int t = 0; t < CH; ++t) {
+            const float4 y = *reinterpret_cast<const float4*>(&src[4 * (q + 8 * t)]);
+            acc[t][0] = fmaf(x, y.x, acc[t][0]); acc[t][1] = fmaf(x, y.y, acc[t][1]);
+            acc[t][2] = fmaf(x, y.z, acc[t][2]); acc[t][3] = fmaf(x, y.w, acc[t][3]);
+          }
+        }
+#pragma unroll
+        for (int t = 0; t < CH; ++t)
+          *reinterpret_cast<float4*>(&L[i * LDA + 4 * (q + 8 * t)]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+      }
+      for (int e = tid; e < nd * D; e += NT) L[(K + e / D) * LDA + e % D] = Qt[defl_row[e / D] * LDA + e % D];
+      __syncthreads();
+      if (tid < D) de[tid].x = tid < K ? kd[korg[tid]] + kmu[tid] : defl_d[tid - K];
+      float* swap = Qt; Qt = L; L = swap;
     }
+    __syncthreads();
+  }
+  // the factor of the sign rule (its space served the prologue and the merge)
+  if (a.lift) {
+    const double* F = a.lift + mat;
+    for (int e = tid; e < D * D; e += NT) L[(e / D) * LDA + e % D] = (float)F[e];
   }
   __syncthreads();
 
@@ -475,7 +709,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
 }
 
 int launch_pca(const PcaArgs& args, int count, int D, cudaStream_t st) {
-  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 2 * D + 4 * D + 4 + 4 * D) + 8 * sizeof(int);
+  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 6 * D + 4 + 8 * D + 16 * D) + 16 * sizeof(int);
   if (D == 64) {
     auto k = eigh_tql_kernel<64>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));

@@ -196,17 +196,38 @@ def within_cluster_scatter(Y, perm, c):
     return total / N
 
 
+# The orientation of a component is itself a decision taken in floating point: the sign of the entry
+# of largest magnitude of a column of R E.  Where the two largest magnitudes of that column lie this
+# close (relative) and carry opposite signs, either orientation is a valid outcome of the rule.
+SIGN_GAP = 2e-3
+
+
 def check_coordinates(label, w, Qh, Kh, Yq_dev, Yk_dev, pq_dev, pk_dev, adaptive=False):
     """The device's chain from Q and K to the split coordinates against the oracle's own chain.
     Components whose variance is separated from both neighbours by more than 1 % of the largest
     variance must agree element by element (the sign rule is the same on both sides); closer ones
     may rotate inside their pair, in proportion to float32 rounding over the gap, and must still
-    point the same way.  The first split of the two chains is compared before differences can
-    cascade: same coordinate, and the rows that change sides lie no further from the threshold
-    than the two key columns differ.  Last, the two clusterings are equally tight."""
-    Yq_orc, Yk_orc = orc.split_coordinates(Qh, Kh, adaptive=adaptive)
-    for side, Yd, Yo, perm, n in (("queries", Yq_dev, Yq_orc, pq_dev, w.n_q), ("keys", Yk_dev, Yk_orc, pk_dev, w.n_k)):
+    point the same way.  A component that comes out mirrored is accepted only where the sign rule
+    itself is at a near-tie (counted and printed); it is mirrored back for the checks that follow.
+    The first split of the two chains is compared before differences can cascade: same coordinate,
+    and the rows that change sides lie no further from the threshold than the two key columns
+    differ.  Last, the two clusterings are equally tight."""
+    Yq_orc, Yk_orc, Wq, Wk = orc.split_coordinates(Qh, Kh, adaptive=adaptive, return_maps=True)
+    for side, Yd, Yo, Wmap, perm, n in (("queries", Yq_dev, Yq_orc, Wq, pq_dev, w.n_q),
+                                        ("keys", Yk_dev, Yk_orc, Wk, pk_dev, w.n_k)):
         a = coordinates_agreement(Yd, Yo)
+        mirrored = np.nonzero((a["cos"] < 0) & (a["gap"] > 1e-4))[0]
+        if len(mirrored):
+            for t in mirrored:
+                col = Wmap[:, t]
+                top = np.argsort(-np.abs(col))[:2]
+                rel = (abs(col[top[0]]) - abs(col[top[1]])) / abs(col[top[0]])
+                print(f"{label} {side}: component {t} is mirrored; the two largest entries of its column of R E "
+                      f"differ by {rel:.2e} (relative) with signs {np.sign(col[top[0]]):+.0f} / {np.sign(col[top[1]]):+.0f}")
+                assert rel < SIGN_GAP and col[top[0]] * col[top[1]] < 0, "a mirrored component away from a sign near-tie"
+            Yd = np.array(Yd, copy=True)
+            Yd[:, mirrored] *= -1.0
+            a = coordinates_agreement(Yd, Yo)
         sep = a["gap"] > 1e-2
         print(f"{label} {side}: {int(sep.sum())} of {len(sep)} components separated by > 1 % of the largest variance: "
               f"max deviation {a['dev'][sep].max() if sep.any() else 0:.2e} sqrt(var0); all components: "
