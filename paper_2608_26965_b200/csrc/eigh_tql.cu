@@ -19,12 +19,21 @@
 // of Qt in registers for the whole phase (the loops are bound by instruction
 // issue and latency, not by arithmetic); the eight owners of row k+1 build the
 // next reflector right after their update, inside their warp, so no third
-// barrier is needed.  Phase 2: warp 0 runs the QL iteration on (diag, sub-diag)
-// -- the search for a negligible sub-diagonal entry uses all lanes, the rotation
-// chase is one dependent chain on lane 0 -- and hands each chase's rotations
-// through a double-buffered list to d consumer threads, which apply them to the
-// rows of Qt (thread t owns column t), pipelined with the next chase by named
-// barriers.
+// barrier is needed.  Phase 2, divide and conquer: the QL iteration is one
+// dependent chain of about 0.9 n^2 plane rotations for n rows, so the tridiagonal
+// matrix is cut in the middle (T = diag(T1, T2) + rho u u^T) and the two halves are
+// iterated side by side, a quarter of the chain each: per half one warp runs the
+// iteration on (diag, sub-diag) -- the search for a negligible sub-diagonal entry
+// uses all lanes, the rotation chase is one dependent chain on lane 0 -- and hands
+// each chase's rotations through a double-buffered list to consumer threads, which
+// apply them to the rows of Qt of that half (a thread per column), pipelined with
+// the next chase by named barriers.  An extra column that starts as u goes through
+// the same rotations and ends as z = Q^T u.  The merge solves diag(d) + rho z z^T:
+// poles sorted, negligible weights and coinciding poles deflated, the roots of the
+// secular equation by bisection on the offset from the nearer pole (eight threads
+// per root; offsets keep the differences d_j - x accurate), the weights recomputed
+// from the roots (Gu and Eisenstat) so that the eigenvectors stay orthogonal to
+// rounding, and one d x d x d product with the halves' eigenvectors.
 //
 // Epilogue.  Components in order of descending eigenvalue.  With E the
 // eigenvectors and F the factor that produced the transformed rows, the map from
@@ -221,7 +230,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   float* beta = ubuf + 3 * D;                          // [2] (+2)
   float* rot = beta + 4;                               // [2][2][2D] per half: (c, s) of the rotation of rows (i, i+1) at 2i
   int* hdr = reinterpret_cast<int*>(rot + 8 * D);      // [2][2][4]  highest i, lowest i, end marker
-  float* scratch = reinterpret_cast<float*>(hdr + 16); // [16 D]     arrays of the merge
+  float* scratch = reinterpret_cast<float*>(hdr + 16); // [17 D]     arrays of the merge
   __shared__ double s_scale;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -474,7 +483,8 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
     int* gb = ga + D;
     int* defl_row = gb + D;                                // deflated: row of Qt, eigenvalue
     float* defl_d = reinterpret_cast<float*>(defl_row + D);
-    int* counts = reinterpret_cast<int*>(defl_d + D);      // kept, rotations, deflated, skip
+    float* kz2 = defl_d + D;                               // squared weights of the kept poles
+    int* counts = reinterpret_cast<int*>(kz2 + D);         // kept, rotations, deflated, skip
     if (tid < D) {
       const float mine = de[tid].x;
       int rank = 0;
@@ -502,13 +512,14 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         counts[3] = 0;
         for (int j = 0; j < D; ++j) {
           if (rho2 * fabsf(zs[j]) <= tol) { defl_row[nd] = ord[j]; defl_d[nd] = ds[j]; ++nd; continue; }
-          if (prev >= 0) {
+          // two poles coincide when |t c s| <= tol, c = z_j / tau, s = -z_prev / tau, tau^2 = z_j^2 + z_prev^2;
+          // the test is made without the root and the divisions, which only a deflation needs
+          if (prev >= 0 && fabsf((ds[j] - ds[prev]) * zs[j] * zs[prev]) <= tol * fmaf(zs[j], zs[j], zs[prev] * zs[prev])) {
             float sn = zs[prev], cs = zs[j];
             const float tau = sqrtf(fmaf(cs, cs, sn * sn));
-            const float t = ds[j] - ds[prev];
             cs = cs / tau;
             sn = -sn / tau;
-            if (fabsf(t * cs * sn) <= tol) {               // the two poles coincide: rotate the weight into one
+            {                                              // rotate the weight into one of the two
               zs[j] = tau;
               zs[prev] = 0.f;
               gc[ng] = cs; gs[ng] = sn; ga[ng] = ord[prev]; gb[ng] = ord[j]; ++ng;
@@ -523,7 +534,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
           prev = j;
         }
         float z2 = 0.f;
-        for (int j = 0; j < K; ++j) z2 = fmaf(kz[j], kz[j], z2);
+        for (int j = 0; j < K; ++j) { kz2[j] = kz[j] * kz[j]; z2 += kz2[j]; }
         s_z2sum = z2;
       }
       counts[0] = K; counts[1] = ng; counts[2] = nd;
@@ -548,7 +559,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         auto fval = [&](int org, float m) {
           const float d0 = kd[org];
           float acc = 0.f;
-          for (int j = sub; j < K; j += 8) acc += (kz[j] * kz[j]) / ((kd[j] - d0) - m);
+          for (int j = sub; j < K; j += 8) acc += __fdividef(kz2[j], (kd[j] - d0) - m);
           acc += __shfl_xor_sync(0xffffffffu, acc, 1);
           acc += __shfl_xor_sync(0xffffffffu, acc, 2);
           acc += __shfl_xor_sync(0xffffffffu, acc, 4);
@@ -565,7 +576,9 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
           if (f_mid >= 0.f) hi_m = mid;                    // root in the left half: offset from pole i
           else { org = i + 1; lo_m = -mid; hi_m = 0.f; }   // offset from pole i + 1
         }
-        for (int it = 0; it < 64; ++it) {                  // a fixed count: the groups of a warp stay in step
+        for (int it = 0; it < 44; ++it) {                  // a fixed count: the groups of a warp stay in step
+          // (44 halvings take an interval of width w down to the float spacing of offsets >= 2^-20 w;
+          // a root closer to its pole than that belongs to a weight that the deflation has removed)
           const float m = 0.5f * (lo_m + hi_m);
           const float fm = fval(org, m);
           if (m != lo_m && m != hi_m) {
@@ -709,7 +722,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
 }
 
 int launch_pca(const PcaArgs& args, int count, int D, cudaStream_t st) {
-  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 6 * D + 4 + 8 * D + 16 * D) + 16 * sizeof(int);
+  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 6 * D + 4 + 8 * D + 17 * D) + 16 * sizeof(int);
   if (D == 64) {
     auto k = eigh_tql_kernel<64>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
