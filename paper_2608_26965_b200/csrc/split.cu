@@ -101,6 +101,64 @@ __device__ __forceinline__ void staged_variances(const float* tiles, int ng, Row
   }
 }
 
+// The same estimate for `ng` subsets at once, the sample rows read straight from the coordinates
+// in global memory (sub[gi * D + j]: row of sample j of subset gi, -1 beyond its m rows).  Same
+// operations in the same order as staged_variances, hence the same bits; what differs is the
+// parallelism: every (subset, residue, coordinate) is a thread's task, so a round of many small
+// subsets keeps all warps busy between two barriers, and a task's loads (one per sample row of its
+// residue) are all in flight together.
+template <int D, typename RowsOf>
+__device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, const int* sub, int ng, RowsOf rows_of,
+                                                   float* part, float* out, int tid, int nt) {
+  constexpr int PER = D / 8;                       // sample rows of a residue
+  constexpr int Q4 = D / 4;                        // 16-byte vectors of a row
+  constexpr int B = 4;                             // loads in flight per task
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int task = tid; task < ng * 8 * Q4; task += nt) {
+      const int gi = task / (8 * Q4), r = (task / Q4) % 8, t4 = task % Q4;
+      const int m = rows_of(gi);
+      float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (pass == 1) mean = *reinterpret_cast<const float4*>(out + gi * D + 4 * t4);
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int k0 = 0; k0 < PER; k0 += B) {
+        float4 x[B];
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+          const int j = r + 8 * (k0 + k);
+          const int row = j < m ? sub[gi * D + j] : -1;
+          x[k] = row >= 0 ? __ldg(reinterpret_cast<const float4*>(Y + (size_t)row * D) + t4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+          if (r + 8 * (k0 + k) < m) {
+            if (pass == 0) {
+              acc.x = __fadd_rn(acc.x, x[k].x); acc.y = __fadd_rn(acc.y, x[k].y);
+              acc.z = __fadd_rn(acc.z, x[k].z); acc.w = __fadd_rn(acc.w, x[k].w);
+            } else {
+              const float dx = __fsub_rn(x[k].x, mean.x), dy = __fsub_rn(x[k].y, mean.y);
+              const float dz = __fsub_rn(x[k].z, mean.z), dw = __fsub_rn(x[k].w, mean.w);
+              acc.x = __fadd_rn(acc.x, __fmul_rn(dx, dx)); acc.y = __fadd_rn(acc.y, __fmul_rn(dy, dy));
+              acc.z = __fadd_rn(acc.z, __fmul_rn(dz, dz)); acc.w = __fadd_rn(acc.w, __fmul_rn(dw, dw));
+            }
+          }
+        }
+      }
+      *reinterpret_cast<float4*>(part + (gi * 8 + r) * D + 4 * t4) = acc;
+    }
+    __syncthreads();
+    for (int task = tid; task < ng * D; task += nt) {
+      const int gi = task / D, t = task % D;
+      const float* p = part + gi * 8 * D + t;
+      const float tot = __fadd_rn(__fadd_rn(__fadd_rn(p[0], p[D]), __fadd_rn(p[2 * D], p[3 * D])),
+                                  __fadd_rn(__fadd_rn(p[4 * D], p[5 * D]), __fadd_rn(p[6 * D], p[7 * D])));
+      const int m = rows_of(gi);
+      out[task] = m > 0 ? __fdiv_rn(tot, (float)m) : -1.0f;
+    }
+    __syncthreads();
+  }
+}
+
 // 16-byte asynchronous copy global -> shared (no registers held while in flight)
 __device__ __forceinline__ void cp_async16(void* smem_dst, const void* gmem_src) {
   const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(smem_dst));
@@ -409,35 +467,30 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
     int32_t* rows_next = sm.rows[cur ^ 1];
 
     // ---- 1. coordinate of largest subsample variance for every subset that still splits.
-    // The subsamples are staged, a few subsets at a time, in the 64 KB that keys/scan/hist
-    // occupy later in the level.
+    // Rounds of up to 1024 / D subsets: their sample rows are located (one division per row), then
+    // every (subset, residue, coordinate) is a thread's task that reads its sample values straight
+    // from the coordinates; partial sums, means and variances live in the 64 KB that keys, scan and
+    // hist occupy later in the level.
     {
-      float* stage = reinterpret_cast<float*>(sm.keys);
-      constexpr int per_group = (16384 / (D * D)) > 0 ? 16384 / (D * D) : 1;     // 4 (d=64) or 1 (d=128)
-      constexpr int q = D / 4;
-      for (int g0 = 0; g0 < nseg; g0 += per_group) {
-        const int ng = min(per_group, nseg - g0);
-        // rows of the subsamples (one division per row), then the tiles by asynchronous copies
+      float* part = reinterpret_cast<float*>(sm.keys);                 // [G][8][D]
+      constexpr int G = 1024 / D;
+      float* vout = part + G * 8 * D;                                  // [G][D] means, then variances
+      int* sub_rows = reinterpret_cast<int*>(vout + G * D);            // [G][D]
+      for (int g0 = 0; g0 < nseg; g0 += G) {
+        const int ng = min(G, nseg - g0);
         for (int e = tid; e < ng * D; e += nt) {
           const int gi = e / D, j = e % D;
           const int a = slo[g0 + gi], sz = slo[g0 + gi + 1] - a;
           const int m = min(D, sz);
-          sm.sub_rows[e] = (sz > c && j < m) ? rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)] : -1;
+          sub_rows[e] = (sz > c && j < m) ? rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)] : -1;
         }
         __syncthreads();
-        for (int e = tid; e < ng * D * q; e += nt) {
-          const int row = sm.sub_rows[e / q];
-          if (row >= 0)
-            cp_async16(reinterpret_cast<float4*>(stage) + e, reinterpret_cast<const float4*>(Y + (size_t)row * D) + (e % q));
-        }
-        cp_async_wait_all();
-        __syncthreads();
-        staged_variances<D>(stage, ng,
-                         [&](int gi) { const int sz = slo[g0 + gi + 1] - slo[g0 + gi]; return sz > c ? min(D, sz) : 0; },
-                         sm.vpart, sm.vout, tid, nt);
+        gathered_variances<D>(Y, sub_rows, ng,
+                              [&](int gi) { const int sz = slo[g0 + gi + 1] - slo[g0 + gi]; return sz > c ? min(D, sz) : 0; },
+                              part, vout, tid, nt);
         for (int task = tid; task < ng * D; task += nt) {
           const int gi = task / D, t = task % D, g = g0 + gi;
-          float v = sm.vout[task];                     // -1 for a subset that is already final
+          float v = vout[task];                        // -1 for a subset that is already final
           // argmax inside the warp (32 consecutive coordinates), lowest coordinate on ties
           int at = t;
           for (int o = 16; o > 0; o >>= 1) {
