@@ -76,6 +76,12 @@ struct TcCfg {
   static constexpr int K_LEAD = 2;
   static constexpr int K_LEAD_CEN = 1;
   static constexpr int PV_N = D;
+  // How the softmax notices a probability above 2^threshold.  d = 128: it keeps the largest
+  // exponent of the half-step.  d = 64: no exponent is tracked; such a probability shows in its
+  // chunk's row sum, and the sum bounds it from above, so the reference moves up by the sum's
+  // exponent (too far by at most log2(32), which costs nothing in fp32 / bf16).  Measured: d = 64
+  // 0.916 -> 0.895 ms without the tracking, d = 128 2.90 -> 2.95 ms.
+  static constexpr bool TRACK_MAX = D != 64;
   static constexpr bool Q_IN_TMEM = false;
   static constexpr int TMEM_Q = 0;
   // shared memory layout (offsets from a 1024-byte aligned base)
@@ -385,8 +391,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       const int qrow = (p * prm.n_qc + qc) * prm.c_q + half * kTile + (row < q_rows ? row : 0);
       row_sc *= prm.q_scale[qrow];
     }
-    bool ok = true;
-    for (int u = 0; u < steps && ok; ++u) {
+    // A warp whose wait gave up goes through the remaining half-steps without touching anything
+    // (`dead`), so that it still meets the other softmax warps at the barriers they share.
+    bool dead = false;
+    for (int u = 0; u < steps; ++u) {
       const int b = u & 1;                               // half of a 128-row tile (geometry of the keys)
       const int buf = u % C::NBUF;                       // score buffer
       const uint32_t t_s = tmem_s + lane_addr + buf * kHalf;
@@ -421,6 +429,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         if (st < kHalf) bz[st] = use ? log2f((float)cnt[min(j, prm.n_kc - 1)]) : -INFINITY;
       }
       if (masked) asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (dead) continue;
       // scale of this half-step's scores.  A zero scale (an all-zero query row or key group) makes
       // every logit 0: the raw scores are then dropped and the additive terms enter with scale 1.
       float sc_used = prm.scale_log2;
@@ -433,8 +442,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         sc_used = keep_raw ? sc_eff : (masked ? 1.f : 0.f);
       }
 
-      ok = __all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
-      if (!ok) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(b_s_full(u % C::NBAR), (u / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit))) {
+        dead = true;
+        continue;
+      }
       tc_fence_after();
       if (quarter * 32 >= q_rows) {          // this warp's rows are padding of a 64-row query cluster
         tc_fence_before();
@@ -510,8 +521,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         l_run *= alpha;
         if (u > 0) {
           // products complete in the order of their issue: once P V (u-1) is complete, all earlier are
-          ok = __all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit));
-          if (!ok) break;
+          if (!__all_sync(0xffffffffu, mbar_wait(b_pv_done((u - 1) % C::NBAR), ((u - 1) / C::NBAR) & 1, abort_flag, prm.status, prm.wait_limit))) {
+            dead = true;
+            continue;
+          }
           tc_fence_after();
 #pragma unroll 1
           for (int c4 = 0; c4 < D / 32; ++c4) {
@@ -529,6 +542,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
       float neg_m = (m_ref == -INFINITY) ? 0.f : -m_ref;
       const f32x2 sc2 = pack2(sc_used, sc_used);
       float cm0 = -INFINITY, cm1 = -INFINITY;            // maximum of x - m_ref over the half-step
+      float big = 0.f;                                   // larger of the two chunk sums of the half-step
 #pragma unroll 1
       for (int c4 = 0; c4 < 2; ++c4) {
         uint32_t r[32];
@@ -552,8 +566,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         for (int g = 0; g < 10; ++g) {
           if (g < 8) {
             const int j = 4 * g;
-            cm0 = max3(cm0, x[j], x[j + 1]);
-            cm1 = max3(cm1, x[j + 2], x[j + 3]);
+            if (C::TRACK_MAX) {
+              cm0 = max3(cm0, x[j], x[j + 1]);
+              cm1 = max3(cm1, x[j + 2], x[j + 3]);
+            }
 #pragma unroll
             for (int e = j; e < j + 4; ++e) x[e] = ex2_approx(x[e]);
           }
@@ -571,12 +587,17 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
         unpack2(s23, sc, sd);
         const float chunk_sum = (sa + sb) + (sc + sd);
         l_run += chunk_sum;
+        if (!C::TRACK_MAX) big = fmaxf(big, chunk_sum);
         tmem_st16(t_s + c4 * 16, pk);
       }
-      {
+      if (C::TRACK_MAX) {
         const float hm = fmaxf(cm0, cm1);
         if (hm > kRescaleThreshold) pend = ceilf(hm);
         if (__any_sync(0xffffffffu, hm > kDanger)) *redo_flag = 1;
+      } else {
+        // a sum that is not below 2^kDanger (infinite or NaN included) marks the tile
+        if (big > 256.0f) pend = ceilf(log2f(big));
+        if (__any_sync(0xffffffffu, !(big < 7.9228163e28f))) *redo_flag = 1;
       }
       // one arrival per warp: 128 arrivals on one barrier word would be serialised in shared memory
       tmem_wait_st();
@@ -586,6 +607,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__
     }
 
     // epilogue: O / l, rows back to their original positions
+    bool ok = !dead;
     if (ok) ok = __all_sync(0xffffffffu, mbar_wait(b_o_done, 0, abort_flag, prm.status, prm.wait_limit));
     tc_fence_after();
     if (ok) {                                          // warp-uniform: TMEM loads are warp-collective

@@ -3,8 +3,8 @@
 // for k = 0, 1, ..., product and sum rounded separately, no fused multiply-add),
 // so the scores -- and with them the selection -- are reproducible bit for bit;
 // the k best per query cluster by (score descending, index ascending), written
-// in ascending index order.  With few key clusters one kernel scores and
-// selects; with many, the scores are computed in tiles first (score_tile_kernel).
+// in ascending index order.  With fewer than 128 key clusters one kernel scores
+// and selects; otherwise the scores are computed in tiles first (score_tile_kernel).
 // The second half of the file is the adaptive (mass-recall) selection.
 #include "kernels.h"
 
@@ -12,7 +12,9 @@ namespace ca {
 
 constexpr int kSelectThreads = 256;
 constexpr int kSelectQT = 4;          // query clusters per CTA (key centroids are read once for all)
-constexpr int kSelectTiledMinClusters = 2048;   // from here on the scores are computed in tiles first
+// From this many key clusters on the scores are computed in tiles first: measured faster from 128
+// clusters up (0.041 -> 0.030 ms at 512 x 128 clusters of 16 heads, 0.75 -> 0.56 ms at 1024 x 1024).
+constexpr int kSelectTiledMinClusters = 128;
 
 __device__ __forceinline__ uint32_t score_key(float s) {
   if (s == 0.0f) s = 0.0f;                        // -0 and +0 compare equal
