@@ -195,23 +195,66 @@ __device__ __forceinline__ void ql_consumer(float* Qt, int lda, int t, int ncols
 
 }  // namespace
 
-// this thread's columns j = 4 (q + 8 t) + c of  acc[j] = sum_k x(k) Y[k][j]
-template <int D, typename XF>
-__device__ __forceinline__ void row_times_matrix(XF x_of_k, const float* __restrict__ Y, int lda, int q,
-                                                 float (&acc)[D / 32][4]) {
+// d x d x d products in shared memory, a 4 x 4 tile of the result per thread (the first d^2 / 16
+// threads; every shared-memory load feeds four or sixteen multiply-adds, and the lanes of a
+// quarter-warp read distinct banks).  Terms are added for k = 0, 1, ... in that order.
+//   XT = false: acc[a][b] = sum_k X[(4 ti + a) lda + k] Y[k lda + 4 tj + b]
+//   XT = true:  acc[a][b] = sum_k X[k lda + 4 ti + a]   Y[k lda + 4 tj + b]
+template <int D, bool XT>
+__device__ __forceinline__ void tile_product(const float* __restrict__ X, const float* __restrict__ Y, int lda,
+                                             int ti, int tj, float (&acc)[4][4]) {
 #pragma unroll
-  for (int t = 0; t < D / 32; ++t)
+  for (int x = 0; x < 4; ++x)
 #pragma unroll
-    for (int c = 0; c < 4; ++c) acc[t][c] = 0.f;
-#pragma unroll 4
-  for (int k = 0; k < D; ++k) {
-    const float x = x_of_k(k);
+    for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+#pragma unroll 2
+  for (int k0 = 0; k0 < D; k0 += 4) {
+    float xa[4][4];                                    // [row][k]
 #pragma unroll
-    for (int t = 0; t < D / 32; ++t) {
-      const float4 y = *reinterpret_cast<const float4*>(&Y[k * lda + 4 * (q + 8 * t)]);
-      acc[t][0] = fmaf(x, y.x, acc[t][0]); acc[t][1] = fmaf(x, y.y, acc[t][1]);
-      acc[t][2] = fmaf(x, y.z, acc[t][2]); acc[t][3] = fmaf(x, y.w, acc[t][3]);
+    for (int e = 0; e < 4; ++e) {
+      if (XT) {
+        const float4 v = *reinterpret_cast<const float4*>(&X[(k0 + e) * lda + 4 * ti]);
+        xa[0][e] = v.x; xa[1][e] = v.y; xa[2][e] = v.z; xa[3][e] = v.w;
+      } else {
+        const float4 v = *reinterpret_cast<const float4*>(&X[(4 * ti + e) * lda + k0]);
+        xa[e][0] = v.x; xa[e][1] = v.y; xa[e][2] = v.z; xa[e][3] = v.w;
+      }
     }
+#pragma unroll
+    for (int kk = 0; kk < 4; ++kk) {
+      const float4 y = *reinterpret_cast<const float4*>(&Y[(k0 + kk) * lda + 4 * tj]);
+#pragma unroll
+      for (int x = 0; x < 4; ++x) {
+        acc[x][0] = fmaf(xa[x][kk], y.x, acc[x][0]); acc[x][1] = fmaf(xa[x][kk], y.y, acc[x][1]);
+        acc[x][2] = fmaf(xa[x][kk], y.z, acc[x][2]); acc[x][3] = fmaf(xa[x][kk], y.w, acc[x][3]);
+      }
+    }
+  }
+}
+
+// acc[a][c] = sum_k X[(4 ti + a) lda + k] Yr[(tj + (D / 4) c) lda + k]   (both operands by rows)
+template <int D>
+__device__ __forceinline__ void tile_product_rows(const float* __restrict__ X, const float* __restrict__ Yr, int lda,
+                                                  int ti, int tj, float (&acc)[4][4]) {
+#pragma unroll
+  for (int x = 0; x < 4; ++x)
+#pragma unroll
+    for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+#pragma unroll 2
+  for (int k0 = 0; k0 < D; k0 += 4) {
+    float4 xv[4], yv[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      xv[e] = *reinterpret_cast<const float4*>(&X[(4 * ti + e) * lda + k0]);
+      yv[e] = *reinterpret_cast<const float4*>(&Yr[(tj + (D / 4) * e) * lda + k0]);
+    }
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+      for (int y = 0; y < 4; ++y) {
+        acc[x][y] = fmaf(xv[x].x, yv[y].x, acc[x][y]); acc[x][y] = fmaf(xv[x].y, yv[y].y, acc[x][y]);
+        acc[x][y] = fmaf(xv[x].z, yv[y].z, acc[x][y]); acc[x][y] = fmaf(xv[x].w, yv[y].w, acc[x][y]);
+      }
   }
 }
 
@@ -236,6 +279,9 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int r = tid >> 3, q = tid & 7;
   const size_t mat = (size_t)blockIdx.x * D * D;
+  // d x d x d products: a 4 x 4 tile per thread, the first d^2 / 16 threads
+  constexpr int TILE_THREADS = D * D / 16;
+  const int tile_i = tid / (D / 4), tile_j = tid % (D / 4);
 
   // ---- prologue: the matrix to decompose, in A
   if (a.lift) {
@@ -253,18 +299,22 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
       A[i * LDA + j] = (float)fma(-cn * sm[i], sm[j], G[e] * cs);
     }
     __syncthreads();
-    float acc[CH][4];
-    row_times_matrix<D>([&](int k) { return L[k * LDA + r]; }, A, LDA, q, acc);        // (F^T C)[r][.]
+    float acc[4][4];
+    if (tid < TILE_THREADS) {
+      tile_product<D, true>(L, A, LDA, tile_i, tile_j, acc);                              // F^T C
 #pragma unroll
-    for (int t = 0; t < CH; ++t)
-      *reinterpret_cast<float4*>(&Qt[r * LDA + 4 * (q + 8 * t)]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+      for (int x = 0; x < 4; ++x)
+        *reinterpret_cast<float4*>(&Qt[(4 * tile_i + x) * LDA + 4 * tile_j]) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+    }
     __syncthreads();
-    row_times_matrix<D>([&](int k) { return Qt[r * LDA + k]; }, L, LDA, q, acc);       // ((F^T C) F)[r][.]
-    const float al = (float)a.alpha;
+    if (tid < TILE_THREADS) {
+      tile_product<D, false>(Qt, L, LDA, tile_i, tile_j, acc);                            // (F^T C) F
+      const float al = (float)a.alpha;
 #pragma unroll
-    for (int t = 0; t < CH; ++t)
-      *reinterpret_cast<float4*>(&A[r * LDA + 4 * (q + 8 * t)]) =
-          make_float4(al * acc[t][0], al * acc[t][1], al * acc[t][2], al * acc[t][3]);
+      for (int x = 0; x < 4; ++x)
+        *reinterpret_cast<float4*>(&A[(4 * tile_i + x) * LDA + 4 * tile_j]) =
+            make_float4(al * acc[x][0], al * acc[x][1], al * acc[x][2], al * acc[x][3]);
+    }
   } else if (a.mode == kPcaQueries) {
     // covariance of the stored representation: gram / n - mean mean^T
     const double* G = a.gram + mat;
@@ -620,25 +670,45 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
       }
       __syncthreads();
       // rows of the merged basis into L: row i = sum_j A[i][j] Qt[keep_row[j]] (i < K), then the deflated rows
-      for (int i = r; i < K; i += NT / 8) {
-        float acc[CH][4];
+      // (a 4 x 4 tile per thread, terms in the order of j)
+      if (tid < TILE_THREADS && 4 * tile_i < K) {
+        const int i0 = 4 * tile_i;
+        float acc[4][4];
 #pragma unroll
-        for (int t = 0; t < CH; ++t)
+        for (int x = 0; x < 4; ++x)
 #pragma unroll
-          for (int c = 0; c < 4; ++c) acc[t][c] = 0.f;
-        for (int j = 0; j < K; ++j) {
-          const float x = A[i * LDA + j];
-          const float* src = Qt + keep_row[j] * LDA;
+          for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+        int j = 0;
+        for (; j + 4 <= K; j += 4) {
+          float xa[4][4];
 #pragma unroll
-          for (int t = 0; t < CH; ++t) {
-            const float4 y = *reinterpret_cast<const float4*>(&src[4 * (q + 8 * t)]);
-            acc[t][0] = fmaf(x, y.x, acc[t][0]); acc[t][1] = fmaf(x, y.y, acc[t][1]);
-            acc[t][2] = fmaf(x, y.z, acc[t][2]); acc[t][3] = fmaf(x, y.w, acc[t][3]);
+          for (int x = 0; x < 4; ++x) {
+            const float4 v = *reinterpret_cast<const float4*>(&A[(i0 + x) * LDA + j]);
+            xa[x][0] = v.x; xa[x][1] = v.y; xa[x][2] = v.z; xa[x][3] = v.w;
+          }
+#pragma unroll
+          for (int kk = 0; kk < 4; ++kk) {
+            const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j + kk] * LDA + 4 * tile_j]);
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              acc[x][0] = fmaf(xa[x][kk], y.x, acc[x][0]); acc[x][1] = fmaf(xa[x][kk], y.y, acc[x][1]);
+              acc[x][2] = fmaf(xa[x][kk], y.z, acc[x][2]); acc[x][3] = fmaf(xa[x][kk], y.w, acc[x][3]);
+            }
+          }
+        }
+        for (; j < K; ++j) {
+          const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j] * LDA + 4 * tile_j]);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            const float xv = A[(i0 + x) * LDA + j];
+            acc[x][0] = fmaf(xv, y.x, acc[x][0]); acc[x][1] = fmaf(xv, y.y, acc[x][1]);
+            acc[x][2] = fmaf(xv, y.z, acc[x][2]); acc[x][3] = fmaf(xv, y.w, acc[x][3]);
           }
         }
 #pragma unroll
-        for (int t = 0; t < CH; ++t)
-          *reinterpret_cast<float4*>(&L[i * LDA + 4 * (q + 8 * t)]) = make_float4(acc[t][0], acc[t][1], acc[t][2], acc[t][3]);
+        for (int x = 0; x < 4; ++x)
+          if (i0 + x < K)
+            *reinterpret_cast<float4*>(&L[(i0 + x) * LDA + 4 * tile_j]) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
       }
       for (int e = tid; e < nd * D; e += NT) L[(K + e / D) * LDA + e % D] = Qt[defl_row[e / D] * LDA + e % D];
       __syncthreads();
@@ -655,22 +725,13 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   __syncthreads();
 
   // ---- the map from the original space, W = F E (W[i][j] = sum_k F[i][k] Qt[j][k]), into A
-  constexpr int PER = D / 8;
-  if (a.lift) {
-    float acc[PER];
+  if (a.lift && tid < TILE_THREADS) {
+    float acc[4][4];
+    tile_product_rows<D>(L, Qt, LDA, tile_i, tile_j, acc);
 #pragma unroll
-    for (int t = 0; t < PER; ++t) acc[t] = 0.f;
-    for (int k = 0; k < D; k += 4) {
-      const float4 f = *reinterpret_cast<const float4*>(&L[r * LDA + k]);
+    for (int x = 0; x < 4; ++x)
 #pragma unroll
-      for (int t = 0; t < PER; ++t) {
-        const float4 ev = *reinterpret_cast<const float4*>(&Qt[(q + 8 * t) * LDA + k]);
-        acc[t] = fmaf(f.x, ev.x, acc[t]); acc[t] = fmaf(f.y, ev.y, acc[t]);
-        acc[t] = fmaf(f.z, ev.z, acc[t]); acc[t] = fmaf(f.w, ev.w, acc[t]);
-      }
-    }
-#pragma unroll
-    for (int t = 0; t < PER; ++t) A[r * LDA + q + 8 * t] = acc[t];
+      for (int y = 0; y < 4; ++y) A[(4 * tile_i + x) * LDA + tile_j + (D / 4) * y] = acc[x][y];
   }
   // ---- order, sign, bias
   double* lam = reinterpret_cast<double*>(vbuf);             // [D] doubles over vbuf's 2D floats
