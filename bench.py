@@ -44,8 +44,8 @@ FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustain
 # was captured from: sha256 of csrc/attn_tc.cu + csrc/tc_ptx.cuh, first 16 hex digits.  When the
 # source has changed since, the bench prints null instead of a stale figure.
 NCU_TRAFFIC = {
-    "tabular": {"bytes": 568.3e6, "source": "6b538db0b9316f3e", "commit": "8346370"},
-    "video480": {"bytes": 1274.8e6, "source": "6b538db0b9316f3e", "commit": "8346370"},
+    "tabular": {"bytes": 577.2e6, "source": "932f684fa31e5a09", "commit": "3110b1f"},
+    "video480": {"bytes": 1264.8e6, "source": "932f684fa31e5a09", "commit": "3110b1f"},
 }
 # FP32 FMA rate of the CUDA cores, the roof of kernels bound by plain arithmetic (centroid scoring,
 # the fp32 attention kernel): 148 SMs x 128 FMA lanes x 2 flops x 1.965 GHz (the maximum SM clock).
