@@ -159,6 +159,51 @@ def oracle_sample_step(w, Q, K, V, n_query_clusters=8, budget_rows=32768):
     return flops, dt, desc
 
 
+def decision_report(w, keep, flags, Qh, Kh, Vh, dev, head=0):
+    """Part of the cpu_baseline leg: the integer decisions the device takes for one head of the timed
+    workload (cluster permutations, block lists) against the oracle -- bit for bit against its
+    float32 restatement on the device's own coordinates and centroids, and counted against its
+    float64 definitions (differing split nodes, rows that end in another cluster, differing lists)."""
+    import numpy as np
+    import torch
+
+    from oracle import clusterattn_oracle as orc
+    from paper_2608_26965_b200 import binding
+    from tests import decisions as dec
+
+    w1 = w.scaled(heads=1)
+    p1 = binding.problem_from_workload(w1, keep=keep, flags=flags)
+    plan = binding.Plan(p1, dev, keep_y=True)
+    dt = binding.torch_dtype(p1)
+    Q, K, V = (torch.from_numpy(a[head:head + 1][None]).to(dt).to(dev) for a in (Qh, Kh, Vh))
+    plan.cluster_qk(Q, K, V)
+    plan.select_blocks()
+    torch.cuda.synchronize()
+    c = w.cluster
+    out = {"head": head, "sides": {}}
+    for side, Y, perm in (("queries", plan.Yq, plan.perm_q), ("keys", plan.Yk, plan.perm_k)):
+        Yh, ph = Y[0, 0].cpu().numpy(), perm[0, 0].cpu().numpy()
+        exact = bool(np.array_equal(ph, orc.recursive_split_f32(Yh, c)))
+        rec = {"permutation_equals_float32_restatement": exact}
+        if exact:
+            a = dec.split_agreement(Yh, c, ph)
+            rec.update(rows=a["rows"], split_nodes=a["nodes"], nodes_differing_from_float64=a["differing_nodes"],
+                       of_them_not_near_ties=a["differing_nodes_not_near_tie"],
+                       rows_in_another_cluster=a["rows_moved"],
+                       rows_near_a_threshold=a["near_threshold_rows"], near_means="within 1e-6 of the spread of the set's keys")
+        out["sides"][side] = rec
+    cq, ck = plan.cq[0, 0].cpu().numpy(), plan.ck[0, 0].cpu().numpy()
+    idx = plan.block_idx[0, 0].cpu().numpy()
+    exact = bool(np.array_equal(idx, orc.select_blocks_f32(cq, ck, keep)))
+    sel = {"lists_equal_float32_restatement": exact}
+    if exact:
+        a = dec.selection_agreement(cq, ck, keep, idx)
+        sel.update(lists=a["lists"], lists_differing_from_float64=a["differing_lists"],
+                   of_them_not_near_ties=a["differing_lists_not_near_tie"], near_tie_lists=a["near_tie_lists"])
+    out["selection"] = sel
+    return out
+
+
 def run_reference(args, w):
     from paper_2608_26965_b200 import inputs
     rank = int(os.environ.get("RANK", "0"))
@@ -692,6 +737,8 @@ def run_ours(args, w):
         line["cpu_baseline"] = {"value": flops / secs / 1e12, "unit": UNIT, "cores": host_cores(),
                                 "kind": "oracle", "seconds": secs,
                                 "sample": f"{used} of {heads} heads in full (all stages, fp64 numpy)"}
+        if not adaptive and not basic:
+            line["decisions_vs_oracle"] = decision_report(w, keep, p.flags, Qh, Kh, Vh, dev)
     print(json.dumps(line))
     replicas.shutdown()
 

@@ -52,3 +52,11 @@ def test_bench_line_has_the_contract_keys():
     assert dense["speedup_vs_fastest_dense"] > 1.0
     sec = line["secondary"]
     assert sec["workload"] == "video480" and sec["head_dim"] == 128 and 0 < sec["roofline"]["frac"] < 1.2
+    # the device's integer decisions for one head of the timed workload against the oracle
+    dec = line["decisions_vs_oracle"]
+    for side in ("queries", "keys"):
+        rec = dec["sides"][side]
+        assert rec["permutation_equals_float32_restatement"] is True
+        assert rec["of_them_not_near_ties"] == 0 and rec["rows_in_another_cluster"] < 1e-3 * rec["rows"]
+    assert dec["selection"]["lists_equal_float32_restatement"] is True
+    assert dec["selection"]["of_them_not_near_ties"] == 0
