@@ -538,6 +538,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
     if (tid < D) {
       const float mine = de[tid].x;
       int rank = 0;
+#pragma unroll 16
       for (int k = 0; k < D; ++k) {
         const float other = de[k].x;
         rank += (other < mine) || (other == mine && k < tid);
@@ -550,49 +551,71 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
       zs[tid] = Qt[ord[tid] * LDA + D] * 0.70710678f;
     }
     __syncthreads();
-    if (tid == 0) {
+    if (tid < 32) {
       const float rho2 = 2.f * s_rho;
       float dmax = 0.f, zmax = 0.f;
-      for (int j = 0; j < D; ++j) { dmax = fmaxf(dmax, fabsf(ds[j])); zmax = fmaxf(zmax, fabsf(zs[j])); }
+      for (int j = lane; j < D; j += 32) { dmax = fmaxf(dmax, fabsf(ds[j])); zmax = fmaxf(zmax, fabsf(zs[j])); }
+      for (int o = 16; o > 0; o >>= 1) {
+        dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+        zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+      }
       const float tol = 8.f * 6e-8f * fmaxf(dmax, zmax);
-      int K = 0, ng = 0, nd = 0, prev = -1;
-      if (rho2 * zmax <= tol) {
+      int K = 0, ng = 0, nd = 0;
+      if (tid != 0) {
+        // the scan below is one thread's
+      } else if (rho2 * zmax <= tol) {
         counts[3] = 1;                                     // the halves do not couple: nothing to merge
       } else {
         counts[3] = 0;
+        // one pass over the sorted poles; the last kept pole and the next pole travel in registers
+        // (every step would otherwise wait for the shared-memory round trip of the step before)
+        float d_prev = 0.f, z_prev = 0.f;
+        int o_prev = -1;
+        float dj = ds[0], zj = zs[0];
+        int oj = ord[0];
         for (int j = 0; j < D; ++j) {
-          if (rho2 * fabsf(zs[j]) <= tol) { defl_row[nd] = ord[j]; defl_d[nd] = ds[j]; ++nd; continue; }
-          // two poles coincide when |t c s| <= tol, c = z_j / tau, s = -z_prev / tau, tau^2 = z_j^2 + z_prev^2;
-          // the test is made without the root and the divisions, which only a deflation needs
-          if (prev >= 0 && fabsf((ds[j] - ds[prev]) * zs[j] * zs[prev]) <= tol * fmaf(zs[j], zs[j], zs[prev] * zs[prev])) {
-            float sn = zs[prev], cs = zs[j];
-            const float tau = sqrtf(fmaf(cs, cs, sn * sn));
-            cs = cs / tau;
-            sn = -sn / tau;
-            {                                              // rotate the weight into one of the two
-              zs[j] = tau;
-              zs[prev] = 0.f;
-              gc[ng] = cs; gs[ng] = sn; ga[ng] = ord[prev]; gb[ng] = ord[j]; ++ng;
-              const float tt = ds[prev] * cs * cs + ds[j] * sn * sn;
-              ds[j] = ds[prev] * sn * sn + ds[j] * cs * cs;
-              ds[prev] = tt;
-              --K;                                         // prev is the last kept pole
-              defl_row[nd] = ord[prev]; defl_d[nd] = tt; ++nd;
+          const int jn = j + 1 < D ? j + 1 : j;
+          const float dn = ds[jn], zn = zs[jn];
+          const int on = ord[jn];
+          if (rho2 * fabsf(zj) <= tol) {
+            defl_row[nd] = oj; defl_d[nd] = dj; ++nd;
+          } else {
+            // two poles coincide when |t c s| <= tol, c = z_j / tau, s = -z_prev / tau, tau^2 = z_j^2 + z_prev^2;
+            // the test is made without the root and the divisions, which only a deflation needs
+            if (o_prev >= 0 && fabsf((dj - d_prev) * zj * z_prev) <= tol * fmaf(zj, zj, z_prev * z_prev)) {
+              float sn = z_prev, cs = zj;
+              const float tau = sqrtf(fmaf(cs, cs, sn * sn));
+              cs = cs / tau;
+              sn = -sn / tau;
+              // rotate the weight into pole j; the other of the two is deflated
+              gc[ng] = cs; gs[ng] = sn; ga[ng] = o_prev; gb[ng] = oj; ++ng;
+              const float tt = d_prev * cs * cs + dj * sn * sn;
+              dj = d_prev * sn * sn + dj * cs * cs;
+              zj = tau;
+              --K;                                         // the last kept pole gives way
+              defl_row[nd] = o_prev; defl_d[nd] = tt; ++nd;
             }
+            keep_row[K] = oj; kd[K] = dj; kz[K] = zj; ++K;
+            d_prev = dj; z_prev = zj; o_prev = oj;
           }
-          keep_row[K] = ord[j]; kd[K] = ds[j]; kz[K] = zs[j]; ++K;
-          prev = j;
+          dj = dn; zj = zn; oj = on;
         }
-        float z2 = 0.f;
-        for (int j = 0; j < K; ++j) { kz2[j] = kz[j] * kz[j]; z2 += kz2[j]; }
-        s_z2sum = z2;
       }
-      counts[0] = K; counts[1] = ng; counts[2] = nd;
+      if (tid == 0) { counts[0] = K; counts[1] = ng; counts[2] = nd; }
     }
     __syncthreads();
     if (!counts[3]) {
       const int K = counts[0], ng = counts[1], nd = counts[2];
       const float rho2 = 2.f * s_rho;
+      // squared weights of the kept poles and their sum (the last root's bracket)
+      if (tid < D) kz2[tid] = tid < K ? kz[tid] * kz[tid] : 0.f;
+      if (tid < 32) {
+        float z2 = 0.f;
+        for (int j = lane; j < K; j += 32) z2 = fmaf(kz[j], kz[j], z2);
+        for (int o = 16; o > 0; o >>= 1) z2 += __shfl_xor_sync(0xffffffffu, z2, o);
+        if (tid == 0) s_z2sum = z2;
+      }
+      __syncthreads();
       // rotations of the deflation on the rows of Qt (one column per thread, in the order recorded)
       if (tid < D) {
         for (int g = 0; g < ng; ++g) {
@@ -606,10 +629,32 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
       const bool live = gi < K;
       {
         const int i = live ? gi : 0;
-        auto fval = [&](int org, float m) {
+        // this thread's poles j = sub + 8 t and their squared weights stay in registers for all the
+        // halvings (past the last pole: weight 0 at a far distance); two terms share one reciprocal:
+        // a / p + b / q = (a q + b p) / (p q)
+        constexpr int TPR = D / 8;
+        float pole[TPR], wgt[TPR];
+#pragma unroll
+        for (int t = 0; t < TPR; ++t) {
+          const int j = sub + 8 * t;
+          pole[t] = j < K ? kd[j] : 0.f;
+          wgt[t] = j < K ? kz2[j] : 0.f;
+        }
+        float dist[TPR];                                   // d_j - d_org
+        auto set_origin = [&](int org) {
           const float d0 = kd[org];
+#pragma unroll
+          for (int t = 0; t < TPR; ++t) dist[t] = (sub + 8 * t < K) ? pole[t] - d0 : 1e18f;
+        };
+        auto fval = [&](float m) {
           float acc = 0.f;
-          for (int j = sub; j < K; j += 8) acc += __fdividef(kz2[j], (kd[j] - d0) - m);
+#pragma unroll
+          for (int t = 0; t < TPR; t += 2) {
+            const float p0 = dist[t] - m, p1 = dist[t + 1] - m;
+            float inv;                                      // one special-function operation, no rounding fix-up
+            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(p0 * p1));
+            acc = fmaf(fmaf(wgt[t], p1, wgt[t + 1] * p0), inv, acc);
+          }
           acc += __shfl_xor_sync(0xffffffffu, acc, 1);
           acc += __shfl_xor_sync(0xffffffffu, acc, 2);
           acc += __shfl_xor_sync(0xffffffffu, acc, 4);
@@ -620,17 +665,19 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         const bool last = i >= K - 1;
         const float width = last ? rho2 * s_z2sum : kd[i + 1] - kd[i];
         const float mid = 0.5f * width;
-        const float f_mid = fval(i, mid);                  // every thread of the warp takes part
+        set_origin(i);
+        const float f_mid = fval(mid);                     // every thread of the warp takes part
         float lo_m = 0.f, hi_m = width;
         if (!last) {
           if (f_mid >= 0.f) hi_m = mid;                    // root in the left half: offset from pole i
           else { org = i + 1; lo_m = -mid; hi_m = 0.f; }   // offset from pole i + 1
         }
+        set_origin(org);
         for (int it = 0; it < 44; ++it) {                  // a fixed count: the groups of a warp stay in step
           // (44 halvings take an interval of width w down to the float spacing of offsets >= 2^-20 w;
           // a root closer to its pole than that belongs to a weight that the deflation has removed)
           const float m = 0.5f * (lo_m + hi_m);
-          const float fm = fval(org, m);
+          const float fm = fval(m);
           if (m != lo_m && m != hi_m) {
             if (fm > 0.f) hi_m = m; else lo_m = m;
           }
@@ -747,12 +794,14 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   if (tid < D) {
     const double mine = lam[tid];
     int rank = 0;
+#pragma unroll 16
     for (int k = 0; k < D; ++k) {
       const double other = lam[k];
       rank += (other > mine) || (other == mine && k < tid);
     }
     // sign rule on column tid of F E (of E when no factor is given); bias = -mean . (output column)
     float best = -1.f, sgn = 1.f, dot = 0.f;
+#pragma unroll 8
     for (int i = 0; i < D; ++i) {
       const float e_i = Qt[tid * LDA + i];
       const float w_i = a.lift ? A[i * LDA + tid] : e_i;
