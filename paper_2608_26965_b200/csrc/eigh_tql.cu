@@ -106,9 +106,12 @@ __device__ __forceinline__ void ql_producer(float2* de, int l0, int l1, float* r
       if (lane == 0) {
         float2* rt = reinterpret_cast<float2*>(rot + bsel * rot_stride);
         const float2 top = de[l];
-        float g = (de[l + 1].x - top.x) / (2.f * top.y);
-        float rr = sqrtf(fmaf(g, g, 1.f));
-        g = de[m].x - top.x + top.y / (g + (g >= 0.f ? rr : -rr));
+        // the shift only steers the convergence (the rotations are formed from the matrix itself), so
+        // approximate division and root are enough for it
+        float g = __fdividef(de[l + 1].x - top.x, 2.f * top.y);
+        float rr;
+        asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rr) : "f"(fmaf(g, g, 1.f)));
+        g = de[m].x - top.x + __fdividef(top.y, g + (g >= 0.f ? rr : -rr));
         float s = 1.f, c = 1.f, p = 0.f;
         bool under = false;
         int i = m - 1;
