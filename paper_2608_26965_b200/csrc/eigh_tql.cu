@@ -451,10 +451,14 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         float bn = 0.f, alpha = x0, v0 = 0.f;
         const bool reflect = rest > 1e-30f;       // already tridiagonal in this column otherwise
         if (reflect) {
-          const float rt = sqrtf(sig);
+          // approximate root and reciprocal (a unit in the last place or two): the reflector stays
+          // orthogonal to the same order as the float32 updates that apply it, and the two IEEE
+          // operations were on the critical path of every one of the d - 2 steps
+          float rt;
+          asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(rt) : "f"(sig));
           alpha = x0 >= 0.f ? -rt : rt;
           v0 = x0 - alpha;
-          bn = 1.f / (sig + fabsf(x0) * rt);
+          asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(bn) : "f"(sig + fabsf(x0) * rt));
         }
         float* vn = vbuf + (kn & 1) * D;
 #pragma unroll
@@ -694,7 +698,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         float prod = 1.f;
         for (int i = sub; i < K; i += 8) {
           const float num = (kd[korg[i]] - kd[j]) + kmu[i];
-          prod *= (i == j) ? num / rho2 : num / (kd[i] - kd[j]);
+          prod *= __fdividef(num, (i == j) ? rho2 : kd[i] - kd[j]);
         }
         prod *= __shfl_xor_sync(0xffffffffu, prod, 1);
         prod *= __shfl_xor_sync(0xffffffffu, prod, 2);
@@ -708,7 +712,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         const float d0 = kd[korg[i]], mu = kmu[i];
         float nrm = 0.f;
         for (int j = sub; j < K; j += 8) {
-          const float v = kzh[j] / ((kd[j] - d0) - mu);
+          const float v = __fdividef(kzh[j], (kd[j] - d0) - mu);
           nrm = fmaf(v, v, nrm);
         }
         nrm += __shfl_xor_sync(0xffffffffu, nrm, 1);
@@ -716,7 +720,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
         nrm += __shfl_xor_sync(0xffffffffu, nrm, 4);
         const float inv = rsqrtf(nrm);
         if (live)
-          for (int j = sub; j < K; j += 8) A[gi * LDA + j] = kzh[j] / ((kd[j] - d0) - mu) * inv;
+          for (int j = sub; j < K; j += 8) A[gi * LDA + j] = __fdividef(kzh[j], (kd[j] - d0) - mu) * inv;
       }
       __syncthreads();
       // rows of the merged basis into L: row i = sum_j A[i][j] Qt[keep_row[j]] (i < K), then the deflated rows
