@@ -27,23 +27,6 @@ namespace ca {
 // pivot, also a step ahead.  A dropped pivot (reciprocal 0) leaves the trailing block alone and
 // gives a zero column.
 // ---------------------------------------------------------------------------
-// 1 / x for a pivot: a float32 estimate refined by two Newton steps in the working precision (the
-// IEEE division is a long dependent sequence, and this one sits on every column's critical path)
-__device__ __forceinline__ double fast_recip(double x) {
-  if (!(x > 1e-30 && x < 1e30)) return 1.0 / x;          // outside float32's comfortable range: the plain division
-  float e;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"((float)x));
-  double y = (double)e;
-  y = y * fma(-x, y, 2.0);
-  y = y * fma(-x, y, 2.0);
-  return y;
-}
-__device__ __forceinline__ float fast_recip(float x) {
-  float e;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(x));
-  return e * fmaf(-x, e, 2.0f);
-}
-
 template <int D, typename T>
 __global__ void __launch_bounds__(8 * D) cholesky_factor_kernel(const double* __restrict__ gram,
                                                                 const double* __restrict__ sum, double n,
@@ -97,7 +80,7 @@ __global__ void __launch_bounds__(8 * D) cholesky_factor_kernel(const double* __
           a[t] -= f * col[k];
           if (k == j + 1) {                               // column j + 1 is complete: publish it
             colbuf[(j + 1) & 1][r] = a[t];
-            if (r == j + 1) s_ip[(j + 1) & 1] = a[t] > tol ? fast_recip(a[t]) : (T)0;
+            if (r == j + 1) s_ip[(j + 1) & 1] = a[t] > tol ? (T)1 / a[t] : (T)0;
           }
         }
       }

@@ -193,7 +193,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   extern __shared__ __align__(16) unsigned char smem_raw[];
   uint32_t* s_keys = reinterpret_cast<uint32_t*>(smem_raw);                  // [smem_rows]
   int32_t* s_rows = reinterpret_cast<int32_t*>(s_keys + prm.smem_rows);      // [smem_rows]
-  __shared__ int s_hist[256];
+  __shared__ int s_hist2[2][256];  // digit counts of this slice, two in rotation over the passes
   __shared__ int s_total[256];
   __shared__ float s_var[128];
   __shared__ float s_part[8 * 128];
@@ -201,6 +201,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   __shared__ int s_warp[2 * 32];
   __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank, 3: chunk total
   __shared__ int s_counts[2];      // this CTA's (less, equal) totals
+  int* const s_hist = s_hist2[1];  // scratch of the partition (the last pass counts in the other array)
 
   const int which = blockIdx.y / prm.problems;
   const int p = blockIdx.y % prm.problems;
@@ -295,15 +296,19 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
     }
   }
   }
+  for (int b = tid; b < 256; b += nt) s_hist2[1][b] = 0;      // the first pass (shift 24) counts here
   __syncthreads();
 
-  // ---- radix selection of the L-th smallest key of the whole set (8 bits per pass)
+  // ---- radix selection of the L-th smallest key of the whole set (8 bits per pass).  The slices'
+  // counts alternate between two arrays: a peer may still be adding up one pass's counts while
+  // this CTA counts the next pass, and an array is cleared only after the cluster barrier of the
+  // pass after the one that used it, when every peer has finished reading it.
   const int L = sd.c * ((s + sd.c) / (2 * sd.c));
   uint32_t prefix = 0, mask = 0;
   int remaining = L;                                // 1-based rank among the candidates
   for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int b = tid; b < 256; b += nt) s_hist[b] = 0;
-    __syncthreads();
+    int* const hist = s_hist2[(shift >> 3) & 1];
+    int* const hist_next = s_hist2[((shift >> 3) & 1) ^ 1];
     for (int i0 = 0; i0 < cs; i0 += nt) {
       const int i = i0 + tid;
       const bool ok = i < cs;
@@ -313,22 +318,23 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
       if (shift == 24) {
         // leading digit: few distinct values in a warp (sign and exponent bits), one atomic per value
         const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&s_hist[bin], __popc(peers));
+        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
       } else if (cand) {
-        atomicAdd(&s_hist[bin], 1);                 // lower digits are spread out: plain atomics
+        atomicAdd(&hist[bin], 1);                   // lower digits are spread out: plain atomics
       }
     }
     if (csize > 1) {
       cluster.sync();                                // every slice has counted
       for (int b = tid; b < 256; b += nt) {
         int sum = 0;
-        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(s_hist, r)[b];
+        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(hist, r)[b];
         s_total[b] = sum;
       }
     } else {
       __syncthreads();
-      for (int b = tid; b < 256; b += nt) s_total[b] = s_hist[b];
+      for (int b = tid; b < 256; b += nt) s_total[b] = hist[b];
     }
+    for (int b = tid; b < 256; b += nt) hist_next[b] = 0;
     __syncthreads();
     if (warp == 0) {
       int local[8]; int sum = 0;
@@ -349,11 +355,11 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
         before += local[j];
       }
     }
-    if (csize > 1) cluster.sync(); else __syncthreads();   // peers are done reading s_hist
+    __syncthreads();
     prefix |= (uint32_t)s_scalar[1] << shift;
     mask |= 255u << shift;
     remaining = s_scalar[2];
-    __syncthreads();
+    // (s_scalar is written again only after the next pass's barriers)
   }
   const uint32_t thr = prefix;
   const int eq_left = remaining;        // how many rows equal to the threshold go down
