@@ -521,25 +521,35 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
     }
     __syncthreads();
 
-    // ---- 2. keys; each position finds its subset by bisection of the start offsets
-    int my_seg[kTailRowsMax / kSplitThreads];
-#pragma unroll
-    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
-      const int i = tid + u * nt;
+    // ---- 2. keys.  A thread owns four consecutive positions for the rest of the level (their
+    // keys stay in registers); the first finds its subset by bisection of the start offsets, the
+    // others walk on from there.
+    constexpr int PT = kTailRowsMax / kSplitThreads;     // positions per thread
+    static_assert(PT == 4 && kSplitThreads == 1024, "the scan below stores four counts per thread and scans 32 warp totals");
+    int my_seg[PT];
+    uint32_t my_key[PT];
+    {
+      const int i0 = PT * tid;
       int g = 0;
-      if (i < s0) {
-        int hi = nseg;                                // slo[g] <= i < slo[g+1]
-        while (hi - g > 1) { const int mid = (g + hi) >> 1; if (slo[mid] <= i) g = mid; else hi = mid; }
-        const bool splits = slo[g + 1] - slo[g] > c;
-        if (splits) sm.keys[i] = order_key(Yt ? __ldg(Yt + (size_t)sm.seg_coord[g] * sd.n + rows[i])
-                                              : __ldg(Y + (size_t)rows[i] * D + sm.seg_coord[g]));
-        else g = -1 - g;                              // final subset: carried over unchanged
-      } else {
-        g = INT_MIN;
+      if (i0 < s0) {
+        int hi = nseg;                                  // slo[g] <= i0 < slo[g+1]
+        while (hi - g > 1) { const int mid = (g + hi) >> 1; if (slo[mid] <= i0) g = mid; else hi = mid; }
       }
-      my_seg[u] = g;
+#pragma unroll
+      for (int u = 0; u < PT; ++u) {
+        const int i = i0 + u;
+        my_key[u] = 0u;
+        if (i < s0) {
+          while (slo[g + 1] <= i) ++g;
+          const bool splits = slo[g + 1] - slo[g] > c;
+          if (splits) my_key[u] = order_key(Yt ? __ldg(Yt + (size_t)sm.seg_coord[g] * sd.n + rows[i])
+                                               : __ldg(Y + (size_t)rows[i] * D + sm.seg_coord[g]));
+          my_seg[u] = splits ? g : -1 - g;              // final subset: carried over unchanged
+        } else {
+          my_seg[u] = INT_MIN;
+        }
+      }
     }
-    __syncthreads();
 
     // ---- radix selection, all subsets side by side
     uint32_t mask = 0;
@@ -547,10 +557,10 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
       for (int e = tid; e < nseg * 256; e += nt) (&sm.hist[0][0])[e] = 0;
       __syncthreads();
 #pragma unroll
-      for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
+      for (int u = 0; u < PT; ++u) {
         const int g = my_seg[u];
         const bool live = g >= 0;
-        const uint32_t k = live ? sm.keys[tid + u * nt] : 0u;
+        const uint32_t k = my_key[u];
         const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
         const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
         if (shift == 24) {
@@ -588,45 +598,53 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
       __syncthreads();
     }
 
-    // ---- 3. stable partition of every subset: one scan over all positions
-    int carry = 0;
+    // ---- 3. stable partition of every subset: one scan of (less | equal << 16) over all positions
+    // (a thread's four, then the warp, then the warps' totals by warp 0)
+    uint32_t my_scan[PT];
+    {
+      int run = 0;
 #pragma unroll
-    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
-      const int i = tid + u * nt;
-      const int g = my_seg[u];
-      int packed = 0;
-      if (g >= 0) {
-        const uint32_t k = sm.keys[i], thr = sm.seg_prefix[g];
-        packed = (k < thr ? 1 : 0) | (k == thr ? 1 << 16 : 0);
+      for (int u = 0; u < PT; ++u) {
+        if (my_seg[u] >= 0) {
+          const uint32_t k = my_key[u], thr = sm.seg_prefix[my_seg[u]];
+          run += (k < thr ? 1 : 0) | (k == thr ? 1 << 16 : 0);
+        }
+        my_scan[u] = (uint32_t)run;
       }
-      int incl = packed;
+      int incl = run;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += v;
       }
       if (lane == 31) sm.warp_tot[warp] = incl;
       __syncthreads();
-      int wbase = 0, total = 0;
-      for (int w = 0; w < nt / 32; ++w) {              // 32 broadcast reads
-        const int v = sm.warp_tot[w];
-        if (w < warp) wbase += v;
-        total += v;
+      if (warp == 0) {
+        const int v = sm.warp_tot[lane];                 // nt / 32 == 32 warps
+        int wi = v;
+        for (int o = 1; o < 32; o <<= 1) {
+          const int x = __shfl_up_sync(0xffffffffu, wi, o);
+          if (lane >= o) wi += x;
+        }
+        sm.warp_tot[lane] = wi - v;                      // totals of the warps before this one
       }
-      if (i < kTailRowsMax) sm.scan[i] = (uint32_t)(carry + wbase + incl);
-      carry += total;
+      __syncthreads();
+      const uint32_t before = (uint32_t)(sm.warp_tot[warp] + incl - run);
+#pragma unroll
+      for (int u = 0; u < PT; ++u) my_scan[u] += before;
+      *reinterpret_cast<uint4*>(&sm.scan[PT * tid]) = make_uint4(my_scan[0], my_scan[1], my_scan[2], my_scan[3]);
       __syncthreads();
     }
 #pragma unroll
-    for (int u = 0; u < kTailRowsMax / kSplitThreads; ++u) {
-      const int i = tid + u * nt;
+    for (int u = 0; u < PT; ++u) {
+      const int i = PT * tid + u;
       const int g = my_seg[u];
       if (g == INT_MIN) continue;
       if (g < 0) { rows_next[i] = rows[i]; continue; }
       const int a = slo[g];
       const uint32_t base = a > 0 ? sm.scan[a - 1] : 0u;
-      const uint32_t k = sm.keys[i], thr = sm.seg_prefix[g];
+      const uint32_t k = my_key[u], thr = sm.seg_prefix[g];
       const int is_less = k < thr, is_eq = k == thr;
-      const uint32_t excl = sm.scan[i] - base - (uint32_t)(is_less | (is_eq << 16));
+      const uint32_t excl = my_scan[u] - base - (uint32_t)(is_less | (is_eq << 16));
       const int less_here = (int)(excl & 0xffffu), eq_here = (int)(excl >> 16);
       const int eq_left = sm.seg_rem[g], L = sm.seg_L[g];
       const bool down = is_less || (is_eq && eq_here < eq_left);
