@@ -443,29 +443,31 @@ static bool map_2d(CUtensorMap* map, const void* base, size_t rows, int D, int b
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Chunks of rows per problem, one CTA each, one CTA per SM: the count that fills whole rounds of
-// the SMs best (a last round that is nearly empty costs a full round's time: 320 CTAs on 148 SMs
-// run as long as 444), among counts of up to about three rounds and chunks of at least four tiles;
-// of equally good counts the smallest (fewer partial sums to write and add up).
-int gram_tc_chunking(int n_rows, int problems, int* chunk_rows, int* n_chunks) {
+// Chunks of rows per problem, one CTA each, `ctas_per_sm` of them resident per SM: the count that
+// minimises rounds x (tiles per chunk + 3), the time of the launch in tiles when every CTA pays
+// about three tiles' worth of start-up and epilogue and a last round that is nearly empty costs a
+// full round (320 CTAs on 148 slots run as long as 444); chunks of at least four tiles.
+int gram_tc_chunking(int n_rows, int problems, int ctas_per_sm, int* chunk_rows, int* n_chunks) {
   int sms = 148, dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||
       cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
     (void)cudaGetLastError();
     sms = 148;
   }
+  const long long slots = (long long)sms * (ctas_per_sm > 0 ? ctas_per_sm : 1);
   const int tiles = ceil_div(n_rows, kRows);
   int best_c = 1, best_cr = tiles * kRows;
-  double best_eff = -1.0;
+  long long best_cost = -1;
   for (int c = 1; c <= tiles; ++c) {
-    const int cr = ceil_div(tiles, c) * kRows;             // rows per chunk, whole tiles
-    if (c > 1 && cr < 4 * kRows) break;
+    const int ct = ceil_div(tiles, c);                     // tiles per chunk
+    if (c > 1 && ct < 4) break;
+    const int cr = ct * kRows;
     const int chunks = ceil_div(n_rows, cr);
     const long long total = (long long)chunks * problems;
-    if (total > 3LL * sms + sms / 2 && best_eff >= 0.0) break;
-    const long long rounds = (total + sms - 1) / sms;
-    const double eff = (double)total / (double)(rounds * sms);
-    if (eff > best_eff + 1e-9) { best_eff = eff; best_c = chunks; best_cr = cr; }
+    const long long rounds = (total + slots - 1) / slots;
+    const long long cost = rounds * (ct + 3);
+    if (best_cost < 0 || cost < best_cost) { best_cost = cost; best_c = chunks; best_cr = cr; }
+    if (rounds > 8) break;
   }
   // the buffer of partial sums is sized for the chunk count of the CUDA-core moments kernel
   int m_cr, m_chunks;
@@ -482,7 +484,6 @@ int gram_tc_chunking(int n_rows, int problems, int* chunk_rows, int* n_chunks) {
 int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows, int D, float* partial,
                    double* gram, double* colsum, int* status, cudaStream_t st) {
   GramParams prm;
-  gram_tc_chunking(n_rows, problems, &prm.chunk_rows, &prm.n_chunks);
   prm.partial = partial; prm.status = status; prm.n_rows = n_rows; prm.has_lo = X_lo ? 1 : 0;
   const int tile = kRows * D * 2 * (X_lo ? 2 : 1);
   prm.stages = (200 * 1024 - 4096) / tile;
@@ -491,6 +492,13 @@ int launch_gram_tc(const void* X_hi, const void* X_lo, int problems, int n_rows,
   // start-up and epilogue overlap the other's streaming (video480: 0.36 -> 0.34 ms for the step's
   // three launches)
   if (!X_lo && prm.stages > 3) prm.stages = 3;
+  {
+    const size_t smem_cta = 1024 + (size_t)prm.stages * tile + 2048 + 8 * (2 * prm.stages + 1) + 64 + 1024;
+    int per_sm = (int)((227 * 1024) / smem_cta);
+    const int by_tmem = 512 / ((D + 16 <= 128) ? 128 : 256);
+    if (per_sm > by_tmem) per_sm = by_tmem;
+    gram_tc_chunking(n_rows, problems, per_sm, &prm.chunk_rows, &prm.n_chunks);
+  }
   CUtensorMap mh, ml;
   if (!map_3d(&mh, X_hi, problems, n_rows, D, 2, 64, kRows)) return CA_ERR_CUDA;
   if (!map_3d(&ml, X_lo ? X_lo : X_hi, problems, n_rows, D, 2, 64, kRows)) return CA_ERR_CUDA;
