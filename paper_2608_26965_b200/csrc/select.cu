@@ -216,8 +216,10 @@ score_tile_kernel(const float* __restrict__ cq, const float* __restrict__ ck, in
   const int tid = threadIdx.x;
   const float* cqp = cq + (size_t)p * n_qc * D;
   const float* ckp = ck + (size_t)p * n_kc * D;
+  // lanes take consecutive rows of one 16-byte column group: the transposing stores below then fall
+  // in consecutive banks (with consecutive column groups per lane they all hit one bank)
   for (int e = tid; e < 64 * (D / 4); e += 256) {
-    const int r = e / (D / 4), k4 = e % (D / 4);
+    const int r = e % 64, k4 = e / 64;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
     if (i0 + r < row_end) a = __ldg(reinterpret_cast<const float4*>(cqp + (size_t)(i0 + r) * D) + k4);
     if (j0 + r < n_kc) b = __ldg(reinterpret_cast<const float4*>(ckp + (size_t)(j0 + r) * D) + k4);
