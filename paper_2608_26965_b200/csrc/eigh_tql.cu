@@ -21,19 +21,21 @@
 // next reflector right after their update, inside their warp, so no third
 // barrier is needed.  Phase 2, divide and conquer: the QL iteration is one
 // dependent chain of about 0.9 n^2 plane rotations for n rows, so the tridiagonal
-// matrix is cut in the middle (T = diag(T1, T2) + rho u u^T) and the two halves are
-// iterated side by side, a quarter of the chain each: per half one warp runs the
-// iteration on (diag, sub-diag) -- the search for a negligible sub-diagonal entry
-// uses all lanes, the rotation chase is one dependent chain on lane 0 -- and hands
-// each chase's rotations through a double-buffered list to consumer threads, which
-// apply them to the rows of Qt of that half (a thread per column), pipelined with
-// the next chase by named barriers.  An extra column that starts as u goes through
-// the same rotations and ends as z = Q^T u.  The merge solves diag(d) + rho z z^T:
-// poles sorted, negligible weights and coinciding poles deflated, the roots of the
-// secular equation by bisection on the offset from the nearer pole (eight threads
-// per root; offsets keep the differences d_j - x accurate), the weights recomputed
-// from the roots (Gu and Eisenstat) so that the eigenvectors stay orthogonal to
-// rounding, and one d x d x d product with the halves' eigenvectors.
+// matrix is cut three times (a cut writes T = diag(T1, T2) + rho u u^T) and the four
+// quarters are iterated side by side, a sixteenth of the chain each: per quarter
+// one warp runs the iteration on (diag, sub-diag) -- the search for a negligible
+// sub-diagonal entry uses all lanes, the rotation chase is one dependent chain on
+// lane 0 -- and hands each chase's rotations through a list (two in rotation) to
+// consumer threads, which apply them to the rows of Qt of that quarter (a thread
+// per column), pipelined with the next chase by two named barriers.  Two extra
+// columns that start as the u of the cuts go through the same rotations and end
+// as z = Q^T u.  A merge solves diag(d) + rho z z^T: poles sorted, negligible
+// weights and coinciding poles deflated, the roots of the secular equation by
+// bisection on the offset from the nearer pole (eight threads per root; offsets
+// keep the differences d_j - x accurate), the weights recomputed from the roots
+// (Gu and Eisenstat) so that the eigenvectors stay orthogonal to rounding, and one
+// product with the blocks' eigenvectors.  The quarters are merged into halves by
+// the two halves of the CTA side by side, then the halves into the whole.
 //
 // Epilogue.  Components in order of descending eigenvalue.  With E the
 // eigenvectors and F the factor that produced the transformed rows, the map from
@@ -50,42 +52,41 @@ namespace ca {
 
 namespace {
 
-// barrier ids are immediates so that the kernel reserves only the barriers it names
+// named barriers with the id as an immediate (ids 1-8: the four QL groups, 9-10: the two half merges;
+// barrier 0 stays the CTA's own: threads that finish early wait there while others still use theirs)
+#define CA_BAR_CASE(OP, ID) case ID: asm volatile(OP " " #ID ", %0;" ::"r"(count) : "memory"); break;
 __device__ __forceinline__ void named_sync(int id, int count) {
   switch (id) {
-    case 1: asm volatile("bar.sync 1, %0;" ::"r"(count) : "memory"); break;
-    case 2: asm volatile("bar.sync 2, %0;" ::"r"(count) : "memory"); break;
-    case 3: asm volatile("bar.sync 3, %0;" ::"r"(count) : "memory"); break;
-    case 4: asm volatile("bar.sync 4, %0;" ::"r"(count) : "memory"); break;
-    case 5: asm volatile("bar.sync 5, %0;" ::"r"(count) : "memory"); break;
-    case 6: asm volatile("bar.sync 6, %0;" ::"r"(count) : "memory"); break;
-    case 7: asm volatile("bar.sync 7, %0;" ::"r"(count) : "memory"); break;
-    default: asm volatile("bar.sync 8, %0;" ::"r"(count) : "memory"); break;
+    CA_BAR_CASE("bar.sync", 0) CA_BAR_CASE("bar.sync", 1) CA_BAR_CASE("bar.sync", 2) CA_BAR_CASE("bar.sync", 3)
+    CA_BAR_CASE("bar.sync", 4) CA_BAR_CASE("bar.sync", 5) CA_BAR_CASE("bar.sync", 6) CA_BAR_CASE("bar.sync", 7)
+    CA_BAR_CASE("bar.sync", 8) CA_BAR_CASE("bar.sync", 9) CA_BAR_CASE("bar.sync", 10) CA_BAR_CASE("bar.sync", 11)
+    CA_BAR_CASE("bar.sync", 12) CA_BAR_CASE("bar.sync", 13) CA_BAR_CASE("bar.sync", 14)
+    default: asm volatile("bar.sync 15, %0;" ::"r"(count) : "memory"); break;
   }
 }
 __device__ __forceinline__ void named_arrive(int id, int count) {
   switch (id) {
-    case 1: asm volatile("bar.arrive 1, %0;" ::"r"(count) : "memory"); break;
-    case 2: asm volatile("bar.arrive 2, %0;" ::"r"(count) : "memory"); break;
-    case 3: asm volatile("bar.arrive 3, %0;" ::"r"(count) : "memory"); break;
-    case 4: asm volatile("bar.arrive 4, %0;" ::"r"(count) : "memory"); break;
-    case 5: asm volatile("bar.arrive 5, %0;" ::"r"(count) : "memory"); break;
-    case 6: asm volatile("bar.arrive 6, %0;" ::"r"(count) : "memory"); break;
-    case 7: asm volatile("bar.arrive 7, %0;" ::"r"(count) : "memory"); break;
-    default: asm volatile("bar.arrive 8, %0;" ::"r"(count) : "memory"); break;
+    CA_BAR_CASE("bar.arrive", 0) CA_BAR_CASE("bar.arrive", 1) CA_BAR_CASE("bar.arrive", 2) CA_BAR_CASE("bar.arrive", 3)
+    CA_BAR_CASE("bar.arrive", 4) CA_BAR_CASE("bar.arrive", 5) CA_BAR_CASE("bar.arrive", 6) CA_BAR_CASE("bar.arrive", 7)
+    CA_BAR_CASE("bar.arrive", 8) CA_BAR_CASE("bar.arrive", 9) CA_BAR_CASE("bar.arrive", 10) CA_BAR_CASE("bar.arrive", 11)
+    CA_BAR_CASE("bar.arrive", 12) CA_BAR_CASE("bar.arrive", 13) CA_BAR_CASE("bar.arrive", 14)
+    default: asm volatile("bar.arrive 15, %0;" ::"r"(count) : "memory"); break;
   }
 }
+#undef CA_BAR_CASE
 
 constexpr int kMaxQlIterations = 64;
 
 // ---- implicit-shift QL on rows [l0, l1) of a tridiagonal matrix (de[i] = (diagonal i, coupling of
 // i and i + 1); the coupling at l1 - 1 is not part of the block).  One warp: the search for a
 // negligible sub-diagonal entry uses all lanes, the rotation chase is one dependent chain on lane 0.
-// Each chase's rotations go through a double-buffered list (rot, hdr) to the consumer threads, which
-// apply them to the rows of Qt; bar_full / bar_empty are the first of two named barriers each.
+// Each chase's rotations go through a list (rot, hdr; two in rotation, so that the next chase is
+// written while the last one is applied) to the consumer threads, which apply them to the rows of
+// Qt.  Two named barriers: bar_full hands a list over, bar_empty hands it back; a list is handed over
+// only after the one before it has come back, so each barrier has one generation in flight.
 __device__ __forceinline__ void ql_producer(float2* de, int l0, int l1, float* rot, int* hdr, int rot_stride,
                                             int bar_full, int bar_empty, int parties, int lane) {
-  int bsel = 0;
+  int bsel = 0, nlist = 0;
   const float eps = 6e-8f;
   for (int l = l0; l < l1; ++l) {
     for (int iter = 0; iter < kMaxQlIterations; ++iter) {
@@ -102,7 +103,6 @@ __device__ __forceinline__ void ql_producer(float2* de, int l0, int l1, float* r
         if (bal) { m = base + __ffs(bal) - 1; break; }
       }
       if (m == l) break;
-      named_sync(bar_empty + bsel, parties);             // the list's previous contents have been applied
       if (lane == 0) {
         float2* rt = reinterpret_cast<float2*>(rot + bsel * rot_stride);
         const float2 top = de[l];
@@ -157,26 +157,25 @@ __device__ __forceinline__ void ql_producer(float2* de, int l0, int l1, float* r
       }
       __syncwarp();
       __threadfence_block();
-      named_arrive(bar_full + bsel, parties);
+      if (nlist > 0) named_sync(bar_empty, parties);     // the list before this one has been applied
+      named_arrive(bar_full, parties);
+      ++nlist;
       bsel ^= 1;
     }
   }
-  named_sync(bar_empty + bsel, parties);
   if (lane == 0) hdr[bsel * 4 + 2] = 1;                    // end marker
   __syncwarp();
   __threadfence_block();
-  named_arrive(bar_full + bsel, parties);
-  named_sync(bar_empty + (bsel ^ 1), parties);             // the other list's last hand-back
+  if (nlist > 0) named_sync(bar_empty, parties);
+  named_arrive(bar_full, parties);
 }
 
 // consumer thread of column t (t >= ncols: only keeps the barriers going)
 __device__ __forceinline__ void ql_consumer(float* Qt, int lda, int t, int ncols, const float* rot, const int* hdr,
                                             int rot_stride, int bar_full, int bar_empty, int parties) {
-  named_arrive(bar_empty + 0, parties);                    // both lists start out free
-  named_arrive(bar_empty + 1, parties);
   int bsel = 0;
   while (true) {
-    named_sync(bar_full + bsel, parties);
+    named_sync(bar_full, parties);
     if (hdr[bsel * 4 + 2]) break;
     if (t < ncols) {
       const int hi = hdr[bsel * 4 + 0], lo = hdr[bsel * 4 + 1];
@@ -191,7 +190,7 @@ __device__ __forceinline__ void ql_consumer(float* Qt, int lda, int t, int ncols
       Qt[lo * lda + t] = carry;
     }
     __threadfence_block();
-    named_arrive(bar_empty + bsel, parties);
+    named_arrive(bar_empty, parties);
     bsel ^= 1;
   }
 }
@@ -261,6 +260,287 @@ __device__ __forceinline__ void tile_product_rows(const float* __restrict__ X, c
   }
 }
 
+// ---- merge of two adjacent blocks of the tridiagonal matrix whose eigen-decompositions are known
+// (rows [b0, b0 + NB) of Qt are their eigenvectors, de[].x their eigenvalues, column `zcol` of
+// those rows z = Q^T u): eigen-decomposition of diag(d) + rho2 z z^T with z scaled to unit length
+// (rho2 = 2 rho).  Sorted poles, deflation of negligible weights and of poles that coincide (a plane
+// rotation of their two eigenvectors), the roots of the secular equation
+// 1 + rho2 sum_j z_j^2 / (d_j - x) = 0 by bisection on the offset from the nearer pole (eight threads
+// per root), the weights recomputed from the roots so that the eigenvectors come out orthogonal
+// (Gu and Eisenstat), eigenvectors u_i[j] = zhat_j / (d_j - x_i), and the product with the blocks'
+// eigenvectors.  Run by a group of GT threads (lt = index in the group, `sync` its barrier); the new
+// rows go to rows [b0, b0 + NB) of L, with `carry` more columns after the D of the basis (the z of
+// an enclosing merge); every array of `scratch` is used at [b0, b0 + NB), so groups on disjoint
+// blocks run side by side.
+template <int D, int NB, int GT, typename Sync>
+__device__ __forceinline__ void merge_blocks(float* __restrict__ Qt, float* __restrict__ L, float* __restrict__ A,
+                                             float2* de, float* scratch, int b0, int zcol, int carry, float rho,
+                                             int lt, int grp, Sync sync) {
+  constexpr int LDA = D + 4;
+  static_assert(GT >= 8 * NB && GT >= D + 4 && (NB / 8) % 2 == 0, "eight threads per root, a thread per column");
+  const int lane = lt & 31;
+  float* ds = scratch + b0;                                // poles in ascending order
+  float* zs = ds + D;
+  int* ord = reinterpret_cast<int*>(zs + D);               // sorted position -> row of Qt
+  int* keep_row = ord + D;                                 // kept pole -> row of Qt
+  float* kd = reinterpret_cast<float*>(keep_row + D);      // kept poles, weights
+  float* kz = kd + D;
+  int* korg = reinterpret_cast<int*>(kz + D);              // root -> pole its offset is measured from
+  float* kmu = reinterpret_cast<float*>(korg + D);
+  float* kzh = kmu + D;
+  float* gc = kzh + D;                                     // plane rotations of the deflation
+  float* gs = gc + D;
+  int* ga = reinterpret_cast<int*>(gs + D);
+  int* gb = ga + D;
+  int* defl_row = gb + D;                                  // deflated: row of Qt, eigenvalue
+  float* defl_d = reinterpret_cast<float*>(defl_row + D);
+  float* kz2 = defl_d + D;                                 // squared weights of the kept poles
+  int* counts = reinterpret_cast<int*>(scratch + 16 * D) + 8 * grp;   // kept, rotations, deflated, skip
+  float* z2sum = reinterpret_cast<float*>(counts + 4);
+  const int W = D + carry;                                 // columns of a row that travel
+  if (lt < NB) {
+    const float mine = de[b0 + lt].x;
+    int rank = 0;
+#pragma unroll 16
+    for (int k = 0; k < NB; ++k) {
+      const float other = de[b0 + k].x;
+      rank += (other < mine) || (other == mine && k < lt);
+    }
+    ord[rank] = b0 + lt;
+  }
+  sync();
+  if (lt < NB) {
+    ds[lt] = de[ord[lt]].x;
+    zs[lt] = Qt[ord[lt] * LDA + zcol] * 0.70710678f;
+  }
+  sync();
+  if (lt < 32) {
+    const float rho2 = 2.f * rho;
+    float dmax = 0.f, zmax = 0.f;
+    for (int j = lane; j < NB; j += 32) { dmax = fmaxf(dmax, fabsf(ds[j])); zmax = fmaxf(zmax, fabsf(zs[j])); }
+    for (int o = 16; o > 0; o >>= 1) {
+      dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
+      zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
+    }
+    const float tol = 8.f * 6e-8f * fmaxf(dmax, zmax);
+    int K = 0, ng = 0, nd = 0;
+    if (lt != 0) {
+      // the scan below is one thread's
+    } else if (rho2 * zmax <= tol) {
+      counts[3] = 1;                                       // the blocks do not couple: nothing to merge
+    } else {
+      counts[3] = 0;
+      // one pass over the sorted poles; the last kept pole and the next pole travel in registers
+      // (every step would otherwise wait for the shared-memory round trip of the step before)
+      float d_prev = 0.f, z_prev = 0.f;
+      int o_prev = -1;
+      float dj = ds[0], zj = zs[0];
+      int oj = ord[0];
+      for (int j = 0; j < NB; ++j) {
+        const int jn = j + 1 < NB ? j + 1 : j;
+        const float dn = ds[jn], zn = zs[jn];
+        const int on = ord[jn];
+        if (rho2 * fabsf(zj) <= tol) {
+          defl_row[nd] = oj; defl_d[nd] = dj; ++nd;
+        } else {
+          // two poles coincide when |t c s| <= tol, c = z_j / tau, s = -z_prev / tau, tau^2 = z_j^2 + z_prev^2;
+          // the test is made without the root and the divisions, which only a deflation needs
+          if (o_prev >= 0 && fabsf((dj - d_prev) * zj * z_prev) <= tol * fmaf(zj, zj, z_prev * z_prev)) {
+            float sn = z_prev, cs = zj;
+            const float tau = sqrtf(fmaf(cs, cs, sn * sn));
+            cs = cs / tau;
+            sn = -sn / tau;
+            // rotate the weight into pole j; the other of the two is deflated
+            gc[ng] = cs; gs[ng] = sn; ga[ng] = o_prev; gb[ng] = oj; ++ng;
+            const float tt = d_prev * cs * cs + dj * sn * sn;
+            dj = d_prev * sn * sn + dj * cs * cs;
+            zj = tau;
+            --K;                                           // the last kept pole gives way
+            defl_row[nd] = o_prev; defl_d[nd] = tt; ++nd;
+          }
+          keep_row[K] = oj; kd[K] = dj; kz[K] = zj; ++K;
+          d_prev = dj; z_prev = zj; o_prev = oj;
+        }
+        dj = dn; zj = zn; oj = on;
+      }
+    }
+    if (lt == 0) { counts[0] = K; counts[1] = ng; counts[2] = nd; }
+  }
+  sync();
+  if (counts[3]) {
+    // nothing to merge: the rows move as they are, so that every block ends in L
+    for (int e = lt; e < NB * W; e += GT) L[(b0 + e / W) * LDA + e % W] = Qt[(b0 + e / W) * LDA + e % W];
+    sync();
+    return;
+  }
+  const int K = counts[0], ng = counts[1], nd = counts[2];
+  const float rho2 = 2.f * rho;
+  // squared weights of the kept poles and their sum (the last root's bracket)
+  if (lt < NB) kz2[lt] = lt < K ? kz[lt] * kz[lt] : 0.f;
+  if (lt < 32) {
+    float z2 = 0.f;
+    for (int j = lane; j < K; j += 32) z2 = fmaf(kz[j], kz[j], z2);
+    for (int o = 16; o > 0; o >>= 1) z2 += __shfl_xor_sync(0xffffffffu, z2, o);
+    if (lt == 0) *z2sum = z2;
+  }
+  sync();
+  // rotations of the deflation on the rows of Qt (one column per thread, in the order recorded)
+  if (lt < W) {
+    for (int g = 0; g < ng; ++g) {
+      const float x = Qt[ga[g] * LDA + lt], y = Qt[gb[g] * LDA + lt];
+      Qt[ga[g] * LDA + lt] = gc[g] * x + gs[g] * y;
+      Qt[gb[g] * LDA + lt] = gc[g] * y - gs[g] * x;
+    }
+  }
+  // roots: group i = lt / 8 of eight threads, each with the poles j = sub (mod 8)
+  const int gi = lt >> 3, sub = lt & 7;
+  const bool live = gi < K;
+  {
+    const int i = live ? gi : 0;
+    // this thread's poles j = sub + 8 t and their squared weights stay in registers for all the
+    // halvings (past the last pole: weight 0 at a far distance); two terms share one reciprocal:
+    // a / p + b / q = (a q + b p) / (p q)
+    constexpr int TPR = NB / 8;
+    float pole[TPR], wgt[TPR];
+#pragma unroll
+    for (int t = 0; t < TPR; ++t) {
+      const int j = sub + 8 * t;
+      pole[t] = j < K ? kd[j] : 0.f;
+      wgt[t] = j < K ? kz2[j] : 0.f;
+    }
+    float dist[TPR];                                       // d_j - d_org
+    auto set_origin = [&](int org) {
+      const float d0 = kd[org];
+#pragma unroll
+      for (int t = 0; t < TPR; ++t) dist[t] = (sub + 8 * t < K) ? pole[t] - d0 : 1e18f;
+    };
+    auto fval = [&](float m) {
+      float acc = 0.f;
+#pragma unroll
+      for (int t = 0; t < TPR; t += 2) {
+        const float p0 = dist[t] - m, p1 = dist[t + 1] - m;
+        float inv;                                          // one special-function operation, no rounding fix-up
+        asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(p0 * p1));
+        acc = fmaf(fmaf(wgt[t], p1, wgt[t + 1] * p0), inv, acc);
+      }
+      acc += __shfl_xor_sync(0xffffffffu, acc, 1);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 2);
+      acc += __shfl_xor_sync(0xffffffffu, acc, 4);
+      return fmaf(rho2, acc, 1.f);
+    };
+    // the last root lies in (d_{K-1}, d_{K-1} + rho2 |z|^2); every other one between two poles
+    int org = i;
+    const bool last = i >= K - 1;
+    const float width = last ? rho2 * *z2sum : kd[i + 1] - kd[i];
+    const float mid = 0.5f * width;
+    set_origin(i);
+    const float f_mid = fval(mid);                         // every thread of the warp takes part
+    float lo_m = 0.f, hi_m = width;
+    if (!last) {
+      if (f_mid >= 0.f) hi_m = mid;                        // root in the left half: offset from pole i
+      else { org = i + 1; lo_m = -mid; hi_m = 0.f; }       // offset from pole i + 1
+    }
+    set_origin(org);
+    for (int it = 0; it < 44; ++it) {                      // a fixed count: the groups of a warp stay in step
+      // (44 halvings take an interval of width w down to the float spacing of offsets >= 2^-20 w;
+      // a root closer to its pole than that belongs to a weight that the deflation has removed)
+      const float m = 0.5f * (lo_m + hi_m);
+      const float fm = fval(m);
+      if (m != lo_m && m != hi_m) {
+        if (fm > 0.f) hi_m = m; else lo_m = m;
+      }
+    }
+    if (live && sub == 0) { korg[gi] = org; kmu[gi] = 0.5f * (lo_m + hi_m); }
+  }
+  sync();
+  // weights recomputed from the roots: zhat_j^2 = prod_i (x_i - d_j) / (rho2 prod_{i != j} (d_i - d_j))
+  {
+    const int j = live ? gi : 0;
+    float prod = 1.f;
+    for (int i = sub; i < K; i += 8) {
+      const float num = (kd[korg[i]] - kd[j]) + kmu[i];
+      prod *= __fdividef(num, (i == j) ? rho2 : kd[i] - kd[j]);
+    }
+    prod *= __shfl_xor_sync(0xffffffffu, prod, 1);
+    prod *= __shfl_xor_sync(0xffffffffu, prod, 2);
+    prod *= __shfl_xor_sync(0xffffffffu, prod, 4);
+    if (live && sub == 0) kzh[gi] = copysignf(sqrtf(fabsf(prod)), kz[gi]);
+  }
+  sync();
+  // eigenvector i over the kept poles, normalised, as row b0 + i of A
+  {
+    const int i = live ? gi : 0;
+    const float d0 = kd[korg[i]], mu = kmu[i];
+    float nrm = 0.f;
+    for (int j = sub; j < K; j += 8) {
+      const float v = __fdividef(kzh[j], (kd[j] - d0) - mu);
+      nrm = fmaf(v, v, nrm);
+    }
+    nrm += __shfl_xor_sync(0xffffffffu, nrm, 1);
+    nrm += __shfl_xor_sync(0xffffffffu, nrm, 2);
+    nrm += __shfl_xor_sync(0xffffffffu, nrm, 4);
+    const float inv = rsqrtf(nrm);
+    if (live)
+      for (int j = sub; j < K; j += 8) A[(b0 + gi) * LDA + j] = __fdividef(kzh[j], (kd[j] - d0) - mu) * inv;
+  }
+  sync();
+  // rows of the merged basis into L: row b0 + i = sum_j A[b0 + i][j] Qt[keep_row[j]] (i < K), then
+  // the deflated rows (a 4 x 4 tile per thread, terms in the order of j)
+  {
+    const int tile_i = lt / (D / 4), tile_j = lt % (D / 4);
+    if (lt < NB * D / 16 && 4 * tile_i < K) {
+      const int i0 = 4 * tile_i;
+      float acc[4][4];
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
+      int j = 0;
+      for (; j + 4 <= K; j += 4) {
+        float xa[4][4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const float4 v = *reinterpret_cast<const float4*>(&A[(b0 + i0 + x) * LDA + j]);
+          xa[x][0] = v.x; xa[x][1] = v.y; xa[x][2] = v.z; xa[x][3] = v.w;
+        }
+#pragma unroll
+        for (int kk = 0; kk < 4; ++kk) {
+          const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j + kk] * LDA + 4 * tile_j]);
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            acc[x][0] = fmaf(xa[x][kk], y.x, acc[x][0]); acc[x][1] = fmaf(xa[x][kk], y.y, acc[x][1]);
+            acc[x][2] = fmaf(xa[x][kk], y.z, acc[x][2]); acc[x][3] = fmaf(xa[x][kk], y.w, acc[x][3]);
+          }
+        }
+      }
+      for (; j < K; ++j) {
+        const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j] * LDA + 4 * tile_j]);
+#pragma unroll
+        for (int x = 0; x < 4; ++x) {
+          const float xv = A[(b0 + i0 + x) * LDA + j];
+          acc[x][0] = fmaf(xv, y.x, acc[x][0]); acc[x][1] = fmaf(xv, y.y, acc[x][1]);
+          acc[x][2] = fmaf(xv, y.z, acc[x][2]); acc[x][3] = fmaf(xv, y.w, acc[x][3]);
+        }
+      }
+#pragma unroll
+      for (int x = 0; x < 4; ++x)
+        if (i0 + x < K)
+          *reinterpret_cast<float4*>(&L[(b0 + i0 + x) * LDA + 4 * tile_j]) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
+    }
+  }
+  // the columns that travel with the rows (the z of the enclosing merge)
+  for (int e = lt; e < K * carry; e += GT) {
+    const int i = e / carry, col = D + e % carry;
+    float acc = 0.f;
+    for (int j = 0; j < K; ++j) acc = fmaf(A[(b0 + i) * LDA + j], Qt[keep_row[j] * LDA + col], acc);
+    L[(b0 + i) * LDA + col] = acc;
+  }
+  for (int e = lt; e < nd * W; e += GT) L[(b0 + K + e / W) * LDA + e % W] = Qt[defl_row[e / W] * LDA + e % W];
+  sync();
+  if (lt < NB) de[b0 + lt].x = lt < K ? kd[korg[lt]] + kmu[lt] : defl_d[lt - K];
+  sync();
+}
+
 template <int D>
 __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   constexpr int NT = 8 * D, LDA = D + 4;
@@ -274,9 +554,9 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
   float* ubuf = pbuf + D;                              // [D]
   float2* de = reinterpret_cast<float2*>(ubuf + D);    // [D]        (diagonal i, sub-diagonal coupling i and i+1)
   float* beta = ubuf + 3 * D;                          // [2] (+2)
-  float* rot = beta + 4;                               // [2][2][2D] per half: (c, s) of the rotation of rows (i, i+1) at 2i
-  int* hdr = reinterpret_cast<int*>(rot + 8 * D);      // [2][2][4]  highest i, lowest i, end marker
-  float* scratch = reinterpret_cast<float*>(hdr + 16); // [17 D]     arrays of the merge
+  float* rot = beta + 4;                               // [2][2D] (+4D) per buffer: (c, s) of the rotation of rows (i, i+1) at 2i
+  int* hdr = reinterpret_cast<int*>(rot + 8 * D);      // [4][2][4]  per quarter and buffer: highest i, lowest i, end marker
+  float* scratch = reinterpret_cast<float*>(hdr + 32); // [17 D]     arrays of the merge
   __shared__ double s_scale;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -488,289 +768,52 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
     for (int c = 0; c < 4; ++c) Qt[(4 * (q + 8 * t) + c) * LDA + r] = qreg[t][c];
   __syncthreads();
 
-  // ---- phase 2: divide and conquer.  T = diag(T1, T2) + rho u u^T with rho = |b|, b the coupling of
-  // rows KH-1 and KH, u = e_{KH-1} + sign(b) e_{KH}, and b subtracted from the two diagonal entries it
-  // touches.  The two halves are independent tridiagonal problems: each gets its own QL warp and its
-  // own consumer threads (rows of Qt of its half), side by side.  An extra column of Qt (index D, in
-  // the row padding) starts as u and goes through the same rotations: afterwards it holds z = Q^T u.
-  constexpr int KH = D / 2;
-  constexpr int kParties = D + 64;                         // a QL warp + D + 1 columns rounded up to warps
-  float* rot_top = rot;
-  float* rot_bot = rot + 4 * D;
-  int* hdr_top = hdr;
-  int* hdr_bot = hdr + 8;
-  __shared__ float s_rho, s_theta, s_z2sum;
+  // ---- phase 2: divide and conquer.  A cut between rows k-1 and k writes T = diag(T1, T2) + rho u u^T
+  // with rho = |b|, b the coupling of the two rows, u = e_{k-1} + sign(b) e_k, and b subtracted from the
+  // two diagonal entries it touches.  Three cuts make four quarters, independent tridiagonal
+  // problems: each gets its own QL warp and its own consumer threads (the rows of Qt of its
+  // quarter), side by side -- a sixteenth of the rotation chain of the whole matrix each.  Two extra
+  // columns of Qt (in the row padding) start as the u of the middle cut (column D) and of the two
+  // outer cuts (column D + 1, disjoint rows) and go through the same rotations: afterwards they hold
+  // z = Q^T u.  The quarters are merged pairwise into halves by the two halves of the CTA side by
+  // side (column D travels through that merge), then the halves into the whole.
+  constexpr int KH = D / 2, KQ = D / 4;
+  constexpr int kParties = D + 64;                         // a QL warp + D + 2 columns rounded up to warps
+  constexpr int kGroup = D + 32;                           // consumer threads of a quarter
+  __shared__ float s_rho[3], s_theta[3];                   // cuts at KQ, KH, 3 KQ
+  if (tid < 3) {
+    const int k = (tid + 1) * KQ;
+    const float bk = de[k - 1].y;
+    s_rho[tid] = fabsf(bk);
+    s_theta[tid] = bk < 0.f ? -1.f : 1.f;
+    de[k - 1] = make_float2(de[k - 1].x - fabsf(bk), 0.f);
+    de[k].x -= fabsf(bk);
+  }
+  for (int i = tid; i < D; i += NT) { Qt[i * LDA + D] = 0.f; Qt[i * LDA + D + 1] = 0.f; }
+  __syncthreads();
   if (tid == 0) {
-    const float bk = de[KH - 1].y;
-    s_rho = fabsf(bk);
-    s_theta = bk < 0.f ? -1.f : 1.f;
-    de[KH - 1] = make_float2(de[KH - 1].x - fabsf(bk), 0.f);
-    de[KH].x -= fabsf(bk);
+    Qt[(KH - 1) * LDA + D] = 1.f;          Qt[KH * LDA + D] = s_theta[1];
+    Qt[(KQ - 1) * LDA + D + 1] = 1.f;      Qt[KQ * LDA + D + 1] = s_theta[0];
+    Qt[(3 * KQ - 1) * LDA + D + 1] = 1.f;  Qt[3 * KQ * LDA + D + 1] = s_theta[2];
   }
-  for (int i = tid; i < D; i += NT) Qt[i * LDA + D] = 0.f;
   __syncthreads();
-  if (tid == 0) { Qt[(KH - 1) * LDA + D] = 1.f; Qt[KH * LDA + D] = s_theta; }
+  // rotation lists: one array per buffer parity, indexed by the row, shared by the quarters
+  if (warp < 4) {
+    ql_producer(de, warp * KQ, (warp + 1) * KQ, rot, hdr + 8 * warp, 2 * D, 1 + 2 * warp, 2 + 2 * warp, kParties, lane);
+  } else if (tid < 128 + 4 * kGroup) {
+    const int g = (tid - 128) / kGroup;
+    ql_consumer(Qt, LDA, (tid - 128) % kGroup, D + 2, rot, hdr + 8 * g, 2 * D, 1 + 2 * g, 2 + 2 * g, kParties);
+  }
   __syncthreads();
-  if (warp == 0) ql_producer(de, 0, KH, rot_top, hdr_top, 2 * D, 1, 3, kParties, lane);
-  else if (warp == 1) ql_producer(de, KH, D, rot_bot, hdr_bot, 2 * D, 5, 7, kParties, lane);
-  else if (tid < 64 + D + 32) ql_consumer(Qt, LDA, tid - 64, D + 1, rot_top, hdr_top, 2 * D, 1, 3, kParties);
-  else if (tid < 64 + 2 * (D + 32)) ql_consumer(Qt, LDA, tid - 64 - (D + 32), D + 1, rot_bot, hdr_bot, 2 * D, 5, 7, kParties);
-  __syncthreads();
-
-  // ---- merge: eigen-decomposition of diag(d) + rho2 z z^T, d the eigenvalues of the halves, z scaled
-  // to unit length (rho2 = 2 rho).  Sorted poles, deflation of negligible weights and of poles that
-  // coincide (a plane rotation of their two eigenvectors), the roots of the secular equation
-  // 1 + rho2 sum_j z_j^2 / (d_j - x) = 0 by bisection on the offset from the nearer pole (eight threads
-  // per root), the weights recomputed from the roots so that the eigenvectors come out orthogonal
-  // (Gu and Eisenstat), eigenvectors u_i[j] = zhat_j / (d_j - x_i), and the product with the halves'
-  // eigenvectors.
   {
-    float* ds = scratch;                                   // poles in ascending order
-    float* zs = ds + D;
-    int* ord = reinterpret_cast<int*>(zs + D);             // sorted position -> row of Qt
-    int* keep_row = ord + D;                               // kept pole -> row of Qt
-    float* kd = reinterpret_cast<float*>(keep_row + D);    // kept poles, weights
-    float* kz = kd + D;
-    int* korg = reinterpret_cast<int*>(kz + D);            // root -> pole its offset is measured from
-    float* kmu = reinterpret_cast<float*>(korg + D);
-    float* kzh = kmu + D;
-    float* gc = kzh + D;                                   // plane rotations of the deflation
-    float* gs = gc + D;
-    int* ga = reinterpret_cast<int*>(gs + D);
-    int* gb = ga + D;
-    int* defl_row = gb + D;                                // deflated: row of Qt, eigenvalue
-    float* defl_d = reinterpret_cast<float*>(defl_row + D);
-    float* kz2 = defl_d + D;                               // squared weights of the kept poles
-    int* counts = reinterpret_cast<int*>(kz2 + D);         // kept, rotations, deflated, skip
-    if (tid < D) {
-      const float mine = de[tid].x;
-      int rank = 0;
-#pragma unroll 16
-      for (int k = 0; k < D; ++k) {
-        const float other = de[k].x;
-        rank += (other < mine) || (other == mine && k < tid);
-      }
-      ord[rank] = tid;
-    }
-    __syncthreads();
-    if (tid < D) {
-      ds[tid] = de[ord[tid]].x;
-      zs[tid] = Qt[ord[tid] * LDA + D] * 0.70710678f;
-    }
-    __syncthreads();
-    if (tid < 32) {
-      const float rho2 = 2.f * s_rho;
-      float dmax = 0.f, zmax = 0.f;
-      for (int j = lane; j < D; j += 32) { dmax = fmaxf(dmax, fabsf(ds[j])); zmax = fmaxf(zmax, fabsf(zs[j])); }
-      for (int o = 16; o > 0; o >>= 1) {
-        dmax = fmaxf(dmax, __shfl_xor_sync(0xffffffffu, dmax, o));
-        zmax = fmaxf(zmax, __shfl_xor_sync(0xffffffffu, zmax, o));
-      }
-      const float tol = 8.f * 6e-8f * fmaxf(dmax, zmax);
-      int K = 0, ng = 0, nd = 0;
-      if (tid != 0) {
-        // the scan below is one thread's
-      } else if (rho2 * zmax <= tol) {
-        counts[3] = 1;                                     // the halves do not couple: nothing to merge
-      } else {
-        counts[3] = 0;
-        // one pass over the sorted poles; the last kept pole and the next pole travel in registers
-        // (every step would otherwise wait for the shared-memory round trip of the step before)
-        float d_prev = 0.f, z_prev = 0.f;
-        int o_prev = -1;
-        float dj = ds[0], zj = zs[0];
-        int oj = ord[0];
-        for (int j = 0; j < D; ++j) {
-          const int jn = j + 1 < D ? j + 1 : j;
-          const float dn = ds[jn], zn = zs[jn];
-          const int on = ord[jn];
-          if (rho2 * fabsf(zj) <= tol) {
-            defl_row[nd] = oj; defl_d[nd] = dj; ++nd;
-          } else {
-            // two poles coincide when |t c s| <= tol, c = z_j / tau, s = -z_prev / tau, tau^2 = z_j^2 + z_prev^2;
-            // the test is made without the root and the divisions, which only a deflation needs
-            if (o_prev >= 0 && fabsf((dj - d_prev) * zj * z_prev) <= tol * fmaf(zj, zj, z_prev * z_prev)) {
-              float sn = z_prev, cs = zj;
-              const float tau = sqrtf(fmaf(cs, cs, sn * sn));
-              cs = cs / tau;
-              sn = -sn / tau;
-              // rotate the weight into pole j; the other of the two is deflated
-              gc[ng] = cs; gs[ng] = sn; ga[ng] = o_prev; gb[ng] = oj; ++ng;
-              const float tt = d_prev * cs * cs + dj * sn * sn;
-              dj = d_prev * sn * sn + dj * cs * cs;
-              zj = tau;
-              --K;                                         // the last kept pole gives way
-              defl_row[nd] = o_prev; defl_d[nd] = tt; ++nd;
-            }
-            keep_row[K] = oj; kd[K] = dj; kz[K] = zj; ++K;
-            d_prev = dj; z_prev = zj; o_prev = oj;
-          }
-          dj = dn; zj = zn; oj = on;
-        }
-      }
-      if (tid == 0) { counts[0] = K; counts[1] = ng; counts[2] = nd; }
-    }
-    __syncthreads();
-    if (!counts[3]) {
-      const int K = counts[0], ng = counts[1], nd = counts[2];
-      const float rho2 = 2.f * s_rho;
-      // squared weights of the kept poles and their sum (the last root's bracket)
-      if (tid < D) kz2[tid] = tid < K ? kz[tid] * kz[tid] : 0.f;
-      if (tid < 32) {
-        float z2 = 0.f;
-        for (int j = lane; j < K; j += 32) z2 = fmaf(kz[j], kz[j], z2);
-        for (int o = 16; o > 0; o >>= 1) z2 += __shfl_xor_sync(0xffffffffu, z2, o);
-        if (tid == 0) s_z2sum = z2;
-      }
-      __syncthreads();
-      // rotations of the deflation on the rows of Qt (one column per thread, in the order recorded)
-      if (tid < D) {
-        for (int g = 0; g < ng; ++g) {
-          const float x = Qt[ga[g] * LDA + tid], y = Qt[gb[g] * LDA + tid];
-          Qt[ga[g] * LDA + tid] = gc[g] * x + gs[g] * y;
-          Qt[gb[g] * LDA + tid] = gc[g] * y - gs[g] * x;
-        }
-      }
-      // roots: group i = tid / 8 of eight threads, each with the poles j = sub (mod 8)
-      const int gi = tid >> 3, sub = tid & 7;
-      const bool live = gi < K;
-      {
-        const int i = live ? gi : 0;
-        // this thread's poles j = sub + 8 t and their squared weights stay in registers for all the
-        // halvings (past the last pole: weight 0 at a far distance); two terms share one reciprocal:
-        // a / p + b / q = (a q + b p) / (p q)
-        constexpr int TPR = D / 8;
-        float pole[TPR], wgt[TPR];
-#pragma unroll
-        for (int t = 0; t < TPR; ++t) {
-          const int j = sub + 8 * t;
-          pole[t] = j < K ? kd[j] : 0.f;
-          wgt[t] = j < K ? kz2[j] : 0.f;
-        }
-        float dist[TPR];                                   // d_j - d_org
-        auto set_origin = [&](int org) {
-          const float d0 = kd[org];
-#pragma unroll
-          for (int t = 0; t < TPR; ++t) dist[t] = (sub + 8 * t < K) ? pole[t] - d0 : 1e18f;
-        };
-        auto fval = [&](float m) {
-          float acc = 0.f;
-#pragma unroll
-          for (int t = 0; t < TPR; t += 2) {
-            const float p0 = dist[t] - m, p1 = dist[t + 1] - m;
-            float inv;                                      // one special-function operation, no rounding fix-up
-            asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(inv) : "f"(p0 * p1));
-            acc = fmaf(fmaf(wgt[t], p1, wgt[t + 1] * p0), inv, acc);
-          }
-          acc += __shfl_xor_sync(0xffffffffu, acc, 1);
-          acc += __shfl_xor_sync(0xffffffffu, acc, 2);
-          acc += __shfl_xor_sync(0xffffffffu, acc, 4);
-          return fmaf(rho2, acc, 1.f);
-        };
-        // the last root lies in (d_{K-1}, d_{K-1} + rho2 |z|^2); every other one between two poles
-        int org = i;
-        const bool last = i >= K - 1;
-        const float width = last ? rho2 * s_z2sum : kd[i + 1] - kd[i];
-        const float mid = 0.5f * width;
-        set_origin(i);
-        const float f_mid = fval(mid);                     // every thread of the warp takes part
-        float lo_m = 0.f, hi_m = width;
-        if (!last) {
-          if (f_mid >= 0.f) hi_m = mid;                    // root in the left half: offset from pole i
-          else { org = i + 1; lo_m = -mid; hi_m = 0.f; }   // offset from pole i + 1
-        }
-        set_origin(org);
-        for (int it = 0; it < 44; ++it) {                  // a fixed count: the groups of a warp stay in step
-          // (44 halvings take an interval of width w down to the float spacing of offsets >= 2^-20 w;
-          // a root closer to its pole than that belongs to a weight that the deflation has removed)
-          const float m = 0.5f * (lo_m + hi_m);
-          const float fm = fval(m);
-          if (m != lo_m && m != hi_m) {
-            if (fm > 0.f) hi_m = m; else lo_m = m;
-          }
-        }
-        if (live && sub == 0) { korg[gi] = org; kmu[gi] = 0.5f * (lo_m + hi_m); }
-      }
-      __syncthreads();
-      // weights recomputed from the roots: zhat_j^2 = prod_i (x_i - d_j) / (rho2 prod_{i != j} (d_i - d_j))
-      {
-        const int j = live ? gi : 0;
-        float prod = 1.f;
-        for (int i = sub; i < K; i += 8) {
-          const float num = (kd[korg[i]] - kd[j]) + kmu[i];
-          prod *= __fdividef(num, (i == j) ? rho2 : kd[i] - kd[j]);
-        }
-        prod *= __shfl_xor_sync(0xffffffffu, prod, 1);
-        prod *= __shfl_xor_sync(0xffffffffu, prod, 2);
-        prod *= __shfl_xor_sync(0xffffffffu, prod, 4);
-        if (live && sub == 0) kzh[gi] = copysignf(sqrtf(fabsf(prod)), kz[gi]);
-      }
-      __syncthreads();
-      // eigenvector i over the kept poles, normalised, as row i of A; its eigenvalue
-      {
-        const int i = live ? gi : 0;
-        const float d0 = kd[korg[i]], mu = kmu[i];
-        float nrm = 0.f;
-        for (int j = sub; j < K; j += 8) {
-          const float v = __fdividef(kzh[j], (kd[j] - d0) - mu);
-          nrm = fmaf(v, v, nrm);
-        }
-        nrm += __shfl_xor_sync(0xffffffffu, nrm, 1);
-        nrm += __shfl_xor_sync(0xffffffffu, nrm, 2);
-        nrm += __shfl_xor_sync(0xffffffffu, nrm, 4);
-        const float inv = rsqrtf(nrm);
-        if (live)
-          for (int j = sub; j < K; j += 8) A[gi * LDA + j] = __fdividef(kzh[j], (kd[j] - d0) - mu) * inv;
-      }
-      __syncthreads();
-      // rows of the merged basis into L: row i = sum_j A[i][j] Qt[keep_row[j]] (i < K), then the deflated rows
-      // (a 4 x 4 tile per thread, terms in the order of j)
-      if (tid < TILE_THREADS && 4 * tile_i < K) {
-        const int i0 = 4 * tile_i;
-        float acc[4][4];
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-#pragma unroll
-          for (int y = 0; y < 4; ++y) acc[x][y] = 0.f;
-        int j = 0;
-        for (; j + 4 <= K; j += 4) {
-          float xa[4][4];
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const float4 v = *reinterpret_cast<const float4*>(&A[(i0 + x) * LDA + j]);
-            xa[x][0] = v.x; xa[x][1] = v.y; xa[x][2] = v.z; xa[x][3] = v.w;
-          }
-#pragma unroll
-          for (int kk = 0; kk < 4; ++kk) {
-            const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j + kk] * LDA + 4 * tile_j]);
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              acc[x][0] = fmaf(xa[x][kk], y.x, acc[x][0]); acc[x][1] = fmaf(xa[x][kk], y.y, acc[x][1]);
-              acc[x][2] = fmaf(xa[x][kk], y.z, acc[x][2]); acc[x][3] = fmaf(xa[x][kk], y.w, acc[x][3]);
-            }
-          }
-        }
-        for (; j < K; ++j) {
-          const float4 y = *reinterpret_cast<const float4*>(&Qt[keep_row[j] * LDA + 4 * tile_j]);
-#pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const float xv = A[(i0 + x) * LDA + j];
-            acc[x][0] = fmaf(xv, y.x, acc[x][0]); acc[x][1] = fmaf(xv, y.y, acc[x][1]);
-            acc[x][2] = fmaf(xv, y.z, acc[x][2]); acc[x][3] = fmaf(xv, y.w, acc[x][3]);
-          }
-        }
-#pragma unroll
-        for (int x = 0; x < 4; ++x)
-          if (i0 + x < K)
-            *reinterpret_cast<float4*>(&L[(i0 + x) * LDA + 4 * tile_j]) = make_float4(acc[x][0], acc[x][1], acc[x][2], acc[x][3]);
-      }
-      for (int e = tid; e < nd * D; e += NT) L[(K + e / D) * LDA + e % D] = Qt[defl_row[e / D] * LDA + e % D];
-      __syncthreads();
-      if (tid < D) de[tid].x = tid < K ? kd[korg[tid]] + kmu[tid] : defl_d[tid - K];
-      float* swap = Qt; Qt = L; L = swap;
-    }
-    __syncthreads();
+    const int g2 = tid / (NT / 2);
+    merge_blocks<D, KH, NT / 2>(Qt, L, A, de, scratch, g2 * KH, D + 1, 1, s_rho[g2 ? 2 : 0], tid % (NT / 2), g2,
+                                [&]() { named_sync(9 + g2, NT / 2); });
   }
+  __syncthreads();
+  { float* swap = Qt; Qt = L; L = swap; }
+  merge_blocks<D, D, NT>(Qt, L, A, de, scratch, 0, D, 0, s_rho[1], tid, 0, [&]() { __syncthreads(); });
+  { float* swap = Qt; Qt = L; L = swap; }
   // the factor of the sign rule (its space served the prologue and the merge)
   if (a.lift) {
     const double* F = a.lift + mat;
@@ -839,7 +882,7 @@ __global__ void __launch_bounds__(8 * D) eigh_tql_kernel(const PcaArgs a) {
 }
 
 int launch_pca(const PcaArgs& args, int count, int D, cudaStream_t st) {
-  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 6 * D + 4 + 8 * D + 17 * D) + 16 * sizeof(int);
+  const size_t smem = sizeof(float) * ((size_t)3 * D * (D + 4) + 6 * D + 4 + 8 * D + 17 * D) + 32 * sizeof(int);
   if (D == 64) {
     auto k = eigh_tql_kernel<64>;
     CA_RETURN_IF_CUDA(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
