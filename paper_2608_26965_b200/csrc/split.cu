@@ -440,6 +440,121 @@ struct TailSmem {
   int more;
 };
 
+// Selection and partition of one level of a subtree, all of its subsets side by side: radix
+// selection of every subset's threshold key (seg_L, seg_rem, seg_prefix set up by the caller), then
+// the stable partition into rows_next.  A thread owns the four consecutive positions 4 tid .. 4 tid + 3
+// (my_seg: subset of a position, -1 - g in a final subset, INT_MIN past the end; my_key: its key).
+template <typename Smem>
+__device__ __forceinline__ void tail_select_partition(Smem& sm, const int (&my_seg)[kTailRowsMax / kSplitThreads],
+                                                      const uint32_t (&my_key)[kTailRowsMax / kSplitThreads],
+                                                      int nseg, const int* slo, const int32_t* rows,
+                                                      int32_t* rows_next, int tid, int* hist, uint32_t* scan) {
+  constexpr int nt = kSplitThreads;
+  constexpr int PT = kTailRowsMax / kSplitThreads;
+  const int lane = tid & 31, warp = tid >> 5;
+  // ---- radix selection, all subsets side by side
+  uint32_t mask = 0;
+  for (int shift = 24; shift >= 0; shift -= 8) {
+    for (int e = tid; e < nseg * 256; e += nt) hist[e] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int u = 0; u < PT; ++u) {
+      const int g = my_seg[u];
+      const bool live = g >= 0;
+      const uint32_t k = my_key[u];
+      const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
+      const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
+      if (shift == 24) {
+        const unsigned peers = __match_any_sync(0xffffffffu, bin);
+        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
+      } else if (cand) {
+        atomicAdd(&hist[bin], 1);
+      }
+    }
+    __syncthreads();
+    for (int g = warp; g < nseg; g += nt / 32) {
+      const int remaining = sm.seg_rem[g];
+      if (sm.seg_L[g] == 0) continue;               // warp-uniform
+      int local[8]; int sum = 0;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { local[j] = hist[g * 256 + lane * 8 + j]; sum += local[j]; }
+      int incl = sum;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+      }
+      int before = incl - sum;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        if (before < remaining && remaining <= before + local[j]) {
+          sm.seg_digit[g] = lane * 8 + j;
+          sm.seg_rem[g] = remaining - before;
+        }
+        before += local[j];
+      }
+      __syncwarp();
+      if (lane == 0) sm.seg_prefix[g] |= (uint32_t)sm.seg_digit[g] << shift;
+    }
+    mask |= 255u << shift;
+    __syncthreads();
+  }
+
+  // ---- 3. stable partition of every subset: one scan of (less | equal << 16) over all positions
+  // (a thread's four, then the warp, then the warps' totals by warp 0)
+  uint32_t my_scan[PT];
+  {
+    int run = 0;
+#pragma unroll
+    for (int u = 0; u < PT; ++u) {
+      if (my_seg[u] >= 0) {
+        const uint32_t k = my_key[u], thr = sm.seg_prefix[my_seg[u]];
+        run += (k < thr ? 1 : 0) | (k == thr ? 1 << 16 : 0);
+      }
+      my_scan[u] = (uint32_t)run;
+    }
+    int incl = run;
+    for (int o = 1; o < 32; o <<= 1) {
+      const int v = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += v;
+    }
+    if (lane == 31) sm.warp_tot[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+      const int v = sm.warp_tot[lane];                 // nt / 32 == 32 warps
+      int wi = v;
+      for (int o = 1; o < 32; o <<= 1) {
+        const int x = __shfl_up_sync(0xffffffffu, wi, o);
+        if (lane >= o) wi += x;
+      }
+      sm.warp_tot[lane] = wi - v;                      // totals of the warps before this one
+    }
+    __syncthreads();
+    const uint32_t before = (uint32_t)(sm.warp_tot[warp] + incl - run);
+#pragma unroll
+    for (int u = 0; u < PT; ++u) my_scan[u] += before;
+    *reinterpret_cast<uint4*>(&scan[PT * tid]) = make_uint4(my_scan[0], my_scan[1], my_scan[2], my_scan[3]);
+    __syncthreads();
+  }
+#pragma unroll
+  for (int u = 0; u < PT; ++u) {
+    const int i = PT * tid + u;
+    const int g = my_seg[u];
+    if (g == INT_MIN) continue;
+    if (g < 0) { rows_next[i] = rows[i]; continue; }
+    const int a = slo[g];
+    const uint32_t base = a > 0 ? scan[a - 1] : 0u;
+    const uint32_t k = my_key[u], thr = sm.seg_prefix[g];
+    const int is_less = k < thr, is_eq = k == thr;
+    const uint32_t excl = my_scan[u] - base - (uint32_t)(is_less | (is_eq << 16));
+    const int less_here = (int)(excl & 0xffffu), eq_here = (int)(excl >> 16);
+    const int eq_left = sm.seg_rem[g], L = sm.seg_L[g];
+    const bool down = is_less || (is_eq && eq_here < eq_left);
+    const int down_before = less_here + min(eq_here, eq_left);
+    const int dst = down ? a + down_before : a + L + (i - a - down_before);
+    rows_next[dst] = rows[i];
+  }
+}
+
 template <int D>
 __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitParams prm) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -551,107 +666,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
       }
     }
 
-    // ---- radix selection, all subsets side by side
-    uint32_t mask = 0;
-    for (int shift = 24; shift >= 0; shift -= 8) {
-      for (int e = tid; e < nseg * 256; e += nt) (&sm.hist[0][0])[e] = 0;
-      __syncthreads();
-#pragma unroll
-      for (int u = 0; u < PT; ++u) {
-        const int g = my_seg[u];
-        const bool live = g >= 0;
-        const uint32_t k = my_key[u];
-        const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
-        const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
-        if (shift == 24) {
-          const unsigned peers = __match_any_sync(0xffffffffu, bin);
-          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&(&sm.hist[0][0])[bin], __popc(peers));
-        } else if (cand) {
-          atomicAdd(&(&sm.hist[0][0])[bin], 1);
-        }
-      }
-      __syncthreads();
-      for (int g = warp; g < nseg; g += nt / 32) {
-        const int remaining = sm.seg_rem[g];
-        if (sm.seg_L[g] == 0) continue;               // warp-uniform
-        int local[8]; int sum = 0;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) { local[j] = sm.hist[g][lane * 8 + j]; sum += local[j]; }
-        int incl = sum;
-        for (int o = 1; o < 32; o <<= 1) {
-          const int v = __shfl_up_sync(0xffffffffu, incl, o);
-          if (lane >= o) incl += v;
-        }
-        int before = incl - sum;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          if (before < remaining && remaining <= before + local[j]) {
-            sm.seg_digit[g] = lane * 8 + j;
-            sm.seg_rem[g] = remaining - before;
-          }
-          before += local[j];
-        }
-        __syncwarp();
-        if (lane == 0) sm.seg_prefix[g] |= (uint32_t)sm.seg_digit[g] << shift;
-      }
-      mask |= 255u << shift;
-      __syncthreads();
-    }
-
-    // ---- 3. stable partition of every subset: one scan of (less | equal << 16) over all positions
-    // (a thread's four, then the warp, then the warps' totals by warp 0)
-    uint32_t my_scan[PT];
-    {
-      int run = 0;
-#pragma unroll
-      for (int u = 0; u < PT; ++u) {
-        if (my_seg[u] >= 0) {
-          const uint32_t k = my_key[u], thr = sm.seg_prefix[my_seg[u]];
-          run += (k < thr ? 1 : 0) | (k == thr ? 1 << 16 : 0);
-        }
-        my_scan[u] = (uint32_t)run;
-      }
-      int incl = run;
-      for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-      }
-      if (lane == 31) sm.warp_tot[warp] = incl;
-      __syncthreads();
-      if (warp == 0) {
-        const int v = sm.warp_tot[lane];                 // nt / 32 == 32 warps
-        int wi = v;
-        for (int o = 1; o < 32; o <<= 1) {
-          const int x = __shfl_up_sync(0xffffffffu, wi, o);
-          if (lane >= o) wi += x;
-        }
-        sm.warp_tot[lane] = wi - v;                      // totals of the warps before this one
-      }
-      __syncthreads();
-      const uint32_t before = (uint32_t)(sm.warp_tot[warp] + incl - run);
-#pragma unroll
-      for (int u = 0; u < PT; ++u) my_scan[u] += before;
-      *reinterpret_cast<uint4*>(&sm.scan[PT * tid]) = make_uint4(my_scan[0], my_scan[1], my_scan[2], my_scan[3]);
-      __syncthreads();
-    }
-#pragma unroll
-    for (int u = 0; u < PT; ++u) {
-      const int i = PT * tid + u;
-      const int g = my_seg[u];
-      if (g == INT_MIN) continue;
-      if (g < 0) { rows_next[i] = rows[i]; continue; }
-      const int a = slo[g];
-      const uint32_t base = a > 0 ? sm.scan[a - 1] : 0u;
-      const uint32_t k = my_key[u], thr = sm.seg_prefix[g];
-      const int is_less = k < thr, is_eq = k == thr;
-      const uint32_t excl = my_scan[u] - base - (uint32_t)(is_less | (is_eq << 16));
-      const int less_here = (int)(excl & 0xffffu), eq_here = (int)(excl >> 16);
-      const int eq_left = sm.seg_rem[g], L = sm.seg_L[g];
-      const bool down = is_less || (is_eq && eq_here < eq_left);
-      const int down_before = less_here + min(eq_here, eq_left);
-      const int dst = down ? a + down_before : a + L + (i - a - down_before);
-      rows_next[dst] = rows[i];
-    }
+    tail_select_partition(sm, my_seg, my_key, nseg, slo, rows, rows_next, tid, &sm.hist[0][0], sm.scan);
     // ---- next level's subsets
     if (tid == 0) {
       int* nlo = sm.seg_lo[cur ^ 1];
@@ -814,8 +829,16 @@ struct BasicParams {
 };
 
 __device__ __forceinline__ float seq_norm(const float* v, int d) {
+  // d is a multiple of 8; the squares are formed eight at a time and added in order
   float s = 0.f;
-  for (int j = 0; j < d; ++j) s = __fadd_rn(s, __fmul_rn(v[j], v[j]));
+#pragma unroll 1
+  for (int j0 = 0; j0 < d; j0 += 8) {
+    float sq[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) sq[j] = __fmul_rn(v[j0 + j], v[j0 + j]);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) s = __fadd_rn(s, sq[j]);
+  }
   return __fsqrt_rn(s);
 }
 
@@ -951,6 +974,294 @@ __global__ void __launch_bounds__(256) basic_keys_kernel(const BasicParams prm) 
   sd.keybuf[(size_t)p * sd.n + i] = order_key(t);
 }
 
+// ---------------------------------------------------------------------------
+// Subtree of the basic variant: a set of at most kTailRowsMax rows finished by one CTA, so that
+// the deepest levels are one launch instead of three per level.  Per level: the directions of all
+// subsets that still split (a team of D threads per subset; the operations of
+// basic_direction_kernel in the same order -- the sample rows are staged as stored and centred
+// where they are used, which yields the same float32 values), the projection of every row onto its
+// subset's direction (the sum of basic_keys_kernel), then the selection and partition of the
+// diagonalized subtree kernel.
+// ---------------------------------------------------------------------------
+// staged sample rows (later the scan and the digit counts): 16 subsets of 64 bf16 rows at d = 64, 4 at d = 128
+template <int D> struct BasicStage { static constexpr int BYTES = D == 64 ? 135168 : 133120; };
+
+template <int D>
+struct BasicTailSmem {
+  static constexpr int TEAMS = kSplitThreads / D;
+  int32_t rows[2][kTailRowsMax];
+  __align__(16) unsigned char stage[BasicStage<D>::BYTES];
+  float dirs[2][kTailSegs][D];            // directions of this level's subsets and of the level above
+  float mu[TEAMS][D], u[TEAMS][D], v[TEAMS][D], w[TEAMS][D], y[TEAMS][D], g[TEAMS][D];
+  int seg_lo[2][2 * kTailSegs + 2];
+  int seg_slot[2][2 * kTailSegs + 2];     // slot of a subset in the tree, at the level it stands on
+  int seg_par[2][2 * kTailSegs + 2];      // subset of the level above it came from
+  int seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
+  uint32_t seg_prefix[kTailSegs];
+  int split_list[kTailSegs];              // the subsets that still split
+  int warp_tot[32];
+  int nseg[2];
+  int nsplit;
+  int more;
+};
+
+template <typename T>
+__device__ __forceinline__ float stored_value(const T* p);
+template <>
+__device__ __forceinline__ float stored_value<float>(const float* p) { return *p; }
+template <>
+__device__ __forceinline__ float stored_value<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+template <typename T, int D>
+__global__ void __launch_bounds__(kSplitThreads) basic_tail_kernel(const BasicParams prm, const SplitParams sp) {
+  using Sm = BasicTailSmem<D>;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  Sm& sm = *reinterpret_cast<Sm*>(smem_raw);
+  constexpr int nt = kSplitThreads;
+  constexpr int LD = D + (sizeof(T) == 2 ? 2 : 1);      // row stride of the staged rows (elements): odd in 4-byte words
+  constexpr int NODE_BYTES = D * LD * (int)sizeof(T);
+  constexpr int ROUND = (BasicStage<D>::BYTES / NODE_BYTES) < Sm::TEAMS ? (BasicStage<D>::BYTES / NODE_BYTES) : Sm::TEAMS;
+  static_assert(ROUND >= 1, "a subset's sample must fit the staging area");
+  constexpr int PT = kTailRowsMax / kSplitThreads;
+  static_assert(PT == 4 && kTailRowsMax * 4 + kTailSegs * 256 * 4 <= BasicStage<D>::BYTES, "scan and digit counts live in the staging area");
+  uint32_t* scan = reinterpret_cast<uint32_t*>(sm.stage);
+  int* hist = reinterpret_cast<int*>(sm.stage + kTailRowsMax * 4);
+
+  const int which = blockIdx.y / prm.problems, p = blockIdx.y % prm.problems;
+  const BasicSide bs = prm.side[which];
+  const SplitSide sd = sp.side[which];
+  const int level0 = sd.tail_level;
+  if (!sd.active || (int)blockIdx.x >= (1 << level0)) return;
+  const SegmentRef root = locate_segment(sd.n, sd.c, level0, blockIdx.x);
+  if (!root.active) return;
+  const int tid = threadIdx.x;
+  const int team = tid / D, member = tid % D;
+  const int c = sd.c;
+  const T* X = static_cast<const T*>(bs.X) + (size_t)p * sd.n * D;
+  const float* Am = bs.A + (size_t)p * D * D;
+  const float* noise = bs.noise + (size_t)p * bs.nodes * D;
+  const int32_t* pin = sd.perm_in ? sd.perm_in + (size_t)p * sd.n : nullptr;
+  int32_t* pout = sd.perm_out + (size_t)p * sd.n;
+  const int lo = root.lo, s0 = root.size;
+
+  for (int i = tid; i < s0; i += nt) sm.rows[0][i] = pin ? pin[lo + i] : lo + i;
+  if (tid == 0) {
+    sm.seg_lo[0][0] = 0; sm.seg_lo[0][1] = s0; sm.nseg[0] = 1; sm.more = s0 > c;
+    sm.seg_slot[0][0] = (int)blockIdx.x; sm.seg_par[0][0] = -1;
+    sm.split_list[0] = 0; sm.nsplit = s0 > c ? 1 : 0;
+  }
+  __syncthreads();
+
+  int cur = 0, level = level0;
+  while (sm.more) {
+    const int nseg = sm.nseg[cur];
+    const int* slo = sm.seg_lo[cur];
+    const int32_t* rows = sm.rows[cur];
+    int32_t* rows_next = sm.rows[cur ^ 1];
+    const int nsplit = sm.nsplit;
+    float (*dir_now)[D] = sm.dirs[cur];
+    float (*dir_up)[D] = sm.dirs[cur ^ 1];
+
+    // ---- 1. directions, ROUND subsets at a time (every stage boundary is a barrier of the CTA; teams
+    // without a subset go through them idle)
+    for (int r0 = 0; r0 < nsplit; r0 += ROUND) {
+      const bool active = team < ROUND && r0 + team < nsplit;
+      const int g = active ? sm.split_list[r0 + team] : 0;
+      const int a = slo[g], sz = slo[g + 1] - a, m = min(D, sz);
+      T* xs = reinterpret_cast<T*>(sm.stage + (size_t)(team < ROUND ? team : 0) * NODE_BYTES);
+      if (active) {
+        if (member < m) {
+          const int pos = a + (int)(((long long)member * sz) / m);
+          const T* xr = X + (size_t)rows[pos] * D;
+          uint32_t* dst = reinterpret_cast<uint32_t*>(xs + (size_t)member * LD);     // LD * sizeof(T) is a multiple of 4
+          constexpr int V = D * (int)sizeof(T) / 16;                                 // 16-byte loads of a row
+#pragma unroll
+          for (int k0 = 0; k0 < V; k0 += 8) {
+            uint4 q[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) if (k0 + k < V) q[k] = __ldg(reinterpret_cast<const uint4*>(xr) + k0 + k);
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              if (k0 + k < V) {
+                dst[(k0 + k) * 4 + 0] = q[k].x; dst[(k0 + k) * 4 + 1] = q[k].y;
+                dst[(k0 + k) * 4 + 2] = q[k].z; dst[(k0 + k) * 4 + 3] = q[k].w;
+              }
+          }
+        }
+        const int node = (1 << level) - 1 + sm.seg_slot[cur][g];
+        sm.g[team][member] = noise[(size_t)node * D + member];
+      }
+      __syncthreads();
+      if (active) {
+        float mu = 0.f;                                      // column `member`, rows in order
+        for (int i = 0; i < m; ++i) mu = __fadd_rn(mu, stored_value(xs + i * LD + member));
+        mu = __fdiv_rn(mu, (float)m);
+        sm.mu[team][member] = mu;
+        const float gn = __fdiv_rn(sm.g[team][member], seq_norm(sm.g[team], D));
+        float start = gn;
+        if (level > 0) {
+          const int par = sm.seg_par[cur][g];
+          const float up = par >= 0 ? dir_up[par][member]
+                                    : bs.dirs[((size_t)p * bs.nodes + (1 << (level - 1)) - 1 + (sm.seg_slot[cur][g] >> 1)) * D + member];
+          start = __fmul_rn(__fadd_rn(up, gn), 0.5f);
+        }
+        sm.u[team][member] = start;
+      }
+      __syncthreads();
+      for (int it = 0; it < prm.iterations; ++it) {
+        if (active && member < m) {
+          // (terms formed eight at a time, then added in order: the loads do not wait for the sum)
+          float acc = 0.f;
+#pragma unroll 1
+          for (int k0 = 0; k0 < D; k0 += 8) {
+            float term[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              term[k] = __fmul_rn(__fsub_rn(stored_value(xs + member * LD + k0 + k), sm.mu[team][k0 + k]), sm.u[team][k0 + k]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc = __fadd_rn(acc, term[k]);
+          }
+          sm.v[team][member] = acc;
+        }
+        __syncthreads();
+        if (active) {
+          const float mk = sm.mu[team][member];
+          float acc = 0.f;
+          int i = 0;
+#pragma unroll 1
+          for (; i + 8 <= m; i += 8) {
+            float term[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+              term[k] = __fmul_rn(__fsub_rn(stored_value(xs + (i + k) * LD + member), mk), sm.v[team][i + k]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc = __fadd_rn(acc, term[k]);
+          }
+          for (; i < m; ++i)
+            acc = __fadd_rn(acc, __fmul_rn(__fsub_rn(stored_value(xs + i * LD + member), mk), sm.v[team][i]));
+          sm.w[team][member] = acc;
+        }
+        __syncthreads();
+        if (active) {
+          const float4* Ar = reinterpret_cast<const float4*>(Am + (size_t)member * D);
+          float acc = 0.f;
+#pragma unroll 1
+          for (int k0 = 0; k0 < D; k0 += 8) {
+            const float4 a0 = __ldg(Ar + k0 / 4), a1 = __ldg(Ar + k0 / 4 + 1);
+            const float av[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            float term[8];
+#pragma unroll
+            for (int k = 0; k < 8; ++k) term[k] = __fmul_rn(av[k], sm.w[team][k0 + k]);
+#pragma unroll
+            for (int k = 0; k < 8; ++k) acc = __fadd_rn(acc, term[k]);
+          }
+          sm.y[team][member] = acc;
+        }
+        __syncthreads();
+        if (active) {
+          const float nrm = seq_norm(sm.y[team], D);          // every thread takes the same sequential sum
+          if (nrm > 0.f && isfinite(nrm)) sm.u[team][member] = __fdiv_rn(sm.y[team][member], nrm);
+        }
+        __syncthreads();
+      }
+      if (active) dir_now[g][member] = sm.u[team][member];
+      __syncthreads();
+    }
+    if (tid < nseg) {
+      const int a = slo[tid], sz = slo[tid + 1] - a;
+      sm.seg_L[tid] = sz > c ? c * ((sz + c) / (2 * c)) : 0;
+      sm.seg_prefix[tid] = 0u;
+      sm.seg_rem[tid] = sm.seg_L[tid];
+    }
+
+    // ---- 2. keys: the projection of a row onto its subset's direction, terms in the order of the columns
+    int my_seg[PT];
+    uint32_t my_key[PT];
+    {
+      const int i0 = PT * tid;
+      int g = 0;
+      if (i0 < s0) {
+        int hi = nseg;                                  // slo[g] <= i0 < slo[g+1]
+        while (hi - g > 1) { const int mid = (g + hi) >> 1; if (slo[mid] <= i0) g = mid; else hi = mid; }
+      }
+#pragma unroll 1
+      for (int u = 0; u < PT; ++u) {
+        const int i = i0 + u;
+        my_key[u] = 0u;
+        if (i < s0) {
+          while (slo[g + 1] <= i) ++g;
+          const bool splits = slo[g + 1] - slo[g] > c;
+          if (splits) {
+            const T* xr = X + (size_t)rows[i] * D;
+            const float* uu = dir_now[g];
+            float t = 0.f;
+            constexpr int E = 16 / (int)sizeof(T);       // elements of a 16-byte load
+#pragma unroll
+            for (int k0 = 0; k0 < D; k0 += 4 * E) {      // four loads in flight, then their terms in order
+              uint4 q[4];
+#pragma unroll
+              for (int k = 0; k < 4; ++k) q[k] = __ldg(reinterpret_cast<const uint4*>(xr + k0) + k);
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const uint32_t wds[4] = {q[k].x, q[k].y, q[k].z, q[k].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                  if (sizeof(T) == 2) {
+                    const float x0 = __uint_as_float(wds[e] << 16), x1 = __uint_as_float(wds[e] & 0xffff0000u);
+                    t = __fadd_rn(t, __fmul_rn(x0, uu[k0 + k * E + 2 * e]));
+                    t = __fadd_rn(t, __fmul_rn(x1, uu[k0 + k * E + 2 * e + 1]));
+                  } else {
+                    t = __fadd_rn(t, __fmul_rn(__uint_as_float(wds[e]), uu[k0 + k * E + e]));
+                  }
+                }
+              }
+            }
+            my_key[u] = order_key(t);
+          }
+          my_seg[u] = splits ? g : -1 - g;              // final subset: carried over unchanged
+        } else {
+          my_seg[u] = INT_MIN;
+        }
+      }
+    }
+    __syncthreads();                                    // the staging area becomes the scan and the digit counts
+
+    tail_select_partition(sm, my_seg, my_key, nseg, slo, rows, rows_next, tid, hist, scan);
+
+    // ---- next level's subsets
+    if (tid == 0) {
+      int* nlo = sm.seg_lo[cur ^ 1];
+      int* nslot = sm.seg_slot[cur ^ 1];
+      int* npar = sm.seg_par[cur ^ 1];
+      int n2 = 0, more = 0, ns = 0;
+      for (int g = 0; g < nseg; ++g) {
+        const int a = slo[g], sz = slo[g + 1] - a;
+        if (sz > c) {
+          const int L = sm.seg_L[g];
+          nlo[n2] = a;     nslot[n2] = 2 * sm.seg_slot[cur][g];     npar[n2] = g;
+          if (L > c) sm.split_list[ns++] = n2;
+          ++n2;
+          nlo[n2] = a + L; nslot[n2] = 2 * sm.seg_slot[cur][g] + 1; npar[n2] = g;
+          if (sz - L > c) sm.split_list[ns++] = n2;
+          ++n2;
+          more |= (L > c) | (sz - L > c);
+        } else {
+          nlo[n2] = a; nslot[n2] = 0; npar[n2] = g;      // a final subset: only carried along
+          ++n2;
+        }
+      }
+      nlo[n2] = s0;
+      sm.nseg[cur ^ 1] = n2;
+      sm.nsplit = ns;
+      sm.more = more;
+    }
+    __syncthreads();
+    cur ^= 1;
+    ++level;
+  }
+  for (int i = tid; i < s0; i += nt) pout[lo + i] = sm.rows[cur][i];
+}
+
 template <typename T>
 static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const float* A_k, const float* noise_q,
                                 const float* noise_k, float* dirs_q, float* dirs_k, int iterations, int problems,
@@ -960,39 +1271,49 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
   auto level_kernel = D == 64 ? split_level_kernel<64> : split_level_kernel<128>;
   CA_RETURN_IF_CUDA(cudaFuncSetAttribute(level_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRowsMax * 8));
   const int lev_q = split_levels_for(n_q, c_q), lev_k = split_levels_for(n_k, c_k);
-  // a side without any split still needs one launch to write the identity permutation
-  const int run_q = lev_q > 0 ? lev_q : 1, run_k = lev_k > 0 ? lev_k : 1;
-  const int top = run_q > run_k ? run_q : run_k;
+  // Sets of more than kTailRowsMax rows take three launches per level (directions, projections,
+  // select + partition); the subtree kernel finishes the rest.  Per-level launches write alternately
+  // to tmp/out so that the subtree kernel, which runs last, reads the buffer that is not the output.
+  const int tail_q = tail_level_for(n_q, c_q), tail_k = tail_level_for(n_k, c_k);
+  const int top = tail_q > tail_k ? tail_q : tail_k;
   BasicParams bp;
   bp.problems = problems; bp.iterations = iterations;
   SplitParams prm;
   prm.D = D; prm.problems = problems; prm.keys_in = 1;
-  for (int level = 0; level < top; ++level) {
+  auto fill = [&](int level) {
     for (int w = 0; w < 2; ++w) {
-      const int run = w == 0 ? run_q : run_k;
+      const int tail = w == 0 ? tail_q : tail_k;
       int32_t* out = w == 0 ? perm_q_out : perm_k_out;
       int32_t* tmp = w == 0 ? perm_q_tmp : perm_k_tmp;
-      // the last level of a side writes its output buffer, the ones before alternate
-      const bool to_tmp = ((run - 1 - level) % 2) != 0;
       SplitSide& sd = prm.side[w];
       sd.Y = nullptr;
       sd.Yt = nullptr;
       sd.keybuf = w == 0 ? keybuf_q : keybuf_k;
       sd.n = w == 0 ? n_q : n_k; sd.c = w == 0 ? c_q : c_k;
       sd.levels = w == 0 ? lev_q : lev_k;
-      sd.tail_level = run;                               // every level runs as a launch of its own
+      sd.tail_level = tail;
       sd.active = 1;
-      sd.perm_out = to_tmp ? tmp : out;
-      sd.perm_in = level == 0 ? nullptr : (to_tmp ? out : tmp);
+      const bool to_tmp = ((tail - 1 - level) % 2) == 0;
+      if (level < tail) {
+        sd.perm_out = to_tmp ? tmp : out;
+        sd.perm_in = level == 0 ? nullptr : (to_tmp ? out : tmp);
+      } else {
+        sd.perm_out = out;
+        sd.perm_in = tail == 0 ? nullptr : tmp;
+      }
       BasicSide& bs = bp.side[w];
       bs.X = w == 0 ? static_cast<const void*>(Q) : static_cast<const void*>(K);
       bs.A = w == 0 ? A_q : A_k;
       bs.noise = w == 0 ? noise_q : noise_k;
       bs.dirs = w == 0 ? dirs_q : dirs_k;
       bs.perm_in = sd.perm_in; bs.keybuf = sd.keybuf;
-      bs.n = sd.n; bs.c = sd.c; bs.levels = sd.levels;
+      bs.n = sd.n; bs.c = sd.c;
+      bs.levels = tail;                                    // the per-level kernels stop where the subtrees begin
       bs.nodes = (1 << (sd.levels > 0 ? sd.levels : 1)) - 1;
     }
+  };
+  for (int level = 0; level < top; ++level) {
+    fill(level);
     bp.level = level; prm.level = level;
     const size_t dsmem = (size_t)D * (D + 1) * sizeof(float);
     if (D == 64) {
@@ -1010,15 +1331,14 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
     else basic_keys_kernel<T, 128><<<dim3(ceil_div(n_max, 256), 2 * problems), 256, 0, st>>>(bp);
     CA_LAUNCH_CHECK();
     int max_seg = 1;
-    if (level < run_q) max_seg = max_segment_at_level(n_q, c_q, level);
-    if (level < run_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
+    if (level < tail_q) max_seg = max_segment_at_level(n_q, c_q, level);
+    if (level < tail_k) { const int ms = max_segment_at_level(n_k, c_k, level); if (ms > max_seg) max_seg = ms; }
     int csize = 1;
     while (csize < kMaxCluster && max_seg > csize * 16384) csize *= 2;
     const int per_cta = (max_seg + csize - 1) / csize;
     prm.smem_rows = per_cta < kSmemRowsMax ? per_cta : kSmemRowsMax;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((1u << level) * csize, 2 * problems);
-    // deep levels hold many small sets: a CTA per set with about four rows per thread
     int threads = 128;
     while (threads < kSplitThreads && threads * 4 < per_cta) threads *= 2;
     cfg.blockDim = dim3(threads);
@@ -1031,6 +1351,19 @@ static int launch_split_basic_t(const T* Q, const T* K, const float* A_q, const 
     CA_RETURN_IF_CUDA(cudaLaunchKernelEx(&cfg, level_kernel, prm));
     CA_LAUNCH_CHECK();
   }
+  fill(top);
+  bp.level = top; prm.level = top;
+  const int slots = 1 << top;
+  if (D == 64) {
+    auto tk = basic_tail_kernel<T, 64>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(tk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BasicTailSmem<64>)));
+    tk<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(BasicTailSmem<64>), st>>>(bp, prm);
+  } else {
+    auto tk = basic_tail_kernel<T, 128>;
+    CA_RETURN_IF_CUDA(cudaFuncSetAttribute(tk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sizeof(BasicTailSmem<128>)));
+    tk<<<dim3(slots, 2 * problems), kSplitThreads, sizeof(BasicTailSmem<128>), st>>>(bp, prm);
+  }
+  CA_LAUNCH_CHECK();
   return CA_OK;
 }
 
