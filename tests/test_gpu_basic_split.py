@@ -34,6 +34,7 @@ CASES = [
     (1, 3000, 4099, 128, 128, 128, "bf16", 3),
     (1, 2048, 40000, 64, 128, 128, "bf16", 1),       # sets larger than the shared-memory window
     (1, 640, 704, 128, 256, 16, "bf16", 0),          # no iteration: the start vectors decide
+    (1, 700, 5000, 128, 64, 128, "fp32", 2),         # float32 rows at d = 128: two subsets staged per round
 ]
 
 
