@@ -292,6 +292,15 @@ int ca_attn_recomputed(const void* ws);
  * memory and returns, and the output of the call is undefined; -1 restores normal operation. */
 void ca_debug_attn_wait(long long wait_limit_cycles, int skip_key_load);
 
+/* Diagnostic: the symmetric eigen-decomposition that cluster_qk uses for the principal components
+ * (Section 3.2.1, diagonalized variant), on matrices of the caller's.  A: `count` symmetric d x d
+ * matrices in double precision, row-major (device, read only); d = 64 or 128.  Written (device):
+ * W [count][d][d] float32, eigenvector t in column t, eigenvalues in descending order, each column
+ * oriented so that its entry of largest magnitude is positive; evals [count][d] double, or NULL.
+ * The arithmetic is float32 (the components only feed float32 coordinates).  Enqueued on `stream`;
+ * returns CA_ERR_UNSUPPORTED for another d, CA_ERR_INVALID_ARG for null or misaligned pointers. */
+int ca_debug_eigh(const double* A, int count, int d, float* W, double* evals, void* stream);
+
 /*
  * Per-kernel-group device times (a measuring aid; process-wide, not thread-safe).
  * ca_profile(1) switches the timers on: every call issued afterwards records CUDA events around

@@ -29,7 +29,7 @@ CA_Y_IN, CA_ATTN_FP32, CA_QUERY_UNNORMALIZED, CA_METRIC_IN, CA_ATTN_FP8_QK = 1, 
 EXPORTS = ("ca_workspace_bytes", "cluster_qk", "select_blocks", "cluster_attention_fwd",
            "ca_last_status", "ca_attn_recomputed", "ca_version", "ca_kernel_launches", "cluster_attention_fwd_static",
            "ca_static_scratch_bytes", "ca_static_last_status", "select_blocks_adaptive",
-           "cluster_attention_fwd_ragged", "ca_basic_workspace_bytes", "cluster_qk_basic", "ca_debug_attn_wait",
+           "cluster_attention_fwd_ragged", "ca_basic_workspace_bytes", "cluster_qk_basic", "ca_debug_attn_wait", "ca_debug_eigh",
            "ca_profile", "ca_profile_read")
 
 
@@ -106,6 +106,9 @@ def load_library() -> ctypes.CDLL:
     lib.ca_static_last_status.restype = ctypes.c_int
     lib.ca_debug_attn_wait.argtypes = [ctypes.c_longlong, ctypes.c_int]
     lib.ca_debug_attn_wait.restype = None
+    lib.ca_debug_eigh.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                                  ctypes.c_void_p]
+    lib.ca_debug_eigh.restype = ctypes.c_int
     lib.ca_profile.argtypes = [ctypes.c_int]
     lib.ca_profile.restype = ctypes.c_int
     lib.ca_profile_read.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_char_p), ctypes.POINTER(ctypes.c_float),
@@ -178,6 +181,20 @@ def problem_from_workload(w, heads: Optional[int] = None, **kw) -> CaProblem:
                 compensate=w.compensate)
     args.update(kw)
     return make_problem(**args)
+
+
+def debug_eigh(A: torch.Tensor, stream=None):
+    """ca_debug_eigh of the C library: A [count, d, d] float64 symmetric (CUDA).  Returns
+    (W [count, d, d] float32 with eigenvector t in column t, evals [count, d] float64, descending)."""
+    _require_cuda(A, "A")
+    if A.dtype != torch.float64 or A.dim() != 3 or A.shape[1] != A.shape[2]:
+        raise ClusterAttnError("A must be [count, d, d] float64")
+    lib = load_library()
+    count, d = int(A.shape[0]), int(A.shape[1])
+    W = torch.empty((count, d, d), dtype=torch.float32, device=A.device)
+    ev = torch.empty((count, d), dtype=torch.float64, device=A.device)
+    _check(lib.ca_debug_eigh(_ptr(A), count, d, _ptr(W), _ptr(ev), _stream_ptr(stream)), "ca_debug_eigh")
+    return W, ev
 
 
 def workspace_bytes(problem: CaProblem) -> Dict[str, int]:

@@ -557,6 +557,17 @@ void ca_debug_attn_wait(long long wait_limit_cycles, int skip_key_load) {
   attn_tc_set_debug(wait_limit_cycles, skip_key_load);
 }
 
+int ca_debug_eigh(const double* A, int count, int d, float* W, double* evals, void* stream) {
+  if (!A || !W || !aligned16(A) || !aligned16(W) || count < 1) return CA_ERR_INVALID_ARG;
+  if (d != 64 && d != 128) return CA_ERR_UNSUPPORTED;
+  PcaArgs a{};
+  a.mode = kPcaMatrix;
+  a.A_in = A;
+  a.W32 = W;
+  a.evals = evals;
+  return launch_pca(a, count, d, static_cast<cudaStream_t>(stream));
+}
+
 int ca_last_status(const void* ws) {
   if (!ws) return CA_ERR_INVALID_ARG;
   int status = 0;
