@@ -101,12 +101,38 @@ __device__ __forceinline__ void staged_variances(const float* tiles, int ng, Row
   }
 }
 
+// Two fp32 values in one 64-bit register and the instructions that work on both halves at once
+// (each half rounded to nearest on its own: the same bits as two scalar operations).
+typedef unsigned long long pair2;
+__device__ __forceinline__ pair2 pair(float lo, float hi) {
+  pair2 d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "f"(lo), "f"(hi));
+  return d;
+}
+__device__ __forceinline__ void unpair(pair2 v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ pair2 add_pair(pair2 a, pair2 b) {
+  pair2 d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ pair2 mul_pair(pair2 a, pair2 b) {
+  pair2 d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 // The same estimate for `ng` subsets at once, the sample rows read straight from the coordinates
-// in global memory (sub[gi * D + j]: row of sample j of subset gi, -1 beyond its m rows).  Same
-// operations in the same order as staged_variances, hence the same bits; what differs is the
-// parallelism: every (subset, residue, coordinate) is a thread's task, so a round of many small
-// subsets keeps all warps busy between two barriers, and a task's loads (one per sample row of its
-// residue) are all in flight together.
+// in global memory.  `sub` holds the sample rows residue-major: sub[gi * D + r * (D / 8) + k] is
+// the row of sample r + 8 k of subset gi, -1 beyond its m rows.  Same operations in the same order
+// as staged_variances, hence the same bits; what differs is the parallelism: every (subset,
+// residue, coordinate) is a thread's task, so a round of many small subsets keeps all warps busy
+// between two barriers, and a task's loads (one per sample row of its residue) are in flight four
+// at a time.  The stage is bound by the instructions it issues, so a subset with all D sample rows
+// (every subset that still splits when the cluster size is at least D) runs without a test per
+// row; a missing row otherwise reads as 0 in the pass of the sums and as the mean in the pass of
+// the squares, which adds an exact zero.
 template <int D, typename RowsOf>
 __device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, const int* sub, int ng, RowsOf rows_of,
                                                    float* part, float* out, int tid, int nt) {
@@ -119,31 +145,40 @@ __device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, 
       const int m = rows_of(gi);
       float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
       if (pass == 1) mean = *reinterpret_cast<const float4*>(out + gi * D + 4 * t4);
-      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      pair2 acc_a = pair(0.f, 0.f), acc_b = acc_a;
+      const pair2 nmean_a = pair(-mean.x, -mean.y), nmean_b = pair(-mean.z, -mean.w);
+      const int4* idx = reinterpret_cast<const int4*>(sub + gi * D + r * PER);
+      const float4* Yv = reinterpret_cast<const float4*>(Y) + t4;
+      const bool full = m == D;                    // all PER rows of the residue are there
 #pragma unroll
       for (int k0 = 0; k0 < PER; k0 += B) {
+        const int4 ri = idx[k0 / B];
+        const int row[B] = {ri.x, ri.y, ri.z, ri.w};
         float4 x[B];
+        if (full) {
 #pragma unroll
-        for (int k = 0; k < B; ++k) {
-          const int j = r + 8 * (k0 + k);
-          const int row = j < m ? sub[gi * D + j] : -1;
-          x[k] = row >= 0 ? __ldg(reinterpret_cast<const float4*>(Y + (size_t)row * D) + t4) : make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int k = 0; k < B; ++k) x[k] = __ldg(Yv + (size_t)row[k] * Q4);
+        } else {
+#pragma unroll
+          for (int k = 0; k < B; ++k) x[k] = row[k] >= 0 ? __ldg(Yv + (size_t)row[k] * Q4) : mean;
         }
+        // two values per instruction, each rounded on its own as the scalar operations are
 #pragma unroll
         for (int k = 0; k < B; ++k) {
-          if (r + 8 * (k0 + k) < m) {
-            if (pass == 0) {
-              acc.x = __fadd_rn(acc.x, x[k].x); acc.y = __fadd_rn(acc.y, x[k].y);
-              acc.z = __fadd_rn(acc.z, x[k].z); acc.w = __fadd_rn(acc.w, x[k].w);
-            } else {
-              const float dx = __fsub_rn(x[k].x, mean.x), dy = __fsub_rn(x[k].y, mean.y);
-              const float dz = __fsub_rn(x[k].z, mean.z), dw = __fsub_rn(x[k].w, mean.w);
-              acc.x = __fadd_rn(acc.x, __fmul_rn(dx, dx)); acc.y = __fadd_rn(acc.y, __fmul_rn(dy, dy));
-              acc.z = __fadd_rn(acc.z, __fmul_rn(dz, dz)); acc.w = __fadd_rn(acc.w, __fmul_rn(dw, dw));
-            }
+          const pair2 xa = pair(x[k].x, x[k].y), xb = pair(x[k].z, x[k].w);
+          if (pass == 0) {
+            acc_a = add_pair(acc_a, xa);
+            acc_b = add_pair(acc_b, xb);
+          } else {
+            const pair2 da = add_pair(xa, nmean_a), db = add_pair(xb, nmean_b);   // x - mean
+            acc_a = add_pair(acc_a, mul_pair(da, da));
+            acc_b = add_pair(acc_b, mul_pair(db, db));
           }
         }
       }
+      float4 acc;
+      unpair(acc_a, acc.x, acc.y);
+      unpair(acc_b, acc.z, acc.w);
       *reinterpret_cast<float4*>(part + (gi * 8 + r) * D + 4 * t4) = acc;
     }
     __syncthreads();
@@ -603,7 +638,9 @@ __global__ void __launch_bounds__(kSplitThreads) split_tail_kernel(const SplitPa
           const int gi = e / D, j = e % D;
           const int a = slo[g0 + gi], sz = slo[g0 + gi + 1] - a;
           const int m = min(D, sz);
-          sub_rows[e] = (sz > c && j < m) ? rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)] : -1;
+          // residue-major: sample j sits at (j % 8) * (D / 8) + j / 8 of its subset's D entries
+          sub_rows[gi * D + (j & 7) * (D / 8) + (j >> 3)] =
+              (sz > c && j < m) ? rows[a + (int)(((unsigned)j * (unsigned)sz) / (unsigned)m)] : -1;
         }
         __syncthreads();
         gathered_variances<D>(Y, sub_rows, ng,
