@@ -117,11 +117,6 @@ __device__ __forceinline__ pair2 add_pair(pair2 a, pair2 b) {
   asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
 }
-__device__ __forceinline__ pair2 mul_pair(pair2 a, pair2 b) {
-  pair2 d;
-  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
 
 // The same estimate for `ng` subsets at once, the sample rows read straight from the coordinates
 // in global memory.  `sub` holds the sample rows residue-major: sub[gi * D + r * (D / 8) + k] is
@@ -146,6 +141,7 @@ __device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, 
       float4 mean = make_float4(0.f, 0.f, 0.f, 0.f);
       if (pass == 1) mean = *reinterpret_cast<const float4*>(out + gi * D + 4 * t4);
       pair2 acc_a = pair(0.f, 0.f), acc_b = acc_a;
+      float4 sq = make_float4(0.f, 0.f, 0.f, 0.f);
       const pair2 nmean_a = pair(-mean.x, -mean.y), nmean_b = pair(-mean.z, -mean.w);
       const int4* idx = reinterpret_cast<const int4*>(sub + gi * D + r * PER);
       const float4* Yv = reinterpret_cast<const float4*>(Y) + t4;
@@ -162,7 +158,10 @@ __device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, 
 #pragma unroll
           for (int k = 0; k < B; ++k) x[k] = row[k] >= 0 ? __ldg(Yv + (size_t)row[k] * Q4) : mean;
         }
-        // two values per instruction, each rounded on its own as the scalar operations are
+        // Sums and differences two values per instruction (each half rounded on its own: the bits
+        // of two scalar additions).  The squares and their sums stay scalar operations that are
+        // never contracted: a two-value multiply followed by a two-value add is merged into one
+        // fused multiply-add by the assembler, which rounds once where the definition rounds twice.
 #pragma unroll
         for (int k = 0; k < B; ++k) {
           const pair2 xa = pair(x[k].x, x[k].y), xb = pair(x[k].z, x[k].w);
@@ -170,15 +169,19 @@ __device__ __forceinline__ void gathered_variances(const float* __restrict__ Y, 
             acc_a = add_pair(acc_a, xa);
             acc_b = add_pair(acc_b, xb);
           } else {
-            const pair2 da = add_pair(xa, nmean_a), db = add_pair(xb, nmean_b);   // x - mean
-            acc_a = add_pair(acc_a, mul_pair(da, da));
-            acc_b = add_pair(acc_b, mul_pair(db, db));
+            float dx, dy, dz, dw;
+            unpair(add_pair(xa, nmean_a), dx, dy);                                // x - mean
+            unpair(add_pair(xb, nmean_b), dz, dw);
+            sq.x = __fadd_rn(sq.x, __fmul_rn(dx, dx)); sq.y = __fadd_rn(sq.y, __fmul_rn(dy, dy));
+            sq.z = __fadd_rn(sq.z, __fmul_rn(dz, dz)); sq.w = __fadd_rn(sq.w, __fmul_rn(dw, dw));
           }
         }
       }
-      float4 acc;
-      unpair(acc_a, acc.x, acc.y);
-      unpair(acc_b, acc.z, acc.w);
+      float4 acc = sq;
+      if (pass == 0) {
+        unpair(acc_a, acc.x, acc.y);
+        unpair(acc_b, acc.z, acc.w);
+      }
       *reinterpret_cast<float4*>(part + (gi * 8 + r) * D + 4 * t4) = acc;
     }
     __syncthreads();
@@ -464,6 +467,8 @@ struct TailSmem {
   int hist[kTailSegs][256];
   int seg_lo[2][2 * kTailSegs + 2];       // start of each subset (relative), +1 sentinel
   int seg_coord[kTailSegs], seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
+  int seg_cand[kTailSegs];                // candidates left after the first two digits; -1: threshold found
+  int overflow;                           // some subset has more candidates than a warp takes
   uint32_t seg_prefix[kTailSegs];
   float vpart[4 * 8 * 64];                // partial sums of the variance stage ([ng][8][D])
   float vout[4 * 64];
@@ -487,17 +492,63 @@ __device__ __forceinline__ void tail_select_partition(Smem& sm, const int (&my_s
   constexpr int nt = kSplitThreads;
   constexpr int PT = kTailRowsMax / kSplitThreads;
   const int lane = tid & 31, warp = tid >> 5;
-  // ---- radix selection, all subsets side by side
+  // ---- radix selection, all subsets side by side: two digits of eight bits by counting; then the
+  // keys that share those sixteen bits with the threshold are few (a handful per subset unless keys
+  // repeat), and a warp ranks them directly.  A subset with more than 32 of them goes on with the two
+  // remaining digits.  (The digit counts are cleared once per level: the warp that picks a subset's
+  // digit clears the counts it has read, ready for the next pass.)
   uint32_t mask = 0;
+  for (int e = tid; e < nseg * 256; e += nt) hist[e] = 0;
+  if (tid < nseg) sm.seg_cand[tid] = 0;
+  if (tid == 0) sm.overflow = 0;
+  __syncthreads();
   for (int shift = 24; shift >= 0; shift -= 8) {
-    for (int e = tid; e < nseg * 256; e += nt) hist[e] = 0;
-    __syncthreads();
+    uint32_t pre[PT];                               // read ahead of the atomics, which order memory accesses
+#pragma unroll
+    for (int u = 0; u < PT; ++u) pre[u] = sm.seg_prefix[my_seg[u] >= 0 ? my_seg[u] : 0];
+    if (shift == 8) {
+      // candidates of every subset into its list (the scan array is free until the partition)
+#pragma unroll
+      for (int u = 0; u < PT; ++u) {
+        const int g = my_seg[u];
+        if (g >= 0 && (my_key[u] & mask) == pre[u]) {
+          const int slot = atomicAdd(&sm.seg_cand[g], 1);
+          if (slot < 32) scan[g * 32 + slot] = my_key[u];
+        }
+      }
+      __syncthreads();
+      for (int g = warp; g < nseg; g += nt / 32) {
+        if (sm.seg_L[g] == 0) continue;             // warp-uniform
+        const int n = sm.seg_cand[g];
+        if (n > 32) {
+          if (lane == 0) sm.overflow = 1;
+          continue;
+        }
+        const int remaining = sm.seg_rem[g];        // 1 <= remaining <= n
+        const uint32_t key = lane < n ? scan[g * 32 + lane] : 0xffffffffu;
+        int less = 0, eq_before = 0;
+        for (int j = 0; j < n; ++j) {
+          const uint32_t kj = __shfl_sync(0xffffffffu, key, j);
+          less += kj < key ? 1 : 0;
+          eq_before += (kj == key && j < lane) ? 1 : 0;
+        }
+        if (lane < n && less + eq_before == remaining - 1) {   // exactly one lane
+          sm.seg_prefix[g] = key;
+          sm.seg_rem[g] = remaining - less;          // how many of the keys equal to the threshold go down
+          sm.seg_cand[g] = -1;
+        }
+      }
+      __syncthreads();
+      if (!sm.overflow) break;                      // uniform: every threshold is found
+#pragma unroll
+      for (int u = 0; u < PT; ++u) pre[u] = sm.seg_prefix[my_seg[u] >= 0 ? my_seg[u] : 0];
+    }
 #pragma unroll
     for (int u = 0; u < PT; ++u) {
       const int g = my_seg[u];
       const bool live = g >= 0;
       const uint32_t k = my_key[u];
-      const bool cand = live && ((k & mask) == sm.seg_prefix[live ? g : 0]);
+      const bool cand = live && ((k & mask) == pre[u]);
       const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
       if (shift == 24) {
         const unsigned peers = __match_any_sync(0xffffffffu, bin);
@@ -511,8 +562,17 @@ __device__ __forceinline__ void tail_select_partition(Smem& sm, const int (&my_s
       const int remaining = sm.seg_rem[g];
       if (sm.seg_L[g] == 0) continue;               // warp-uniform
       int local[8]; int sum = 0;
+      {
+        int4* h4 = reinterpret_cast<int4*>(&hist[g * 256 + lane * 8]);
+        const int4 h0 = h4[0], h1 = h4[1];
+        h4[0] = make_int4(0, 0, 0, 0);
+        h4[1] = make_int4(0, 0, 0, 0);
+        local[0] = h0.x; local[1] = h0.y; local[2] = h0.z; local[3] = h0.w;
+        local[4] = h1.x; local[5] = h1.y; local[6] = h1.z; local[7] = h1.w;
+      }
+      if (sm.seg_cand[g] < 0) continue;             // found by the direct ranking (its keys were still counted)
 #pragma unroll
-      for (int j = 0; j < 8; ++j) { local[j] = hist[g * 256 + lane * 8 + j]; sum += local[j]; }
+      for (int j = 0; j < 8; ++j) sum += local[j];
       int incl = sum;
       for (int o = 1; o < 32; o <<= 1) {
         const int v = __shfl_up_sync(0xffffffffu, incl, o);
@@ -1034,6 +1094,8 @@ struct BasicTailSmem {
   int seg_slot[2][2 * kTailSegs + 2];     // slot of a subset in the tree, at the level it stands on
   int seg_par[2][2 * kTailSegs + 2];      // subset of the level above it came from
   int seg_digit[kTailSegs], seg_rem[kTailSegs], seg_L[kTailSegs];
+  int seg_cand[kTailSegs];                // candidates left after the first two digits; -1: threshold found
+  int overflow;                           // some subset has more candidates than a warp takes
   uint32_t seg_prefix[kTailSegs];
   int split_list[kTailSegs];              // the subsets that still split
   int warp_tot[32];

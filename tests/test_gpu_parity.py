@@ -97,6 +97,40 @@ def test_split_and_gather_bit_exact(H, n_q, n_k, d, c_q, c_k, dtype, ties):
             assert np.abs(got[0, h].cpu().numpy() - want).max() < 2e-6 * max(1.0, np.abs(want).max())
 
 
+# Coordinates whose columns are permutations of one set of values: every column has the same
+# variance in exact arithmetic, so which coordinate a set is split on is decided by the last bit of
+# every rounding in the variance estimate.  A device sum that rounds once where the float32
+# restatement rounds twice (a multiply and an add merged into a fused multiply-add) picks another
+# coordinate for about two sets in three.  Shapes: sets with fewer rows than coordinates (a partly
+# filled subsample), sets with at least d rows, and sets large enough for the per-level kernels.
+EQUAL_VARIANCE_CASES = [
+    # n, d, c
+    (96, 128, 32), (300, 64, 16), (1500, 128, 16), (4096, 64, 128), (5000, 128, 64), (40000, 64, 128), (20000, 128, 128),
+]
+
+
+@pytest.mark.parametrize("n,d,c", EQUAL_VARIANCE_CASES)
+def test_split_follows_the_float32_restatement_when_every_column_has_the_same_variance(n, d, c):
+    H = 2
+    r = np.random.default_rng(n * 131 + d)
+    Y = np.empty((H, n, d), np.float32)
+    for h in range(H):
+        base = r.standard_normal(n).astype(np.float32)
+        if h == 1:
+            base = np.round(base * 4.0) / 4.0            # repeated values on top
+        for t in range(d):
+            Y[h, :, t] = r.permutation(base)
+    X = inputs.round_to_bf16(r.standard_normal((H, n, d)).astype(np.float32))
+    p = binding.make_problem(1, H, n, n, d, "bf16", c, c, 1, flags=binding.CA_Y_IN)
+    plan = binding.Plan(p, DEV)
+    plan.cluster_qk(store(p, X), store(p, X), store(p, X), Yq=to_dev(Y[None]), Yk=to_dev(Y[None, :, ::-1].copy()))
+    torch.cuda.synchronize()
+    assert all(v == 0 for v in plan.last_status().values())
+    for h in range(H):
+        assert np.array_equal(plan.perm_q[0, h].cpu().numpy(), orc.recursive_split_f32(Y[h], c)), f"queries, head {h}"
+        assert np.array_equal(plan.perm_k[0, h].cpu().numpy(), orc.recursive_split_f32(Y[h, ::-1], c)), f"keys, head {h}"
+
+
 # ----------------------------------------------------------------------------
 # Full clustering stage: the device computes its own coordinates.  The oracle's
 # splitter run on the device's coordinates must give the same permutation, and
