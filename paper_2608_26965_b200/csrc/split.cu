@@ -34,6 +34,7 @@ namespace cg = cooperative_groups;
 constexpr int kSplitThreads = 1024;
 constexpr int kSmemRowsMax = 24576;      // rows a CTA stages (8 bytes each)
 constexpr int kMaxCluster = 8;
+constexpr int kLevelListMax = 1024;      // candidates that the level kernel ranks from a list after two digits
 constexpr int kTailRowsMax = 4096;
 constexpr int kTailSegs = 32;            // subsets a tail CTA splits side by side
 
@@ -239,6 +240,9 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   __shared__ int s_warp[2 * 32];
   __shared__ int s_scalar[4];      // 0: coordinate, 1: digit, 2: remaining rank, 3: chunk total
   __shared__ int s_counts[2];      // this CTA's (less, equal) totals
+  __shared__ uint32_t s_list[kLevelListMax];   // the keys that share the first two digits with the threshold
+  __shared__ int s_list_n;         // entries of the list (counted in the cluster's first CTA)
+  __shared__ int s_ncand;          // keys in the digit that the last pass chose
   int* const s_hist = s_hist2[1];  // scratch of the partition (the last pass counts in the other array)
 
   const int which = blockIdx.y / prm.problems;
@@ -335,40 +339,72 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
   }
   }
   for (int b = tid; b < 256; b += nt) s_hist2[1][b] = 0;      // the first pass (shift 24) counts here
+  if (tid == 0) s_list_n = 0;
   __syncthreads();
 
   // ---- radix selection of the L-th smallest key of the whole set (8 bits per pass).  The slices'
   // counts alternate between two arrays: a peer may still be adding up one pass's counts while
   // this CTA counts the next pass, and an array is cleared only after the cluster barrier of the
   // pass after the one that used it, when every peer has finished reading it.
+  // After two digits the keys that share them with the threshold are usually few: if they fit the
+  // list, every slice appends its candidates to the list of the cluster's first CTA (one more
+  // cluster barrier), every CTA takes a copy, and the last two digits are counted over that list
+  // alone, with no sweep over the slice, no cluster barrier and no sums over the peers.
   const int L = sd.c * ((s + sd.c) / (2 * sd.c));
   uint32_t prefix = 0, mask = 0;
   int remaining = L;                                // 1-based rank among the candidates
+  bool listed = false;
+  int n_list = 0;
   for (int shift = 24; shift >= 0; shift -= 8) {
     int* const hist = s_hist2[(shift >> 3) & 1];
     int* const hist_next = s_hist2[((shift >> 3) & 1) ^ 1];
-    for (int i0 = 0; i0 < cs; i0 += nt) {
-      const int i = i0 + tid;
-      const bool ok = i < cs;
-      const uint32_t k = ok ? keys[i] : 0u;
-      const bool cand = ok && ((k & mask) == prefix);
-      const int bin = cand ? (int)((k >> shift) & 255u) : -1;
-      if (shift == 24) {
-        // leading digit: few distinct values in a warp (sign and exponent bits), one atomic per value
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
-      } else if (cand) {
-        atomicAdd(&hist[bin], 1);                   // lower digits are spread out: plain atomics
+    if (shift == 8 && s_ncand <= kLevelListMax) {   // uniform over the cluster: every CTA holds the same totals
+      listed = true;
+      n_list = s_ncand;
+      uint32_t* const list0 = csize > 1 ? cluster.map_shared_rank(s_list, 0) : s_list;
+      int* const count0 = csize > 1 ? cluster.map_shared_rank(&s_list_n, 0) : &s_list_n;
+      for (int i = tid; i < cs; i += nt) {
+        const uint32_t k = keys[i];
+        if ((k & mask) == prefix) list0[atomicAdd(count0, 1)] = k;   // n_list such keys in the whole set
       }
+      if (csize > 1) {
+        cluster.sync();                              // the list is complete (and every peer is past the second pass)
+        if (crank != 0)
+          for (int i = tid; i < n_list; i += nt) s_list[i] = list0[i];
+      }
+      __syncthreads();
     }
-    if (csize > 1) {
-      cluster.sync();                                // every slice has counted
-      for (int b = tid; b < 256; b += nt) {
-        int sum = 0;
-        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(hist, r)[b];
-        s_total[b] = sum;
+    if (!listed) {
+      for (int i0 = 0; i0 < cs; i0 += nt) {
+        const int i = i0 + tid;
+        const bool ok = i < cs;
+        const uint32_t k = ok ? keys[i] : 0u;
+        const bool cand = ok && ((k & mask) == prefix);
+        const int bin = cand ? (int)((k >> shift) & 255u) : -1;
+        if (shift == 24) {
+          // leading digit: few distinct values in a warp (sign and exponent bits), one atomic per value
+          const unsigned peers = __match_any_sync(0xffffffffu, bin);
+          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
+        } else if (cand) {
+          atomicAdd(&hist[bin], 1);                 // lower digits are spread out: plain atomics
+        }
+      }
+      if (csize > 1) {
+        cluster.sync();                              // every slice has counted
+        for (int b = tid; b < 256; b += nt) {
+          int sum = 0;
+          for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(hist, r)[b];
+          s_total[b] = sum;
+        }
+      } else {
+        __syncthreads();
+        for (int b = tid; b < 256; b += nt) s_total[b] = hist[b];
       }
     } else {
+      for (int i = tid; i < n_list; i += nt) {
+        const uint32_t k = s_list[i];
+        if ((k & mask) == prefix) atomicAdd(&hist[(k >> shift) & 255u], 1);
+      }
       __syncthreads();
       for (int b = tid; b < 256; b += nt) s_total[b] = hist[b];
     }
@@ -389,6 +425,7 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
         if (before < remaining && remaining <= before + local[j]) {
           s_scalar[1] = lane * 8 + j;
           s_scalar[2] = remaining - before;
+          s_ncand = local[j];
         }
         before += local[j];
       }
