@@ -379,15 +379,10 @@ __global__ void __launch_bounds__(kSplitThreads) split_level_kernel(const SplitP
         const int i = i0 + tid;
         const bool ok = i < cs;
         const uint32_t k = ok ? keys[i] : 0u;
-        const bool cand = ok && ((k & mask) == prefix);
-        const int bin = cand ? (int)((k >> shift) & 255u) : -1;
-        if (shift == 24) {
-          // leading digit: few distinct values in a warp (sign and exponent bits), one atomic per value
-          const unsigned peers = __match_any_sync(0xffffffffu, bin);
-          if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
-        } else if (cand) {
-          atomicAdd(&hist[bin], 1);                 // lower digits are spread out: plain atomics
-        }
+        // one atomic per candidate key, also for the leading digit with its few distinct values:
+        // a sweep of plain atomics costs the same whatever the digit's spread, and a warp match per
+        // position to merge equal digits costs three times as much
+        if (ok && ((k & mask) == prefix)) atomicAdd(&hist[(k >> shift) & 255u], 1);
       }
       if (csize > 1) {
         cluster.sync();                              // every slice has counted
@@ -585,14 +580,7 @@ __device__ __forceinline__ void tail_select_partition(Smem& sm, const int (&my_s
       const int g = my_seg[u];
       const bool live = g >= 0;
       const uint32_t k = my_key[u];
-      const bool cand = live && ((k & mask) == pre[u]);
-      const int bin = cand ? ((g << 8) | (int)((k >> shift) & 255u)) : -1;
-      if (shift == 24) {
-        const unsigned peers = __match_any_sync(0xffffffffu, bin);
-        if (cand && lane == (__ffs(peers) - 1)) atomicAdd(&hist[bin], __popc(peers));
-      } else if (cand) {
-        atomicAdd(&hist[bin], 1);
-      }
+      if (live && ((k & mask) == pre[u])) atomicAdd(&hist[(g << 8) | (int)((k >> shift) & 255u)], 1);
     }
     __syncthreads();
     for (int g = warp; g < nseg; g += nt / 32) {
